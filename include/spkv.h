@@ -1,0 +1,230 @@
+/*
+ * spkv.h -- C ABI of the SP-KV (Self-Pruned Key-Value attention) inference library
+ * for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the inference-time hot path of SP-KV: every new key/value
+ * pair gets a utility logit from a small predictor (Eq. 1), lives in a ring of the w
+ * most recent pairs (the always-visible local window), and when it leaves the ring it
+ * is appended to a per-(layer, sequence, KV head) compact cache only if its utility
+ * reaches the threshold tau (Eq. 2).  Attention for the query heads of a KV head then
+ * runs over window U compact cache (Eq. 3-5) under grouped-query attention.
+ *
+ * General rules of this interface
+ *   - Every function returns an int status: SPKV_OK (0) or a negative SPKV_E_* code.
+ *     Nothing throws, aborts or traps the device.
+ *   - "d_" arguments are DEVICE pointers, "h_" arguments are HOST pointers.  All device
+ *     memory (arena, inputs, outputs, workspaces) is allocated, owned and freed by the
+ *     caller; the library never allocates or frees device memory.
+ *   - `stream` is a cudaStream_t passed as a plain pointer (NULL = default stream).
+ *     Calls only enqueue work on it; the only calls that synchronise are spkv_status,
+ *     spkv_cache_stats and the spkv_read_* helpers.
+ *   - bf16 tensors are dense, row-major, 16-byte aligned.  head_dim is 128.
+ *   - Argument errors are reported synchronously.  Errors found on the device (pool
+ *     exhausted, context overflow, a bounded wait that ran out) are recorded in a sticky
+ *     status word inside the arena and reported by spkv_status.
+ *   - One host thread at a time per cache.  A sequence id may appear at most once in
+ *     the seq-id list of a call.
+ *
+ * A "unit" is one (layer, sequence, KV head).  Units are independent of each other.
+ * Positions: a unit that has received t pairs holds positions 0..t-1; the ring holds
+ * positions max(0,t-w)..t-1; the compact cache holds the positions s <= t-1-w whose
+ * logit passed the threshold, in ascending order.
+ */
+#ifndef SPKV_H_
+#define SPKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct spkv_cache spkv_cache_t; /* opaque host-side handle */
+typedef void *spkv_stream_t;            /* cudaStream_t */
+
+enum {
+  SPKV_OK = 0,
+  SPKV_E_INVALID = -1,          /* bad argument                                        */
+  SPKV_E_ARENA_TOO_SMALL = -2,  /* arena_bytes < spkv_arena_bytes(cfg)                 */
+  SPKV_E_UNSUPPORTED = -3,      /* head_dim != 128, page_tokens != 64, group size > 16 */
+  SPKV_E_CUDA = -4,             /* a CUDA runtime call failed                          */
+  SPKV_E_POOL_EXHAUSTED = -5,   /* device: no free page; the pair was NOT stored       */
+  SPKV_E_CONTEXT_OVERFLOW = -6, /* device: a unit's page table is full                 */
+  SPKV_E_WORKSPACE = -7,        /* workspace missing or too small                      */
+  SPKV_E_TIMEOUT = -8,          /* device: a bounded wait on a copy ran out            */
+  SPKV_E_BOUNDS = -9            /* device: a sequence id outside [0, max_seqs)         */
+};
+
+typedef struct {
+  int32_t n_layers;
+  int32_t max_seqs;     /* sequence slots; seq ids are 0..max_seqs-1                    */
+  int32_t n_q_heads;    /* multiple of n_kv_heads; group size G = n_q_heads/n_kv_heads  */
+  int32_t n_kv_heads;
+  int32_t head_dim;     /* must be 128                                                  */
+  int32_t window;       /* w >= 1: pairs always visible (paper default 128)             */
+  int32_t page_tokens;  /* must be 64                                                   */
+  int32_t max_context;  /* upper bound on kept pairs per unit (sizes the page tables)   */
+  int64_t pool_pages;   /* pages shared by all compact caches                           */
+  float tau;            /* utility threshold in [0,1]; <= 0 keeps all, >= 1 keeps none  */
+  int32_t flags;        /* reserved, 0                                                  */
+} spkv_config_t;
+
+/* Utility predictor f of Eq. 1 (the sigmoid is never evaluated: the decision is taken
+ * in logit space, u >= tau  <=>  logit >= log(tau/(1-tau))).
+ *   kind 0, linear:  logit[h] = <W1[h,:], x> + b1[h]            W1 [n_kv_heads, d_in]
+ *   kind 1, MLP   :  logit[h] = <W2[h,:], SiLU(W1 x + b1)> + b2[h]
+ *                    W1 [hidden, d_in], b1 [hidden], W2 [n_kv_heads, hidden], b2 [n_kv_heads]
+ *                    (two-layer perceptron of the paper's reference listing)
+ * Weights are bf16, biases float32, all device pointers.  d_in and hidden are multiples
+ * of 8. */
+typedef struct {
+  int32_t kind;
+  int32_t d_in;
+  int32_t hidden; /* kind 1 only */
+  int32_t reserved;
+  const void *d_W1;
+  const float *d_b1;
+  const void *d_W2;
+  const float *d_b2;
+} spkv_predictor_t;
+
+typedef struct {
+  int64_t units;           /* n_layers * max_seqs * n_kv_heads                          */
+  int64_t pairs_seen;      /* sum over units of t                                       */
+  int64_t pairs_kept;      /* sum over units of compact-cache lengths                   */
+  int64_t pairs_in_window; /* sum over units of min(t, w)                               */
+  int64_t pairs_evicted;   /* sum over units of max(t - w, 0)                           */
+  int64_t gates_open;      /* number of pairs, window included, with logit >= tau_logit */
+  int64_t pages_in_use;    /* pool pages held by compact caches                         */
+  int64_t pages_free;
+  int64_t bytes_resident;  /* K/V bytes a decode step reads: kept + window pairs        */
+  double density_all;      /* Eq. 8: gates_open / pairs_seen                            */
+  double density_cache;    /* pairs_kept / pairs_evicted (fraction kept in the
+                              long-term cache, the figure the paper reports)           */
+} spkv_stats_t;
+
+/* ---- cache lifetime ---------------------------------------------------------------- */
+
+/* Bytes of device memory a cache with this configuration needs (host only). */
+int spkv_arena_bytes(const spkv_config_t *cfg, size_t *out_bytes);
+
+/* Lays the cache out inside the caller's arena (256-byte aligned device memory of at
+ * least spkv_arena_bytes bytes) and enqueues its initialisation on `stream`.  The arena
+ * must stay alive and untouched by the caller until spkv_cache_destroy.
+ * Paper: Appendix "Inference Kernels" (paged pool, per-head page-index arrays, ring
+ * window kept by metadata); here the capacity is fixed at creation instead of grown. */
+int spkv_cache_create(const spkv_config_t *cfg, void *d_arena, size_t arena_bytes,
+                      spkv_stream_t stream, spkv_cache_t **out);
+
+/* Frees the host handle only (the arena belongs to the caller). */
+int spkv_cache_destroy(spkv_cache_t *cache);
+
+/* Empties every unit of sequence `seq` (all layers) and returns its pages to the pool. */
+int spkv_cache_reset_seq(spkv_cache_t *cache, int32_t seq, spkv_stream_t stream);
+
+/* Changes tau for all FUTURE evictions (the paper adjusts sparsity a posteriori by
+ * changing the threshold; pairs already dropped stay dropped). */
+int spkv_set_tau(spkv_cache_t *cache, float tau);
+
+/* ---- the hot path ------------------------------------------------------------------ */
+
+/* Step 1, score + threshold (Eq. 1-2).  d_x [n_tok, d_in] bf16 -> d_logits_out
+ * [n_tok, n_kv_heads] float32 (fp32 accumulation).  d_flags_out (optional, may be NULL)
+ * [n_tok, n_kv_heads] uint8 = 1 where logit >= tau_logit under the current tau. */
+int spkv_score(spkv_cache_t *cache, const spkv_predictor_t *pred, const void *d_x,
+               int32_t n_tok, float *d_logits_out, uint8_t *d_flags_out,
+               spkv_stream_t stream);
+
+/* Step 2, append + evict, one new pair per listed sequence and KV head (Appendix
+ * "Inference Kernels": fused token append).  For each unit: the new pair (position t)
+ * goes to ring slot t mod w; if t >= w the pair of position t-w leaves the ring first
+ * and is appended to the unit's compact cache iff its stored logit >= tau_logit.
+ *   d_seq_ids [B] int32, d_k/d_v [B, n_kv_heads, 128] bf16, d_logits [B, n_kv_heads] f32.
+ * On SPKV_E_POOL_EXHAUSTED / SPKV_E_CONTEXT_OVERFLOW the evicted pair is dropped, the
+ * unit's length is unchanged and the sticky status is set. */
+int spkv_append_evict(spkv_cache_t *cache, int32_t layer, const int32_t *d_seq_ids, int32_t B,
+                      const void *d_k, const void *d_v, const float *d_logits,
+                      spkv_stream_t stream);
+
+/* Workspace bytes spkv_decode_attention needs for a batch of B sequences. */
+size_t spkv_decode_workspace_bytes(const spkv_config_t *cfg, int32_t B);
+
+/* Step 3, decode attention (Eq. 3-5) for the query whose pair was appended last:
+ * out[b, j, :] = softmax(<q[b,j], K_vis> * sm_scale) V_vis with K_vis = ring U compact
+ * cache of KV head floor(j / G).  Split over the keys across thread blocks, partial
+ * results merged by their log-sum-exp weights.
+ *   d_q [B, n_q_heads, 128] bf16 -> d_out [B, n_q_heads, 128] bf16;
+ *   d_lse_opt [B, n_q_heads] float32 natural-log sum-exp of the scaled scores, or NULL;
+ *   d_workspace: >= spkv_decode_workspace_bytes(cfg, B) bytes, 256-byte aligned; its
+ *   contents need not be preserved between calls, but it must have been zero-filled
+ *   once before its first use. */
+int spkv_decode_attention(spkv_cache_t *cache, int32_t layer, const int32_t *d_seq_ids,
+                          int32_t B, const void *d_q, void *d_out, float *d_lse_opt,
+                          float sm_scale, void *d_workspace, size_t workspace_bytes,
+                          spkv_stream_t stream);
+
+/* Workspace bytes spkv_prefill needs for a chunk of C pairs. */
+size_t spkv_prefill_workspace_bytes(const spkv_config_t *cfg, int32_t C);
+
+/* Companion path, chunked prefill of C pairs for one sequence and layer: equivalent to
+ * C x (spkv_append_evict, spkv_decode_attention) -- the paper's chunked-prefill protocol
+ * with the cache compressed after each chunk -- done as: stream compaction of the pairs
+ * that leave the window (ballot + prefix sum, ascending position), tensor-core attention
+ * of every query of the chunk over compact cache U window (Eq. 3-5), ring update.
+ *   d_q [C, n_q_heads, 128], d_k/d_v [C, n_kv_heads, 128] bf16, d_logits [C, n_kv_heads],
+ *   d_out [C, n_q_heads, 128] bf16.  d_q = d_out = NULL builds the cache state only. */
+int spkv_prefill(spkv_cache_t *cache, int32_t layer, int32_t seq, int32_t C, const void *d_q,
+                 const void *d_k, const void *d_v, const float *d_logits, void *d_out,
+                 float sm_scale, void *d_workspace, size_t workspace_bytes,
+                 spkv_stream_t stream);
+
+/* One decode step of one layer from HOST buffers (pinned memory recommended): copies
+ * x, q, k, v to the device staging area, runs score -> append/evict -> decode attention,
+ * copies the output back, all enqueued on `stream` (no synchronisation).
+ *   h_x [B, d_in], h_q [B, n_q_heads, 128], h_k/h_v [B, n_kv_heads, 128] bf16,
+ *   h_out [B, n_q_heads, 128] bf16;
+ *   d_staging: >= spkv_decode_step_staging_bytes(cfg, B, d_in) bytes (inputs, logits,
+ *   output and the decode workspace live there; zero-filled once before first use). */
+size_t spkv_decode_step_staging_bytes(const spkv_config_t *cfg, int32_t B, int32_t d_in);
+int spkv_decode_step_host(spkv_cache_t *cache, int32_t layer, const spkv_predictor_t *pred,
+                          const int32_t *d_seq_ids, int32_t B, const void *h_x, const void *h_q,
+                          const void *h_k, const void *h_v, void *h_out, float sm_scale,
+                          void *d_staging, size_t staging_bytes, spkv_stream_t stream);
+
+/* ---- introspection ----------------------------------------------------------------- */
+
+/* Synchronises `stream` and returns the sticky device status (SPKV_OK or the first
+ * device-side error).  spkv_clear_status resets it. */
+int spkv_status(spkv_cache_t *cache, spkv_stream_t stream);
+int spkv_clear_status(spkv_cache_t *cache, spkv_stream_t stream);
+
+/* Gate density (Eq. 8) and memory accounting; synchronises `stream`. */
+int spkv_cache_stats(spkv_cache_t *cache, spkv_stream_t stream, spkv_stats_t *out);
+
+/* Lengths of one layer: h_len / h_t [max_seqs, n_kv_heads] int32 (kept pairs / pairs
+ * received); either may be NULL.  Synchronises `stream`. */
+int spkv_read_lengths(spkv_cache_t *cache, int32_t layer, int32_t *h_len, int32_t *h_t,
+                      spkv_stream_t stream);
+
+/* Compact cache of one unit in logical (ascending position) order: up to `cap` pairs.
+ * h_pos [cap] int32, h_k/h_v [cap,128] bf16 (each may be NULL); *n_out = stored length.
+ * Synchronises `stream`. */
+int spkv_read_kept(spkv_cache_t *cache, int32_t layer, int32_t seq, int32_t kvh, int32_t *h_pos,
+                   void *h_k, void *h_v, int32_t cap, int32_t *n_out, spkv_stream_t stream);
+
+/* Ring of one unit in ascending position order: min(t, w) pairs.  h_pos [w] int32,
+ * h_k/h_v [w,128] bf16, h_logits [w] float32 (each may be NULL).  Synchronises. */
+int spkv_read_window(spkv_cache_t *cache, int32_t layer, int32_t seq, int32_t kvh,
+                     int32_t *h_pos, void *h_k, void *h_v, float *h_logits, int32_t *n_out,
+                     spkv_stream_t stream);
+
+/* The float32 logit-space threshold currently in force. */
+float spkv_tau_logit(const spkv_cache_t *cache);
+
+const char *spkv_error_string(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPKV_H_ */

@@ -1,0 +1,111 @@
+// Step 2 of the hot path: fused append + evict (paper, Appendix "Inference Kernels").
+//
+// One warp owns one unit (layer, sequence, KV head) for the duration of the call, so a
+// unit's ring, length, page table and pages have a single writer and no locks are
+// needed.  The only atomic is the pop from the shared free-page stack.
+//
+// Bytes per unit and step: 512 B read (new k, v) + 512 B written to the ring slot, and,
+// when the pair leaving the ring is kept, 512 B read back + 512 B written to its page.
+#include "spkv_internal.cuh"
+
+namespace spkv {
+
+// Pops a free page (lane 0) and clears its value block, so that rows past a page's
+// valid count always hold zeros (the attention kernels multiply them by weight 0).
+// Returns the global page index or -1.
+__device__ inline int alloc_page(const CacheView &c, int lane) {
+  int page = -1;
+  if (lane == 0) {
+    int top = atomicSub(&c.status[1], 1);
+    if (top <= 0) {
+      atomicAdd(&c.status[1], 1);
+    } else {
+      page = c.free_stack[top - 1];
+    }
+  }
+  page = __shfl_sync(0xffffffffu, page, 0);
+  if (page >= 0) {
+    uint4 *vb = reinterpret_cast<uint4 *>(c.pages + (int64_t)page * kPageElems + kBlockElems);
+    for (int i = lane; i < kBlockElems * 2 / 16; i += 32) vb[i] = make_uint4(0, 0, 0, 0);
+  }
+  return page;
+}
+
+__global__ void __launch_bounds__(128)
+append_evict_kernel(CacheView c, int layer, const int32_t *__restrict__ seq_ids, int B,
+                    const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new,
+                    const float *__restrict__ logits, float tau_logit) {
+  const int lane = threadIdx.x & 31;
+  const int item = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (item >= B * c.Hkv) return;
+  const int b = item / c.Hkv, kvh = item % c.Hkv;
+  const int seq = seq_ids[b];
+  if (seq < 0 || seq >= c.S) {
+    if (lane == 0) set_status(c, SPKV_E_BOUNDS);
+    return;
+  }
+  const int u = unit_index(c, layer, seq, kvh);
+  const int t = c.t[u];
+  const int slot = t % c.w;
+  const int row = slot % kP;
+  // lanes 0-15 move the key row, lanes 16-31 the value row, one 16-byte chunk each
+  const int chunk = lane & 15;
+  const int blk = (lane >> 4) * kBlockElems;
+  __nv_bfloat16 *ring = c.pages + ring_page(c, u, slot / kP) * kPageElems;
+  uint4 *ring_cell = reinterpret_cast<uint4 *>(ring + blk + swz_off(row, chunk));
+
+  if (t >= c.w) {
+    // the pair of position t - w leaves the window: threshold decision on its stored logit
+    const float lg = c.ring_logit[(size_t)u * c.w + slot];
+    if (lg >= tau_logit) {
+      const int n = c.len[u];
+      const int pj = n / kP, prow = n % kP;
+      int page = -1, err = 0;
+      if (pj >= c.max_pages) {
+        err = SPKV_E_CONTEXT_OVERFLOW;
+      } else if (prow == 0) {
+        page = alloc_page(c, lane);
+        if (page < 0) err = SPKV_E_POOL_EXHAUSTED;
+        else if (lane == 0) c.table[(size_t)u * c.max_pages + pj] = page;
+      } else {
+        page = c.table[(size_t)u * c.max_pages + pj];
+      }
+      if (err) {
+        if (lane == 0) set_status(c, err);
+      } else {
+        __syncwarp();
+        __nv_bfloat16 *dst = c.pages + (int64_t)page * kPageElems;
+        *reinterpret_cast<uint4 *>(dst + blk + swz_off(prow, chunk)) = *ring_cell;
+        if (lane == 0) {
+          c.pos_pool[((int64_t)page - c.n_ring_pages_total) * kP + prow] = t - c.w;
+          c.len[u] = n + 1;
+        }
+      }
+    }
+  }
+  const uint4 *src = (lane < 16 ? k_new : v_new) + (size_t)item * 16 + chunk;
+  *ring_cell = *src;
+  if (lane == 0) {
+    c.ring_logit[(size_t)u * c.w + slot] = logits[item];
+    c.t[u] = t + 1;
+  }
+}
+
+}  // namespace spkv
+
+using namespace spkv;
+
+extern "C" int spkv_append_evict(spkv_cache_t *cache, int32_t layer, const int32_t *d_seq_ids,
+                                 int32_t B, const void *d_k, const void *d_v,
+                                 const float *d_logits, spkv_stream_t stream) {
+  if (!cache || layer < 0 || layer >= cache->cfg.n_layers || B < 0 || B > cache->cfg.max_seqs)
+    return SPKV_E_INVALID;
+  if (B == 0) return SPKV_OK;
+  if (!d_seq_ids || !d_k || !d_v || !d_logits) return SPKV_E_INVALID;
+  if (((uintptr_t)d_k | (uintptr_t)d_v) & 15) return SPKV_E_INVALID;
+  const int items = B * cache->view.Hkv;
+  append_evict_kernel<<<(items + 3) / 4, 128, 0, as_stream(stream)>>>(
+      cache->view, layer, d_seq_ids, B, static_cast<const uint4 *>(d_k),
+      static_cast<const uint4 *>(d_v), d_logits, cache->tau_logit);
+  return check_stream_error(cudaGetLastError());
+}

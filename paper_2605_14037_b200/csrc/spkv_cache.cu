@@ -1,0 +1,327 @@
+// Cache lifetime, bookkeeping and read-back (host side + small maintenance kernels).
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "spkv_internal.cuh"
+
+namespace spkv {
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int check_stream_error(cudaError_t e) { return e == cudaSuccess ? SPKV_OK : SPKV_E_CUDA; }
+
+// Eq. 2 moved to logit space: u >= tau  <=>  logit >= log(tau / (1 - tau)).
+float tau_to_logit(float tau) {
+  if (!(tau > 0.0f)) return -INFINITY;
+  if (!(tau < 1.0f)) return INFINITY;
+  return (float)log((double)tau / (1.0 - (double)tau));
+}
+
+static int validate(const spkv_config_t *c) {
+  if (!c) return SPKV_E_INVALID;
+  if (c->n_layers < 1 || c->max_seqs < 1 || c->n_kv_heads < 1 || c->n_q_heads < 1) return SPKV_E_INVALID;
+  if (c->n_q_heads % c->n_kv_heads) return SPKV_E_INVALID;
+  if (c->window < 1 || c->max_context < 1 || c->pool_pages < 0) return SPKV_E_INVALID;
+  if (c->head_dim != kD || c->page_tokens != kP) return SPKV_E_UNSUPPORTED;
+  if (c->n_q_heads / c->n_kv_heads > kMaxGroup) return SPKV_E_UNSUPPORTED;
+  if (c->tau != c->tau) return SPKV_E_INVALID;
+  int64_t units = (int64_t)c->n_layers * c->max_seqs * c->n_kv_heads;
+  int64_t ring_pages = (c->window + kP - 1) / kP;
+  if (units > (1 << 24)) return SPKV_E_INVALID;
+  if (units * ring_pages + c->pool_pages > 0x7fffffffLL) return SPKV_E_INVALID;
+  return SPKV_OK;
+}
+
+static void make_layout(const spkv_config_t *c, Layout *l) {
+  size_t units = (size_t)c->n_layers * c->max_seqs * c->n_kv_heads;
+  size_t ring_pages = (c->window + kP - 1) / kP;
+  size_t max_pages = ((size_t)c->max_context + kP - 1) / kP;
+  size_t o = 0;
+  l->off_header = o; o = align_up(o + 256, 256);
+  l->off_t = o;      o = align_up(o + units * 4, 256);
+  l->off_len = o;    o = align_up(o + units * 4, 256);
+  l->off_table = o;  o = align_up(o + units * max_pages * 4, 256);
+  l->off_free = o;   o = align_up(o + (size_t)c->pool_pages * 4, 256);
+  l->off_pos = o;    o = align_up(o + (size_t)c->pool_pages * kP * 4, 256);
+  l->off_rlogit = o; o = align_up(o + units * (size_t)c->window * 4, 256);
+  o = align_up(o, 1024);
+  l->off_pages = o;  o += (units * ring_pages + (size_t)c->pool_pages) * kPageBytes;
+  l->total = o;
+}
+
+__global__ void init_free_stack_kernel(int32_t *stack, int32_t *free_top, int64_t pool_pages,
+                                       int64_t first) {
+  int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i == 0) *free_top = (int32_t)pool_pages;
+  // popped from the top: ascending page order for a fresh cache
+  if (i < pool_pages) stack[i] = (int32_t)(first + (pool_pages - 1 - i));
+}
+
+// One block per (layer, kvh) of the sequence being reset.
+__global__ void reset_seq_kernel(CacheView c, int seq) {
+  const int layer = blockIdx.x / c.Hkv, kvh = blockIdx.x % c.Hkv;
+  const int u = unit_index(c, layer, seq, kvh);
+  const int n_pages = (c.len[u] + kP - 1) / kP;
+  __shared__ int base;
+  if (threadIdx.x == 0) base = n_pages ? atomicAdd(&c.status[1], n_pages) : 0;
+  __syncthreads();
+  for (int j = threadIdx.x; j < n_pages; j += blockDim.x)
+    c.free_stack[base + j] = c.table[(size_t)u * c.max_pages + j];
+  uint4 *ring = reinterpret_cast<uint4 *>(c.pages + ring_page(c, u, 0) * kPageElems);
+  const int n16 = c.ring_pages * (kPageBytes / 16);
+  for (int i = threadIdx.x; i < n16; i += blockDim.x) ring[i] = make_uint4(0, 0, 0, 0);
+  for (int i = threadIdx.x; i < c.w; i += blockDim.x) c.ring_logit[(size_t)u * c.w + i] = 0.f;
+  __syncthreads();
+  if (threadIdx.x == 0) { c.len[u] = 0; c.t[u] = 0; }
+}
+
+}  // namespace spkv
+
+using namespace spkv;
+
+extern "C" int spkv_arena_bytes(const spkv_config_t *cfg, size_t *out_bytes) {
+  int rc = validate(cfg);
+  if (rc) return rc;
+  if (!out_bytes) return SPKV_E_INVALID;
+  Layout l;
+  make_layout(cfg, &l);
+  *out_bytes = l.total;
+  return SPKV_OK;
+}
+
+extern "C" int spkv_cache_create(const spkv_config_t *cfg, void *d_arena, size_t arena_bytes,
+                                 spkv_stream_t stream, spkv_cache_t **out) {
+  int rc = validate(cfg);
+  if (rc) return rc;
+  if (!d_arena || !out || ((uintptr_t)d_arena & 255)) return SPKV_E_INVALID;
+  Layout l;
+  make_layout(cfg, &l);
+  if (arena_bytes < l.total) return SPKV_E_ARENA_TOO_SMALL;
+  spkv_cache *c = new (std::nothrow) spkv_cache();
+  if (!c) return SPKV_E_INVALID;
+  c->cfg = *cfg;
+  c->layout = l;
+  c->arena = d_arena;
+  c->tau_logit = tau_to_logit(cfg->tau);
+  char *base = static_cast<char *>(d_arena);
+  CacheView &v = c->view;
+  v.L = cfg->n_layers; v.S = cfg->max_seqs; v.Hq = cfg->n_q_heads; v.Hkv = cfg->n_kv_heads;
+  v.G = cfg->n_q_heads / cfg->n_kv_heads;
+  v.w = cfg->window;
+  v.ring_pages = (cfg->window + kP - 1) / kP;
+  v.max_pages = (cfg->max_context + kP - 1) / kP;
+  v.n_units = cfg->n_layers * cfg->max_seqs * cfg->n_kv_heads;
+  v.pool_pages = cfg->pool_pages;
+  v.n_ring_pages_total = (int64_t)v.n_units * v.ring_pages;
+  v.status = reinterpret_cast<int32_t *>(base + l.off_header);
+  v.t = reinterpret_cast<int32_t *>(base + l.off_t);
+  v.len = reinterpret_cast<int32_t *>(base + l.off_len);
+  v.table = reinterpret_cast<int32_t *>(base + l.off_table);
+  v.free_stack = reinterpret_cast<int32_t *>(base + l.off_free);
+  v.pos_pool = reinterpret_cast<int32_t *>(base + l.off_pos);
+  v.ring_logit = reinterpret_cast<float *>(base + l.off_rlogit);
+  v.pages = reinterpret_cast<__nv_bfloat16 *>(base + l.off_pages);
+
+  int dev = 0;
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+    delete c;
+    return SPKV_E_CUDA;
+  }
+  c->sm_count = prop.multiProcessorCount;
+
+  cudaStream_t s = as_stream(stream);
+  // metadata and ring pages start at zero; pool pages are zeroed when first allocated
+  cudaError_t e = cudaMemsetAsync(base, 0, l.off_pages + (size_t)v.n_ring_pages_total * kPageBytes, s);
+  if (e == cudaSuccess && v.pool_pages > 0) {
+    int64_t n = v.pool_pages;
+    init_free_stack_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(v.free_stack, &v.status[1], n,
+                                                                      v.n_ring_pages_total);
+    e = cudaGetLastError();
+  }
+  if (e != cudaSuccess) {
+    delete c;
+    return SPKV_E_CUDA;
+  }
+  *out = c;
+  return SPKV_OK;
+}
+
+extern "C" int spkv_cache_destroy(spkv_cache_t *cache) {
+  if (!cache) return SPKV_E_INVALID;
+  delete cache;
+  return SPKV_OK;
+}
+
+extern "C" int spkv_cache_reset_seq(spkv_cache_t *cache, int32_t seq, spkv_stream_t stream) {
+  if (!cache || seq < 0 || seq >= cache->cfg.max_seqs) return SPKV_E_INVALID;
+  reset_seq_kernel<<<cache->view.L * cache->view.Hkv, 256, 0, as_stream(stream)>>>(cache->view, seq);
+  return check_stream_error(cudaGetLastError());
+}
+
+extern "C" int spkv_set_tau(spkv_cache_t *cache, float tau) {
+  if (!cache || tau != tau) return SPKV_E_INVALID;
+  cache->cfg.tau = tau;
+  cache->tau_logit = tau_to_logit(tau);
+  return SPKV_OK;
+}
+
+extern "C" float spkv_tau_logit(const spkv_cache_t *cache) { return cache ? cache->tau_logit : NAN; }
+
+extern "C" int spkv_status(spkv_cache_t *cache, spkv_stream_t stream) {
+  if (!cache) return SPKV_E_INVALID;
+  int32_t st = 0;
+  if (cudaStreamSynchronize(as_stream(stream)) != cudaSuccess) return SPKV_E_CUDA;
+  if (cudaMemcpy(&st, cache->view.status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return SPKV_E_CUDA;
+  return st;
+}
+
+extern "C" int spkv_clear_status(spkv_cache_t *cache, spkv_stream_t stream) {
+  if (!cache) return SPKV_E_INVALID;
+  return check_stream_error(cudaMemsetAsync(cache->view.status, 0, 4, as_stream(stream)));
+}
+
+extern "C" int spkv_read_lengths(spkv_cache_t *cache, int32_t layer, int32_t *h_len, int32_t *h_t,
+                                 spkv_stream_t stream) {
+  if (!cache || layer < 0 || layer >= cache->cfg.n_layers) return SPKV_E_INVALID;
+  const CacheView &v = cache->view;
+  if (cudaStreamSynchronize(as_stream(stream)) != cudaSuccess) return SPKV_E_CUDA;
+  size_t n = (size_t)v.S * v.Hkv, off = (size_t)layer * n;
+  if (h_len && cudaMemcpy(h_len, v.len + off, n * 4, cudaMemcpyDeviceToHost) != cudaSuccess) return SPKV_E_CUDA;
+  if (h_t && cudaMemcpy(h_t, v.t + off, n * 4, cudaMemcpyDeviceToHost) != cudaSuccess) return SPKV_E_CUDA;
+  return SPKV_OK;
+}
+
+// Copies one page to the host and undoes the row swizzle for rows [0, n_rows).
+static int fetch_page(const CacheView &v, int64_t gpage, int n_rows, uint16_t *tmp, uint16_t *h_k,
+                      uint16_t *h_v) {
+  if (cudaMemcpy(tmp, v.pages + gpage * kPageElems, kPageBytes, cudaMemcpyDeviceToHost) != cudaSuccess)
+    return SPKV_E_CUDA;
+  for (int r = 0; r < n_rows; ++r)
+    for (int ch = 0; ch < 16; ++ch) {
+      if (h_k) memcpy(h_k + (size_t)r * kD + ch * 8, tmp + swz_off(r, ch), 16);
+      if (h_v) memcpy(h_v + (size_t)r * kD + ch * 8, tmp + kBlockElems + swz_off(r, ch), 16);
+    }
+  return SPKV_OK;
+}
+
+extern "C" int spkv_read_kept(spkv_cache_t *cache, int32_t layer, int32_t seq, int32_t kvh,
+                              int32_t *h_pos, void *h_k, void *h_v, int32_t cap, int32_t *n_out,
+                              spkv_stream_t stream) {
+  if (!cache || layer < 0 || layer >= cache->cfg.n_layers || seq < 0 || seq >= cache->cfg.max_seqs ||
+      kvh < 0 || kvh >= cache->cfg.n_kv_heads || cap < 0)
+    return SPKV_E_INVALID;
+  const CacheView &v = cache->view;
+  if (cudaStreamSynchronize(as_stream(stream)) != cudaSuccess) return SPKV_E_CUDA;
+  const int u = (layer * v.S + seq) * v.Hkv + kvh;
+  int32_t len = 0;
+  if (cudaMemcpy(&len, v.len + u, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return SPKV_E_CUDA;
+  if (n_out) *n_out = len;
+  int n = len < cap ? len : cap;
+  int n_pages = (n + kP - 1) / kP;
+  if (n_pages == 0) return SPKV_OK;
+  std::vector<int32_t> table(n_pages);
+  if (cudaMemcpy(table.data(), v.table + (size_t)u * v.max_pages, (size_t)n_pages * 4,
+                 cudaMemcpyDeviceToHost) != cudaSuccess)
+    return SPKV_E_CUDA;
+  std::vector<uint16_t> tmp(kPageElems);
+  for (int j = 0; j < n_pages; ++j) {
+    int rows = n - j * kP < kP ? n - j * kP : kP;
+    int64_t g = table[j];
+    if (g < v.n_ring_pages_total || g >= v.n_ring_pages_total + v.pool_pages) return SPKV_E_INVALID;
+    int rc = fetch_page(v, g, rows, tmp.data(),
+                        h_k ? (uint16_t *)h_k + (size_t)j * kP * kD : nullptr,
+                        h_v ? (uint16_t *)h_v + (size_t)j * kP * kD : nullptr);
+    if (rc) return rc;
+    if (h_pos && cudaMemcpy(h_pos + (size_t)j * kP, v.pos_pool + (g - v.n_ring_pages_total) * kP,
+                            (size_t)rows * 4, cudaMemcpyDeviceToHost) != cudaSuccess)
+      return SPKV_E_CUDA;
+  }
+  return SPKV_OK;
+}
+
+extern "C" int spkv_read_window(spkv_cache_t *cache, int32_t layer, int32_t seq, int32_t kvh,
+                                int32_t *h_pos, void *h_k, void *h_v, float *h_logits,
+                                int32_t *n_out, spkv_stream_t stream) {
+  if (!cache || layer < 0 || layer >= cache->cfg.n_layers || seq < 0 || seq >= cache->cfg.max_seqs ||
+      kvh < 0 || kvh >= cache->cfg.n_kv_heads)
+    return SPKV_E_INVALID;
+  const CacheView &v = cache->view;
+  if (cudaStreamSynchronize(as_stream(stream)) != cudaSuccess) return SPKV_E_CUDA;
+  const int u = (layer * v.S + seq) * v.Hkv + kvh;
+  int32_t t = 0;
+  if (cudaMemcpy(&t, v.t + u, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return SPKV_E_CUDA;
+  const int n = t < v.w ? t : v.w;
+  if (n_out) *n_out = n;
+  std::vector<uint16_t> ring((size_t)v.ring_pages * kPageElems);
+  std::vector<float> lg(v.w);
+  if (cudaMemcpy(ring.data(), v.pages + (int64_t)u * v.ring_pages * kPageElems,
+                 ring.size() * 2, cudaMemcpyDeviceToHost) != cudaSuccess)
+    return SPKV_E_CUDA;
+  if (cudaMemcpy(lg.data(), v.ring_logit + (size_t)u * v.w, (size_t)v.w * 4, cudaMemcpyDeviceToHost) !=
+      cudaSuccess)
+    return SPKV_E_CUDA;
+  for (int j = 0; j < n; ++j) {
+    const int s = t - n + j, slot = s % v.w, pg = slot / kP, r = slot % kP;
+    const uint16_t *page = ring.data() + (size_t)pg * kPageElems;
+    if (h_pos) h_pos[j] = s;
+    if (h_logits) h_logits[j] = lg[slot];
+    for (int ch = 0; ch < 16; ++ch) {
+      if (h_k) memcpy((uint16_t *)h_k + (size_t)j * kD + ch * 8, page + swz_off(r, ch), 16);
+      if (h_v) memcpy((uint16_t *)h_v + (size_t)j * kD + ch * 8, page + kBlockElems + swz_off(r, ch), 16);
+    }
+  }
+  return SPKV_OK;
+}
+
+extern "C" int spkv_cache_stats(spkv_cache_t *cache, spkv_stream_t stream, spkv_stats_t *out) {
+  if (!cache || !out) return SPKV_E_INVALID;
+  const CacheView &v = cache->view;
+  if (cudaStreamSynchronize(as_stream(stream)) != cudaSuccess) return SPKV_E_CUDA;
+  std::vector<int32_t> t(v.n_units), len(v.n_units);
+  std::vector<float> lg((size_t)v.n_units * v.w);
+  int32_t hdr[2];
+  if (cudaMemcpy(t.data(), v.t, (size_t)v.n_units * 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
+      cudaMemcpy(len.data(), v.len, (size_t)v.n_units * 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
+      cudaMemcpy(lg.data(), v.ring_logit, lg.size() * 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
+      cudaMemcpy(hdr, v.status, 8, cudaMemcpyDeviceToHost) != cudaSuccess)
+    return SPKV_E_CUDA;
+  memset(out, 0, sizeof *out);
+  out->units = v.n_units;
+  for (int u = 0; u < v.n_units; ++u) {
+    const int nw = t[u] < v.w ? t[u] : v.w;
+    out->pairs_seen += t[u];
+    out->pairs_kept += len[u];
+    out->pairs_in_window += nw;
+    out->pairs_evicted += t[u] > v.w ? t[u] - v.w : 0;
+    out->pages_in_use += (len[u] + kP - 1) / kP;
+    out->gates_open += len[u];
+    for (int s = 0; s < nw; ++s)
+      if (lg[(size_t)u * v.w + s] >= cache->tau_logit) out->gates_open++;
+  }
+  out->pages_free = hdr[1];
+  out->bytes_resident = (out->pairs_kept + out->pairs_in_window) * 2 * kRowBytes;
+  out->density_all = out->pairs_seen ? (double)out->gates_open / (double)out->pairs_seen : 0.0;
+  out->density_cache = out->pairs_evicted ? (double)out->pairs_kept / (double)out->pairs_evicted : 0.0;
+  return SPKV_OK;
+}
+
+extern "C" const char *spkv_error_string(int code) {
+  switch (code) {
+    case SPKV_OK: return "ok";
+    case SPKV_E_INVALID: return "invalid argument";
+    case SPKV_E_ARENA_TOO_SMALL: return "arena too small";
+    case SPKV_E_UNSUPPORTED: return "unsupported configuration";
+    case SPKV_E_CUDA: return "CUDA runtime error";
+    case SPKV_E_POOL_EXHAUSTED: return "page pool exhausted";
+    case SPKV_E_CONTEXT_OVERFLOW: return "unit page table full";
+    case SPKV_E_WORKSPACE: return "workspace missing or too small";
+    case SPKV_E_TIMEOUT: return "bounded device wait ran out";
+    case SPKV_E_BOUNDS: return "sequence id out of range";
+    default: return "unknown error";
+  }
+}

@@ -1,0 +1,83 @@
+// Internal declarations shared by the translation units of libspkv.so.
+//
+// Arena layout (all offsets 256-byte aligned, computed by spkv_layout()):
+//   header      : status word, free-page counter
+//   t[]         : pairs received per unit                       int32 [n_units]
+//   len[]       : kept pairs per unit                           int32 [n_units]
+//   table[]     : page table per unit (global page indices)     int32 [n_units][max_pages]
+//   free_stack[]: LIFO of free pool pages (global page indices) int32 [pool_pages]
+//   pos_pool[]  : position of every kept pair, by pool page     int32 [pool_pages][P]
+//   ring_logit[]: stored logit per ring slot                    f32   [n_units][w]
+//   pages       : ring pages of every unit ([n_units][ring_pages]) followed by the pool
+//
+// A page holds P = 64 pairs: a 16 KB key block followed by a 16 KB value block.  Each
+// block is 64 rows of 256 B (one row per pair, 128 bf16).  Inside a row the sixteen
+// 16-byte chunks are stored XOR-swizzled by the row number, chunk' = chunk ^ (row & 7):
+// the page in HBM is exactly the shared-memory image the attention kernels want, so one
+// linear bulk copy brings it in and `ldmatrix` reads it without bank conflicts.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/spkv.h"
+
+namespace spkv {
+
+constexpr int kD = 128;            // head_dim
+constexpr int kP = 64;             // pairs per page
+constexpr int kRowBytes = kD * 2;  // 256
+constexpr int kBlockElems = kP * kD;        // bf16 elements in a key (or value) block
+constexpr int kPageElems = 2 * kBlockElems; // 16384 elements = 32 KB
+constexpr int kPageBytes = kPageElems * 2;
+constexpr int kMaxGroup = 16;      // query heads per KV head supported by the kernels
+
+struct CacheView {
+  int32_t L, S, Hq, Hkv, G, w, ring_pages, max_pages, n_units;
+  int64_t pool_pages, n_ring_pages_total;
+  int32_t *status;      // [0] sticky status, [1] free_top
+  int32_t *t;
+  int32_t *len;
+  int32_t *table;
+  int32_t *free_stack;
+  int32_t *pos_pool;
+  float *ring_logit;
+  __nv_bfloat16 *pages;
+};
+
+struct Layout {
+  size_t off_header, off_t, off_len, off_table, off_free, off_pos, off_rlogit, off_pages, total;
+};
+
+// element offset of (row, 16-byte chunk) inside a key or value block
+__host__ __device__ inline int swz_off(int row, int chunk) {
+  return row * kD + ((chunk ^ (row & 7)) << 3);
+}
+
+__device__ inline int unit_index(const CacheView &c, int layer, int seq, int kvh) {
+  return (layer * c.S + seq) * c.Hkv + kvh;
+}
+
+__device__ inline void set_status(const CacheView &c, int code) { atomicCAS(c.status, 0, code); }
+
+// global page index of ring page j of a unit
+__device__ inline int64_t ring_page(const CacheView &c, int unit, int j) {
+  return (int64_t)unit * c.ring_pages + j;
+}
+
+}  // namespace spkv
+
+struct spkv_cache {
+  spkv_config_t cfg;
+  spkv::CacheView view;
+  spkv::Layout layout;
+  void *arena;
+  float tau_logit;
+  int sm_count;
+};
+
+namespace spkv {
+int check_stream_error(cudaError_t e);
+inline cudaStream_t as_stream(spkv_stream_t s) { return reinterpret_cast<cudaStream_t>(s); }
+float tau_to_logit(float tau);
+}  // namespace spkv

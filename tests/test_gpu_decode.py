@@ -1,0 +1,114 @@
+"""GPU parity, step 3 (decode attention): outputs against the oracle's streaming form
+within |gpu - ref| <= 2e-3 + 1e-2 |ref| per element (bf16 inputs and output, fp32
+accumulation), log-sum-exp within 1e-3."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gpu_util import D, Workload, assert_attn_close, dev, load, to_dev_bf16
+from paper_2605_14037_b200 import spkv as _unused  # noqa: F401  (fails loudly if the library is missing)
+
+pytestmark = pytest.mark.gpu
+
+
+def run_and_check(spkv, w, T, Hq, Hkv, n_seq, tau, rates, check_steps, seed, sm_scale=None,
+                  pool_pages=200, max_context=8192):
+    cache = spkv.Cache(n_layers=2, max_seqs=n_seq + 1, n_q_heads=Hq, n_kv_heads=Hkv,
+                       max_context=max_context, pool_pages=pool_pages, window=w, tau=tau)
+    tl = cache.spkv_tau_logit()
+    G = Hq // Hkv
+    wl = Workload(seed, T, n_seq, Hq, Hkv, rates, tl)
+    seq_ids = list(range(n_seq, 0, -1))          # slots n_seq..1, reversed order
+    ids = torch.tensor(seq_ids, dtype=torch.int32, device=dev())
+    K, V, Q = to_dev_bf16(wl.K), to_dev_bf16(wl.V), to_dev_bf16(wl.q)
+    lg = torch.from_numpy(wl.logit).to(dev())
+    units = [[oracle.Unit(w, D) for _ in range(Hkv)] for _ in range(n_seq)]
+    scale = 1.0 / math.sqrt(D) if sm_scale is None else sm_scale
+    layer = 1
+    lse = torch.empty((n_seq, Hq), dtype=torch.float32, device=dev())
+    worst = 0.0
+    for t in range(T):
+        cache.spkv_append_evict(layer, ids, K[t], V[t], lg[t])
+        for s in range(n_seq):
+            for h in range(Hkv):
+                units[s][h].append(wl.K[t, s, h], wl.V[t, s, h], wl.logit[t, s, h], tl)
+        if t in check_steps:
+            out = cache.spkv_decode_attention(layer, ids, Q[t], lse=lse, sm_scale=sm_scale)
+            got = spkv.bits_from_bf16(out)                      # [n_seq, Hq, D]
+            got_lse = lse.cpu().numpy()
+            for s in range(n_seq):
+                for h in range(Hkv):
+                    ref, ref_lse = units[s][h].attend(
+                        np.ascontiguousarray(wl.q[t, s, h * G:(h + 1) * G]), scale, want_lse=True)
+                    worst = max(worst, assert_attn_close(got[s, h * G:(h + 1) * G], ref,
+                                                         f"t={t} seq={s} kvh={h}"))
+                    assert np.abs(got_lse[s, h * G:(h + 1) * G] - ref_lse).max() < 1e-3
+    assert cache.spkv_status() == 0
+    return worst
+
+
+@pytest.mark.parametrize("w,G,Hkv", [(128, 4, 2), (128, 1, 2), (128, 8, 1), (4, 4, 2), (1, 4, 1),
+                                     (100, 2, 2), (128, 16, 1), (128, 3, 2)])
+def test_decode_small_every_phase(w, G, Hkv):
+    """From the first token (t < w, partially filled ring) across page boundaries."""
+    spkv = load()
+    T = 330
+    steps = set(range(0, 8)) | {w - 2, w - 1, w, w + 1, 63, 64, 65, 127, 128, 129, 191, 192, 193,
+                                255, 256, 257, T - 1}
+    run_and_check(spkv, w, T, G * Hkv, Hkv, 2, 0.5, np.linspace(0.2, 0.9, Hkv), steps, 50 + w + G)
+
+
+@pytest.mark.parametrize("tau,rates", [(-math.inf, [0.3, 0.3]), (math.inf, [0.7, 0.7]),
+                                       (0.5, [0.0, 1.0]), (0.9, [0.05, 0.5])])
+def test_decode_limits(tau, rates):
+    """tau = -inf: full causal attention; tau = +inf: sliding window; r = 0 and r = 1 heads."""
+    spkv = load()
+    run_and_check(spkv, 128, 700, 8, 2, 2, tau, rates, {0, 127, 128, 300, 699}, 60)
+
+
+def test_decode_many_segments_and_ragged_batch():
+    """Units from 2 to ~80 pages in one call: ranges cut inside units, several merges."""
+    spkv = load()
+    run_and_check(spkv, 128, 5200, 32, 8, 2, 0.5,
+                  [0.0, 0.02, 0.1, 0.2, 0.35, 0.5, 0.8, 1.0], {4000, 5199}, 70,
+                  pool_pages=700, max_context=8192)
+
+
+def test_decode_scale_and_batch_of_one():
+    spkv = load()
+    run_and_check(spkv, 16, 400, 4, 1, 1, 0.5, [0.5], {0, 15, 16, 399}, 80, sm_scale=0.3)
+
+
+def test_decode_output_is_deterministic_and_repeatable():
+    spkv = load()
+    cache = spkv.Cache(n_layers=1, max_seqs=2, n_q_heads=8, n_kv_heads=2, max_context=4096,
+                       pool_pages=100, window=128, tau=0.5)
+    wl = Workload(90, 1500, 2, 8, 2, [0.4, 0.9], 0.0)
+    ids = torch.tensor([0, 1], dtype=torch.int32, device=dev())
+    K, V, Q = to_dev_bf16(wl.K), to_dev_bf16(wl.V), to_dev_bf16(wl.q)
+    lg = torch.from_numpy(wl.logit).to(dev())
+    for t in range(wl.T):
+        cache.spkv_append_evict(0, ids, K[t], V[t], lg[t])
+    a = cache.spkv_decode_attention(0, ids, Q[-1]).clone()
+    for _ in range(3):
+        b = cache.spkv_decode_attention(0, ids, Q[-1])
+        assert torch.equal(a, b)
+    # a sub-batch cuts the page ranges elsewhere: same rows up to summation order
+    one = cache.spkv_decode_attention(0, ids[1:], Q[-1][1:].contiguous())
+    assert torch.allclose(one[0].float(), a[1].float(), atol=2e-3, rtol=1e-2)
+
+
+def test_decode_workspace_checked():
+    spkv = load()
+    import ctypes as C
+    cache = spkv.Cache(n_layers=1, max_seqs=1, n_q_heads=2, n_kv_heads=1, max_context=64,
+                       pool_pages=1, window=4)
+    ids = torch.zeros(1, dtype=torch.int32, device=dev())
+    q = torch.zeros((1, 2, 128), dtype=torch.bfloat16, device=dev())
+    rc = spkv.lib().spkv_decode_attention(cache._h, 0, C.c_void_p(ids.data_ptr()), 1,
+                                          C.c_void_p(q.data_ptr()), C.c_void_p(q.data_ptr()), None,
+                                          0.1, None, 0, None)
+    assert rc == -7

@@ -1,0 +1,96 @@
+"""GPU parity, step 1 (score + threshold): float32 logits against the double-precision
+oracle, and decisions that agree wherever the logit is not within rounding of tau."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gpu_util import dev, load, to_dev_bf16
+from paper_2605_14037_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+# bf16 products are exact in float32; a length-d float32 accumulation of O(1) terms errs
+# by about d * 2^-24 * |partial sums| -- far below 1e-3 for d <= 8192.
+LOGIT_TOL = 1e-3
+
+
+def make_cache(spkv, Hkv, tau=0.5):
+    return spkv.Cache(n_layers=1, max_seqs=1, n_q_heads=Hkv, n_kv_heads=Hkv, max_context=64,
+                      pool_pages=1, window=4, tau=tau)
+
+
+@pytest.mark.parametrize("n_tok,d_in,Hkv", [(1, 512, 2), (16, 512, 8), (1000, 512, 8),
+                                            (37, 8, 1), (5, 4096, 3)])
+def test_linear_predictor(n_tok, d_in, Hkv):
+    spkv = load()
+    rng = np.random.default_rng(20 + n_tok)
+    cache = make_cache(spkv, Hkv, tau=0.7)
+    tl = cache.spkv_tau_logit()
+    x = synth.normal_bf16(rng, (n_tok, d_in))
+    W = synth.linear_predictor(rng, Hkv, d_in)
+    b = synth.bias_for_keep_rate(W, np.linspace(0.1, 0.9, Hkv), tl)
+    pred = spkv.make_predictor(to_dev_bf16(W), torch.from_numpy(b).to(dev()))
+    flags = torch.zeros((n_tok, Hkv), dtype=torch.uint8, device=dev())
+    got = cache.spkv_score(pred, to_dev_bf16(x), flags=flags).cpu().numpy()
+    ref = oracle.score_linear(x, W, b)
+    assert np.abs(got - ref).max() < LOGIT_TOL
+    f = flags.cpu().numpy().astype(bool)
+    assert np.array_equal(f, got >= np.float32(tl))            # flag == decision on the fp32 logit
+    differ = f != (ref >= float(tl))
+    assert (np.abs(ref[differ] - float(tl)) < LOGIT_TOL).all()  # only inside the rounding band
+    assert 0.2 < f.mean() < 0.8 or n_tok < 30
+
+
+@pytest.mark.parametrize("n_tok,d_in,hidden,Hkv", [(1, 512, 64, 2), (16, 512, 256, 8),
+                                                   (300, 256, 64, 4), (3, 1024, 8, 1)])
+def test_mlp_predictor(n_tok, d_in, hidden, Hkv):
+    spkv = load()
+    rng = np.random.default_rng(30 + n_tok)
+    cache = make_cache(spkv, Hkv)
+    tl = cache.spkv_tau_logit()
+    x = synth.normal_bf16(rng, (n_tok, d_in))
+    W1, b1, W2, b2 = synth.mlp_predictor(rng, Hkv, d_in, hidden)
+    pred = spkv.make_predictor(to_dev_bf16(W1), torch.from_numpy(b1).to(dev()),
+                               to_dev_bf16(W2), torch.from_numpy(b2).to(dev()))
+    flags = torch.zeros((n_tok, Hkv), dtype=torch.uint8, device=dev())
+    got = cache.spkv_score(pred, to_dev_bf16(x), flags=flags).cpu().numpy()
+    ref = oracle.score_mlp(x, W1, b1, W2, b2)
+    assert np.abs(got - ref).max() < LOGIT_TOL
+    f = flags.cpu().numpy().astype(bool)
+    assert np.array_equal(f, got >= np.float32(tl))
+    differ = f != (ref >= float(tl))
+    assert (np.abs(ref[differ] - float(tl)) < LOGIT_TOL).all()
+
+
+def test_score_then_append_chain_is_bit_exact_outside_the_guard_band():
+    """Tokens whose oracle logit lies within the rounding band of tau are resampled, after
+    which GPU-scored logits drive the same keep decisions as oracle-scored ones."""
+    spkv = load()
+    rng = np.random.default_rng(40)
+    Hkv, d_in, T, w = 2, 512, 500, 16
+    cache = spkv.Cache(n_layers=1, max_seqs=1, n_q_heads=Hkv, n_kv_heads=Hkv, max_context=1024,
+                       pool_pages=20, window=w, tau=0.5)
+    tl = cache.spkv_tau_logit()
+    W = synth.linear_predictor(rng, Hkv, d_in)
+    b = synth.bias_for_keep_rate(W, [0.2, 0.5], tl)
+    x = synth.normal_bf16(rng, (T, d_in))
+    for _ in range(10):
+        ref = oracle.score_linear(x, W, b)
+        near = (np.abs(ref - float(tl)) < LOGIT_TOL).any(axis=1)
+        if not near.any():
+            break
+        x[near] = synth.normal_bf16(rng, (int(near.sum()), d_in))
+    K, V = synth.normal_bf16(rng, (T, Hkv, 128)), synth.normal_bf16(rng, (T, Hkv, 128))
+    pred = spkv.make_predictor(to_dev_bf16(W), torch.from_numpy(b).to(dev()))
+    xd, Kd, Vd = to_dev_bf16(x), to_dev_bf16(K), to_dev_bf16(V)
+    ids = torch.zeros(1, dtype=torch.int32, device=dev())
+    for t in range(T):
+        lg = cache.spkv_score(pred, xd[t:t + 1])
+        cache.spkv_append_evict(0, ids, Kd[t:t + 1], Vd[t:t + 1], lg)
+    for h in range(Hkv):
+        u = oracle.Unit(w, 128)
+        u.prefill(np.ascontiguousarray(K[:, h]), np.ascontiguousarray(V[:, h]),
+                  ref[:, h].astype(np.float32), tl)
+        pos, k, v = cache.spkv_read_kept(0, 0, h)
+        assert np.array_equal(pos, u.kept()[0]) and np.array_equal(k, u.kept()[1])
