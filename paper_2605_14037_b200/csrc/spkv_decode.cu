@@ -137,7 +137,10 @@ __global__ void __launch_bounds__(128) decode_simt_kernel(DecodeArgs a) {
   block_exclusive_scan(s_np, s_pre, n, s_tmp);
   const int NP = s_pre[n];
   if (NP == 0) return;
-  const int nb = gridDim.x;
+  // with fewer pages than blocks only the first NP blocks work (every range non-empty,
+  // so the segments of a unit sit in consecutive blocks)
+  const int nb = min((int)gridDim.x, NP);
+  if ((int)blockIdx.x >= nb) return;
   int p = range_start(blockIdx.x, NP, nb);
   const int p_end = range_start(blockIdx.x + 1, NP, nb);
   if (p >= p_end) return;

@@ -125,18 +125,19 @@ def test_reset_returns_pages_and_replay_is_identical():
     spkv = load()
     w, T, Hkv = 16, 500, 2
     cache = spkv.Cache(n_layers=2, max_seqs=2, n_q_heads=4, n_kv_heads=Hkv, max_context=1024,
-                       pool_pages=40, window=w, tau=0.5)
+                       pool_pages=60, window=w, tau=0.5)
     tl = cache.spkv_tau_logit()
     wl = Workload(10, T, 2, 4, Hkv, [0.5, 0.8], tl, with_q=False)
     for layer in (0, 1):
         run_appends(cache, layer, [0, 1], wl)
+    assert cache.spkv_status() == 0
     before = cache.spkv_cache_stats()
     first = [cache.spkv_read_kept(1, 1, h) for h in range(Hkv)]
     cache.spkv_cache_reset_seq(1)
     st = cache.spkv_cache_stats()
     ln, tt = cache.spkv_read_lengths(1)
     assert ln[1].tolist() == [0, 0] and tt[1].tolist() == [0, 0] and tt[0].tolist() == [T, T]
-    assert st.pages_free + st.pages_in_use == 40 and st.pages_in_use < before.pages_in_use
+    assert st.pages_free + st.pages_in_use == 60 and st.pages_in_use < before.pages_in_use
     # replay sequence 1 alone in both layers: same logical content as the first time
     wl1 = Workload(10, T, 2, 4, Hkv, [0.5, 0.8], tl, with_q=False)
     wl1.K, wl1.V, wl1.logit = wl.K[:, 1:], wl.V[:, 1:], wl.logit[:, 1:]

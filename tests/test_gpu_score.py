@@ -39,7 +39,6 @@ def test_linear_predictor(n_tok, d_in, Hkv):
     assert np.array_equal(f, got >= np.float32(tl))            # flag == decision on the fp32 logit
     differ = f != (ref >= float(tl))
     assert (np.abs(ref[differ] - float(tl)) < LOGIT_TOL).all()  # only inside the rounding band
-    assert 0.2 < f.mean() < 0.8 or n_tok < 30
 
 
 @pytest.mark.parametrize("n_tok,d_in,hidden,Hkv", [(1, 512, 64, 2), (16, 512, 256, 8),
