@@ -1,13 +1,378 @@
-// Companion path: chunked prefill (placeholder until the kernels land).
+// Companion path: chunked prefill of C pairs for one (layer, sequence).
+//
+// By definition the result equals C x (append/evict, decode attention) -- the paper's
+// chunked-prefill protocol, cache compressed after every chunk (Section "Sparse decoding
+// approximation"), attention per Eq. 3-5.  It is computed in four launches:
+//
+//  A  plan     one block per KV head: thresholds the old ring pairs and the chunk pairs in
+//              position order ("staging" sequence of N = min(t0,w) + C pairs), exclusive
+//              prefix sum of the flags (warp ballot + popc, block carry), pops the pages
+//              the unit will need and extends its page table.
+//  B  scatter  stream compaction proper: every flagged staging pair whose position is
+//              <= t_last - w is copied to compact-cache index len0 + E[j] (ascending
+//              position, so order and indices are unique and bit-exact).
+//  ATT attention of every query of the chunk (tensor cores, bf16 mma.sync m16n8k16, fp32
+//              accumulation, online softmax) over
+//                (a) the first nvis(t) = len0 + E[t - w - p0 + 1] pairs of the compact cache
+//                    (the kept pairs with position <= t - w: a prefix, because the cache is in
+//                    ascending position order), and
+//                (b) the dense band t-w < s <= t, read from the not-yet-updated ring and the
+//                    chunk's own K/V.
+//              A kept pair inside the band is counted once: the prefix (a) stops at t - w.
+//  C  ring     the last min(C, w) pairs of the chunk overwrite their ring slots; t and len
+//              are advanced.
+//
+// Workspace per KV head: a 64-int header followed by E[0..N] (int32).
 #include "spkv_internal.cuh"
+#include "spkv_mma.cuh"
 
-extern "C" size_t spkv_prefill_workspace_bytes(const spkv_config_t *cfg, int32_t C) {
-  (void)cfg; (void)C;
-  return 256;
+namespace spkv {
+
+constexpr int kHdrInts = 64;
+enum { H_T0 = 0, H_LEN0, H_NOLD, H_N, H_NCOMMIT, H_LEN1, H_FAIL };
+
+struct PrefillArgs {
+  CacheView c;
+  int layer, seq, C;
+  const __nv_bfloat16 *q, *k, *v;  // [C][Hq][128], [C][Hkv][128]
+  const float *logits;             // [C][Hkv]
+  __nv_bfloat16 *out;              // [C][Hq][128]
+  float tau_logit, scale_log2;
+  int32_t *ws;                     // [Hkv][ws_stride]
+  int ws_stride;
+};
+
+__device__ inline int32_t *unit_ws(const PrefillArgs &a, int kvh) { return a.ws + (size_t)kvh * a.ws_stride; }
+
+// ---------------------------------------------------------------- A: plan (flags + scan)
+__global__ void __launch_bounds__(1024) prefill_plan_kernel(PrefillArgs a) {
+  const CacheView &c = a.c;
+  const int kvh = blockIdx.x;
+  const int u = unit_index(c, a.layer, a.seq, kvh);
+  int32_t *hdr = unit_ws(a, kvh);
+  int32_t *E = hdr + kHdrInts;
+  const int t0 = c.t[u], len0 = c.len[u];
+  const int n_old = min(t0, c.w), p0 = t0 - n_old;
+  const int N = n_old + a.C;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  __shared__ int s_warp[32];
+  __shared__ int s_carry, s_pages_base, s_fail;
+  if (tid == 0) { s_carry = 0; s_fail = 0; }
+  __syncthreads();
+  for (int base = 0; base < N; base += 1024) {
+    const int j = base + tid;
+    bool flag = false;
+    if (j < N) {
+      const float lg = j < n_old ? c.ring_logit[(size_t)u * c.w + (p0 + j) % c.w]
+                                 : a.logits[(size_t)(j - n_old) * c.Hkv + kvh];
+      flag = lg >= a.tau_logit;  // Eq. 2 on the float32 logit
+    }
+    const unsigned ballot = __ballot_sync(0xffffffffu, flag);
+    const int before = __popc(ballot & ((1u << lane) - 1u));
+    if (lane == 31) s_warp[warp] = __popc(ballot);
+    __syncthreads();
+    if (warp == 0) {
+      int v = s_warp[lane], incl = v;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int x = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += x;
+      }
+      s_warp[lane] = incl - v;
+      if (lane == 31) s_pages_base = incl;  // tile total (reusing the slot)
+    }
+    __syncthreads();
+    if (j < N) E[j] = s_carry + s_warp[warp] + before;
+    __syncthreads();
+    if (tid == 0) s_carry += s_pages_base;
+    __syncthreads();
+  }
+  if (tid == 0) E[N] = s_carry;
+  __syncthreads();
+  // pairs leaving the window in this call: staging index j < N - w
+  const int n_leave = max(N - c.w, 0);
+  const int n_commit = E[n_leave];  // written by this block above
+  const int len1 = len0 + n_commit;
+  const int pages0 = (len0 + kP - 1) / kP, pages1 = (len1 + kP - 1) / kP;
+  const int n_new = pages1 - pages0;
+  if (tid == 0) {
+    int fail = 0;
+    if (pages1 > c.max_pages) {
+      fail = SPKV_E_CONTEXT_OVERFLOW;
+    } else if (n_new > 0) {
+      const int top = atomicSub(&c.status[1], n_new);
+      if (top < n_new) {
+        atomicAdd(&c.status[1], n_new);
+        fail = SPKV_E_POOL_EXHAUSTED;
+      } else {
+        s_pages_base = top;
+      }
+    }
+    if (fail) set_status(c, fail);
+    s_fail = fail;
+    hdr[H_T0] = t0; hdr[H_LEN0] = len0; hdr[H_NOLD] = n_old; hdr[H_N] = N;
+    hdr[H_NCOMMIT] = fail ? 0 : n_commit;
+    hdr[H_LEN1] = fail ? len0 : len1;
+    hdr[H_FAIL] = fail;
+  }
+  __syncthreads();
+  if (s_fail || n_new == 0) return;
+  for (int i = tid; i < n_new; i += blockDim.x)
+    c.table[(size_t)u * c.max_pages + pages0 + i] = c.free_stack[s_pages_base - 1 - i];
+  __syncthreads();
+  // rows past the final length of a freshly popped last page must read as zeros
+  if (len1 % kP) {
+    const int last = c.table[(size_t)u * c.max_pages + pages1 - 1];
+    uint4 *vb = reinterpret_cast<uint4 *>(c.pages + (int64_t)last * kPageElems + kBlockElems);
+    for (int i = tid; i < kBlockElems * 2 / 16; i += blockDim.x) vb[i] = make_uint4(0, 0, 0, 0);
+  }
 }
 
-extern "C" int spkv_prefill(spkv_cache_t *, int32_t, int32_t, int32_t, const void *, const void *,
-                            const void *, const float *, void *, float, void *, size_t,
-                            spkv_stream_t) {
-  return SPKV_E_UNSUPPORTED;
+// Source row of staging pair j: old ring slot (swizzled page) or chunk input (linear).
+struct SrcRow {
+  const __nv_bfloat16 *k, *v;
+  int row;  // >= 0: swizzled with this row; -1: linear
+};
+__device__ inline SrcRow staging_row(const PrefillArgs &a, int u, int kvh, int t0, int n_old, int j) {
+  SrcRow r;
+  if (j < n_old) {
+    const int slot = (t0 - n_old + j) % a.c.w;
+    const __nv_bfloat16 *pg = a.c.pages + ring_page(a.c, u, slot / kP) * kPageElems;
+    r.row = slot % kP;
+    r.k = pg + r.row * kD;
+    r.v = pg + kBlockElems + r.row * kD;
+  } else {
+    const size_t off = ((size_t)(j - n_old) * a.c.Hkv + kvh) * kD;
+    r.row = -1;
+    r.k = a.k + off;
+    r.v = a.v + off;
+  }
+  return r;
+}
+__device__ inline uint4 load_chunk(const __nv_bfloat16 *rowbase, int row, int chunk) {
+  const int cc = row >= 0 ? (chunk ^ (row & 7)) : chunk;
+  return *reinterpret_cast<const uint4 *>(rowbase + cc * 8);
+}
+
+// ------------------------------------------------------------------ B: scatter (compact)
+// grid (ceil(n_leave_max / 64), Hkv); each warp moves 8 consecutive staging pairs.
+__global__ void __launch_bounds__(256) prefill_scatter_kernel(PrefillArgs a) {
+  const CacheView &c = a.c;
+  const int kvh = blockIdx.y;
+  const int32_t *hdr = unit_ws(a, kvh);
+  const int32_t *E = hdr + kHdrInts;
+  if (hdr[H_FAIL]) return;
+  const int t0 = hdr[H_T0], len0 = hdr[H_LEN0], n_old = hdr[H_NOLD], N = hdr[H_N];
+  const int n_leave = max(N - c.w, 0);
+  const int u = unit_index(c, a.layer, a.seq, kvh);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int chunk = lane & 15, blk = (lane >> 4) * kBlockElems;
+  const int j0 = (blockIdx.x * 8 + warp) * 8;
+  for (int j = j0; j < min(j0 + 8, n_leave); ++j) {
+    const int e = E[j];
+    if (E[j + 1] == e) continue;  // not flagged
+    const int idx = len0 + e;
+    const int page = c.table[(size_t)u * c.max_pages + idx / kP];
+    const int drow = idx % kP;
+    const SrcRow s = staging_row(a, u, kvh, t0, n_old, j);
+    const uint4 val = load_chunk(lane < 16 ? s.k : s.v, s.row, chunk);
+    *reinterpret_cast<uint4 *>(c.pages + (int64_t)page * kPageElems + blk + swz_off(drow, chunk)) = val;
+    if (lane == 0) c.pos_pool[((int64_t)page - c.n_ring_pages_total) * kP + drow] = t0 - n_old + j;
+  }
+}
+
+// --------------------------------------------------------------------- C: ring update
+// grid (ceil(min(C,w) / 8), Hkv); one warp per pair.
+__global__ void __launch_bounds__(256) prefill_ring_kernel(PrefillArgs a) {
+  const CacheView &c = a.c;
+  const int kvh = blockIdx.y;
+  const int32_t *hdr = unit_ws(a, kvh);
+  const int t0 = hdr[H_T0];
+  const int u = unit_index(c, a.layer, a.seq, kvh);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int first = max(a.C - c.w, 0);
+  const int i = first + blockIdx.x * 8 + warp;
+  if (i < a.C) {
+    const int slot = (t0 + i) % c.w, row = slot % kP;
+    __nv_bfloat16 *pg = c.pages + ring_page(c, u, slot / kP) * kPageElems;
+    const int chunk = lane & 15, blk = (lane >> 4) * kBlockElems;
+    const size_t off = ((size_t)i * c.Hkv + kvh) * kD;
+    const uint4 val = *reinterpret_cast<const uint4 *>((lane < 16 ? a.k : a.v) + off + chunk * 8);
+    *reinterpret_cast<uint4 *>(pg + blk + swz_off(row, chunk)) = val;
+    if (lane == 0) c.ring_logit[(size_t)u * c.w + slot] = a.logits[(size_t)i * c.Hkv + kvh];
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    c.t[u] = t0 + a.C;
+    c.len[u] = hdr[H_LEN1];
+  }
+}
+
+// ------------------------------------------------------------------ ATT: chunk attention
+// grid (ceil(C/64), Hq); 4 warps x 16 query rows; K/V tiles of 64 keys, double buffered.
+constexpr int kAttnSmem = 2 * kPageBytes;
+
+__global__ void __launch_bounds__(128) prefill_attn_kernel(PrefillArgs a) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  const CacheView &c = a.c;
+  const int hq = blockIdx.y, kvh = hq / c.G;
+  const int i0 = blockIdx.x * 64;
+  const int32_t *hdr = unit_ws(a, kvh);
+  const int32_t *E = hdr + kHdrInts;
+  const int t0 = hdr[H_T0], len0 = hdr[H_LEN0], n_old = hdr[H_NOLD], N = hdr[H_N];
+  const int p0 = t0 - n_old;
+  const int u = unit_index(c, a.layer, a.seq, kvh);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int g = lane >> 2;
+
+  // kept pairs visible to chunk query i: those with position <= t0 + i - w
+  auto nvis = [&](int i) { return len0 + E[min(max(i + n_old - c.w + 1, 0), N)]; };
+  const int i_last = min(i0 + 63, a.C - 1);
+  const int nv_lo = nvis(i0), nv_hi = nvis(i_last);
+  const int n_ptiles = (nv_hi + kP - 1) / kP;
+  const int s_lo = max(p0, t0 + i0 - c.w + 1), s_hi = t0 + i_last;  // band positions
+  const int n_btiles = (s_hi - s_lo + 1 + 63) / 64;
+  const int n_tiles = n_ptiles + n_btiles;
+
+  // rows of this thread
+  const int ra = i0 + warp * 16 + g, rb = ra + 8;
+  const int nv_a = ra < a.C ? nvis(ra) : 0, nv_b = rb < a.C ? nvis(rb) : 0;
+  const int ta = t0 + ra, tb = t0 + rb;
+
+  uint32_t qf[8][4];
+  load_q_frags(qf, [&](int r) -> const __nv_bfloat16 * {
+    const int i = i0 + warp * 16 + r;
+    return i < a.C ? a.q + ((size_t)i * c.Hq + hq) * kD : nullptr;
+  }, lane);
+
+  auto load_tile = [&](int tile, int buf) {
+    unsigned char *dst = smem + buf * kPageBytes;
+    if (tile < n_ptiles) {
+      const int page = c.table[(size_t)u * c.max_pages + tile];
+      const unsigned char *src = reinterpret_cast<const unsigned char *>(c.pages + (int64_t)page * kPageElems);
+      for (int x = tid; x < kPageBytes / 16; x += 128) cp_async16(smem_u32(dst + x * 16), src + x * 16);
+    } else {
+      // gather 64 band rows (ring slots or chunk rows) into the swizzled image
+      const int s_base = s_lo + (tile - n_ptiles) * 64;
+      for (int x = tid; x < 64 * 32; x += 128) {
+        const int r = x >> 5, part = x & 31, chunk = part & 15, isv = part >> 4;
+        const int s = s_base + r;
+        const uint32_t d = smem_u32(dst + isv * (kBlockElems * 2)) + blk_off(r, chunk);
+        if (s <= s_hi) {
+          const SrcRow sr = staging_row(a, u, kvh, t0, n_old, s - p0);
+          const __nv_bfloat16 *rowp = isv ? sr.v : sr.k;
+          const int cc = sr.row >= 0 ? (chunk ^ (sr.row & 7)) : chunk;
+          cp_async16(d, rowp + cc * 8);
+        } else {
+          *reinterpret_cast<uint4 *>(dst + isv * (kBlockElems * 2) + blk_off(r, chunk)) = make_uint4(0, 0, 0, 0);
+        }
+      }
+    }
+    cp_async_commit();
+  };
+
+  float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f}, o[16][4];
+#pragma unroll
+  for (int n = 0; n < 16; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
+
+  load_tile(0, 0);
+  for (int tile = 0; tile < n_tiles; ++tile) {
+    const int buf = tile & 1;
+    if (tile + 1 < n_tiles) {
+      load_tile(tile + 1, buf ^ 1);
+      cp_async_wait<1>();
+    } else {
+      cp_async_wait<0>();
+    }
+    __syncthreads();
+    const uint32_t sK = smem_u32(smem + buf * kPageBytes), sV = sK + kBlockElems * 2;
+    float s[8][4];
+    qk_tile<64>(s, qf, sK, 0, lane);
+    if (tile < n_ptiles) {
+      const int base = tile * kP;
+      if (base + kP <= nv_lo) {
+        softmax_pv_tile<64>(s, [](int, int) { return true; }, a.scale_log2, m, l, o, sV, 0, lane);
+      } else {
+        softmax_pv_tile<64>(s, [&](int h, int col) { return base + col < (h ? nv_b : nv_a); },
+                            a.scale_log2, m, l, o, sV, 0, lane);
+      }
+    } else {
+      const int s_base = s_lo + (tile - n_ptiles) * 64;
+      softmax_pv_tile<64>(s, [&](int h, int col) {
+        const int sp = s_base + col, tq = h ? tb : ta;
+        return sp <= tq && sp > tq - c.w && sp <= s_hi;
+      }, a.scale_log2, m, l, o, sV, 0, lane);
+    }
+    __syncthreads();
+  }
+  // finish: reduce l over the quad, normalise, store bf16
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    l[h] += __shfl_xor_sync(0xffffffffu, l[h], 1);
+    l[h] += __shfl_xor_sync(0xffffffffu, l[h], 2);
+  }
+  const int t4 = lane & 3;
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const int i = h ? rb : ra;
+    if (i >= a.C) continue;
+    const float inv = 1.f / l[h];
+    __nv_bfloat16 *orow = a.out + ((size_t)i * c.Hq + hq) * kD;
+#pragma unroll
+    for (int n = 0; n < 16; ++n)
+      *reinterpret_cast<uint32_t *>(orow + n * 8 + t4 * 2) = pack_bf16(o[n][2 * h] * inv, o[n][2 * h + 1] * inv);
+  }
+}
+
+static size_t prefill_ws_stride_ints(int C, int w) {
+  size_t ints = kHdrInts + (size_t)C + w + 2;
+  return (ints + 63) / 64 * 64;
+}
+
+}  // namespace spkv
+
+using namespace spkv;
+
+extern "C" size_t spkv_prefill_workspace_bytes(const spkv_config_t *cfg, int32_t C) {
+  if (!cfg || C < 0) return 0;
+  return prefill_ws_stride_ints(C, cfg->window) * 4 * (size_t)cfg->n_kv_heads;
+}
+
+extern "C" int spkv_prefill(spkv_cache_t *cache, int32_t layer, int32_t seq, int32_t C,
+                            const void *d_q, const void *d_k, const void *d_v,
+                            const float *d_logits, void *d_out, float sm_scale, void *d_workspace,
+                            size_t workspace_bytes, spkv_stream_t stream) {
+  if (!cache || layer < 0 || layer >= cache->cfg.n_layers || seq < 0 || seq >= cache->cfg.max_seqs || C < 0)
+    return SPKV_E_INVALID;
+  if (C == 0) return SPKV_OK;
+  if (!d_k || !d_v || !d_logits || ((d_q == nullptr) != (d_out == nullptr))) return SPKV_E_INVALID;
+  if (((uintptr_t)d_k | (uintptr_t)d_v | (uintptr_t)d_q | (uintptr_t)d_out) & 15) return SPKV_E_INVALID;
+  const CacheView &v = cache->view;
+  if (!d_workspace || ((uintptr_t)d_workspace & 255) ||
+      workspace_bytes < spkv_prefill_workspace_bytes(&cache->cfg, C))
+    return SPKV_E_WORKSPACE;
+  PrefillArgs a;
+  a.c = v; a.layer = layer; a.seq = seq; a.C = C;
+  a.q = static_cast<const __nv_bfloat16 *>(d_q);
+  a.k = static_cast<const __nv_bfloat16 *>(d_k);
+  a.v = static_cast<const __nv_bfloat16 *>(d_v);
+  a.logits = d_logits;
+  a.out = static_cast<__nv_bfloat16 *>(d_out);
+  a.tau_logit = cache->tau_logit;
+  a.scale_log2 = sm_scale * 1.4426950408889634f;
+  a.ws = static_cast<int32_t *>(d_workspace);
+  a.ws_stride = (int)prefill_ws_stride_ints(C, v.w);
+  cudaStream_t s = as_stream(stream);
+
+  prefill_plan_kernel<<<v.Hkv, 1024, 0, s>>>(a);
+  // at most max(min(t0,w) + C - w, 0) <= C pairs leave the window
+  prefill_scatter_kernel<<<dim3((C + 63) / 64, v.Hkv), 256, 0, s>>>(a);
+  if (d_q) {
+    if (cudaFuncSetAttribute(prefill_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             kAttnSmem) != cudaSuccess)
+      return SPKV_E_CUDA;
+    prefill_attn_kernel<<<dim3((C + 63) / 64, v.Hq), 128, kAttnSmem, s>>>(a);
+  }
+  const int n_ring = C < v.w ? C : v.w;
+  prefill_ring_kernel<<<dim3((n_ring + 7) / 8, v.Hkv), 256, 0, s>>>(a);
+  return check_stream_error(cudaGetLastError());
 }
