@@ -1,0 +1,430 @@
+#!/usr/bin/env python
+"""SP-KV decode benchmark (one JSON line).
+
+A step = one decode token for every sequence of the batch through the whole layer stack:
+per layer  spkv_score -> spkv_append_evict -> spkv_decode_attention  (the library is the
+attention path only; there are no projections or MLPs).  Inputs are synthetic and seeded,
+shaped like the paper's decode workloads (see paper_2605_14037_b200/synth.py); the cache is
+brought to the configured context length with spkv_prefill before timing.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 2] [--impl reference]
+
+value        whole-job decode tokens/s, inputs resident in HBM, one CUDA-graph replay per step
+e2e          the same through spkv_decode_step_host with pinned HOST buffers (H2D + D2H timed)
+roofline     decode-attention kernel: algorithmic bytes (kept + window K/V, Q, O) per launch
+             over its CUDA-event duration, against the measured HBM copy bandwidth
+dense        same library, tau = -inf (every pair kept): the full-cache decode baseline
+cpu_baseline the CPU oracle timed on a bounded sample of the same workload
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+CONFIGS = {
+    # name: layers, batch, q heads, kv heads, context, beta(a, b) of per-head keep rates
+    1: dict(name="config1_1layer_b1_ctx4k", L=1, B=1, Hq=8, Hkv=2, T=4096, beta=None, rate=0.2),
+    2: dict(name="config2_llama8b_b16_ctx32k", L=32, B=16, Hq=32, Hkv=8, T=32768, beta=(0.5, 2.0)),
+    3: dict(name="config3_llama8b_b4_ctx128k", L=32, B=4, Hq=32, Hkv=8, T=131072, beta=(0.3, 3.0)),
+    5: dict(name="config5_llama70b_b8_ctx64k", L=80, B=8, Hq=64, Hkv=8, T=65536, beta=(0.5, 2.5)),
+}
+W, D_IN, TAU, CHUNK = 128, 512, 0.5, 8192
+
+
+def peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while a region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc = index, None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+        return self
+
+    def __exit__(self, *exc):
+        self.result = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if not self.proc:
+            return
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            return
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if sm:
+            sm.sort()
+            self.result = {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(mx), "reasons": sorted(reasons)}
+
+
+def build_workload(spkv, synth, torch, cfg, dev, dense, total_steps, seed=0):
+    """Creates the cache, per-layer predictors and brings every sequence to context T."""
+    import numpy as np
+    L, B, Hq, Hkv, T = cfg["L"], cfg["B"], cfg["Hq"], cfg["Hkv"], cfg["T"]
+    rng = np.random.default_rng(seed)
+    tau = -math.inf if dense else TAU
+    if cfg["beta"] is None:
+        rates = np.full((L, Hkv), cfg["rate"])
+    else:
+        rates = synth.keep_rates(rng, L, Hkv, *cfg["beta"])
+    eff = np.ones_like(rates) if dense else rates
+    t_final = T + total_steps
+    pages_per_unit = np.ceil(eff * (t_final - W) * 1.03 / 64).astype(np.int64) + 2
+    pool_pages = int(pages_per_unit.sum() * B)
+    cache = spkv.Cache(n_layers=L, max_seqs=B, n_q_heads=Hq, n_kv_heads=Hkv,
+                       max_context=t_final + 64, pool_pages=pool_pages, window=W, tau=tau, device=dev)
+    tl = 0.0  # logit-space threshold of tau = 0.5 (the dense run ignores it)
+    preds, keep = [], []
+    for l in range(L):
+        Wl = synth.linear_predictor(rng, Hkv, D_IN)
+        bl = synth.bias_for_keep_rate(Wl, rates[l], tl)
+        Wd, bd = spkv.bf16_from_bits(Wl, dev), torch.from_numpy(bl).to(dev)
+        preds.append(spkv.make_predictor(Wd, bd))
+        keep.append((Wd, bd))
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(seed)
+    # state build: device-generated chunks through score + prefill (state only, no attention)
+    kv_pool = [torch.randn((CHUNK, Hkv, 128), generator=gen, device=dev, dtype=torch.float32)
+               .to(torch.bfloat16) for _ in range(4)]
+    for l in range(L):
+        for b in range(B):
+            done = 0
+            while done < T:
+                c = min(CHUNK, T - done)
+                x = torch.randn((c, D_IN), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+                lg = cache.spkv_score(preds[l], x)
+                k, v = kv_pool[(l + b + done // CHUNK) % 4][:c], kv_pool[(l + b + 1 + done // CHUNK) % 4][:c]
+                cache.spkv_prefill(l, b, k, v, lg)
+                done += c
+    cache.check()
+    return cache, preds, rates, gen
+
+
+def run_ours(args):
+    import numpy as np
+    import torch
+
+    from paper_2605_14037_b200 import build as spkv_build
+    spkv_build.build()
+    from paper_2605_14037_b200 import spkv, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dev = torch.device(f"cuda:{local}")
+    torch.cuda.set_device(dev)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    cfg = CONFIGS[args.config]
+    L, B, Hq, Hkv = cfg["L"], cfg["B"], cfg["Hq"], cfg["Hkv"]
+    K, Wm = args.steps, args.warmup
+    e2e_steps = min(K, args.e2e_steps)
+    roof_steps = min(K, 8)
+    total_steps = Wm + K + e2e_steps + 3 + roof_steps + 3
+    hbm_peak, peak_kind = peaks()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x):
+        if dist is None:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def measure(dense):
+        cache, preds, rates, gen = build_workload(spkv, synth, torch, cfg, dev, dense, total_steps)
+        ids = torch.arange(B, dtype=torch.int32, device=dev)
+        n_in = 4  # distinct q/k/v input sets cycled over the steps
+        q_in = torch.randn((n_in, L, B, Hq, 128), generator=gen, device=dev).to(torch.bfloat16)
+        k_in = torch.randn((n_in, L, B, Hkv, 128), generator=gen, device=dev).to(torch.bfloat16)
+        v_in = torch.randn((n_in, L, B, Hkv, 128), generator=gen, device=dev).to(torch.bfloat16)
+        x_all = torch.randn((total_steps, L, B, D_IN), generator=gen, device=dev).to(torch.bfloat16)
+        xs, qs, ks, vs = (torch.empty_like(t[0]) for t in (x_all, q_in, k_in, v_in))
+        out = torch.empty((L, B, Hq, 128), dtype=torch.bfloat16, device=dev)
+        logits = torch.empty((L, B, Hkv), dtype=torch.float32, device=dev)
+        cache.decode_workspace(B)
+        step_no = [0]
+
+        def stage_inputs():
+            s = step_no[0]
+            xs.copy_(x_all[s]); qs.copy_(q_in[s % n_in]); ks.copy_(k_in[s % n_in]); vs.copy_(v_in[s % n_in])
+            step_no[0] += 1
+
+        def layer_calls(stream=None, events=None):
+            for l in range(L):
+                cache.spkv_score(preds[l], xs[l], logits=logits[l], stream=stream)
+                cache.spkv_append_evict(l, ids, ks[l], vs[l], logits[l], stream=stream)
+                if events is not None:
+                    events[l][0].record()
+                cache.spkv_decode_attention(l, ids, qs[l], out=out[l], stream=stream)
+                if events is not None:
+                    events[l][1].record()
+
+        graph = None
+        if not args.no_graph:
+            side = torch.cuda.Stream(device=dev)
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                stage_inputs(); layer_calls()          # warm the lazily loaded kernels
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                layer_calls()
+
+        def step():
+            stage_inputs()
+            if graph is not None:
+                graph.replay()
+            else:
+                layer_calls()
+
+        for _ in range(Wm):
+            step()
+        cache.check()
+        st0 = cache.spkv_cache_stats()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with ClockSampler(local) as clk:
+            e0.record()
+            for _ in range(K):
+                step()
+            e1.record()
+            torch.cuda.synchronize()
+        barrier()
+        ms = max_over_ranks(e0.elapsed_time(e1))
+        cache.check()
+        st1 = cache.spkv_cache_stats()
+
+        # decode-kernel duration, measured with events around every launch (no graph)
+        evs = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                for _ in range(L)] for _ in range(roof_steps)]
+        for _ in range(3):
+            stage_inputs(); layer_calls()
+        torch.cuda.synchronize()
+        for s in range(roof_steps):
+            stage_inputs(); layer_calls(events=evs[s])
+        torch.cuda.synchronize()
+        dec_ms = [a.elapsed_time(b) for row in evs for (a, b) in row]
+        st2 = cache.spkv_cache_stats()
+        kv_bytes = 0.5 * (st1.bytes_resident + st2.bytes_resident)     # all layers, one step
+        qo_bytes = L * B * Hq * 128 * 2 * 2
+        launch_bytes = (kv_bytes + qo_bytes) / L
+        launch_s = (sum(dec_ms) / len(dec_ms)) * 1e-3
+
+        res = dict(ms_per_step=ms / K, tokens_per_s=world * B * K / (ms * 1e-3),
+                   kv_gb_per_step=0.5 * (st0.bytes_resident + st1.bytes_resident) / 1e9,
+                   density=st1.density_cache, launch_bytes=launch_bytes, launch_s=launch_s,
+                   clocks=clk.result, graph=graph is not None)
+
+        # end to end through the host-buffer entry point
+        if not dense and e2e_steps > 0:
+            pin = lambda t: t.cpu().pin_memory()
+            hx, hq, hk, hv = pin(x_all[:4]), pin(q_in), pin(k_in), pin(v_in)
+            hout = torch.empty((L, B, Hq, 128), dtype=torch.bfloat16).pin_memory()
+
+            def e2e_step(s):
+                for l in range(L):
+                    cache.spkv_decode_step_host(l, preds[l], ids, hx[s % 4, l], hq[s % n_in, l],
+                                                hk[s % n_in, l], hv[s % n_in, l], hout[l])
+                torch.cuda.current_stream().synchronize()   # the step's result is read on the host
+                return float(hout[L - 1, 0, 0, 0])
+
+            for s in range(3):
+                e2e_step(s)
+            barrier()
+            t0 = time.perf_counter()
+            for s in range(e2e_steps):
+                e2e_step(s)
+            torch.cuda.synchronize()
+            dt = max_over_ranks(time.perf_counter() - t0)
+            cache.check()
+            res["e2e"] = {
+                "value": world * B * e2e_steps / dt, "unit": "tokens/s",
+                "h2d_bytes_per_step": L * B * (D_IN + Hq * 128 + 2 * Hkv * 128) * 2,
+                "d2h_bytes_per_step": L * B * Hq * 128 * 2, "steps": e2e_steps,
+                "api": "spkv_decode_step_host"}
+        cache.close()
+        del cache
+        torch.cuda.empty_cache()
+        return res
+
+    sp = measure(dense=False)
+    dn = measure(dense=True) if args.dense else None
+
+    if rank != 0:
+        return
+    achieved = sp["launch_bytes"] / sp["launch_s"] / 1e9
+    line = {
+        "metric": "SP-KV decode tokens/s at 32K ctx; achieved HBM GB/s vs peak (surviving bytes)",
+        "value": sp["tokens_per_s"], "unit": "tokens/s", "n_gpus": world, "steps": K, "warmup": Wm,
+        "ms_per_step": sp["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": cfg["name"], "layers": L, "batch": B, "q_heads": Hq, "kv_heads": Hkv,
+                   "head_dim": 128, "context": cfg["T"], "window": W, "tau": TAU,
+                   "keep_rates": ("beta%s" % (cfg["beta"],) if cfg["beta"] else cfg["rate"]),
+                   "density": sp["density"], "kv_gb_per_step": sp["kv_gb_per_step"],
+                   "l2": "inputs larger than L2 (K/V read per step >> 126 MB)" if sp["kv_gb_per_step"] > 0.5
+                         else "working set smaller than L2: latency-bound case",
+                   "cuda_graph": sp["graph"], "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "clocks": sp["clocks"],
+        "gpu_launches": 3 * L * K,
+        "roofline": {"bound": "hbm", "kernel": "decode_tc_kernel", "achieved": achieved, "peak": hbm_peak,
+                     "unit": "GB/s", "frac": achieved / hbm_peak, "peak_kind": f"of {peak_kind}",
+                     "frac_of_nominal_8TBs": achieved / 8000.0,
+                     "bytes_per_launch": sp["launch_bytes"], "launch_us": sp["launch_s"] * 1e6,
+                     "traffic": load_traffic(cfg["name"], sp["launch_bytes"])},
+        "e2e": sp.get("e2e"),
+    }
+    if dn is not None:
+        dn_ach = dn["launch_bytes"] / dn["launch_s"] / 1e9
+        line["dense"] = {"tokens_per_s": dn["tokens_per_s"], "ms_per_step": dn["ms_per_step"],
+                         "kv_gb_per_step": dn["kv_gb_per_step"], "achieved_gbs": dn_ach,
+                         "frac": dn_ach / hbm_peak,
+                         "speedup_spkv_over_dense": sp["tokens_per_s"] / dn["tokens_per_s"],
+                         "cache_reduction": dn["kv_gb_per_step"] / sp["kv_gb_per_step"]}
+    if world == 1 and not args.no_cpu:
+        line["cpu_baseline"] = cpu_baseline(cfg, budget_s=args.cpu_seconds)
+    print(json.dumps(line))
+
+
+def load_traffic(workload, launch_bytes):
+    """DRAM bytes per decode launch from the committed ncu summary, if there is one."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "decode_traffic.json")) as f:
+            t = json.load(f)
+        # measured on a smaller case; traffic grows in proportion to the algorithmic bytes
+        return t["dram_bytes_per_launch"] / t["algorithmic_bytes_per_launch"] * launch_bytes
+    except Exception:
+        return None
+
+
+def cpu_baseline(cfg, budget_s=20.0, steps=None):
+    """The oracle, as it stands, on a bounded sample: the units of `n_seq` sequences of one
+    layer at the configured context, a few decode steps; scaled to whole-job tokens/s."""
+    import numpy as np
+
+    import oracle
+    from paper_2605_14037_b200 import synth
+    rng = np.random.default_rng(1)
+    Hq, Hkv, T, B, L = cfg["Hq"], cfg["Hkv"], cfg["T"], cfg["B"], cfg["L"]
+    G = Hq // Hkv
+    n_seq = 2 if B >= 2 else 1
+    rates = (np.full(Hkv, cfg["rate"]) if cfg["beta"] is None
+             else synth.keep_rates(np.random.default_rng(0), L, Hkv, *cfg["beta"])[0])
+    units = [oracle.Unit(W, 128) for _ in range(n_seq * Hkv)]
+    Tb = min(T, 32768)        # state built with min(T, 32768) pairs per unit to bound the set-up
+    for i, u in enumerate(units):
+        k, v = synth.normal_bf16(rng, (Tb, 128)), synth.normal_bf16(rng, (Tb, 128))
+        lg = synth.logits_with_keep_rate(rng, (Tb,), float(rates[i % Hkv]) * T / Tb if Tb < T else float(rates[i % Hkv]), 0.0)
+        u.prefill(k, v, lg, 0.0)
+    n = len(units)
+    scale = 1.0 / math.sqrt(128)
+    t_used, done = 0.0, 0
+    while (steps is None and t_used < budget_s and done < 64) or (steps is not None and done < steps):
+        k, v = synth.normal_bf16(rng, (n, 128)), synth.normal_bf16(rng, (n, 128))
+        q = synth.normal_bf16(rng, (n, G, 128))
+        lg = rng.standard_normal(n).astype(np.float32)
+        t0 = time.perf_counter()
+        oracle.step_batch(units, k, v, lg, 0.0, q, scale)
+        t_used += time.perf_counter() - t0
+        done += 1
+    per_step_full = (t_used / done) * (L * B * Hkv / n)
+    return {"value": B / per_step_full, "unit": "tokens/s", "cores": oracle.threads(), "kind": "oracle",
+            "sample": f"{n} units ({n_seq} sequences x {Hkv} KV heads of one layer, context {T}), "
+                      f"{done} decode steps (append + attend), scaled by units to {L} layers x batch {B}",
+            "seconds": t_used}
+
+
+def run_reference(args):
+    """Reference arm = the CPU oracle on a bounded sample per step (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    cfg = CONFIGS[args.config]
+    steps = max(1, min(args.steps, 16))
+    cb = cpu_baseline(cfg, steps=steps + min(args.warmup, 2))
+    L, B = cfg["L"], cfg["B"]
+    line = {
+        "impl": "reference",
+        "metric": "SP-KV decode tokens/s at 32K ctx; achieved HBM GB/s vs peak (surviving bytes)",
+        "value": cb["value"], "unit": "tokens/s", "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": steps, "warmup": min(args.warmup, 2), "ms_per_step": 1e3 * B / cb["value"],
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": cfg["name"], "layers": L, "batch": B, "context": cfg["T"], "window": W,
+                   "tau": TAU},
+        "cpu_baseline": {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")},
+        "e2e": {"value": cb["value"], "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=256)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2, choices=sorted(CONFIGS))
+    ap.add_argument("--no-graph", action="store_true", help="launch every kernel from the host")
+    ap.add_argument("--no-dense", dest="dense", action="store_false", help="skip the dense baseline")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
+    ap.add_argument("--e2e-steps", type=int, default=32)
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -15,7 +15,10 @@
 // because consecutive segments differ in block or item -- and bumps the unit's arrival
 // counter; the block that arrives last merges all slots of the unit by their
 // log-sum-exp weights and resets the counter.  Nobody ever waits.
+#include <stdlib.h>
+
 #include "spkv_internal.cuh"
+#include "spkv_mma.cuh"
 
 namespace spkv {
 
@@ -295,6 +298,279 @@ __global__ void __launch_bounds__(128) decode_simt_kernel(DecodeArgs a) {
   }
 }
 
+
+// ------------------------------------------------------------------------------------
+// Main kernel: one persistent block per SM, a pipeline of whole pages.
+//
+//   warp 4, lane 0 (producer): for every page of the block's range, one 32 KB linear bulk
+//       copy HBM -> shared memory (cp.async.bulk, completion counted on an mbarrier).
+//       The page in HBM already is the swizzled shared-memory image, so nothing is
+//       rearranged on the way.  n_stages pages (5-6, i.e. 160-192 KB per SM) are in flight.
+//   warps 0-3 (consumers): each takes 16 of the page's 64 pairs.  The group's G query
+//       heads form the rows of a 16-row tile (padded), so S = Q K^T and O += P V are small
+//       dense products done with mma.sync m16n8k16 (bf16 in, fp32 accumulate), operands
+//       read with ldmatrix; masking, online softmax (exp2, quad shuffles) in registers.
+//       A warp keeps its own (m, l, O) for its quarter of every page of a segment; the
+//       four are merged through shared memory once per segment.
+//
+// Why tensor cores in a bandwidth-bound kernel: per 512 B pair the group needs 2*G*128
+// multiply-adds.  On the CUDA cores (kernel above) that is, with bf16 unpacking and the
+// reductions, several hundred issue slots per pair and SM -- the issue rate, not HBM, then
+// limits the kernel at G >= 4.  As MMA tiles the same arithmetic is 2 x 16 instructions per
+// page and warp, and the kernel is limited by the page stream alone.
+//
+// Every wait is bounded: if a copy never lands the waiting thread records
+// SPKV_E_TIMEOUT, raises the block's abort flag, and all threads run to the end without
+// waiting again (control flow stays uniform, outputs are then meaningless).
+// ------------------------------------------------------------------------------------
+constexpr int kListCap = 512;
+constexpr int kTcThreads = 160;
+
+struct TcSmem {  // offsets into dynamic shared memory, computed on host and device alike
+  int n_stages, off_bar, off_np, off_pre, off_tmp, off_list, off_meta, off_red, off_flags, total;
+};
+__host__ __device__ inline TcSmem tc_smem_layout(int n_items, int GP, int n_stages) {
+  TcSmem L;
+  L.n_stages = n_stages;
+  int o = n_stages * kPageBytes;
+  L.off_bar = o;   o += 2 * 8 * 8;  // up to 8 stages: full[8], empty[8]
+  L.off_np = o;    o += n_items * 4;
+  L.off_pre = o;   o += (n_items + 1) * 4;
+  L.off_tmp = o;   o += 64 * 4;
+  L.off_list = o;  o += kListCap * 4;
+  L.off_meta = o;  o += kListCap * 4;
+  o = (o + 15) / 16 * 16;
+  L.off_red = o;   o += 4 * GP * 132 * 4;
+  L.off_flags = o; o += 16;
+  L.total = o;
+  return L;
+}
+
+__device__ inline void consumer_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+__device__ inline void wait_or_abort(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
+                                     const CacheView &c) {
+  if (*abort_flag) return;
+  if (!mbar_wait_bounded(bar, parity)) {
+    *abort_flag = 1;
+    set_status(c, SPKV_E_TIMEOUT);
+  }
+}
+
+__global__ void __launch_bounds__(kTcThreads, 1) decode_tc_kernel(DecodeArgs a, int GP, int n_stages) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  const CacheView &c = a.c;
+  const int n = a.n_items;
+  const TcSmem L = tc_smem_layout(n, GP, n_stages);
+  uint64_t *full = reinterpret_cast<uint64_t *>(smem + L.off_bar);
+  uint64_t *empty = full + 8;
+  int *s_np = reinterpret_cast<int *>(smem + L.off_np);
+  int *s_pre = reinterpret_cast<int *>(smem + L.off_pre);
+  int *s_tmp = reinterpret_cast<int *>(smem + L.off_tmp);
+  int *s_list = reinterpret_cast<int *>(smem + L.off_list);
+  int *s_meta = reinterpret_cast<int *>(smem + L.off_meta);
+  float *s_red = reinterpret_cast<float *>(smem + L.off_red);
+  volatile int *s_abort = reinterpret_cast<volatile int *>(smem + L.off_flags);
+  volatile int *s_last = s_abort + 1;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  if (tid == 0) {
+    for (int i = 0; i < n_stages; ++i) {
+      mbar_init(&full[i], 1);
+      mbar_init(&empty[i], 4);
+    }
+    mbar_fence_init();
+    *s_abort = 0;
+    *s_last = 0;
+  }
+  for (int i = tid; i < n; i += kTcThreads) {
+    const int b = i / c.Hkv, kvh = i % c.Hkv;
+    const int seq = a.seq_ids[b];
+    int np = 0;
+    if (seq >= 0 && seq < c.S) {
+      const int u = unit_index(c, a.layer, seq, kvh);
+      np = (c.len[u] + kP - 1) / kP + (min(c.t[u], c.w) + kP - 1) / kP;
+    } else if (blockIdx.x == 0) {
+      set_status(c, SPKV_E_BOUNDS);
+    }
+    s_np[i] = np;
+    if (np == 0 && blockIdx.x == 0) {
+      for (int g = 0; g < a.G; ++g) {
+        __nv_bfloat16 *o = a.out + ((size_t)b * c.Hq + kvh * a.G + g) * kD;
+        for (int d = 0; d < kD; ++d) o[d] = __float2bfloat16(0.f);
+        if (a.lse) a.lse[(size_t)b * c.Hq + kvh * a.G + g] = -INFINITY;
+      }
+    }
+  }
+  __syncthreads();
+  block_exclusive_scan(s_np, s_pre, n, s_tmp);
+  const int NP = s_pre[n];
+  if (NP == 0) return;
+  const int nb = min((int)gridDim.x, NP);
+  if ((int)blockIdx.x >= nb) return;
+  const int p_begin = range_start(blockIdx.x, NP, nb);
+  const int p_end = range_start(blockIdx.x + 1, NP, nb);
+
+  // consumer state
+  uint32_t qf[8][4];
+  float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f}, o[16][4];
+  int k_page = 0;  // pages handled so far by this block (same count in producer and consumers)
+
+  for (int round = p_begin; round < p_end; round += kListCap) {
+    const int cnt = min(kListCap, p_end - round);
+    __syncthreads();  // the previous round's list is no longer in use
+    for (int i = tid; i < cnt; i += kTcThreads) {
+      const int pp = round + i;
+      int lo = 0, hi = n;
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (s_pre[mid] <= pp) lo = mid; else hi = mid;
+      }
+      const int item = lo, j = pp - s_pre[item];
+      const int u = unit_index(c, a.layer, a.seq_ids[item / c.Hkv], item % c.Hkv);
+      const int len = c.len[u], nk = (len + kP - 1) / kP;
+      int gpage, valid;
+      if (j < nk) {
+        gpage = c.table[(size_t)u * c.max_pages + j];
+        valid = min(kP, len - j * kP);
+      } else {
+        gpage = (int)ring_page(c, u, j - nk);
+        valid = min(kP, min(c.t[u], c.w) - (j - nk) * kP);
+      }
+      const int seg_begin = (pp == p_begin) || (j == 0);
+      const int seg_end = (pp == p_end - 1) || (j == s_np[item] - 1);
+      s_list[i] = gpage;
+      s_meta[i] = valid | (seg_end << 8) | (seg_begin << 9) | (item << 10);
+    }
+    __syncthreads();
+
+    if (warp == 4) {
+      if (lane == 0) {
+        for (int i = 0; i < cnt; ++i) {
+          const int k = k_page + i, stage = k % n_stages, use = k / n_stages;
+          if (use > 0) wait_or_abort(&empty[stage], (use - 1) & 1, s_abort, c);
+          mbar_arrive_expect_tx(&full[stage], kPageBytes);
+          bulk_load(smem + (size_t)stage * kPageBytes, c.pages + (int64_t)s_list[i] * kPageElems,
+                    kPageBytes, &full[stage]);
+        }
+      }
+    } else {
+      for (int i = 0; i < cnt; ++i) {
+        const int k = k_page + i, stage = k % n_stages, use = k / n_stages;
+        const int meta = s_meta[i];
+        const int valid = meta & 255, item = meta >> 10;
+        const int b = item / c.Hkv, kvh = item % c.Hkv;
+        if (meta & 512) {  // first page of a segment
+          load_q_frags(qf, [&](int r) -> const __nv_bfloat16 * {
+            return r < a.G ? a.q + ((size_t)b * c.Hq + kvh * a.G + r) * kD : nullptr;
+          }, lane);
+          m[0] = m[1] = -INFINITY;
+          l[0] = l[1] = 0.f;
+#pragma unroll
+          for (int x = 0; x < 16; ++x) o[x][0] = o[x][1] = o[x][2] = o[x][3] = 0.f;
+        }
+        wait_or_abort(&full[stage], use & 1, s_abort, c);
+        const int tok0 = warp * 16;
+        if (tok0 < valid) {
+          const uint32_t sK = smem_u32(smem + (size_t)stage * kPageBytes), sV = sK + kBlockElems * 2;
+          float s[2][4];
+          qk_tile<16>(s, qf, sK, tok0, lane);
+          softmax_pv_tile<16>(s, [&](int, int col) { return col < valid; }, a.scale_log2, m, l, o, sV,
+                              tok0, lane);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty[stage]);
+
+        if (meta & 256) {  // last page of the segment: merge the four warps, emit
+          const int g = lane >> 2, t4 = lane & 3;
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            l[h] += __shfl_xor_sync(0xffffffffu, l[h], 1);
+            l[h] += __shfl_xor_sync(0xffffffffu, l[h], 2);
+            const int row = g + 8 * h;
+            if (row < a.G) {
+              float *dst = s_red + ((size_t)warp * GP + row) * 132;
+#pragma unroll
+              for (int x = 0; x < 16; ++x) {
+                dst[x * 8 + t4 * 2] = o[x][2 * h];
+                dst[x * 8 + t4 * 2 + 1] = o[x][2 * h + 1];
+              }
+              if (t4 == 0) { dst[128] = m[h]; dst[129] = l[h]; }
+            }
+          }
+          consumer_bar();
+          const int c_first = block_of_page(s_pre[item], NP, nb);
+          const int c_last = block_of_page(s_pre[item + 1] - 1, NP, nb);
+          const int nseg = c_last - c_first + 1;
+          const int slot = blockIdx.x + item;
+          for (int gh = 0; gh < a.G; ++gh) {
+            float M = -INFINITY;
+#pragma unroll
+            for (int w4 = 0; w4 < 4; ++w4) M = fmaxf(M, s_red[((size_t)w4 * GP + gh) * 132 + 128]);
+            float Ls = 0.f, Os = 0.f;
+#pragma unroll
+            for (int w4 = 0; w4 < 4; ++w4) {
+              const float *src = s_red + ((size_t)w4 * GP + gh) * 132;
+              const float f = src[128] == -INFINITY ? 0.f : exp2f(src[128] - M);
+              Ls += src[129] * f;
+              Os += src[tid] * f;
+            }
+            const size_t row = (size_t)b * c.Hq + kvh * a.G + gh;
+            if (nseg == 1) {
+              a.out[row * kD + tid] = __float2bfloat16(Os / Ls);
+              if (a.lse && tid == 0) a.lse[row] = (M + log2f(Ls)) * kLn2;
+            } else {
+              a.part_acc[((size_t)slot * a.G + gh) * kD + tid] = Os;
+              if (tid == 0) {
+                a.part_ml[((size_t)slot * a.G + gh) * 2 + 0] = M;
+                a.part_ml[((size_t)slot * a.G + gh) * 2 + 1] = Ls;
+              }
+            }
+          }
+          if (nseg > 1) {
+            __threadfence();
+            consumer_bar();
+            if (tid == 0) {
+              const int old = atomicAdd(&a.counters[item], 1);
+              const int last = old == nseg - 1;
+              if (last) a.counters[item] = 0;
+              *s_last = last;
+            }
+            consumer_bar();
+            if (*s_last) {
+              __threadfence();
+              for (int gh = 0; gh < a.G; ++gh) {
+                float Mx = -INFINITY;
+                for (int sidx = c_first; sidx <= c_last; ++sidx)
+                  Mx = fmaxf(Mx, __ldcg(&a.part_ml[((size_t)(sidx + item) * a.G + gh) * 2]));
+                float Ls = 0.f, Os = 0.f;
+                for (int sidx = c_first; sidx <= c_last; ++sidx) {
+                  const size_t base = (size_t)(sidx + item) * a.G + gh;
+                  const float f = exp2f(__ldcg(&a.part_ml[base * 2]) - Mx);
+                  Ls += __ldcg(&a.part_ml[base * 2 + 1]) * f;
+                  Os += __ldcg(&a.part_acc[base * kD + tid]) * f;
+                }
+                const size_t row = (size_t)b * c.Hq + kvh * a.G + gh;
+                a.out[row * kD + tid] = __float2bfloat16(Os / Ls);
+                if (a.lse && tid == 0) a.lse[row] = (Mx + log2f(Ls)) * kLn2;
+              }
+            }
+          }
+          consumer_bar();  // s_red and s_last are free again
+        }
+      }
+    }
+    k_page += cnt;
+  }
+  // after an abort, do not leave while copies may still be landing in shared memory
+  __syncthreads();
+  if (*s_abort && tid == 0) {
+    const int first = max(0, k_page - n_stages);
+    for (int k = first; k < k_page; ++k) mbar_wait_bounded(&full[k % n_stages], (k / n_stages) & 1);
+  }
+}
+
 template <int GP>
 static int launch_simt(const DecodeArgs &a, int grid, size_t smem, cudaStream_t s) {
   if (smem > 48 * 1024 &&
@@ -353,10 +629,25 @@ extern "C" int spkv_decode_attention(spkv_cache_t *cache, int32_t layer, const i
 
   int GP = 1;
   while (GP < v.G) GP <<= 1;
+  cudaStream_t s = as_stream(stream);
+  static const bool use_simt = [] {
+    const char *e = getenv("SPKV_DECODE_KERNEL");  // "simt": the CUDA-core comparison kernel
+    return e && e[0] == 's';
+  }();
+  if (!use_simt) {
+    if (n_items > 1024) return SPKV_E_UNSUPPORTED;
+    int n_stages = 6;
+    TcSmem L = tc_smem_layout(n_items, GP, n_stages);
+    while (L.total > 227 * 1024 && n_stages > 2) L = tc_smem_layout(n_items, GP, --n_stages);
+    if (cudaFuncSetAttribute(decode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total) !=
+        cudaSuccess)
+      return SPKV_E_CUDA;
+    decode_tc_kernel<<<min(kMaxGrid, cache->sm_count), kTcThreads, L.total, s>>>(a, GP, n_stages);
+    return check_stream_error(cudaGetLastError());
+  }
   const int grid = min(kMaxGrid, cache->sm_count * 4);
   const size_t smem = (size_t)(n_items + n_items + 1 + 64) * 4 + (size_t)n_items * sizeof(ItemInfo) +
                       (size_t)4 * GP * 130 * 4;
-  cudaStream_t s = as_stream(stream);
   switch (GP) {
     case 1: return launch_simt<1>(a, grid, smem, s);
     case 2: return launch_simt<2>(a, grid, smem, s);
