@@ -2,7 +2,7 @@
 """SP-KV decode benchmark (one JSON line).
 
 A step = one decode token for every sequence of the batch through the whole layer stack:
-per layer  spkv_score -> spkv_append_evict -> spkv_decode_attention  (the library is the
+per layer  spkv_score_append_evict (score + append/evict fused) -> spkv_decode_attention  (the library is the
 attention path only; there are no projections or MLPs).  Inputs are synthetic and seeded,
 shaped like the paper's decode workloads (see paper_2605_14037_b200/synth.py); the cache is
 brought to the configured context length with spkv_prefill before timing.
@@ -157,7 +157,10 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
-    cfg = CONFIGS[args.config]
+    cfg = dict(CONFIGS[args.config])
+    if args.layers > 0:
+        cfg["L"] = args.layers
+        cfg["name"] += f"_{args.layers}layers_only"
     L, B, Hq, Hkv = cfg["L"], cfg["B"], cfg["Hq"], cfg["Hkv"]
     K, Wm = args.steps, args.warmup
     e2e_steps = min(K, args.e2e_steps)
@@ -198,8 +201,8 @@ def run_ours(args):
 
         def layer_calls(stream=None, events=None):
             for l in range(L):
-                cache.spkv_score(preds[l], xs[l], logits=logits[l], stream=stream)
-                cache.spkv_append_evict(l, ids, ks[l], vs[l], logits[l], stream=stream)
+                cache.spkv_score_append_evict(l, preds[l], ids, xs[l], ks[l], vs[l],
+                                              logits_out=logits[l], stream=stream)
                 if events is not None:
                     events[l][0].record()
                 cache.spkv_decode_attention(l, ids, qs[l], out=out[l], stream=stream)
@@ -314,7 +317,7 @@ def run_ours(args):
                          else "working set smaller than L2: latency-bound case",
                    "cuda_graph": sp["graph"], "parallelism": "replicas only" if world > 1 else "single GPU"},
         "clocks": sp["clocks"],
-        "gpu_launches": 3 * L * K,
+        "gpu_launches": 2 * L * K,
         "roofline": {"bound": "hbm", "kernel": "decode_tc_kernel", "achieved": achieved, "peak": hbm_peak,
                      "unit": "GB/s", "frac": achieved / hbm_peak, "peak_kind": f"of {peak_kind}",
                      "frac_of_nominal_8TBs": achieved / 8000.0,
@@ -416,6 +419,8 @@ def main():
     ap.add_argument("--no-dense", dest="dense", action="store_false", help="skip the dense baseline")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
     ap.add_argument("--e2e-steps", type=int, default=32)
+    ap.add_argument("--layers", type=int, default=0,
+                    help="override the layer count (small profiling captures only; not a bench line)")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":

@@ -147,6 +147,14 @@ int spkv_append_evict(spkv_cache_t *cache, int32_t layer, const int32_t *d_seq_i
                       const void *d_k, const void *d_v, const float *d_logits,
                       spkv_stream_t stream);
 
+/* Steps 1 + 2 in one launch: scores the B new tokens with `pred` (Eq. 1; same float32
+ * logits as spkv_score, bit for bit) and appends them as spkv_append_evict does.
+ *   d_x [B, d_in] bf16; d_logits_out [B, n_kv_heads] float32, optional for the linear
+ *   predictor (may be NULL), required for the two-layer one (scored by its own kernel). */
+int spkv_score_append_evict(spkv_cache_t *cache, int32_t layer, const spkv_predictor_t *pred,
+                            const int32_t *d_seq_ids, int32_t B, const void *d_x, const void *d_k,
+                            const void *d_v, float *d_logits_out, spkv_stream_t stream);
+
 /* Workspace bytes spkv_decode_attention needs for a batch of B sequences. */
 size_t spkv_decode_workspace_bytes(const spkv_config_t *cfg, int32_t B);
 

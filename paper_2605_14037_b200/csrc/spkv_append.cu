@@ -34,7 +34,9 @@ __device__ inline int alloc_page(const CacheView &c, int lane) {
 __global__ void __launch_bounds__(128)
 append_evict_kernel(CacheView c, int layer, const int32_t *__restrict__ seq_ids, int B,
                     const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new,
-                    const float *__restrict__ logits, float tau_logit) {
+                    const float *__restrict__ logits, float tau_logit,
+                    const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__restrict__ W,
+                    const float *__restrict__ bias, int d_in, float *__restrict__ logits_out) {
   const int lane = threadIdx.x & 31;
   const int item = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (item >= B * c.Hkv) return;
@@ -45,6 +47,14 @@ append_evict_kernel(CacheView c, int layer, const int32_t *__restrict__ seq_ids,
     return;
   }
   const int u = unit_index(c, layer, seq, kvh);
+  // fused scoring (Eq. 1, linear predictor): this unit's logit for the new pair
+  float new_logit;
+  if (x) {
+    new_logit = warp_dot_bf16(x + (size_t)b * d_in, W + (size_t)kvh * d_in, d_in, lane) + bias[kvh];
+    if (logits_out && lane == 0) logits_out[item] = new_logit;
+  } else {
+    new_logit = logits[item];
+  }
   const int t = c.t[u];
   const int slot = t % c.w;
   const int row = slot % kP;
@@ -86,7 +96,7 @@ append_evict_kernel(CacheView c, int layer, const int32_t *__restrict__ seq_ids,
   const uint4 *src = (lane < 16 ? k_new : v_new) + (size_t)item * 16 + chunk;
   *ring_cell = *src;
   if (lane == 0) {
-    c.ring_logit[(size_t)u * c.w + slot] = logits[item];
+    c.ring_logit[(size_t)u * c.w + slot] = new_logit;
     c.t[u] = t + 1;
   }
 }
@@ -106,6 +116,33 @@ extern "C" int spkv_append_evict(spkv_cache_t *cache, int32_t layer, const int32
   const int items = B * cache->view.Hkv;
   append_evict_kernel<<<(items + 3) / 4, 128, 0, as_stream(stream)>>>(
       cache->view, layer, d_seq_ids, B, static_cast<const uint4 *>(d_k),
-      static_cast<const uint4 *>(d_v), d_logits, cache->tau_logit);
+      static_cast<const uint4 *>(d_v), d_logits, cache->tau_logit, nullptr, nullptr, nullptr, 0, nullptr);
+  return check_stream_error(cudaGetLastError());
+}
+
+extern "C" int spkv_score_append_evict(spkv_cache_t *cache, int32_t layer, const spkv_predictor_t *pred,
+                                       const int32_t *d_seq_ids, int32_t B, const void *d_x,
+                                       const void *d_k, const void *d_v, float *d_logits_out,
+                                       spkv_stream_t stream) {
+  if (!cache || !pred || layer < 0 || layer >= cache->cfg.n_layers || B < 0 || B > cache->cfg.max_seqs)
+    return SPKV_E_INVALID;
+  if (B == 0) return SPKV_OK;
+  if (!d_seq_ids || !d_x || !d_k || !d_v) return SPKV_E_INVALID;
+  if (pred->kind != 0) {
+    // two-layer predictor: the hidden layer is shared by the KV heads, so it is scored by
+    // its own kernel first
+    if (!d_logits_out) return SPKV_E_INVALID;
+    int rc = spkv_score(cache, pred, d_x, B, d_logits_out, nullptr, stream);
+    if (rc) return rc;
+    return spkv_append_evict(cache, layer, d_seq_ids, B, d_k, d_v, d_logits_out, stream);
+  }
+  if (!pred->d_W1 || !pred->d_b1 || pred->d_in < 8 || (pred->d_in & 7)) return SPKV_E_INVALID;
+  if (((uintptr_t)d_k | (uintptr_t)d_v | (uintptr_t)d_x | (uintptr_t)pred->d_W1) & 15) return SPKV_E_INVALID;
+  const int items = B * cache->view.Hkv;
+  append_evict_kernel<<<(items + 3) / 4, 128, 0, as_stream(stream)>>>(
+      cache->view, layer, d_seq_ids, B, static_cast<const uint4 *>(d_k),
+      static_cast<const uint4 *>(d_v), nullptr, cache->tau_logit,
+      static_cast<const __nv_bfloat16 *>(d_x), static_cast<const __nv_bfloat16 *>(pred->d_W1),
+      pred->d_b1, pred->d_in, d_logits_out);
   return check_stream_error(cudaGetLastError());
 }

@@ -65,6 +65,32 @@ __device__ inline int64_t ring_page(const CacheView &c, int unit, int j) {
   return (int64_t)unit * c.ring_pages + j;
 }
 
+// ---- dot product used by the utility predictor (fixed summation order: the logit of a
+// token is bit-identical whichever kernel computes it) -------------------------------------
+__device__ inline float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// <a, b> over d elements (d % 8 == 0), a and b bf16, one warp, 16-byte loads.
+__device__ inline float warp_dot_bf16(const __nv_bfloat16 *a, const __nv_bfloat16 *b, int d, int lane) {
+  float acc = 0.f;
+  for (int i = lane * 8; i < d; i += 256) {
+    const uint4 av = *reinterpret_cast<const uint4 *>(a + i);
+    const uint4 bv = *reinterpret_cast<const uint4 *>(b + i);
+    const __nv_bfloat162 *a2 = reinterpret_cast<const __nv_bfloat162 *>(&av);
+    const __nv_bfloat162 *b2 = reinterpret_cast<const __nv_bfloat162 *>(&bv);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float2 fa = __bfloat1622float2(a2[j]), fb = __bfloat1622float2(b2[j]);
+      acc = fmaf(fa.x, fb.x, acc);
+      acc = fmaf(fa.y, fb.y, acc);
+    }
+  }
+  return warp_sum(acc);
+}
+
 }  // namespace spkv
 
 struct spkv_cache {

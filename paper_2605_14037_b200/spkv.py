@@ -76,6 +76,7 @@ def lib():
         "spkv_set_tau": (C.c_int, [vp, f32]),
         "spkv_score": (C.c_int, [vp, pp, vp, i32, vp, vp, vp]),
         "spkv_append_evict": (C.c_int, [vp, i32, vp, i32, vp, vp, vp, vp]),
+        "spkv_score_append_evict": (C.c_int, [vp, i32, pp, vp, i32, vp, vp, vp, vp, vp]),
         "spkv_decode_workspace_bytes": (sz, [cfgp, i32]),
         "spkv_decode_attention": (C.c_int, [vp, i32, vp, i32, vp, vp, vp, f32, vp, sz, vp]),
         "spkv_prefill_workspace_bytes": (sz, [cfgp, i32]),
@@ -190,6 +191,12 @@ class Cache:
                                        _ptr(k, torch.bfloat16), _ptr(v, torch.bfloat16),
                                        _ptr(logits, torch.float32), _stream(stream)),
                "spkv_append_evict")
+
+    def spkv_score_append_evict(self, layer, pred, seq_ids, x, k, v, logits_out=None, stream=None):
+        _check(lib().spkv_score_append_evict(
+            self._h, layer, C.byref(pred), _ptr(seq_ids, torch.int32), seq_ids.numel(),
+            _ptr(x, torch.bfloat16), _ptr(k, torch.bfloat16), _ptr(v, torch.bfloat16),
+            _ptr(logits_out, torch.float32), _stream(stream)), "spkv_score_append_evict")
 
     def spkv_decode_attention(self, layer, seq_ids, q, out=None, lse=None, sm_scale=None,
                               stream=None):

@@ -93,3 +93,39 @@ def test_score_then_append_chain_is_bit_exact_outside_the_guard_band():
                   ref[:, h].astype(np.float32), tl)
         pos, k, v = cache.spkv_read_kept(0, 0, h)
         assert np.array_equal(pos, u.kept()[0]) and np.array_equal(k, u.kept()[1])
+
+
+@pytest.mark.parametrize("kind", ["linear", "mlp"])
+def test_fused_score_append_equals_separate_calls(kind):
+    """spkv_score_append_evict == spkv_score followed by spkv_append_evict, bit for bit."""
+    spkv = load()
+    rng = np.random.default_rng(41)
+    Hkv, d_in, T, w, B = 4, 512, 300, 8, 3
+    mk = lambda: spkv.Cache(n_layers=1, max_seqs=B, n_q_heads=Hkv, n_kv_heads=Hkv, max_context=1024,
+                            pool_pages=40, window=w, tau=0.5)
+    a, b = mk(), mk()
+    if kind == "linear":
+        W = synth.linear_predictor(rng, Hkv, d_in)
+        bias = synth.bias_for_keep_rate(W, [0.1, 0.3, 0.6, 0.9], 0.0)
+        pred = spkv.make_predictor(to_dev_bf16(W), torch.from_numpy(bias).to(dev()))
+    else:
+        W1, b1, W2, b2 = synth.mlp_predictor(rng, Hkv, d_in, 64)
+        pred = spkv.make_predictor(to_dev_bf16(W1), torch.from_numpy(b1).to(dev()),
+                                   to_dev_bf16(W2), torch.from_numpy(b2).to(dev()))
+    x = to_dev_bf16(synth.normal_bf16(rng, (T, B, d_in)))
+    K = to_dev_bf16(synth.normal_bf16(rng, (T, B, Hkv, 128)))
+    V = to_dev_bf16(synth.normal_bf16(rng, (T, B, Hkv, 128)))
+    ids = torch.tensor([2, 0, 1], dtype=torch.int32, device=dev())
+    lg_f = torch.empty((B, Hkv), dtype=torch.float32, device=dev())
+    for t in range(T):
+        lg = a.spkv_score(pred, x[t])
+        a.spkv_append_evict(0, ids, K[t], V[t], lg)
+        b.spkv_score_append_evict(0, pred, ids, x[t], K[t], V[t], logits_out=lg_f)
+        assert torch.equal(lg, lg_f)
+    for s in range(B):
+        for h in range(Hkv):
+            for p, q in zip(a.spkv_read_kept(0, s, h), b.spkv_read_kept(0, s, h)):
+                assert np.array_equal(p, q)
+            for p, q in zip(a.spkv_read_window(0, s, h), b.spkv_read_window(0, s, h)):
+                assert np.array_equal(p, q)
+    assert a.spkv_status() == 0 and b.spkv_status() == 0
