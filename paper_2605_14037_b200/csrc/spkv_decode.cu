@@ -53,6 +53,7 @@ namespace spkv {
 
 constexpr int kTcThreads = 192;  // 4 consumer warps, producer warp, epilogue warp
 constexpr int kMaxStages = 8;
+constexpr int kMergeCap = 256;  // (slot, head) pairs staged in shared memory by a merge
 enum { F_BEGIN = 1, F_END = 2, F_STOP = 4 };
 
 struct StageMeta {
@@ -61,7 +62,7 @@ struct StageMeta {
 
 struct TcSmem {  // offsets into dynamic shared memory, computed on host and device alike
   int n_stages, red_bufs, stage_bytes, off_bar, off_meta, off_np, off_pre, off_unit, off_len, off_ring,
-      off_tmp, off_red, off_flags, total;
+      off_tmp, off_red, off_mrg, off_flags, total;
 };
 __host__ __device__ inline TcSmem tc_smem_layout(int n_items, int GP, int n_stages, int red_bufs) {
   TcSmem L;
@@ -80,6 +81,7 @@ __host__ __device__ inline TcSmem tc_smem_layout(int n_items, int GP, int n_stag
   L.off_tmp = o;   o += 64 * 4;
   o = (o + 15) / 16 * 16;
   L.off_red = o;   o += red_bufs * 4 * GP * 132 * 4;
+  L.off_mrg = o;   o += kMergeCap * 8;
   L.off_flags = o; o += 16;
   L.total = o;
   return L;
@@ -98,7 +100,7 @@ __device__ inline unsigned long long gtimer() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-#define SPKV_STAMP_T(i, cond) do { if (cond) reinterpret_cast<unsigned long long *>(a.part_acc + (size_t)3000 * a.G * kD)[blockIdx.x * 8 + (i)] = gtimer(); } while (0)
+#define SPKV_STAMP_T(i, cond) do { if (cond) reinterpret_cast<unsigned long long *>(a.part_acc + (size_t)3000 * a.G * kD)[blockIdx.x * 16 + (i)] = gtimer(); } while (0)
 #else
 #define SPKV_STAMP_T(i, cond)
 #endif
@@ -127,6 +129,7 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
   int *s_tmp = reinterpret_cast<int *>(smem + L.off_tmp);
   float *s_red = reinterpret_cast<float *>(smem + L.off_red);
   uint64_t *red_full = empty + kMaxStages, *red_empty = red_full + 2;
+  float2 *s_mrg = reinterpret_cast<float2 *>(smem + L.off_mrg);
   volatile int *s_redmeta = reinterpret_cast<volatile int *>(smem + L.off_flags);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -386,6 +389,7 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
       __syncwarp();
       if (lane == 0) mbar_arrive(&red_empty[rb]);
       if (nseg > 1) {
+        SPKV_STAMP_T(2, lane == 0);
         __threadfence();
         __syncwarp();
         int last = 0;
@@ -394,41 +398,77 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
           if (last) a.counters[item] = 0;
         }
         last = __shfl_sync(0xffffffffu, last, 0);
+        SPKV_STAMP_T(6, lane == 0);
+        SPKV_STAMP_T(7, lane == 0 && last);
         if (last) {
           __threadfence();
-          for (int gh = 0; gh < a.G; ++gh) {
-            float Mx = -INFINITY;
-            for (int sidx = c_first; sidx <= c_last; ++sidx)
-              Mx = fmaxf(Mx, __ldcg(&a.part_ml[((size_t)(sidx + item) * a.G + gh) * 2]));
-            float Ls = 0.f;
-            float4 Os = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int sidx = c_first; sidx <= c_last; ++sidx) {
-              const size_t base = (size_t)(sidx + item) * a.G + gh;
-              const float f = fast_exp2(__ldcg(&a.part_ml[base * 2]) - Mx);
-              const float4 v = __ldcg(reinterpret_cast<const float4 *>(a.part_acc + base * kD + lane * 4));
-              Ls += __ldcg(&a.part_ml[base * 2 + 1]) * f;
-              Os.x += v.x * f; Os.y += v.y * f; Os.z += v.z * f; Os.w += v.w * f;
-            }
-            const size_t row = (size_t)b * c.Hq + kvh * a.G + gh;
-            const float inv = 1.f / Ls;
-            uint2 pk;
-            pk.x = pack_bf16(Os.x * inv, Os.y * inv);
-            pk.y = pack_bf16(Os.z * inv, Os.w * inv);
-            *reinterpret_cast<uint2 *>(a.out + row * kD + lane * 4) = pk;
-            if (a.lse && lane == 0) a.lse[row] = (Mx + log2f(Ls)) * kLn2;
+          SPKV_STAMP_T(8, lane == 0);
+          // (m, l) of every slot and head go through shared memory first (one round of
+          // loads for the whole warp); the accumulator loads below are then independent
+          const int n_ml = nseg * a.G;
+          const bool staged = n_ml <= kMergeCap;
+          if (staged) {
+            for (int idx = lane; idx < n_ml; idx += 32)
+              s_mrg[idx] = __ldcg(reinterpret_cast<const float2 *>(a.part_ml) + (size_t)(c_first + item) * a.G + idx);
+            __syncwarp();
           }
+          SPKV_STAMP_T(9, lane == 0);
+#ifdef SPKV_PHASE_TIMING
+          if (lane == 0) reinterpret_cast<unsigned long long *>(a.part_acc + (size_t)3000 * a.G * kD)[blockIdx.x * 16 + 11] = nseg;
+#endif
+          const float2 *g_ml = reinterpret_cast<const float2 *>(a.part_ml) + (size_t)(c_first + item) * a.G;
+          const float *g_acc = a.part_acc + (size_t)(c_first + item) * a.G * kD + lane * 4;
+          auto ml_of = [&](int si, int gh) { return staged ? s_mrg[si * a.G + gh] : __ldcg(g_ml + si * a.G + gh); };
+          // four heads x eight slots at a time: 32 independent 16-byte loads in flight
+          for (int gh0 = 0; gh0 < a.G; gh0 += 4) {
+            float Mx[4], Ls[4];
+            float4 Os[4];
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+              Mx[h] = -INFINITY; Ls[h] = 0.f; Os[h] = make_float4(0.f, 0.f, 0.f, 0.f);
+              if (gh0 + h < a.G)
+                for (int si = 0; si < nseg; ++si) Mx[h] = fmaxf(Mx[h], ml_of(si, gh0 + h).x);
+            }
+            for (int s0 = 0; s0 < nseg; s0 += 8) {
+              float4 v[8][4];
+#pragma unroll
+              for (int x = 0; x < 8; ++x)
+#pragma unroll
+                for (int h = 0; h < 4; ++h)
+                  v[x][h] = (s0 + x < nseg && gh0 + h < a.G)
+                                ? __ldcg(reinterpret_cast<const float4 *>(
+                                      g_acc + ((size_t)(s0 + x) * a.G + gh0 + h) * kD))
+                                : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+              for (int x = 0; x < 8; ++x)
+#pragma unroll
+                for (int h = 0; h < 4; ++h)
+                  if (s0 + x < nseg && gh0 + h < a.G) {
+                    const float2 ml = ml_of(s0 + x, gh0 + h);
+                    const float f = fast_exp2(ml.x - Mx[h]);
+                    Ls[h] += ml.y * f;
+                    Os[h].x += v[x][h].x * f; Os[h].y += v[x][h].y * f;
+                    Os[h].z += v[x][h].z * f; Os[h].w += v[x][h].w * f;
+                  }
+            }
+#pragma unroll
+            for (int h = 0; h < 4; ++h)
+              if (gh0 + h < a.G) {
+                const size_t row = (size_t)b * c.Hq + kvh * a.G + gh0 + h;
+                const float inv = 1.f / Ls[h];
+                uint2 pk;
+                pk.x = pack_bf16(Os[h].x * inv, Os[h].y * inv);
+                pk.y = pack_bf16(Os[h].z * inv, Os[h].w * inv);
+                *reinterpret_cast<uint2 *>(a.out + row * kD + lane * 4) = pk;
+                if (a.lse && lane == 0) a.lse[row] = (Mx[h] + log2f(Ls[h])) * kLn2;
+              }
+          }
+          SPKV_STAMP_T(10, lane == 0);
         }
       }
     }
   }
   SPKV_STAMP_T(4, tid == 0);
-#ifdef SPKV_PHASE_TIMING
-  if (tid == 0) {
-    unsigned long long *dbg = reinterpret_cast<unsigned long long *>(a.part_acc + (size_t)3000 * a.G * kD);
-    dbg[blockIdx.x * 8 + 6] = dbg_pages;
-    dbg[blockIdx.x * 8 + 7] = dbg_segs;
-  }
-#endif
   __syncthreads();
   SPKV_STAMP_T(5, tid == 0);
 }
