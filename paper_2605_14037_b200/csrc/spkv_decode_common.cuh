@@ -6,7 +6,7 @@
 namespace spkv {
 
 constexpr int kMaxGrid = 1024;
-constexpr int kMaxSlots = 3328;  // upper bound on the number of page ranges ("chunks") of a launch
+constexpr int kMaxSlots = kMaxGrid;  // one partial slot per (block + item): see the merge
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
