@@ -53,7 +53,8 @@ enum {
   SPKV_E_CONTEXT_OVERFLOW = -6, /* device: a unit's page table is full                 */
   SPKV_E_WORKSPACE = -7,        /* workspace missing or too small                      */
   SPKV_E_TIMEOUT = -8,          /* device: a bounded wait on a copy ran out            */
-  SPKV_E_BOUNDS = -9            /* device: a sequence id outside [0, max_seqs)         */
+  SPKV_E_BOUNDS = -9,           /* device: a sequence id outside [0, max_seqs)         */
+  SPKV_E_SCRATCH_LIMIT = -10    /* request larger than the library's built-in scratch  */
 };
 
 typedef struct {
@@ -171,6 +172,31 @@ int spkv_decode_attention(spkv_cache_t *cache, int32_t layer, const int32_t *d_s
                           int32_t B, const void *d_q, void *d_out, float *d_lse_opt,
                           float sm_scale, void *d_workspace, size_t workspace_bytes,
                           spkv_stream_t stream);
+
+/* (No counterpart in the paper: an addition for integration.)
+ * spkv_decode_attention for callers that must not allocate device memory -- code running
+ * inside someone else's memory plan, where every cudaMalloc is forbidden or already spoken
+ * for (a serving engine that has handed all free HBM to its own KV pool, a plugin loaded
+ * into a host application, a latency-critical loop that may not touch the allocator).
+ * It computes exactly what spkv_decode_attention computes, but its split-K scratch is a
+ * fixed SPKV_STATIC_SCRATCH_BYTES array that is part of the library image on every GPU,
+ * so no workspace is passed and nothing is allocated or freed, here or in any library
+ * routine it calls.  Inputs and outputs are still the caller's.
+ *   - Sizes: B and the head configuration must satisfy
+ *     spkv_decode_workspace_bytes(cfg, B) <= SPKV_STATIC_SCRATCH_BYTES, otherwise the call
+ *     returns SPKV_E_SCRATCH_LIMIT and does nothing (with 8 KV heads: every supported batch
+ *     at 4 query heads per KV head, batches up to 32 at 8 per KV head; beyond that use
+ *     spkv_decode_attention with a workspace of your own).
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current).  Make that first call outside of any stream capture.
+ *   - All calls on a device share the one array and it keeps the previous call's contents;
+ *     the entry point clears the part that must start at zero on `stream` before the
+ *     kernel.  Two calls whose GPU work overlaps (different streams, no dependency) race on
+ *     it: keep such calls ordered. */
+#define SPKV_STATIC_SCRATCH_BYTES (6u << 20)
+int spkv_decode_attention_static(spkv_cache_t *cache, int32_t layer, const int32_t *d_seq_ids,
+                                 int32_t B, const void *d_q, void *d_out, float *d_lse_opt,
+                                 float sm_scale, spkv_stream_t stream);
 
 /* Workspace bytes spkv_prefill needs for a chunk of C pairs. */
 size_t spkv_prefill_workspace_bytes(const spkv_config_t *cfg, int32_t C);

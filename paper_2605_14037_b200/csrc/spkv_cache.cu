@@ -322,6 +322,7 @@ extern "C" const char *spkv_error_string(int code) {
     case SPKV_E_WORKSPACE: return "workspace missing or too small";
     case SPKV_E_TIMEOUT: return "bounded device wait ran out";
     case SPKV_E_BOUNDS: return "sequence id out of range";
+    case SPKV_E_SCRATCH_LIMIT: return "request exceeds the built-in scratch area";
     default: return "unknown error";
   }
 }

@@ -532,6 +532,45 @@ extern "C" int spkv_decode_attention(spkv_cache_t *cache, int32_t layer, const i
   return check_stream_error(cudaGetLastError());
 }
 
+// ---- decode attention for callers that cannot allocate device memory ---------------------
+//
+// The split-K scratch (arrival counters and partial results) of this variant lives in a
+// fixed array inside the library's device image instead of a caller-supplied workspace.
+// Every GPU that loads the library carries these 6 MiB until the process exits.
+static __device__ __align__(256) unsigned char g_static_scratch[SPKV_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void *g_scratch_ptr[kMaxDevices];  // device address of g_static_scratch, per device
+bool g_scratch_ready[kMaxDevices];
+}  // namespace
+
+extern "C" int spkv_decode_attention_static(spkv_cache_t *cache, int32_t layer, const int32_t *d_seq_ids,
+                                            int32_t B, const void *d_q, void *d_out, float *d_lse_opt,
+                                            float sm_scale, spkv_stream_t stream) {
+  if (!cache || B < 0) return SPKV_E_INVALID;
+  const size_t need = spkv_decode_workspace_bytes(&cache->cfg, B);
+  if (need > (size_t)SPKV_STATIC_SCRATCH_BYTES) return SPKV_E_SCRATCH_LIMIT;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SPKV_E_CUDA;
+  if (!g_scratch_ready[dev]) {
+    // In host code `g_static_scratch` names a host-side stand-in, not device memory: the
+    // address a kernel may use has to be asked for, once per device, with that device current.
+    void *p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return SPKV_E_CUDA;
+    g_scratch_ptr[dev] = p;
+    g_scratch_ready[dev] = true;
+  }
+  void *scratch = g_scratch_ptr[dev];
+  if (B > 0) {
+    // the array keeps whatever the previous call left: the arrival counters must start at zero
+    const size_t counters = (size_t)B * cache->cfg.n_kv_heads * 4;
+    if (cudaMemsetAsync(scratch, 0, counters, as_stream(stream)) != cudaSuccess) return SPKV_E_CUDA;
+  }
+  return spkv_decode_attention(cache, layer, d_seq_ids, B, d_q, d_out, d_lse_opt, sm_scale, scratch,
+                               SPKV_STATIC_SCRATCH_BYTES, stream);
+}
+
 static size_t a256(size_t x) { return (x + 255) / 256 * 256; }
 
 extern "C" size_t spkv_decode_step_staging_bytes(const spkv_config_t *cfg, int32_t B, int32_t d_in) {

@@ -23,7 +23,7 @@ SPKV_OK = 0
 ERRORS = {
     -1: "SPKV_E_INVALID", -2: "SPKV_E_ARENA_TOO_SMALL", -3: "SPKV_E_UNSUPPORTED", -4: "SPKV_E_CUDA",
     -5: "SPKV_E_POOL_EXHAUSTED", -6: "SPKV_E_CONTEXT_OVERFLOW", -7: "SPKV_E_WORKSPACE",
-    -8: "SPKV_E_TIMEOUT", -9: "SPKV_E_BOUNDS",
+    -8: "SPKV_E_TIMEOUT", -9: "SPKV_E_BOUNDS", -10: "SPKV_E_SCRATCH_LIMIT",
 }
 
 
@@ -79,6 +79,7 @@ def lib():
         "spkv_score_append_evict": (C.c_int, [vp, i32, pp, vp, i32, vp, vp, vp, vp, vp]),
         "spkv_decode_workspace_bytes": (sz, [cfgp, i32]),
         "spkv_decode_attention": (C.c_int, [vp, i32, vp, i32, vp, vp, vp, f32, vp, sz, vp]),
+        "spkv_decode_attention_static": (C.c_int, [vp, i32, vp, i32, vp, vp, vp, f32, vp]),
         "spkv_prefill_workspace_bytes": (sz, [cfgp, i32]),
         "spkv_prefill": (C.c_int, [vp, i32, i32, i32, vp, vp, vp, vp, vp, f32, vp, sz, vp]),
         "spkv_decode_step_staging_bytes": (sz, [cfgp, i32, i32]),
@@ -209,6 +210,20 @@ class Cache:
             _ptr(out, torch.bfloat16), _ptr(lse, torch.float32),
             self.default_scale if sm_scale is None else sm_scale, _ptr(ws), ws.numel(),
             _stream(stream)), "spkv_decode_attention")
+        return out
+
+    def spkv_decode_attention_static(self, layer, seq_ids, q, out=None, lse=None, sm_scale=None,
+                                     stream=None):
+        """Same result as spkv_decode_attention, for callers that may not allocate device
+        memory: the scratch is a fixed array inside the library (no workspace tensor)."""
+        B = seq_ids.numel()
+        if out is None:
+            out = torch.empty_like(q)
+        _check(lib().spkv_decode_attention_static(
+            self._h, layer, _ptr(seq_ids, torch.int32), B, _ptr(q, torch.bfloat16),
+            _ptr(out, torch.bfloat16), _ptr(lse, torch.float32),
+            self.default_scale if sm_scale is None else sm_scale, _stream(stream)),
+            "spkv_decode_attention_static")
         return out
 
     def spkv_prefill(self, layer, seq, k, v, logits, q=None, out=None, sm_scale=None, stream=None):

@@ -85,8 +85,8 @@ def test_workspace_sizes_and_error_strings(spkv):
     assert l.spkv_decode_step_staging_bytes(C.byref(c), 3, 512) > b
     assert l.spkv_prefill_workspace_bytes(C.byref(c), 8192) > 0
     assert l.spkv_error_string(0) == b"ok"
-    seen = {l.spkv_error_string(code) for code in range(-9, 1)}
-    assert len(seen) == 10 and b"unknown error" not in seen
+    seen = {l.spkv_error_string(code) for code in range(-10, 1)}
+    assert len(seen) == 11 and b"unknown error" not in seen
     assert l.spkv_error_string(-99) == b"unknown error"
     # null handles are rejected, not dereferenced
     assert l.spkv_cache_destroy(None) == -1
