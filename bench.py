@@ -96,6 +96,23 @@ class ClockSampler:
             self.result = {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(mx), "reasons": sorted(reasons)}
 
 
+def max_over_ranks(x, dist=None, device=None):
+    """Largest value of x over the ranks of the job (x itself without a process group)."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return float(x)
+    import torch
+    t = torch.tensor([float(x)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(units_per_rank, seconds_local, dist=None, device=None):
+    """Replicas only: every rank processes `units_per_rank` units; the job's rate is all
+    ranks' units over the slowest rank's time."""
+    world = dist.get_world_size() if dist is not None and dist.is_initialized() else 1
+    return world * units_per_rank / max_over_ranks(seconds_local, dist, device)
+
+
 def build_workload(spkv, synth, torch, cfg, dev, dense, total_steps, seed=0):
     """Creates the cache, per-layer predictors and brings every sequence to context T."""
     import numpy as np
@@ -173,12 +190,8 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    def max_over_ranks(x):
-        if dist is None:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    def max_ranks(x):
+        return max_over_ranks(x, dist, dev)
 
     def measure(dense):
         cache, preds, rates, gen = build_workload(spkv, synth, torch, cfg, dev, dense, total_steps)
@@ -241,7 +254,7 @@ def run_ours(args):
             e1.record()
             torch.cuda.synchronize()
         barrier()
-        ms = max_over_ranks(e0.elapsed_time(e1))
+        ms = max_ranks(e0.elapsed_time(e1))
         cache.check()
         st1 = cache.spkv_cache_stats()
 
@@ -286,7 +299,7 @@ def run_ours(args):
             for s in range(e2e_steps):
                 e2e_step(s)
             torch.cuda.synchronize()
-            dt = max_over_ranks(time.perf_counter() - t0)
+            dt = max_ranks(time.perf_counter() - t0)
             cache.check()
             res["e2e"] = {
                 "value": world * B * e2e_steps / dt, "unit": "tokens/s",

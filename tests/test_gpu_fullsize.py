@@ -1,0 +1,103 @@
+"""Parity at the benchmark's full size and launch configuration: one layer of the
+Llama-3-8B-shaped decode workload (batch 16, 32 query / 8 KV heads, context 32768, window 128,
+per-head keep rates ~ Beta(0.5, 2)).  The cache is built with 8192-pair prefill chunks and
+then stepped with batch-16 calls exactly as bench.py does.  Checked:
+  * compact-cache length of all 128 units == count of logits >= tau_logit among the pairs that
+    left the window (kept-set identity), bit-exact;
+  * for two sampled sequences (16 units, CPU-generated K/V): kept positions and bytes bit-exact
+    against the oracle, sampled prefill outputs against the oracle's mask form, and the decode
+    outputs of three steps against the oracle's streaming form, within the attention tolerance.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gpu_util import D, assert_attn_close, compare_state, dev, load, to_dev_bf16
+from paper_2605_14037_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def test_config2_one_layer_full_size():
+    spkv = load()
+    B, Hq, Hkv, T, w, C, steps = 16, 32, 8, 32768, 128, 8192, 3
+    G = Hq // Hkv
+    sampled = [3, 11]
+    rng = np.random.default_rng(1234)
+    rates = synth.keep_rates(rng, 1, Hkv, 0.5, 2.0)[0]
+    rates[0], rates[5] = 0.0, 0.97                       # a local-only head and a near-full head
+    pages = int(np.ceil(rates * (T + steps) * 1.05 / 64 + 2).sum()) * B
+    cache = spkv.Cache(n_layers=1, max_seqs=B, n_q_heads=Hq, n_kv_heads=Hkv, max_context=T + 128,
+                       pool_pages=pages, window=w, tau=0.5)
+    tl = cache.spkv_tau_logit()
+    Tt = T + steps
+    logit = np.stack([synth.logits_with_keep_rate(rng, (Tt, B), float(r), tl) for r in rates], axis=-1)
+    Ks = {s: synth.normal_bf16(rng, (Tt, Hkv, D)) for s in sampled}
+    Vs = {s: synth.normal_bf16(rng, (Tt, Hkv, D)) for s in sampled}
+    q_last = {s: synth.normal_bf16(rng, (C, Hq, D)) for s in sampled}      # queries of the last chunk
+    gen = torch.Generator(device=dev())
+    gen.manual_seed(7)
+    lg_dev = torch.from_numpy(logit).to(dev())
+    prefill_out = {}
+    for s in range(B):
+        if s in sampled:
+            Kd, Vd = to_dev_bf16(Ks[s][:T]), to_dev_bf16(Vs[s][:T])
+        else:
+            Kd = torch.randn((T, Hkv, D), generator=gen, device=dev()).to(torch.bfloat16)
+            Vd = torch.randn((T, Hkv, D), generator=gen, device=dev()).to(torch.bfloat16)
+        for a in range(0, T, C):
+            last = a + C == T and s in sampled
+            o = cache.spkv_prefill(0, s, Kd[a:a + C], Vd[a:a + C], lg_dev[a:a + C, s].contiguous(),
+                                   q=to_dev_bf16(q_last[s]) if last else None)
+            if last:
+                prefill_out[s] = spkv.bits_from_bf16(o)
+    assert cache.spkv_status() == 0
+
+    # sampled prefill queries against the mask form (Eq. 2-5 written out)
+    scale = 1.0 / math.sqrt(D)
+    for s in sampled:
+        for t in (T - C, T - C + 127, T - C + 128, T - 4097, T - 1):
+            for h in (0, 3, 5):
+                ref = oracle.mask_attend_row(
+                    np.ascontiguousarray(Ks[s][:T, h]), np.ascontiguousarray(Vs[s][:T, h]),
+                    np.ascontiguousarray(logit[:T, s, h]), t, w, tl,
+                    np.ascontiguousarray(q_last[s][t - (T - C), h * G:(h + 1) * G]), scale)
+                assert_attn_close(prefill_out[s][t - (T - C), h * G:(h + 1) * G], ref, f"prefill s={s} t={t} h={h}")
+
+    # oracle streaming state of the sampled units
+    units = {s: [oracle.Unit(w, D) for _ in range(Hkv)] for s in sampled}
+    for s in sampled:
+        for h in range(Hkv):
+            units[s][h].prefill(np.ascontiguousarray(Ks[s][:T, h]), np.ascontiguousarray(Vs[s][:T, h]),
+                                np.ascontiguousarray(logit[:T, s, h]), tl)
+
+    ids = torch.arange(B, dtype=torch.int32, device=dev())
+    for step in range(steps):
+        t = T + step
+        k_new = torch.randn((B, Hkv, D), generator=gen, device=dev()).to(torch.bfloat16)
+        v_new = torch.randn((B, Hkv, D), generator=gen, device=dev()).to(torch.bfloat16)
+        q_new = torch.randn((B, Hq, D), generator=gen, device=dev()).to(torch.bfloat16)
+        for s in sampled:
+            k_new[s], v_new[s] = to_dev_bf16(Ks[s][t]), to_dev_bf16(Vs[s][t])
+        cache.spkv_append_evict(0, ids, k_new, v_new, lg_dev[t].contiguous())
+        out = spkv.bits_from_bf16(cache.spkv_decode_attention(0, ids, q_new))
+        q_bits = spkv.bits_from_bf16(q_new)
+        for s in sampled:
+            for h in range(Hkv):
+                units[s][h].append(Ks[s][t, h], Vs[s][t, h], logit[t, s, h], tl)
+                ref = units[s][h].attend(np.ascontiguousarray(q_bits[s, h * G:(h + 1) * G]), scale)
+                assert_attn_close(out[s, h * G:(h + 1) * G], ref, f"decode step={step} s={s} h={h}")
+    assert cache.spkv_status() == 0
+
+    ln, tt = cache.spkv_read_lengths(0)
+    want = (logit[:Tt - w] >= np.float32(tl)).sum(axis=0)          # [B, Hkv]
+    assert np.array_equal(ln, want.astype(np.int32)) and (tt == Tt).all()
+    assert ln[:, 0].max() == 0 and ln[:, 5].min() > 0.9 * T
+    for s in sampled:
+        for h in (0, 2, 5):
+            compare_state(cache, 0, s, h, units[s][h])
+    st = cache.spkv_cache_stats()
+    assert abs(st.density_cache - want.sum() / (B * Hkv * (Tt - w))) < 1e-12
