@@ -68,8 +68,16 @@ typedef struct {
   int32_t max_context;  /* upper bound on kept pairs per unit (sizes the page tables)   */
   int64_t pool_pages;   /* pages shared by all compact caches                           */
   float tau;            /* utility threshold in [0,1]; <= 0 keeps all, >= 1 keeps none  */
-  int32_t flags;        /* reserved, 0                                                  */
+  int32_t flags;        /* 0 or SPKV_FLAG_NO_OVERLAP                                    */
 } spkv_config_t;
+
+/* By default consecutive hot-path launches on one stream overlap where they share no data
+ * (programmatic dependent launch): the append of layer l+1 may run beside the decode attention
+ * of layer l, and the decode attention of layer l+1 starts on the SMs that the one of layer l
+ * has already left.  What the caller has to respect: two decode calls issued back to back,
+ * with nothing but this library's append between them, must not write the same d_out.
+ * SPKV_FLAG_NO_OVERLAP turns this off (every launch then waits for the previous one). */
+#define SPKV_FLAG_NO_OVERLAP 1
 
 /* Utility predictor f of Eq. 1 (the sigmoid is never evaluated: the decision is taken
  * in logit space, u >= tau  <=>  logit >= log(tau/(1-tau))).
@@ -165,9 +173,9 @@ size_t spkv_decode_workspace_bytes(const spkv_config_t *cfg, int32_t B);
  * results merged by their log-sum-exp weights.
  *   d_q [B, n_q_heads, 128] bf16 -> d_out [B, n_q_heads, 128] bf16;
  *   d_lse_opt [B, n_q_heads] float32 natural-log sum-exp of the scaled scores, or NULL;
- *   d_workspace: >= spkv_decode_workspace_bytes(cfg, B) bytes, 256-byte aligned; its
- *   contents need not be preserved between calls, but it must have been zero-filled
- *   once before its first use. */
+ *   d_workspace: >= spkv_decode_workspace_bytes(cfg, B) bytes, 256-byte aligned, used by
+ *   this cache only; it must have been zero-filled once before its first use and is then
+ *   left alone by the caller (consecutive calls alternate between its two halves). */
 int spkv_decode_attention(spkv_cache_t *cache, int32_t layer, const int32_t *d_seq_ids,
                           int32_t B, const void *d_q, void *d_out, float *d_lse_opt,
                           float sm_scale, void *d_workspace, size_t workspace_bytes,

@@ -36,7 +36,14 @@ append_evict_kernel(CacheView c, int layer, const int32_t *__restrict__ seq_ids,
                     const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new,
                     const float *__restrict__ logits, float tau_logit,
                     const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__restrict__ W,
-                    const float *__restrict__ bias, int d_in, float *__restrict__ logits_out) {
+                    const float *__restrict__ bias, int d_in, float *__restrict__ logits_out,
+                    int wait_prev) {
+  // The previous kernel of the stream may still be running (see launch_overlapped).  The host
+  // passes wait_prev = 0 only when that kernel was a decode/append of ANOTHER layer of this
+  // cache: it shares no data with this launch, and ordering with everything older is kept by
+  // the decode kernels, which always wait.
+  if (wait_prev) pdl_wait();
+  pdl_trigger();
   const int lane = threadIdx.x & 31;
   const int item = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (item >= B * c.Hkv) return;
@@ -105,6 +112,19 @@ append_evict_kernel(CacheView c, int layer, const int32_t *__restrict__ seq_ids,
 
 using namespace spkv;
 
+// Records this append as the cache's latest launch and tells whether it has to wait for the
+// kernel before it: always, unless that kernel was a decode/append of a different layer of
+// this cache on the same stream.
+static int append_must_wait(spkv_cache *cache, int layer, cudaStream_t s) {
+  const bool independent = (cache->last_kind == kLastDecode || cache->last_kind == kLastAppend) &&
+                           cache->last_layer != layer && cache->last_stream == s &&
+                           !(cache->cfg.flags & SPKV_FLAG_NO_OVERLAP);
+  cache->last_kind = kLastAppend;
+  cache->last_layer = layer;
+  cache->last_stream = s;
+  return independent ? 0 : 1;
+}
+
 extern "C" int spkv_append_evict(spkv_cache_t *cache, int32_t layer, const int32_t *d_seq_ids,
                                  int32_t B, const void *d_k, const void *d_v,
                                  const float *d_logits, spkv_stream_t stream) {
@@ -114,10 +134,12 @@ extern "C" int spkv_append_evict(spkv_cache_t *cache, int32_t layer, const int32
   if (!d_seq_ids || !d_k || !d_v || !d_logits) return SPKV_E_INVALID;
   if (((uintptr_t)d_k | (uintptr_t)d_v) & 15) return SPKV_E_INVALID;
   const int items = B * cache->view.Hkv;
-  append_evict_kernel<<<(items + 3) / 4, 128, 0, as_stream(stream)>>>(
-      cache->view, layer, d_seq_ids, B, static_cast<const uint4 *>(d_k),
-      static_cast<const uint4 *>(d_v), d_logits, cache->tau_logit, nullptr, nullptr, nullptr, 0, nullptr);
-  return check_stream_error(cudaGetLastError());
+  const int wait_prev = append_must_wait(cache, layer, as_stream(stream));
+  return check_stream_error(launch_overlapped(
+      append_evict_kernel, dim3((items + 3) / 4), dim3(128), 0, as_stream(stream), cache->view, layer,
+      d_seq_ids, B, static_cast<const uint4 *>(d_k), static_cast<const uint4 *>(d_v), d_logits,
+      cache->tau_logit, (const __nv_bfloat16 *)nullptr, (const __nv_bfloat16 *)nullptr,
+      (const float *)nullptr, 0, (float *)nullptr, wait_prev));
 }
 
 extern "C" int spkv_score_append_evict(spkv_cache_t *cache, int32_t layer, const spkv_predictor_t *pred,
@@ -134,15 +156,16 @@ extern "C" int spkv_score_append_evict(spkv_cache_t *cache, int32_t layer, const
     if (!d_logits_out) return SPKV_E_INVALID;
     int rc = spkv_score(cache, pred, d_x, B, d_logits_out, nullptr, stream);
     if (rc) return rc;
+    cache->last_kind = kLastOther;
     return spkv_append_evict(cache, layer, d_seq_ids, B, d_k, d_v, d_logits_out, stream);
   }
   if (!pred->d_W1 || !pred->d_b1 || pred->d_in < 8 || (pred->d_in & 7)) return SPKV_E_INVALID;
   if (((uintptr_t)d_k | (uintptr_t)d_v | (uintptr_t)d_x | (uintptr_t)pred->d_W1) & 15) return SPKV_E_INVALID;
   const int items = B * cache->view.Hkv;
-  append_evict_kernel<<<(items + 3) / 4, 128, 0, as_stream(stream)>>>(
-      cache->view, layer, d_seq_ids, B, static_cast<const uint4 *>(d_k),
-      static_cast<const uint4 *>(d_v), nullptr, cache->tau_logit,
-      static_cast<const __nv_bfloat16 *>(d_x), static_cast<const __nv_bfloat16 *>(pred->d_W1),
-      pred->d_b1, pred->d_in, d_logits_out);
-  return check_stream_error(cudaGetLastError());
+  const int wait_prev = append_must_wait(cache, layer, as_stream(stream));
+  return check_stream_error(launch_overlapped(
+      append_evict_kernel, dim3((items + 3) / 4), dim3(128), 0, as_stream(stream), cache->view, layer,
+      d_seq_ids, B, static_cast<const uint4 *>(d_k), static_cast<const uint4 *>(d_v),
+      (const float *)nullptr, cache->tau_logit, static_cast<const __nv_bfloat16 *>(d_x),
+      static_cast<const __nv_bfloat16 *>(pred->d_W1), pred->d_b1, pred->d_in, d_logits_out, wait_prev));
 }

@@ -107,6 +107,10 @@ extern "C" int spkv_cache_create(const spkv_config_t *cfg, void *d_arena, size_t
   c->layout = l;
   c->arena = d_arena;
   c->tau_logit = tau_to_logit(cfg->tau);
+  c->last_kind = kLastOther;
+  c->last_layer = -1;
+  c->last_stream = nullptr;
+  c->ws_toggle = 0;
   char *base = static_cast<char *>(d_arena);
   CacheView &v = c->view;
   v.L = cfg->n_layers; v.S = cfg->max_seqs; v.Hq = cfg->n_q_heads; v.Hkv = cfg->n_kv_heads;
@@ -159,6 +163,7 @@ extern "C" int spkv_cache_destroy(spkv_cache_t *cache) {
 
 extern "C" int spkv_cache_reset_seq(spkv_cache_t *cache, int32_t seq, spkv_stream_t stream) {
   if (!cache || seq < 0 || seq >= cache->cfg.max_seqs) return SPKV_E_INVALID;
+  cache->last_kind = kLastOther;
   reset_seq_kernel<<<cache->view.L * cache->view.Hkv, 256, 0, as_stream(stream)>>>(cache->view, seq);
   return check_stream_error(cudaGetLastError());
 }

@@ -24,10 +24,11 @@
 //       32 lanes in parallel, then issues one 32 KB linear bulk copy HBM -> shared memory
 //       per page (cp.async.bulk on an mbarrier) plus, at the start of a segment, the
 //       G query rows.  The page in HBM already is the swizzled shared-memory image.
-//   consumers each take 16 of the page's 64 pairs.  The group's G query heads are the rows
-//       of a 16-row tile, so S = Q K^T and O += P V are small dense products done with
-//       mma.sync m16n8k16 (bf16 in, fp32 accumulate), operands read with ldmatrix; mask,
-//       online softmax (exp2, quad shuffles) in registers.  Each warp keeps (m, l, O) for
+//   consumers each take 16 of the page's 64 pairs.  The 16 keys are the rows and the group's
+//       G query heads the (8-wide) columns of the tiles, so S^T = K Q^T and O^T += V^T P^T are
+//       small dense products done with mma.sync m16n8k16 (bf16 in, fp32 accumulate): 8 + 16
+//       MMAs per warp and page, operands read with ldmatrix; mask, online softmax (exp2,
+//       shuffles over the keys) in registers.  Each warp keeps (m, l, O) for
 //       its quarter of every page of a segment and drops it into one of two shared-memory
 //       buffers at the segment's end, then carries straight on with the next segment.
 //   epilogue  merges the four warps' results of a finished segment, writes the output (or
@@ -36,7 +37,7 @@
 // Why tensor cores in a bandwidth-bound kernel: per 512 B pair the group needs 2*G*128
 // multiply-adds.  On the CUDA cores (spkv_decode_simt.cu) that is, with bf16 unpacking and
 // the reductions, several hundred issue slots per pair and SM, and the issue rate, not
-// HBM, limits the kernel from G = 4 on.  As MMA tiles it is 48 instructions per page and
+// HBM, limits the kernel from G = 4 on.  As MMA tiles it is 24 instructions per page and
 // warp, and the page stream alone sets the pace.
 //
 // Every wait is bounded (about a second).  A consumer warp whose page never lands records
@@ -87,7 +88,8 @@ __host__ __device__ inline TcSmem tc_smem_layout(int n_items, int GP, int n_stag
   return L;
 }
 
-// Equal cut of the axis of VP positions into nb ranges.
+// Equal cut of the axis of VP positions into nb ranges (exact integer arithmetic: every block
+// must compute identical boundaries).
 struct Ranges {
   int VP, nb;
   __device__ int start(int c) const { return (int)(((long long)c * VP) / nb); }
@@ -112,6 +114,7 @@ __device__ inline bool wait_or_flag(uint64_t *bar, uint32_t parity, const CacheV
   return false;
 }
 
+template <int NH>  // 8-head tiles on the N side: 1 for G <= 8, 2 for G <= 16
 __global__ void __launch_bounds__(kTcThreads, 1)
 decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
   extern __shared__ __align__(1024) unsigned char smem[];
@@ -156,6 +159,10 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
     reinterpret_cast<uint4 *>(smem + (size_t)st * L.stage_bytes + kPageBytes + a.G * kRowBytes)[r] =
         make_uint4(0, 0, 0, 0);
   }
+  // Everything above touched only this block's shared memory and may overlap the tail of the
+  // previous kernel of the stream; from here on its results (lengths, pages) are read.
+  pdl_wait();
+  pdl_trigger();
   for (int i = tid; i < n; i += kTcThreads) {
     const int b = i / c.Hkv, kvh = i % c.Hkv;
     const int seq = a.seq_ids[b];
@@ -273,8 +280,8 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
     }
   } else if (warp < 4) {
     // ----------------------------------------------------------------- consumer warps
-    uint32_t qf[8][4];
-    float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f}, o[16][4];
+    uint32_t qb[NH][8][2];
+    float m[NH][2], l[NH][2], o[NH][8][4];
     const int g = lane >> 2, t4 = lane & 3;
     int n_seg = 0;
     for (int k = 0;; ++k) {
@@ -287,20 +294,27 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
       unsigned char *sbase = smem + (size_t)stage * L.stage_bytes;
       if (flags & F_BEGIN) {
         const __nv_bfloat16 *qs = reinterpret_cast<const __nv_bfloat16 *>(sbase + kPageBytes);
-        load_q_frags(qf, [&](int r) -> const __nv_bfloat16 * { return r < GP ? qs + r * kD : nullptr; }, lane);
-        m[0] = m[1] = -INFINITY;
-        l[0] = l[1] = 0.f;
+        load_q_frags_t<NH>(qb, [&](int h) -> const __nv_bfloat16 * { return h < GP ? qs + h * kD : nullptr; },
+                           lane);
 #pragma unroll
-        for (int x = 0; x < 16; ++x) o[x][0] = o[x][1] = o[x][2] = o[x][3] = 0.f;
+        for (int hn = 0; hn < NH; ++hn) {
+          m[hn][0] = m[hn][1] = -INFINITY;
+          l[hn][0] = l[hn][1] = 0.f;
+#pragma unroll
+          for (int mt = 0; mt < 8; ++mt) o[hn][mt][0] = o[hn][mt][1] = o[hn][mt][2] = o[hn][mt][3] = 0.f;
+        }
       }
       const int tok0 = warp * 16;
+#ifndef SPKV_PROBE_NOCOMPUTE
       if (tok0 < valid) {
         const uint32_t sK = smem_u32(sbase), sV = sK + kBlockElems * 2;
-        float s[2][4];
-        qk_tile<16>(s, qf, sK, tok0, lane);
-        softmax_pv_tile<16>(s, [&](int, int col) { return col < valid; }, a.scale_log2, m, l, o, sV, tok0,
-                            lane);
+        float s[NH][4];
+        qk_tile_t<NH>(s, qb, sK, tok0, lane);
+        softmax_pv_tile_t<NH>(s, valid, a.scale_log2, m, l, o, sV, tok0, lane);
       }
+#else
+      if (tok0 < valid) { m[0][0] = 0.f; l[0][0] = 1.f; }
+#endif
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty[stage]);
 #ifdef SPKV_PHASE_TIMING
@@ -315,18 +329,24 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
       if (ruse > 0 && !wait_or_flag(&red_empty[rb], (ruse - 1) & 1, c)) break;
       float *red = s_red + (size_t)rb * 4 * GP * 132;
 #pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        l[h] += __shfl_xor_sync(0xffffffffu, l[h], 1);
-        l[h] += __shfl_xor_sync(0xffffffffu, l[h], 2);
-        const int row = g + 8 * h;
-        if (row < a.G) {
-          float *dst = red + ((size_t)warp * GP + row) * 132;
+      for (int hn = 0; hn < NH; ++hn)
 #pragma unroll
-          for (int x = 0; x < 16; ++x)
-            *reinterpret_cast<float2 *>(dst + x * 8 + t4 * 2) = make_float2(o[x][2 * h], o[x][2 * h + 1]);
-          if (t4 == 0) { dst[128] = m[h]; dst[129] = l[h]; }
+        for (int j = 0; j < 2; ++j) {
+          float lv = l[hn][j];
+          lv += __shfl_xor_sync(0xffffffffu, lv, 4);
+          lv += __shfl_xor_sync(0xffffffffu, lv, 8);
+          lv += __shfl_xor_sync(0xffffffffu, lv, 16);
+          const int h = hn * 8 + t4 * 2 + j;
+          if (h < a.G) {
+            float *dst = red + ((size_t)warp * GP + h) * 132;
+#pragma unroll
+            for (int mt = 0; mt < 8; ++mt) {
+              dst[mt * 16 + g] = o[hn][mt][j];
+              dst[mt * 16 + 8 + g] = o[hn][mt][2 + j];
+            }
+            if (g == 0) { dst[128] = m[hn][j]; dst[129] = lv; }
+          }
         }
-      }
       if (tid == 0) s_redmeta[rb] = item;
       __syncwarp();
       if (lane == 0) mbar_arrive(&red_full[rb]);
@@ -479,7 +499,7 @@ using namespace spkv;
 
 extern "C" size_t spkv_decode_workspace_bytes(const spkv_config_t *cfg, int32_t B) {
   if (!cfg || B < 0 || cfg->n_kv_heads < 1) return 0;
-  return decode_ws_layout(B * cfg->n_kv_heads, cfg->n_q_heads / cfg->n_kv_heads).total;
+  return 2 * decode_ws_layout(B * cfg->n_kv_heads, cfg->n_q_heads / cfg->n_kv_heads).total;
 }
 
 extern "C" int spkv_decode_attention(spkv_cache_t *cache, int32_t layer, const int32_t *d_seq_ids,
@@ -495,7 +515,7 @@ extern "C" int spkv_decode_attention(spkv_cache_t *cache, int32_t layer, const i
   const int n_items = B * v.Hkv;
   if (n_items > 1024) return SPKV_E_UNSUPPORTED;
   const DecodeWs wl = decode_ws_layout(n_items, v.G);
-  if (!d_workspace || ((uintptr_t)d_workspace & 255) || workspace_bytes < wl.total) return SPKV_E_WORKSPACE;
+  if (!d_workspace || ((uintptr_t)d_workspace & 255) || workspace_bytes < 2 * wl.total) return SPKV_E_WORKSPACE;
 
   DecodeArgs a;
   a.c = v; a.layer = layer; a.B = B; a.n_items = n_items; a.G = v.G;
@@ -504,7 +524,14 @@ extern "C" int spkv_decode_attention(spkv_cache_t *cache, int32_t layer, const i
   a.out = static_cast<__nv_bfloat16 *>(d_out);
   a.lse = d_lse_opt;
   a.scale_log2 = sm_scale * kLog2e;
-  char *ws = static_cast<char *>(d_workspace);
+  // Two consecutive decode launches may overlap (the next one starts on the SMs this one
+  // has left): they alternate between the two halves of the workspace.  A third cannot
+  // join: it needs every block of the second resident, i.e. every SM left by the first.
+  char *ws = static_cast<char *>(d_workspace) + (size_t)cache->ws_toggle * wl.total;
+  cache->ws_toggle ^= 1;
+  cache->last_kind = kLastDecode;
+  cache->last_layer = layer;
+  cache->last_stream = as_stream(stream);
   a.counters = reinterpret_cast<int32_t *>(ws);
   a.part_ml = reinterpret_cast<float *>(ws + wl.off_ml);
   a.part_acc = reinterpret_cast<float *>(ws + wl.off_acc);
@@ -525,11 +552,19 @@ extern "C" int spkv_decode_attention(spkv_cache_t *cache, int32_t layer, const i
   TcSmem L = tc_smem_layout(n_items, GP, n_stages, red_bufs);
   while (L.total > limit && n_stages > 2) L = tc_smem_layout(n_items, GP, --n_stages, red_bufs);
   if (L.total > limit) return SPKV_E_UNSUPPORTED;
-  if (cudaFuncSetAttribute(decode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total) !=
-      cudaSuccess)
+  void (*kernel)(DecodeArgs, int, int, int) = GP > 8 ? decode_tc_kernel<2> : decode_tc_kernel<1>;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total) != cudaSuccess)
     return SPKV_E_CUDA;
-  decode_tc_kernel<<<min(kMaxGrid, cache->sm_count), kTcThreads, L.total, s>>>(a, GP, n_stages, red_bufs);
-  return check_stream_error(cudaGetLastError());
+  int grid = min(kMaxGrid, cache->sm_count);
+#ifdef SPKV_PROBE_GRID
+  if (const char *e = getenv("SPKV_DECODE_GRID")) grid = atoi(e);
+#endif
+  if (cache->cfg.flags & SPKV_FLAG_NO_OVERLAP) {
+    kernel<<<grid, kTcThreads, L.total, s>>>(a, GP, n_stages, red_bufs);
+    return check_stream_error(cudaGetLastError());
+  }
+  return check_stream_error(
+      launch_overlapped(kernel, dim3(grid), dim3(kTcThreads), (size_t)L.total, s, a, GP, n_stages, red_bufs));
 }
 
 // ---- decode attention for callers that cannot allocate device memory ---------------------
@@ -565,7 +600,10 @@ extern "C" int spkv_decode_attention_static(spkv_cache_t *cache, int32_t layer, 
   if (B > 0) {
     // the array keeps whatever the previous call left: the arrival counters must start at zero
     const size_t counters = (size_t)B * cache->cfg.n_kv_heads * 4;
-    if (cudaMemsetAsync(scratch, 0, counters, as_stream(stream)) != cudaSuccess) return SPKV_E_CUDA;
+    for (int half = 0; half < 2; ++half)
+      if (cudaMemsetAsync(static_cast<char *>(scratch) + half * (need / 2), 0, counters,
+                          as_stream(stream)) != cudaSuccess)
+        return SPKV_E_CUDA;
   }
   return spkv_decode_attention(cache, layer, d_seq_ids, B, d_q, d_out, d_lse_opt, sm_scale, scratch,
                                SPKV_STATIC_SCRATCH_BYTES, stream);

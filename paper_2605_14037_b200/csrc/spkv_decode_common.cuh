@@ -5,7 +5,7 @@
 
 namespace spkv {
 
-constexpr int kMaxGrid = 1024;
+constexpr int kMaxGrid = 256;   // blocks per decode launch (one per SM; B200 has 148)
 constexpr int kMaxSlots = kMaxGrid;  // one partial slot per (block + item): see the merge
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;

@@ -91,6 +91,31 @@ __device__ inline float warp_dot_bf16(const __nv_bfloat16 *a, const __nv_bfloat1
   return warp_sum(acc);
 }
 
+// ---- programmatic dependent launch ---------------------------------------------------------
+// Kernels launched with launch_overlapped() may begin while the previous kernel of the stream
+// is still running, once all of its blocks have executed pdl_trigger() (or exited).
+// pdl_wait() blocks until that previous kernel has completed and its writes are visible.
+__device__ inline void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ inline void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <class... KArgs, class... Args>
+inline cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                     cudaStream_t stream, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
+enum { kLastOther = 0, kLastAppend = 1, kLastDecode = 2 };
+
 }  // namespace spkv
 
 struct spkv_cache {
@@ -100,6 +125,11 @@ struct spkv_cache {
   void *arena;
   float tau_logit;
   int sm_count;
+  // what the previous launch on this cache was (decides whether an append may overlap it)
+  int last_kind;        // 0 other, 1 append, 2 decode
+  int last_layer;
+  cudaStream_t last_stream;
+  int ws_toggle;        // decode workspace half used by the next decode launch
 };
 
 namespace spkv {

@@ -159,6 +159,128 @@ __device__ inline void softmax_pv_tile(float (&s)[NT / 8][4], Visible visible, f
   }
 }
 
+// ---- "keys as rows" tiles for decode --------------------------------------------------------
+// In decode the query side has only G <= 16 rows (the heads of one group), the key side 64 per
+// page.  Putting the 16 keys of a warp on the M side and the heads on the N side (8 per tile)
+// wastes nothing for G = 8 and half for G = 4, and needs 8 + 16 MMAs per warp and page instead
+// of 16 + 32:
+//   S^T (16 keys x 8 heads)  = K (16 x 128) . Q^T          A = K rows (ldmatrix), B = Q
+//   O^T (128 dims x 8 heads) += V^T (128 x 16) . P^T        A = V (ldmatrix.trans), B = P^T
+// P^T is obtained from the S^T accumulator layout with movmatrix (8x8 transpose in registers).
+// Accumulator layout of a 16 x 8 tile (g = lane >> 2, t = lane & 3):
+//   e=0: (row g, col 2t)  e=1: (row g, col 2t+1)  e=2: (row g+8, col 2t)  e=3: (row g+8, col 2t+1)
+
+__device__ inline uint32_t movmatrix_trans(uint32_t a) {
+  uint32_t d;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
+}
+
+// B fragments of Q^T for head tile hn: qb[hn][kk][0..1].  q_row(h) -> address of head h's 128
+// bf16 (shared or global memory) or nullptr for a padding head.
+template <int NH, class RowPtr>
+__device__ inline void load_q_frags_t(uint32_t (&qb)[NH][8][2], RowPtr q_row, int lane) {
+  const int g = lane >> 2, t = lane & 3;
+#pragma unroll
+  for (int hn = 0; hn < NH; ++hn) {
+    const __nv_bfloat16 *r = q_row(hn * 8 + g);
+#pragma unroll
+    for (int kk = 0; kk < 8; ++kk) {
+      qb[hn][kk][0] = r ? *reinterpret_cast<const uint32_t *>(r + kk * 16 + t * 2) : 0u;
+      qb[hn][kk][1] = r ? *reinterpret_cast<const uint32_t *>(r + kk * 16 + 8 + t * 2) : 0u;
+    }
+  }
+}
+
+// s[hn][.] = scores of keys tok0..tok0+15 (rows) against heads 8hn..8hn+7 (cols), unscaled.
+// Two accumulators per tile (even / odd k-steps) halve the dependent MMA chain.
+template <int NH>
+__device__ inline void qk_tile_t(float (&s)[NH][4], const uint32_t (&qb)[NH][8][2], uint32_t sK, int tok0,
+                                 int lane) {
+  float s2[NH][4];
+#pragma unroll
+  for (int hn = 0; hn < NH; ++hn)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) s[hn][e] = s2[hn][e] = 0.f;
+  const int mi = lane >> 3, ri = lane & 7;
+  const int row = tok0 + (mi & 1) * 8 + ri;
+#pragma unroll
+  for (int kk = 0; kk < 8; ++kk) {
+    uint32_t a[4];
+    ldsm_x4(a, sK + blk_off(row, 2 * kk + (mi >> 1)));
+#pragma unroll
+    for (int hn = 0; hn < NH; ++hn) {
+      if (kk & 1) mma_bf16_16816(s2[hn], a, qb[hn][kk][0], qb[hn][kk][1]);
+      else mma_bf16_16816(s[hn], a, qb[hn][kk][0], qb[hn][kk][1]);
+    }
+  }
+#pragma unroll
+  for (int hn = 0; hn < NH; ++hn)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) s[hn][e] += s2[hn][e];
+}
+
+// Online softmax over the 16 keys of this warp + O^T += V^T P^T.  n_valid: keys tok0.. that are
+// < n_valid (page-local index) are visible.  m, l: per head (2 per thread and head tile: heads
+// 8hn+2t, 8hn+2t+1); l is a per-thread partial (reduce over lanes with equal t at the end).
+// o[hn][mt][e]: dims 16mt + g + 8(e>>1), head 8hn + 2t + (e&1).
+template <int NH>
+__device__ inline void softmax_pv_tile_t(float (&s)[NH][4], int n_valid, float scale_log2, float (&m)[NH][2],
+                                         float (&l)[NH][2], float (&o)[NH][8][4], uint32_t sV, int tok0,
+                                         int lane) {
+  const int g = lane >> 2;
+  const bool vis0 = tok0 + g < n_valid, vis1 = tok0 + g + 8 < n_valid;
+  uint32_t bhi[NH][2], blo[NH][2];
+#pragma unroll
+  for (int hn = 0; hn < NH; ++hn) {
+    float v[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) v[e] = ((e >> 1) ? vis1 : vis0) ? s[hn][e] * scale_log2 : -INFINITY;
+    float corr[2], ms[2];
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      float mx = fmaxf(v[j], v[j + 2]);
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+      const float mn = fmaxf(m[hn][j], mx);
+      ms[j] = mn == -INFINITY ? 0.f : mn;
+      corr[j] = fast_exp2(m[hn][j] - ms[j]);
+      m[hn][j] = mn;
+      l[hn][j] *= corr[j];
+    }
+#pragma unroll
+    for (int mt = 0; mt < 8; ++mt)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) o[hn][mt][e] *= corr[e & 1];
+    float p[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      p[e] = fast_exp2(v[e] - ms[e & 1]);
+      l[hn][e & 1] += p[e];
+    }
+    // P = hi + lo in bf16 (see softmax_pv_tile), transposed into B-fragment layout
+    const __nv_bfloat162 h0 = __floats2bfloat162_rn(p[0], p[1]), h1 = __floats2bfloat162_rn(p[2], p[3]);
+    const float2 f0 = __bfloat1622float2(h0), f1 = __bfloat1622float2(h1);
+    bhi[hn][0] = movmatrix_trans(*reinterpret_cast<const uint32_t *>(&h0));
+    bhi[hn][1] = movmatrix_trans(*reinterpret_cast<const uint32_t *>(&h1));
+    blo[hn][0] = movmatrix_trans(pack_bf16(p[0] - f0.x, p[1] - f0.y));
+    blo[hn][1] = movmatrix_trans(pack_bf16(p[2] - f1.x, p[3] - f1.y));
+  }
+  const int mi = lane >> 3, ri = lane & 7;
+  const int row = tok0 + (mi >> 1) * 8 + ri;
+#pragma unroll
+  for (int mt = 0; mt < 8; ++mt) {
+    uint32_t a[4];
+    ldsm_x4_trans(a, sV + blk_off(row, 2 * mt + (mi & 1)));
+#pragma unroll
+    for (int hn = 0; hn < NH; ++hn) {
+      mma_bf16_16816(o[hn][mt], a, bhi[hn][0], bhi[hn][1]);
+      mma_bf16_16816(o[hn][mt], a, blo[hn][0], blo[hn][1]);
+    }
+  }
+}
+
 // ---- mbarrier + bulk copy (global -> shared, completion counted in bytes) -------------
 
 __device__ inline void mbar_init(uint64_t *bar, uint32_t count) {

@@ -362,6 +362,7 @@ extern "C" int spkv_prefill(spkv_cache_t *cache, int32_t layer, int32_t seq, int
   a.ws = static_cast<int32_t *>(d_workspace);
   a.ws_stride = (int)prefill_ws_stride_ints(C, v.w);
   cudaStream_t s = as_stream(stream);
+  cache->last_kind = kLastOther;
 
   prefill_plan_kernel<<<v.Hkv, 1024, 0, s>>>(a);
   // at most max(min(t0,w) + C - w, 0) <= C pairs leave the window

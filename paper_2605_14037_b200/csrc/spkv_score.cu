@@ -69,6 +69,7 @@ extern "C" int spkv_score(spkv_cache_t *cache, const spkv_predictor_t *p, const 
     return SPKV_E_INVALID;
   const int Hkv = cache->view.Hkv;
   cudaStream_t s = as_stream(stream);
+  cache->last_kind = kLastOther;
   const __nv_bfloat16 *x = static_cast<const __nv_bfloat16 *>(d_x);
   if (p->kind == 0) {
     score_linear_kernel<<<(n_tok + 7) / 8, 256, 0, s>>>(
