@@ -18,20 +18,21 @@
 // bumps the unit's arrival counter; the block that arrives last merges all slots of the
 // unit by their log-sum-exp weights and resets the counter.  Nobody ever waits.
 //
-// Block = 4 consumer warps + producer warp + epilogue warp, one block per SM, a pipeline of
-// whole pages:
+// Block = 8 consumer warps (two groups of four that take alternate pages, so that one group's
+// waits overlap the other's arithmetic) + producer warp + epilogue warp, one block per SM, a
+// pipeline of whole pages:
 //   producer  walks the block's range, resolves each page (unit, page-table entry, valid rows) with its
 //       32 lanes in parallel, then issues one 32 KB linear bulk copy HBM -> shared memory
 //       per page (cp.async.bulk on an mbarrier) plus, at the start of a segment, the
 //       G query rows.  The page in HBM already is the swizzled shared-memory image.
-//   consumers each take 16 of the page's 64 pairs.  The 16 keys are the rows and the group's
+//   consumers each take 16 of the 64 pairs of their group's pages.  The 16 keys are the rows and the group's
 //       G query heads the (8-wide) columns of the tiles, so S^T = K Q^T and O^T += V^T P^T are
 //       small dense products done with mma.sync m16n8k16 (bf16 in, fp32 accumulate): 8 + 16
 //       MMAs per warp and page, operands read with ldmatrix; mask, online softmax (exp2,
 //       shuffles over the keys) in registers.  Each warp keeps (m, l, O) for
 //       its quarter of every page of a segment and drops it into one of two shared-memory
 //       buffers at the segment's end, then carries straight on with the next segment.
-//   epilogue  merges the four warps' results of a finished segment, writes the output (or
+//   epilogue  merges the eight warps' results of a finished segment, writes the output (or
 //       the partial + arrival count + last-arriver merge) while the consumers stream on.
 //
 // Why tensor cores in a bandwidth-bound kernel: per 512 B pair the group needs 2*G*128
@@ -52,13 +53,14 @@
 
 namespace spkv {
 
-constexpr int kTcThreads = 192;  // 4 consumer warps, producer warp, epilogue warp
+constexpr int kConsumerWarps = 8;  // two groups of four: group g takes the pages with k % 2 == g
+constexpr int kTcThreads = (kConsumerWarps + 2) * 32;  // + producer warp + epilogue warp
 constexpr int kMaxStages = 8;
 constexpr int kMergeCap = 256;  // (slot, head) pairs staged in shared memory by a merge
 enum { F_BEGIN = 1, F_END = 2, F_STOP = 4 };
 
-struct StageMeta {
-  int valid, flags, item, pad;
+struct StageMeta {  // valid rows (bits 0-7) | flags (8-11) | item (12+)
+  int packed, pad[3];
 };
 
 struct TcSmem {  // offsets into dynamic shared memory, computed on host and device alike
@@ -81,7 +83,7 @@ __host__ __device__ inline TcSmem tc_smem_layout(int n_items, int GP, int n_stag
   L.off_ring = o;  o += n_items * 4;
   L.off_tmp = o;   o += 64 * 4;
   o = (o + 15) / 16 * 16;
-  L.off_red = o;   o += red_bufs * 4 * GP * 132 * 4;
+  L.off_red = o;   o += red_bufs * kConsumerWarps * GP * 132 * 4;
   L.off_mrg = o;   o += kMergeCap * 8;
   L.off_flags = o; o += 16;
   L.total = o;
@@ -139,15 +141,16 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
   SPKV_STAMP_T(0, tid == 0);
 #ifdef SPKV_PHASE_TIMING
   int dbg_pages = 0, dbg_segs = 0;
+  long long dbg_c[5] = {0, 0, 0, 0, 0};
 #endif
 
   if (tid == 0) {
     for (int i = 0; i < n_stages; ++i) {
       mbar_init(&full[i], 1);
-      mbar_init(&empty[i], 4);
+      mbar_init(&empty[i], kConsumerWarps);
     }
     for (int i = 0; i < 2; ++i) {
-      mbar_init(&red_full[i], 4);
+      mbar_init(&red_full[i], kConsumerWarps);
       mbar_init(&red_empty[i], 1);
     }
     mbar_fence_init();
@@ -191,7 +194,7 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
   const Ranges rg = {VP, max(1, min((int)gridDim.x, VP))};
   SPKV_STAMP_T(1, tid == 0);
 
-  if (warp == 4) {
+  if (warp == kConsumerWarps) {
     // ------------------------------------------------------------------ producer warp
     // Pages are resolved in groups of up to 32 (one per lane) of the block's range.
     // The next group is resolved before the current
@@ -249,8 +252,7 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
           break;
         }
         if (lane == 0) {
-          s_meta[stage].valid = va; s_meta[stage].flags = fl;
-          s_meta[stage].item = it;
+          s_meta[stage].packed = va | (fl << 8) | (it << 12);
           unsigned char *dst = smem + (size_t)stage * L.stage_bytes;
           const uint32_t qbytes = (fl & F_BEGIN) ? (uint32_t)(a.G * kRowBytes) : 0u;
           mbar_arrive_expect_tx(&full[stage], kPageBytes + qbytes);
@@ -267,7 +269,7 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
     if (lane == 0 && !gave_up) {  // tell the consumers that nothing follows
       const int stage = k % n_stages, use = k / n_stages;
       if (use == 0 || wait_or_flag(&empty[stage], (use - 1) & 1, c)) {
-        s_meta[stage].flags = F_STOP;
+        s_meta[stage].packed = F_STOP << 8;
         mbar_arrive(&full[stage]);
       } else {
         gave_up = 1;
@@ -278,7 +280,7 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
       for (int kk = max(0, k - n_stages); kk < k; ++kk)
         mbar_wait_bounded(&full[kk % n_stages], (kk / n_stages) & 1);
     }
-  } else if (warp < 4) {
+  } else if (warp < kConsumerWarps) {
     // ----------------------------------------------------------------- consumer warps
     uint32_t qb[NH][8][2];
     float m[NH][2], l[NH][2], o[NH][8][4];
@@ -286,11 +288,18 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
     int n_seg = 0;
     for (int k = 0;; ++k) {
       const int stage = k % n_stages, use = k / n_stages;
+#ifdef SPKV_PHASE_TIMING
+      const long long c0 = clock64();
+#endif
       if (!wait_or_flag(&full[stage], use & 1, c)) break;
+#ifdef SPKV_PHASE_TIMING
+      const long long c1 = clock64();
+#endif
       SPKV_STAMP_T(3, tid == 0 && k == 0);
-      const int flags = s_meta[stage].flags;
+      const int meta = s_meta[stage].packed;
+      const int flags = (meta >> 8) & 15;
       if (flags & F_STOP) break;
-      const int valid = s_meta[stage].valid, item = s_meta[stage].item;
+      const int valid = meta & 255, item = meta >> 12;
       unsigned char *sbase = smem + (size_t)stage * L.stage_bytes;
       if (flags & F_BEGIN) {
         const __nv_bfloat16 *qs = reinterpret_cast<const __nv_bfloat16 *>(sbase + kPageBytes);
@@ -304,13 +313,23 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
           for (int mt = 0; mt < 8; ++mt) o[hn][mt][0] = o[hn][mt][1] = o[hn][mt][2] = o[hn][mt][3] = 0.f;
         }
       }
-      const int tok0 = warp * 16;
+      const int tok0 = (warp & 3) * 16;
 #ifndef SPKV_PROBE_NOCOMPUTE
-      if (tok0 < valid) {
+      if ((k & 1) == (warp >> 2) && tok0 < valid) {
         const uint32_t sK = smem_u32(sbase), sV = sK + kBlockElems * 2;
         float s[NH][4];
+#ifdef SPKV_PHASE_TIMING
+        const long long c2 = clock64();
+#endif
         qk_tile_t<NH>(s, qb, sK, tok0, lane);
+#ifdef SPKV_PHASE_TIMING
+        const long long c3 = clock64();
+        dbg_c[1] += c2 - c1; dbg_c[2] += c3 - c2;
+#endif
         softmax_pv_tile_t<NH>(s, valid, a.scale_log2, m, l, o, sV, tok0, lane);
+#ifdef SPKV_PHASE_TIMING
+        dbg_c[3] += clock64() - c3;
+#endif
       }
 #else
       if (tok0 < valid) { m[0][0] = 0.f; l[0][0] = 1.f; }
@@ -318,6 +337,7 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty[stage]);
 #ifdef SPKV_PHASE_TIMING
+      dbg_c[0] += c1 - c0; dbg_c[4] += clock64() - c0;
       dbg_pages++;
       if (flags & F_END) dbg_segs++;
 #endif
@@ -327,7 +347,7 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
       const int rb = n_seg & 1, ruse = n_seg >> 1;
       ++n_seg;
       if (ruse > 0 && !wait_or_flag(&red_empty[rb], (ruse - 1) & 1, c)) break;
-      float *red = s_red + (size_t)rb * 4 * GP * 132;
+      float *red = s_red + (size_t)rb * kConsumerWarps * GP * 132;
 #pragma unroll
       for (int hn = 0; hn < NH; ++hn)
 #pragma unroll
@@ -371,7 +391,7 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
       if (!wait_or_flag(&red_full[rb], (e >> 1) & 1, c)) break;
       const int item = s_redmeta[rb];
       if (item < 0) break;
-      const float *red = s_red + (size_t)rb * 4 * GP * 132;
+      const float *red = s_red + (size_t)rb * kConsumerWarps * GP * 132;
       const int b = item / c.Hkv, kvh = item % c.Hkv;
       const int c_first = rg.of_pos(s_pre[item] + 1), c_last = rg.of_pos(s_pre[item + 1] - 1);
       const int nseg = c_last - c_first + 1;
@@ -379,11 +399,11 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
       for (int gh = 0; gh < a.G; ++gh) {
         float M = -INFINITY;
 #pragma unroll
-        for (int w4 = 0; w4 < 4; ++w4) M = fmaxf(M, red[((size_t)w4 * GP + gh) * 132 + 128]);
+        for (int w4 = 0; w4 < kConsumerWarps; ++w4) M = fmaxf(M, red[((size_t)w4 * GP + gh) * 132 + 128]);
         float Ls = 0.f;
         float4 Os = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int w4 = 0; w4 < 4; ++w4) {
+        for (int w4 = 0; w4 < kConsumerWarps; ++w4) {
           const float *src = red + ((size_t)w4 * GP + gh) * 132;
           const float f = src[128] == -INFINITY ? 0.f : fast_exp2(src[128] - M);
           const float4 v = *reinterpret_cast<const float4 *>(src + lane * 4);
@@ -434,27 +454,27 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
           }
           SPKV_STAMP_T(9, lane == 0);
 #ifdef SPKV_PHASE_TIMING
-          if (lane == 0) reinterpret_cast<unsigned long long *>(a.part_acc + (size_t)600 * a.G * kD)[blockIdx.x * 16 + 11] = nseg;
+          if (lane == 0) reinterpret_cast<unsigned long long *>(a.part_acc + (size_t)600 * a.G * kD)[blockIdx.x * 16 + 10] = nseg;
 #endif
           const float2 *g_ml = reinterpret_cast<const float2 *>(a.part_ml) + (size_t)(c_first + item) * a.G;
           const float *g_acc = a.part_acc + (size_t)(c_first + item) * a.G * kD + lane * 4;
           auto ml_of = [&](int si, int gh) { return staged ? s_mrg[si * a.G + gh] : __ldcg(g_ml + si * a.G + gh); };
-          // four heads x eight slots at a time: 32 independent 16-byte loads in flight
-          for (int gh0 = 0; gh0 < a.G; gh0 += 4) {
-            float Mx[4], Ls[4];
-            float4 Os[4];
+          // two heads x eight slots at a time: 16 independent 16-byte loads in flight
+          for (int gh0 = 0; gh0 < a.G; gh0 += 2) {
+            float Mx[2], Ls[2];
+            float4 Os[2];
 #pragma unroll
-            for (int h = 0; h < 4; ++h) {
+            for (int h = 0; h < 2; ++h) {
               Mx[h] = -INFINITY; Ls[h] = 0.f; Os[h] = make_float4(0.f, 0.f, 0.f, 0.f);
               if (gh0 + h < a.G)
                 for (int si = 0; si < nseg; ++si) Mx[h] = fmaxf(Mx[h], ml_of(si, gh0 + h).x);
             }
             for (int s0 = 0; s0 < nseg; s0 += 8) {
-              float4 v[8][4];
+              float4 v[8][2];
 #pragma unroll
               for (int x = 0; x < 8; ++x)
 #pragma unroll
-                for (int h = 0; h < 4; ++h)
+                for (int h = 0; h < 2; ++h)
                   v[x][h] = (s0 + x < nseg && gh0 + h < a.G)
                                 ? __ldcg(reinterpret_cast<const float4 *>(
                                       g_acc + ((size_t)(s0 + x) * a.G + gh0 + h) * kD))
@@ -462,7 +482,7 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
 #pragma unroll
               for (int x = 0; x < 8; ++x)
 #pragma unroll
-                for (int h = 0; h < 4; ++h)
+                for (int h = 0; h < 2; ++h)
                   if (s0 + x < nseg && gh0 + h < a.G) {
                     const float2 ml = ml_of(s0 + x, gh0 + h);
                     const float f = fast_exp2(ml.x - Mx[h]);
@@ -472,7 +492,7 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
                   }
             }
 #pragma unroll
-            for (int h = 0; h < 4; ++h)
+            for (int h = 0; h < 2; ++h)
               if (gh0 + h < a.G) {
                 const size_t row = (size_t)b * c.Hq + kvh * a.G + gh0 + h;
                 const float inv = 1.f / Ls[h];
@@ -489,6 +509,12 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
     }
   }
   SPKV_STAMP_T(4, tid == 0);
+#ifdef SPKV_PHASE_TIMING
+  if (tid == 0) {
+    unsigned long long *dbg = reinterpret_cast<unsigned long long *>(a.part_acc + (size_t)600 * a.G * kD);
+    for (int i = 0; i < 5; ++i) dbg[blockIdx.x * 16 + 11 + i] = dbg_pages ? dbg_c[i] / dbg_pages : 0;
+  }
+#endif
   __syncthreads();
   SPKV_STAMP_T(5, tid == 0);
 }

@@ -193,15 +193,19 @@ __device__ inline void load_q_frags_t(uint32_t (&qb)[NH][8][2], RowPtr q_row, in
 }
 
 // s[hn][.] = scores of keys tok0..tok0+15 (rows) against heads 8hn..8hn+7 (cols), unscaled.
-// Two accumulators per tile (even / odd k-steps) halve the dependent MMA chain.
+// mma.sync results come back after a long pipeline, and a warp issues in order: a chain of MMAs
+// on one accumulator stalls for that latency at every link.  The eight k-steps therefore go to
+// four accumulators (chains of two) that are summed at the end.
 template <int NH>
 __device__ inline void qk_tile_t(float (&s)[NH][4], const uint32_t (&qb)[NH][8][2], uint32_t sK, int tok0,
                                  int lane) {
-  float s2[NH][4];
+  float acc[4][NH][4];
 #pragma unroll
-  for (int hn = 0; hn < NH; ++hn)
+  for (int c4 = 0; c4 < 4; ++c4)
 #pragma unroll
-    for (int e = 0; e < 4; ++e) s[hn][e] = s2[hn][e] = 0.f;
+    for (int hn = 0; hn < NH; ++hn)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc[c4][hn][e] = 0.f;
   const int mi = lane >> 3, ri = lane & 7;
   const int row = tok0 + (mi & 1) * 8 + ri;
 #pragma unroll
@@ -209,15 +213,13 @@ __device__ inline void qk_tile_t(float (&s)[NH][4], const uint32_t (&qb)[NH][8][
     uint32_t a[4];
     ldsm_x4(a, sK + blk_off(row, 2 * kk + (mi >> 1)));
 #pragma unroll
-    for (int hn = 0; hn < NH; ++hn) {
-      if (kk & 1) mma_bf16_16816(s2[hn], a, qb[hn][kk][0], qb[hn][kk][1]);
-      else mma_bf16_16816(s[hn], a, qb[hn][kk][0], qb[hn][kk][1]);
-    }
+    for (int hn = 0; hn < NH; ++hn) mma_bf16_16816(acc[kk & 3][hn], a, qb[hn][kk][0], qb[hn][kk][1]);
   }
 #pragma unroll
   for (int hn = 0; hn < NH; ++hn)
 #pragma unroll
-    for (int e = 0; e < 4; ++e) s[hn][e] += s2[hn][e];
+    for (int e = 0; e < 4; ++e)
+      s[hn][e] = (acc[0][hn][e] + acc[1][hn][e]) + (acc[2][hn][e] + acc[3][hn][e]);
 }
 
 // Online softmax over the 16 keys of this warp + O^T += V^T P^T.  n_valid: keys tok0.. that are
@@ -267,18 +269,20 @@ __device__ inline void softmax_pv_tile_t(float (&s)[NH][4], int n_valid, float s
     blo[hn][0] = movmatrix_trans(pack_bf16(p[0] - f0.x, p[1] - f0.y));
     blo[hn][1] = movmatrix_trans(pack_bf16(p[2] - f1.x, p[3] - f1.y));
   }
+  // all "hi" products first, then all "lo" products: no MMA waits for its predecessor
   const int mi = lane >> 3, ri = lane & 7;
   const int row = tok0 + (mi >> 1) * 8 + ri;
+  uint32_t a[8][4];
 #pragma unroll
   for (int mt = 0; mt < 8; ++mt) {
-    uint32_t a[4];
-    ldsm_x4_trans(a, sV + blk_off(row, 2 * mt + (mi & 1)));
+    ldsm_x4_trans(a[mt], sV + blk_off(row, 2 * mt + (mi & 1)));
 #pragma unroll
-    for (int hn = 0; hn < NH; ++hn) {
-      mma_bf16_16816(o[hn][mt], a, bhi[hn][0], bhi[hn][1]);
-      mma_bf16_16816(o[hn][mt], a, blo[hn][0], blo[hn][1]);
-    }
+    for (int hn = 0; hn < NH; ++hn) mma_bf16_16816(o[hn][mt], a[mt], bhi[hn][0], bhi[hn][1]);
   }
+#pragma unroll
+  for (int mt = 0; mt < 8; ++mt)
+#pragma unroll
+    for (int hn = 0; hn < NH; ++hn) mma_bf16_16816(o[hn][mt], a[mt], blo[hn][0], blo[hn][1]);
 }
 
 // ---- mbarrier + bulk copy (global -> shared, completion counted in bytes) -------------
