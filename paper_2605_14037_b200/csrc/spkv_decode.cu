@@ -104,7 +104,7 @@ __device__ inline unsigned long long gtimer() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-#define SPKV_STAMP_T(i, cond) do { if (cond) reinterpret_cast<unsigned long long *>(a.part_acc + (size_t)600 * a.G * kD)[blockIdx.x * 16 + (i)] = gtimer(); } while (0)
+#define SPKV_STAMP_T(i, cond) do { if (cond) reinterpret_cast<unsigned long long *>(a.part_acc + (size_t)300 * a.G * kD)[blockIdx.x * 16 + (i)] = gtimer(); } while (0)
 #else
 #define SPKV_STAMP_T(i, cond)
 #endif
@@ -454,7 +454,7 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
           }
           SPKV_STAMP_T(9, lane == 0);
 #ifdef SPKV_PHASE_TIMING
-          if (lane == 0) reinterpret_cast<unsigned long long *>(a.part_acc + (size_t)600 * a.G * kD)[blockIdx.x * 16 + 10] = nseg;
+          if (lane == 0) reinterpret_cast<unsigned long long *>(a.part_acc + (size_t)300 * a.G * kD)[blockIdx.x * 16 + 10] = nseg;
 #endif
           const float2 *g_ml = reinterpret_cast<const float2 *>(a.part_ml) + (size_t)(c_first + item) * a.G;
           const float *g_acc = a.part_acc + (size_t)(c_first + item) * a.G * kD + lane * 4;
@@ -511,7 +511,7 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
   SPKV_STAMP_T(4, tid == 0);
 #ifdef SPKV_PHASE_TIMING
   if (tid == 0) {
-    unsigned long long *dbg = reinterpret_cast<unsigned long long *>(a.part_acc + (size_t)600 * a.G * kD);
+    unsigned long long *dbg = reinterpret_cast<unsigned long long *>(a.part_acc + (size_t)300 * a.G * kD);
     for (int i = 0; i < 5; ++i) dbg[blockIdx.x * 16 + 11 + i] = dbg_pages ? dbg_c[i] / dbg_pages : 0;
   }
 #endif
