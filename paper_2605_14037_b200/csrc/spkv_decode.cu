@@ -90,12 +90,33 @@ __host__ __device__ inline TcSmem tc_smem_layout(int n_items, int GP, int n_stag
   return L;
 }
 
-// Equal cut of the axis of VP positions into nb ranges (exact integer arithmetic: every block
-// must compute identical boundaries).
+// Cut of the axis of VP positions into nb ranges: equal lengths (exact integer arithmetic,
+// every block must compute identical boundaries), except that a cut that falls within
+// `snap` positions of a unit boundary moves onto it -- the unit is then not split, which saves
+// two partial results and a merge at the price of a few pages of imbalance.
 struct Ranges {
-  int VP, nb;
-  __device__ int start(int c) const { return (int)(((long long)c * VP) / nb); }
-  __device__ int of_pos(int p) const { return (int)((((long long)p + 1) * nb - 1) / VP); }
+  int VP, nb, snap, n;
+  const int *pre;  // prefix sums of the unit lengths (shared memory), pre[n] = VP
+  __device__ int ideal(int c) const { return (int)(((long long)c * VP) / nb); }
+  __device__ int start(int c) const {
+    if (c <= 0) return 0;
+    if (c >= nb) return VP;
+    const int p = ideal(c);
+    int lo = 0, hi = n;  // unit containing position p
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (pre[mid] <= p) lo = mid; else hi = mid;
+    }
+    if (p - pre[lo] <= snap) return pre[lo];
+    if (pre[lo + 1] - p <= snap) return pre[lo + 1];
+    return p;
+  }
+  __device__ int of_pos(int p) const {  // block whose range holds position p
+    int c = (int)((((long long)p + 1) * nb - 1) / VP);
+    while (c > 0 && start(c) > p) --c;
+    while (c + 1 < nb && start(c + 1) <= p) ++c;
+    return c;
+  }
 };
 
 #ifdef SPKV_PHASE_TIMING
@@ -191,7 +212,10 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
   __syncthreads();
   block_exclusive_scan(s_np, s_pre, n, s_tmp);
   const int VP = s_pre[n];
-  const Ranges rg = {VP, max(1, min((int)gridDim.x, VP))};
+  // at least four positions per block (tiny calls would otherwise be cut into single pages
+  // and spend their time merging); snapping distance: a.snap positions, less for short ranges
+  const int nb_eff = max(1, min((int)gridDim.x, (VP + 3) / 4));
+  const Ranges rg = {VP, nb_eff, min(a.snap, VP / nb_eff / 4), n, s_pre};
   SPKV_STAMP_T(1, tid == 0);
 
   if (warp == kConsumerWarps) {
@@ -550,6 +574,11 @@ extern "C" int spkv_decode_attention(spkv_cache_t *cache, int32_t layer, const i
   a.out = static_cast<__nv_bfloat16 *>(d_out);
   a.lse = d_lse_opt;
   a.scale_log2 = sm_scale * kLog2e;
+  static const int snap_env = [] {
+    const char *e = getenv("SPKV_DECODE_SNAP");  // tuning knob: snapping distance of the range cuts
+    return e ? atoi(e) : 6;
+  }();
+  a.snap = snap_env;
   // Two consecutive decode launches may overlap (the next one starts on the SMs this one
   // has left): they alternate between the two halves of the workspace.  A third cannot
   // join: it needs every block of the second resident, i.e. every SM left by the first.

@@ -18,6 +18,7 @@ struct DecodeArgs {
   __nv_bfloat16 *out;      // [B][Hq][128]
   float *lse;              // [B][Hq] or null
   float scale_log2;        // sm_scale * log2(e)
+  int snap;                // range cuts within this many positions of a unit boundary move onto it
   int32_t *counters;       // [n_items] arrival counters
   float *part_ml;          // [slots][G][2]
   float *part_acc;         // [slots][G][128]
