@@ -65,7 +65,7 @@ struct StageMeta {  // valid rows (bits 0-7) | flags (8-11) | item (12+)
 
 struct TcSmem {  // offsets into dynamic shared memory, computed on host and device alike
   int n_stages, red_bufs, stage_bytes, off_bar, off_meta, off_np, off_pre, off_unit, off_len, off_ring,
-      off_tmp, off_red, off_mrg, off_flags, total;
+      off_tmp, off_cut, off_red, off_mrg, off_flags, total;
 };
 __host__ __device__ inline TcSmem tc_smem_layout(int n_items, int GP, int n_stages, int red_bufs) {
   TcSmem L;
@@ -82,6 +82,7 @@ __host__ __device__ inline TcSmem tc_smem_layout(int n_items, int GP, int n_stag
   L.off_len = o;   o += n_items * 4;
   L.off_ring = o;  o += n_items * 4;
   L.off_tmp = o;   o += 64 * 4;
+  L.off_cut = o;   o += (kMaxGrid + 1) * 4;
   o = (o + 15) / 16 * 16;
   L.off_red = o;   o += red_bufs * kConsumerWarps * GP * 132 * 4;
   L.off_mrg = o;   o += kMergeCap * 8;
@@ -91,31 +92,34 @@ __host__ __device__ inline TcSmem tc_smem_layout(int n_items, int GP, int n_stag
 }
 
 // Cut of the axis of VP positions into nb ranges: equal lengths (exact integer arithmetic,
-// every block must compute identical boundaries), except that a cut that falls within
-// `snap` positions of a unit boundary moves onto it -- the unit is then not split, which saves
-// two partial results and a merge at the price of a few pages of imbalance.
+// every block computes identical boundaries), except that a cut that falls within `snap`
+// positions of a unit boundary moves onto it -- the unit is then not split, which saves two
+// partial results and a merge at the price of a few pages of imbalance.  The nb + 1 cuts are
+// computed once per block, in parallel, into shared memory.
+__device__ inline int range_cut(int c, int nb, int VP, int snap, const int *pre, int n) {
+  if (c <= 0) return 0;
+  if (c >= nb) return VP;
+  const int p = (int)(((unsigned long long)(unsigned)c * (unsigned)VP) / (unsigned)nb);
+  int lo = 0, hi = n;  // unit containing position p
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (pre[mid] <= p) lo = mid; else hi = mid;
+  }
+  if (p - pre[lo] <= snap) return pre[lo];
+  if (pre[lo + 1] - p <= snap) return pre[lo + 1];
+  return p;
+}
 struct Ranges {
-  int VP, nb, snap, n;
-  const int *pre;  // prefix sums of the unit lengths (shared memory), pre[n] = VP
-  __device__ int ideal(int c) const { return (int)(((long long)c * VP) / nb); }
-  __device__ int start(int c) const {
-    if (c <= 0) return 0;
-    if (c >= nb) return VP;
-    const int p = ideal(c);
-    int lo = 0, hi = n;  // unit containing position p
+  int nb;
+  const int *cut;  // [nb + 1], non-decreasing, cut[0] = 0, cut[nb] = VP
+  __device__ int start(int c) const { return cut[min(c, nb)]; }
+  __device__ int of_pos(int p) const {  // last block c with cut[c] <= p (its range is non-empty)
+    int lo = 0, hi = nb;
     while (hi - lo > 1) {
       const int mid = (lo + hi) >> 1;
-      if (pre[mid] <= p) lo = mid; else hi = mid;
+      if (cut[mid] <= p) lo = mid; else hi = mid;
     }
-    if (p - pre[lo] <= snap) return pre[lo];
-    if (pre[lo + 1] - p <= snap) return pre[lo + 1];
-    return p;
-  }
-  __device__ int of_pos(int p) const {  // block whose range holds position p
-    int c = (int)((((long long)p + 1) * nb - 1) / VP);
-    while (c > 0 && start(c) > p) --c;
-    while (c + 1 < nb && start(c + 1) <= p) ++c;
-    return c;
+    return lo;
   }
 };
 
@@ -153,6 +157,7 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
   int *s_len = reinterpret_cast<int *>(smem + L.off_len);
   int *s_ring = reinterpret_cast<int *>(smem + L.off_ring);
   int *s_tmp = reinterpret_cast<int *>(smem + L.off_tmp);
+  int *s_cut = reinterpret_cast<int *>(smem + L.off_cut);
   float *s_red = reinterpret_cast<float *>(smem + L.off_red);
   uint64_t *red_full = empty + kMaxStages, *red_empty = red_full + 2;
   float2 *s_mrg = reinterpret_cast<float2 *>(smem + L.off_mrg);
@@ -215,7 +220,10 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
   // at least four positions per block (tiny calls would otherwise be cut into single pages
   // and spend their time merging); snapping distance: a.snap positions, less for short ranges
   const int nb_eff = max(1, min((int)gridDim.x, (VP + 3) / 4));
-  const Ranges rg = {VP, nb_eff, min(a.snap, VP / nb_eff / 4), n, s_pre};
+  for (int cc = tid; cc <= nb_eff; cc += kTcThreads)
+    s_cut[cc] = range_cut(cc, nb_eff, VP, min(a.snap, VP / nb_eff / 4), s_pre, n);
+  __syncthreads();
+  const Ranges rg = {nb_eff, s_cut};
   SPKV_STAMP_T(1, tid == 0);
 
   if (warp == kConsumerWarps) {
@@ -415,11 +423,20 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
       if (!wait_or_flag(&red_full[rb], (e >> 1) & 1, c)) break;
       const int item = s_redmeta[rb];
       if (item < 0) break;
+#ifdef SPKV_PHASE_TIMING
+      const long long ec0 = clock64();
+#endif
       const float *red = s_red + (size_t)rb * kConsumerWarps * GP * 132;
       const int b = item / c.Hkv, kvh = item % c.Hkv;
-      const int c_first = rg.of_pos(s_pre[item] + 1), c_last = rg.of_pos(s_pre[item + 1] - 1);
+      // blocks that share the unit (searched only when it sticks out of this block's range)
+      const int u_first = s_pre[item] + 1, u_last = s_pre[item + 1] - 1;
+      const int c_first = u_first >= rg.start(cidx) ? cidx : rg.of_pos(u_first);
+      const int c_last = u_last < rg.start(cidx + 1) ? cidx : rg.of_pos(u_last);
       const int nseg = c_last - c_first + 1;
       const int slot = cidx + item;
+#ifdef SPKV_PHASE_TIMING
+      const long long ec1 = clock64();
+#endif
       for (int gh = 0; gh < a.G; ++gh) {
         float M = -INFINITY;
 #pragma unroll
@@ -452,8 +469,15 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(&red_empty[rb]);
+#ifdef SPKV_PHASE_TIMING
+      if (lane == 0) {
+        unsigned long long *dbg = reinterpret_cast<unsigned long long *>(a.part_acc + (size_t)300 * a.G * kD);
+        dbg[blockIdx.x * 16 + 6] += clock64() - ec0;
+        dbg[blockIdx.x * 16 + 7] += 1;
+        dbg[blockIdx.x * 16 + 2] += ec1 - ec0;
+      }
+#endif
       if (nseg > 1) {
-        SPKV_STAMP_T(2, lane == 0);
         __threadfence();
         __syncwarp();
         int last = 0;
@@ -462,8 +486,6 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
           if (last) a.counters[item] = 0;
         }
         last = __shfl_sync(0xffffffffu, last, 0);
-        SPKV_STAMP_T(6, lane == 0);
-        SPKV_STAMP_T(7, lane == 0 && last);
         if (last) {
           __threadfence();
           SPKV_STAMP_T(8, lane == 0);
