@@ -11,10 +11,12 @@
 //   pages       : ring pages of every unit ([n_units][ring_pages]) followed by the pool
 //
 // A page holds P = 64 pairs: a 16 KB key block followed by a 16 KB value block.  Each
-// block is 64 rows of 256 B (one row per pair, 128 bf16).  Inside a row the sixteen
-// 16-byte chunks are stored XOR-swizzled by the row number, chunk' = chunk ^ (row & 7):
-// the page in HBM is exactly the shared-memory image the attention kernels want, so one
-// linear bulk copy brings it in and `ldmatrix` reads it without bank conflicts.
+// block is two 8 KB slabs (dims 0-63, dims 64-127) of 64 rows x 128 B, one row per pair;
+// inside a row the eight 16-byte chunks are XOR-swizzled by the row number,
+// chunk' = chunk ^ (row & 7) -- the 128-byte-swizzle operand layout of the tensor cores.
+// The page in HBM is exactly the shared-memory image the attention kernels want: one
+// linear bulk copy brings it in, `ldmatrix` reads it without bank conflicts, and
+// tcgen05.mma can take a slab as a K-major (keys) or MN-major (values) operand as it is.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -51,7 +53,7 @@ struct Layout {
 
 // element offset of (row, 16-byte chunk) inside a key or value block
 __host__ __device__ inline int swz_off(int row, int chunk) {
-  return row * kD + ((chunk ^ (row & 7)) << 3);
+  return (chunk >> 3) * (kP * 64) + row * 64 + (((chunk & 7) ^ (row & 7)) << 3);
 }
 
 __device__ inline int unit_index(const CacheView &c, int layer, int seq, int kvh) {

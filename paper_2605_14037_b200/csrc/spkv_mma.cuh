@@ -2,10 +2,10 @@
 // (mma.sync m16n8k16, operands fetched with ldmatrix from swizzled shared memory),
 // the online-softmax update, and the mbarrier / bulk-copy primitives of the page pipeline.
 //
-// Shared-memory image of a key or value block (identical to its image in HBM):
-// 64 rows of 256 B, 16-byte chunk c of row r stored at chunk position c ^ (r & 7).
-// Eight consecutive rows at a fixed logical chunk therefore hit eight different
-// 16-byte bank groups: every ldmatrix phase is conflict-free.
+// Shared-memory image of a key or value block (identical to its image in HBM): two slabs
+// (dims 0-63 | 64-127) of 64 rows x 128 B; 16-byte chunk c (0-7) of a slab row r is stored at
+// chunk position c ^ (r & 7).  Eight consecutive rows at a fixed logical chunk therefore hit
+// eight different 16-byte bank groups: every ldmatrix phase is conflict-free.
 //
 // Fragment conventions (g = lane >> 2, t = lane & 3), m16n8k16, A row-major, B col-major:
 //   A: a0 (row g,   k 2t..2t+1)  a1 (row g+8, k 2t..2t+1)  a2 (row g, k 2t+8..)  a3 (row g+8, k 2t+8..)
@@ -48,7 +48,7 @@ __device__ inline float fast_exp2(float x) {
 
 // Byte offset of (row, logical 16-byte chunk) inside a swizzled key/value block.
 __device__ inline uint32_t blk_off(int row, int chunk) {
-  return (uint32_t)(row * 256 + ((chunk ^ (row & 7)) << 4));
+  return (uint32_t)((chunk >> 3) * 8192 + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
 }
 
 // Loads the A fragments of a 16 x 128 query tile straight from global memory.

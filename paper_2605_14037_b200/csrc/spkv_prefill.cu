@@ -130,8 +130,8 @@ __global__ void __launch_bounds__(1024) prefill_plan_kernel(PrefillArgs a) {
 
 // Source row of staging pair j: old ring slot (swizzled page) or chunk input (linear).
 struct SrcRow {
-  const __nv_bfloat16 *k, *v;
-  int row;  // >= 0: swizzled with this row; -1: linear
+  const __nv_bfloat16 *k, *v;  // row >= 0: base of the key / value block; row < 0: the row itself
+  int row;                     // >= 0: row of a swizzled block; -1: linear row
 };
 __device__ inline SrcRow staging_row(const PrefillArgs &a, int u, int kvh, int t0, int n_old, int j) {
   SrcRow r;
@@ -139,8 +139,8 @@ __device__ inline SrcRow staging_row(const PrefillArgs &a, int u, int kvh, int t
     const int slot = (t0 - n_old + j) % a.c.w;
     const __nv_bfloat16 *pg = a.c.pages + ring_page(a.c, u, slot / kP) * kPageElems;
     r.row = slot % kP;
-    r.k = pg + r.row * kD;
-    r.v = pg + kBlockElems + r.row * kD;
+    r.k = pg;
+    r.v = pg + kBlockElems;
   } else {
     const size_t off = ((size_t)(j - n_old) * a.c.Hkv + kvh) * kD;
     r.row = -1;
@@ -150,8 +150,7 @@ __device__ inline SrcRow staging_row(const PrefillArgs &a, int u, int kvh, int t
   return r;
 }
 __device__ inline uint4 load_chunk(const __nv_bfloat16 *rowbase, int row, int chunk) {
-  const int cc = row >= 0 ? (chunk ^ (row & 7)) : chunk;
-  return *reinterpret_cast<const uint4 *>(rowbase + cc * 8);
+  return *reinterpret_cast<const uint4 *>(rowbase + (row >= 0 ? swz_off(row, chunk) : chunk * 8));
 }
 
 // ------------------------------------------------------------------ B: scatter (compact)
@@ -260,8 +259,7 @@ __global__ void __launch_bounds__(128) prefill_attn_kernel(PrefillArgs a) {
         if (s <= s_hi) {
           const SrcRow sr = staging_row(a, u, kvh, t0, n_old, s - p0);
           const __nv_bfloat16 *rowp = isv ? sr.v : sr.k;
-          const int cc = sr.row >= 0 ? (chunk ^ (sr.row & 7)) : chunk;
-          cp_async16(d, rowp + cc * 8);
+          cp_async16(d, rowp + (sr.row >= 0 ? swz_off(sr.row, chunk) : chunk * 8));
         } else {
           *reinterpret_cast<uint4 *>(dst + isv * (kBlockElems * 2) + blk_off(r, chunk)) = make_uint4(0, 0, 0, 0);
         }
