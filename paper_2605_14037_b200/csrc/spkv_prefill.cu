@@ -23,26 +23,12 @@
 //              are advanced.
 //
 // Workspace per KV head: a 64-int header followed by E[0..N] (int32).
-#include "spkv_internal.cuh"
+#include <stdlib.h>
+
+#include "spkv_prefill_common.cuh"
 #include "spkv_mma.cuh"
 
 namespace spkv {
-
-constexpr int kHdrInts = 64;
-enum { H_T0 = 0, H_LEN0, H_NOLD, H_N, H_NCOMMIT, H_LEN1, H_FAIL };
-
-struct PrefillArgs {
-  CacheView c;
-  int layer, seq, C;
-  const __nv_bfloat16 *q, *k, *v;  // [C][Hq][128], [C][Hkv][128]
-  const float *logits;             // [C][Hkv]
-  __nv_bfloat16 *out;              // [C][Hq][128]
-  float tau_logit, scale_log2;
-  int32_t *ws;                     // [Hkv][ws_stride]
-  int ws_stride;
-};
-
-__device__ inline int32_t *unit_ws(const PrefillArgs &a, int kvh) { return a.ws + (size_t)kvh * a.ws_stride; }
 
 // ---------------------------------------------------------------- A: plan (flags + scan)
 __global__ void __launch_bounds__(1024) prefill_plan_kernel(PrefillArgs a) {
@@ -330,9 +316,16 @@ static size_t prefill_ws_stride_ints(int C, int w) {
 
 using namespace spkv;
 
+static size_t prefill_plan_bytes(const spkv_config_t *cfg, int C) {
+  size_t b = prefill_ws_stride_ints(C, cfg->window) * 4 * (size_t)cfg->n_kv_heads;
+  return (b + 1023) / 1024 * 1024;
+}
+static int prefill_stage_pages(const spkv_config_t *cfg, int C) { return (C + cfg->window + kP - 1) / kP; }
+
 extern "C" size_t spkv_prefill_workspace_bytes(const spkv_config_t *cfg, int32_t C) {
   if (!cfg || C < 0) return 0;
-  return prefill_ws_stride_ints(C, cfg->window) * 4 * (size_t)cfg->n_kv_heads;
+  // plan (header + prefix sums per KV head), then the staging pages of the chunk attention
+  return prefill_plan_bytes(cfg, C) + (size_t)cfg->n_kv_heads * prefill_stage_pages(cfg, C) * kPageBytes;
 }
 
 extern "C" int spkv_prefill(spkv_cache_t *cache, int32_t layer, int32_t seq, int32_t C,
@@ -359,13 +352,23 @@ extern "C" int spkv_prefill(spkv_cache_t *cache, int32_t layer, int32_t seq, int
   a.scale_log2 = sm_scale * 1.4426950408889634f;
   a.ws = static_cast<int32_t *>(d_workspace);
   a.ws_stride = (int)prefill_ws_stride_ints(C, v.w);
+  a.stage_pages = reinterpret_cast<__nv_bfloat16 *>(static_cast<char *>(d_workspace) +
+                                                    prefill_plan_bytes(&cache->cfg, C));
+  a.n_stage_pages = prefill_stage_pages(&cache->cfg, C);
   cudaStream_t s = as_stream(stream);
   cache->last_kind = kLastOther;
 
   prefill_plan_kernel<<<v.Hkv, 1024, 0, s>>>(a);
   // at most max(min(t0,w) + C - w, 0) <= C pairs leave the window
   prefill_scatter_kernel<<<dim3((C + 63) / 64, v.Hkv), 256, 0, s>>>(a);
-  if (d_q) {
+  static const bool use_mma_sync = [] {
+    const char *e = getenv("SPKV_PREFILL_KERNEL");  // "mma": the mma.sync comparison kernel
+    return e && e[0] == 'm';
+  }();
+  if (d_q && !use_mma_sync) {
+    int rc = launch_prefill_attn_tc5(a, s);
+    if (rc) return rc;
+  } else if (d_q) {
     if (cudaFuncSetAttribute(prefill_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              kAttnSmem) != cudaSuccess)
       return SPKV_E_CUDA;
