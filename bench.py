@@ -34,6 +34,8 @@ CONFIGS = {
     1: dict(name="config1_1layer_b1_ctx4k", L=1, B=1, Hq=8, Hkv=2, T=4096, beta=None, rate=0.2),
     2: dict(name="config2_llama8b_b16_ctx32k", L=32, B=16, Hq=32, Hkv=8, T=32768, beta=(0.5, 2.0)),
     3: dict(name="config3_llama8b_b4_ctx128k", L=32, B=4, Hq=32, Hkv=8, T=131072, beta=(0.3, 3.0)),
+    4: dict(name="config4_ragged_b64_prefill8_decode56", L=32, B=64, Hq=32, Hkv=8, T=65536, beta=(0.5, 2.0),
+            t_min=4096, n_prefill=8, chunk=8192),
     5: dict(name="config5_llama70b_b8_ctx64k", L=80, B=8, Hq=64, Hkv=8, T=65536, beta=(0.5, 2.5)),
 }
 W, D_IN, TAU, CHUNK = 128, 512, 0.5, 8192
@@ -124,9 +126,15 @@ def build_workload(spkv, synth, torch, cfg, dev, dense, total_steps, seed=0):
     else:
         rates = synth.keep_rates(rng, L, Hkv, *cfg["beta"])
     eff = np.ones_like(rates) if dense else rates
-    t_final = T + total_steps
+    t_list = cfg.get("t_list")          # per-sequence contexts (ragged batch), else uniform T
+    grow = cfg.get("grow", total_steps)  # pairs every sequence may still receive
+    t_final = T + grow
     pages_per_unit = np.ceil(eff * (t_final - W) * 1.03 / 64).astype(np.int64) + 2
     pool_pages = int(pages_per_unit.sum() * B)
+    if t_list is not None:
+        g_list = np.asarray(cfg.get("grow_list", [grow] * B))
+        per_seq = np.ceil(eff[:, None, :] * (np.asarray(t_list) + g_list)[None, :, None] * 1.03 / 64) + 2
+        pool_pages = int(per_seq.sum())
     cache = spkv.Cache(n_layers=L, max_seqs=B, n_q_heads=Hq, n_kv_heads=Hkv,
                        max_context=t_final + 64, pool_pages=pool_pages, window=W, tau=tau, device=dev)
     tl = 0.0  # logit-space threshold of tau = 0.5 (the dense run ignores it)
@@ -144,9 +152,9 @@ def build_workload(spkv, synth, torch, cfg, dev, dense, total_steps, seed=0):
                .to(torch.bfloat16) for _ in range(4)]
     for l in range(L):
         for b in range(B):
-            done = 0
-            while done < T:
-                c = min(CHUNK, T - done)
+            done, T_b = 0, (T if t_list is None else int(t_list[b]))
+            while done < T_b:
+                c = min(CHUNK, T_b - done)
                 x = torch.randn((c, D_IN), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
                 lg = cache.spkv_score(preds[l], x)
                 k, v = kv_pool[(l + b + done // CHUNK) % 4][:c], kv_pool[(l + b + 1 + done // CHUNK) % 4][:c]
@@ -373,6 +381,106 @@ def run_ours(args):
     print(json.dumps(line))
 
 
+def run_config4(args):
+    """Ragged serving batch: every step 8 sequences run an 8192-pair prefill chunk (score,
+    compaction, tensor-core chunk attention) while 56 sequences decode one token each."""
+    import numpy as np
+    import torch
+
+    from paper_2605_14037_b200 import build as spkv_build
+    spkv_build.build()
+    from paper_2605_14037_b200 import spkv, synth
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    cfg = dict(CONFIGS[4])
+    if args.layers > 0:
+        cfg["L"] = args.layers
+        cfg["name"] += f"_{args.layers}layers_only"
+    L, B, Hq, Hkv, C, NP = cfg["L"], cfg["B"], cfg["Hq"], cfg["Hkv"], cfg["chunk"], cfg["n_prefill"]
+    K, Wm = max(1, min(args.steps, 8)), 3
+    rng = np.random.default_rng(4)
+    cfg["t_list"] = rng.integers(cfg["t_min"], cfg["T"] + 1, size=B)
+    cfg["grow"] = (K + Wm) * C + 64
+    cfg["grow_list"] = [cfg["grow"] if b < NP else K + Wm + 64 for b in range(B)]
+    cache, preds, rates, gen = build_workload(spkv, synth, torch, cfg, dev, False, 0)
+    hbm_peak, peak_kind = peaks()
+    dec_ids = torch.arange(NP, B, dtype=torch.int32, device=dev)          # sequences 8..63 decode
+    nd = B - NP
+    rnd = lambda *shape: torch.randn(shape, generator=gen, device=dev).to(torch.bfloat16)
+    xq, qd, kd, vd = rnd(L, nd, D_IN), rnd(L, nd, Hq, 128), rnd(L, nd, Hkv, 128), rnd(L, nd, Hkv, 128)
+    xp, qp, kp, vp = rnd(C, D_IN), rnd(C, Hq, 128), rnd(C, Hkv, 128), rnd(C, Hkv, 128)
+    out_d = torch.empty((L, nd, Hq, 128), dtype=torch.bfloat16, device=dev)
+    out_p = torch.empty((C, Hq, 128), dtype=torch.bfloat16, device=dev)
+    lg_p = torch.empty((C, Hkv), dtype=torch.float32, device=dev)
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def step(timers=None):
+        for l in range(L):
+            a, b, c_ = ev(), ev(), ev()
+            a.record()
+            for s in range(NP):                                           # sequences 0..7 prefill
+                cache.spkv_score(preds[l], xp, logits=lg_p)
+                cache.spkv_prefill(l, s, kp, vp, lg_p, q=qp, out=out_p)
+            b.record()
+            cache.spkv_score_append_evict(l, preds[l], dec_ids, xq[l], kd[l], vd[l])
+            cache.spkv_decode_attention(l, dec_ids, qd[l], out=out_d[l])
+            c_.record()
+            if timers is not None:
+                timers.append((a, b, c_))
+
+    for _ in range(Wm):
+        step()
+    cache.check()
+    st0 = cache.spkv_cache_stats()
+    lens0 = [cache.spkv_read_lengths(l)[0][:NP].astype(np.int64) for l in range(L)]
+    torch.cuda.synchronize()
+    timers, e0, e1 = [], ev(), ev()
+    with ClockSampler(0) as clk:
+        e0.record()
+        for _ in range(K):
+            step(timers)
+        e1.record()
+        torch.cuda.synchronize()
+    cache.check()
+    ms = e0.elapsed_time(e1)
+    pre_ms = sum(a.elapsed_time(b) for a, b, _ in timers)
+    dec_ms = sum(b.elapsed_time(c_) for _, b, c_ in timers)
+    st1 = cache.spkv_cache_stats()
+    # useful prefill flops: visible keys per (query, head) = kept before + kept inside the chunk so far + window
+    keys = 0.0
+    for l in range(L):
+        for kk in range(K):
+            kept_before = lens0[l].sum(axis=0) + kk * NP * rates[l] * C      # [Hkv], summed over the 8 sequences
+            keys += float(((kept_before + NP * (rates[l] * C / 2 + W)) * (Hq // Hkv) * C).sum())
+    pre_tflops = keys * 4 * 128 / (pre_ms * 1e-3) / 1e12
+    # decode bytes: kept + window pairs of the 56 decoding sequences (their share of the resident bytes)
+    lens_all = np.stack([cache.spkv_read_lengths(l)[0] for l in range(L)]).astype(np.int64)   # [L, B, Hkv]
+    dec_bytes = float((lens_all[:, NP:].sum() + L * nd * Hkv * W) * 512 + L * nd * Hq * 512)
+    dec_gbs = dec_bytes * K / (dec_ms * 1e-3) / 1e9
+    tokens = K * (NP * C + nd)
+    line = {
+        "metric": "SP-KV mixed prefill + decode tokens/s (ragged batch 64)", "value": tokens / (ms * 1e-3),
+        "unit": "tokens/s", "n_gpus": 1, "steps": K, "warmup": Wm, "ms_per_step": ms / K,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": cfg["name"], "layers": L, "batch": B, "prefilling": NP, "chunk": C,
+                   "contexts": "uniform[4096, 65536], seeded", "keep_rates": "beta(0.5, 2.0)",
+                   "density": st1.density_cache, "resident_gb": st1.bytes_resident / 1e9,
+                   "l2": "inputs larger than L2", "cuda_graph": False},
+        "clocks": clk.result, "gpu_launches": K * L * (NP * 6 + 2),
+        "decode": {"tokens_per_s": K * nd / (dec_ms * 1e-3), "ms_per_step": dec_ms / K, "achieved_gbs": dec_gbs,
+                   "frac_of_measured_hbm": dec_gbs / hbm_peak},
+        "prefill": {"tokens_per_s": K * NP * C / (pre_ms * 1e-3), "ms_per_step": pre_ms / K,
+                    "useful_tflops": pre_tflops, "frac_of_sustained_bf16": pre_tflops / 1356.9,
+                    "kernel": "prefill_attn_tc5_kernel (tcgen05)"},
+        "roofline": {"bound": "tensor", "kernel": "prefill_attn_tc5_kernel", "achieved": pre_tflops, "peak": 1356.9,
+                     "unit": "TFLOP/s", "frac": pre_tflops / 1356.9, "peak_kind": "of measured (sustained)",
+                     "traffic": None},
+        "e2e": None, "dense": None,
+        "note": "dense K/V of this batch (~292 GB) does not fit one GPU: no dense run for this config",
+    }
+    print(json.dumps(line))
+
+
 def load_traffic(workload, launch_bytes):
     """DRAM bytes per decode launch from the committed ncu summary, if there is one."""
     try:
@@ -463,6 +571,9 @@ def main():
         args.warmup = 3
     if args.impl == "reference":
         run_reference(args)
+    elif args.config == 4:
+        if int(os.environ.get("RANK", "0")) == 0:
+            run_config4(args)
     else:
         run_ours(args)
 
