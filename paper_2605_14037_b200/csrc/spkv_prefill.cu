@@ -365,7 +365,7 @@ extern "C" int spkv_prefill(spkv_cache_t *cache, int32_t layer, int32_t seq, int
     const char *e = getenv("SPKV_PREFILL_KERNEL");  // "mma": the mma.sync comparison kernel
     return e && e[0] == 'm';
   }();
-  if (d_q && !use_mma_sync) {
+  if (d_q && !use_mma_sync && sm_scale > 0.f) {  // the tcgen05 kernel folds a positive scale into the exponent
     int rc = launch_prefill_attn_tc5(a, s);
     if (rc) return rc;
   } else if (d_q) {

@@ -253,24 +253,28 @@ __global__ void __launch_bounds__(tc5::kThreads, 1) prefill_attn_tc5_kernel(Pref
       tmem_ld_wait();
       fence_before();
       mbar_arrive(&bar[B_S_FREE + s]);
-      // visibility: compact-cache page j -> first nv pairs; staging page -> the band of this row
+      // visibility: compact-cache page j -> first nv pairs; staging page -> the band of this row.
+      // v keeps the raw scores (masked ones become -inf); the scale is folded into the exponent
+      // below, and pages that every row of the warp sees in full skip the masking altogether.
       float mx = -INFINITY;
       if (j < n_ptiles) {
         const int base = j * kP;
+        const bool all_visible = __all_sync(0xffffffffu, base + kP <= nv);
+        if (!all_visible) {
 #pragma unroll
-        for (int x = 0; x < 64; ++x) {
-          v[x] = (base + x < nv) ? v[x] * a.scale_log2 : -INFINITY;
-          mx = fmaxf(mx, v[x]);
+          for (int x = 0; x < 64; ++x) v[x] = (base + x < nv) ? v[x] : -INFINITY;
         }
       } else {
         const int base = (sp_lo + j - n_ptiles) * kP;
 #pragma unroll
         for (int x = 0; x < 64; ++x) {
           const int jj = base + x;
-          v[x] = (row_ok && jj <= jq && jj > jq - c.w) ? v[x] * a.scale_log2 : -INFINITY;
-          mx = fmaxf(mx, v[x]);
+          v[x] = (row_ok && jj <= jq && jj > jq - c.w) ? v[x] : -INFINITY;
         }
       }
+#pragma unroll
+      for (int x = 0; x < 64; ++x) mx = fmaxf(mx, v[x]);
+      mx *= a.scale_log2;  // scale > 0 (checked on the host): the maximum commutes with it
       // the reference maximum moves only when the row maximum outgrows it by 2^8
       const bool grow = mx > m_ref + 8.f;
       const float m_new = grow ? mx : m_ref;
@@ -300,7 +304,8 @@ __global__ void __launch_bounds__(tc5::kThreads, 1) prefill_attn_tc5_kernel(Pref
         uint32_t hi[4], lo[4];
 #pragma unroll
         for (int x = 0; x < 4; ++x) {
-          const float p0 = fast_exp2(v[ch * 8 + 2 * x] - ms), p1 = fast_exp2(v[ch * 8 + 2 * x + 1] - ms);
+          const float p0 = fast_exp2(fmaf(v[ch * 8 + 2 * x], a.scale_log2, -ms));
+          const float p1 = fast_exp2(fmaf(v[ch * 8 + 2 * x + 1], a.scale_log2, -ms));
           l += p0 + p1;
           const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
           const float2 hf = __bfloat1622float2(h);
