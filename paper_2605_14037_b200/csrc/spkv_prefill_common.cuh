@@ -23,6 +23,8 @@ struct PrefillArgs {
 __device__ inline int32_t *unit_ws(const PrefillArgs &a, int kvh) { return a.ws + (size_t)kvh * a.ws_stride; }
 
 
+// staging pages + chunk attention on tcgen05 (two heads per block when G is even)
 int launch_prefill_attn_tc5(const PrefillArgs &a, cudaStream_t s);
+int launch_prefill_attn_tc5x2(const PrefillArgs &a, cudaStream_t s);
 
 }  // namespace spkv

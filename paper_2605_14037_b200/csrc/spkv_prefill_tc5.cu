@@ -18,8 +18,10 @@
 //
 // Warps: 0-3 softmax/correction/epilogue (thread = query row = TMEM lane), 4 page loader (one
 // lane) and TMEM allocation, 5 MMA issue (one lane).  All waits are bounded.
-#include "spkv_mma.cuh"
+#include <stdlib.h>
+
 #include "spkv_prefill_common.cuh"
+#include "spkv_tc5.cuh"
 
 namespace spkv {
 
@@ -35,54 +37,6 @@ constexpr int kSBar = kSP + 32768;           // barriers
 constexpr int kSmemBytes = kSBar + 256;
 
 enum { B_KV_FULL = 0, B_KV_EMPTY = 4, B_S_FULL = 8, B_S_FREE = 10, B_P_FULL = 12, B_O_DONE = 13, B_COUNT = 14 };
-
-__device__ inline uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-  // shared-memory matrix descriptor: start address, leading / stride byte offsets (in 16-byte
-  // units), descriptor version 1, 128-byte swizzle
-  return (uint64_t)((saddr & 0x3FFFF) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
-         ((uint64_t)(sbo_bytes >> 4) << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
-}
-// instruction descriptor, kind::f16: fp32 accumulate, bf16 x bf16, A K-major
-__host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool b_mn_major) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(N >> 3) << 17) |
-         ((uint32_t)(M >> 4) << 24);
-}
-__device__ inline void umma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ inline void umma_commit(uint64_t *bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
-               : "memory");
-}
-__device__ inline void fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ inline void fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ inline void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-
-// 16 consecutive fp32 columns of this thread's TMEM lane
-__device__ inline void tmem_ld16(uint32_t taddr, float (&v)[16]) {
-  uint32_t r[16];
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr));
-#pragma unroll
-  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
-}
-__device__ inline void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ inline void tmem_st16(uint32_t taddr, const float (&v)[16]) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};\n"
-      ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
-      "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])),
-      "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])),
-      "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])),
-      "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15]))
-      : "memory");
-}
-__device__ inline void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 }  // namespace tc5
 
@@ -354,7 +308,12 @@ int launch_prefill_attn_tc5(const PrefillArgs &a, cudaStream_t s) {
   if (cudaFuncSetAttribute(prefill_attn_tc5_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            tc5::kSmemBytes) != cudaSuccess)
     return SPKV_E_CUDA;
+  static const bool one_head = [] {
+    const char *e = getenv("SPKV_PREFILL_KERNEL");  // "tc5x1": one query head per block
+    return e && e[0] == 't' && e[1] == 'c' && e[2] == '5' && e[3] == 'x' && e[4] == '1';
+  }();
   prefill_stage_kernel<<<dim3(a.n_stage_pages, a.c.Hkv), 256, 0, s>>>(a);
+  if (a.c.G % 2 == 0 && !one_head) return launch_prefill_attn_tc5x2(a, s);
   prefill_attn_tc5_kernel<<<dim3((a.C + 127) / 128, a.c.Hq), tc5::kThreads, tc5::kSmemBytes, s>>>(a);
   return check_stream_error(cudaGetLastError());
 }

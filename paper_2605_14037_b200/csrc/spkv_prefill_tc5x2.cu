@@ -1,0 +1,290 @@
+// Chunk attention of spkv_prefill on tcgen05, two query heads per block.
+//
+// One block = 128 consecutive queries of TWO query heads that share a KV head (GQA, Eq. 5:
+// head j reads KV head j / G).  Both heads walk the same page list, so each 32 KB page is
+// fetched once and feeds both.  Each head owns one "softmax group" of 128 threads (thread =
+// query row = TMEM lane) and its own S / O accumulators in tensor memory; the single MMA
+// thread alternates between the two heads, so while one group computes its softmax the
+// tensor core works for the other:
+//
+//   tensor core :  PV0(j-1) QK0(j) | PV1(j-1) QK1(j) | PV0(j) QK0(j+1) | ...
+//   group 0     :                  | softmax0(j)      |                  softmax0(j+1) ...
+//   group 1     :  softmax1(j-1)   |                  | softmax1(j)      | ...
+//
+// P = exp2(S - m) is split into hi + lo bf16 terms and written back into the tensor-memory
+// columns S came from (two bf16 per 32-bit column); the P.V MMAs take it from there as their A
+// operand, so P never touches shared memory.  tcgen05.mma instructions execute in issue order:
+// QK(j+1) of a head cannot overwrite P(j) before PV(j) has read it.
+//
+// Tensor memory (512 columns): S/P of head 0 [0,64), of head 1 [64,128); O of head 0
+// [128,256), of head 1 [256,384).  Shared memory: Q of both heads (64 KB) + 5 page stages.
+// Warps 0-3 group 0, 4-7 group 1, 8 page loader + TMEM allocation, 9 MMA issue.  All waits
+// are bounded.
+#include "spkv_prefill_common.cuh"
+#include "spkv_tc5.cuh"
+
+namespace spkv {
+
+namespace tc5x2 {
+constexpr int kThreads = 320;
+constexpr int kTmemCols = 512;
+constexpr int kSQ = 0;                     // 2 x 32 KB: Q of head 0, head 1 (two slabs of 128 rows x 128 B each)
+constexpr int kStages = 5;
+constexpr int kSKV = 65536;                // kStages x 32 KB
+constexpr int kSBar = kSKV + kStages * kPageBytes;
+constexpr int kSmemBytes = kSBar + 256;
+enum { B_KV_FULL = 0, B_KV_EMPTY = 8, B_S_FULL = 16, B_P_FULL = 18, B_COUNT = 20 };
+}  // namespace tc5x2
+
+__global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(PrefillArgs a) {
+  using namespace tc5;
+  using namespace tc5x2;
+  extern __shared__ __align__(1024) unsigned char smem[];
+  const CacheView &c = a.c;
+  uint64_t *bar = reinterpret_cast<uint64_t *>(smem + kSBar);
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + kSBar + B_COUNT * 8);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int pairs_per_kvh = c.G >> 1;
+  const int kvh = blockIdx.y / pairs_per_kvh, hq0 = kvh * c.G + (blockIdx.y % pairs_per_kvh) * 2;
+  const int i0 = blockIdx.x * 128;
+  const int32_t *hdr = unit_ws(a, kvh);
+  const int32_t *E = hdr + kHdrInts;
+  const int len0 = hdr[H_LEN0], n_old = hdr[H_NOLD], N = hdr[H_N];
+  const int u = unit_index(c, a.layer, a.seq, kvh);
+  // kept pairs visible to chunk query i: the first nvis(i) pairs of the compact cache
+  auto nvis = [&](int i) { return len0 + E[min(max(i + n_old - c.w + 1, 0), N)]; };
+  const int i_last = min(i0 + 127, a.C - 1);
+  const int n_ptiles = (nvis(i_last) + kP - 1) / kP;
+  // band, in staging indices (query i is staging pair n_old + i)
+  const int sp_lo = max(0, i0 + n_old - c.w + 1) / kP, sp_hi = (i_last + n_old) / kP;
+  const int n_tiles = n_ptiles + (sp_hi - sp_lo + 1);
+
+  if (tid == 0) {
+    for (int i = 0; i < kStages; ++i) {
+      mbar_init(&bar[B_KV_FULL + i], 1);
+      mbar_init(&bar[B_KV_EMPTY + i], 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&bar[B_S_FULL + i], 1);
+      mbar_init(&bar[B_P_FULL + i], 128);
+    }
+    mbar_fence_init();
+  }
+  // Q tiles -> per head two slabs of 128 rows x 128 B, 128-byte swizzle (rows past the chunk are zero)
+  for (int x = tid; x < 2 * 128 * 16; x += kThreads) {
+    const int h = x >> 11, r = (x >> 4) & 127, ch = x & 15;
+    uint4 val = make_uint4(0, 0, 0, 0);
+    if (i0 + r < a.C) val = *reinterpret_cast<const uint4 *>(a.q + ((size_t)(i0 + r) * c.Hq + hq0 + h) * kD + ch * 8);
+    *reinterpret_cast<uint4 *>(smem + kSQ + h * 32768 + (ch >> 3) * 16384 + r * 128 + (((ch & 7) ^ (r & 7)) << 4)) = val;
+  }
+  fence_async_smem();
+  if (warp == 8) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "n"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  fence_before();
+  __syncthreads();
+  fence_after();
+  const uint32_t tbase = *tmem_slot;
+  bool failed = false;
+
+  if (warp == 8) {
+    // ---------------------------------------------------------------- page loader
+    int j = 0;
+    for (int base = 0; base < n_tiles && !failed; base += 32) {
+      const int jl = base + lane;
+      int64_t src_off = 0;
+      if (jl < n_ptiles) src_off = (int64_t)c.table[(size_t)u * c.max_pages + jl] * kPageElems;
+      const int cnt = min(32, n_tiles - base);
+      for (int x = 0; x < cnt; ++x, ++j) {
+        const int64_t off = __shfl_sync(0xffffffffu, src_off, x);
+        if (lane == 0) {
+          const int s = j % kStages;
+          if (j >= kStages && !mbar_wait_bounded(&bar[B_KV_EMPTY + s], ((j / kStages) - 1) & 1)) failed = true;
+          if (!failed) {
+            const __nv_bfloat16 *src =
+                j < n_ptiles ? c.pages + off
+                             : a.stage_pages + ((size_t)kvh * a.n_stage_pages + sp_lo + (j - n_ptiles)) * kPageElems;
+            mbar_arrive_expect_tx(&bar[B_KV_FULL + s], kPageBytes);
+            bulk_load(smem + kSKV + s * kPageBytes, src, kPageBytes, &bar[B_KV_FULL + s]);
+          }
+        }
+        failed = __shfl_sync(0xffffffffu, (int)failed, 0) != 0;
+        if (failed) break;
+      }
+    }
+    if (failed && lane == 0)  // do not leave while copies may still be landing
+      for (int k = max(0, j - kStages); k < j; ++k)
+        mbar_wait_bounded(&bar[B_KV_FULL + (k % kStages)], (k / kStages) & 1);
+  } else if (warp == 9) {
+    // ---------------------------------------------------------------- MMA issue
+    if (lane == 0) {
+      constexpr uint32_t idesc_qk = instr_desc(128, 64, false), idesc_pv = instr_desc(128, 128, true);
+      const uint32_t sQ = smem_u32(smem + kSQ);
+      // O_h += P_h(jj) . V(jj): A from tensor memory (hi in columns [0,32) of the head's S
+      // region, lo in [32,64)), B = the page's value block, MN-major
+      auto issue_pv = [&](int h, int jj) {
+        if (!mbar_wait_bounded(&bar[B_P_FULL + h], jj & 1)) { failed = true; return; }
+        fence_after();
+        const uint32_t sV = smem_u32(smem + kSKV + (jj % kStages) * kPageBytes) + kBlockElems * 2;
+#pragma unroll
+        for (int part = 0; part < 2; ++part)
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk)
+            umma_ts(tbase + 128 + h * 128, tbase + h * 64 + part * 32 + kk * 8, smem_desc(sV + kk * 2048, 8192, 1024),
+                    idesc_pv, (jj > 0 || part > 0 || kk > 0) ? 1u : 0u);
+      };
+      for (int j = 0; j < n_tiles && !failed; ++j) {
+        const int ks = j % kStages;
+        const uint32_t sK = smem_u32(smem + kSKV + ks * kPageBytes);
+        for (int h = 0; h < 2 && !failed; ++h) {
+          if (j >= 1) {
+            issue_pv(h, j - 1);
+            if (failed) break;
+            if (h == 1) umma_commit(&bar[B_KV_EMPTY + ((j - 1) % kStages)]);  // page j-1 has no reader left
+          }
+          if (h == 0) {
+            if (!mbar_wait_bounded(&bar[B_KV_FULL + ks], (j / kStages) & 1)) { failed = true; break; }
+            fence_after();
+          }
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk)
+            umma(tbase + h * 64, smem_desc(sQ + h * 32768 + (kk >> 2) * 16384 + (kk & 3) * 32, 16, 1024),
+                 smem_desc(sK + (kk >> 2) * 8192 + (kk & 3) * 32, 16, 1024), idesc_qk, kk > 0 ? 1u : 0u);
+          umma_commit(&bar[B_S_FULL + h]);  // also: PV_h(j-1) has completed, O_h is stable
+        }
+      }
+      for (int h = 0; h < 2 && !failed; ++h) {
+        issue_pv(h, n_tiles - 1);
+        if (!failed) umma_commit(&bar[B_S_FULL + h]);  // completion n_tiles: O_h is final
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- softmax groups
+    const int h = warp >> 2, row = tid & 127, i = i0 + row, hq = hq0 + h;
+    const bool row_ok = i < a.C;
+    const int nv = row_ok ? nvis(i) : 0;
+    const int jq = n_old + i;  // staging index of this row's own pair
+    const uint32_t t_lane = tbase + ((uint32_t)((warp & 3) * 32) << 16);
+    const uint32_t t_s = t_lane + h * 64, t_o = t_lane + 128 + h * 128;
+    float m_ref = -INFINITY, l = 0.f;
+    for (int j = 0; j < n_tiles; ++j) {
+      if (!mbar_wait_bounded(&bar[B_S_FULL + h], j & 1)) { failed = true; break; }
+      fence_after();
+      float v[64];
+#pragma unroll
+      for (int q4 = 0; q4 < 4; ++q4) {
+        float t16[16];
+        tmem_ld16(t_s + q4 * 16, t16);
+#pragma unroll
+        for (int x = 0; x < 16; ++x) v[q4 * 16 + x] = t16[x];
+      }
+      tmem_ld_wait();
+      // visibility: compact-cache page j -> first nv pairs; staging page -> the band of this row.
+      // v keeps the raw scores (masked ones become -inf); the scale is folded into the exponent,
+      // and pages that every row of the warp sees in full skip the masking altogether.
+      if (j < n_ptiles) {
+        const int base = j * kP;
+        if (!__all_sync(0xffffffffu, base + kP <= nv)) {
+#pragma unroll
+          for (int x = 0; x < 64; ++x) v[x] = (base + x < nv) ? v[x] : -INFINITY;
+        }
+      } else {
+        const int base = (sp_lo + j - n_ptiles) * kP;
+#pragma unroll
+        for (int x = 0; x < 64; ++x) {
+          const int jj = base + x;
+          v[x] = (row_ok && jj <= jq && jj > jq - c.w) ? v[x] : -INFINITY;
+        }
+      }
+      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+      for (int x = 0; x < 64; x += 4) {
+        mx0 = fmaxf(mx0, v[x]);
+        mx1 = fmaxf(mx1, v[x + 1]);
+        mx2 = fmaxf(mx2, v[x + 2]);
+        mx3 = fmaxf(mx3, v[x + 3]);
+      }
+      const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * a.scale_log2;  // scale > 0 (host-checked)
+      // the reference maximum moves only when the row maximum outgrows it by 2^8
+      const bool grow = mx > m_ref + 8.f;
+      const float m_new = grow ? mx : m_ref;
+      if (j > 0 && __any_sync(0xffffffffu, grow)) {
+        // S_FULL(j) completed after PV(j-1): O is stable until this group hands P(j) over
+        const float f = grow ? fast_exp2(m_ref - m_new) : 1.f;  // m_ref = -inf -> 0
+#pragma unroll
+        for (int q8 = 0; q8 < 8; ++q8) {
+          float t16[16];
+          tmem_ld16(t_o + q8 * 16, t16);
+          tmem_ld_wait();
+#pragma unroll
+          for (int x = 0; x < 16; ++x) t16[x] *= f;
+          tmem_st16(t_o + q8 * 16, t16);
+        }
+        l *= f;
+      }
+      m_ref = m_new;
+      const float ms = m_ref == -INFINITY ? 0.f : m_ref;
+      float l0 = 0.f, l1 = 0.f;
+#pragma unroll
+      for (int q2 = 0; q2 < 2; ++q2) {  // 32 keys -> 16 columns of hi, 16 of lo
+        uint32_t hi[16], lo[16];
+#pragma unroll
+        for (int x = 0; x < 16; ++x) {
+          const float p0 = fast_exp2(fmaf(v[q2 * 32 + 2 * x], a.scale_log2, -ms));
+          const float p1 = fast_exp2(fmaf(v[q2 * 32 + 2 * x + 1], a.scale_log2, -ms));
+          l0 += p0;
+          l1 += p1;
+          const __nv_bfloat162 hb = __floats2bfloat162_rn(p0, p1);
+          const float2 hf = __bfloat1622float2(hb);
+          hi[x] = *reinterpret_cast<const uint32_t *>(&hb);
+          lo[x] = pack_bf16(p0 - hf.x, p1 - hf.y);
+        }
+        tmem_st16u(t_s + q2 * 16, hi);
+        tmem_st16u(t_s + 32 + q2 * 16, lo);
+      }
+      l += l0 + l1;
+      tmem_st_wait();
+      fence_before();
+      mbar_arrive(&bar[B_P_FULL + h]);
+    }
+    if (!failed && mbar_wait_bounded(&bar[B_S_FULL + h], n_tiles & 1)) {
+      fence_after();
+      const float inv = l > 0.f ? 1.f / l : 0.f;
+      __nv_bfloat16 *orow = a.out + ((size_t)i * c.Hq + hq) * kD;
+#pragma unroll
+      for (int q8 = 0; q8 < 8; ++q8) {
+        float t16[16];
+        tmem_ld16(t_o + q8 * 16, t16);
+        tmem_ld_wait();
+        if (row_ok) {
+          uint4 w0, w1;
+          w0.x = pack_bf16(t16[0] * inv, t16[1] * inv);   w0.y = pack_bf16(t16[2] * inv, t16[3] * inv);
+          w0.z = pack_bf16(t16[4] * inv, t16[5] * inv);   w0.w = pack_bf16(t16[6] * inv, t16[7] * inv);
+          w1.x = pack_bf16(t16[8] * inv, t16[9] * inv);   w1.y = pack_bf16(t16[10] * inv, t16[11] * inv);
+          w1.z = pack_bf16(t16[12] * inv, t16[13] * inv); w1.w = pack_bf16(t16[14] * inv, t16[15] * inv);
+          *reinterpret_cast<uint4 *>(orow + q8 * 16) = w0;
+          *reinterpret_cast<uint4 *>(orow + q8 * 16 + 8) = w1;
+        }
+      }
+    } else {
+      failed = true;
+    }
+  }
+  if (failed) set_status(c, SPKV_E_TIMEOUT);
+  fence_before();
+  __syncthreads();
+  if (warp == 8)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tbase), "n"(tc5x2::kTmemCols) : "memory");
+}
+
+int launch_prefill_attn_tc5x2(const PrefillArgs &a, cudaStream_t s) {
+  if (cudaFuncSetAttribute(prefill_attn_tc5x2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           tc5x2::kSmemBytes) != cudaSuccess)
+    return SPKV_E_CUDA;
+  prefill_attn_tc5x2_kernel<<<dim3((a.C + 127) / 128, a.c.Hkv * (a.c.G / 2)), tc5x2::kThreads, tc5x2::kSmemBytes, s>>>(a);
+  return check_stream_error(cudaGetLastError());
+}
+
+}  // namespace spkv
