@@ -17,7 +17,7 @@
 // whatever reference maximum the row carries).
 //
 // Warps: 0-3 softmax/correction/epilogue (thread = query row = TMEM lane), 4 page loader (one
-// lane) and TMEM allocation, 5 MMA issue (one lane).  All waits are bounded.
+// lane) and TMEM allocation, 5 MMA issue (one elected lane).  All waits are bounded.
 #include <stdlib.h>
 
 #include "spkv_prefill_common.cuh"
@@ -152,8 +152,8 @@ __global__ void __launch_bounds__(tc5::kThreads, 1) prefill_attn_tc5_kernel(Pref
       for (int k = max(0, j - kStages); k < j; ++k)
         mbar_wait_bounded(&bar[B_KV_FULL + (k % kStages)], (k / kStages) & 1);
   } else if (warp == 5) {
-    // ---------------------------------------------------------------- MMA issue
-    if (lane == 0) {
+    // ---------------------------------------------------------------- MMA issue (whole warp, one elected lane issues)
+    {
       constexpr uint32_t idesc_qk = instr_desc(128, 64, false), idesc_pv = instr_desc(128, 128, true);
       const uint32_t sQ = smem_u32(smem + kSQ), sP = smem_u32(smem + kSP);
       auto issue_pv = [&](int jj) {

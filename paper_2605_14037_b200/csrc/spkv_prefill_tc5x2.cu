@@ -3,21 +3,22 @@
 // One block = 128 consecutive queries of TWO query heads that share a KV head (GQA, Eq. 5:
 // head j reads KV head j / G).  Both heads walk the same page list, so each 32 KB page is
 // fetched once and feeds both.  Each head owns one "softmax group" of 128 threads (thread =
-// query row = TMEM lane) and its own S / O accumulators in tensor memory; the single MMA
-// thread alternates between the two heads, so while one group computes its softmax the
-// tensor core works for the other:
+// query row = TMEM lane), two S buffers and one O accumulator in tensor memory.  The single MMA
+// thread runs two pages ahead with Q.K^T, so a group finds the scores of its next page ready
+// when it finishes the current one, and the issue-to-completion latency of the MMAs of one head
+// hides under the softmax of both:
 //
-//   tensor core :  PV0(j-1) QK0(j) | PV1(j-1) QK1(j) | PV0(j) QK0(j+1) | ...
-//   group 0     :                  | softmax0(j)      |                  softmax0(j+1) ...
-//   group 1     :  softmax1(j-1)   |                  | softmax1(j)      | ...
+//   MMA thread, per page j:  wait P0(j) | PV0(j) QK0(j+2) | wait P1(j) | PV1(j) QK1(j+2)
+//   group h               :  softmax_h(j) softmax_h(j+1) softmax_h(j+2) ...
 //
 // P = exp2(S - m) is split into hi + lo bf16 terms and written back into the tensor-memory
 // columns S came from (two bf16 per 32-bit column); the P.V MMAs take it from there as their A
 // operand, so P never touches shared memory.  tcgen05.mma instructions execute in issue order:
-// QK(j+1) of a head cannot overwrite P(j) before PV(j) has read it.
+// QK(j+2) of a head cannot overwrite P(j) before PV(j) has read it.  O is rescaled only when a
+// row's maximum grows by more than 2^8; a group that has to rescale first waits for PV(j-1).
 //
-// Tensor memory (512 columns): S/P of head 0 [0,64), of head 1 [64,128); O of head 0
-// [128,256), of head 1 [256,384).  Shared memory: Q of both heads (64 KB) + 5 page stages.
+// Tensor memory (512 columns): S/P buffer b of head h at [(2h+b) 64, +64); O of head h at
+// [256 + 128 h, +128).  Shared memory: Q of both heads (64 KB) + 5 page stages.
 // Warps 0-3 group 0, 4-7 group 1, 8 page loader + TMEM allocation, 9 MMA issue.  All waits
 // are bounded.
 #include "spkv_prefill_common.cuh"
@@ -33,8 +34,15 @@ constexpr int kStages = 5;
 constexpr int kSKV = 65536;                // kStages x 32 KB
 constexpr int kSBar = kSKV + kStages * kPageBytes;
 constexpr int kSmemBytes = kSBar + 256;
-enum { B_KV_FULL = 0, B_KV_EMPTY = 8, B_S_FULL = 16, B_P_FULL = 18, B_COUNT = 20 };
+enum { B_KV_FULL = 0, B_KV_EMPTY = 8, B_S_FULL = 16 /* [2h+b] */, B_P_FULL = 20 /* [2h+b] */, B_O_DONE = 24 /* [2h+b] */, B_COUNT = 28 };
 }  // namespace tc5x2
+
+#ifdef SPKV_TC5_TRACE
+__device__ long long g_tc5_trace[12][2048];
+#define TC5_STAMP(cond, who, j) do { if ((cond) && (j) < 2048) g_tc5_trace[who][j] = clock64(); } while (0)
+#else
+#define TC5_STAMP(cond, who, j) do { } while (0)
+#endif
 
 __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(PrefillArgs a) {
   using namespace tc5;
@@ -64,9 +72,15 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
       mbar_init(&bar[B_KV_FULL + i], 1);
       mbar_init(&bar[B_KV_EMPTY + i], 1);
     }
-    for (int i = 0; i < 2; ++i) {
+    // One barrier per head and page parity: a parity wait only tells adjacent phases apart, and
+    // producer and waiter of S, P and O can be two pages apart (a group may finish page j+1
+    // before the MMA thread has looked at P(j); PV(j-1) and PV(j) can both be in flight).
+    // Per parity they are at most one phase apart: S_FULL(j) completes after every MMA issued
+    // before it, PV(j-2) included.
+    for (int i = 0; i < 4; ++i) {
       mbar_init(&bar[B_S_FULL + i], 1);
       mbar_init(&bar[B_P_FULL + i], 128);
+      mbar_init(&bar[B_O_DONE + i], 1);
     }
     mbar_fence_init();
   }
@@ -88,6 +102,9 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
   fence_after();
   const uint32_t tbase = *tmem_slot;
   bool failed = false;
+#ifdef SPKV_TC5_TRACE
+  const bool traced = blockIdx.x == gridDim.x - 1 && blockIdx.y == gridDim.y - 1;
+#endif
 
   if (warp == 8) {
     // ---------------------------------------------------------------- page loader
@@ -118,46 +135,55 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
       for (int k = max(0, j - kStages); k < j; ++k)
         mbar_wait_bounded(&bar[B_KV_FULL + (k % kStages)], (k / kStages) & 1);
   } else if (warp == 9) {
-    // ---------------------------------------------------------------- MMA issue
-    if (lane == 0) {
+    // ---------------------------------------------------------------- MMA issue (whole warp, one elected lane issues)
+    {
       constexpr uint32_t idesc_qk = instr_desc(128, 64, false), idesc_pv = instr_desc(128, 128, true);
       const uint32_t sQ = smem_u32(smem + kSQ);
-      // O_h += P_h(jj) . V(jj): A from tensor memory (hi in columns [0,32) of the head's S
-      // region, lo in [32,64)), B = the page's value block, MN-major
+      auto issue_qk = [&](int h, int jj) {  // S_h[jj & 1] = Q_h . K(jj)^T
+        const uint32_t sK = smem_u32(smem + kSKV + (jj % kStages) * kPageBytes);
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk)
+          umma(tbase + (2 * h + (jj & 1)) * 64, smem_desc(sQ + h * 32768 + (kk >> 2) * 16384 + (kk & 3) * 32, 16, 1024),
+               smem_desc(sK + (kk >> 2) * 8192 + (kk & 3) * 32, 16, 1024), idesc_qk, kk > 0 ? 1u : 0u);
+        umma_commit(&bar[B_S_FULL + 2 * h + (jj & 1)]);
+      };
+      // O_h += P_h(jj) . V(jj): A from tensor memory (hi in columns [0,32) of the S buffer the
+      // scores came from, lo in [32,64)), B = the page's value block, MN-major
       auto issue_pv = [&](int h, int jj) {
-        if (!mbar_wait_bounded(&bar[B_P_FULL + h], jj & 1)) { failed = true; return; }
+        if (!mbar_wait_bounded(&bar[B_P_FULL + 2 * h + (jj & 1)], (jj >> 1) & 1)) { failed = true; return; }
+        TC5_STAMP(traced && lane == 0, 8 + h, jj);
         fence_after();
         const uint32_t sV = smem_u32(smem + kSKV + (jj % kStages) * kPageBytes) + kBlockElems * 2;
+        const uint32_t tP = tbase + (2 * h + (jj & 1)) * 64;
 #pragma unroll
         for (int part = 0; part < 2; ++part)
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk)
-            umma_ts(tbase + 128 + h * 128, tbase + h * 64 + part * 32 + kk * 8, smem_desc(sV + kk * 2048, 8192, 1024),
-                    idesc_pv, (jj > 0 || part > 0 || kk > 0) ? 1u : 0u);
+            umma_ts(tbase + 256 + h * 128, tP + part * 32 + kk * 8, smem_desc(sV + kk * 2048, 8192, 1024), idesc_pv,
+                    (jj > 0 || part > 0 || kk > 0) ? 1u : 0u);
+        umma_commit(&bar[B_O_DONE + 2 * h + (jj & 1)]);
       };
-      for (int j = 0; j < n_tiles && !failed; ++j) {
-        const int ks = j % kStages;
-        const uint32_t sK = smem_u32(smem + kSKV + ks * kPageBytes);
-        for (int h = 0; h < 2 && !failed; ++h) {
-          if (j >= 1) {
-            issue_pv(h, j - 1);
-            if (failed) break;
-            if (h == 1) umma_commit(&bar[B_KV_EMPTY + ((j - 1) % kStages)]);  // page j-1 has no reader left
-          }
-          if (h == 0) {
-            if (!mbar_wait_bounded(&bar[B_KV_FULL + ks], (j / kStages) & 1)) { failed = true; break; }
-            fence_after();
-          }
-#pragma unroll
-          for (int kk = 0; kk < 8; ++kk)
-            umma(tbase + h * 64, smem_desc(sQ + h * 32768 + (kk >> 2) * 16384 + (kk & 3) * 32, 16, 1024),
-                 smem_desc(sK + (kk >> 2) * 8192 + (kk & 3) * 32, 16, 1024), idesc_qk, kk > 0 ? 1u : 0u);
-          umma_commit(&bar[B_S_FULL + h]);  // also: PV_h(j-1) has completed, O_h is stable
-        }
+      auto wait_page = [&](int jj) {
+        if (!mbar_wait_bounded(&bar[B_KV_FULL + jj % kStages], (jj / kStages) & 1)) failed = true;
+        TC5_STAMP(traced && lane == 0, 10, jj);
+        fence_after();
+      };
+      for (int jj = 0; jj < 2 && jj < n_tiles && !failed; ++jj) {
+        wait_page(jj);
+        if (failed) break;
+        issue_qk(0, jj);
+        issue_qk(1, jj);
       }
-      for (int h = 0; h < 2 && !failed; ++h) {
-        issue_pv(h, n_tiles - 1);
-        if (!failed) umma_commit(&bar[B_S_FULL + h]);  // completion n_tiles: O_h is final
+      for (int j = 0; j < n_tiles && !failed; ++j) {
+        for (int h = 0; h < 2 && !failed; ++h) {
+          issue_pv(h, j);
+          if (failed) break;
+          if (h == 1) umma_commit(&bar[B_KV_EMPTY + (j % kStages)]);  // page j has no reader left
+          if (j + 2 < n_tiles) {
+            if (h == 0) wait_page(j + 2);
+            if (!failed) issue_qk(h, j + 2);
+          }
+        }
       }
     }
   } else {
@@ -167,10 +193,12 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
     const int nv = row_ok ? nvis(i) : 0;
     const int jq = n_old + i;  // staging index of this row's own pair
     const uint32_t t_lane = tbase + ((uint32_t)((warp & 3) * 32) << 16);
-    const uint32_t t_s = t_lane + h * 64, t_o = t_lane + 128 + h * 128;
+    const uint32_t t_o = t_lane + 256 + h * 128;
     float m_ref = -INFINITY, l = 0.f;
     for (int j = 0; j < n_tiles; ++j) {
-      if (!mbar_wait_bounded(&bar[B_S_FULL + h], j & 1)) { failed = true; break; }
+      const uint32_t t_s = t_lane + (2 * h + (j & 1)) * 64;
+      if (!mbar_wait_bounded(&bar[B_S_FULL + 2 * h + (j & 1)], (j >> 1) & 1)) { failed = true; break; }
+      TC5_STAMP(traced && row == 0, h * 4 + 0, j);
       fence_after();
       float v[64];
 #pragma unroll
@@ -181,6 +209,7 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
         for (int x = 0; x < 16; ++x) v[q4 * 16 + x] = t16[x];
       }
       tmem_ld_wait();
+      TC5_STAMP(traced && row == 0, h * 4 + 1, j);
       // visibility: compact-cache page j -> first nv pairs; staging page -> the band of this row.
       // v keeps the raw scores (masked ones become -inf); the scale is folded into the exponent,
       // and pages that every row of the warp sees in full skip the masking altogether.
@@ -211,7 +240,9 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
       const bool grow = mx > m_ref + 8.f;
       const float m_new = grow ? mx : m_ref;
       if (j > 0 && __any_sync(0xffffffffu, grow)) {
-        // S_FULL(j) completed after PV(j-1): O is stable until this group hands P(j) over
+        // O is stable between the completion of PV(j-1) and the hand-over of P(j)
+        if (!mbar_wait_bounded(&bar[B_O_DONE + 2 * h + ((j - 1) & 1)], ((j - 1) >> 1) & 1)) { failed = true; break; }
+        fence_after();
         const float f = grow ? fast_exp2(m_ref - m_new) : 1.f;  // m_ref = -inf -> 0
 #pragma unroll
         for (int q8 = 0; q8 < 8; ++q8) {
@@ -225,6 +256,7 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
         l *= f;
       }
       m_ref = m_new;
+      TC5_STAMP(traced && row == 0, h * 4 + 2, j);
       const float ms = m_ref == -INFINITY ? 0.f : m_ref;
       float l0 = 0.f, l1 = 0.f;
 #pragma unroll
@@ -247,9 +279,10 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
       l += l0 + l1;
       tmem_st_wait();
       fence_before();
-      mbar_arrive(&bar[B_P_FULL + h]);
+      mbar_arrive(&bar[B_P_FULL + 2 * h + (j & 1)]);
+      TC5_STAMP(traced && row == 0, h * 4 + 3, j);
     }
-    if (!failed && mbar_wait_bounded(&bar[B_S_FULL + h], n_tiles & 1)) {
+    if (!failed && mbar_wait_bounded(&bar[B_O_DONE + 2 * h + ((n_tiles - 1) & 1)], ((n_tiles - 1) >> 1) & 1)) {
       fence_after();
       const float inv = l > 0.f ? 1.f / l : 0.f;
       __nv_bfloat16 *orow = a.out + ((size_t)i * c.Hq + hq) * kD;
@@ -278,6 +311,12 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
   if (warp == 8)
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tbase), "n"(tc5x2::kTmemCols) : "memory");
 }
+
+#ifdef SPKV_TC5_TRACE
+extern "C" int spkv_debug_tc5_trace(long long *host_out) {
+  return cudaMemcpyFromSymbol(host_out, g_tc5_trace, sizeof(g_tc5_trace)) == cudaSuccess ? 0 : -1;
+}
+#endif
 
 int launch_prefill_attn_tc5x2(const PrefillArgs &a, cudaStream_t s) {
   if (cudaFuncSetAttribute(prefill_attn_tc5x2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
