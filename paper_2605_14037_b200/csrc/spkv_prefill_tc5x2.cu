@@ -19,15 +19,18 @@
 //
 // Tensor memory (512 columns): S/P buffer b of head h at [(2h+b) 64, +64); O of head h at
 // [256 + 128 h, +128).  Shared memory: Q of both heads (64 KB) + 5 page stages.
-// Warps 0-3 group 0, 4-7 group 1, 8 page loader + TMEM allocation, 9 MMA issue.  All waits
-// are bounded.
+// Warps: 0 MMA issue, 1 page loader + TMEM allocation, 2-3 idle, 4-7 group 0, 8-11 group 1
+// (a warp reaches the TMEM lanes 32 (warp % 4) ...).  The MMA warp comes first because the
+// warp schedulers favour lower-numbered warps when several are ready: as warp 9, behind two
+// always-ready softmax warps on its scheduler, it got an issue slot every ~9 cycles and the
+// tensor pipe starved.  All waits are bounded.
 #include "spkv_prefill_common.cuh"
 #include "spkv_tc5.cuh"
 
 namespace spkv {
 
 namespace tc5x2 {
-constexpr int kThreads = 320;
+constexpr int kThreads = 384;
 constexpr int kTmemCols = 512;
 constexpr int kSQ = 0;                     // 2 x 32 KB: Q of head 0, head 1 (two slabs of 128 rows x 128 B each)
 constexpr int kStages = 5;
@@ -38,7 +41,7 @@ enum { B_KV_FULL = 0, B_KV_EMPTY = 8, B_S_FULL = 16 /* [2h+b] */, B_P_FULL = 20 
 }  // namespace tc5x2
 
 #ifdef SPKV_TC5_TRACE
-__device__ long long g_tc5_trace[12][2048];
+__device__ long long g_tc5_trace[16][2048];
 #define TC5_STAMP(cond, who, j) do { if ((cond) && (j) < 2048) g_tc5_trace[who][j] = clock64(); } while (0)
 #else
 #define TC5_STAMP(cond, who, j) do { } while (0)
@@ -76,7 +79,8 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
     // producer and waiter of S, P and O can be two pages apart (a group may finish page j+1
     // before the MMA thread has looked at P(j); PV(j-1) and PV(j) can both be in flight).
     // Per parity they are at most one phase apart: S_FULL(j) completes after every MMA issued
-    // before it, PV(j-2) included.
+    // before it, PV(j-2) included.  O_DONE is committed for the last two pages only (one use
+    // per barrier).
     for (int i = 0; i < 4; ++i) {
       mbar_init(&bar[B_S_FULL + i], 1);
       mbar_init(&bar[B_P_FULL + i], 128);
@@ -92,7 +96,7 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
     *reinterpret_cast<uint4 *>(smem + kSQ + h * 32768 + (ch >> 3) * 16384 + r * 128 + (((ch & 7) ^ (r & 7)) << 4)) = val;
   }
   fence_async_smem();
-  if (warp == 8) {
+  if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
                  "n"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -106,7 +110,7 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
   const bool traced = blockIdx.x == gridDim.x - 1 && blockIdx.y == gridDim.y - 1;
 #endif
 
-  if (warp == 8) {
+  if (warp == 1) {
     // ---------------------------------------------------------------- page loader
     int j = 0;
     for (int base = 0; base < n_tiles && !failed; base += 32) {
@@ -134,34 +138,31 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
     if (failed && lane == 0)  // do not leave while copies may still be landing
       for (int k = max(0, j - kStages); k < j; ++k)
         mbar_wait_bounded(&bar[B_KV_FULL + (k % kStages)], (k / kStages) & 1);
-  } else if (warp == 9) {
+  } else if (warp == 0) {
     // ---------------------------------------------------------------- MMA issue (whole warp, one elected lane issues)
     {
       constexpr uint32_t idesc_qk = instr_desc(128, 64, false), idesc_pv = instr_desc(128, 128, true);
       const uint32_t sQ = smem_u32(smem + kSQ);
       auto issue_qk = [&](int h, int jj) {  // S_h[jj & 1] = Q_h . K(jj)^T
         const uint32_t sK = smem_u32(smem + kSKV + (jj % kStages) * kPageBytes);
-#pragma unroll
-        for (int kk = 0; kk < 8; ++kk)
-          umma(tbase + (2 * h + (jj & 1)) * 64, smem_desc(sQ + h * 32768 + (kk >> 2) * 16384 + (kk & 3) * 32, 16, 1024),
-               smem_desc(sK + (kk >> 2) * 8192 + (kk & 3) * 32, 16, 1024), idesc_qk, kk > 0 ? 1u : 0u);
+        umma_qk_page<16384 / 16, 8192 / 16>(tbase + (2 * h + (jj & 1)) * 64, smem_desc(sQ + h * 32768, 16, 1024),
+                                            smem_desc(sK, 16, 1024), idesc_qk);
         umma_commit(&bar[B_S_FULL + 2 * h + (jj & 1)]);
+        TC5_STAMP(traced && lane == 0, 12 + 2 * h, jj);
       };
       // O_h += P_h(jj) . V(jj): A from tensor memory (hi in columns [0,32) of the S buffer the
       // scores came from, lo in [32,64)), B = the page's value block, MN-major
       auto issue_pv = [&](int h, int jj) {
+        TC5_STAMP(traced && lane == 0 && h == 0, 15, jj);
         if (!mbar_wait_bounded(&bar[B_P_FULL + 2 * h + (jj & 1)], (jj >> 1) & 1)) { failed = true; return; }
         TC5_STAMP(traced && lane == 0, 8 + h, jj);
         fence_after();
         const uint32_t sV = smem_u32(smem + kSKV + (jj % kStages) * kPageBytes) + kBlockElems * 2;
         const uint32_t tP = tbase + (2 * h + (jj & 1)) * 64;
-#pragma unroll
-        for (int part = 0; part < 2; ++part)
-#pragma unroll
-          for (int kk = 0; kk < 4; ++kk)
-            umma_ts(tbase + 256 + h * 128, tP + part * 32 + kk * 8, smem_desc(sV + kk * 2048, 8192, 1024), idesc_pv,
-                    (jj > 0 || part > 0 || kk > 0) ? 1u : 0u);
-        umma_commit(&bar[B_O_DONE + 2 * h + (jj & 1)]);
+        umma_pv_page(tbase + 256 + h * 128, tP, smem_desc(sV, 8192, 1024), idesc_pv, jj > 0 ? 1u : 0u);
+        // the last two PVs have no later QK whose S_FULL would vouch for their completion
+        if (jj + 2 >= n_tiles) umma_commit(&bar[B_O_DONE + 2 * h + (jj & 1)]);
+        TC5_STAMP(traced && lane == 0, 11 + 2 * h, jj);
       };
       auto wait_page = [&](int jj) {
         if (!mbar_wait_bounded(&bar[B_KV_FULL + jj % kStages], (jj / kStages) & 1)) failed = true;
@@ -186,9 +187,9 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
         }
       }
     }
-  } else {
+  } else if (warp >= 4) {
     // ---------------------------------------------------------------- softmax groups
-    const int h = warp >> 2, row = tid & 127, i = i0 + row, hq = hq0 + h;
+    const int h = (warp >> 2) - 1, row = tid & 127, i = i0 + row, hq = hq0 + h;
     const bool row_ok = i < a.C;
     const int nv = row_ok ? nvis(i) : 0;
     const int jq = n_old + i;  // staging index of this row's own pair
@@ -209,7 +210,7 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
         for (int x = 0; x < 16; ++x) v[q4 * 16 + x] = t16[x];
       }
       tmem_ld_wait();
-      TC5_STAMP(traced && row == 0, h * 4 + 1, j);
+      
       // visibility: compact-cache page j -> first nv pairs; staging page -> the band of this row.
       // v keeps the raw scores (masked ones become -inf); the scale is folded into the exponent,
       // and pages that every row of the warp sees in full skip the masking altogether.
@@ -240,8 +241,14 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
       const bool grow = mx > m_ref + 8.f;
       const float m_new = grow ? mx : m_ref;
       if (j > 0 && __any_sync(0xffffffffu, grow)) {
-        // O is stable between the completion of PV(j-1) and the hand-over of P(j)
-        if (!mbar_wait_bounded(&bar[B_O_DONE + 2 * h + ((j - 1) & 1)], ((j - 1) >> 1) & 1)) { failed = true; break; }
+        // O is stable between the completion of PV(j-1) and the hand-over of P(j).  QK(j+1) was
+        // issued right after PV(j-1), so S_FULL(j+1) vouches for it (waiting on it here does not
+        // consume the phase); the last page has its own barrier.
+        if (!(j + 1 < n_tiles ? mbar_wait_bounded(&bar[B_S_FULL + 2 * h + ((j + 1) & 1)], ((j + 1) >> 1) & 1)
+                              : mbar_wait_bounded(&bar[B_O_DONE + 2 * h + ((j - 1) & 1)], 0))) {
+          failed = true;
+          break;
+        }
         fence_after();
         const float f = grow ? fast_exp2(m_ref - m_new) : 1.f;  // m_ref = -inf -> 0
 #pragma unroll
@@ -256,7 +263,7 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
         l *= f;
       }
       m_ref = m_new;
-      TC5_STAMP(traced && row == 0, h * 4 + 2, j);
+      
       const float ms = m_ref == -INFINITY ? 0.f : m_ref;
       float l0 = 0.f, l1 = 0.f;
 #pragma unroll
@@ -281,8 +288,9 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
       fence_before();
       mbar_arrive(&bar[B_P_FULL + 2 * h + (j & 1)]);
       TC5_STAMP(traced && row == 0, h * 4 + 3, j);
+      TC5_STAMP(traced && h == 0 && lane == 0 && warp > 4, warp - 4, j);  // rows 1-3: P arrival of warps 1-3 (trace only)
     }
-    if (!failed && mbar_wait_bounded(&bar[B_O_DONE + 2 * h + ((n_tiles - 1) & 1)], ((n_tiles - 1) >> 1) & 1)) {
+    if (!failed && mbar_wait_bounded(&bar[B_O_DONE + 2 * h + ((n_tiles - 1) & 1)], 0)) {
       fence_after();
       const float inv = l > 0.f ? 1.f / l : 0.f;
       __nv_bfloat16 *orow = a.out + ((size_t)i * c.Hq + hq) * kD;
@@ -308,7 +316,7 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
   if (failed) set_status(c, SPKV_E_TIMEOUT);
   fence_before();
   __syncthreads();
-  if (warp == 8)
+  if (warp == 1)
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tbase), "n"(tc5x2::kTmemCols) : "memory");
 }
 

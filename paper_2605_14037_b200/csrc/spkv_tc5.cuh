@@ -67,6 +67,48 @@ __device__ inline void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc,
       " @e tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n"
       ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// One page of scores: D (128 x 64) = Q (128 x 128) . K^T, eight K=16 steps in one asm block with a
+// single election.  adesc/bdesc are the descriptors of k-step 0; a step advances both by 32 bytes
+// (2 descriptor units) inside a 64-dim slab, the second slab starts a_slab / b_slab units later.
+template <int kASlabUnits, int kBSlabUnits>
+__device__ inline void umma_qk_page(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
+  asm volatile(
+      "{\n .reg .pred e;\n .reg .b64 a1, a2, a3, a4, a5, a6, a7, b1, b2, b3, b4, b5, b6, b7;\n"
+      " elect.sync _|e, 0xffffffff;\n"
+      " add.u64 a1, %1, 2; add.u64 a2, %1, 4; add.u64 a3, %1, 6;\n"
+      " add.u64 a4, %1, %4; add.u64 a5, a4, 2; add.u64 a6, a4, 4; add.u64 a7, a4, 6;\n"
+      " add.u64 b1, %2, 2; add.u64 b2, %2, 4; add.u64 b3, %2, 6;\n"
+      " add.u64 b4, %2, %5; add.u64 b5, b4, 2; add.u64 b6, b4, 4; add.u64 b7, b4, 6;\n"
+      " @e tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, 0;\n"
+      " @e tcgen05.mma.cta_group::1.kind::f16 [%0], a1, b1, %3, 1;\n"
+      " @e tcgen05.mma.cta_group::1.kind::f16 [%0], a2, b2, %3, 1;\n"
+      " @e tcgen05.mma.cta_group::1.kind::f16 [%0], a3, b3, %3, 1;\n"
+      " @e tcgen05.mma.cta_group::1.kind::f16 [%0], a4, b4, %3, 1;\n"
+      " @e tcgen05.mma.cta_group::1.kind::f16 [%0], a5, b5, %3, 1;\n"
+      " @e tcgen05.mma.cta_group::1.kind::f16 [%0], a6, b6, %3, 1;\n"
+      " @e tcgen05.mma.cta_group::1.kind::f16 [%0], a7, b7, %3, 1;\n}\n"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "n"(kASlabUnits), "n"(kBSlabUnits) : "memory");
+}
+// One page of P.V: D (128 x 128) (+)= P_hi . V + P_lo . V with P in tensor memory (hi at a_tmem,
+// lo 32 columns later, 8 columns per K=16 step) and V MN-major (a k-step = 16 value rows =
+// 2048 bytes = 128 descriptor units).  `first` = 0 overwrites D with the first product.
+__device__ inline void umma_pv_page(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t first) {
+  asm volatile(
+      "{\n .reg .pred e, p;\n .reg .b64 b1, b2, b3;\n .reg .b32 t1, t2, t3, t4, t5, t6, t7;\n"
+      " elect.sync _|e, 0xffffffff;\n setp.ne.b32 p, %4, 0;\n"
+      " add.u64 b1, %2, 128; add.u64 b2, %2, 256; add.u64 b3, %2, 384;\n"
+      " add.u32 t1, %1, 8; add.u32 t2, %1, 16; add.u32 t3, %1, 24; add.u32 t4, %1, 32;\n"
+      " add.u32 t5, %1, 40; add.u32 t6, %1, 48; add.u32 t7, %1, 56;\n"
+      " @e tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n"
+      " @e tcgen05.mma.cta_group::1.kind::f16 [%0], [t1], b1, %3, 1;\n"
+      " @e tcgen05.mma.cta_group::1.kind::f16 [%0], [t2], b2, %3, 1;\n"
+      " @e tcgen05.mma.cta_group::1.kind::f16 [%0], [t3], b3, %3, 1;\n"
+      " @e tcgen05.mma.cta_group::1.kind::f16 [%0], [t4], %2, %3, 1;\n"
+      " @e tcgen05.mma.cta_group::1.kind::f16 [%0], [t5], b1, %3, 1;\n"
+      " @e tcgen05.mma.cta_group::1.kind::f16 [%0], [t6], b2, %3, 1;\n"
+      " @e tcgen05.mma.cta_group::1.kind::f16 [%0], [t7], b3, %3, 1;\n}\n"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(first) : "memory");
+}
 __device__ inline void tmem_st16u(uint32_t taddr, const uint32_t (&r)[16]) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};\n"
