@@ -230,11 +230,11 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
       }
       float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-      for (int x = 0; x < 64; x += 4) {
-        mx0 = fmaxf(mx0, v[x]);
-        mx1 = fmaxf(mx1, v[x + 1]);
-        mx2 = fmaxf(mx2, v[x + 2]);
-        mx3 = fmaxf(mx3, v[x + 3]);
+      for (int x = 0; x < 64; x += 8) {
+        mx0 = max3(mx0, v[x], v[x + 1]);
+        mx1 = max3(mx1, v[x + 2], v[x + 3]);
+        mx2 = max3(mx2, v[x + 4], v[x + 5]);
+        mx3 = max3(mx3, v[x + 6], v[x + 7]);
       }
       const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * a.scale_log2;  // scale > 0 (host-checked)
       // the reference maximum moves only when the row maximum outgrows it by 2^8
@@ -265,25 +265,32 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
       m_ref = m_new;
       
       const float ms = m_ref == -INFINITY ? 0.f : m_ref;
-      float l0 = 0.f, l1 = 0.f;
+      // two elements per instruction where the hardware has a packed form (fma, add, sub)
+      const uint64_t sc2 = pack2(a.scale_log2, a.scale_log2), nms2 = pack2(-ms, -ms);
+      uint64_t l2a = pack2(0.f, 0.f), l2b = l2a;
 #pragma unroll
       for (int q2 = 0; q2 < 2; ++q2) {  // 32 keys -> 16 columns of hi, 16 of lo
         uint32_t hi[16], lo[16];
 #pragma unroll
         for (int x = 0; x < 16; ++x) {
-          const float p0 = fast_exp2(fmaf(v[q2 * 32 + 2 * x], a.scale_log2, -ms));
-          const float p1 = fast_exp2(fmaf(v[q2 * 32 + 2 * x + 1], a.scale_log2, -ms));
-          l0 += p0;
-          l1 += p1;
+          float e0, e1, r0, r1;
+          unpack2(fma2(pack2(v[q2 * 32 + 2 * x], v[q2 * 32 + 2 * x + 1]), sc2, nms2), e0, e1);
+          const float p0 = fast_exp2(e0), p1 = fast_exp2(e1);
+          const uint64_t p2 = pack2(p0, p1);
+          if (x & 1) l2b = add2(l2b, p2); else l2a = add2(l2a, p2);
           const __nv_bfloat162 hb = __floats2bfloat162_rn(p0, p1);
-          const float2 hf = __bfloat1622float2(hb);
           hi[x] = *reinterpret_cast<const uint32_t *>(&hb);
-          lo[x] = pack_bf16(p0 - hf.x, p1 - hf.y);
+          unpack2(sub2(p2, pack2(__uint_as_float(hi[x] << 16), __uint_as_float(hi[x] & 0xffff0000u))), r0, r1);
+          lo[x] = pack_bf16(r0, r1);
         }
         tmem_st16u(t_s + q2 * 16, hi);
         tmem_st16u(t_s + 32 + q2 * 16, lo);
       }
-      l += l0 + l1;
+      {
+        float la, lb;
+        unpack2(add2(l2a, l2b), la, lb);
+        l += la + lb;
+      }
       tmem_st_wait();
       fence_before();
       mbar_arrive(&bar[B_P_FULL + 2 * h + (j & 1)]);
