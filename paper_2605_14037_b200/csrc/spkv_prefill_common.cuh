@@ -22,6 +22,32 @@ struct PrefillArgs {
 
 __device__ inline int32_t *unit_ws(const PrefillArgs &a, int kvh) { return a.ws + (size_t)kvh * a.ws_stride; }
 
+// Work order of the tensor-core attention kernels (1-D grid, blocks start in index order):
+// heaviest blocks first, so that the last wave is made of short ones.  A block's length is the
+// number of pages it walks: KV heads are taken by descending number of kept pairs after the
+// chunk (the plan kernel has counted them), and inside a head the query tiles run from the end
+// of the chunk backwards.  Item -> (KV head, which of its `blocks_per_kvh` head groups, query
+// tile).  Called by whole warps at kernel entry; every warp computes the same answer.
+__device__ inline void prefill_work_item(const PrefillArgs &a, int item, int n_xtiles, int blocks_per_kvh, int &kvh,
+                                         int &sub, int &xtile) {
+  const int r = item / n_xtiles, rank = r / blocks_per_kvh, lane = threadIdx.x & 31, Hkv = a.c.Hkv;
+  xtile = n_xtiles - 1 - item % n_xtiles;
+  sub = r % blocks_per_kvh;
+  kvh = rank;
+  if (Hkv > 32) return;  // more KV heads than lanes: plain order
+  int key = -1;
+  if (lane < Hkv) {
+    const int32_t *hdr = unit_ws(a, lane);
+    key = hdr[H_LEN0] + hdr[kHdrInts + hdr[H_N]];
+  }
+  int my_rank = 0;
+  for (int k = 0; k < Hkv; ++k) {
+    const int other = __shfl_sync(0xffffffffu, key, k);
+    my_rank += (other > key || (other == key && k < lane)) ? 1 : 0;
+  }
+  kvh = __ffs(__ballot_sync(0xffffffffu, lane < Hkv && my_rank == rank)) - 1;
+}
+
 
 // staging pages + chunk attention on tcgen05 (two heads per block when G is even)
 int launch_prefill_attn_tc5(const PrefillArgs &a, cudaStream_t s);

@@ -77,7 +77,9 @@ __global__ void __launch_bounds__(tc5::kThreads, 1) prefill_attn_tc5_kernel(Pref
   uint64_t *bar = reinterpret_cast<uint64_t *>(smem + kSBar);
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + kSBar + B_COUNT * 8);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int hq = blockIdx.y, kvh = hq / c.G, i0 = blockIdx.x * 128;
+  int kvh, sub, xtile;
+  prefill_work_item(a, blockIdx.x, (a.C + 127) / 128, c.G, kvh, sub, xtile);
+  const int hq = kvh * c.G + sub, i0 = xtile * 128;
   const int32_t *hdr = unit_ws(a, kvh);
   const int32_t *E = hdr + kHdrInts;
   const int len0 = hdr[H_LEN0], n_old = hdr[H_NOLD], N = hdr[H_N];
@@ -314,7 +316,7 @@ int launch_prefill_attn_tc5(const PrefillArgs &a, cudaStream_t s) {
   }();
   prefill_stage_kernel<<<dim3(a.n_stage_pages, a.c.Hkv), 256, 0, s>>>(a);
   if (a.c.G % 2 == 0 && !one_head) return launch_prefill_attn_tc5x2(a, s);
-  prefill_attn_tc5_kernel<<<dim3((a.C + 127) / 128, a.c.Hq), tc5::kThreads, tc5::kSmemBytes, s>>>(a);
+  prefill_attn_tc5_kernel<<<dim3(((a.C + 127) / 128) * a.c.Hq), tc5::kThreads, tc5::kSmemBytes, s>>>(a);
   return check_stream_error(cudaGetLastError());
 }
 

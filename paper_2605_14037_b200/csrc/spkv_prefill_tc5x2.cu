@@ -55,9 +55,9 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
   uint64_t *bar = reinterpret_cast<uint64_t *>(smem + kSBar);
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + kSBar + B_COUNT * 8);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int pairs_per_kvh = c.G >> 1;
-  const int kvh = blockIdx.y / pairs_per_kvh, hq0 = kvh * c.G + (blockIdx.y % pairs_per_kvh) * 2;
-  const int i0 = blockIdx.x * 128;
+  int kvh, pair, xtile;
+  prefill_work_item(a, blockIdx.x, (a.C + 127) / 128, c.G >> 1, kvh, pair, xtile);
+  const int hq0 = kvh * c.G + pair * 2, i0 = xtile * 128;
   const int32_t *hdr = unit_ws(a, kvh);
   const int32_t *E = hdr + kHdrInts;
   const int len0 = hdr[H_LEN0], n_old = hdr[H_NOLD], N = hdr[H_N];
@@ -107,7 +107,7 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
   const uint32_t tbase = *tmem_slot;
   bool failed = false;
 #ifdef SPKV_TC5_TRACE
-  const bool traced = blockIdx.x == gridDim.x - 1 && blockIdx.y == gridDim.y - 1;
+  const bool traced = blockIdx.x == 0;
 #endif
 
   if (warp == 1) {
@@ -337,7 +337,7 @@ int launch_prefill_attn_tc5x2(const PrefillArgs &a, cudaStream_t s) {
   if (cudaFuncSetAttribute(prefill_attn_tc5x2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            tc5x2::kSmemBytes) != cudaSuccess)
     return SPKV_E_CUDA;
-  prefill_attn_tc5x2_kernel<<<dim3((a.C + 127) / 128, a.c.Hkv * (a.c.G / 2)), tc5x2::kThreads, tc5x2::kSmemBytes, s>>>(a);
+  prefill_attn_tc5x2_kernel<<<dim3(((a.C + 127) / 128) * a.c.Hkv * (a.c.G / 2)), tc5x2::kThreads, tc5x2::kSmemBytes, s>>>(a);
   return check_stream_error(cudaGetLastError());
 }
 
