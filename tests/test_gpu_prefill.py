@@ -66,12 +66,15 @@ def test_prefill_chunkings_match_oracle(chunk):
     (1, 4, 1, 0.5, [0.5]), (4, 1, 2, 0.2, [0.3, 0.6]), (100, 8, 1, 0.5, [0.4]),
     (200, 2, 2, 0.9, [0.1, 0.9]), (128, 4, 2, -math.inf, [0.2, 0.2]),
     (128, 4, 2, math.inf, [0.8, 0.8]), (128, 16, 1, 0.5, [0.0]), (128, 3, 2, 0.5, [1.0, 0.5]),
+    # more KV heads than lanes (the heaviest-first order falls back to plain order), and exactly 32
+    (128, 2, 33, 0.5, [((7 * i) % 33) / 33.0 for i in range(33)]),
+    (128, 2, 32, 0.5, [((5 * i) % 32) / 40.0 for i in range(32)]),
 ])
 def test_prefill_windows_groups_thresholds(w, G, Hkv, tau, rates):
     spkv = load()
     T, Hq = 700, G * Hkv
     cache = spkv.Cache(n_layers=1, max_seqs=1, n_q_heads=Hq, n_kv_heads=Hkv, max_context=2048,
-                       pool_pages=40, window=w, tau=tau)
+                       pool_pages=40 + 12 * Hkv, window=w, tau=tau)
     tl = cache.spkv_tau_logit()
     wl = Workload(210 + w + G, T, 1, Hq, Hkv, rates, tl)
     got = prefill_in_chunks(spkv, cache, 0, 0, wl, 0, [70, 1, 200, 129, 300])
