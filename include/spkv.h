@@ -140,7 +140,11 @@ int spkv_set_tau(spkv_cache_t *cache, float tau);
 
 /* Step 1, score + threshold (Eq. 1-2).  d_x [n_tok, d_in] bf16 -> d_logits_out
  * [n_tok, n_kv_heads] float32 (fp32 accumulation).  d_flags_out (optional, may be NULL)
- * [n_tok, n_kv_heads] uint8 = 1 where logit >= tau_logit under the current tau. */
+ * [n_tok, n_kv_heads] uint8 = 1 where logit >= tau_logit under the current tau.
+ * The two-layer form runs on the tensor cores for n_tok >= 64 when hidden is a multiple of 16
+ * up to 256 (and hidden * n_kv_heads rounded up to 8 is at most 4096), on the CUDA cores
+ * otherwise; the two differ in the last bits of a logit, and the flag always follows the
+ * logit written. */
 int spkv_score(spkv_cache_t *cache, const spkv_predictor_t *pred, const void *d_x,
                int32_t n_tok, float *d_logits_out, uint8_t *d_flags_out,
                spkv_stream_t stream);

@@ -138,4 +138,6 @@ namespace spkv {
 int check_stream_error(cudaError_t e);
 inline cudaStream_t as_stream(spkv_stream_t s) { return reinterpret_cast<cudaStream_t>(s); }
 float tau_to_logit(float tau);
+int launch_score_mlp_tc(spkv_cache *cache, const spkv_predictor_t *p, const void *d_x, int n_tok, float *d_logits,
+                        uint8_t *d_flags, cudaStream_t s);
 }  // namespace spkv

@@ -77,6 +77,10 @@ extern "C" int spkv_score(spkv_cache_t *cache, const spkv_predictor_t *p, const 
         cache->tau_logit, d_logits_out, d_flags_out);
   } else if (p->kind == 1) {
     if (!p->d_W2 || !p->d_b2 || p->hidden < 1 || p->hidden > 8192) return SPKV_E_INVALID;
+    // chunks of tokens at model width go to the tensor cores; a handful of tokens (decode) or an
+    // unusual shape stay on the CUDA cores.  Each token is scored once, by one of the two.
+    const int rc = launch_score_mlp_tc(cache, p, d_x, n_tok, d_logits_out, d_flags_out, s);
+    if (rc <= 0) return rc;
     score_mlp_kernel<<<n_tok, 256, (size_t)p->hidden * 4, s>>>(
         x, n_tok, p->d_in, static_cast<const __nv_bfloat16 *>(p->d_W1), p->d_b1, p->hidden,
         static_cast<const __nv_bfloat16 *>(p->d_W2), p->d_b2, Hkv, cache->tau_logit,

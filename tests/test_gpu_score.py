@@ -41,8 +41,15 @@ def test_linear_predictor(n_tok, d_in, Hkv):
     assert (np.abs(ref[differ] - float(tl)) < LOGIT_TOL).all()  # only inside the rounding band
 
 
+# 64 tokens and more go to the tensor-core kernel when hidden is a multiple of 16 up to 256 and
+# hidden x heads (rounded up to 8) <= 4096; the other cases run on the CUDA cores
 @pytest.mark.parametrize("n_tok,d_in,hidden,Hkv", [(1, 512, 64, 2), (16, 512, 256, 8),
-                                                   (300, 256, 64, 4), (3, 1024, 8, 1)])
+                                                   (300, 256, 64, 4), (3, 1024, 8, 1),
+                                                   (2000, 4096, 256, 8),     # model width, ragged last tile
+                                                   (129, 520, 48, 3),        # d_in not a multiple of 64
+                                                   (64, 64, 16, 16), (1000, 512, 128, 32),
+                                                   (500, 512, 256, 24),      # second layer too big for shared memory
+                                                   (256, 8192, 240, 5)])
 def test_mlp_predictor(n_tok, d_in, hidden, Hkv):
     spkv = load()
     rng = np.random.default_rng(30 + n_tok)
