@@ -57,6 +57,15 @@ def lib():
         l.orcB_attend_row.restype = None
         l.orcB_attend_row.argtypes = [_u16p, _u16p, _f32p, C.c_int, C.c_int, C.c_int, C.c_float,
                                       _u16p, C.c_int, C.c_int, C.c_double, _f64p, C.c_void_p]
+        l.orcB_attend_row_sinks.restype = None
+        l.orcB_attend_row_sinks.argtypes = [_u16p, _u16p, _f32p, C.c_int, C.c_int, C.c_int, C.c_float,
+                                            C.c_int, _u16p, C.c_int, C.c_int, C.c_double, _f64p,
+                                            C.c_void_p]
+        l.orcB_attend_all_sinks.restype = None
+        l.orcB_attend_all_sinks.argtypes = [_u16p, _u16p, _f32p, C.c_int, C.c_int, C.c_float, C.c_int,
+                                            _u16p, C.c_int, C.c_int, C.c_double, _f64p]
+        l.orcA_set_sinks.restype = None
+        l.orcA_set_sinks.argtypes = [C.c_void_p, C.c_int]
         l.orcB_attend_all.restype = None
         l.orcB_attend_all.argtypes = [_u16p, _u16p, _f32p, C.c_int, C.c_int, C.c_float, _u16p,
                                       C.c_int, C.c_int, C.c_double, _f64p]
@@ -142,25 +151,27 @@ def score_mlp(x, W1, b1, W2, b2) -> np.ndarray:
     return out
 
 
-def mask_attend_row(K, V, logit, t, w, tau_l, q, scale, want_lse=False):
-    """Mask form (Eq. 2-5), one query position t.  K,V [T,D]; q [G,D] -> [G,D]."""
+def mask_attend_row(K, V, logit, t, w, tau_l, q, scale, want_lse=False, n_sink=0):
+    """Mask form (Eq. 2-5), one query position t.  K,V [T,D]; q [G,D] -> [G,D].
+    n_sink > 0: the sink-token variant (first n_sink positions always retained)."""
     K, V, q, logit = _u16(K), _u16(V), _u16(q), _f32(logit)
     T, D = K.shape
     G = q.shape[0]
     out = np.empty((G, D), np.float64)
     lse = np.empty(G, np.float64)
-    lib().orcB_attend_row(K, V, logit, T, int(t), int(w), float(tau_l), q, G, D, float(scale),
-                          out, lse.ctypes.data)
+    lib().orcB_attend_row_sinks(K, V, logit, T, int(t), int(w), float(tau_l), int(n_sink), q, G, D,
+                                float(scale), out, lse.ctypes.data)
     return (out, lse) if want_lse else out
 
 
-def mask_attend_all(K, V, logit, w, tau_l, q, scale):
+def mask_attend_all(K, V, logit, w, tau_l, q, scale, n_sink=0):
     """Mask form for every position.  q [T,G,D] -> [T,G,D] (O(T^2))."""
     K, V, q, logit = _u16(K), _u16(V), _u16(q), _f32(logit)
     T, D = K.shape
     G = q.shape[1]
     out = np.empty((T, G, D), np.float64)
-    lib().orcB_attend_all(K, V, logit, T, int(w), float(tau_l), q, G, D, float(scale), out)
+    lib().orcB_attend_all_sinks(K, V, logit, T, int(w), float(tau_l), int(n_sink), q, G, D,
+                                float(scale), out)
     return out
 
 
@@ -175,9 +186,11 @@ def density(logit, w, tau_l):
 class Unit:
     """Streaming form: ring of w pairs + append-only kept list, one (layer, seq, KV head)."""
 
-    def __init__(self, w: int, D: int = 128):
-        self.w, self.D = int(w), int(D)
+    def __init__(self, w: int, D: int = 128, n_sink: int = 0):
+        self.w, self.D, self.n_sink = int(w), int(D), int(n_sink)
         self._h = C.c_void_p(lib().orcA_new(self.w, self.D))
+        if self.n_sink:
+            lib().orcA_set_sinks(self._h, self.n_sink)
 
     def __del__(self):
         try:

@@ -115,16 +115,18 @@ void orc_score_mlp(const uint16_t *x, int n_tok, int d_in, const uint16_t *W1,
  * Every position s in [0,T) gets a bias: 0 when causal and (gated on or inside
  * the window), -inf otherwise; the softmax runs over the whole row.
  */
-void orcB_attend_row(const uint16_t *K, const uint16_t *V, const float *logit, int T,
-                     int t, int w, float tau_logit, const uint16_t *q, int G, int D,
-                     double scale, double *out, double *lse) {
+void orcB_attend_row_sinks(const uint16_t *K, const uint16_t *V, const float *logit, int T,
+                           int t, int w, float tau_logit, int n_sink, const uint16_t *q, int G,
+                           int D, double scale, double *out, double *lse) {
   double *score = (double *)malloc(sizeof(double) * (size_t)T);
   for (int g = 0; g < G; ++g) {
     double mx = -INFINITY;
     for (int s = 0; s < T; ++s) {
       int z = (logit[s] >= tau_logit) ? 1 : 0;                 /* Eq. 2 */
       int in_win = (t - s >= 0) && (t - s < w);                /* window indicator */
-      double gate = (z || in_win) ? 0.0 : -INFINITY;           /* Eq. 3 */
+      int sink = s < n_sink;     /* "Fixed Attention Sinks" variant: the first n_sink
+                                    positions are retained whatever their gate says */
+      double gate = (z || in_win || sink) ? 0.0 : -INFINITY;   /* Eq. 3 */
       double causal = (s <= t) ? 0.0 : -INFINITY;
       double bias = causal + gate;                             /* Eq. 4 */
       double dot = 0.0;
@@ -146,13 +148,26 @@ void orcB_attend_row(const uint16_t *K, const uint16_t *V, const float *logit, i
   free(score);
 }
 
+/* The method as the paper defines it (no sink tokens). */
+void orcB_attend_row(const uint16_t *K, const uint16_t *V, const float *logit, int T,
+                     int t, int w, float tau_logit, const uint16_t *q, int G, int D,
+                     double scale, double *out, double *lse) {
+  orcB_attend_row_sinks(K, V, logit, T, t, w, tau_logit, 0, q, G, D, scale, out, lse);
+}
+
 /* Whole-sequence mask form: out[t][g][:] for every t (O(T^2); tiny T only). */
+void orcB_attend_all_sinks(const uint16_t *K, const uint16_t *V, const float *logit, int T,
+                           int w, float tau_logit, int n_sink, const uint16_t *q /*[T][G][D]*/,
+                           int G, int D, double scale, double *out /*[T][G][D]*/) {
+  for (int t = 0; t < T; ++t)
+    orcB_attend_row_sinks(K, V, logit, T, t, w, tau_logit, n_sink, q + (size_t)t * G * D, G, D,
+                          scale, out + (size_t)t * G * D, NULL);
+}
+
 void orcB_attend_all(const uint16_t *K, const uint16_t *V, const float *logit, int T,
                      int w, float tau_logit, const uint16_t *q /*[T][G][D]*/, int G, int D,
                      double scale, double *out /*[T][G][D]*/) {
-  for (int t = 0; t < T; ++t)
-    orcB_attend_row(K, V, logit, T, t, w, tau_logit, q + (size_t)t * G * D, G, D, scale,
-                    out + (size_t)t * G * D, NULL);
+  orcB_attend_all_sinks(K, V, logit, T, w, tau_logit, 0, q, G, D, scale, out);
 }
 
 /* Eq. 8 gate density over one (layer, head): mean of z over all T positions,
@@ -173,6 +188,7 @@ void orcB_density(const float *logit, int T, int w, float tau_logit, double *rho
 
 typedef struct orcA_unit {
   int w, D;
+  int n_sink;        /* positions < n_sink are kept whatever their logit (0: none) */
   long t;            /* number of pairs appended so far = next position        */
   uint16_t *ring_k;  /* [w][D]  slot (s mod w) holds position s                 */
   uint16_t *ring_v;
@@ -191,6 +207,8 @@ orcA_unit *orcA_new(int w, int D) {
   u->ring_logit = (float *)calloc((size_t)w, sizeof(float));
   return u;
 }
+
+void orcA_set_sinks(orcA_unit *u, int n_sink) { u->n_sink = n_sink; }
 
 void orcA_free(orcA_unit *u) {
   if (!u) return;
@@ -214,13 +232,14 @@ static void orcA_keep(orcA_unit *u, long pos, const uint16_t *k, const uint16_t 
 
 /* Append the pair of position t.  When the ring is full, the pair of position
  * t - w leaves it: it joins the kept list iff its stored logit >= tau_logit
- * (threshold applied at window exit, with the threshold current at that time),
- * otherwise it is gone for good. */
+ * (threshold applied at window exit, with the threshold current at that time)
+ * or it is one of the first n_sink positions (sink-token variant); otherwise it
+ * is gone for good. */
 void orcA_append(orcA_unit *u, const uint16_t *k, const uint16_t *v, float logit,
                  float tau_logit) {
   long slot = u->t % u->w;
   if (u->t >= u->w) {
-    if (u->ring_logit[slot] >= tau_logit)
+    if (u->ring_logit[slot] >= tau_logit || u->t - u->w < u->n_sink)
       orcA_keep(u, u->t - u->w, u->ring_k + (size_t)slot * u->D, u->ring_v + (size_t)slot * u->D);
   }
   memcpy(u->ring_k + (size_t)slot * u->D, k, 2 * (size_t)u->D);
