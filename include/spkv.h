@@ -69,6 +69,10 @@ typedef struct {
   int64_t pool_pages;   /* pages shared by all compact caches                           */
   float tau;            /* utility threshold in [0,1]; <= 0 keeps all, >= 1 keeps none  */
   int32_t flags;        /* 0 or SPKV_FLAG_NO_OVERLAP                                    */
+  int32_t sink_tokens;  /* >= 0: the first sink_tokens positions of every sequence are
+                           kept in the compact cache whatever their utility (the paper's
+                           "Fixed Attention Sinks" ablation; its evaluation protocol uses
+                           4).  0 = the method as defined by Eq. 2-4.                      */
 } spkv_config_t;
 
 /* By default consecutive hot-path launches on one stream overlap where they share no data

@@ -28,7 +28,7 @@ static int validate(const spkv_config_t *c) {
   if (c->window < 1 || c->max_context < 1 || c->pool_pages < 0) return SPKV_E_INVALID;
   if (c->head_dim != kD || c->page_tokens != kP) return SPKV_E_UNSUPPORTED;
   if (c->n_q_heads / c->n_kv_heads > kMaxGroup) return SPKV_E_UNSUPPORTED;
-  if (c->tau != c->tau) return SPKV_E_INVALID;
+  if (c->tau != c->tau || c->sink_tokens < 0) return SPKV_E_INVALID;
   int64_t units = (int64_t)c->n_layers * c->max_seqs * c->n_kv_heads;
   int64_t ring_pages = (c->window + kP - 1) / kP;
   if (units > (1 << 24)) return SPKV_E_INVALID;
@@ -116,6 +116,7 @@ extern "C" int spkv_cache_create(const spkv_config_t *cfg, void *d_arena, size_t
   v.L = cfg->n_layers; v.S = cfg->max_seqs; v.Hq = cfg->n_q_heads; v.Hkv = cfg->n_kv_heads;
   v.G = cfg->n_q_heads / cfg->n_kv_heads;
   v.w = cfg->window;
+  v.n_sink = cfg->sink_tokens;
   v.ring_pages = (cfg->window + kP - 1) / kP;
   v.max_pages = (cfg->max_context + kP - 1) / kP;
   v.n_units = cfg->n_layers * cfg->max_seqs * cfg->n_kv_heads;

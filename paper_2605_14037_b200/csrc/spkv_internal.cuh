@@ -36,6 +36,7 @@ constexpr int kMaxGroup = 16;      // query heads per KV head supported by the k
 
 struct CacheView {
   int32_t L, S, Hq, Hkv, G, w, ring_pages, max_pages, n_units;
+  int32_t n_sink;       // positions < n_sink are kept whatever their logit (sink tokens)
   int64_t pool_pages, n_ring_pages_total;
   int32_t *status;      // [0] sticky status, [1] free_top
   int32_t *t;

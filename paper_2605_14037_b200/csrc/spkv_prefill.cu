@@ -51,7 +51,7 @@ __global__ void __launch_bounds__(1024) prefill_plan_kernel(PrefillArgs a) {
     if (j < N) {
       const float lg = j < n_old ? c.ring_logit[(size_t)u * c.w + (p0 + j) % c.w]
                                  : a.logits[(size_t)(j - n_old) * c.Hkv + kvh];
-      flag = lg >= a.tau_logit;  // Eq. 2 on the float32 logit
+      flag = lg >= a.tau_logit || p0 + j < c.n_sink;  // Eq. 2 on the float32 logit; sink positions always
     }
     const unsigned ballot = __ballot_sync(0xffffffffu, flag);
     const int before = __popc(ballot & ((1u << lane) - 1u));
