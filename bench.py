@@ -115,17 +115,36 @@ def whole_job_rate(units_per_rank, seconds_local, dist=None, device=None):
     return world * units_per_rank / max_over_ranks(seconds_local, dist, device)
 
 
-def build_workload(spkv, synth, torch, cfg, dev, dense, total_steps, seed=0):
-    """Creates the cache, per-layer predictors and brings every sequence to context T."""
+def build_workload(spkv, synth, torch, cfg, dev, dense, total_steps, seed=0, tau=None):
+    """Creates the cache, per-layer predictors and brings every sequence to context T.
+    The predictors are calibrated so that head (l, h) keeps a fraction rates[l, h] at tau = 0.5;
+    another `tau` (threshold sweep) moves every head's rate along its Gaussian logit
+    distribution, as sweeping the threshold of a trained predictor does."""
     import numpy as np
     L, B, Hq, Hkv, T = cfg["L"], cfg["B"], cfg["Hq"], cfg["Hkv"], cfg["T"]
     rng = np.random.default_rng(seed)
-    tau = -math.inf if dense else TAU
+    tau = TAU if tau is None else tau
+    tau = -math.inf if dense else tau
     if cfg["beta"] is None:
         rates = np.full((L, Hkv), cfg["rate"])
     else:
         rates = synth.keep_rates(rng, L, Hkv, *cfg["beta"])
-    eff = np.ones_like(rates) if dense else rates
+    tl = 0.0  # logit-space threshold of tau = 0.5, where the biases are calibrated
+    pred_np = []
+    for l in range(L):
+        Wl = synth.linear_predictor(rng, Hkv, D_IN)
+        pred_np.append((Wl, synth.bias_for_keep_rate(Wl, rates[l], tl)))
+    if dense:
+        eff = np.ones_like(rates)
+    elif tau == TAU:
+        eff = rates
+    else:  # P(w.x + b >= tau_logit) for x ~ N(0, I): Phi((b - tau_logit) / |w|)
+        tl_run = math.log(tau / (1.0 - tau)) if 0.0 < tau < 1.0 else (-math.inf if tau <= 0.0 else math.inf)
+        eff = np.empty_like(rates)
+        for l, (Wl, bl) in enumerate(pred_np):
+            norms = np.sqrt((synth.bf16_bits_to_f32(Wl).astype(np.float64) ** 2).sum(axis=1))
+            z = (bl.astype(np.float64) - tl_run) / norms
+            eff[l] = [0.5 * math.erfc(-float(v) / math.sqrt(2.0)) for v in z]
     t_list = cfg.get("t_list")          # per-sequence contexts (ragged batch), else uniform T
     grow = cfg.get("grow", total_steps)  # pairs every sequence may still receive
     t_final = T + grow
@@ -137,11 +156,9 @@ def build_workload(spkv, synth, torch, cfg, dev, dense, total_steps, seed=0):
         pool_pages = int(per_seq.sum())
     cache = spkv.Cache(n_layers=L, max_seqs=B, n_q_heads=Hq, n_kv_heads=Hkv,
                        max_context=t_final + 64, pool_pages=pool_pages, window=W, tau=tau, device=dev)
-    tl = 0.0  # logit-space threshold of tau = 0.5 (the dense run ignores it)
     preds, keep = [], []
     for l in range(L):
-        Wl = synth.linear_predictor(rng, Hkv, D_IN)
-        bl = synth.bias_for_keep_rate(Wl, rates[l], tl)
+        Wl, bl = pred_np[l]
         Wd, bd = spkv.bf16_from_bits(Wl, dev), torch.from_numpy(bl).to(dev)
         preds.append(spkv.make_predictor(Wd, bd))
         keep.append((Wd, bd))
@@ -201,7 +218,7 @@ def run_ours(args):
     def max_ranks(x):
         return max_over_ranks(x, dist, dev)
 
-    def measure(dense):
+    def measure(dense, tau=None):
         nonlocal L
         cfg_run, L_full = cfg, cfg["L"]
         if dense:
@@ -212,12 +229,12 @@ def run_ours(args):
                 cfg_run = dict(cfg, L=max(1, int(cfg["L"] * 140e9 / dense_bytes)))
         L = cfg_run["L"]
         try:
-            return _measure(dense, cfg_run, L_full)
+            return _measure(dense, cfg_run, L_full, tau)
         finally:
             L = L_full
 
-    def _measure(dense, cfg, L_full):
-        cache, preds, rates, gen = build_workload(spkv, synth, torch, cfg, dev, dense, total_steps)
+    def _measure(dense, cfg, L_full, tau):
+        cache, preds, rates, gen = build_workload(spkv, synth, torch, cfg, dev, dense, total_steps, tau=tau)
         ids = torch.arange(B, dtype=torch.int32, device=dev)
         n_in = 4  # distinct q/k/v input sets cycled over the steps
         q_in = torch.randn((n_in, L, B, Hq, 128), generator=gen, device=dev).to(torch.bfloat16)
@@ -305,7 +322,7 @@ def run_ours(args):
                    clocks=clk.result, graph=graph is not None)
 
         # end to end through the host-buffer entry point
-        if not dense and e2e_steps > 0:
+        if not dense and e2e_steps > 0 and tau is None:
             pin = lambda t: t.cpu().pin_memory()
             hx, hq, hk, hv = pin(x_all[:4]), pin(q_in), pin(k_in), pin(v_in)
             hout = torch.empty((L, B, Hq, 128), dtype=torch.bfloat16).pin_memory()
@@ -336,6 +353,19 @@ def run_ours(args):
         torch.cuda.empty_cache()
         return res
 
+    if args.sweep_tau:
+        # threshold sweep (the deployment-time density control of the paper's section on
+        # controlling sparsity at inference time): one line per tau, same predictors, state rebuilt
+        for tau in [float(t) for t in args.sweep_tau.split(",")]:
+            r = measure(dense=False, tau=tau)
+            if rank == 0:
+                ach = r["launch_bytes"] / r["launch_s"] / 1e9
+                print(json.dumps({"sweep": "tau", "tau": tau, "workload": cfg["name"], "density": r["density"],
+                                  "kv_gb_per_step": r["kv_gb_per_step"], "tokens_per_s": r["tokens_per_s"],
+                                  "ms_per_step": r["ms_per_step"], "decode_kernel_gbs": ach,
+                                  "frac_of_hbm_peak": ach / hbm_peak, "steps": K, "warmup": Wm,
+                                  "clocks": r["clocks"]}), flush=True)
+        return
     sp = measure(dense=False)
     dn = measure(dense=True) if args.dense else None
 
@@ -566,6 +596,8 @@ def main():
     ap.add_argument("--layers", type=int, default=0,
                     help="override the layer count (small profiling captures only; not a bench line)")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--sweep-tau", default="",
+                    help="comma-separated thresholds: one decode measurement per tau, nothing else")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
