@@ -331,6 +331,7 @@ def run_ours(args):
                 for l in range(L):
                     cache.spkv_decode_step_host(l, preds[l], ids, hx[s % 4, l], hq[s % n_in, l],
                                                 hk[s % n_in, l], hv[s % n_in, l], hout[l])
+                cache.spkv_decode_step_host_flush()
                 torch.cuda.current_stream().synchronize()   # the step's result is read on the host
                 return float(hout[L - 1, 0, 0, 0])
 

@@ -229,18 +229,25 @@ int spkv_prefill(spkv_cache_t *cache, int32_t layer, int32_t seq, int32_t C, con
                  float sm_scale, void *d_workspace, size_t workspace_bytes,
                  spkv_stream_t stream);
 
-/* One decode step of one layer from HOST buffers (pinned memory recommended): copies
- * x, q, k, v to the device staging area, runs score -> append/evict -> decode attention,
- * copies the output back, all enqueued on `stream` (no synchronisation).
+/* One decode step of one layer from HOST buffers (pinned memory, or the copies are not
+ * asynchronous): score -> append/evict -> decode attention with the inputs copied in and the
+ * output copied out.  The copies run on two streams of the cache's own, double-buffered, so
+ * that the transfers of one call overlap the kernels of its neighbours; the kernels run on
+ * `stream`.  Nothing synchronises with the host.  Completion: after call i, `stream` has
+ * waited for the output of call i-1; spkv_decode_step_host_flush makes `stream` wait for the
+ * output of the last call -- synchronise (or order later work) after that.  The host input
+ * buffers of a call must stay untouched until its copies have run (flush + synchronise).
  *   h_x [B, d_in], h_q [B, n_q_heads, 128], h_k/h_v [B, n_kv_heads, 128] bf16,
  *   h_out [B, n_q_heads, 128] bf16;
- *   d_staging: >= spkv_decode_step_staging_bytes(cfg, B, d_in) bytes (inputs, logits,
- *   output and the decode workspace live there; zero-filled once before first use). */
+ *   d_staging: >= spkv_decode_step_staging_bytes(cfg, B, d_in) bytes (two slots of inputs,
+ *   logits and output, and the decode workspace; zero-filled once before first use).  Pass
+ *   the same buffer to consecutive calls; flush and synchronise before freeing or reusing it. */
 size_t spkv_decode_step_staging_bytes(const spkv_config_t *cfg, int32_t B, int32_t d_in);
 int spkv_decode_step_host(spkv_cache_t *cache, int32_t layer, const spkv_predictor_t *pred,
                           const int32_t *d_seq_ids, int32_t B, const void *h_x, const void *h_q,
                           const void *h_k, const void *h_v, void *h_out, float sm_scale,
                           void *d_staging, size_t staging_bytes, spkv_stream_t stream);
+int spkv_decode_step_host_flush(spkv_cache_t *cache, spkv_stream_t stream);
 
 /* ---- introspection ----------------------------------------------------------------- */
 

@@ -111,6 +111,8 @@ extern "C" int spkv_cache_create(const spkv_config_t *cfg, void *d_arena, size_t
   c->last_layer = -1;
   c->last_stream = nullptr;
   c->ws_toggle = 0;
+  c->host_ready = false;
+  c->host_calls = 0;
   char *base = static_cast<char *>(d_arena);
   CacheView &v = c->view;
   v.L = cfg->n_layers; v.S = cfg->max_seqs; v.Hq = cfg->n_q_heads; v.Hkv = cfg->n_kv_heads;
@@ -158,6 +160,15 @@ extern "C" int spkv_cache_create(const spkv_config_t *cfg, void *d_arena, size_t
 
 extern "C" int spkv_cache_destroy(spkv_cache_t *cache) {
   if (!cache) return SPKV_E_INVALID;
+  if (cache->host_ready) {  // host-side objects of the host-buffer pipeline
+    for (int i = 0; i < 2; ++i) {
+      cudaEventDestroy(cache->ev_in[i]);
+      cudaEventDestroy(cache->ev_k[i]);
+      cudaEventDestroy(cache->ev_out[i]);
+    }
+    cudaStreamDestroy(cache->copy_in);
+    cudaStreamDestroy(cache->copy_out);
+  }
   delete cache;
   return SPKV_OK;
 }

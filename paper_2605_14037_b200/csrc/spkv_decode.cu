@@ -688,11 +688,36 @@ extern "C" int spkv_decode_attention_static(spkv_cache_t *cache, int32_t layer, 
 
 static size_t a256(size_t x) { return (x + 255) / 256 * 256; }
 
+// ---- decode step from host buffers: a two-slot pipeline over three streams ----------------
+//   copy_in : [wait kernels of call i-2]  x, q, k, v -> slot            record ev_in[slot]
+//   stream  : [wait ev_in[slot], ev_out[slot] of call i-2] score+append, decode   record ev_k[slot]
+//             [wait ev_out of call i-1]
+//   copy_out: [wait ev_k[slot]]  out -> host                            record ev_out[slot]
+// so the copies of one layer run under the kernels of its neighbours.  After call i the
+// caller's stream has waited for the output of call i-1; spkv_decode_step_host_flush makes it
+// wait for the last one.
+static size_t host_slot_bytes(const spkv_config_t *cfg, int32_t B, int32_t d_in) {
+  const size_t q = a256((size_t)B * cfg->n_q_heads * kD * 2), kv = a256((size_t)B * cfg->n_kv_heads * kD * 2);
+  return a256((size_t)B * d_in * 2) + 2 * q + 2 * kv + a256((size_t)B * cfg->n_kv_heads * 4);
+}
+
 extern "C" size_t spkv_decode_step_staging_bytes(const spkv_config_t *cfg, int32_t B, int32_t d_in) {
   if (!cfg || B < 0 || d_in < 0) return 0;
-  const size_t q = a256((size_t)B * cfg->n_q_heads * kD * 2), kv = a256((size_t)B * cfg->n_kv_heads * kD * 2);
-  return a256((size_t)B * d_in * 2) + 2 * q + 2 * kv + a256((size_t)B * cfg->n_kv_heads * 4) +
-         spkv_decode_workspace_bytes(cfg, B);
+  return 2 * host_slot_bytes(cfg, B, d_in) + spkv_decode_workspace_bytes(cfg, B);
+}
+
+static int host_pipeline_init(spkv_cache *c) {
+  if (c->host_ready) return SPKV_OK;
+  if (cudaStreamCreateWithFlags(&c->copy_in, cudaStreamNonBlocking) != cudaSuccess) return SPKV_E_CUDA;
+  if (cudaStreamCreateWithFlags(&c->copy_out, cudaStreamNonBlocking) != cudaSuccess) return SPKV_E_CUDA;
+  for (int i = 0; i < 2; ++i)
+    if (cudaEventCreateWithFlags(&c->ev_in[i], cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&c->ev_k[i], cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&c->ev_out[i], cudaEventDisableTiming) != cudaSuccess)
+      return SPKV_E_CUDA;
+  c->host_calls = 0;
+  c->host_ready = true;
+  return SPKV_OK;
 }
 
 extern "C" int spkv_decode_step_host(spkv_cache_t *cache, int32_t layer, const spkv_predictor_t *pred,
@@ -704,26 +729,52 @@ extern "C" int spkv_decode_step_host(spkv_cache_t *cache, int32_t layer, const s
   if (!d_staging || ((uintptr_t)d_staging & 255) ||
       staging_bytes < spkv_decode_step_staging_bytes(&cache->cfg, B, pred->d_in))
     return SPKV_E_WORKSPACE;
+  int rc = host_pipeline_init(cache);
+  if (rc) return rc;
   const spkv_config_t &cfg = cache->cfg;
   const size_t xb = (size_t)B * pred->d_in * 2, qb = (size_t)B * cfg.n_q_heads * kD * 2,
-               kvb = (size_t)B * cfg.n_kv_heads * kD * 2;
-  char *p = static_cast<char *>(d_staging);
+               kvb = (size_t)B * cfg.n_kv_heads * kD * 2, slot_bytes = host_slot_bytes(&cfg, B, pred->d_in);
+  const long long call = cache->host_calls++;
+  const int slot = (int)(call & 1);
+  char *p = static_cast<char *>(d_staging) + slot * slot_bytes;
   char *d_x = p; p += a256(xb);
   char *d_q = p; p += a256(qb);
   char *d_o = p; p += a256(qb);
   char *d_k = p; p += a256(kvb);
   char *d_v = p; p += a256(kvb);
-  float *d_lg = reinterpret_cast<float *>(p); p += a256((size_t)B * cfg.n_kv_heads * 4);
+  float *d_lg = reinterpret_cast<float *>(p);
+  void *d_ws = static_cast<char *>(d_staging) + 2 * slot_bytes;
   cudaStream_t s = as_stream(stream);
-  if (cudaMemcpyAsync(d_x, h_x, xb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-      cudaMemcpyAsync(d_q, h_q, qb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-      cudaMemcpyAsync(d_k, h_k, kvb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-      cudaMemcpyAsync(d_v, h_v, kvb, cudaMemcpyHostToDevice, s) != cudaSuccess)
+  // inputs: this slot was last read by the kernels of call - 2
+  if (call >= 2 && cudaStreamWaitEvent(cache->copy_in, cache->ev_k[slot], 0) != cudaSuccess) return SPKV_E_CUDA;
+  if (cudaMemcpyAsync(d_x, h_x, xb, cudaMemcpyHostToDevice, cache->copy_in) != cudaSuccess ||
+      cudaMemcpyAsync(d_q, h_q, qb, cudaMemcpyHostToDevice, cache->copy_in) != cudaSuccess ||
+      cudaMemcpyAsync(d_k, h_k, kvb, cudaMemcpyHostToDevice, cache->copy_in) != cudaSuccess ||
+      cudaMemcpyAsync(d_v, h_v, kvb, cudaMemcpyHostToDevice, cache->copy_in) != cudaSuccess ||
+      cudaEventRecord(cache->ev_in[slot], cache->copy_in) != cudaSuccess)
     return SPKV_E_CUDA;
-  int rc = spkv_score_append_evict(cache, layer, pred, d_seq_ids, B, d_x, d_k, d_v, d_lg, stream);
+  // kernels: after the inputs have landed and the slot's previous output has left
+  if (cudaStreamWaitEvent(s, cache->ev_in[slot], 0) != cudaSuccess) return SPKV_E_CUDA;
+  if (call >= 2 && cudaStreamWaitEvent(s, cache->ev_out[slot], 0) != cudaSuccess) return SPKV_E_CUDA;
+  rc = spkv_score_append_evict(cache, layer, pred, d_seq_ids, B, d_x, d_k, d_v, d_lg, stream);
   if (rc) return rc;
-  rc = spkv_decode_attention(cache, layer, d_seq_ids, B, d_q, d_o, nullptr, sm_scale, p,
+  rc = spkv_decode_attention(cache, layer, d_seq_ids, B, d_q, d_o, nullptr, sm_scale, d_ws,
                              spkv_decode_workspace_bytes(&cfg, B), stream);
   if (rc) return rc;
-  return check_stream_error(cudaMemcpyAsync(h_out, d_o, qb, cudaMemcpyDeviceToHost, s));
+  if (cudaEventRecord(cache->ev_k[slot], s) != cudaSuccess) return SPKV_E_CUDA;
+  // output
+  if (cudaStreamWaitEvent(cache->copy_out, cache->ev_k[slot], 0) != cudaSuccess ||
+      cudaMemcpyAsync(h_out, d_o, qb, cudaMemcpyDeviceToHost, cache->copy_out) != cudaSuccess ||
+      cudaEventRecord(cache->ev_out[slot], cache->copy_out) != cudaSuccess)
+    return SPKV_E_CUDA;
+  // the caller's stream answers for the output of the call before this one
+  if (call >= 1 && cudaStreamWaitEvent(s, cache->ev_out[slot ^ 1], 0) != cudaSuccess) return SPKV_E_CUDA;
+  return check_stream_error(cudaGetLastError());
+}
+
+extern "C" int spkv_decode_step_host_flush(spkv_cache_t *cache, spkv_stream_t stream) {
+  if (!cache) return SPKV_E_INVALID;
+  if (!cache->host_ready || cache->host_calls == 0) return SPKV_OK;
+  const int last = (int)((cache->host_calls - 1) & 1);
+  return check_stream_error(cudaStreamWaitEvent(as_stream(stream), cache->ev_out[last], 0));
 }

@@ -133,6 +133,11 @@ struct spkv_cache {
   int last_layer;
   cudaStream_t last_stream;
   int ws_toggle;        // decode workspace half used by the next decode launch
+  // spkv_decode_step_host: copy streams and events of its two-slot pipeline (made on first use)
+  cudaStream_t copy_in, copy_out;
+  cudaEvent_t ev_in[2], ev_k[2], ev_out[2];   // per slot: inputs landed, kernels done, output landed
+  long long host_calls;                        // calls so far; slot = call & 1
+  bool host_ready;
 };
 
 namespace spkv {

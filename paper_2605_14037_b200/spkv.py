@@ -84,6 +84,7 @@ def lib():
         "spkv_prefill": (C.c_int, [vp, i32, i32, i32, vp, vp, vp, vp, vp, f32, vp, sz, vp]),
         "spkv_decode_step_staging_bytes": (sz, [cfgp, i32, i32]),
         "spkv_decode_step_host": (C.c_int, [vp, i32, pp, vp, i32, vp, vp, vp, vp, vp, f32, vp, sz, vp]),
+        "spkv_decode_step_host_flush": (C.c_int, [vp, vp]),
         "spkv_status": (C.c_int, [vp, vp]),
         "spkv_clear_status": (C.c_int, [vp, vp]),
         "spkv_cache_stats": (C.c_int, [vp, vp, C.POINTER(Stats)]),
@@ -240,10 +241,16 @@ class Cache:
 
     def spkv_decode_step_host(self, layer, pred, seq_ids, h_x, h_q, h_k, h_v, h_out, sm_scale=None,
                               stream=None):
-        """Host (pinned) tensors in, host tensor out; enqueues copies + the three kernels."""
+        """Host (pinned) tensors in, host tensor out; enqueues the copies (on the cache's own
+        copy streams) and the kernels.  h_out is complete after spkv_decode_step_host_flush()
+        and a synchronisation of the stream."""
         B = seq_ids.numel()
         nbytes = lib().spkv_decode_step_staging_bytes(C.byref(self.cfg), B, pred.d_in)
-        st = self._workspace(("staging", layer), nbytes)
+        old = self._ws.get("staging")
+        if old is not None and old.numel() < nbytes:   # growing: drain the pipeline that uses the old one
+            self.spkv_decode_step_host_flush(stream)
+            torch.cuda.synchronize(self.device)
+        st = self._workspace("staging", nbytes)
         for t in (h_x, h_q, h_k, h_v, h_out):
             assert not t.is_cuda and t.is_contiguous() and t.dtype == torch.bfloat16
         _check(lib().spkv_decode_step_host(
@@ -252,6 +259,10 @@ class Cache:
             C.c_void_p(h_v.data_ptr()), C.c_void_p(h_out.data_ptr()),
             self.default_scale if sm_scale is None else sm_scale, _ptr(st), st.numel(),
             _stream(stream)), "spkv_decode_step_host")
+
+    def spkv_decode_step_host_flush(self, stream=None):
+        """Makes the stream wait for the output copy of the last spkv_decode_step_host call."""
+        _check(lib().spkv_decode_step_host_flush(self._h, _stream(stream)), "spkv_decode_step_host_flush")
 
     # -- maintenance / introspection ---------------------------------------------------
     def spkv_cache_reset_seq(self, seq, stream=None):

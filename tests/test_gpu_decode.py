@@ -10,6 +10,7 @@ import torch
 import oracle
 from gpu_util import D, Workload, assert_attn_close, dev, load, to_dev_bf16
 from paper_2605_14037_b200 import spkv as _unused  # noqa: F401  (fails loudly if the library is missing)
+from paper_2605_14037_b200 import synth
 
 pytestmark = pytest.mark.gpu
 
@@ -112,3 +113,40 @@ def test_decode_workspace_checked():
                                           C.c_void_p(q.data_ptr()), C.c_void_p(q.data_ptr()), None,
                                           0.1, None, 0, None)
     assert rc == -7
+
+
+def test_decode_step_host_pipeline_matches_device_calls():
+    """spkv_decode_step_host (pinned host buffers, copies on the cache's own streams, two
+    slots in flight) gives bit for bit what the device-pointer calls give, layer after layer
+    and step after step, and its outputs are complete after flush + synchronize."""
+    spkv = load()
+    rng = np.random.default_rng(91)
+    L, B, Hq, Hkv, d_in, w, steps = 3, 5, 8, 2, 64, 16, 40
+    mk = lambda: spkv.Cache(n_layers=L, max_seqs=B, n_q_heads=Hq, n_kv_heads=Hkv, max_context=512,
+                            pool_pages=L * B * Hkv * 2, window=w, tau=0.5)
+    ca, cb = mk(), mk()
+    tl = ca.spkv_tau_logit()
+    preds = []
+    for l in range(L):
+        W = synth.linear_predictor(rng, Hkv, d_in)
+        b = synth.bias_for_keep_rate(W, [0.3, 0.6], tl)
+        preds.append(spkv.make_predictor(to_dev_bf16(W), torch.from_numpy(b).to(dev())))
+    ids = torch.arange(B, dtype=torch.int32, device=dev())
+    bf = lambda shape: torch.from_numpy(synth.normal_bf16(rng, shape).view(np.int16)).view(torch.bfloat16)
+    for t in range(steps):
+        hx, hq = bf((L, B, d_in)).pin_memory(), bf((L, B, Hq, D)).pin_memory()
+        hk, hv = bf((L, B, Hkv, D)).pin_memory(), bf((L, B, Hkv, D)).pin_memory()
+        hout = torch.zeros((L, B, Hq, D), dtype=torch.bfloat16).pin_memory()
+        for l in range(L):
+            ca.spkv_decode_step_host(l, preds[l], ids, hx[l], hq[l], hk[l], hv[l], hout[l])
+        ca.spkv_decode_step_host_flush()
+        torch.cuda.current_stream().synchronize()
+        for l in range(L):
+            cb.spkv_score_append_evict(l, preds[l], ids, hx[l].to(dev()), hk[l].to(dev()), hv[l].to(dev()))
+            want = cb.spkv_decode_attention(l, ids, hq[l].to(dev())).cpu()
+            assert torch.equal(hout[l].view(torch.int16), want.view(torch.int16)), (t, l)
+    assert ca.spkv_status() == 0 and cb.spkv_status() == 0
+    for l in range(L):
+        la, _ = ca.spkv_read_lengths(l)
+        lb, _ = cb.spkv_read_lengths(l)
+        assert np.array_equal(la, lb)
