@@ -140,6 +140,16 @@ int spkv_cache_reset_seq(spkv_cache_t *cache, int32_t seq, spkv_stream_t stream)
  * changing the threshold; pairs already dropped stay dropped). */
 int spkv_set_tau(spkv_cache_t *cache, float tau);
 
+/* Static hybrid layouts (the paper's hand-designed local/global mixes, e.g. a 3:1 ratio of
+ * sliding-window to global heads): a (layer, KV head) may carry a threshold of its own, in
+ * force for its future evictions, on the stream given.  tau >= 1 makes the head local-only
+ * (window attention, nothing is ever kept: its compact cache and page table stay empty),
+ * tau <= 0 makes it a full-attention head, NaN returns it to the cache-wide threshold.
+ * kv_head = -1 addresses every KV head of the layer.  spkv_score's optional flags follow the
+ * cache-wide threshold only. */
+int spkv_set_head_tau(spkv_cache_t *cache, int32_t layer, int32_t kv_head, float tau,
+                      spkv_stream_t stream);
+
 /* ---- the hot path ------------------------------------------------------------------ */
 
 /* Step 1, score + threshold (Eq. 1-2).  d_x [n_tok, d_in] bf16 -> d_logits_out

@@ -75,7 +75,7 @@ append_evict_kernel(CacheView c, int layer, const int32_t *__restrict__ seq_ids,
     // the pair of position t - w leaves the window: threshold decision on its stored logit
     // (sink positions are kept regardless)
     const float lg = c.ring_logit[(size_t)u * c.w + slot];
-    if (lg >= tau_logit || t - c.w < c.n_sink) {
+    if (lg >= head_threshold(c, layer, kvh, tau_logit) || t - c.w < c.n_sink) {
       const int n = c.len[u];
       const int pj = n / kP, prow = n % kP;
       int page = -1, err = 0;

@@ -48,9 +48,16 @@ static void make_layout(const spkv_config_t *c, Layout *l) {
   l->off_free = o;   o = align_up(o + (size_t)c->pool_pages * 4, 256);
   l->off_pos = o;    o = align_up(o + (size_t)c->pool_pages * kP * 4, 256);
   l->off_rlogit = o; o = align_up(o + units * (size_t)c->window * 4, 256);
+  l->off_htau = o;   o = align_up(o + (size_t)c->n_layers * c->n_kv_heads * 4, 256);
   o = align_up(o, 1024);
   l->off_pages = o;  o += (units * ring_pages + (size_t)c->pool_pages) * kPageBytes;
   l->total = o;
+}
+
+// value = NaN clears the override
+__global__ void set_head_tau_kernel(float *head_tau, int first, int count, float value) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < count) head_tau[first + i] = value;
 }
 
 __global__ void init_free_stack_kernel(int32_t *stack, int32_t *free_top, int64_t pool_pages,
@@ -131,6 +138,7 @@ extern "C" int spkv_cache_create(const spkv_config_t *cfg, void *d_arena, size_t
   v.free_stack = reinterpret_cast<int32_t *>(base + l.off_free);
   v.pos_pool = reinterpret_cast<int32_t *>(base + l.off_pos);
   v.ring_logit = reinterpret_cast<float *>(base + l.off_rlogit);
+  v.head_tau = reinterpret_cast<float *>(base + l.off_htau);
   v.pages = reinterpret_cast<__nv_bfloat16 *>(base + l.off_pages);
 
   int dev = 0;
@@ -144,6 +152,10 @@ extern "C" int spkv_cache_create(const spkv_config_t *cfg, void *d_arena, size_t
   cudaStream_t s = as_stream(stream);
   // metadata and ring pages start at zero; pool pages are zeroed when first allocated
   cudaError_t e = cudaMemsetAsync(base, 0, l.off_pages + (size_t)v.n_ring_pages_total * kPageBytes, s);
+  if (e == cudaSuccess) {
+    const int nh = v.L * v.Hkv;
+    set_head_tau_kernel<<<(nh + 255) / 256, 256, 0, s>>>(v.head_tau, 0, nh, NAN);
+  }
   if (e == cudaSuccess && v.pool_pages > 0) {
     int64_t n = v.pool_pages;
     init_free_stack_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(v.free_stack, &v.status[1], n,
@@ -185,6 +197,18 @@ extern "C" int spkv_set_tau(spkv_cache_t *cache, float tau) {
   cache->cfg.tau = tau;
   cache->tau_logit = tau_to_logit(tau);
   return SPKV_OK;
+}
+
+extern "C" int spkv_set_head_tau(spkv_cache_t *cache, int32_t layer, int32_t kv_head, float tau,
+                                 spkv_stream_t stream) {
+  if (!cache || layer < 0 || layer >= cache->view.L || kv_head < -1 || kv_head >= cache->view.Hkv)
+    return SPKV_E_INVALID;
+  const float value = tau != tau ? NAN : tau_to_logit(tau);
+  const int first = layer * cache->view.Hkv + (kv_head < 0 ? 0 : kv_head);
+  const int count = kv_head < 0 ? cache->view.Hkv : 1;
+  cache->last_kind = kLastOther;
+  set_head_tau_kernel<<<1, 256, 0, as_stream(stream)>>>(cache->view.head_tau, first, count, value);
+  return check_stream_error(cudaGetLastError());
 }
 
 extern "C" float spkv_tau_logit(const spkv_cache_t *cache) { return cache ? cache->tau_logit : NAN; }
@@ -300,9 +324,10 @@ extern "C" int spkv_cache_stats(spkv_cache_t *cache, spkv_stream_t stream, spkv_
   const CacheView &v = cache->view;
   if (cudaStreamSynchronize(as_stream(stream)) != cudaSuccess) return SPKV_E_CUDA;
   std::vector<int32_t> t(v.n_units), len(v.n_units);
-  std::vector<float> lg((size_t)v.n_units * v.w);
+  std::vector<float> lg((size_t)v.n_units * v.w), htau((size_t)v.L * v.Hkv);
   int32_t hdr[2];
-  if (cudaMemcpy(t.data(), v.t, (size_t)v.n_units * 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
+  if (cudaMemcpy(htau.data(), v.head_tau, htau.size() * 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
+      cudaMemcpy(t.data(), v.t, (size_t)v.n_units * 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
       cudaMemcpy(len.data(), v.len, (size_t)v.n_units * 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
       cudaMemcpy(lg.data(), v.ring_logit, lg.size() * 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
       cudaMemcpy(hdr, v.status, 8, cudaMemcpyDeviceToHost) != cudaSuccess)
@@ -317,8 +342,10 @@ extern "C" int spkv_cache_stats(spkv_cache_t *cache, spkv_stream_t stream, spkv_
     out->pairs_evicted += t[u] > v.w ? t[u] - v.w : 0;
     out->pages_in_use += (len[u] + kP - 1) / kP;
     out->gates_open += len[u];
+    const float own = htau[(size_t)(u / (v.S * v.Hkv)) * v.Hkv + u % v.Hkv];  // unit = (layer * S + seq) * Hkv + kvh
+    const float thr = own != own ? cache->tau_logit : own;
     for (int s = 0; s < nw; ++s)
-      if (lg[(size_t)u * v.w + s] >= cache->tau_logit) out->gates_open++;
+      if (lg[(size_t)u * v.w + s] >= thr) out->gates_open++;
   }
   out->pages_free = hdr[1];
   out->bytes_resident = (out->pairs_kept + out->pairs_in_window) * 2 * kRowBytes;

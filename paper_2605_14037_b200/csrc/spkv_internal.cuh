@@ -8,6 +8,7 @@
 //   free_stack[]: LIFO of free pool pages (global page indices) int32 [pool_pages]
 //   pos_pool[]  : position of every kept pair, by pool page     int32 [pool_pages][P]
 //   ring_logit[]: stored logit per ring slot                    f32   [n_units][w]
+//   head_tau[]  : per-(layer, KV head) threshold override       f32   [L][Hkv]  (NaN: none)
 //   pages       : ring pages of every unit ([n_units][ring_pages]) followed by the pool
 //
 // A page holds P = 64 pairs: a 16 KB key block followed by a 16 KB value block.  Each
@@ -45,11 +46,12 @@ struct CacheView {
   int32_t *free_stack;
   int32_t *pos_pool;
   float *ring_logit;
+  float *head_tau;      // [L][Hkv] logit-space threshold of a (layer, KV head); NaN = the cache-wide one
   __nv_bfloat16 *pages;
 };
 
 struct Layout {
-  size_t off_header, off_t, off_len, off_table, off_free, off_pos, off_rlogit, off_pages, total;
+  size_t off_header, off_t, off_len, off_table, off_free, off_pos, off_rlogit, off_htau, off_pages, total;
 };
 
 // element offset of (row, 16-byte chunk) inside a key or value block
@@ -62,6 +64,12 @@ __device__ inline int unit_index(const CacheView &c, int layer, int seq, int kvh
 }
 
 __device__ inline void set_status(const CacheView &c, int code) { atomicCAS(c.status, 0, code); }
+
+// threshold in force for a (layer, KV head): its own if one was set, else the cache-wide one
+__device__ inline float head_threshold(const CacheView &c, int layer, int kvh, float tau_logit) {
+  const float own = c.head_tau[layer * c.Hkv + kvh];
+  return own != own ? tau_logit : own;
+}
 
 // global page index of ring page j of a unit
 __device__ inline int64_t ring_page(const CacheView &c, int unit, int j) {

@@ -38,6 +38,7 @@ __global__ void __launch_bounds__(1024) prefill_plan_kernel(PrefillArgs a) {
   int32_t *hdr = unit_ws(a, kvh);
   int32_t *E = hdr + kHdrInts;
   const int t0 = c.t[u], len0 = c.len[u];
+  const float thr = head_threshold(c, a.layer, kvh, a.tau_logit);
   const int n_old = min(t0, c.w), p0 = t0 - n_old;
   const int N = n_old + a.C;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -51,7 +52,7 @@ __global__ void __launch_bounds__(1024) prefill_plan_kernel(PrefillArgs a) {
     if (j < N) {
       const float lg = j < n_old ? c.ring_logit[(size_t)u * c.w + (p0 + j) % c.w]
                                  : a.logits[(size_t)(j - n_old) * c.Hkv + kvh];
-      flag = lg >= a.tau_logit || p0 + j < c.n_sink;  // Eq. 2 on the float32 logit; sink positions always
+      flag = lg >= thr || p0 + j < c.n_sink;  // Eq. 2 on the float32 logit; sink positions always
     }
     const unsigned ballot = __ballot_sync(0xffffffffu, flag);
     const int before = __popc(ballot & ((1u << lane) - 1u));

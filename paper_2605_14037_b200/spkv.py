@@ -74,6 +74,7 @@ def lib():
         "spkv_cache_destroy": (C.c_int, [vp]),
         "spkv_cache_reset_seq": (C.c_int, [vp, i32, vp]),
         "spkv_set_tau": (C.c_int, [vp, f32]),
+        "spkv_set_head_tau": (C.c_int, [vp, i32, i32, f32, vp]),
         "spkv_score": (C.c_int, [vp, pp, vp, i32, vp, vp, vp]),
         "spkv_append_evict": (C.c_int, [vp, i32, vp, i32, vp, vp, vp, vp]),
         "spkv_score_append_evict": (C.c_int, [vp, i32, pp, vp, i32, vp, vp, vp, vp, vp]),
@@ -270,6 +271,10 @@ class Cache:
 
     def spkv_set_tau(self, tau):
         _check(lib().spkv_set_tau(self._h, tau), "spkv_set_tau")
+
+    def spkv_set_head_tau(self, layer, kv_head, tau, stream=None):
+        """Threshold of one (layer, KV head) (kv_head = -1: the whole layer); NaN clears it."""
+        _check(lib().spkv_set_head_tau(self._h, layer, kv_head, tau, _stream(stream)), "spkv_set_head_tau")
 
     def spkv_tau_logit(self) -> float:
         return float(lib().spkv_tau_logit(self._h))
