@@ -113,13 +113,14 @@ struct Ranges {
   int nb;
   const int *cut;  // [nb + 1], non-decreasing, cut[0] = 0, cut[nb] = VP
   __device__ int start(int c) const { return cut[min(c, nb)]; }
-  __device__ int of_pos(int p) const {  // last block c with cut[c] <= p (its range is non-empty)
-    int lo = 0, hi = nb;
-    while (hi - lo > 1) {
-      const int mid = (lo + hi) >> 1;
-      if (cut[mid] <= p) lo = mid; else hi = mid;
-    }
-    return lo;
+  // last block c with cut[c] <= p (its range is non-empty).  The cuts sit within `snap` positions
+  // of c * VP / nb, so the proportional guess is off by a step or two at most.
+  __device__ int of_pos(int p) const {
+    const unsigned VP = (unsigned)cut[nb];
+    int c = min(nb - 1, (int)(((unsigned long long)(unsigned)p * (unsigned)nb) / VP));
+    while (c > 0 && cut[c] > p) --c;
+    while (c + 1 < nb && cut[c + 1] <= p) ++c;
+    return c;
   }
 };
 
@@ -139,6 +140,80 @@ __device__ inline bool wait_or_flag(uint64_t *bar, uint32_t parity, const CacheV
   if (mbar_wait_bounded(bar, parity)) return true;
   set_status(c, SPKV_E_TIMEOUT);
   return false;
+}
+
+// Epilogue warp: merge the consumer warps' (m, l, O) of one finished segment for all GG heads of
+// the group, fully unrolled so that every shared-memory load is issued before the first use
+// (a loop over the heads pays the load latency once per head and lets finished segments queue
+// up behind the epilogue warp when a block's range ends in several short units).
+template <int GG>
+__device__ inline void merge_warps(const float *red, int GP, int lane, float (&M)[GG], float (&Ls)[GG],
+                                   float4 (&Os)[GG]) {
+  float m[kConsumerWarps][GG], l[kConsumerWarps][GG];
+  float4 v[kConsumerWarps][GG];
+#pragma unroll
+  for (int w4 = 0; w4 < kConsumerWarps; ++w4)
+#pragma unroll
+    for (int gh = 0; gh < GG; ++gh) {
+      const float *src = red + ((size_t)w4 * GP + gh) * 132;
+      m[w4][gh] = src[128];
+      l[w4][gh] = src[129];
+      v[w4][gh] = *reinterpret_cast<const float4 *>(src + lane * 4);
+    }
+#pragma unroll
+  for (int gh = 0; gh < GG; ++gh) {
+    M[gh] = -INFINITY;
+#pragma unroll
+    for (int w4 = 0; w4 < kConsumerWarps; ++w4) M[gh] = fmaxf(M[gh], m[w4][gh]);
+    Ls[gh] = 0.f;
+    Os[gh] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int w4 = 0; w4 < kConsumerWarps; ++w4) {
+      const float f = m[w4][gh] == -INFINITY ? 0.f : fast_exp2(m[w4][gh] - M[gh]);
+      Ls[gh] += l[w4][gh] * f;
+      Os[gh].x += v[w4][gh].x * f; Os[gh].y += v[w4][gh].y * f;
+      Os[gh].z += v[w4][gh].z * f; Os[gh].w += v[w4][gh].w * f;
+    }
+  }
+}
+
+// Last-arriver merge of a unit whose (slot, head) partials number at most 16: every accumulator
+// load of the warp (one float4 per lane, slot and head) is issued before the first use, so the
+// merge costs one trip to L2 instead of one per pair of heads.  s_ml: the (m, l) pairs, slot-major.
+template <int GG>
+__device__ inline void merge_parts_fast(const float *g_acc /* + lane * 4 */, const float2 *s_ml, int nseg,
+                                        __nv_bfloat16 *out_rows /* head 0 of the group */, float *lse_rows,
+                                        int lane) {
+  constexpr int NS = 16 / GG;
+  float4 v[NS][GG];
+#pragma unroll
+  for (int si = 0; si < NS; ++si)
+#pragma unroll
+    for (int gh = 0; gh < GG; ++gh)
+      v[si][gh] = si < nseg ? __ldcg(reinterpret_cast<const float4 *>(g_acc + ((size_t)si * GG + gh) * kD))
+                            : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+  for (int gh = 0; gh < GG; ++gh) {
+    float mx = -INFINITY, ls = 0.f;
+    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int si = 0; si < NS; ++si)
+      if (si < nseg) mx = fmaxf(mx, s_ml[si * GG + gh].x);
+#pragma unroll
+    for (int si = 0; si < NS; ++si)
+      if (si < nseg) {
+        const float2 ml = s_ml[si * GG + gh];
+        const float f = fast_exp2(ml.x - mx);
+        ls += ml.y * f;
+        o.x += v[si][gh].x * f; o.y += v[si][gh].y * f; o.z += v[si][gh].z * f; o.w += v[si][gh].w * f;
+      }
+    const float inv = 1.f / ls;
+    uint2 pk;
+    pk.x = pack_bf16(o.x * inv, o.y * inv);
+    pk.y = pack_bf16(o.z * inv, o.w * inv);
+    *reinterpret_cast<uint2 *>(out_rows + (size_t)gh * kD + lane * 4) = pk;
+    if (lse_rows && lane == 0) lse_rows[gh] = (mx + log2f(ls)) * kLn2;
+  }
 }
 
 template <int NH>  // 8-head tiles on the N side: 1 for G <= 8, 2 for G <= 16
@@ -437,20 +512,8 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
 #ifdef SPKV_PHASE_TIMING
       const long long ec1 = clock64();
 #endif
-      for (int gh = 0; gh < a.G; ++gh) {
-        float M = -INFINITY;
-#pragma unroll
-        for (int w4 = 0; w4 < kConsumerWarps; ++w4) M = fmaxf(M, red[((size_t)w4 * GP + gh) * 132 + 128]);
-        float Ls = 0.f;
-        float4 Os = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-        for (int w4 = 0; w4 < kConsumerWarps; ++w4) {
-          const float *src = red + ((size_t)w4 * GP + gh) * 132;
-          const float f = src[128] == -INFINITY ? 0.f : fast_exp2(src[128] - M);
-          const float4 v = *reinterpret_cast<const float4 *>(src + lane * 4);
-          Ls += src[129] * f;
-          Os.x += v.x * f; Os.y += v.y * f; Os.z += v.z * f; Os.w += v.w * f;
-        }
+      // writes one head's merged result: the output if the unit lies inside this block, else a partial
+      auto emit = [&](int gh, float M, float Ls, const float4 &Os) {
         const size_t row = (size_t)b * c.Hq + kvh * a.G + gh;
         if (nseg == 1) {
           const float inv = 1.f / Ls;
@@ -465,6 +528,26 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
             a.part_ml[((size_t)slot * a.G + gh) * 2 + 0] = M;
             a.part_ml[((size_t)slot * a.G + gh) * 2 + 1] = Ls;
           }
+        }
+      };
+      if (a.G == 4) {
+        float M[4], Ls[4];
+        float4 Os[4];
+        merge_warps<4>(red, GP, lane, M, Ls, Os);
+#pragma unroll
+        for (int gh = 0; gh < 4; ++gh) emit(gh, M[gh], Ls[gh], Os[gh]);
+      } else if (a.G == 2) {
+        float M[2], Ls[2];
+        float4 Os[2];
+        merge_warps<2>(red, GP, lane, M, Ls, Os);
+#pragma unroll
+        for (int gh = 0; gh < 2; ++gh) emit(gh, M[gh], Ls[gh], Os[gh]);
+      } else {
+        for (int gh = 0; gh < a.G; ++gh) {
+          float M[1], Ls[1];
+          float4 Os[1];
+          merge_warps<1>(red + (size_t)gh * 132, GP, lane, M, Ls, Os);
+          emit(gh, M[0], Ls[0], Os[0]);
         }
       }
       __syncwarp();
@@ -505,8 +588,18 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
           const float2 *g_ml = reinterpret_cast<const float2 *>(a.part_ml) + (size_t)(c_first + item) * a.G;
           const float *g_acc = a.part_acc + (size_t)(c_first + item) * a.G * kD + lane * 4;
           auto ml_of = [&](int si, int gh) { return staged ? s_mrg[si * a.G + gh] : __ldcg(g_ml + si * a.G + gh); };
-          // two heads x eight slots at a time: 16 independent 16-byte loads in flight
-          for (int gh0 = 0; gh0 < a.G; gh0 += 2) {
+          const bool fast = staged && nseg * a.G <= 16 && (a.G == 1 || a.G == 2 || a.G == 4 || a.G == 8);
+          if (fast) {
+            const size_t row0 = (size_t)b * c.Hq + kvh * a.G;
+            __nv_bfloat16 *orow = a.out + row0 * kD;
+            float *lrow = a.lse ? a.lse + row0 : nullptr;
+            if (a.G == 4) merge_parts_fast<4>(g_acc, s_mrg, nseg, orow, lrow, lane);
+            else if (a.G == 8) merge_parts_fast<8>(g_acc, s_mrg, nseg, orow, lrow, lane);
+            else if (a.G == 2) merge_parts_fast<2>(g_acc, s_mrg, nseg, orow, lrow, lane);
+            else merge_parts_fast<1>(g_acc, s_mrg, nseg, orow, lrow, lane);
+          }
+          // general case: two heads x eight slots at a time, 16 independent 16-byte loads in flight
+          for (int gh0 = fast ? a.G : 0; gh0 < a.G; gh0 += 2) {
             float Mx[2], Ls[2];
             float4 Os[2];
 #pragma unroll
