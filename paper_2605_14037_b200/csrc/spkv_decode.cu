@@ -57,6 +57,8 @@ constexpr int kConsumerWarps = 8;  // two groups of four: group g takes the page
 constexpr int kTcThreads = (kConsumerWarps + 2) * 32;  // + producer warp + epilogue warp
 constexpr int kMaxStages = 8;
 constexpr int kMergeCap = 256;  // (slot, head) pairs staged in shared memory by a merge
+constexpr int kMergeGroup = 8;  // blocks per first-level merge group of a unit split over many blocks
+constexpr int kMaxMergeGroups = kMaxGrid / kMergeGroup;
 enum { F_BEGIN = 1, F_END = 2, F_STOP = 4 };
 
 struct StageMeta {  // valid rows (bits 0-7) | flags (8-11) | item (12+)
@@ -130,7 +132,7 @@ __device__ inline unsigned long long gtimer() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-#define SPKV_STAMP_T(i, cond) do { if (cond) reinterpret_cast<unsigned long long *>(a.part_acc + (size_t)300 * a.G * kD)[blockIdx.x * 16 + (i)] = gtimer(); } while (0)
+#define SPKV_STAMP_T(i, cond) do { if (cond) reinterpret_cast<unsigned long long *>(a.part_acc + (size_t)(148 + a.n_items) * a.G * kD)[blockIdx.x * 16 + (i)] = gtimer(); } while (0)
 #else
 #define SPKV_STAMP_T(i, cond)
 #endif
@@ -177,42 +179,41 @@ __device__ inline void merge_warps(const float *red, int GP, int lane, float (&M
   }
 }
 
-// Last-arriver merge of a unit whose (slot, head) partials number at most 16: every accumulator
-// load of the warp (one float4 per lane, slot and head) is issued before the first use, so the
-// merge costs one trip to L2 instead of one per pair of heads.  s_ml: the (m, l) pairs, slot-major.
+// Merge of `cnt` partial slots (slot si at row offset si * stride slots from g_acc) for all GG heads
+// of a group.  s_ml: the (m, l) pairs staged in shared memory, [cnt][GG].  The accumulator rows
+// are fetched 16 at a time with unconditional loads (indices past the end are clamped and get
+// weight 0), so every load of a round is in flight before the first use: a round costs one
+// trip to L2 whatever the shape.  Lane l owns dims 4l..4l+3.
 template <int GG>
-__device__ inline void merge_parts_fast(const float *g_acc /* + lane * 4 */, const float2 *s_ml, int nseg,
-                                        __nv_bfloat16 *out_rows /* head 0 of the group */, float *lse_rows,
-                                        int lane) {
+__device__ inline void merge_rows(const float *g_acc /* first slot, + lane * 4 */, const float2 *s_ml, int stride,
+                                  int cnt, float (&M)[GG], float (&L)[GG], float4 (&O)[GG]) {
   constexpr int NS = 16 / GG;
-  float4 v[NS][GG];
-#pragma unroll
-  for (int si = 0; si < NS; ++si)
-#pragma unroll
-    for (int gh = 0; gh < GG; ++gh)
-      v[si][gh] = si < nseg ? __ldcg(reinterpret_cast<const float4 *>(g_acc + ((size_t)si * GG + gh) * kD))
-                            : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
   for (int gh = 0; gh < GG; ++gh) {
-    float mx = -INFINITY, ls = 0.f;
-    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+    M[gh] = -INFINITY;
+    L[gh] = 0.f;
+    O[gh] = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  for (int si = 0; si < cnt; ++si)
 #pragma unroll
-    for (int si = 0; si < NS; ++si)
-      if (si < nseg) mx = fmaxf(mx, s_ml[si * GG + gh].x);
+    for (int gh = 0; gh < GG; ++gh) M[gh] = fmaxf(M[gh], s_ml[si * GG + gh].x);
+  for (int s0 = 0; s0 < cnt; s0 += NS) {
+    float4 v[NS][GG];
 #pragma unroll
-    for (int si = 0; si < NS; ++si)
-      if (si < nseg) {
-        const float2 ml = s_ml[si * GG + gh];
-        const float f = fast_exp2(ml.x - mx);
-        ls += ml.y * f;
-        o.x += v[si][gh].x * f; o.y += v[si][gh].y * f; o.z += v[si][gh].z * f; o.w += v[si][gh].w * f;
+    for (int x = 0; x < NS; ++x) {
+      const size_t row = (size_t)min(s0 + x, cnt - 1) * stride * GG;
+#pragma unroll
+      for (int gh = 0; gh < GG; ++gh) v[x][gh] = __ldcg(reinterpret_cast<const float4 *>(g_acc + (row + gh) * kD));
+    }
+#pragma unroll
+    for (int x = 0; x < NS; ++x)
+#pragma unroll
+      for (int gh = 0; gh < GG; ++gh) {
+        const float2 ml = s_ml[min(s0 + x, cnt - 1) * GG + gh];
+        const float f = (s0 + x < cnt && ml.x != -INFINITY) ? fast_exp2(ml.x - M[gh]) : 0.f;
+        L[gh] += ml.y * f;
+        O[gh].x += v[x][gh].x * f; O[gh].y += v[x][gh].y * f; O[gh].z += v[x][gh].z * f; O[gh].w += v[x][gh].w * f;
       }
-    const float inv = 1.f / ls;
-    uint2 pk;
-    pk.x = pack_bf16(o.x * inv, o.y * inv);
-    pk.y = pack_bf16(o.z * inv, o.w * inv);
-    *reinterpret_cast<uint2 *>(out_rows + (size_t)gh * kD + lane * 4) = pk;
-    if (lse_rows && lane == 0) lse_rows[gh] = (mx + log2f(ls)) * kLn2;
   }
 }
 
@@ -554,77 +555,100 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
       if (lane == 0) mbar_arrive(&red_empty[rb]);
 #ifdef SPKV_PHASE_TIMING
       if (lane == 0) {
-        unsigned long long *dbg = reinterpret_cast<unsigned long long *>(a.part_acc + (size_t)300 * a.G * kD);
+        unsigned long long *dbg = reinterpret_cast<unsigned long long *>(a.part_acc + (size_t)(148 + a.n_items) * a.G * kD);
         dbg[blockIdx.x * 16 + 6] += clock64() - ec0;
         dbg[blockIdx.x * 16 + 7] += 1;
         dbg[blockIdx.x * 16 + 2] += ec1 - ec0;
       }
 #endif
       if (nseg > 1) {
-        __threadfence();
-        __syncwarp();
-        int last = 0;
-        if (lane == 0) {
-          last = atomicAdd(&a.counters[item], 1) == nseg - 1;
-          if (last) a.counters[item] = 0;
-        }
-        last = __shfl_sync(0xffffffffu, last, 0);
-        if (last) {
-          __threadfence();
-          SPKV_STAMP_T(8, lane == 0);
-          // (m, l) of every slot and head go through shared memory first (one round of
-          // loads for the whole warp); the accumulator loads below are then independent
-          const int n_ml = nseg * a.G;
+        // Merge of `cnt` partial slots first, first + stride, ... of this unit (one warp; lane l owns
+        // dims 4l..4l+3).  dst_slot < 0: normalise and write the output rows; otherwise write the
+        // merged (m, l, O) back as a partial into dst_slot.
+        auto merge_slots = [&](int first, int stride, int cnt, int dst_slot) {
+          // (m, l) of every slot and head go through shared memory first (one round of loads for
+          // the whole warp); the accumulator loads below are then independent
+          const int n_ml = cnt * a.G;
           const bool staged = n_ml <= kMergeCap;
+          const float2 *g_ml = reinterpret_cast<const float2 *>(a.part_ml) + (size_t)first * a.G;
           if (staged) {
             for (int idx = lane; idx < n_ml; idx += 32)
-              s_mrg[idx] = __ldcg(reinterpret_cast<const float2 *>(a.part_ml) + (size_t)(c_first + item) * a.G + idx);
+              s_mrg[idx] = __ldcg(g_ml + (size_t)(idx / a.G) * stride * a.G + idx % a.G);
             __syncwarp();
           }
           SPKV_STAMP_T(9, lane == 0);
-#ifdef SPKV_PHASE_TIMING
-          if (lane == 0) reinterpret_cast<unsigned long long *>(a.part_acc + (size_t)300 * a.G * kD)[blockIdx.x * 16 + 10] = nseg;
-#endif
-          const float2 *g_ml = reinterpret_cast<const float2 *>(a.part_ml) + (size_t)(c_first + item) * a.G;
-          const float *g_acc = a.part_acc + (size_t)(c_first + item) * a.G * kD + lane * 4;
-          auto ml_of = [&](int si, int gh) { return staged ? s_mrg[si * a.G + gh] : __ldcg(g_ml + si * a.G + gh); };
-          const bool fast = staged && nseg * a.G <= 16 && (a.G == 1 || a.G == 2 || a.G == 4 || a.G == 8);
-          if (fast) {
-            const size_t row0 = (size_t)b * c.Hq + kvh * a.G;
-            __nv_bfloat16 *orow = a.out + row0 * kD;
-            float *lrow = a.lse ? a.lse + row0 : nullptr;
-            if (a.G == 4) merge_parts_fast<4>(g_acc, s_mrg, nseg, orow, lrow, lane);
-            else if (a.G == 8) merge_parts_fast<8>(g_acc, s_mrg, nseg, orow, lrow, lane);
-            else if (a.G == 2) merge_parts_fast<2>(g_acc, s_mrg, nseg, orow, lrow, lane);
-            else merge_parts_fast<1>(g_acc, s_mrg, nseg, orow, lrow, lane);
+          const float *g_acc = a.part_acc + (size_t)first * a.G * kD + lane * 4;
+          auto ml_of = [&](int si, int gh) {
+            return staged ? s_mrg[si * a.G + gh] : __ldcg(g_ml + ((size_t)si * stride) * a.G + gh);
+          };
+          const size_t row0 = (size_t)b * c.Hq + kvh * a.G;
+          // writes one head's merged (m, l, O): normalised output row, or a partial into dst_slot
+          auto put = [&](int gh, float Mx, float Ls, const float4 &Os) {
+            if (dst_slot < 0) {
+              const float inv = 1.f / Ls;
+              uint2 pk;
+              pk.x = pack_bf16(Os.x * inv, Os.y * inv);
+              pk.y = pack_bf16(Os.z * inv, Os.w * inv);
+              *reinterpret_cast<uint2 *>(a.out + (row0 + gh) * kD + lane * 4) = pk;
+              if (a.lse && lane == 0) a.lse[row0 + gh] = (Mx + log2f(Ls)) * kLn2;
+            } else {
+              *reinterpret_cast<float4 *>(a.part_acc + ((size_t)dst_slot * a.G + gh) * kD + lane * 4) = Os;
+              if (lane == 0) {
+                a.part_ml[((size_t)dst_slot * a.G + gh) * 2 + 0] = Mx;
+                a.part_ml[((size_t)dst_slot * a.G + gh) * 2 + 1] = Ls;
+              }
+            }
+          };
+          if (staged && (a.G == 1 || a.G == 2 || a.G == 4 || a.G == 8)) {
+            if (a.G == 4) {
+              float M[4], L[4]; float4 O[4];
+              merge_rows<4>(g_acc, s_mrg, stride, cnt, M, L, O);
+#pragma unroll
+              for (int gh = 0; gh < 4; ++gh) put(gh, M[gh], L[gh], O[gh]);
+            } else if (a.G == 8) {
+              float M[8], L[8]; float4 O[8];
+              merge_rows<8>(g_acc, s_mrg, stride, cnt, M, L, O);
+#pragma unroll
+              for (int gh = 0; gh < 8; ++gh) put(gh, M[gh], L[gh], O[gh]);
+            } else if (a.G == 2) {
+              float M[2], L[2]; float4 O[2];
+              merge_rows<2>(g_acc, s_mrg, stride, cnt, M, L, O);
+#pragma unroll
+              for (int gh = 0; gh < 2; ++gh) put(gh, M[gh], L[gh], O[gh]);
+            } else {
+              float M[1], L[1]; float4 O[1];
+              merge_rows<1>(g_acc, s_mrg, stride, cnt, M, L, O);
+              put(0, M[0], L[0], O[0]);
+            }
+            return;
           }
           // general case: two heads x eight slots at a time, 16 independent 16-byte loads in flight
-          for (int gh0 = fast ? a.G : 0; gh0 < a.G; gh0 += 2) {
+          for (int gh0 = 0; gh0 < a.G; gh0 += 2) {
             float Mx[2], Ls[2];
             float4 Os[2];
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
               Mx[h] = -INFINITY; Ls[h] = 0.f; Os[h] = make_float4(0.f, 0.f, 0.f, 0.f);
               if (gh0 + h < a.G)
-                for (int si = 0; si < nseg; ++si) Mx[h] = fmaxf(Mx[h], ml_of(si, gh0 + h).x);
+                for (int si = 0; si < cnt; ++si) Mx[h] = fmaxf(Mx[h], ml_of(si, gh0 + h).x);
             }
-            for (int s0 = 0; s0 < nseg; s0 += 8) {
+            for (int s0 = 0; s0 < cnt; s0 += 8) {
               float4 v[8][2];
 #pragma unroll
               for (int x = 0; x < 8; ++x)
 #pragma unroll
                 for (int h = 0; h < 2; ++h)
-                  v[x][h] = (s0 + x < nseg && gh0 + h < a.G)
+                  v[x][h] = (s0 + x < cnt && gh0 + h < a.G)
                                 ? __ldcg(reinterpret_cast<const float4 *>(
-                                      g_acc + ((size_t)(s0 + x) * a.G + gh0 + h) * kD))
+                                      g_acc + (((size_t)(s0 + x) * stride) * a.G + gh0 + h) * kD))
                                 : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
               for (int x = 0; x < 8; ++x)
 #pragma unroll
                 for (int h = 0; h < 2; ++h)
-                  if (s0 + x < nseg && gh0 + h < a.G) {
+                  if (s0 + x < cnt && gh0 + h < a.G) {
                     const float2 ml = ml_of(s0 + x, gh0 + h);
-                    const float f = fast_exp2(ml.x - Mx[h]);
+                    const float f = ml.x == -INFINITY ? 0.f : fast_exp2(ml.x - Mx[h]);
                     Ls[h] += ml.y * f;
                     Os[h].x += v[x][h].x * f; Os[h].y += v[x][h].y * f;
                     Os[h].z += v[x][h].z * f; Os[h].w += v[x][h].w * f;
@@ -632,17 +656,44 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
             }
 #pragma unroll
             for (int h = 0; h < 2; ++h)
-              if (gh0 + h < a.G) {
-                const size_t row = (size_t)b * c.Hq + kvh * a.G + gh0 + h;
-                const float inv = 1.f / Ls[h];
-                uint2 pk;
-                pk.x = pack_bf16(Os[h].x * inv, Os[h].y * inv);
-                pk.y = pack_bf16(Os[h].z * inv, Os[h].w * inv);
-                *reinterpret_cast<uint2 *>(a.out + row * kD + lane * 4) = pk;
-                if (a.lse && lane == 0) a.lse[row] = (Mx[h] + log2f(Ls[h])) * kLn2;
-              }
+              if (gh0 + h < a.G) put(gh0 + h, Mx[h], Ls[h], Os[h]);
           }
-          SPKV_STAMP_T(10, lane == 0);
+        };
+        // this block's arrival on a counter; true for the last of `target` arrivals (which also
+        // resets the counter for the next launch)
+        auto arrive_last = [&](int32_t *counter, int target) {
+          __threadfence();
+          __syncwarp();
+          int last = 0;
+          if (lane == 0) {
+            last = atomicAdd(counter, 1) == target - 1;
+            if (last) *counter = 0;
+          }
+          last = __shfl_sync(0xffffffffu, last, 0);
+          if (last) __threadfence();
+          return last != 0;
+        };
+        // A unit split over up to kMergeGroup blocks is merged by its last arriver.  A longer one
+        // (a near-full head at 128 K spans dozens of blocks) is merged on two levels, so that no
+        // single warp has to pull dozens of partials through its own few loads in flight: the
+        // parts form groups of kMergeGroup consecutive blocks, the last arriver of a group merges
+        // it into the group's first slot, and the last group to finish merges the group results.
+        const int first_slot = c_first + item, part = cidx - c_first;
+        if (nseg <= kMergeGroup) {
+          if (arrive_last(&a.counters[item], nseg)) {
+            SPKV_STAMP_T(8, lane == 0);
+            merge_slots(first_slot, 1, nseg, -1);
+            SPKV_STAMP_T(10, lane == 0);
+          }
+        } else {
+          const int g = part / kMergeGroup, n_groups = (nseg + kMergeGroup - 1) / kMergeGroup;
+          const int g_parts = min(kMergeGroup, nseg - g * kMergeGroup);
+          if (arrive_last(&a.group_counters[(size_t)item * kMaxMergeGroups + g], g_parts)) {
+            SPKV_STAMP_T(8, lane == 0);
+            if (g_parts > 1) merge_slots(first_slot + g * kMergeGroup, 1, g_parts, first_slot + g * kMergeGroup);
+            if (arrive_last(&a.counters[item], n_groups)) merge_slots(first_slot, kMergeGroup, n_groups, -1);
+            SPKV_STAMP_T(10, lane == 0);
+          }
         }
       }
     }
@@ -650,7 +701,7 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
   SPKV_STAMP_T(4, tid == 0);
 #ifdef SPKV_PHASE_TIMING
   if (tid == 0) {
-    unsigned long long *dbg = reinterpret_cast<unsigned long long *>(a.part_acc + (size_t)300 * a.G * kD);
+    unsigned long long *dbg = reinterpret_cast<unsigned long long *>(a.part_acc + (size_t)(148 + a.n_items) * a.G * kD);
     for (int i = 0; i < 5; ++i) dbg[blockIdx.x * 16 + 11 + i] = dbg_pages ? dbg_c[i] / dbg_pages : 0;
   }
 #endif
@@ -703,6 +754,7 @@ extern "C" int spkv_decode_attention(spkv_cache_t *cache, int32_t layer, const i
   cache->last_layer = layer;
   cache->last_stream = as_stream(stream);
   a.counters = reinterpret_cast<int32_t *>(ws);
+  a.group_counters = reinterpret_cast<int32_t *>(ws + wl.off_gcnt);
   a.part_ml = reinterpret_cast<float *>(ws + wl.off_ml);
   a.part_acc = reinterpret_cast<float *>(ws + wl.off_acc);
 
@@ -769,7 +821,8 @@ extern "C" int spkv_decode_attention_static(spkv_cache_t *cache, int32_t layer, 
   void *scratch = g_scratch_ptr[dev];
   if (B > 0) {
     // the array keeps whatever the previous call left: the arrival counters must start at zero
-    const size_t counters = (size_t)B * cache->cfg.n_kv_heads * 4;
+    const size_t counters =
+        decode_ws_layout(B * cache->cfg.n_kv_heads, cache->cfg.n_q_heads / cache->cfg.n_kv_heads).off_ml;
     for (int half = 0; half < 2; ++half)
       if (cudaMemsetAsync(static_cast<char *>(scratch) + half * (need / 2), 0, counters,
                           as_stream(stream)) != cudaSuccess)

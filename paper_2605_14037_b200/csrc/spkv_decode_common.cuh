@@ -20,6 +20,7 @@ struct DecodeArgs {
   float scale_log2;        // sm_scale * log2(e)
   int snap;                // range cuts within this many positions of a unit boundary move onto it
   int32_t *counters;       // [n_items] arrival counters
+  int32_t *group_counters; // [n_items][kMaxGrid / 8] arrival counters of the first-level merge groups
   float *part_ml;          // [slots][G][2]
   float *part_acc;         // [slots][G][128]
 };
@@ -66,12 +67,13 @@ __device__ inline void block_exclusive_scan(const int *s_np, int *s_pre, int n, 
 
 
 struct DecodeWs {
-  size_t off_ml, off_acc, total;
+  size_t off_gcnt, off_ml, off_acc, total;
 };
 inline DecodeWs decode_ws_layout(int n_items, int G) {
   DecodeWs w;
   const size_t slots = (size_t)kMaxSlots + n_items;
-  w.off_ml = ((size_t)(n_items + 2) * 4 + 255) / 256 * 256;
+  w.off_gcnt = ((size_t)(n_items + 2) * 4 + 255) / 256 * 256;
+  w.off_ml = w.off_gcnt + ((size_t)n_items * (kMaxGrid / 8) * 4 + 255) / 256 * 256;
   w.off_acc = w.off_ml + (slots * G * 2 * 4 + 255) / 256 * 256;
   w.total = w.off_acc + slots * G * kD * 4;
   return w;

@@ -150,3 +150,43 @@ def test_decode_step_host_pipeline_matches_device_calls():
         la, _ = ca.spkv_read_lengths(l)
         lb, _ = cb.spkv_read_lengths(l)
         assert np.array_equal(la, lb)
+
+
+@pytest.mark.parametrize("T", [40000, 8 * 64 * 20 + 70])
+def test_units_split_over_dozens_of_blocks_merge_on_two_levels(T):
+    """Two full-attention units of tens of thousands of pairs are the whole launch: each is cut
+    into dozens of block ranges, more than one first-level merge group holds, so the partial
+    results are merged group by group and then across groups.  Output and log-sum-exp against
+    the oracle; repeated launches are bit-identical (the counters reset themselves)."""
+    spkv = load()
+    rng = np.random.default_rng(5 + T)
+    w, Hq, Hkv, G, B, C = 128, 4, 1, 4, 2, 8192
+    cache = spkv.Cache(n_layers=1, max_seqs=B, n_q_heads=Hq, n_kv_heads=Hkv, max_context=T + 64,
+                       pool_pages=B * (T // 64 + 2), window=w, tau=-math.inf)
+    tl = cache.spkv_tau_logit()
+    K = synth.normal_bf16(rng, (B, T, Hkv, D))
+    V = synth.normal_bf16(rng, (B, T, Hkv, D))
+    q = synth.normal_bf16(rng, (B, Hq, D))
+    lg = torch.zeros((C, Hkv), dtype=torch.float32, device=dev())
+    units = []
+    for s in range(B):
+        Kd, Vd = to_dev_bf16(K[s]), to_dev_bf16(V[s])
+        for a in range(0, T, C):
+            n = min(C, T - a)
+            cache.spkv_prefill(0, s, Kd[a:a + n], Vd[a:a + n], lg[:n])
+        u = oracle.Unit(w, D)
+        u.prefill(np.ascontiguousarray(K[s, :, 0]), np.ascontiguousarray(V[s, :, 0]),
+                  np.zeros(T, np.float32), tl)
+        units.append(u)
+    ids = torch.arange(B, dtype=torch.int32, device=dev())
+    lse = torch.empty((B, Hq), dtype=torch.float32, device=dev())
+    scale = 1.0 / math.sqrt(D)
+    out = cache.spkv_decode_attention(0, ids, to_dev_bf16(q), lse=lse).clone()
+    again = cache.spkv_decode_attention(0, ids, to_dev_bf16(q))
+    assert torch.equal(out.view(torch.int16), again.view(torch.int16))
+    assert cache.spkv_status() == 0
+    got = spkv.bits_from_bf16(out)
+    for s in range(B):
+        ref, ref_lse = units[s].attend(q[s], scale, want_lse=True)
+        assert_attn_close(got[s], ref, f"long unit {s}")
+        assert np.abs(lse[s].cpu().numpy() - ref_lse).max() < 1e-3
