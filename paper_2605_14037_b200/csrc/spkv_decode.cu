@@ -702,7 +702,8 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
 #ifdef SPKV_PHASE_TIMING
   if (tid == 0) {
     unsigned long long *dbg = reinterpret_cast<unsigned long long *>(a.part_acc + (size_t)(148 + a.n_items) * a.G * kD);
-    for (int i = 0; i < 5; ++i) dbg[blockIdx.x * 16 + 11 + i] = dbg_pages ? dbg_c[i] / dbg_pages : 0;
+    for (int i = 0; i < 4; ++i) dbg[blockIdx.x * 16 + 11 + i] = dbg_pages ? dbg_c[i] / dbg_pages : 0;
+    { unsigned smid; asm volatile("mov.u32 %0, %%smid;" : "=r"(smid)); dbg[blockIdx.x * 16 + 15] = smid; }
   }
 #endif
   __syncthreads();
