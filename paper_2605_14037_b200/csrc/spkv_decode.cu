@@ -16,7 +16,10 @@
 // unit writes the output directly.  Otherwise it stores (m, l, acc) in workspace slot
 // (chunk + item) -- unique because consecutive segments differ in chunk or item -- and
 // bumps the unit's arrival counter; the block that arrives last merges all slots of the
-// unit by their log-sum-exp weights and resets the counter.  Nobody ever waits.
+// unit by their log-sum-exp weights and resets the counter.  A unit cut into more than
+// kMergeGroup ranges is merged on two levels: groups of kMergeGroup consecutive ranges, each
+// by the last arriver of the group into the group's first slot, then the group results by
+// the last group.  Nobody ever waits.
 //
 // Block = 8 consumer warps (two groups of four that take alternate pages, so that one group's
 // waits overlap the other's arithmetic) + producer warp + epilogue warp, one block per SM, a
