@@ -237,11 +237,15 @@ def run_ours(args):
         cache, preds, rates, gen = build_workload(spkv, synth, torch, cfg, dev, dense, total_steps, tau=tau)
         ids = torch.arange(B, dtype=torch.int32, device=dev)
         n_in = 4  # distinct q/k/v input sets cycled over the steps
-        q_in = torch.randn((n_in, L, B, Hq, 128), generator=gen, device=dev).to(torch.bfloat16)
-        k_in = torch.randn((n_in, L, B, Hkv, 128), generator=gen, device=dev).to(torch.bfloat16)
-        v_in = torch.randn((n_in, L, B, Hkv, 128), generator=gen, device=dev).to(torch.bfloat16)
+        # q, k, v of a step live in one flat buffer (one staging copy per step instead of three)
+        nq, nkv = L * B * Hq * 128, L * B * Hkv * 128
+        qkv_in = torch.randn((n_in, nq + 2 * nkv), generator=gen, device=dev).to(torch.bfloat16)
+        q_in = qkv_in[:, :nq].view(n_in, L, B, Hq, 128)
+        k_in = qkv_in[:, nq:nq + nkv].view(n_in, L, B, Hkv, 128)
+        v_in = qkv_in[:, nq + nkv:].view(n_in, L, B, Hkv, 128)
         x_all = torch.randn((total_steps, L, B, D_IN), generator=gen, device=dev).to(torch.bfloat16)
-        xs, qs, ks, vs = (torch.empty_like(t[0]) for t in (x_all, q_in, k_in, v_in))
+        xs, qkv = torch.empty_like(x_all[0]), torch.empty_like(qkv_in[0])
+        qs, ks, vs = qkv[:nq].view(L, B, Hq, 128), qkv[nq:nq + nkv].view(L, B, Hkv, 128), qkv[nq + nkv:].view(L, B, Hkv, 128)
         out = torch.empty((L, B, Hq, 128), dtype=torch.bfloat16, device=dev)
         logits = torch.empty((L, B, Hkv), dtype=torch.float32, device=dev)
         cache.decode_workspace(B)
@@ -249,7 +253,7 @@ def run_ours(args):
 
         def stage_inputs():
             s = step_no[0]
-            xs.copy_(x_all[s]); qs.copy_(q_in[s % n_in]); ks.copy_(k_in[s % n_in]); vs.copy_(v_in[s % n_in])
+            xs.copy_(x_all[s]); qkv.copy_(qkv_in[s % n_in])
             step_no[0] += 1
 
         def layer_calls(stream=None, events=None):
@@ -323,7 +327,7 @@ def run_ours(args):
 
         # end to end through the host-buffer entry point
         if not dense and e2e_steps > 0 and tau is None:
-            pin = lambda t: t.cpu().pin_memory()
+            pin = lambda t: t.contiguous().cpu().pin_memory()
             hx, hq, hk, hv = pin(x_all[:4]), pin(q_in), pin(k_in), pin(v_in)
             hout = torch.empty((L, B, Hq, 128), dtype=torch.bfloat16).pin_memory()
 
