@@ -547,7 +547,15 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
 #pragma unroll
         for (int gh = 0; gh < 2; ++gh) emit(gh, M[gh], Ls[gh], Os[gh]);
       } else {
-        for (int gh = 0; gh < a.G; ++gh) {
+        int gh = 0;
+        for (; gh + 4 <= a.G; gh += 4) {  // G = 8, 12, 16: four heads at a time
+          float M[4], Ls[4];
+          float4 Os[4];
+          merge_warps<4>(red + (size_t)gh * 132, GP, lane, M, Ls, Os);
+#pragma unroll
+          for (int x = 0; x < 4; ++x) emit(gh + x, M[x], Ls[x], Os[x]);
+        }
+        for (; gh < a.G; ++gh) {
           float M[1], Ls[1];
           float4 Os[1];
           merge_warps<1>(red + (size_t)gh * 132, GP, lane, M, Ls, Os);
@@ -571,6 +579,7 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
         auto merge_slots = [&](int first, int stride, int cnt, int dst_slot) {
           // (m, l) of every slot and head go through shared memory first (one round of loads for
           // the whole warp); the accumulator loads below are then independent
+          SPKV_STAMP_T(11, lane == 0);
           const int n_ml = cnt * a.G;
           const bool staged = n_ml <= kMergeCap;
           const float2 *g_ml = reinterpret_cast<const float2 *>(a.part_ml) + (size_t)first * a.G;
@@ -606,11 +615,13 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
             if (a.G == 4) {
               float M[4], L[4]; float4 O[4];
               merge_rows<4>(g_acc, s_mrg, stride, cnt, M, L, O);
+              SPKV_STAMP_T(12, lane == 0);
 #pragma unroll
               for (int gh = 0; gh < 4; ++gh) put(gh, M[gh], L[gh], O[gh]);
             } else if (a.G == 8) {
               float M[8], L[8]; float4 O[8];
               merge_rows<8>(g_acc, s_mrg, stride, cnt, M, L, O);
+              SPKV_STAMP_T(12, lane == 0);
 #pragma unroll
               for (int gh = 0; gh < 8; ++gh) put(gh, M[gh], L[gh], O[gh]);
             } else if (a.G == 2) {
@@ -694,6 +705,7 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
           if (arrive_last(&a.group_counters[(size_t)item * kMaxMergeGroups + g], g_parts)) {
             SPKV_STAMP_T(8, lane == 0);
             if (g_parts > 1) merge_slots(first_slot + g * kMergeGroup, 1, g_parts, first_slot + g * kMergeGroup);
+            SPKV_STAMP_T(13, lane == 0);
             if (arrive_last(&a.counters[item], n_groups)) merge_slots(first_slot, kMergeGroup, n_groups, -1);
             SPKV_STAMP_T(10, lane == 0);
           }
@@ -705,7 +717,6 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
 #ifdef SPKV_PHASE_TIMING
   if (tid == 0) {
     unsigned long long *dbg = reinterpret_cast<unsigned long long *>(a.part_acc + (size_t)(148 + a.n_items) * a.G * kD);
-    for (int i = 0; i < 4; ++i) dbg[blockIdx.x * 16 + 11 + i] = dbg_pages ? dbg_c[i] / dbg_pages : 0;
     { unsigned smid; asm volatile("mov.u32 %0, %%smid;" : "=r"(smid)); dbg[blockIdx.x * 16 + 15] = smid; }
   }
 #endif
