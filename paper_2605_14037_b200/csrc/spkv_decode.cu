@@ -676,15 +676,18 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
         // this block's arrival on a counter; true for the last of `target` arrivals (which also
         // resets the counter for the next launch)
         auto arrive_last = [&](int32_t *counter, int target) {
-          __threadfence();
+          // The warp's partial stores are ordered before lane 0's release by the warp barrier
+          // (release is cumulative), and the other lanes' later loads after its acquire the same
+          // way: one acq_rel atomic instead of fence + atomic + fence.
           __syncwarp();
           int last = 0;
           if (lane == 0) {
-            last = atomicAdd(counter, 1) == target - 1;
+            int old;
+            asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(counter) : "memory");
+            last = old == target - 1;
             if (last) *counter = 0;
           }
           last = __shfl_sync(0xffffffffu, last, 0);
-          if (last) __threadfence();
           return last != 0;
         };
         // A unit split over up to kMergeGroup blocks is merged by its last arriver.  A longer one
