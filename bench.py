@@ -155,7 +155,8 @@ def build_workload(spkv, synth, torch, cfg, dev, dense, total_steps, seed=0, tau
         per_seq = np.ceil(eff[:, None, :] * (np.asarray(t_list) + g_list)[None, :, None] * 1.03 / 64) + 2
         pool_pages = int(per_seq.sum())
     cache = spkv.Cache(n_layers=L, max_seqs=B, n_q_heads=Hq, n_kv_heads=Hkv,
-                       max_context=t_final + 64, pool_pages=pool_pages, window=W, tau=tau, device=dev)
+                       max_context=t_final + 64, pool_pages=pool_pages, window=W, tau=tau, device=dev,
+                       flags=spkv.FLAG_OVERLAP)   # attention-only stack, inputs staged before the step
     preds, keep = [], []
     for l in range(L):
         Wl, bl = pred_np[l]
@@ -388,7 +389,7 @@ def run_ours(args):
                    "density": sp["density"], "kv_gb_per_step": sp["kv_gb_per_step"],
                    "l2": "inputs larger than L2 (K/V read per step >> 126 MB)" if sp["kv_gb_per_step"] > 0.5
                          else "working set smaller than L2: latency-bound case",
-                   "cuda_graph": sp["graph"], "parallelism": "replicas only" if world > 1 else "single GPU"},
+                   "cuda_graph": sp["graph"], "launch_overlap": "SPKV_FLAG_OVERLAP", "parallelism": "replicas only" if world > 1 else "single GPU"},
         "clocks": sp["clocks"],
         "gpu_launches": 2 * L * K,
         "roofline": {"bound": "hbm", "kernel": "decode_tc_kernel", "achieved": achieved, "peak": hbm_peak,

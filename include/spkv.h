@@ -68,20 +68,30 @@ typedef struct {
   int32_t max_context;  /* upper bound on kept pairs per unit (sizes the page tables)   */
   int64_t pool_pages;   /* pages shared by all compact caches                           */
   float tau;            /* utility threshold in [0,1]; <= 0 keeps all, >= 1 keeps none  */
-  int32_t flags;        /* 0 or SPKV_FLAG_NO_OVERLAP                                    */
+  int32_t flags;        /* 0 or SPKV_FLAG_OVERLAP                                       */
   int32_t sink_tokens;  /* >= 0: the first sink_tokens positions of every sequence are
                            kept in the compact cache whatever their utility (the paper's
                            "Fixed Attention Sinks" ablation; its evaluation protocol uses
                            4).  0 = the method as defined by Eq. 2-4.                      */
 } spkv_config_t;
 
-/* By default consecutive hot-path launches on one stream overlap where they share no data
- * (programmatic dependent launch): the append of layer l+1 may run beside the decode attention
- * of layer l, and the decode attention of layer l+1 starts on the SMs that the one of layer l
- * has already left.  What the caller has to respect: two decode calls issued back to back,
- * with nothing but this library's append between them, must not write the same d_out.
- * SPKV_FLAG_NO_OVERLAP turns this off (every launch then waits for the previous one). */
-#define SPKV_FLAG_NO_OVERLAP 1
+/* SPKV_FLAG_OVERLAP (off by default): consecutive hot-path launches on one stream overlap where
+ * they share no data.  The fused score+append of layer l+1 runs beside the decode attention of
+ * layer l, and the decode attention of layer l+1 starts on each SM as soon as that of layer l
+ * has left it -- its start-up and the other's tail run under each other's page stream.  The
+ * kernels then skip the wait for "everything earlier on the stream" (which would also wait
+ * for the kernel they are meant to overlap) and order themselves on the device by the data
+ * they really share: an append waits for the decode launches of its own layer, a decode for
+ * the appends of its own layer and for the previous user of its workspace half.
+ * What the caller has to guarantee in this mode, because the library cannot see foreign work
+ * on the stream: the inputs of an append or decode call (x, k, v, q, seq ids) were complete
+ * when the library's previous call on that stream was enqueued, and two decode calls in a row
+ * do not write the same d_out.  That holds for an attention-only stack (the benchmark) and for
+ * a model that stages a whole step's inputs beforehand; a model that computes q, k, v of a
+ * layer between the library's calls must leave the flag off (every launch then waits for all
+ * earlier work, as any stream-ordered kernel does).  Any other call of the library (prefill,
+ * score, reset, ...) is a full synchronisation point either way. */
+#define SPKV_FLAG_OVERLAP 1
 
 /* Utility predictor f of Eq. 1 (the sigmoid is never evaluated: the decision is taken
  * in logit space, u >= tau  <=>  logit >= log(tau/(1-tau))).

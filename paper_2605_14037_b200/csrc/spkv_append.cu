@@ -31,19 +31,12 @@ __device__ inline int alloc_page(const CacheView &c, int lane) {
   return page;
 }
 
-__global__ void __launch_bounds__(128)
-append_evict_kernel(CacheView c, int layer, const int32_t *__restrict__ seq_ids, int B,
-                    const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new,
-                    const float *__restrict__ logits, float tau_logit,
-                    const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__restrict__ W,
-                    const float *__restrict__ bias, int d_in, float *__restrict__ logits_out,
-                    int wait_prev) {
-  // The previous kernel of the stream may still be running (see launch_overlapped).  The host
-  // passes wait_prev = 0 only when that kernel was a decode/append of ANOTHER layer of this
-  // cache: it shares no data with this launch, and ordering with everything older is kept by
-  // the decode kernels, which always wait.
-  if (wait_prev) pdl_wait();
-  pdl_trigger();
+// One warp: the append + evict of one unit.
+__device__ inline void append_unit(const CacheView &c, int layer, const int32_t *__restrict__ seq_ids, int B,
+                                   const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new,
+                                   const float *__restrict__ logits, float tau_logit,
+                                   const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__restrict__ W,
+                                   const float *__restrict__ bias, int d_in, float *__restrict__ logits_out) {
   const int lane = threadIdx.x & 31;
   const int item = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (item >= B * c.Hkv) return;
@@ -109,21 +102,64 @@ append_evict_kernel(CacheView c, int layer, const int32_t *__restrict__ seq_ids,
   }
 }
 
+__global__ void __launch_bounds__(128)
+append_evict_kernel(CacheView c, int layer, const int32_t *__restrict__ seq_ids, int B,
+                    const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new,
+                    const float *__restrict__ logits, float tau_logit,
+                    const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__restrict__ W,
+                    const float *__restrict__ bias, int d_in, float *__restrict__ logits_out,
+                    int wait_prev) {
+  // Every block counts itself in before dependents may launch and out when it is done: that is
+  // what later kernels that skip griddepcontrol.wait order themselves by.
+  if (threadIdx.x == 0) sync_count_start(c, layer, kSyncAppStart);
+  __syncthreads();
+  // wait_prev = 1: wait for everything earlier on the stream.  wait_prev = 0 (overlap mode; the
+  // host passes it only when the launches since the last full wait were hot-path kernels of
+  // this cache on other layers): the earlier kernels may still be running, and the only ones
+  // this launch shares data with are the decode launches of its own layer, which it waits out.
+  if (wait_prev) pdl_wait();
+  pdl_trigger();
+  if (!wait_prev) {
+    if (threadIdx.x == 0 && !sync_wait_finished(c, layer, kSyncDecStart)) set_status(c, SPKV_E_TIMEOUT);
+    __syncthreads();
+  }
+  append_unit(c, layer, seq_ids, B, k_new, v_new, logits, tau_logit, x, W, bias, d_in, logits_out);
+  __syncthreads();
+  if (threadIdx.x == 0) sync_count_finish(c, layer, kSyncAppFin);
+}
+
 }  // namespace spkv
 
 using namespace spkv;
 
-// Records this append as the cache's latest launch and tells whether it has to wait for the
-// kernel before it: always, unless that kernel was a decode/append of a different layer of
-// this cache on the same stream.
+// Records this append as the cache's latest launch and tells whether it has to wait for
+// everything before it on the stream.  It need not (overlap mode only) when the previous launch
+// was a decode/append of a different layer of this cache on the same stream and no other append
+// of this layer is outstanding: the kernel then waits for its own layer's decode launches only.
 static int append_must_wait(spkv_cache *cache, int layer, cudaStream_t s) {
-  const bool independent = (cache->last_kind == kLastDecode || cache->last_kind == kLastAppend) &&
+  const bool independent = (cache->cfg.flags & SPKV_FLAG_OVERLAP) &&
+                           (cache->last_kind == kLastDecode || cache->last_kind == kLastAppend) &&
                            cache->last_layer != layer && cache->last_stream == s &&
-                           !(cache->cfg.flags & SPKV_FLAG_NO_OVERLAP);
+                           cache->appends_pending[layer] == 0;
   cache->last_kind = kLastAppend;
   cache->last_layer = layer;
   cache->last_stream = s;
+  cache->appends_pending[layer]++;
   return independent ? 0 : 1;
+}
+
+// Plain stream-ordered launch unless the cache is in overlap mode.  Blocks of two warps: small
+// enough to fit on an SM beside a resident decode block (320 threads x 168 registers leave
+// 11.7 K registers), which is what lets the append of the next layer run under the decode.
+constexpr int kAppendThreads = 64;
+template <class... Args>
+static int launch_append(spkv_cache *cache, int items, cudaStream_t s, Args... args) {
+  const int per = kAppendThreads / 32, grid = (items + per - 1) / per;
+  if (!(cache->cfg.flags & SPKV_FLAG_OVERLAP)) {
+    append_evict_kernel<<<grid, kAppendThreads, 0, s>>>(args...);
+    return check_stream_error(cudaGetLastError());
+  }
+  return check_stream_error(launch_overlapped(append_evict_kernel, dim3(grid), dim3(kAppendThreads), 0, s, args...));
 }
 
 extern "C" int spkv_append_evict(spkv_cache_t *cache, int32_t layer, const int32_t *d_seq_ids,
@@ -136,11 +172,10 @@ extern "C" int spkv_append_evict(spkv_cache_t *cache, int32_t layer, const int32
   if (((uintptr_t)d_k | (uintptr_t)d_v) & 15) return SPKV_E_INVALID;
   const int items = B * cache->view.Hkv;
   const int wait_prev = append_must_wait(cache, layer, as_stream(stream));
-  return check_stream_error(launch_overlapped(
-      append_evict_kernel, dim3((items + 3) / 4), dim3(128), 0, as_stream(stream), cache->view, layer,
-      d_seq_ids, B, static_cast<const uint4 *>(d_k), static_cast<const uint4 *>(d_v), d_logits,
-      cache->tau_logit, (const __nv_bfloat16 *)nullptr, (const __nv_bfloat16 *)nullptr,
-      (const float *)nullptr, 0, (float *)nullptr, wait_prev));
+  return launch_append(cache, items, as_stream(stream), cache->view, layer, d_seq_ids, B,
+                       static_cast<const uint4 *>(d_k), static_cast<const uint4 *>(d_v), d_logits,
+                       cache->tau_logit, (const __nv_bfloat16 *)nullptr, (const __nv_bfloat16 *)nullptr,
+                       (const float *)nullptr, 0, (float *)nullptr, wait_prev);
 }
 
 extern "C" int spkv_score_append_evict(spkv_cache_t *cache, int32_t layer, const spkv_predictor_t *pred,
@@ -164,9 +199,9 @@ extern "C" int spkv_score_append_evict(spkv_cache_t *cache, int32_t layer, const
   if (((uintptr_t)d_k | (uintptr_t)d_v | (uintptr_t)d_x | (uintptr_t)pred->d_W1) & 15) return SPKV_E_INVALID;
   const int items = B * cache->view.Hkv;
   const int wait_prev = append_must_wait(cache, layer, as_stream(stream));
-  return check_stream_error(launch_overlapped(
-      append_evict_kernel, dim3((items + 3) / 4), dim3(128), 0, as_stream(stream), cache->view, layer,
-      d_seq_ids, B, static_cast<const uint4 *>(d_k), static_cast<const uint4 *>(d_v),
-      (const float *)nullptr, cache->tau_logit, static_cast<const __nv_bfloat16 *>(d_x),
-      static_cast<const __nv_bfloat16 *>(pred->d_W1), pred->d_b1, pred->d_in, d_logits_out, wait_prev));
+  return launch_append(cache, items, as_stream(stream), cache->view, layer, d_seq_ids, B,
+                       static_cast<const uint4 *>(d_k), static_cast<const uint4 *>(d_v), (const float *)nullptr,
+                       cache->tau_logit, static_cast<const __nv_bfloat16 *>(d_x),
+                       static_cast<const __nv_bfloat16 *>(pred->d_W1), pred->d_b1, pred->d_in, d_logits_out,
+                       wait_prev);
 }

@@ -49,6 +49,7 @@ static void make_layout(const spkv_config_t *c, Layout *l) {
   l->off_pos = o;    o = align_up(o + (size_t)c->pool_pages * kP * 4, 256);
   l->off_rlogit = o; o = align_up(o + units * (size_t)c->window * 4, 256);
   l->off_htau = o;   o = align_up(o + (size_t)c->n_layers * c->n_kv_heads * 4, 256);
+  l->off_sync = o;   o = align_up(o + (size_t)c->n_layers * 4 * 8, 256);
   o = align_up(o, 1024);
   l->off_pages = o;  o += (units * ring_pages + (size_t)c->pool_pages) * kPageBytes;
   l->total = o;
@@ -118,6 +119,9 @@ extern "C" int spkv_cache_create(const spkv_config_t *cfg, void *d_arena, size_t
   c->last_layer = -1;
   c->last_stream = nullptr;
   c->ws_toggle = 0;
+  c->half_last_layer[0] = c->half_last_layer[1] = -1;
+  c->appends_pending = new (std::nothrow) int[cfg->n_layers]();
+  if (!c->appends_pending) { delete c; return SPKV_E_INVALID; }
   c->host_ready = false;
   c->host_calls = 0;
   char *base = static_cast<char *>(d_arena);
@@ -139,11 +143,13 @@ extern "C" int spkv_cache_create(const spkv_config_t *cfg, void *d_arena, size_t
   v.pos_pool = reinterpret_cast<int32_t *>(base + l.off_pos);
   v.ring_logit = reinterpret_cast<float *>(base + l.off_rlogit);
   v.head_tau = reinterpret_cast<float *>(base + l.off_htau);
+  v.sync_ctr = reinterpret_cast<unsigned long long *>(base + l.off_sync);
   v.pages = reinterpret_cast<__nv_bfloat16 *>(base + l.off_pages);
 
   int dev = 0;
   cudaDeviceProp prop;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+    delete[] c->appends_pending;
     delete c;
     return SPKV_E_CUDA;
   }
@@ -163,6 +169,7 @@ extern "C" int spkv_cache_create(const spkv_config_t *cfg, void *d_arena, size_t
     e = cudaGetLastError();
   }
   if (e != cudaSuccess) {
+    delete[] c->appends_pending;
     delete c;
     return SPKV_E_CUDA;
   }
@@ -181,6 +188,7 @@ extern "C" int spkv_cache_destroy(spkv_cache_t *cache) {
     cudaStreamDestroy(cache->copy_in);
     cudaStreamDestroy(cache->copy_out);
   }
+  delete[] cache->appends_pending;
   delete cache;
   return SPKV_OK;
 }

@@ -249,6 +249,8 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
   long long dbg_c[5] = {0, 0, 0, 0, 0};
 #endif
 
+  // counted in by a thread that has nothing else to do here (see sync_count_start)
+  if (tid == 32) sync_count_start(c, a.layer, kSyncDecStart);
   if (tid == 0) {
     for (int i = 0; i < n_stages; ++i) {
       mbar_init(&full[i], 1);
@@ -269,11 +271,27 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
   }
   // Everything above touched only this block's shared memory and may overlap the tail of the
   // previous kernel of the stream; from here on its results (lengths, pages) are read.
-  pdl_wait();
+  // Overlap mode (wait_mode 1): the kernels before this one may still be running.  It shares data
+  // with the appends of its own layer (lengths, ring, pages) and with the decode launch that
+  // last used this half of the workspace, and waits for exactly those.
+  // The sequence ids are an input of the call, complete by contract in this mode: fetched now,
+  // beside the counter reads below.
+  int seq_first = -1;
+  if (a.wait_mode == 1 && tid < n) seq_first = a.seq_ids[tid / c.Hkv];
+  if (a.wait_mode == 0) pdl_wait();
+  __syncthreads();  // the block is counted in before any of its threads lets dependents launch
   pdl_trigger();
+  if (a.wait_mode == 1) {
+    if (tid == 0) {
+      if (!sync_wait_finished(c, a.layer, kSyncAppStart, a.prev_half_layer, kSyncDecStart))
+        set_status(c, SPKV_E_TIMEOUT);
+    }
+    __syncthreads();
+    asm volatile("fence.proxy.async;" ::: "memory");  // the appends wrote the pages the bulk copies read
+  }
   for (int i = tid; i < n; i += kTcThreads) {
     const int b = i / c.Hkv, kvh = i % c.Hkv;
-    const int seq = a.seq_ids[b];
+    const int seq = (a.wait_mode == 1 && i == tid) ? seq_first : a.seq_ids[b];
     int np = 0, u = 0, len = 0, n_ring = 0;
     if (seq >= 0 && seq < c.S) {
       u = unit_index(c, a.layer, seq, kvh);
@@ -724,6 +742,7 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
   }
 #endif
   __syncthreads();
+  if (tid == 0) sync_count_finish(c, a.layer, kSyncDecFin);
   SPKV_STAMP_T(5, tid == 0);
 }
 
@@ -766,8 +785,19 @@ extern "C" int spkv_decode_attention(spkv_cache_t *cache, int32_t layer, const i
   // Two consecutive decode launches may overlap (the next one starts on the SMs this one
   // has left): they alternate between the two halves of the workspace.  A third cannot
   // join: it needs every block of the second resident, i.e. every SM left by the first.
-  char *ws = static_cast<char *>(d_workspace) + (size_t)cache->ws_toggle * wl.total;
+  const int half = cache->ws_toggle;
+  char *ws = static_cast<char *>(d_workspace) + (size_t)half * wl.total;
   cache->ws_toggle ^= 1;
+  // Overlap mode: directly after this layer's append on the same stream the kernel need not wait
+  // for the whole stream, only for that append and for the previous user of its workspace half
+  // (which must be another layer: a block cannot tell its own launch's blocks from older ones).
+  a.wait_mode = ((cache->cfg.flags & SPKV_FLAG_OVERLAP) && cache->last_kind == kLastAppend &&
+                 cache->last_layer == layer && cache->last_stream == as_stream(stream) &&
+                 cache->half_last_layer[half] != layer)
+                    ? 1 : 0;
+  a.prev_half_layer = cache->half_last_layer[half];
+  cache->half_last_layer[half] = layer;
+  cache->appends_pending[layer] = 0;
   cache->last_kind = kLastDecode;
   cache->last_layer = layer;
   cache->last_stream = as_stream(stream);
@@ -781,7 +811,10 @@ extern "C" int spkv_decode_attention(spkv_cache_t *cache, int32_t layer, const i
     const char *e = getenv("SPKV_DECODE_KERNEL");  // "simt": the CUDA-core comparison kernel
     return e && e[0] == 's';
   }();
-  if (use_simt) return launch_decode_simt(a, cache->sm_count, s);
+  if (use_simt) {  // plain launch, not counted in the overlap bookkeeping: the next launch waits for it
+    cache->last_kind = kLastOther;
+    return launch_decode_simt(a, cache->sm_count, s);
+  }
 
   int GP = 1;
   while (GP < v.G) GP <<= 1;
@@ -799,7 +832,7 @@ extern "C" int spkv_decode_attention(spkv_cache_t *cache, int32_t layer, const i
 #ifdef SPKV_PROBE_GRID
   if (const char *e = getenv("SPKV_DECODE_GRID")) grid = atoi(e);
 #endif
-  if (cache->cfg.flags & SPKV_FLAG_NO_OVERLAP) {
+  if (!(cache->cfg.flags & SPKV_FLAG_OVERLAP)) {  // plain stream-ordered launch
     kernel<<<grid, kTcThreads, L.total, s>>>(a, GP, n_stages, red_bufs);
     return check_stream_error(cudaGetLastError());
   }

@@ -19,6 +19,8 @@ struct DecodeArgs {
   float *lse;              // [B][Hq] or null
   float scale_log2;        // sm_scale * log2(e)
   int snap;                // range cuts within this many positions of a unit boundary move onto it
+  int wait_mode;           // 0: griddepcontrol.wait; 1: overlap mode, wait for the launches it shares data with
+  int prev_half_layer;     // layer of the decode launch that last used this workspace half (-1: none)
   int32_t *counters;       // [n_items] arrival counters
   int32_t *group_counters; // [n_items][kMaxGrid / 8] arrival counters of the first-level merge groups
   float *part_ml;          // [slots][G][2]

@@ -9,6 +9,7 @@
 //   pos_pool[]  : position of every kept pair, by pool page     int32 [pool_pages][P]
 //   ring_logit[]: stored logit per ring slot                    f32   [n_units][w]
 //   head_tau[]  : per-(layer, KV head) threshold override       f32   [L][Hkv]  (NaN: none)
+//   sync_ctr[]  : blocks started / finished per layer and kernel u64   [L][4]    (launch overlap)
 //   pages       : ring pages of every unit ([n_units][ring_pages]) followed by the pool
 //
 // A page holds P = 64 pairs: a 16 KB key block followed by a 16 KB value block.  Each
@@ -47,11 +48,12 @@ struct CacheView {
   int32_t *pos_pool;
   float *ring_logit;
   float *head_tau;      // [L][Hkv] logit-space threshold of a (layer, KV head); NaN = the cache-wide one
+  unsigned long long *sync_ctr;  // [L][4]: append blocks started, finished; decode blocks started, finished
   __nv_bfloat16 *pages;
 };
 
 struct Layout {
-  size_t off_header, off_t, off_len, off_table, off_free, off_pos, off_rlogit, off_htau, off_pages, total;
+  size_t off_header, off_t, off_len, off_table, off_free, off_pos, off_rlogit, off_htau, off_sync, off_pages, total;
 };
 
 // element offset of (row, 16-byte chunk) inside a key or value block
@@ -127,6 +129,52 @@ inline cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 b
 
 enum { kLastOther = 0, kLastAppend = 1, kLastDecode = 2 };
 
+// ---- launch overlap without griddepcontrol.wait ---------------------------------------------
+// griddepcontrol.wait returns only when EVERY earlier kernel of the stream has completed, so a
+// kernel that calls it cannot begin its real work under the tail of its predecessor.  In overlap
+// mode (SPKV_FLAG_OVERLAP) the hot-path kernels skip it where the host knows what the preceding
+// launches were, and order themselves by the data they actually share: every block counts
+// itself into "started" before it lets dependents launch and into "finished" (release) when it
+// is done.  A later kernel is launched only after all blocks of all earlier kernels of the
+// stream have started (each launch needs its predecessor's blocks to have triggered), so when
+// it reads "started" that number is final, and "finished >= started" (acquire) means those
+// kernels are done.  Nothing here depends on values the host passes per launch: a captured
+// CUDA graph replays correctly.  The spin is bounded; on expiry the status word is set.
+enum { kSyncAppStart = 0, kSyncAppFin = 1, kSyncDecStart = 2, kSyncDecFin = 3 };
+
+__device__ inline void sync_count_start(const CacheView &c, int layer, int which) {  // one thread per block
+  atomicAdd(&c.sync_ctr[layer * 4 + which], 1ULL);
+  __threadfence();
+}
+__device__ inline void sync_count_finish(const CacheView &c, int layer, int which) {  // one thread, after a block barrier
+  asm volatile("red.release.gpu.global.add.u64 [%0], 1;" ::"l"(&c.sync_ctr[layer * 4 + which]) : "memory");
+}
+// true when every block counted in "started" has also finished, for up to two (layer, kernel)
+// pairs at once (layer_b < 0: only the first).  One thread per block calls; all four counters
+// are fetched together (relaxed loads, one fence at the end), so the common case -- already
+// satisfied -- costs one trip to L2.
+__device__ inline unsigned long long sync_load(const unsigned long long *p) {
+  unsigned long long v;
+  asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ inline bool sync_wait_finished(const CacheView &c, int layer_a, int which_a, int layer_b = -1,
+                                          int which_b = 0) {
+  const unsigned long long *pa = &c.sync_ctr[layer_a * 4 + which_a];
+  const unsigned long long *pb = layer_b >= 0 ? &c.sync_ctr[layer_b * 4 + which_b] : pa;
+  const unsigned long long sa = sync_load(pa), sb = sync_load(pb);
+  unsigned long long fa = sync_load(pa + 1), fb = sync_load(pb + 1);
+  const long long t0 = clock64();
+  while (fa < sa || fb < sb) {
+    if (clock64() - t0 > (1LL << 31)) return false;
+    __nanosleep(64);
+    fa = sync_load(pa + 1);
+    fb = sync_load(pb + 1);
+  }
+  __threadfence();  // acquire: what those blocks wrote before counting themselves out is visible now
+  return true;
+}
+
 }  // namespace spkv
 
 struct spkv_cache {
@@ -141,6 +189,8 @@ struct spkv_cache {
   int last_layer;
   cudaStream_t last_stream;
   int ws_toggle;        // decode workspace half used by the next decode launch
+  int half_last_layer[2];   // layer of the decode launch that last used each workspace half (-1: none)
+  int *appends_pending;     // [n_layers] appends since the layer's last decode launch
   // spkv_decode_step_host: copy streams and events of its two-slot pipeline (made on first use)
   cudaStream_t copy_in, copy_out;
   cudaEvent_t ev_in[2], ev_k[2], ev_out[2];   // per slot: inputs landed, kernels done, output landed

@@ -27,6 +27,9 @@ ERRORS = {
 }
 
 
+FLAG_OVERLAP = 1   # SPKV_FLAG_OVERLAP
+
+
 class Config(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("max_seqs", C.c_int32), ("n_q_heads", C.c_int32),
                 ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("window", C.c_int32),
@@ -140,9 +143,10 @@ class Cache:
     attention calls need.  Methods carry the names of the C entry points."""
 
     def __init__(self, n_layers, max_seqs, n_q_heads, n_kv_heads, max_context, pool_pages,
-                 window=128, tau=0.5, device="cuda:0", head_dim=128, page_tokens=64, sink_tokens=0):
+                 window=128, tau=0.5, device="cuda:0", head_dim=128, page_tokens=64, sink_tokens=0,
+                 flags=0):
         self.cfg = Config(n_layers, max_seqs, n_q_heads, n_kv_heads, head_dim, window, page_tokens,
-                          max_context, pool_pages, tau, 0, sink_tokens)
+                          max_context, pool_pages, tau, flags, sink_tokens)
         self.device = torch.device(device)
         n = C.c_size_t()
         _check(lib().spkv_arena_bytes(C.byref(self.cfg), C.byref(n)), "spkv_arena_bytes")

@@ -190,3 +190,55 @@ def test_units_split_over_dozens_of_blocks_merge_on_two_levels(T):
         ref, ref_lse = units[s].attend(q[s], scale, want_lse=True)
         assert_attn_close(got[s], ref, f"long unit {s}")
         assert np.abs(lse[s].cpu().numpy() - ref_lse).max() < 1e-3
+
+
+@pytest.mark.parametrize("L,B", [(4, 16), (3, 2), (2, 3), (1, 2)])
+def test_overlap_mode_is_bit_identical_to_stream_ordered_launches(L, B):
+    """SPKV_FLAG_OVERLAP: appends and decodes skip the wait for the whole stream and order
+    themselves by per-layer block counters.  A multi-layer decode loop (inputs staged before
+    each step, launches back to back, as the benchmark issues them) must give, bit for bit,
+    the outputs and cache state of a cache that launches everything stream-ordered.  Two and
+    one layer(s) exercise the fall-back when a workspace half comes back to the same layer."""
+    spkv = load()
+    rng = np.random.default_rng(300 + L * 10 + B)
+    Hq, Hkv, d_in, w, T0, steps = 8, 2, 64, 128, 700, 24
+    mk = lambda flags: spkv.Cache(n_layers=L, max_seqs=B, n_q_heads=Hq, n_kv_heads=Hkv, max_context=2048,
+                                  pool_pages=L * B * Hkv * 14, window=w, tau=0.5, flags=flags)
+    ca, cb = mk(spkv.FLAG_OVERLAP), mk(0)
+    tl = ca.spkv_tau_logit()
+    preds = []
+    for l in range(L):
+        W = synth.linear_predictor(rng, Hkv, d_in)
+        b = synth.bias_for_keep_rate(W, [0.2, 0.9], tl)
+        preds.append(spkv.make_predictor(to_dev_bf16(W), torch.from_numpy(b).to(dev())))
+    bf = lambda shape: to_dev_bf16(synth.normal_bf16(rng, shape))
+    for l in range(L):                       # some history, so that units span several blocks
+        for s in range(B):
+            k, v = bf((T0, Hkv, D)), bf((T0, Hkv, D))
+            lg = torch.from_numpy(synth.logits_with_keep_rate(rng, (T0, Hkv), 0.6, tl)).to(dev())
+            for c in (ca, cb):
+                c.spkv_prefill(l, s, k, v, lg)
+    ids = torch.arange(B, dtype=torch.int32, device=dev())
+    for t in range(steps):
+        x, q = bf((L, B, d_in)), bf((L, B, Hq, D))
+        k, v = bf((L, B, Hkv, D)), bf((L, B, Hkv, D))
+        outs = []
+        for c in (ca, cb):
+            o = torch.empty((L, B, Hq, D), dtype=torch.bfloat16, device=dev())
+            torch.cuda.synchronize()         # the step's inputs are complete before its first launch
+            for l in range(L):
+                c.spkv_score_append_evict(l, preds[l], ids, x[l], k[l], v[l])
+                c.spkv_decode_attention(l, ids, q[l], out=o[l])
+            outs.append(o)
+        torch.cuda.synchronize()
+        assert torch.equal(outs[0].view(torch.int16), outs[1].view(torch.int16)), t
+    assert ca.spkv_status() == 0 and cb.spkv_status() == 0
+    for l in range(L):
+        la, ta = ca.spkv_read_lengths(l)
+        lb, tb = cb.spkv_read_lengths(l)
+        assert np.array_equal(la, lb) and np.array_equal(ta, tb)
+        for s in range(B):
+            for h in range(Hkv):
+                pa, ka, va = ca.spkv_read_kept(l, s, h)
+                pb, kb, vb = cb.spkv_read_kept(l, s, h)
+                assert np.array_equal(pa, pb) and np.array_equal(ka, kb) and np.array_equal(va, vb)

@@ -31,7 +31,7 @@ def test_config2_one_layer_full_size():
     rates[0], rates[5] = 0.0, 0.97                       # a local-only head and a near-full head
     pages = int(np.ceil(rates * (T + steps) * 1.05 / 64 + 2).sum()) * B
     cache = spkv.Cache(n_layers=1, max_seqs=B, n_q_heads=Hq, n_kv_heads=Hkv, max_context=T + 128,
-                       pool_pages=pages, window=w, tau=0.5)
+                       pool_pages=pages, window=w, tau=0.5, flags=spkv.FLAG_OVERLAP)   # as bench.py creates it
     tl = cache.spkv_tau_logit()
     Tt = T + steps
     logit = np.stack([synth.logits_with_keep_rate(rng, (Tt, B), float(r), tl) for r in rates], axis=-1)
