@@ -147,16 +147,19 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
         const uint32_t sK = smem_u32(smem + kSKV + (jj % kStages) * kPageBytes);
         umma_qk_page<16384 / 16, 8192 / 16>(tbase + (2 * h + (jj & 1)) * 64, smem_desc(sQ + h * 32768, 16, 1024),
                                             smem_desc(sK, 16, 1024), idesc_qk);
-        umma_commit(&bar[B_S_FULL + 2 * h + (jj & 1)]);
-        TC5_STAMP(traced && lane == 0, 12 + 2 * h, jj);
+      };
+      auto commit_s = [&](int jj) {  // both heads' scores of page jj (each also covers the P.V before it)
+        umma_commit(&bar[B_S_FULL + 0 + (jj & 1)]);
+        umma_commit(&bar[B_S_FULL + 2 + (jj & 1)]);
       };
       // O_h += P_h(jj) . V(jj): A from tensor memory (hi in columns [0,32) of the S buffer the
       // scores came from, lo in [32,64)), B = the page's value block, MN-major
-      auto issue_pv = [&](int h, int jj) {
-        TC5_STAMP(traced && lane == 0 && h == 0, 15, jj);
-        if (!mbar_wait_bounded(&bar[B_P_FULL + 2 * h + (jj & 1)], (jj >> 1) & 1)) { failed = true; return; }
+      auto wait_p = [&](int h, int jj) {
+        if (!mbar_wait_bounded(&bar[B_P_FULL + 2 * h + (jj & 1)], (jj >> 1) & 1)) failed = true;
         TC5_STAMP(traced && lane == 0, 8 + h, jj);
         fence_after();
+      };
+      auto issue_pv = [&](int h, int jj) {
         const uint32_t sV = smem_u32(smem + kSKV + (jj % kStages) * kPageBytes) + kBlockElems * 2;
         const uint32_t tP = tbase + (2 * h + (jj & 1)) * 64;
         umma_pv_page(tbase + 256 + h * 128, tP, smem_desc(sV, 8192, 1024), idesc_pv, jj > 0 ? 1u : 0u);
@@ -174,16 +177,24 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
         if (failed) break;
         issue_qk(0, jj);
         issue_qk(1, jj);
+        commit_s(jj);
       }
+      // Both heads' P.V of a page, then both heads' Q.K^T of the page after next: one cluster of
+      // waits and commits per page instead of one per head and page (every wait or commit
+      // between two runs of MMAs lets the tensor pipe run dry for a few dozen clocks).
       for (int j = 0; j < n_tiles && !failed; ++j) {
-        for (int h = 0; h < 2 && !failed; ++h) {
-          issue_pv(h, j);
+        wait_p(0, j);
+        wait_p(1, j);
+        if (failed) break;
+        issue_pv(0, j);
+        issue_pv(1, j);
+        umma_commit(&bar[B_KV_EMPTY + (j % kStages)]);  // page j has no reader left
+        if (j + 2 < n_tiles) {
+          wait_page(j + 2);
           if (failed) break;
-          if (h == 1) umma_commit(&bar[B_KV_EMPTY + (j % kStages)]);  // page j has no reader left
-          if (j + 2 < n_tiles) {
-            if (h == 0) wait_page(j + 2);
-            if (!failed) issue_qk(h, j + 2);
-          }
+          issue_qk(0, j + 2);
+          issue_qk(1, j + 2);
+          commit_s(j + 2);
         }
       }
     }
