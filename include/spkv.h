@@ -269,6 +269,20 @@ int spkv_decode_step_host(spkv_cache_t *cache, int32_t layer, const spkv_predict
                           void *d_staging, size_t staging_bytes, spkv_stream_t stream);
 int spkv_decode_step_host_flush(spkv_cache_t *cache, spkv_stream_t stream);
 
+/* One decode step of the WHOLE layer stack from host buffers, for an attention-only stack whose
+ * inputs all exist before the step: four copies in, per layer score -> append/evict -> decode
+ * attention back to back on `stream` (in overlap mode nothing separates the launches), one copy
+ * out.  Everything is enqueued on `stream`; no synchronisation.
+ *   preds [n_layers] (host array, same d_in); h_x [L, B, d_in], h_q [L, B, n_q_heads, 128],
+ *   h_k/h_v [L, B, n_kv_heads, 128] bf16 -> h_out [L, B, n_q_heads, 128] bf16;
+ *   d_staging: >= spkv_decode_stack_staging_bytes(cfg, B, d_in) bytes, 256-byte aligned,
+ *   zero-filled once before first use. */
+size_t spkv_decode_stack_staging_bytes(const spkv_config_t *cfg, int32_t B, int32_t d_in);
+int spkv_decode_stack_host(spkv_cache_t *cache, const spkv_predictor_t *preds, const int32_t *d_seq_ids,
+                           int32_t B, const void *h_x, const void *h_q, const void *h_k, const void *h_v,
+                           void *h_out, float sm_scale, void *d_staging, size_t staging_bytes,
+                           spkv_stream_t stream);
+
 /* ---- introspection ----------------------------------------------------------------- */
 
 /* Synchronises `stream` and returns the sticky device status (SPKV_OK or the first

@@ -975,3 +975,64 @@ extern "C" int spkv_decode_step_host_flush(spkv_cache_t *cache, spkv_stream_t st
   const int last = (int)((cache->host_calls - 1) & 1);
   return check_stream_error(cudaStreamWaitEvent(as_stream(stream), cache->ev_out[last], 0));
 }
+
+// ---- one decode step of the WHOLE layer stack from host buffers ------------------------------
+// For an attention-only stack every layer's inputs exist before the step starts, so they go to
+// the device in four copies, the 2 L kernels follow back to back on the same stream (nothing
+// between them: in overlap mode each decode launch starts under the tail of the previous one,
+// which the per-layer entry point's event waits prevent), and one copy brings all outputs back.
+static size_t stack_inputs_bytes(const spkv_config_t *cfg, int32_t B, int32_t d_in, size_t *x, size_t *q, size_t *kv,
+                                 size_t *lg) {
+  *x = a256((size_t)cfg->n_layers * B * d_in * 2);
+  *q = a256((size_t)cfg->n_layers * B * cfg->n_q_heads * kD * 2);
+  *kv = a256((size_t)cfg->n_layers * B * cfg->n_kv_heads * kD * 2);
+  *lg = a256((size_t)cfg->n_layers * B * cfg->n_kv_heads * 4);
+  return *x + 2 * *q + 2 * *kv + *lg;
+}
+
+extern "C" size_t spkv_decode_stack_staging_bytes(const spkv_config_t *cfg, int32_t B, int32_t d_in) {
+  if (!cfg || B < 0 || d_in < 0) return 0;
+  size_t x, q, kv, lg;
+  return stack_inputs_bytes(cfg, B, d_in, &x, &q, &kv, &lg) + spkv_decode_workspace_bytes(cfg, B);
+}
+
+extern "C" int spkv_decode_stack_host(spkv_cache_t *cache, const spkv_predictor_t *preds, const int32_t *d_seq_ids,
+                                      int32_t B, const void *h_x, const void *h_q, const void *h_k, const void *h_v,
+                                      void *h_out, float sm_scale, void *d_staging, size_t staging_bytes,
+                                      spkv_stream_t stream) {
+  if (!cache || !preds || !h_x || !h_q || !h_k || !h_v || !h_out || B < 1) return SPKV_E_INVALID;
+  const spkv_config_t &cfg = cache->cfg;
+  const int L = cfg.n_layers, d_in = preds[0].d_in;
+  for (int l = 0; l < L; ++l)
+    if (preds[l].d_in != d_in) return SPKV_E_INVALID;
+  if (!d_staging || ((uintptr_t)d_staging & 255) || staging_bytes < spkv_decode_stack_staging_bytes(&cfg, B, d_in))
+    return SPKV_E_WORKSPACE;
+  size_t xb, qb, kvb, lgb;
+  stack_inputs_bytes(&cfg, B, d_in, &xb, &qb, &kvb, &lgb);
+  char *p = static_cast<char *>(d_staging);
+  char *d_x = p; p += xb;
+  char *d_q = p; p += qb;
+  char *d_o = p; p += qb;
+  char *d_k = p; p += kvb;
+  char *d_v = p; p += kvb;
+  float *d_lg = reinterpret_cast<float *>(p); p += lgb;
+  const size_t x_l = (size_t)B * d_in * 2, q_l = (size_t)B * cfg.n_q_heads * kD * 2,
+               kv_l = (size_t)B * cfg.n_kv_heads * kD * 2;
+  cudaStream_t s = as_stream(stream);
+  if (cudaMemcpyAsync(d_x, h_x, x_l * L, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+      cudaMemcpyAsync(d_q, h_q, q_l * L, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+      cudaMemcpyAsync(d_k, h_k, kv_l * L, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+      cudaMemcpyAsync(d_v, h_v, kv_l * L, cudaMemcpyHostToDevice, s) != cudaSuccess)
+    return SPKV_E_CUDA;
+  cache->last_kind = kLastOther;  // the first append waits for the copies
+  for (int l = 0; l < L; ++l) {
+    int rc = spkv_score_append_evict(cache, l, &preds[l], d_seq_ids, B, d_x + l * x_l, d_k + l * kv_l, d_v + l * kv_l,
+                                     d_lg + (size_t)l * B * cfg.n_kv_heads, stream);
+    if (rc) return rc;
+    rc = spkv_decode_attention(cache, l, d_seq_ids, B, d_q + l * q_l, d_o + l * q_l, nullptr, sm_scale, p,
+                               spkv_decode_workspace_bytes(&cfg, B), stream);
+    if (rc) return rc;
+  }
+  cache->last_kind = kLastOther;
+  return check_stream_error(cudaMemcpyAsync(h_out, d_o, q_l * L, cudaMemcpyDeviceToHost, s));
+}

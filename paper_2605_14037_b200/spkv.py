@@ -89,6 +89,8 @@ def lib():
         "spkv_decode_step_staging_bytes": (sz, [cfgp, i32, i32]),
         "spkv_decode_step_host": (C.c_int, [vp, i32, pp, vp, i32, vp, vp, vp, vp, vp, f32, vp, sz, vp]),
         "spkv_decode_step_host_flush": (C.c_int, [vp, vp]),
+        "spkv_decode_stack_staging_bytes": (sz, [cfgp, i32, i32]),
+        "spkv_decode_stack_host": (C.c_int, [vp, vp, vp, i32, vp, vp, vp, vp, vp, f32, vp, sz, vp]),
         "spkv_status": (C.c_int, [vp, vp]),
         "spkv_clear_status": (C.c_int, [vp, vp]),
         "spkv_cache_stats": (C.c_int, [vp, vp, C.POINTER(Stats)]),
@@ -264,6 +266,23 @@ class Cache:
             C.c_void_p(h_v.data_ptr()), C.c_void_p(h_out.data_ptr()),
             self.default_scale if sm_scale is None else sm_scale, _ptr(st), st.numel(),
             _stream(stream)), "spkv_decode_step_host")
+
+    def spkv_decode_stack_host(self, preds, seq_ids, h_x, h_q, h_k, h_v, h_out, sm_scale=None, stream=None):
+        """One decode step of all layers from host (pinned) tensors [L, B, ...]; enqueues four
+        copies in, the 2 L kernels and one copy out on the stream."""
+        B, L = seq_ids.numel(), self.cfg.n_layers
+        assert len(preds) == L
+        arr = (Predictor * L)(*preds)
+        nbytes = lib().spkv_decode_stack_staging_bytes(C.byref(self.cfg), B, preds[0].d_in)
+        st = self._workspace("stack_staging", nbytes)
+        for t in (h_x, h_q, h_k, h_v, h_out):
+            assert not t.is_cuda and t.is_contiguous() and t.dtype == torch.bfloat16 and t.shape[0] == L
+        _check(lib().spkv_decode_stack_host(
+            self._h, C.cast(arr, C.c_void_p), _ptr(seq_ids, torch.int32), B,
+            C.c_void_p(h_x.data_ptr()), C.c_void_p(h_q.data_ptr()), C.c_void_p(h_k.data_ptr()),
+            C.c_void_p(h_v.data_ptr()), C.c_void_p(h_out.data_ptr()),
+            self.default_scale if sm_scale is None else sm_scale, _ptr(st), st.numel(),
+            _stream(stream)), "spkv_decode_stack_host")
 
     def spkv_decode_step_host_flush(self, stream=None):
         """Makes the stream wait for the output copy of the last spkv_decode_step_host call."""

@@ -242,3 +242,34 @@ def test_overlap_mode_is_bit_identical_to_stream_ordered_launches(L, B):
                 pa, ka, va = ca.spkv_read_kept(l, s, h)
                 pb, kb, vb = cb.spkv_read_kept(l, s, h)
                 assert np.array_equal(pa, pb) and np.array_equal(ka, kb) and np.array_equal(va, vb)
+
+
+@pytest.mark.parametrize("flags", [0, 1])
+def test_decode_stack_host_matches_device_calls(flags):
+    """spkv_decode_stack_host (all layers' inputs copied in at once, kernels back to back, one
+    copy out) against the device-pointer calls, bit for bit, with and without overlap mode."""
+    spkv = load()
+    rng = np.random.default_rng(123 + flags)
+    L, B, Hq, Hkv, d_in, w, steps = 5, 3, 8, 2, 64, 16, 30
+    mk = lambda f: spkv.Cache(n_layers=L, max_seqs=B, n_q_heads=Hq, n_kv_heads=Hkv, max_context=512,
+                              pool_pages=L * B * Hkv * 2, window=w, tau=0.5, flags=f)
+    ca, cb = mk(flags), mk(0)
+    tl = ca.spkv_tau_logit()
+    preds = []
+    for l in range(L):
+        W = synth.linear_predictor(rng, Hkv, d_in)
+        b = synth.bias_for_keep_rate(W, [0.3, 0.6], tl)
+        preds.append(spkv.make_predictor(to_dev_bf16(W), torch.from_numpy(b).to(dev())))
+    ids = torch.arange(B, dtype=torch.int32, device=dev())
+    bf = lambda shape: torch.from_numpy(synth.normal_bf16(rng, shape).view(np.int16)).view(torch.bfloat16)
+    for t in range(steps):
+        hx, hq = bf((L, B, d_in)).pin_memory(), bf((L, B, Hq, D)).pin_memory()
+        hk, hv = bf((L, B, Hkv, D)).pin_memory(), bf((L, B, Hkv, D)).pin_memory()
+        hout = torch.zeros((L, B, Hq, D), dtype=torch.bfloat16).pin_memory()
+        ca.spkv_decode_stack_host(preds, ids, hx, hq, hk, hv, hout)
+        torch.cuda.current_stream().synchronize()
+        for l in range(L):
+            cb.spkv_score_append_evict(l, preds[l], ids, hx[l].to(dev()), hk[l].to(dev()), hv[l].to(dev()))
+            want = cb.spkv_decode_attention(l, ids, hq[l].to(dev())).cpu()
+            assert torch.equal(hout[l].view(torch.int16), want.view(torch.int16)), (t, l)
+    assert ca.spkv_status() == 0 and cb.spkv_status() == 0
