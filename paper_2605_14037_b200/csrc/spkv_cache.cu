@@ -120,6 +120,8 @@ extern "C" int spkv_cache_create(const spkv_config_t *cfg, void *d_arena, size_t
   c->last_stream = nullptr;
   c->ws_toggle = 0;
   c->half_last_layer[0] = c->half_last_layer[1] = -1;
+  c->last_decode_items = -1;
+  c->last_decode_ws = nullptr;
   c->appends_pending = new (std::nothrow) int[cfg->n_layers]();
   if (!c->appends_pending) { delete c; return SPKV_E_INVALID; }
   c->host_ready = false;

@@ -793,8 +793,12 @@ extern "C" int spkv_decode_attention(spkv_cache_t *cache, int32_t layer, const i
   // (which must be another layer: a block cannot tell its own launch's blocks from older ones).
   a.wait_mode = ((cache->cfg.flags & SPKV_FLAG_OVERLAP) && cache->last_kind == kLastAppend &&
                  cache->last_layer == layer && cache->last_stream == as_stream(stream) &&
-                 cache->half_last_layer[half] != layer)
+                 cache->half_last_layer[half] != layer &&
+                 // same workspace, cut into the same halves, as the launch it may run beside
+                 cache->last_decode_items == n_items && cache->last_decode_ws == d_workspace)
                     ? 1 : 0;
+  cache->last_decode_items = n_items;
+  cache->last_decode_ws = d_workspace;
   a.prev_half_layer = cache->half_last_layer[half];
   cache->half_last_layer[half] = layer;
   cache->appends_pending[layer] = 0;

@@ -190,6 +190,8 @@ struct spkv_cache {
   cudaStream_t last_stream;
   int ws_toggle;        // decode workspace half used by the next decode launch
   int half_last_layer[2];   // layer of the decode launch that last used each workspace half (-1: none)
+  int last_decode_items;    // units of the previous decode launch (the workspace halves depend on it)
+  void *last_decode_ws;     // and its workspace
   int *appends_pending;     // [n_layers] appends since the layer's last decode launch
   // spkv_decode_step_host: copy streams and events of its two-slot pipeline (made on first use)
   cudaStream_t copy_in, copy_out;
