@@ -279,16 +279,14 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
   int seq_first = -1;
   if (a.wait_mode == 1 && tid < n) seq_first = a.seq_ids[tid / c.Hkv];
   if (a.wait_mode == 0) pdl_wait();
+  // (the counter reads run beside thread 32's count-in: one trip to L2 for both)
+  if (a.wait_mode == 1 && tid == 0 &&
+      !sync_wait_finished(c, a.layer, kSyncAppStart, a.prev_half_layer, kSyncDecStart))
+    set_status(c, SPKV_E_TIMEOUT);
   __syncthreads();  // the block is counted in before any of its threads lets dependents launch
   pdl_trigger();
-  if (a.wait_mode == 1) {
-    if (tid == 0) {
-      if (!sync_wait_finished(c, a.layer, kSyncAppStart, a.prev_half_layer, kSyncDecStart))
-        set_status(c, SPKV_E_TIMEOUT);
-    }
-    __syncthreads();
+  if (a.wait_mode == 1)
     asm volatile("fence.proxy.async;" ::: "memory");  // the appends wrote the pages the bulk copies read
-  }
   for (int i = tid; i < n; i += kTcThreads) {
     const int b = i / c.Hkv, kvh = i % c.Hkv;
     const int seq = (a.wait_mode == 1 && i == tid) ? seq_first : a.seq_ids[b];
