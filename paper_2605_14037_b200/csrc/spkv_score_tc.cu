@@ -5,11 +5,13 @@
 //   A = SiLU(Z + b1)                      epilogue threads (thread = token = TMEM lane)
 //   logit = A W2^T + b2 [n_tok, n_kv_heads], flag = logit >= tau_logit (Eq. 2)
 //
-// One block = 128 tokens x all hidden units (hidden <= 256 = one accumulator tile).  X and W1
+// One block = 128 tokens x all hidden units (hidden <= 256 = one accumulator tile), or -- when
+// the chunk has fewer token tiles than the GPU has SMs -- a cluster of two blocks that share the
+// tokens and take half of the hidden units each (see the kernel).  X and W1
 // are row-major with the contraction dimension innermost, i.e. K-major operands as they are: a
 // TMA tile load (64 dims x rows, 128-byte swizzle) puts them in shared memory in operand layout.
-// Rows past n_tok and dims past d_in are zero-filled by the TMA unit.  4-stage mbarrier
-// pipeline: warp 4 = TMA producer, warp 5 = MMA issue (whole warp, one elected lane), warps 0-3
+// Rows past n_tok and dims past d_in are zero-filled by the TMA unit.  192 KB mbarrier
+// pipeline (4 stages of 48 KB, or 6 of 32 KB): warp 4 = TMA producer, warp 5 = MMA issue (whole warp, one elected lane), warps 0-3
 // = epilogue.  Traffic: n_tok * d_in * 2 B of activations from HBM once; W1 (hidden * d_in * 2 B)
 // is re-read per block from L2.  All waits are bounded.
 #include <cuda.h>
@@ -24,25 +26,48 @@ namespace sctc {
 constexpr int kThreads = 192;
 constexpr int kTok = 128;      // tokens per block (MMA M)
 constexpr int kKC = 64;        // dims per pipeline stage (one 128-byte swizzle row)
-constexpr int kStages = 4;
 constexpr int kMaxHidden = 256;
 constexpr int kABytes = kTok * kKC * 2;            // 16 KB
-constexpr int kBBytesMax = kMaxHidden * kKC * 2;   // 32 KB
-constexpr int kStageBytes = kABytes + kBBytesMax;  // 48 KB
+constexpr int kBBytesMax = kMaxHidden * kKC * 2;   // 32 KB (16 KB when the hidden units are split over two blocks)
+constexpr int kPipeBytes = 4 * (kABytes + kBBytesMax);  // 192 KB: 4 stages of 48 KB, or 6 of 32 KB
+constexpr int kMaxStages = 6;
 constexpr int kMaxW2Floats = 4096;                 // hidden x (n_kv_heads rounded up to 8)
-constexpr int kSW2 = kStages * kStageBytes;        // [hidden][heads8] fp32
+constexpr int kSW2 = kPipeBytes;                   // [hidden][heads8] fp32
 constexpr int kSB1 = kSW2 + kMaxW2Floats * 4;      // [hidden] fp32
-constexpr int kSBar = kSB1 + kMaxHidden * 4;
+constexpr int kSPart = kSB1 + kMaxHidden * 4;      // split only: [2][128][heads8 <= 16] fp32 partial logits
+constexpr int kSBar = kSPart + 2 * kTok * 16 * 4;
 constexpr int kSmemBytes = kSBar + 128;
-enum { B_FULL = 0, B_EMPTY = 4, B_ACC = 8, B_COUNT = 9 };
+enum { B_FULL = 0, B_EMPTY = kMaxStages, B_ACC = 2 * kMaxStages, B_COUNT = 2 * kMaxStages + 1 };
 
 __device__ inline void tma_load_2d(void *smem_dst, const CUtensorMap *map, int x, int y, uint64_t *bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
 }
+__device__ inline uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// float store into the same shared-memory location of another block of the cluster
+__device__ inline void st_cluster_f32(const float *local_addr, uint32_t rank, float v) {
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(local_addr)), "r"(rank));
+  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
+}
+__device__ inline void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 }  // namespace sctc
 
+// kSplit = 1: one block computes all hidden units of its 128 tokens.  kSplit = 2: a cluster of two
+// blocks shares the tokens, each takes half of the hidden units (its own half of W1, the same X
+// tile -- the second read comes from L2), and block 1 hands its partial logits to block 0 through
+// distributed shared memory.  Twice the blocks, two thirds of the bytes per block and six
+// stages in flight instead of four: the kernel is bound by load latency x bytes in flight per
+// SM and by the number of blocks (a chunk of 8192 tokens is only 64 token tiles on 148 SMs).
+template <int kSplit>
 __global__ void __launch_bounds__(sctc::kThreads, 1)
 score_mlp_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w1, int n_tok,
                     int d_in, int hidden, const float *__restrict__ b1, const __nv_bfloat16 *__restrict__ W2,
@@ -50,12 +75,17 @@ score_mlp_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
                     uint8_t *__restrict__ flags, int32_t *status) {
   using namespace tc5;
   using namespace sctc;
+  constexpr int kStages = kSplit == 2 ? 6 : 4;
+  constexpr int kStageBytes = kPipeBytes / kStages;
   extern __shared__ __align__(1024) unsigned char smem[];
   uint64_t *bar = reinterpret_cast<uint64_t *>(smem + kSBar);
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + kSBar + B_COUNT * 8);
   float *w2s = reinterpret_cast<float *>(smem + kSW2), *b1s = reinterpret_cast<float *>(smem + kSB1);
+  float *part = reinterpret_cast<float *>(smem + kSPart);  // [0]: this block's, [1]: the partner's partial logits
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int tok0 = blockIdx.x * kTok, n_kc = (d_in + kKC - 1) / kKC, heads8 = (Hkv + 7) & ~7;
+  const int rank = kSplit == 2 ? (int)cluster_rank() : 0;
+  const int hl = hidden / kSplit, j_off = rank * hl;  // this block's hidden units
+  const int tok0 = (blockIdx.x / kSplit) * kTok, n_kc = (d_in + kKC - 1) / kKC, heads8 = (Hkv + 7) & ~7;
 
   if (tid == 0) {
     for (int i = 0; i < kStages; ++i) {
@@ -66,11 +96,11 @@ score_mlp_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
     mbar_fence_init();
   }
   // second layer, transposed and padded: w2s[j][h] (zero for h >= Hkv), and the first bias
-  for (int x = tid; x < hidden * heads8; x += kThreads) {
+  for (int x = tid; x < hl * heads8; x += kThreads) {
     const int j = x / heads8, h = x % heads8;
-    w2s[x] = h < Hkv ? __bfloat162float(W2[(size_t)h * hidden + j]) : 0.f;
+    w2s[x] = h < Hkv ? __bfloat162float(W2[(size_t)h * hidden + j_off + j]) : 0.f;
   }
-  for (int x = tid; x < hidden; x += kThreads) b1s[x] = b1[x];
+  for (int x = tid; x < hl; x += kThreads) b1s[x] = b1[j_off + x];
   if (warp == 4) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 256;" ::"r"(smem_u32(tmem_slot)) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -84,21 +114,21 @@ score_mlp_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
   if (warp == 4) {
     // ---------------------------------------------------------------- TMA producer
     if (lane == 0) {
-      const uint32_t stage_tx = kABytes + (uint32_t)hidden * kKC * 2;
+      const uint32_t stage_tx = kABytes + (uint32_t)hl * kKC * 2;
       int kc = 0;
       for (; kc < n_kc; ++kc) {
         const int s = kc % kStages;
         if (kc >= kStages && !mbar_wait_bounded(&bar[B_EMPTY + s], ((kc / kStages) - 1) & 1)) { failed = true; break; }
         mbar_arrive_expect_tx(&bar[B_FULL + s], stage_tx);
         tma_load_2d(smem + s * kStageBytes, &map_x, kc * kKC, tok0, &bar[B_FULL + s]);
-        tma_load_2d(smem + s * kStageBytes + kABytes, &map_w1, kc * kKC, 0, &bar[B_FULL + s]);
+        tma_load_2d(smem + s * kStageBytes + kABytes, &map_w1, kc * kKC, j_off, &bar[B_FULL + s]);
       }
       if (failed)  // do not leave while copies may still be landing
         for (int k = max(0, kc - kStages); k < kc; ++k) mbar_wait_bounded(&bar[B_FULL + (k % kStages)], (k / kStages) & 1);
     }
   } else if (warp == 5) {
     // ---------------------------------------------------------------- MMA issue
-    const uint32_t idesc = instr_desc(kTok, hidden, false);
+    const uint32_t idesc = instr_desc(kTok, hl, false);
     for (int kc = 0; kc < n_kc && !failed; ++kc) {
       const int s = kc % kStages;
       if (!mbar_wait_bounded(&bar[B_FULL + s], (kc / kStages) & 1)) { failed = true; break; }
@@ -120,7 +150,7 @@ score_mlp_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
         float acc[8];
 #pragma unroll
         for (int h = 0; h < 8; ++h) acc[h] = 0.f;
-        for (int j0 = 0; j0 < hidden; j0 += 16) {
+        for (int j0 = 0; j0 < hl; j0 += 16) {
           float z[16];
           tmem_ld16(t_lane + j0, z);
           tmem_ld_wait();
@@ -136,7 +166,14 @@ score_mlp_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
             acc[6] = fmaf(wb.z, act, acc[6]); acc[7] = fmaf(wb.w, act, acc[7]);
           }
         }
-        if (tok < n_tok) {
+        if (kSplit == 2) {
+          // block 0 parks its half, block 1 sends its half to block 0; summed after the cluster barrier
+#pragma unroll
+          for (int h = 0; h < 8; ++h) {
+            if (rank == 0) part[(size_t)tid * heads8 + h0 + h] = acc[h];
+            else st_cluster_f32(part + (size_t)kTok * heads8 + (size_t)tid * heads8 + h0 + h, 0, acc[h]);
+          }
+        } else if (tok < n_tok) {
 #pragma unroll
           for (int h = 0; h < 8; ++h)
             if (h0 + h < Hkv) {
@@ -148,6 +185,18 @@ score_mlp_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
       }
     } else {
       failed = true;
+    }
+  }
+  if (kSplit == 2) {
+    cluster_sync_all();  // every thread of both blocks; block 1's stores are visible to block 0 after it
+    if (rank == 0 && warp < 4) {
+      const int tok = tok0 + tid;
+      if (tok < n_tok)
+        for (int h = 0; h < Hkv; ++h) {
+          const float v = part[(size_t)tid * heads8 + h] + part[(size_t)kTok * heads8 + (size_t)tid * heads8 + h] + b2[h];
+          logits[(size_t)tok * Hkv + h] = v;
+          if (flags) flags[(size_t)tok * Hkv + h] = v >= tau_logit ? 1 : 0;
+        }
     }
   }
   if (failed) atomicCAS(status, 0, SPKV_E_TIMEOUT);
@@ -205,15 +254,32 @@ int launch_score_mlp_tc(spkv_cache *cache, const spkv_predictor_t *p, const void
       p->hidden * heads8 > sctc::kMaxW2Floats || (p->d_in & 7) || ((uintptr_t)d_x & 15) || ((uintptr_t)p->d_W1 & 15) ||
       !encode_tiled())
     return 1;
+  // two blocks per token tile when that gives more blocks than one wave would otherwise hold
+  const int tiles = (n_tok + sctc::kTok - 1) / sctc::kTok;
+  const bool split = (p->hidden % 32) == 0 && heads8 <= 16 && tiles < cache->sm_count;
+  const int hl = split ? p->hidden / 2 : p->hidden;
   CUtensorMap map_x, map_w1;
-  if (!make_map(&map_x, d_x, n_tok, p->d_in, sctc::kTok) || !make_map(&map_w1, p->d_W1, p->hidden, p->d_in, p->hidden))
+  if (!make_map(&map_x, d_x, n_tok, p->d_in, sctc::kTok) || !make_map(&map_w1, p->d_W1, p->hidden, p->d_in, hl))
     return 1;
-  if (cudaFuncSetAttribute(score_mlp_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, sctc::kSmemBytes) !=
-      cudaSuccess)
+  auto kernel = split ? score_mlp_tc_kernel<2> : score_mlp_tc_kernel<1>;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, sctc::kSmemBytes) != cudaSuccess)
     return SPKV_E_CUDA;
-  score_mlp_tc_kernel<<<(n_tok + sctc::kTok - 1) / sctc::kTok, sctc::kThreads, sctc::kSmemBytes, s>>>(
-      map_x, map_w1, n_tok, p->d_in, p->hidden, p->d_b1, static_cast<const __nv_bfloat16 *>(p->d_W2), p->d_b2, Hkv,
-      cache->tau_logit, d_logits, d_flags, cache->view.status);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(tiles * (split ? 2 : 1));
+  cfg.blockDim = dim3(sctc::kThreads);
+  cfg.dynamicSmemBytes = sctc::kSmemBytes;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = split ? 2 : 1;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, kernel, map_x, map_w1, n_tok, (int)p->d_in, (int)p->hidden, p->d_b1,
+                         static_cast<const __nv_bfloat16 *>(p->d_W2), p->d_b2, Hkv, cache->tau_logit, d_logits,
+                         d_flags, cache->view.status) != cudaSuccess)
+    return SPKV_E_CUDA;
   return check_stream_error(cudaGetLastError());
 }
 
