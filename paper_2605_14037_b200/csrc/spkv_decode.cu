@@ -314,7 +314,7 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
   const int VP = s_pre[n];
   // at least four positions per block (tiny calls would otherwise be cut into single pages
   // and spend their time merging); snapping distance: a.snap positions, less for short ranges
-  const int nb_eff = max(1, min((int)gridDim.x, (VP + 3) / 4));
+  const int nb_eff = max(1, min((int)gridDim.x, (VP + a.min_pos - 1) / a.min_pos));
   for (int cc = tid; cc <= nb_eff; cc += kTcThreads)
     s_cut[cc] = range_cut(cc, nb_eff, VP, min(a.snap, VP / nb_eff / 4), s_pre, n);
   __syncthreads();
@@ -780,6 +780,11 @@ extern "C" int spkv_decode_attention(spkv_cache_t *cache, int32_t layer, const i
     return e ? atoi(e) : 6;
   }();
   a.snap = snap_env;
+  static const int min_pos_env = [] {
+    const char *e = getenv("SPKV_DECODE_MINPOS");  // tuning knob: least positions per block
+    return e ? max(1, atoi(e)) : 4;
+  }();
+  a.min_pos = min_pos_env;
   // Two consecutive decode launches may overlap (the next one starts on the SMs this one
   // has left): they alternate between the two halves of the workspace.  A third cannot
   // join: it needs every block of the second resident, i.e. every SM left by the first.
