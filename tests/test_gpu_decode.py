@@ -115,16 +115,17 @@ def test_decode_workspace_checked():
     assert rc == -7
 
 
-def test_decode_step_host_pipeline_matches_device_calls():
+@pytest.mark.parametrize("flags", [0, 1])
+def test_decode_step_host_pipeline_matches_device_calls(flags):
     """spkv_decode_step_host (pinned host buffers, copies on the cache's own streams, two
     slots in flight) gives bit for bit what the device-pointer calls give, layer after layer
     and step after step, and its outputs are complete after flush + synchronize."""
     spkv = load()
     rng = np.random.default_rng(91)
     L, B, Hq, Hkv, d_in, w, steps = 3, 5, 8, 2, 64, 16, 40
-    mk = lambda: spkv.Cache(n_layers=L, max_seqs=B, n_q_heads=Hq, n_kv_heads=Hkv, max_context=512,
-                            pool_pages=L * B * Hkv * 2, window=w, tau=0.5)
-    ca, cb = mk(), mk()
+    mk = lambda f: spkv.Cache(n_layers=L, max_seqs=B, n_q_heads=Hq, n_kv_heads=Hkv, max_context=512,
+                              pool_pages=L * B * Hkv * 2, window=w, tau=0.5, flags=f)
+    ca, cb = mk(flags), mk(0)
     tl = ca.spkv_tau_logit()
     preds = []
     for l in range(L):
