@@ -54,7 +54,11 @@ enum {
   SPKV_E_WORKSPACE = -7,        /* workspace missing or too small                      */
   SPKV_E_TIMEOUT = -8,          /* device: a bounded wait on a copy ran out            */
   SPKV_E_BOUNDS = -9,           /* device: a sequence id outside [0, max_seqs)         */
-  SPKV_E_SCRATCH_LIMIT = -10    /* request larger than the library's built-in scratch  */
+  SPKV_E_SCRATCH_LIMIT = -10,   /* request larger than the library's built-in scratch  */
+  SPKV_E_ORDER_DECODE = -11,    /* device, overlap mode: a decode launch gave up waiting for the
+                                   appends of its layer / the previous user of its workspace */
+  SPKV_E_ORDER_APPEND = -12     /* device, overlap mode: an append gave up waiting for the decode
+                                   launches of its layer                                  */
 };
 
 typedef struct {

@@ -112,17 +112,17 @@ append_evict_kernel(CacheView c, int layer, const int32_t *__restrict__ seq_ids,
   // Every block counts itself in before dependents may launch and out when it is done: that is
   // what later kernels that skip griddepcontrol.wait order themselves by.
   if (threadIdx.x == 0) sync_count_start(c, layer, kSyncAppStart);
-  __syncthreads();
   // wait_prev = 1: wait for everything earlier on the stream.  wait_prev = 0 (overlap mode; the
   // host passes it only when the launches since the last full wait were hot-path kernels of
   // this cache on other layers): the earlier kernels may still be running, and the only ones
   // this launch shares data with are the decode launches of its own layer, which it waits out.
+  // The "started" counter is read BEFORE the block lets dependents launch: the decode launch
+  // that follows counts itself into the same counter and waits for this append, so reading it
+  // later would make the two wait for each other.
   if (wait_prev) pdl_wait();
+  else if (threadIdx.x == 0 && !sync_wait_finished(c, layer, kSyncDecStart)) set_status(c, SPKV_E_ORDER_APPEND);
+  __syncthreads();
   pdl_trigger();
-  if (!wait_prev) {
-    if (threadIdx.x == 0 && !sync_wait_finished(c, layer, kSyncDecStart)) set_status(c, SPKV_E_TIMEOUT);
-    __syncthreads();
-  }
   append_unit(c, layer, seq_ids, B, k_new, v_new, logits, tau_logit, x, W, bias, d_in, logits_out);
   __syncthreads();
   if (threadIdx.x == 0) sync_count_finish(c, layer, kSyncAppFin);

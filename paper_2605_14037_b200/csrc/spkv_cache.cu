@@ -377,6 +377,8 @@ extern "C" const char *spkv_error_string(int code) {
     case SPKV_E_TIMEOUT: return "bounded device wait ran out";
     case SPKV_E_BOUNDS: return "sequence id out of range";
     case SPKV_E_SCRATCH_LIMIT: return "request exceeds the built-in scratch area";
+    case SPKV_E_ORDER_DECODE: return "overlap mode: decode launch gave up waiting for its append / workspace";
+    case SPKV_E_ORDER_APPEND: return "overlap mode: append gave up waiting for its layer's decode launches";
     default: return "unknown error";
   }
 }

@@ -282,7 +282,7 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
   // (the counter reads run beside thread 32's count-in: one trip to L2 for both)
   if (a.wait_mode == 1 && tid == 0 &&
       !sync_wait_finished(c, a.layer, kSyncAppStart, a.prev_half_layer, kSyncDecStart))
-    set_status(c, SPKV_E_TIMEOUT);
+    set_status(c, SPKV_E_ORDER_DECODE);
   __syncthreads();  // the block is counted in before any of its threads lets dependents launch
   pdl_trigger();
   if (a.wait_mode == 1)

@@ -138,8 +138,11 @@ enum { kLastOther = 0, kLastAppend = 1, kLastDecode = 2 };
 // is done.  A later kernel is launched only after all blocks of all earlier kernels of the
 // stream have started (each launch needs its predecessor's blocks to have triggered), so when
 // it reads "started" that number is final, and "finished >= started" (acquire) means those
-// kernels are done.  Nothing here depends on values the host passes per launch: a captured
-// CUDA graph replays correctly.  The spin is bounded; on expiry the status word is set.
+// kernels are done.  A block must read "started" BEFORE it lets dependents launch: a dependent
+// may count itself into the very counter being read and wait for this kernel in turn, and the
+// two would then wait for each other.  Nothing here depends on values the host passes per
+// launch: a captured CUDA graph replays correctly.  The spin is bounded; on expiry the status
+// word is set.
 enum { kSyncAppStart = 0, kSyncAppFin = 1, kSyncDecStart = 2, kSyncDecFin = 3 };
 
 __device__ inline void sync_count_start(const CacheView &c, int layer, int which) {  // one thread per block

@@ -23,7 +23,7 @@ SPKV_OK = 0
 ERRORS = {
     -1: "SPKV_E_INVALID", -2: "SPKV_E_ARENA_TOO_SMALL", -3: "SPKV_E_UNSUPPORTED", -4: "SPKV_E_CUDA",
     -5: "SPKV_E_POOL_EXHAUSTED", -6: "SPKV_E_CONTEXT_OVERFLOW", -7: "SPKV_E_WORKSPACE",
-    -8: "SPKV_E_TIMEOUT", -9: "SPKV_E_BOUNDS", -10: "SPKV_E_SCRATCH_LIMIT",
+    -8: "SPKV_E_TIMEOUT", -9: "SPKV_E_BOUNDS", -10: "SPKV_E_SCRATCH_LIMIT", -11: "SPKV_E_ORDER_DECODE", -12: "SPKV_E_ORDER_APPEND",
 }
 
 

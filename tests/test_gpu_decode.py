@@ -193,16 +193,18 @@ def test_units_split_over_dozens_of_blocks_merge_on_two_levels(T):
         assert np.abs(lse[s].cpu().numpy() - ref_lse).max() < 1e-3
 
 
-@pytest.mark.parametrize("L,B", [(4, 16), (3, 2), (2, 3), (1, 2)])
-def test_overlap_mode_is_bit_identical_to_stream_ordered_launches(L, B):
+@pytest.mark.parametrize("L,B,steps", [(4, 16, 24), (3, 2, 24), (2, 3, 24), (1, 2, 24), (8, 16, 200)])
+def test_overlap_mode_is_bit_identical_to_stream_ordered_launches(L, B, steps):
     """SPKV_FLAG_OVERLAP: appends and decodes skip the wait for the whole stream and order
     themselves by per-layer block counters.  A multi-layer decode loop (inputs staged before
     each step, launches back to back, as the benchmark issues them) must give, bit for bit,
     the outputs and cache state of a cache that launches everything stream-ordered.  Two and
-    one layer(s) exercise the fall-back when a workspace half comes back to the same layer."""
+    one layer(s) exercise the fall-back when a workspace half comes back to the same layer; the
+    long case is there for the orderings that only show up now and then (a dependency wait that
+    runs out sets the status word)."""
     spkv = load()
     rng = np.random.default_rng(300 + L * 10 + B)
-    Hq, Hkv, d_in, w, T0, steps = 8, 2, 64, 128, 700, 24
+    Hq, Hkv, d_in, w, T0 = 8, 2, 64, 128, 700
     mk = lambda flags: spkv.Cache(n_layers=L, max_seqs=B, n_q_heads=Hq, n_kv_heads=Hkv, max_context=2048,
                                   pool_pages=L * B * Hkv * 14, window=w, tau=0.5, flags=flags)
     ca, cb = mk(spkv.FLAG_OVERLAP), mk(0)
