@@ -20,7 +20,7 @@ __device__ inline int alloc_page(const CacheView &c, int lane) {
     if (top <= 0) {
       atomicAdd(&c.status[1], 1);
     } else {
-      page = c.free_stack[top - 1];
+      page = __ldcg(&c.free_stack[top - 1]);
     }
   }
   page = __shfl_sync(0xffffffffu, page, 0);
@@ -55,7 +55,9 @@ __device__ inline void append_unit(const CacheView &c, int layer, const int32_t 
   } else {
     new_logit = logits[item];
   }
-  const int t = c.t[u];
+  // metadata and the evicted pair are read from L2: in overlap mode this kernel does not start at a
+  // stream-wide synchronisation point, and an SM's L1 is not coherent with other SMs' stores
+  const int t = __ldcg(&c.t[u]);
   const int slot = t % c.w;
   const int row = slot % kP;
   // lanes 0-15 move the key row, lanes 16-31 the value row, one 16-byte chunk each
@@ -67,9 +69,9 @@ __device__ inline void append_unit(const CacheView &c, int layer, const int32_t 
   if (t >= c.w) {
     // the pair of position t - w leaves the window: threshold decision on its stored logit
     // (sink positions are kept regardless)
-    const float lg = c.ring_logit[(size_t)u * c.w + slot];
+    const float lg = __ldcg(&c.ring_logit[(size_t)u * c.w + slot]);
     if (lg >= head_threshold(c, layer, kvh, tau_logit) || t - c.w < c.n_sink) {
-      const int n = c.len[u];
+      const int n = __ldcg(&c.len[u]);
       const int pj = n / kP, prow = n % kP;
       int page = -1, err = 0;
       if (pj >= c.max_pages) {
@@ -79,14 +81,14 @@ __device__ inline void append_unit(const CacheView &c, int layer, const int32_t 
         if (page < 0) err = SPKV_E_POOL_EXHAUSTED;
         else if (lane == 0) c.table[(size_t)u * c.max_pages + pj] = page;
       } else {
-        page = c.table[(size_t)u * c.max_pages + pj];
+        page = __ldcg(&c.table[(size_t)u * c.max_pages + pj]);
       }
       if (err) {
         if (lane == 0) set_status(c, err);
       } else {
         __syncwarp();
         __nv_bfloat16 *dst = c.pages + (int64_t)page * kPageElems;
-        *reinterpret_cast<uint4 *>(dst + blk + swz_off(prow, chunk)) = *ring_cell;
+        *reinterpret_cast<uint4 *>(dst + blk + swz_off(prow, chunk)) = __ldcg(ring_cell);
         if (lane == 0) {
           c.pos_pool[((int64_t)page - c.n_ring_pages_total) * kP + prow] = t - c.w;
           c.len[u] = n + 1;

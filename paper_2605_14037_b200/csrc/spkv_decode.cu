@@ -293,8 +293,10 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
     int np = 0, u = 0, len = 0, n_ring = 0;
     if (seq >= 0 && seq < c.S) {
       u = unit_index(c, a.layer, seq, kvh);
-      len = c.len[u];
-      n_ring = min(c.t[u], c.w);
+      // (L2 loads: in overlap mode the writer may be a kernel that ended after this block began,
+      // and an SM's L1 is not coherent with other SMs' stores)
+      len = __ldcg(&c.len[u]);
+      n_ring = min(__ldcg(&c.t[u]), c.w);
       np = (len + kP - 1) / kP + (n_ring + kP - 1) / kP;
     } else if (blockIdx.x == 0) {
       set_status(c, SPKV_E_BOUNDS);
@@ -347,7 +349,7 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
         if (j >= 0) {
           const int u = s_unit[item], len = s_len[item], nk = (len + kP - 1) / kP;
           if (j < nk) {
-            gq.gpage = c.table[(size_t)u * c.max_pages + j];
+            gq.gpage = __ldcg(&c.table[(size_t)u * c.max_pages + j]);
             gq.valid = min(kP, len - j * kP);
           } else {
             gq.gpage = (int)ring_page(c, u, j - nk);

@@ -69,7 +69,7 @@ __device__ inline void set_status(const CacheView &c, int code) { atomicCAS(c.st
 
 // threshold in force for a (layer, KV head): its own if one was set, else the cache-wide one
 __device__ inline float head_threshold(const CacheView &c, int layer, int kvh, float tau_logit) {
-  const float own = c.head_tau[layer * c.Hkv + kvh];
+  const float own = __ldcg(&c.head_tau[layer * c.Hkv + kvh]);
   return own != own ? tau_logit : own;
 }
 
