@@ -314,9 +314,14 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
   __syncthreads();
   block_exclusive_scan(s_np, s_pre, n, s_tmp);
   const int VP = s_pre[n];
-  // at least four positions per block (tiny calls would otherwise be cut into single pages
-  // and spend their time merging); snapping distance: a.snap positions, less for short ranges
-  const int nb_eff = max(1, min((int)gridDim.x, (VP + a.min_pos - 1) / a.min_pos));
+  // Blocks per launch.  A small launch is latency-bound: as many blocks as have four positions
+  // each (tiny calls would otherwise be cut into single pages and spend their time merging).
+  // A launch with at least half a grid of a.min_pos-position ranges gives every block at least
+  // that many: consecutive launches overlap, the SMs this one leaves idle work for its
+  // neighbours, and a block's fixed cost (start-up, merge) is spread over more pages.
+  const int nb_eff = VP >= a.min_pos * ((int)gridDim.x / 2) ? min((int)gridDim.x, (VP + a.min_pos - 1) / a.min_pos)
+                                                            : max(1, min((int)gridDim.x, (VP + 3) / 4));
+  // snapping distance: a.snap positions, less for short ranges
   for (int cc = tid; cc <= nb_eff; cc += kTcThreads)
     s_cut[cc] = range_cut(cc, nb_eff, VP, min(a.snap, VP / nb_eff / 4), s_pre, n);
   __syncthreads();
@@ -783,8 +788,8 @@ extern "C" int spkv_decode_attention(spkv_cache_t *cache, int32_t layer, const i
   }();
   a.snap = snap_env;
   static const int min_pos_env = [] {
-    const char *e = getenv("SPKV_DECODE_MINPOS");  // tuning knob: least positions per block
-    return e ? max(1, atoi(e)) : 4;
+    const char *e = getenv("SPKV_DECODE_MINPOS");  // tuning knob: least positions per block of a large launch
+    return e ? max(4, atoi(e)) : 56;
   }();
   a.min_pos = min_pos_env;
   // Two consecutive decode launches may overlap (the next one starts on the SMs this one

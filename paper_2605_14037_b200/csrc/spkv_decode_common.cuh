@@ -19,7 +19,7 @@ struct DecodeArgs {
   float *lse;              // [B][Hq] or null
   float scale_log2;        // sm_scale * log2(e)
   int snap;                // range cuts within this many positions of a unit boundary move onto it
-  int min_pos;             // a block takes at least this many positions (fewer blocks work on a small launch)
+  int min_pos;             // positions a block takes at least when the launch has half a grid of such ranges
   int wait_mode;           // 0: griddepcontrol.wait; 1: overlap mode, wait for the launches it shares data with
   int prev_half_layer;     // layer of the decode launch that last used this workspace half (-1: none)
   int32_t *counters;       // [n_items] arrival counters
