@@ -448,7 +448,6 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
         }
       }
       const int tok0 = (warp & 3) * 16;
-#ifndef SPKV_PROBE_NOCOMPUTE
       if ((k & 1) == (warp >> 2) && tok0 < valid) {
         const uint32_t sK = smem_u32(sbase), sV = sK + kBlockElems * 2;
         float s[NH][4];
@@ -465,9 +464,6 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
         dbg_c[3] += clock64() - c3;
 #endif
       }
-#else
-      if (tok0 < valid) { m[0][0] = 0.f; l[0][0] = 1.f; }
-#endif
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty[stage]);
 #ifdef SPKV_PHASE_TIMING
@@ -842,10 +838,7 @@ extern "C" int spkv_decode_attention(spkv_cache_t *cache, int32_t layer, const i
   void (*kernel)(DecodeArgs, int, int, int) = GP > 8 ? decode_tc_kernel<2> : decode_tc_kernel<1>;
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total) != cudaSuccess)
     return SPKV_E_CUDA;
-  int grid = min(kMaxGrid, cache->sm_count);
-#ifdef SPKV_PROBE_GRID
-  if (const char *e = getenv("SPKV_DECODE_GRID")) grid = atoi(e);
-#endif
+  const int grid = min(kMaxGrid, cache->sm_count);
   if (!(cache->cfg.flags & SPKV_FLAG_OVERLAP)) {  // plain stream-ordered launch
     kernel<<<grid, kTcThreads, L.total, s>>>(a, GP, n_stages, red_bufs);
     return check_stream_error(cudaGetLastError());
