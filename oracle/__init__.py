@@ -27,7 +27,12 @@ _i32p = np.ctypeslib.ndpointer(np.int32, flags="C_CONTIGUOUS")
 
 
 def build(force: bool = False) -> str:
-    """Compile the oracle with gcc (OpenMP for the unit loop only)."""
+    """Compile the oracle with gcc (OpenMP for the unit loop only).  SPKV_ORACLE_LIB names a
+    ready-made library to load instead (the mutation tests point it at deliberately broken
+    copies to show that the pins catch them)."""
+    override = os.environ.get("SPKV_ORACLE_LIB")
+    if override:
+        return override
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
         tmp = _LIB + f".{os.getpid()}.tmp"
         subprocess.check_call(

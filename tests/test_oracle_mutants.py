@@ -1,0 +1,55 @@
+"""How sharp are the oracle's pins?  Each case plants ONE plausible mistake in a copy of the
+oracle's C source (a wrong comparison, an off-by-one window, a transposed operand, a dropped
+term, ...), builds it, and runs the pin tests against the broken copy in a child process: the
+pins must fail.  A mistake that survives would mean the oracle is not pinned there."""
+import os
+import subprocess
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+SRC = os.path.join(ROOT, "oracle", "spkv_oracle.c")
+
+# (name, text in the source, what it is replaced by, how many times the text occurs)
+MUTANTS = [
+    ("threshold_exclusive_mask", "int z = (logit[s] >= tau_logit) ? 1 : 0;", "int z = (logit[s] > tau_logit) ? 1 : 0;", 1),
+    ("window_one_too_wide", "int in_win = (t - s >= 0) && (t - s < w);", "int in_win = (t - s >= 0) && (t - s <= w);", 1),
+    ("no_causal_mask", "double causal = (s <= t) ? 0.0 : -INFINITY;", "double causal = 0.0;", 1),
+    ("scores_against_values", "dot += bf16_widen(q[(size_t)g * D + i]) * bf16_widen(K[(size_t)s * D + i]);",
+     "dot += bf16_widen(q[(size_t)g * D + i]) * bf16_widen(V[(size_t)s * D + i]);", 1),
+    ("scale_dropped_mask", "score[s] = dot * scale + bias;", "score[s] = dot + bias;", 1),
+    ("scale_dropped_stream", "p[j] = dot * scale;", "p[j] = dot;", 1),
+    ("all_heads_use_head_0", "for (int i = 0; i < D; ++i) dot += bf16_widen(q[(size_t)g * D + i]) * bf16_widen(kr[i]);",
+     "for (int i = 0; i < D; ++i) dot += bf16_widen(q[i]) * bf16_widen(kr[i]);", 1),
+    ("evict_decides_on_new_logit", "if (u->ring_logit[slot] >= tau_logit || u->t - u->w < u->n_sink)",
+     "if (logit >= tau_logit || u->t - u->w < u->n_sink)", 1),
+    ("kept_position_off_by_one", "orcA_keep(u, u->t - u->w, ", "orcA_keep(u, u->t - u->w + 1, ", 1),
+    ("ring_slot_off_by_one", "long slot = u->t % u->w;", "long slot = (u->t + 1) % u->w;", 1),
+    ("sink_one_too_many", "int sink = s < n_sink;", "int sink = s <= n_sink;", 1),
+    ("lse_without_max", "if (lse) lse[g] = mx + log(denom);", "if (lse) lse[g] = log(denom);", 1),
+    ("linear_bias_dropped", "logit_out[(size_t)n * n_kv_heads + h] = acc + (double)b[h];",
+     "logit_out[(size_t)n * n_kv_heads + h] = acc;", 1),
+    ("silu_is_plain_sigmoid", "a[j] = z * orc_sigmoid(z);", "a[j] = orc_sigmoid(z);", 1),
+    ("tau_logit_sign", "return (float)log(tau / (1.0 - tau));", "return (float)log((1.0 - tau) / tau);", 1),
+    ("softmax_without_normalisation", "double p = exp(score[s] - mx) / denom;", "double p = exp(score[s] - mx);", 1),
+    ("keep_all_and_keep_none_swapped", "if (!(tau > 0.0)) return -INFINITY;", "if (!(tau > 0.0)) return INFINITY;", 1),
+]
+
+
+@pytest.mark.parametrize("name,old,new,count", MUTANTS, ids=[m[0] for m in MUTANTS])
+def test_planted_mistake_is_caught(tmp_path, name, old, new, count):
+    text = open(SRC).read()
+    assert text.count(old) == count, f"{name}: source text occurs {text.count(old)} times"
+    mutated = text.replace(old, new)
+    src = tmp_path / "mutant.c"
+    lib = tmp_path / "libmutant.so"
+    src.write_text(mutated)
+    subprocess.check_call(["gcc", "-O1", "-std=c99", "-fPIC", "-shared", "-fopenmp", "-o", str(lib), str(src), "-lm"])
+    env = dict(os.environ, SPKV_ORACLE_LIB=str(lib))
+    r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider",
+                        os.path.join(ROOT, "tests", "test_oracle_pins.py"),
+                        os.path.join(ROOT, "tests", "test_oracle_sinks.py")],
+                       cwd=ROOT, env=env, capture_output=True, text=True, timeout=600)
+    out = r.stdout + r.stderr
+    assert r.returncode == 1 and " failed" in out, f"mutant {name} survived the pins:\n{out[-800:]}"
