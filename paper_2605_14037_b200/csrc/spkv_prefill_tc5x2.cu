@@ -8,7 +8,7 @@
 // when it finishes the current one, and the issue-to-completion latency of the MMAs of one head
 // hides under the softmax of both:
 //
-//   MMA thread, per page j:  wait P0(j) | PV0(j) QK0(j+2) | wait P1(j) | PV1(j) QK1(j+2)
+//   MMA warp, per page j  :  wait P0(j), P1(j) | PV0(j) PV1(j) | wait page j+2 | QK0(j+2) QK1(j+2)
 //   group h               :  softmax_h(j) softmax_h(j+1) softmax_h(j+2) ...
 //
 // P = exp2(S - m) is split into hi + lo bf16 terms and written back into the tensor-memory

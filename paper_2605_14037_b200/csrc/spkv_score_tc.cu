@@ -11,8 +11,8 @@
 // are row-major with the contraction dimension innermost, i.e. K-major operands as they are: a
 // TMA tile load (64 dims x rows, 128-byte swizzle) puts them in shared memory in operand layout.
 // Rows past n_tok and dims past d_in are zero-filled by the TMA unit.  192 KB mbarrier
-// pipeline (4 stages of 48 KB, or 6 of 32 KB): warp 4 = TMA producer, warp 5 = MMA issue (whole warp, one elected lane), warps 0-3
-// = epilogue.  Traffic: n_tok * d_in * 2 B of activations from HBM once; W1 (hidden * d_in * 2 B)
+// pipeline (4 stages of 48 KB, or 6 of 32 KB): warp 4 = TMA producer, warp 5 = MMA issue (whole
+// warp, one elected lane), warps 0-3 = epilogue.  Traffic: n_tok * d_in * 2 B of activations from HBM once; W1 (hidden * d_in * 2 B)
 // is re-read per block from L2.  All waits are bounded.
 #include <cuda.h>
 #include <stdlib.h>
