@@ -97,8 +97,11 @@ __device__ inline void append_unit(const CacheView &c, int layer, const int32_t 
     }
   }
   const uint4 *src = (lane < 16 ? k_new : v_new) + (size_t)item * 16 + chunk;
-  *ring_cell = *src;
+  const uint4 cell = *src;
+  *ring_cell = cell;
+  const uint32_t vm = __reduce_max_sync(0xffffffffu, lane < 16 ? 0u : chunk_abs_max_bf16(cell));
   if (lane == 0) {
+    note_vmax(c, u, vm);
     c.ring_logit[(size_t)u * c.w + slot] = new_logit;
     c.t[u] = t + 1;
   }

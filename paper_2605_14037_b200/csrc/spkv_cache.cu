@@ -50,6 +50,7 @@ static void make_layout(const spkv_config_t *c, Layout *l) {
   l->off_rlogit = o; o = align_up(o + units * (size_t)c->window * 4, 256);
   l->off_htau = o;   o = align_up(o + (size_t)c->n_layers * c->n_kv_heads * 4, 256);
   l->off_sync = o;   o = align_up(o + (size_t)c->n_layers * 4 * 8, 256);
+  l->off_vmax = o;   o = align_up(o + units * 4, 256);
   o = align_up(o, 1024);
   l->off_pages = o;  o += (units * ring_pages + (size_t)c->pool_pages) * kPageBytes;
   l->total = o;
@@ -84,7 +85,7 @@ __global__ void reset_seq_kernel(CacheView c, int seq) {
   for (int i = threadIdx.x; i < n16; i += blockDim.x) ring[i] = make_uint4(0, 0, 0, 0);
   for (int i = threadIdx.x; i < c.w; i += blockDim.x) c.ring_logit[(size_t)u * c.w + i] = 0.f;
   __syncthreads();
-  if (threadIdx.x == 0) { c.len[u] = 0; c.t[u] = 0; }
+  if (threadIdx.x == 0) { c.len[u] = 0; c.t[u] = 0; c.vmax[u] = 0; }
 }
 
 }  // namespace spkv
@@ -146,6 +147,7 @@ extern "C" int spkv_cache_create(const spkv_config_t *cfg, void *d_arena, size_t
   v.ring_logit = reinterpret_cast<float *>(base + l.off_rlogit);
   v.head_tau = reinterpret_cast<float *>(base + l.off_htau);
   v.sync_ctr = reinterpret_cast<unsigned long long *>(base + l.off_sync);
+  v.vmax = reinterpret_cast<uint32_t *>(base + l.off_vmax);
   v.pages = reinterpret_cast<__nv_bfloat16 *>(base + l.off_pages);
 
   int dev = 0;

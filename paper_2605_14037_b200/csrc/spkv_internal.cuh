@@ -9,6 +9,7 @@
 //   pos_pool[]  : position of every kept pair, by pool page     int32 [pool_pages][P]
 //   ring_logit[]: stored logit per ring slot                    f32   [n_units][w]
 //   head_tau[]  : per-(layer, KV head) threshold override       f32   [L][Hkv]  (NaN: none)
+//   vmax[]      : largest finite |value| a unit has received    u32   [n_units] (fp32 bit pattern)
 //   sync_ctr[]  : blocks started / finished per layer and kernel u64   [L][4]    (launch overlap)
 //   pages       : ring pages of every unit ([n_units][ring_pages]) followed by the pool
 //
@@ -49,12 +50,33 @@ struct CacheView {
   float *ring_logit;
   float *head_tau;      // [L][Hkv] logit-space threshold of a (layer, KV head); NaN = the cache-wide one
   unsigned long long *sync_ctr;  // [L][4]: append blocks started, finished; decode blocks started, finished
+  // [n_units] bit pattern of the largest finite |v| the unit has received since its sequence was
+  // reset.  The prefill attention multiplies P.V in fp16 and scales the values by a power of two
+  // taken from this word, so that any bf16 value range fits.
+  uint32_t *vmax;
   __nv_bfloat16 *pages;
 };
 
 struct Layout {
-  size_t off_header, off_t, off_len, off_table, off_free, off_pos, off_rlogit, off_htau, off_sync, off_pages, total;
+  size_t off_header, off_t, off_len, off_table, off_free, off_pos, off_rlogit, off_htau, off_sync, off_vmax, off_pages, total;
 };
+
+// largest finite |x| among the eight bf16 of a 16-byte chunk, as the upper half of an fp32 bit
+// pattern (infinities and NaNs do not count: they come out of the attention as they went in)
+__device__ inline uint32_t chunk_abs_max_bf16(const uint4 &v) {
+  uint32_t m = 0;
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const uint32_t a = w[i] & 0x7fffu, b = (w[i] >> 16) & 0x7fffu;
+    m = max(m, a < 0x7f80u ? a : 0u);
+    m = max(m, b < 0x7f80u ? b : 0u);
+  }
+  return m << 16;
+}
+__device__ inline void note_vmax(const CacheView &c, int u, uint32_t m) {  // one thread
+  if (m > __ldcg(&c.vmax[u])) atomicMax(&c.vmax[u], m);
+}
 
 // element offset of (row, 16-byte chunk) inside a key or value block
 __host__ __device__ inline int swz_off(int row, int chunk) {

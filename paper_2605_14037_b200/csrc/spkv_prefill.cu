@@ -154,6 +154,7 @@ __global__ void __launch_bounds__(256) prefill_scatter_kernel(PrefillArgs a) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int chunk = lane & 15, blk = (lane >> 4) * kBlockElems;
   const int j0 = (blockIdx.x * 8 + warp) * 8;
+  uint32_t vm = 0;  // largest |v| among the chunk's own pairs that this warp keeps
   for (int j = j0; j < min(j0 + 8, n_leave); ++j) {
     const int e = E[j];
     if (E[j + 1] == e) continue;  // not flagged
@@ -163,8 +164,11 @@ __global__ void __launch_bounds__(256) prefill_scatter_kernel(PrefillArgs a) {
     const SrcRow s = staging_row(a, u, kvh, t0, n_old, j);
     const uint4 val = load_chunk(lane < 16 ? s.k : s.v, s.row, chunk);
     *reinterpret_cast<uint4 *>(c.pages + (int64_t)page * kPageElems + blk + swz_off(drow, chunk)) = val;
+    if (lane >= 16 && j >= n_old) vm = max(vm, chunk_abs_max_bf16(val));
     if (lane == 0) c.pos_pool[((int64_t)page - c.n_ring_pages_total) * kP + drow] = t0 - n_old + j;
   }
+  vm = __reduce_max_sync(0xffffffffu, vm);
+  if (lane == 0 && vm) note_vmax(c, u, vm);
 }
 
 // --------------------------------------------------------------------- C: ring update
@@ -185,7 +189,11 @@ __global__ void __launch_bounds__(256) prefill_ring_kernel(PrefillArgs a) {
     const size_t off = ((size_t)i * c.Hkv + kvh) * kD;
     const uint4 val = *reinterpret_cast<const uint4 *>((lane < 16 ? a.k : a.v) + off + chunk * 8);
     *reinterpret_cast<uint4 *>(pg + blk + swz_off(row, chunk)) = val;
-    if (lane == 0) c.ring_logit[(size_t)u * c.w + slot] = a.logits[(size_t)i * c.Hkv + kvh];
+    const uint32_t vm = __reduce_max_sync(0xffffffffu, lane < 16 ? 0u : chunk_abs_max_bf16(val));
+    if (lane == 0) {
+      c.ring_logit[(size_t)u * c.w + slot] = a.logits[(size_t)i * c.Hkv + kvh];
+      if (vm) note_vmax(c, u, vm);
+    }
   }
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     c.t[u] = t0 + a.C;

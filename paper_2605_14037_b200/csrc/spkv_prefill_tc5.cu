@@ -52,6 +52,7 @@ __global__ void __launch_bounds__(256) prefill_stage_kernel(PrefillArgs a) {
   __nv_bfloat16 *page = a.stage_pages + ((size_t)kvh * a.n_stage_pages + sp) * kPageElems;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int chunk = lane & 15, blk = (lane >> 4) * kBlockElems;
+  uint32_t vm = 0;  // largest |v| among the chunk's values this lane moves (old ring pairs are accounted for already)
   for (int r = warp * 8; r < warp * 8 + 8; ++r) {
     const int j = sp * kP + r;
     uint4 val = make_uint4(0, 0, 0, 0);  // rows past the last pair read as zeros
@@ -63,10 +64,13 @@ __global__ void __launch_bounds__(256) prefill_stage_kernel(PrefillArgs a) {
       } else {
         const __nv_bfloat16 *src = (lane < 16 ? a.k : a.v) + ((size_t)(j - n_old) * c.Hkv + kvh) * kD;
         val = *reinterpret_cast<const uint4 *>(src + chunk * 8);
+        if (lane >= 16) vm = max(vm, chunk_abs_max_bf16(val));
       }
     }
     *reinterpret_cast<uint4 *>(page + blk + swz_off(r, chunk)) = val;
   }
+  vm = __reduce_max_sync(0xffffffffu, vm);
+  if (lane == 0 && vm) note_vmax(c, u, vm);
 }
 
 // ------------------------------------------------------------------ chunk attention

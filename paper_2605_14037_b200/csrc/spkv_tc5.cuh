@@ -11,10 +11,11 @@ __device__ inline uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_
   return (uint64_t)((saddr & 0x3FFFF) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
          ((uint64_t)(sbo_bytes >> 4) << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
 }
-// instruction descriptor, kind::f16: fp32 accumulate, bf16 x bf16, A K-major
-__host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool b_mn_major) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(N >> 3) << 17) |
-         ((uint32_t)(M >> 4) << 24);
+// instruction descriptor, kind::f16: fp32 accumulate, A K-major, A and B both bf16 (format 1)
+// or both fp16 (format 0)
+__host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool b_mn_major, bool fp16 = false) {
+  return (1u << 4) | ((fp16 ? 0u : 1u) << 7) | ((fp16 ? 0u : 1u) << 10) | ((b_mn_major ? 1u : 0u) << 16) |
+         ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 // The MMA warp runs its loops with all 32 lanes (convergent control flow lets the compiler keep
 // descriptors and addresses in uniform registers: issuing from inside an `if (lane == 0)` branch
@@ -108,6 +109,32 @@ __device__ inline void umma_pv_page(uint32_t d_tmem, uint32_t a_tmem, uint64_t b
       " @e tcgen05.mma.cta_group::1.kind::f16 [%0], [t6], b2, %3, 1;\n"
       " @e tcgen05.mma.cta_group::1.kind::f16 [%0], [t7], b3, %3, 1;\n}\n"
       ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(first) : "memory");
+}
+// One page of P.V with a single fp16 P (64 keys = 32 columns at a_tmem): four K=16 steps.
+__device__ inline void umma_pv_page_f16(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
+                                        uint32_t first) {
+  asm volatile(
+      "{\n .reg .pred e, p;\n .reg .b64 b1, b2, b3;\n .reg .b32 t1, t2, t3;\n"
+      " elect.sync _|e, 0xffffffff;\n setp.ne.b32 p, %4, 0;\n"
+      " add.u64 b1, %2, 128; add.u64 b2, %2, 256; add.u64 b3, %2, 384;\n"
+      " add.u32 t1, %1, 8; add.u32 t2, %1, 16; add.u32 t3, %1, 24;\n"
+      " @e tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n"
+      " @e tcgen05.mma.cta_group::1.kind::f16 [%0], [t1], b1, %3, 1;\n"
+      " @e tcgen05.mma.cta_group::1.kind::f16 [%0], [t2], b2, %3, 1;\n"
+      " @e tcgen05.mma.cta_group::1.kind::f16 [%0], [t3], b3, %3, 1;\n}\n"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(first) : "memory");
+}
+// two bf16 (one 32-bit word) -> two fp16, each multiplied by `scale` first (a power of two)
+__device__ inline uint32_t bf16x2_to_f16x2(uint32_t x, float scale) {
+  uint32_t d;
+  const float lo = __uint_as_float(x << 16) * scale, hi = __uint_as_float(x & 0xffff0000u) * scale;
+  asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+__device__ inline uint32_t pack_f16(float lo, float hi) {
+  uint32_t d;
+  asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
 }
 // ---- packed fp32 pairs (two lanes per instruction on sm_100) and the three-input maximum
 __device__ inline uint64_t pack2(float a, float b) {
