@@ -525,8 +525,8 @@ def run_config4(args):
                    "frac_of_measured_hbm": dec_gbs / hbm_peak},
         "prefill": {"tokens_per_s": K * NP * C / (pre_ms * 1e-3), "ms_per_step": pre_ms / K,
                     "useful_tflops": pre_tflops, "frac_of_sustained_bf16": pre_tflops / 1356.9,
-                    "kernel": "prefill_attn_tc5x2_kernel (tcgen05)"},
-        "roofline": {"bound": "tensor", "kernel": "prefill_attn_tc5x2_kernel", "achieved": pre_tflops, "peak": 1356.9,
+                    "kernel": "prefill_attn_tc5x2h_kernel (tcgen05, P.V in fp16)"},
+        "roofline": {"bound": "tensor", "kernel": "prefill_attn_tc5x2h_kernel", "achieved": pre_tflops, "peak": 1356.9,
                      "unit": "TFLOP/s", "frac": pre_tflops / 1356.9, "peak_kind": "of measured (sustained)",
                      "traffic": None},
         "e2e": None, "dense": None,

@@ -74,8 +74,10 @@ __device__ inline uint32_t chunk_abs_max_bf16(const uint4 &v) {
   }
   return m << 16;
 }
-__device__ inline void note_vmax(const CacheView &c, int u, uint32_t m) {  // one thread
-  if (m > __ldcg(&c.vmax[u])) atomicMax(&c.vmax[u], m);
+// one thread; the result is not used, so this is a fire-and-forget reduction (reading the word
+// first to skip the atomic would put an L2 round trip at the end of every append)
+__device__ inline void note_vmax(const CacheView &c, int u, uint32_t m) {
+  if (m) atomicMax(&c.vmax[u], m);
 }
 
 // element offset of (row, 16-byte chunk) inside a key or value block

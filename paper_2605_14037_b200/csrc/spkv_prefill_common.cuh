@@ -52,5 +52,6 @@ __device__ inline void prefill_work_item(const PrefillArgs &a, int item, int n_x
 // staging pages + chunk attention on tcgen05 (two heads per block when G is even)
 int launch_prefill_attn_tc5(const PrefillArgs &a, cudaStream_t s);
 int launch_prefill_attn_tc5x2(const PrefillArgs &a, cudaStream_t s);
+int launch_prefill_attn_tc5x2h(const PrefillArgs &a, cudaStream_t s);
 
 }  // namespace spkv

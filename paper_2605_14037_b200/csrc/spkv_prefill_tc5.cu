@@ -318,8 +318,12 @@ int launch_prefill_attn_tc5(const PrefillArgs &a, cudaStream_t s) {
     const char *e = getenv("SPKV_PREFILL_KERNEL");  // "tc5x1": one query head per block
     return e && e[0] == 't' && e[1] == 'c' && e[2] == '5' && e[3] == 'x' && e[4] == '1';
   }();
+  static const bool bf16_pv = [] {
+    const char *e = getenv("SPKV_PREFILL_PV");  // "bf16": the two-term bf16 P.V kernel (comparison)
+    return e && e[0] == 'b';
+  }();
   prefill_stage_kernel<<<dim3(a.n_stage_pages, a.c.Hkv), 256, 0, s>>>(a);
-  if (a.c.G % 2 == 0 && !one_head) return launch_prefill_attn_tc5x2(a, s);
+  if (a.c.G % 2 == 0 && !one_head) return bf16_pv ? launch_prefill_attn_tc5x2(a, s) : launch_prefill_attn_tc5x2h(a, s);
   prefill_attn_tc5_kernel<<<dim3(((a.C + 127) / 128) * a.c.Hq), tc5::kThreads, tc5::kSmemBytes, s>>>(a);
   return check_stream_error(cudaGetLastError());
 }

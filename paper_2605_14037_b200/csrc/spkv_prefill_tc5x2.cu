@@ -1,4 +1,6 @@
-// Chunk attention of spkv_prefill on tcgen05, two query heads per block.
+// Chunk attention of spkv_prefill on tcgen05, two query heads per block, P.V in two bf16 terms.
+// (The comparison kernel, SPKV_PREFILL_PV=bf16; the default is the fp16 P.V kernel in
+// spkv_prefill_tc5x2h.cu, which does a third less tensor work per page.)
 //
 // One block = 128 consecutive queries of TWO query heads that share a KV head (GQA, Eq. 5:
 // head j reads KV head j / G).  Both heads walk the same page list, so each 32 KB page is
@@ -24,9 +26,6 @@
 // warp schedulers favour lower-numbered warps when several are ready: as warp 9, behind two
 // always-ready softmax warps on its scheduler, it got an issue slot every ~9 cycles and the
 // tensor pipe starved.  All waits are bounded.
-#include <cstdlib>
-#include <cstring>
-
 #include "spkv_prefill_common.cuh"
 #include "spkv_tc5.cuh"
 
@@ -39,11 +38,8 @@ constexpr int kSQ = 0;                     // 2 x 32 KB: Q of head 0, head 1 (tw
 constexpr int kStages = 5;
 constexpr int kSKV = 65536;                // kStages x 32 KB
 constexpr int kSBar = kSKV + kStages * kPageBytes;
-constexpr int kSmemBytes = kSBar + 512;
-enum { B_KV_FULL = 0, B_KV_EMPTY = 8, B_S_FULL = 16 /* [2h+b] */, B_P_FULL = 20 /* [2h+b] */, B_O_DONE = 24 /* [2h+b] */,
-       B_V_READY = 28 /* [stage] */, B_COUNT = 36 };
-constexpr int kConvThreads = 64;           // warps 2-3 (fp16 P.V only)
-constexpr float kPBias = 7.f;              // fp16 P is stored as 2^7 p (p <= 2^8 by the lazy rescale)
+constexpr int kSmemBytes = kSBar + 256;
+enum { B_KV_FULL = 0, B_KV_EMPTY = 8, B_S_FULL = 16 /* [2h+b] */, B_P_FULL = 20 /* [2h+b] */, B_O_DONE = 24 /* [2h+b] */, B_COUNT = 28 };
 }  // namespace tc5x2
 
 #ifdef SPKV_TC5_TRACE
@@ -53,7 +49,6 @@ __device__ long long g_tc5_trace[16][2048];
 #define TC5_STAMP(cond, who, j) do { } while (0)
 #endif
 
-template <bool kHalfPV>
 __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(PrefillArgs a) {
   using namespace tc5;
   using namespace tc5x2;
@@ -69,18 +64,6 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
   const int32_t *E = hdr + kHdrInts;
   const int len0 = hdr[H_LEN0], n_old = hdr[H_NOLD], N = hdr[H_N];
   const int u = unit_index(c, a.layer, a.seq, kvh);
-  // fp16 P.V: the values are multiplied by 2^k with the unit's largest |v| brought into
-  // [2^14, 2^15) (every value the unit holds or this chunk brings is covered by vmax); the
-  // epilogue multiplies by 2^-k.  Both are exact.
-  float v_scale = 1.f, v_unscale = 1.f;
-  if (kHalfPV) {
-    const uint32_t vm = c.vmax[u];
-    if (vm) {
-      const int k = min(14 - ((int)(vm >> 23) - 127), 126);
-      v_scale = __int_as_float((127 + k) << 23);
-      v_unscale = __int_as_float((127 - k) << 23);
-    }
-  }
   // kept pairs visible to chunk query i: the first nvis(i) pairs of the compact cache
   auto nvis = [&](int i) { return len0 + E[min(max(i + n_old - c.w + 1, 0), N)]; };
   const int i_last = min(i0 + 127, a.C - 1);
@@ -93,7 +76,6 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
     for (int i = 0; i < kStages; ++i) {
       mbar_init(&bar[B_KV_FULL + i], 1);
       mbar_init(&bar[B_KV_EMPTY + i], 1);
-      mbar_init(&bar[B_V_READY + i], kConvThreads);
     }
     // One barrier per head and page parity: a parity wait only tells adjacent phases apart, and
     // producer and waiter of S, P and O can be two pages apart (a group may finish page j+1
@@ -161,7 +143,7 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
   } else if (warp == 0) {
     // ---------------------------------------------------------------- MMA issue (whole warp, one elected lane issues)
     {
-      constexpr uint32_t idesc_qk = instr_desc(128, 64, false), idesc_pv = instr_desc(128, 128, true, kHalfPV);
+      constexpr uint32_t idesc_qk = instr_desc(128, 64, false), idesc_pv = instr_desc(128, 128, true);
       const uint32_t sQ = smem_u32(smem + kSQ);
       auto issue_qk = [&](int h, int jj) {  // S_h[jj & 1] = Q_h . K(jj)^T
         const uint32_t sK = smem_u32(smem + kSKV + (jj % kStages) * kPageBytes);
@@ -182,8 +164,7 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
       auto issue_pv = [&](int h, int jj) {
         const uint32_t sV = smem_u32(smem + kSKV + (jj % kStages) * kPageBytes) + kBlockElems * 2;
         const uint32_t tP = tbase + (2 * h + (jj & 1)) * 64;
-        if (kHalfPV) umma_pv_page_f16(tbase + 256 + h * 128, tP, smem_desc(sV, 8192, 1024), idesc_pv, jj > 0 ? 1u : 0u);
-        else         umma_pv_page(tbase + 256 + h * 128, tP, smem_desc(sV, 8192, 1024), idesc_pv, jj > 0 ? 1u : 0u);
+        umma_pv_page(tbase + 256 + h * 128, tP, smem_desc(sV, 8192, 1024), idesc_pv, jj > 0 ? 1u : 0u);
         // the last two PVs have no later QK whose S_FULL would vouch for their completion
         if (jj + 2 >= n_tiles) umma_commit(&bar[B_O_DONE + 2 * h + (jj & 1)]);
         TC5_STAMP(traced && lane == 0, 11 + 2 * h, jj);
@@ -204,9 +185,6 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
       // waits and commits per page instead of one per head and page (every wait or commit
       // between two runs of MMAs lets the tensor pipe run dry for a few dozen clocks).
       for (int j = 0; j < n_tiles && !failed; ++j) {
-        TC5_STAMP(traced && lane == 0, 15, j);
-        if (kHalfPV && !mbar_wait_bounded(&bar[B_V_READY + j % kStages], (j / kStages) & 1)) failed = true;
-        TC5_STAMP(traced && lane == 0, 14, j);
         wait_p(0, j);
         wait_p(1, j);
         if (failed) break;
@@ -219,27 +197,8 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
           issue_qk(0, j + 2);
           issue_qk(1, j + 2);
           commit_s(j + 2);
-          TC5_STAMP(traced && lane == 0, 12, j);
         }
       }
-    }
-  } else if (kHalfPV && warp < 4) {
-    // ---------------------------------------------------------------- value converter (warps 2-3)
-    // bf16 -> fp16 in place, in the swizzled layout the copy left (element positions do not move)
-    const int ct = tid - 64;
-    for (int j = 0; j < n_tiles; ++j) {
-      const int s = j % kStages;
-      if (!mbar_wait_bounded(&bar[B_KV_FULL + s], (j / kStages) & 1)) { failed = true; break; }
-      uint4 *vb = reinterpret_cast<uint4 *>(smem + kSKV + s * kPageBytes + kBlockElems * 2) + ct;
-#pragma unroll 8
-      for (int x = 0; x < 16; ++x) {
-        uint4 r = vb[x * kConvThreads];
-        r.x = bf16x2_to_f16x2(r.x, v_scale); r.y = bf16x2_to_f16x2(r.y, v_scale);
-        r.z = bf16x2_to_f16x2(r.z, v_scale); r.w = bf16x2_to_f16x2(r.w, v_scale);
-        vb[x * kConvThreads] = r;
-      }
-      fence_async_smem();
-      mbar_arrive(&bar[B_V_READY + s]);
     }
   } else if (warp >= 4) {
     // ---------------------------------------------------------------- softmax groups
@@ -264,7 +223,7 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
         for (int x = 0; x < 16; ++x) v[q4 * 16 + x] = t16[x];
       }
       tmem_ld_wait();
-      TC5_STAMP(traced && row == 0, h * 4 + 1, j);
+      
       // visibility: compact-cache page j -> first nv pairs; staging page -> the band of this row.
       // v keeps the raw scores (masked ones become -inf); the scale is folded into the exponent,
       // and pages that every row of the warp sees in full skip the masking altogether.
@@ -317,27 +276,11 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
         l *= f;
       }
       m_ref = m_new;
-      TC5_STAMP(traced && row == 0, h * 4 + 2, j);
+      
       const float ms = m_ref == -INFINITY ? 0.f : m_ref;
       // two elements per instruction where the hardware has a packed form (fma, add, sub)
-      const float nms = kHalfPV ? kPBias - ms : -ms;
-      const uint64_t sc2 = pack2(a.scale_log2, a.scale_log2), nms2 = pack2(nms, nms);
+      const uint64_t sc2 = pack2(a.scale_log2, a.scale_log2), nms2 = pack2(-ms, -ms);
       uint64_t l2a = pack2(0.f, 0.f), l2b = l2a;
-      if (kHalfPV) {
-#pragma unroll
-        for (int q2 = 0; q2 < 2; ++q2) {  // 32 keys -> 16 columns of fp16 pairs
-          uint32_t ph[16];
-#pragma unroll
-          for (int x = 0; x < 16; ++x) {
-            float e0, e1;
-            unpack2(fma2(pack2(v[q2 * 32 + 2 * x], v[q2 * 32 + 2 * x + 1]), sc2, nms2), e0, e1);
-            const float p0 = fast_exp2(e0), p1 = fast_exp2(e1);
-            if (x & 1) l2b = add2(l2b, pack2(p0, p1)); else l2a = add2(l2a, pack2(p0, p1));
-            ph[x] = pack_f16(p0, p1);
-          }
-          tmem_st16u(t_s + q2 * 16, ph);
-        }
-      } else {
 #pragma unroll
       for (int q2 = 0; q2 < 2; ++q2) {  // 32 keys -> 16 columns of hi, 16 of lo
         uint32_t hi[16], lo[16];
@@ -356,38 +299,32 @@ __global__ void __launch_bounds__(tc5x2::kThreads, 1) prefill_attn_tc5x2_kernel(
         tmem_st16u(t_s + q2 * 16, hi);
         tmem_st16u(t_s + 32 + q2 * 16, lo);
       }
-      }
       {
         float la, lb;
         unpack2(add2(l2a, l2b), la, lb);
         l += la + lb;
       }
-      TC5_STAMP(traced && row == 0 && h == 0, 6, j);
       tmem_st_wait();
       fence_before();
       mbar_arrive(&bar[B_P_FULL + 2 * h + (j & 1)]);
       TC5_STAMP(traced && row == 0, h * 4 + 3, j);
+      TC5_STAMP(traced && h == 0 && lane == 0 && warp > 4, warp - 4, j);  // rows 1-3: P arrival of warps 1-3 (trace only)
     }
     if (!failed && mbar_wait_bounded(&bar[B_O_DONE + 2 * h + ((n_tiles - 1) & 1)], 0)) {
       fence_after();
-      const float inv = l > 0.f ? 1.f / l : 0.f;  // the bias of P cancels between O and l
+      const float inv = l > 0.f ? 1.f / l : 0.f;
       __nv_bfloat16 *orow = a.out + ((size_t)i * c.Hq + hq) * kD;
 #pragma unroll
       for (int q8 = 0; q8 < 8; ++q8) {
         float t16[16];
         tmem_ld16(t_o + q8 * 16, t16);
         tmem_ld_wait();
-#pragma unroll
-        for (int x = 0; x < 16; ++x) {
-          t16[x] *= inv;                         // |O| / l < 2^15 in the scaled units ...
-          if (kHalfPV) t16[x] *= v_unscale;      // ... and <= max |v| after this: no overflow in between
-        }
         if (row_ok) {
           uint4 w0, w1;
-          w0.x = pack_bf16(t16[0], t16[1]);   w0.y = pack_bf16(t16[2], t16[3]);
-          w0.z = pack_bf16(t16[4], t16[5]);   w0.w = pack_bf16(t16[6], t16[7]);
-          w1.x = pack_bf16(t16[8], t16[9]);   w1.y = pack_bf16(t16[10], t16[11]);
-          w1.z = pack_bf16(t16[12], t16[13]); w1.w = pack_bf16(t16[14], t16[15]);
+          w0.x = pack_bf16(t16[0] * inv, t16[1] * inv);   w0.y = pack_bf16(t16[2] * inv, t16[3] * inv);
+          w0.z = pack_bf16(t16[4] * inv, t16[5] * inv);   w0.w = pack_bf16(t16[6] * inv, t16[7] * inv);
+          w1.x = pack_bf16(t16[8] * inv, t16[9] * inv);   w1.y = pack_bf16(t16[10] * inv, t16[11] * inv);
+          w1.z = pack_bf16(t16[12] * inv, t16[13] * inv); w1.w = pack_bf16(t16[14] * inv, t16[15] * inv);
           *reinterpret_cast<uint4 *>(orow + q8 * 16) = w0;
           *reinterpret_cast<uint4 *>(orow + q8 * 16 + 8) = w1;
         }
@@ -410,14 +347,10 @@ extern "C" int spkv_debug_tc5_trace(long long *host_out) {
 #endif
 
 int launch_prefill_attn_tc5x2(const PrefillArgs &a, cudaStream_t s) {
-  static const bool half_pv = [] {
-    const char *e = getenv("SPKV_PREFILL_PV");  // "bf16": the two-term bf16 P.V (comparison)
-    return !(e != nullptr && strcmp(e, "bf16") == 0);
-  }();
-  auto kern = half_pv ? prefill_attn_tc5x2_kernel<true> : prefill_attn_tc5x2_kernel<false>;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc5x2::kSmemBytes) != cudaSuccess)
+  if (cudaFuncSetAttribute(prefill_attn_tc5x2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           tc5x2::kSmemBytes) != cudaSuccess)
     return SPKV_E_CUDA;
-  kern<<<dim3(((a.C + 127) / 128) * a.c.Hkv * (a.c.G / 2)), tc5x2::kThreads, tc5x2::kSmemBytes, s>>>(a);
+  prefill_attn_tc5x2_kernel<<<dim3(((a.C + 127) / 128) * a.c.Hkv * (a.c.G / 2)), tc5x2::kThreads, tc5x2::kSmemBytes, s>>>(a);
   return check_stream_error(cudaGetLastError());
 }
 

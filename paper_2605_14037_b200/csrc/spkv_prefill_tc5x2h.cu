@@ -1,0 +1,408 @@
+// Chunk attention of spkv_prefill on tcgen05, two query heads per block, P.V in fp16.
+//
+// Same tiling as the two-term bf16 kernel next door (one block = 128 consecutive queries of two
+// query heads that share a KV head, Eq. 5; every 32 KB page is fetched once and feeds both; one
+// softmax group of 128 threads per head, thread = query row = TMEM lane).  Two things differ:
+//
+// * P is ONE fp16 term (11 significant bits; the two-term bf16 split carries 16 but costs a second
+//   P.V pass).  The tensor cores want both operands in the same type, so warps 2-3 rewrite the
+//   value block of every page from bf16 to fp16 in shared memory, multiplied by a power of two
+//   that brings the largest |v| the unit has ever received into [2^14, 2^15) -- any bf16 range
+//   fits, and the epilogue undoes the factor exactly.  P carries a bias of 2^7 (p <= 2^8 under the
+//   lazy rescale), which cancels between O and the row sum.
+//
+// * P has tensor-memory columns of its own instead of overwriting the scores it came from.  A
+//   group copies its row of S into registers and hands the S buffer back at once, so Q.K^T of the
+//   next page runs under the softmax of this one and never waits for P; only P.V does.  With P
+//   aliased onto S, Q.K^T(j+2) had to queue behind P.V(j), and scores, softmax and P.V of a head
+//   formed one dependent loop whose latency, not the tensor pipe, set the pace.
+//
+// Tensor memory (512 columns): S of head h at [64 h, +64); P buffer b of head h at
+// [128 + 32 (2h + b), +32) (two fp16 per column); O of head h at [256 + 128 h, +128).
+// MMA order per page j:  QK0(j+1) | PV0(j) | QK1(j+1) | PV1(j).  The two heads' scores become
+// ready half a page apart, which keeps the two groups out of step: the exponentials of one
+// (special-function unit, the scarce resource) run under the load / maximum / hand-over phases of
+// the other instead of both queueing for the same unit at the same time.
+//
+// What bounds the kernel is shared-memory bandwidth: per page the tensor cores read Q twice over
+// (every K=16 step re-reads its 4 KB slice of Q: 64 KB), K and V once per head (64 KB), the copy
+// engine writes the page (32 KB) and the conversion reads and rewrites V (32 KB) -- about 1500
+// of the ~1750 cycles a page takes at 128 B per cycle.  (Computing part of the exponentials by
+// polynomial on the FMA pipe, which helps when the special-function unit is the limit, only
+// added instructions here and was dropped.)
+// Shared memory: Q of both heads (64 KB) + 5 page stages.
+// Warps: 0 MMA issue, 1 page loader + TMEM allocation, 2-3 value conversion, 4-7 group 0,
+// 8-11 group 1.  All waits are bounded.
+#include <cstdlib>
+#include <cstring>
+
+#include "spkv_prefill_common.cuh"
+#include "spkv_tc5.cuh"
+
+namespace spkv {
+
+namespace tc5x2h {
+constexpr int kThreads = 384;
+constexpr int kTmemCols = 512;
+constexpr int kSQ = 0;                     // 2 x 32 KB: Q of head 0, head 1 (two slabs of 128 rows x 128 B each)
+constexpr int kStages = 5;
+constexpr int kSKV = 65536;                // kStages x 32 KB
+constexpr int kSBar = kSKV + kStages * kPageBytes;
+constexpr int kSmemBytes = kSBar + 512;
+enum { B_KV_FULL = 0, B_KV_EMPTY = 8, B_V_READY = 16 /* [stage] */, B_S_FULL = 24 /* [h] */, B_S_FREE = 26 /* [h] */,
+       B_P_FULL = 28 /* [2h+b] */, B_O_DONE = 32 /* [2h+b] */, B_COUNT = 36 };
+constexpr int kConvThreads = 64;           // warps 2-3
+constexpr float kPBias = 7.f;              // P is stored as 2^7 p
+}  // namespace tc5x2h
+
+#ifdef SPKV_TC5_TRACE
+__device__ long long g_tc5h_trace[16][2048];
+#define TC5H_STAMP(cond, who, j) do { if ((cond) && (j) < 2048) g_tc5h_trace[who][j] = clock64(); } while (0)
+#else
+#define TC5H_STAMP(cond, who, j) do { } while (0)
+#endif
+
+__global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kernel(PrefillArgs a) {
+  using namespace tc5;
+  using namespace tc5x2h;
+  extern __shared__ __align__(1024) unsigned char smem[];
+  const CacheView &c = a.c;
+  uint64_t *bar = reinterpret_cast<uint64_t *>(smem + kSBar);
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + kSBar + B_COUNT * 8);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  int kvh, pair, xtile;
+  prefill_work_item(a, blockIdx.x, (a.C + 127) / 128, c.G >> 1, kvh, pair, xtile);
+  const int hq0 = kvh * c.G + pair * 2, i0 = xtile * 128;
+  const int32_t *hdr = unit_ws(a, kvh);
+  const int32_t *E = hdr + kHdrInts;
+  const int len0 = hdr[H_LEN0], n_old = hdr[H_NOLD], N = hdr[H_N];
+  const int u = unit_index(c, a.layer, a.seq, kvh);
+  // The values are multiplied by 2^k with the unit's largest |v| brought into [2^14, 2^15) (every
+  // value the unit holds or this chunk brings is covered by vmax); the epilogue multiplies by
+  // 2^-k.  Both are exact.
+  float v_scale = 1.f, v_unscale = 1.f;
+  {
+    const uint32_t vm = c.vmax[u];
+    if (vm) {
+      const int k = min(14 - ((int)(vm >> 23) - 127), 126);
+      v_scale = __int_as_float((127 + k) << 23);
+      v_unscale = __int_as_float((127 - k) << 23);
+    }
+  }
+  // kept pairs visible to chunk query i: the first nvis(i) pairs of the compact cache
+  auto nvis = [&](int i) { return len0 + E[min(max(i + n_old - c.w + 1, 0), N)]; };
+  const int i_last = min(i0 + 127, a.C - 1);
+  const int n_ptiles = (nvis(i_last) + kP - 1) / kP;
+  // band, in staging indices (query i is staging pair n_old + i)
+  const int sp_lo = max(0, i0 + n_old - c.w + 1) / kP, sp_hi = (i_last + n_old) / kP;
+  const int n_tiles = n_ptiles + (sp_hi - sp_lo + 1);
+
+  if (tid == 0) {
+    for (int i = 0; i < kStages; ++i) {
+      mbar_init(&bar[B_KV_FULL + i], 1);
+      mbar_init(&bar[B_KV_EMPTY + i], 1);
+      mbar_init(&bar[B_V_READY + i], kConvThreads);
+    }
+    // S_FULL / S_FREE: one barrier per head, one phase per page -- the MMA thread commits the
+    // scores of page j+1 only after the group has freed the buffer of page j, and the group frees
+    // it only after seeing it full, so the two are never more than one phase apart.
+    // P_FULL / O_DONE: one per head and page parity -- a group may hand over P(j+1) before the MMA
+    // thread has looked at P(j).  P(j+2) cannot follow before that: it needs the scores of page
+    // j+2, whose Q.K^T is issued after P.V(j).  O_DONE is committed for the last two pages only.
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&bar[B_S_FULL + i], 1);
+      mbar_init(&bar[B_S_FREE + i], 128);
+    }
+    for (int i = 0; i < 4; ++i) {
+      mbar_init(&bar[B_P_FULL + i], 128);
+      mbar_init(&bar[B_O_DONE + i], 1);
+    }
+    mbar_fence_init();
+  }
+  // Q tiles -> per head two slabs of 128 rows x 128 B, 128-byte swizzle (rows past the chunk are zero)
+  for (int x = tid; x < 2 * 128 * 16; x += kThreads) {
+    const int h = x >> 11, r = (x >> 4) & 127, ch = x & 15;
+    uint4 val = make_uint4(0, 0, 0, 0);
+    if (i0 + r < a.C) val = *reinterpret_cast<const uint4 *>(a.q + ((size_t)(i0 + r) * c.Hq + hq0 + h) * kD + ch * 8);
+    *reinterpret_cast<uint4 *>(smem + kSQ + h * 32768 + (ch >> 3) * 16384 + r * 128 + (((ch & 7) ^ (r & 7)) << 4)) = val;
+  }
+  fence_async_smem();
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "n"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  fence_before();
+  __syncthreads();
+  fence_after();
+  const uint32_t tbase = *tmem_slot;
+  bool failed = false;
+#ifdef SPKV_TC5_TRACE
+  const bool traced = blockIdx.x == 0;
+#endif
+
+  if (warp == 1) {
+    // ---------------------------------------------------------------- page loader
+    int j = 0;
+    for (int base = 0; base < n_tiles && !failed; base += 32) {
+      const int jl = base + lane;
+      int64_t src_off = 0;
+      if (jl < n_ptiles) src_off = (int64_t)c.table[(size_t)u * c.max_pages + jl] * kPageElems;
+      const int cnt = min(32, n_tiles - base);
+      for (int x = 0; x < cnt; ++x, ++j) {
+        const int64_t off = __shfl_sync(0xffffffffu, src_off, x);
+        if (lane == 0) {
+          const int s = j % kStages;
+          if (j >= kStages && !mbar_wait_bounded(&bar[B_KV_EMPTY + s], ((j / kStages) - 1) & 1)) failed = true;
+          if (!failed) {
+            const __nv_bfloat16 *src =
+                j < n_ptiles ? c.pages + off
+                             : a.stage_pages + ((size_t)kvh * a.n_stage_pages + sp_lo + (j - n_ptiles)) * kPageElems;
+            mbar_arrive_expect_tx(&bar[B_KV_FULL + s], kPageBytes);
+            bulk_load(smem + kSKV + s * kPageBytes, src, kPageBytes, &bar[B_KV_FULL + s]);
+          }
+        }
+        failed = __shfl_sync(0xffffffffu, (int)failed, 0) != 0;
+        if (failed) break;
+      }
+    }
+    if (failed && lane == 0)  // do not leave while copies may still be landing
+      for (int k = max(0, j - kStages); k < j; ++k)
+        mbar_wait_bounded(&bar[B_KV_FULL + (k % kStages)], (k / kStages) & 1);
+  } else if (warp == 0) {
+    // ---------------------------------------------------------------- MMA issue (whole warp, one elected lane issues)
+    constexpr uint32_t idesc_qk = instr_desc(128, 64, false), idesc_pv = instr_desc(128, 128, true, true);
+    const uint32_t sQ = smem_u32(smem + kSQ);
+    auto wait_page = [&](int jj) {
+      if (!mbar_wait_bounded(&bar[B_KV_FULL + jj % kStages], (jj / kStages) & 1)) failed = true;
+      fence_after();
+    };
+    auto issue_qk = [&](int h, int jj) {  // S_h = Q_h . K(jj)^T, committed at once
+      const uint32_t sK = smem_u32(smem + kSKV + (jj % kStages) * kPageBytes);
+      umma_qk_page<16384 / 16, 8192 / 16>(tbase + h * 64, smem_desc(sQ + h * 32768, 16, 1024), smem_desc(sK, 16, 1024),
+                                          idesc_qk);
+      umma_commit(&bar[B_S_FULL + h]);
+    };
+    // the group has copied the scores of page jj out of the S buffer
+    auto wait_s_free = [&](int h, int jj) {
+      if (!mbar_wait_bounded(&bar[B_S_FREE + h], jj & 1)) failed = true;
+      fence_after();
+    };
+    // O_h += P_h(jj) . V(jj): A from tensor memory, B = the page's value block (fp16 by now), MN-major
+    auto issue_pv = [&](int h, int jj) {
+      if (!mbar_wait_bounded(&bar[B_P_FULL + 2 * h + (jj & 1)], (jj >> 1) & 1)) failed = true;
+      TC5H_STAMP(traced && lane == 0, 8 + h, jj);
+      fence_after();
+      if (failed) return;
+      const uint32_t sV = smem_u32(smem + kSKV + (jj % kStages) * kPageBytes) + kBlockElems * 2;
+      umma_pv_page_f16(tbase + 256 + h * 128, tbase + 128 + (2 * h + (jj & 1)) * 32, smem_desc(sV, 8192, 1024), idesc_pv,
+                       jj > 0 ? 1u : 0u);
+      // the last two P.V have no later Q.K^T whose S_FULL would vouch for their completion
+      if (jj + 2 >= n_tiles) umma_commit(&bar[B_O_DONE + 2 * h + (jj & 1)]);
+    };
+    wait_page(0);
+    if (!failed) {
+      issue_qk(0, 0);
+      issue_qk(1, 0);
+    }
+    for (int j = 0; j < n_tiles && !failed; ++j) {
+      const bool more = j + 1 < n_tiles;
+      TC5H_STAMP(traced && lane == 0, 15, j);
+      if (more) {
+        wait_page(j + 1);
+        wait_s_free(0, j);
+        if (failed) break;
+        issue_qk(0, j + 1);
+      }
+      TC5H_STAMP(traced && lane == 0, 14, j);
+      if (!mbar_wait_bounded(&bar[B_V_READY + j % kStages], (j / kStages) & 1)) failed = true;
+      if (failed) break;
+      issue_pv(0, j);
+      if (failed) break;
+      TC5H_STAMP(traced && lane == 0, 13, j);
+      if (more) {
+        wait_s_free(1, j);
+        if (failed) break;
+        issue_qk(1, j + 1);
+      }
+      TC5H_STAMP(traced && lane == 0, 12, j);
+      issue_pv(1, j);
+      if (failed) break;
+      umma_commit(&bar[B_KV_EMPTY + (j % kStages)]);  // page j has no reader left
+    }
+  } else if (warp < 4) {
+    // ---------------------------------------------------------------- value converter (warps 2-3)
+    // bf16 -> fp16 in place, in the swizzled layout the copy left (element positions do not move)
+    const int ct = tid - 64;
+    for (int j = 0; j < n_tiles; ++j) {
+      const int s = j % kStages;
+      if (!mbar_wait_bounded(&bar[B_KV_FULL + s], (j / kStages) & 1)) { failed = true; break; }
+      uint4 *vb = reinterpret_cast<uint4 *>(smem + kSKV + s * kPageBytes + kBlockElems * 2) + ct;
+#pragma unroll 8
+      for (int x = 0; x < 16; ++x) {
+        uint4 r = vb[x * kConvThreads];
+        r.x = bf16x2_to_f16x2(r.x, v_scale); r.y = bf16x2_to_f16x2(r.y, v_scale);
+        r.z = bf16x2_to_f16x2(r.z, v_scale); r.w = bf16x2_to_f16x2(r.w, v_scale);
+        vb[x * kConvThreads] = r;
+      }
+      fence_async_smem();
+      mbar_arrive(&bar[B_V_READY + s]);
+    }
+  } else {
+    // ---------------------------------------------------------------- softmax groups
+    const int h = (warp >> 2) - 1, row = tid & 127, i = i0 + row, hq = hq0 + h;
+    const bool row_ok = i < a.C;
+    const int nv = row_ok ? nvis(i) : 0;
+    const int jq = n_old + i;  // staging index of this row's own pair
+    const uint32_t t_lane = tbase + ((uint32_t)((warp & 3) * 32) << 16);
+    const uint32_t t_s = t_lane + h * 64, t_o = t_lane + 256 + h * 128;
+    float m_ref = -INFINITY, l = 0.f;
+    for (int j = 0; j < n_tiles; ++j) {
+      if (!mbar_wait_bounded(&bar[B_S_FULL + h], j & 1)) { failed = true; break; }
+      TC5H_STAMP(traced && row == 0, h * 4 + 0, j);
+      fence_after();
+      float v[64];
+#pragma unroll
+      for (int q4 = 0; q4 < 4; ++q4) {
+        float t16[16];
+        tmem_ld16(t_s + q4 * 16, t16);
+#pragma unroll
+        for (int x = 0; x < 16; ++x) v[q4 * 16 + x] = t16[x];
+      }
+      tmem_ld_wait();
+      // the scores are in registers: Q.K^T of the next page may overwrite the buffer
+      fence_before();
+      mbar_arrive(&bar[B_S_FREE + h]);
+      TC5H_STAMP(traced && row == 0, h * 4 + 1, j);
+      // visibility: compact-cache page j -> first nv pairs; staging page -> the band of this row.
+      // v keeps the raw scores (masked ones become -inf); the scale is folded into the exponent,
+      // and pages that every row of the warp sees in full skip the masking altogether.
+      if (j < n_ptiles) {
+        const int base = j * kP;
+        if (!__all_sync(0xffffffffu, base + kP <= nv)) {
+#pragma unroll
+          for (int x = 0; x < 64; ++x) v[x] = (base + x < nv) ? v[x] : -INFINITY;
+        }
+      } else {
+        const int base = (sp_lo + j - n_ptiles) * kP;
+#pragma unroll
+        for (int x = 0; x < 64; ++x) {
+          const int jj = base + x;
+          v[x] = (row_ok && jj <= jq && jj > jq - c.w) ? v[x] : -INFINITY;
+        }
+      }
+      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+      for (int x = 0; x < 64; x += 8) {
+        mx0 = max3(mx0, v[x], v[x + 1]);
+        mx1 = max3(mx1, v[x + 2], v[x + 3]);
+        mx2 = max3(mx2, v[x + 4], v[x + 5]);
+        mx3 = max3(mx3, v[x + 6], v[x + 7]);
+      }
+      const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * a.scale_log2;  // scale > 0 (host-checked)
+      // the reference maximum moves only when the row maximum outgrows it by 2^8
+      const bool grow = mx > m_ref + 8.f;
+      const float m_new = grow ? mx : m_ref;
+      if (j > 0 && __any_sync(0xffffffffu, grow)) {
+        // O is stable between the completion of PV(j-1) and the hand-over of P(j).  QK(j+1) is
+        // issued after PV(j-1) and needs nothing more from this group (the S buffer is free), so
+        // S_FULL(j+1) vouches for it (waiting on it here does not consume the phase); the last
+        // page has its own barrier.
+        if (!(j + 1 < n_tiles ? mbar_wait_bounded(&bar[B_S_FULL + h], (j + 1) & 1)
+                              : mbar_wait_bounded(&bar[B_O_DONE + 2 * h + ((j - 1) & 1)], 0))) {
+          failed = true;
+          break;
+        }
+        fence_after();
+        const float f = grow ? fast_exp2(m_ref - m_new) : 1.f;  // m_ref = -inf -> 0
+#pragma unroll
+        for (int q8 = 0; q8 < 8; ++q8) {
+          float t16[16];
+          tmem_ld16(t_o + q8 * 16, t16);
+          tmem_ld_wait();
+#pragma unroll
+          for (int x = 0; x < 16; ++x) t16[x] *= f;
+          tmem_st16(t_o + q8 * 16, t16);
+        }
+        l *= f;
+      }
+      m_ref = m_new;
+      TC5H_STAMP(traced && row == 0, h * 4 + 2, j);
+      const float ms = m_ref == -INFINITY ? 0.f : m_ref;
+      // two elements per instruction where the hardware has a packed form (fma, add)
+      const uint64_t sc2 = pack2(a.scale_log2, a.scale_log2), nms2 = pack2(kPBias - ms, kPBias - ms);
+      uint64_t l2a = pack2(0.f, 0.f), l2b = l2a;
+      // P buffer (j & 1) is free: S_FULL(j) completed after P.V(j-2)
+      const uint32_t t_p = t_lane + 128 + (2 * h + (j & 1)) * 32;
+#pragma unroll
+      for (int q2 = 0; q2 < 2; ++q2) {  // 32 keys -> 16 columns of fp16 pairs
+        uint32_t ph[16];
+#pragma unroll
+        for (int x = 0; x < 16; ++x) {
+          float e0, e1;
+          unpack2(fma2(pack2(v[q2 * 32 + 2 * x], v[q2 * 32 + 2 * x + 1]), sc2, nms2), e0, e1);
+          const float p0 = fast_exp2(e0), p1 = fast_exp2(e1);
+          const uint64_t p2 = pack2(p0, p1);
+          if (x & 1) l2b = add2(l2b, p2); else l2a = add2(l2a, p2);
+          ph[x] = pack_f16(p0, p1);
+        }
+        tmem_st16u(t_p + q2 * 16, ph);
+      }
+      {
+        float la, lb;
+        unpack2(add2(l2a, l2b), la, lb);
+        l += la + lb;
+      }
+      tmem_st_wait();
+      fence_before();
+      mbar_arrive(&bar[B_P_FULL + 2 * h + (j & 1)]);
+      TC5H_STAMP(traced && row == 0, h * 4 + 3, j);
+    }
+    if (!failed && mbar_wait_bounded(&bar[B_O_DONE + 2 * h + ((n_tiles - 1) & 1)], 0)) {
+      fence_after();
+      const float inv = l > 0.f ? 1.f / l : 0.f;  // the bias of P cancels between O and l
+      __nv_bfloat16 *orow = a.out + ((size_t)i * c.Hq + hq) * kD;
+#pragma unroll
+      for (int q8 = 0; q8 < 8; ++q8) {
+        float t16[16];
+        tmem_ld16(t_o + q8 * 16, t16);
+        tmem_ld_wait();
+#pragma unroll
+        for (int x = 0; x < 16; ++x) t16[x] = t16[x] * inv * v_unscale;  // |O| / l < 2^15 in the scaled units, then <= max |v|
+        if (row_ok) {
+          uint4 w0, w1;
+          w0.x = pack_bf16(t16[0], t16[1]);   w0.y = pack_bf16(t16[2], t16[3]);
+          w0.z = pack_bf16(t16[4], t16[5]);   w0.w = pack_bf16(t16[6], t16[7]);
+          w1.x = pack_bf16(t16[8], t16[9]);   w1.y = pack_bf16(t16[10], t16[11]);
+          w1.z = pack_bf16(t16[12], t16[13]); w1.w = pack_bf16(t16[14], t16[15]);
+          *reinterpret_cast<uint4 *>(orow + q8 * 16) = w0;
+          *reinterpret_cast<uint4 *>(orow + q8 * 16 + 8) = w1;
+        }
+      }
+    } else {
+      failed = true;
+    }
+  }
+  if (failed) set_status(c, SPKV_E_TIMEOUT);
+  fence_before();
+  __syncthreads();
+  if (warp == 1)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tbase), "n"(tc5x2h::kTmemCols) : "memory");
+}
+
+#ifdef SPKV_TC5_TRACE
+extern "C" int spkv_debug_tc5h_trace(long long *host_out) {
+  return cudaMemcpyFromSymbol(host_out, g_tc5h_trace, sizeof(g_tc5h_trace)) == cudaSuccess ? 0 : -1;
+}
+#endif
+
+int launch_prefill_attn_tc5x2h(const PrefillArgs &a, cudaStream_t s) {
+  if (cudaFuncSetAttribute(prefill_attn_tc5x2h_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           tc5x2h::kSmemBytes) != cudaSuccess)
+    return SPKV_E_CUDA;
+  prefill_attn_tc5x2h_kernel<<<dim3(((a.C + 127) / 128) * a.c.Hkv * (a.c.G / 2)), tc5x2h::kThreads, tc5x2h::kSmemBytes,
+                               s>>>(a);
+  return check_stream_error(cudaGetLastError());
+}
+
+}  // namespace spkv
