@@ -24,12 +24,10 @@
 // (special-function unit, the scarce resource) run under the load / maximum / hand-over phases of
 // the other instead of both queueing for the same unit at the same time.
 //
-// What bounds the kernel is shared-memory bandwidth: per page the tensor cores read Q twice over
-// (every K=16 step re-reads its 4 KB slice of Q: 64 KB), K and V once per head (64 KB), the copy
-// engine writes the page (32 KB) and the conversion reads and rewrites V (32 KB) -- about 1500
-// of the ~1750 cycles a page takes at 128 B per cycle.  (Computing part of the exponentials by
-// polynomial on the FMA pipe, which helps when the special-function unit is the limit, only
-// added instructions here and was dropped.)
+// No unit is saturated (tensor pipe ~54 % active, special-function unit ~41 %, issue slots ~54 %):
+// the page period is the length of the chain scores -> softmax -> P -> MMA warp -> next scores.
+// (Computing part of the exponentials by polynomial on the FMA pipe, which helps when the
+// special-function unit is the limit, only added instructions here and was dropped.)
 // Shared memory: Q of both heads (64 KB) + 5 page stages.
 // Warps: 0 MMA issue, 1 page loader + TMEM allocation, 2-3 value conversion, 4-7 group 0,
 // 8-11 group 1.  All waits are bounded.
