@@ -173,3 +173,33 @@ def test_prefill_pool_exhaustion_reports_and_keeps_length():
     assert cache.spkv_status() == -5
     ln, tt = cache.spkv_read_lengths(0)
     assert ln[0, 0] == 96 and tt[0, 0] == 600
+
+
+@pytest.mark.parametrize("direction", [1.0, -1.0])
+def test_prefill_scores_that_grow_or_fall_with_position(direction):
+    """Raw scores 2t (or -2t) for the first head of every pair: with direction +1 the row maximum
+    grows by ~16 (log2 units, after the 1/sqrt(d) scale) from one 64-key page to the next, so the accumulator is rescaled
+    on every page, the last one included; with -1 everything after a row's first visible page
+    underflows.  The second head of every pair keeps ordinary scores, so the two softmax groups
+    of a block take different paths side by side."""
+    from paper_2605_14037_b200 import synth
+    spkv = load()
+    w, Hq, Hkv, G, chunks = 128, 4, 2, 2, [300, 400, 1, 130]
+    T = sum(chunks)
+    cache = spkv.Cache(n_layers=1, max_seqs=1, n_q_heads=Hq, n_kv_heads=Hkv, max_context=2048,
+                       pool_pages=40, window=w, tau=0.5)
+    tl = cache.spkv_tau_logit()
+    wl = Workload(321, T, 1, Hq, Hkv, [0.5, 0.35], tl)
+    Kf = synth.bf16_bits_to_f32(wl.K)
+    Kf[:, 0, :, 0] = (direction * 0.25 * np.arange(T, dtype=np.float32))[:, None]
+    wl.K = synth.to_bf16_bits(Kf)
+    qf = synth.bf16_bits_to_f32(wl.q)
+    qf[:, 0, 0::2, :] = 0.0
+    qf[:, 0, 0::2, 0] = 8.0
+    wl.q = synth.to_bf16_bits(qf)
+    got = prefill_in_chunks(spkv, cache, 0, 0, wl, 0, chunks)
+    assert cache.spkv_status() == 0
+    units, ref = oracle_prefill(wl, 0, w, tl, G, T, 1.0 / math.sqrt(D))   # 2t / sqrt(128) * log2(e) = 0.255 t
+    for h in range(Hkv):
+        compare_state(cache, 0, 0, h, units[h])
+    assert_attn_close(got, ref, f"direction={direction}")
