@@ -16,12 +16,14 @@ pytestmark = pytest.mark.gpu
 
 
 def run_and_check(spkv, w, T, Hq, Hkv, n_seq, tau, rates, check_steps, seed, sm_scale=None,
-                  pool_pages=200, max_context=8192):
+                  pool_pages=200, max_context=8192, tweak=None):
     cache = spkv.Cache(n_layers=2, max_seqs=n_seq + 1, n_q_heads=Hq, n_kv_heads=Hkv,
                        max_context=max_context, pool_pages=pool_pages, window=w, tau=tau)
     tl = cache.spkv_tau_logit()
     G = Hq // Hkv
     wl = Workload(seed, T, n_seq, Hq, Hkv, rates, tl)
+    if tweak is not None:
+        tweak(wl)
     seq_ids = list(range(n_seq, 0, -1))          # slots n_seq..1, reversed order
     ids = torch.tensor(seq_ids, dtype=torch.int32, device=dev())
     K, V, Q = to_dev_bf16(wl.K), to_dev_bf16(wl.V), to_dev_bf16(wl.q)
@@ -76,6 +78,26 @@ def test_decode_many_segments_and_ragged_batch():
     run_and_check(spkv, 128, 5200, 32, 8, 2, 0.5,
                   [0.0, 0.02, 0.1, 0.2, 0.35, 0.5, 0.8, 1.0], {4000, 5199}, 70,
                   pool_pages=700, max_context=8192)
+
+
+@pytest.mark.parametrize("direction", [1.0, -1.0])
+def test_decode_scores_that_grow_or_fall_with_position(direction):
+    """Raw scores +-0.4 t for every other query head: the running maximum moves on every tile
+    (or never after the first), and the partial results of a unit's page ranges carry maxima
+    hundreds apart into the log-sum-exp merge.  The other heads keep ordinary scores."""
+    spkv = load()
+
+    def tweak(wl):
+        Kf = synth.bf16_bits_to_f32(wl.K)
+        Kf[..., 0] = (direction * 0.05 * np.arange(wl.T, dtype=np.float32))[:, None, None]
+        wl.K = synth.to_bf16_bits(Kf)
+        qf = synth.bf16_bits_to_f32(wl.q)
+        qf[:, :, 0::2, :] = 0.0
+        qf[:, :, 0::2, 0] = 8.0
+        wl.q = synth.to_bf16_bits(qf)
+
+    run_and_check(spkv, 128, 5200, 32, 8, 2, 0.5, [0.0, 0.02, 0.1, 0.2, 0.35, 0.5, 0.8, 1.0],
+                  {130, 4000, 5199}, 71, pool_pages=700, max_context=8192, tweak=tweak)
 
 
 def test_decode_scale_and_batch_of_one():
