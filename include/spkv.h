@@ -213,6 +213,15 @@ int spkv_decode_attention(spkv_cache_t *cache, int32_t layer, const int32_t *d_s
                           float sm_scale, void *d_workspace, size_t workspace_bytes,
                           spkv_stream_t stream);
 
+/* spkv_decode_attention that also returns the output rows in float32, as they are before the
+ * rounding to bf16 (bf16 rounding alone is up to 2^-9 |o|, which hides smaller errors of the
+ * kernel from a comparison): d_out_f32 [B, n_q_heads, 128] float32, device, 16-byte aligned,
+ * required.  d_out is written as usual.  Everything else as spkv_decode_attention. */
+int spkv_decode_attention_f32(spkv_cache_t *cache, int32_t layer, const int32_t *d_seq_ids,
+                              int32_t B, const void *d_q, void *d_out, float *d_out_f32,
+                              float *d_lse_opt, float sm_scale, void *d_workspace,
+                              size_t workspace_bytes, spkv_stream_t stream);
+
 /* (No counterpart in the paper: an addition for integration.)
  * spkv_decode_attention for callers that must not allocate device memory -- code running
  * inside someone else's memory plan, where every cudaMalloc is forbidden or already spoken

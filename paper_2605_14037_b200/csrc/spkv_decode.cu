@@ -307,6 +307,8 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
       for (int g = 0; g < a.G; ++g) {
         __nv_bfloat16 *o = a.out + ((size_t)b * c.Hq + kvh * a.G + g) * kD;
         for (int d = 0; d < kD; ++d) o[d] = __float2bfloat16(0.f);
+        if (a.out_f32)
+          for (int d = 0; d < kD; ++d) a.out_f32[((size_t)b * c.Hq + kvh * a.G + g) * kD + d] = 0.f;
         if (a.lse) a.lse[(size_t)b * c.Hq + kvh * a.G + g] = -INFINITY;
       }
     }
@@ -544,6 +546,9 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
           pk.x = pack_bf16(Os.x * inv, Os.y * inv);
           pk.y = pack_bf16(Os.z * inv, Os.w * inv);
           *reinterpret_cast<uint2 *>(a.out + row * kD + lane * 4) = pk;
+          if (a.out_f32)
+            *reinterpret_cast<float4 *>(a.out_f32 + row * kD + lane * 4) =
+                make_float4(Os.x * inv, Os.y * inv, Os.z * inv, Os.w * inv);
           if (a.lse && lane == 0) a.lse[row] = (M + log2f(Ls)) * kLn2;
         } else {
           *reinterpret_cast<float4 *>(a.part_acc + ((size_t)slot * a.G + gh) * kD + lane * 4) = Os;
@@ -621,6 +626,9 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
               pk.x = pack_bf16(Os.x * inv, Os.y * inv);
               pk.y = pack_bf16(Os.z * inv, Os.w * inv);
               *reinterpret_cast<uint2 *>(a.out + (row0 + gh) * kD + lane * 4) = pk;
+              if (a.out_f32)
+                *reinterpret_cast<float4 *>(a.out_f32 + (row0 + gh) * kD + lane * 4) =
+                    make_float4(Os.x * inv, Os.y * inv, Os.z * inv, Os.w * inv);
               if (a.lse && lane == 0) a.lse[row0 + gh] = (Mx + log2f(Ls)) * kLn2;
             } else {
               *reinterpret_cast<float4 *>(a.part_acc + ((size_t)dst_slot * a.G + gh) * kD + lane * 4) = Os;
@@ -756,15 +764,14 @@ extern "C" size_t spkv_decode_workspace_bytes(const spkv_config_t *cfg, int32_t 
   return 2 * decode_ws_layout(B * cfg->n_kv_heads, cfg->n_q_heads / cfg->n_kv_heads).total;
 }
 
-extern "C" int spkv_decode_attention(spkv_cache_t *cache, int32_t layer, const int32_t *d_seq_ids,
-                                     int32_t B, const void *d_q, void *d_out, float *d_lse_opt,
-                                     float sm_scale, void *d_workspace, size_t workspace_bytes,
-                                     spkv_stream_t stream) {
+static int decode_attention_impl(spkv_cache_t *cache, int32_t layer, const int32_t *d_seq_ids, int32_t B,
+                                 const void *d_q, void *d_out, float *d_out_f32, float *d_lse_opt, float sm_scale,
+                                 void *d_workspace, size_t workspace_bytes, spkv_stream_t stream) {
   if (!cache || layer < 0 || layer >= cache->cfg.n_layers || B < 0 || B > cache->cfg.max_seqs)
     return SPKV_E_INVALID;
   if (B == 0) return SPKV_OK;
   if (!d_seq_ids || !d_q || !d_out) return SPKV_E_INVALID;
-  if (((uintptr_t)d_q | (uintptr_t)d_out) & 15) return SPKV_E_INVALID;
+  if (((uintptr_t)d_q | (uintptr_t)d_out | (uintptr_t)d_out_f32) & 15) return SPKV_E_INVALID;
   const CacheView &v = cache->view;
   const int n_items = B * v.Hkv;
   if (n_items > 1024) return SPKV_E_UNSUPPORTED;
@@ -776,6 +783,7 @@ extern "C" int spkv_decode_attention(spkv_cache_t *cache, int32_t layer, const i
   a.seq_ids = d_seq_ids;
   a.q = static_cast<const __nv_bfloat16 *>(d_q);
   a.out = static_cast<__nv_bfloat16 *>(d_out);
+  a.out_f32 = d_out_f32;
   a.lse = d_lse_opt;
   a.scale_log2 = sm_scale * kLog2e;
   static const int snap_env = [] {
@@ -845,6 +853,23 @@ extern "C" int spkv_decode_attention(spkv_cache_t *cache, int32_t layer, const i
   }
   return check_stream_error(
       launch_overlapped(kernel, dim3(grid), dim3(kTcThreads), (size_t)L.total, s, a, GP, n_stages, red_bufs));
+}
+
+extern "C" int spkv_decode_attention(spkv_cache_t *cache, int32_t layer, const int32_t *d_seq_ids,
+                                     int32_t B, const void *d_q, void *d_out, float *d_lse_opt,
+                                     float sm_scale, void *d_workspace, size_t workspace_bytes,
+                                     spkv_stream_t stream) {
+  return decode_attention_impl(cache, layer, d_seq_ids, B, d_q, d_out, nullptr, d_lse_opt, sm_scale, d_workspace,
+                               workspace_bytes, stream);
+}
+
+extern "C" int spkv_decode_attention_f32(spkv_cache_t *cache, int32_t layer, const int32_t *d_seq_ids,
+                                         int32_t B, const void *d_q, void *d_out, float *d_out_f32,
+                                         float *d_lse_opt, float sm_scale, void *d_workspace,
+                                         size_t workspace_bytes, spkv_stream_t stream) {
+  if (!d_out_f32) return SPKV_E_INVALID;
+  return decode_attention_impl(cache, layer, d_seq_ids, B, d_q, d_out, d_out_f32, d_lse_opt, sm_scale, d_workspace,
+                               workspace_bytes, stream);
 }
 
 // ---- decode attention for callers that cannot allocate device memory ---------------------

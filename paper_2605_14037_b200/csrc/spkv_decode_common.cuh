@@ -16,6 +16,7 @@ struct DecodeArgs {
   const int32_t *seq_ids;
   const __nv_bfloat16 *q;  // [B][Hq][128]
   __nv_bfloat16 *out;      // [B][Hq][128]
+  float *out_f32;          // [B][Hq][128] or null: the same rows before the rounding to bf16
   float *lse;              // [B][Hq] or null
   float scale_log2;        // sm_scale * log2(e)
   int snap;                // range cuts within this many positions of a unit boundary move onto it

@@ -58,6 +58,8 @@ __global__ void __launch_bounds__(128) decode_simt_kernel(DecodeArgs a) {
       for (int g = 0; g < a.G; ++g) {
         __nv_bfloat16 *o = a.out + ((size_t)b * c.Hq + kvh * a.G + g) * kD;
         for (int d = 0; d < kD; ++d) o[d] = __float2bfloat16(0.f);
+        if (a.out_f32)
+          for (int d = 0; d < kD; ++d) a.out_f32[((size_t)b * c.Hq + kvh * a.G + g) * kD + d] = 0.f;
         if (a.lse) a.lse[(size_t)b * c.Hq + kvh * a.G + g] = -INFINITY;
       }
     }
@@ -216,6 +218,7 @@ __global__ void __launch_bounds__(128) decode_simt_kernel(DecodeArgs a) {
         if (g < a.G) {
           const size_t row = (size_t)b * c.Hq + kvh * a.G + g;
           a.out[row * kD + tid] = __float2bfloat16(O[g] / Lsum[g]);
+          if (a.out_f32) a.out_f32[row * kD + tid] = O[g] / Lsum[g];
           if (a.lse && tid == 0) a.lse[row] = (M[g] + log2f(Lsum[g])) * kLn2;
         }
     }

@@ -83,6 +83,7 @@ def lib():
         "spkv_score_append_evict": (C.c_int, [vp, i32, pp, vp, i32, vp, vp, vp, vp, vp]),
         "spkv_decode_workspace_bytes": (sz, [cfgp, i32]),
         "spkv_decode_attention": (C.c_int, [vp, i32, vp, i32, vp, vp, vp, f32, vp, sz, vp]),
+        "spkv_decode_attention_f32": (C.c_int, [vp, i32, vp, i32, vp, vp, vp, vp, f32, vp, sz, vp]),
         "spkv_decode_attention_static": (C.c_int, [vp, i32, vp, i32, vp, vp, vp, f32, vp]),
         "spkv_prefill_workspace_bytes": (sz, [cfgp, i32]),
         "spkv_prefill": (C.c_int, [vp, i32, i32, i32, vp, vp, vp, vp, vp, f32, vp, sz, vp]),
@@ -219,6 +220,23 @@ class Cache:
             self.default_scale if sm_scale is None else sm_scale, _ptr(ws), ws.numel(),
             _stream(stream)), "spkv_decode_attention")
         return out
+
+    def spkv_decode_attention_f32(self, layer, seq_ids, q, out=None, out_f32=None, lse=None, sm_scale=None,
+                                  stream=None):
+        """spkv_decode_attention that also returns the rows before their rounding to bf16;
+        returns (out bf16, out float32)."""
+        B = seq_ids.numel()
+        if out is None:
+            out = torch.empty_like(q)
+        if out_f32 is None:
+            out_f32 = torch.empty(q.shape, dtype=torch.float32, device=q.device)
+        ws = self.decode_workspace(B)
+        _check(lib().spkv_decode_attention_f32(
+            self._h, layer, _ptr(seq_ids, torch.int32), B, _ptr(q, torch.bfloat16),
+            _ptr(out, torch.bfloat16), _ptr(out_f32, torch.float32), _ptr(lse, torch.float32),
+            self.default_scale if sm_scale is None else sm_scale, _ptr(ws), ws.numel(),
+            _stream(stream)), "spkv_decode_attention_f32")
+        return out, out_f32
 
     def spkv_decode_attention_static(self, layer, seq_ids, q, out=None, lse=None, sm_scale=None,
                                      stream=None):
