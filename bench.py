@@ -365,6 +365,10 @@ def run_ours(args):
                 "d2h_bytes_per_step": L * B * Hq * 128 * 2, "steps": e2e_steps,
                 "api": "spkv_decode_stack_host",
                 "per_layer_api": {"value": world * B * e2e_steps / dt_layer, "api": "spkv_decode_step_host"}}
+        if not dense and tau is None:
+            # the read-only ceiling of this GPU, measured by the library's own read stream over
+            # the cache arena (larger than L2 for every config but the tiny one)
+            res["read_ceiling_gbs"] = spkv.spkv_stream_read(cache.arena)
         cache.close()
         del cache
         torch.cuda.empty_cache()
@@ -412,6 +416,11 @@ def run_ours(args):
         "roofline": {"bound": "hbm", "kernel": "decode_tc_kernel", "achieved": in_step, "peak": hbm_peak,
                      "unit": "GB/s", "frac": in_step / hbm_peak, "peak_kind": f"of {peak_kind}",
                      "frac_of_nominal_8TBs": in_step / 8000.0,
+                     "read_ceiling": {"gbs": sp.get("read_ceiling_gbs"),
+                                      "frac": in_step / sp["read_ceiling_gbs"] if sp.get("read_ceiling_gbs") else None,
+                                      "how": "spkv_stream_read over the cache arena: 32 KB bulk copies into shared "
+                                             "memory, one block per SM, nothing else (the measured peak above is a "
+                                             "copy: half writes)"},
                      "bytes_per_launch": sp["launch_bytes"], "launch_period_us": sp["ms_per_step"] * 1e3 / L,
                      "how": "algorithmic K/V, Q, O bytes of a step over the step time measured with CUDA events "
                             "around the timed region (graph replay, launches overlapped, append included)",

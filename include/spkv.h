@@ -328,6 +328,16 @@ float spkv_tau_logit(const spkv_cache_t *cache);
 
 const char *spkv_error_string(int code);
 
+/* Measurement aid (no counterpart in the paper): streams `bytes` bytes (rounded down to whole
+ * 32 KB pages) from device memory through shared memory with the bulk copies the decode kernel
+ * uses, one block per SM, and does nothing else with them.  Timed by the caller with events it
+ * gives the read-only HBM rate of this GPU, the ceiling of a kernel that only reads (the usual
+ * copy figure is half writes).
+ *   d_buf: device, 16-byte aligned; d_sink: device, one 64-bit word (a checksum is added to it);
+ *   d_status: device, one int32, set to SPKV_E_TIMEOUT if a bounded wait ran out.  Asynchronous. */
+int spkv_stream_read(const void *d_buf, size_t bytes, unsigned long long *d_sink, int32_t *d_status,
+                     spkv_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

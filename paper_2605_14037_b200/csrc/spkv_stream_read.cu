@@ -1,0 +1,69 @@
+// Measurement aid (no counterpart in the paper): how fast can this GPU READ from HBM with the
+// copy mechanism the decode kernel uses?  The decode path only reads its K/V pages, while the
+// usual bandwidth figure is a copy (half reads, half writes); this kernel streams a buffer
+// through shared memory in 32 KB bulk copies, six in flight per block, one block per SM, and does
+// nothing else with it (one word per page goes into a checksum so that the copies are not dead).
+#include "spkv_internal.cuh"
+#include "spkv_mma.cuh"
+
+namespace spkv {
+
+namespace {
+constexpr int kReadStages = 6;
+constexpr int kReadSmem = kReadStages * kPageBytes + 64;
+}  // namespace
+
+// grid = SMs, 32 threads; block b takes pages b, b + grid, ...  status[0] != 0 on a timed-out wait.
+__global__ void __launch_bounds__(32) stream_read_kernel(const unsigned char *buf, long long n_pages,
+                                                         unsigned long long *sink, int *status) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  uint64_t *full = reinterpret_cast<uint64_t *>(smem + kReadStages * kPageBytes);
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kReadStages; ++i) mbar_init(&full[i], 1);
+    mbar_fence_init();
+  }
+  __syncwarp();
+  if (threadIdx.x != 0) return;
+  unsigned long long sum = 0;
+  long long k = 0;
+  bool failed = false;
+  for (long long p = blockIdx.x; p < n_pages && !failed; p += gridDim.x, ++k) {
+    const int s = (int)(k % kReadStages);
+    if (k >= kReadStages) {  // the copy that used this stage before has landed
+      if (!mbar_wait_bounded(&full[s], (uint32_t)((k / kReadStages) - 1) & 1)) { failed = true; break; }
+      sum += *reinterpret_cast<const unsigned int *>(smem + s * kPageBytes);
+      // the generic-proxy read above is ordered before the next bulk copy into the stage
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    mbar_arrive_expect_tx(&full[s], kPageBytes);
+    bulk_load(smem + s * kPageBytes, buf + p * (long long)kPageBytes, kPageBytes, &full[s]);
+  }
+  // do not leave while copies may still be landing
+  for (long long j = k > kReadStages ? k - kReadStages : 0; j < k; ++j) {
+    const int s = (int)(j % kReadStages);
+    if (!mbar_wait_bounded(&full[s], (uint32_t)(j / kReadStages) & 1)) failed = true;
+    else sum += *reinterpret_cast<const unsigned int *>(smem + s * kPageBytes);
+  }
+  if (failed) atomicExch(status, SPKV_E_TIMEOUT);
+  atomicAdd(sink, sum);
+}
+
+}  // namespace spkv
+
+using namespace spkv;
+
+extern "C" int spkv_stream_read(const void *d_buf, size_t bytes, unsigned long long *d_sink, int32_t *d_status,
+                                spkv_stream_t stream) {
+  if (!d_buf || !d_sink || !d_status || ((uintptr_t)d_buf & 15)) return SPKV_E_INVALID;
+  const long long n_pages = (long long)(bytes / kPageBytes);
+  if (n_pages == 0) return SPKV_OK;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return SPKV_E_CUDA;
+  if (cudaFuncSetAttribute(stream_read_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kReadSmem) != cudaSuccess)
+    return SPKV_E_CUDA;
+  stream_read_kernel<<<sms, 32, kReadSmem, as_stream(stream)>>>(static_cast<const unsigned char *>(d_buf), n_pages,
+                                                               d_sink, d_status);
+  return check_stream_error(cudaGetLastError());
+}

@@ -83,6 +83,7 @@ def lib():
         "spkv_score_append_evict": (C.c_int, [vp, i32, pp, vp, i32, vp, vp, vp, vp, vp]),
         "spkv_decode_workspace_bytes": (sz, [cfgp, i32]),
         "spkv_decode_attention": (C.c_int, [vp, i32, vp, i32, vp, vp, vp, f32, vp, sz, vp]),
+        "spkv_stream_read": (C.c_int, [vp, sz, vp, vp, vp]),
         "spkv_decode_attention_f32": (C.c_int, [vp, i32, vp, i32, vp, vp, vp, vp, f32, vp, sz, vp]),
         "spkv_decode_attention_static": (C.c_int, [vp, i32, vp, i32, vp, vp, vp, f32, vp]),
         "spkv_prefill_workspace_bytes": (sz, [cfgp, i32]),
@@ -371,6 +372,26 @@ class Cache:
                "spkv_read_window")
         n = n.value
         return pos[:n], k[:n], v[:n], lg[:n]
+
+
+def spkv_stream_read(buf, passes=5, stream=None):
+    """Read-only HBM rate in GB/s: streams the uint8 tensor `buf` through spkv_stream_read
+    `passes` times (after one warm-up pass), timed with CUDA events on the launching stream."""
+    sink = torch.zeros(1, dtype=torch.int64, device=buf.device)
+    status = torch.zeros(1, dtype=torch.int32, device=buf.device)
+    nbytes = buf.numel() // 32768 * 32768
+    call = lambda: _check(lib().spkv_stream_read(_ptr(buf), nbytes, _ptr(sink), _ptr(status), _stream(stream)),
+                          "spkv_stream_read")
+    call()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(passes):
+        call()
+    e1.record()
+    e1.synchronize()
+    if int(status.item()) != 0:
+        raise SpkvError(f"spkv_stream_read: {ERRORS.get(int(status.item()), status.item())}")
+    return nbytes * passes / (e0.elapsed_time(e1) * 1e-3) / 1e9
 
 
 def bf16_from_bits(bits, device):
