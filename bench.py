@@ -601,7 +601,7 @@ def cpu_baseline(cfg, budget_s=20.0, steps=None):
     n = len(units)
     scale = 1.0 / math.sqrt(128)
     t_used, done = 0.0, 0
-    while (steps is None and t_used < budget_s and done < 64) or (steps is not None and done < steps):
+    while (steps is None and t_used < budget_s and done < 512) or (steps is not None and done < steps):
         k, v = synth.normal_bf16(rng, (n, 128)), synth.normal_bf16(rng, (n, 128))
         q = synth.normal_bf16(rng, (n, G, 128))
         lg = rng.standard_normal(n).astype(np.float32)
