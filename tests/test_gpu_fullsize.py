@@ -59,8 +59,10 @@ def test_config2_one_layer_full_size():
     # sampled prefill queries against the mask form (Eq. 2-5 written out)
     scale = 1.0 / math.sqrt(D)
     for s in sampled:
-        for t in (T - C, T - C + 127, T - C + 128, T - 4097, T - 1):
-            for h in (0, 3, 5):
+        ts = sorted({T - C, T - C + 1, T - C + 63, T - C + 64, T - C + 127, T - C + 128, T - 4097, T - 129, T - 1}
+                    | {T - C + int(x) for x in np.linspace(200, C - 200, 24)})   # tile edges and a spread
+        for t in ts:
+            for h in (0, 3, 5, 7):
                 ref = oracle.mask_attend_row(
                     np.ascontiguousarray(Ks[s][:T, h]), np.ascontiguousarray(Vs[s][:T, h]),
                     np.ascontiguousarray(logit[:T, s, h]), t, w, tl,
