@@ -283,9 +283,13 @@ int spkv_decode_step_host(spkv_cache_t *cache, int32_t layer, const spkv_predict
 int spkv_decode_step_host_flush(spkv_cache_t *cache, spkv_stream_t stream);
 
 /* One decode step of the WHOLE layer stack from host buffers, for an attention-only stack whose
- * inputs all exist before the step: four copies in, per layer score -> append/evict -> decode
- * attention back to back on `stream` (in overlap mode nothing separates the launches), one copy
- * out.  Everything is enqueued on `stream`; no synchronisation.
+ * inputs all exist before the step.  The layers go in four chunks: a chunk's inputs are copied
+ * on a stream of the cache's own, its kernels (per layer score -> append/evict -> decode
+ * attention, back to back) run on `stream` once they have landed, and its outputs are copied
+ * back on another stream of the cache's own while the next chunk computes.  `stream` ends up
+ * waiting for the last output copy, so synchronising `stream` means h_out is complete; the host
+ * buffers must stay untouched until then (pinned memory, or the copies serialise).  No
+ * synchronisation inside the call.
  *   preds [n_layers] (host array, same d_in); h_x [L, B, d_in], h_q [L, B, n_q_heads, 128],
  *   h_k/h_v [L, B, n_kv_heads, 128] bf16 -> h_out [L, B, n_q_heads, 128] bf16;
  *   d_staging: >= spkv_decode_stack_staging_bytes(cfg, B, d_in) bytes, 256-byte aligned,

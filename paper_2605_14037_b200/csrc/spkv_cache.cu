@@ -126,6 +126,7 @@ extern "C" int spkv_cache_create(const spkv_config_t *cfg, void *d_arena, size_t
   c->appends_pending = new (std::nothrow) int[cfg->n_layers]();
   if (!c->appends_pending) { delete c; return SPKV_E_INVALID; }
   c->host_ready = false;
+  c->stack_ready = false;
   c->host_calls = 0;
   char *base = static_cast<char *>(d_arena);
   CacheView &v = c->view;
@@ -183,6 +184,14 @@ extern "C" int spkv_cache_create(const spkv_config_t *cfg, void *d_arena, size_t
 
 extern "C" int spkv_cache_destroy(spkv_cache_t *cache) {
   if (!cache) return SPKV_E_INVALID;
+  if (cache->stack_ready) {
+    for (int i = 0; i < 4; ++i) {
+      cudaEventDestroy(cache->ev_st_in[i]);
+      cudaEventDestroy(cache->ev_st_k[i]);
+    }
+    cudaEventDestroy(cache->ev_st_start);
+    cudaEventDestroy(cache->ev_st_done);
+  }
   if (cache->host_ready) {  // host-side objects of the host-buffer pipeline
     for (int i = 0; i < 2; ++i) {
       cudaEventDestroy(cache->ev_in[i]);

@@ -1009,10 +1009,31 @@ extern "C" int spkv_decode_step_host_flush(spkv_cache_t *cache, spkv_stream_t st
 }
 
 // ---- one decode step of the WHOLE layer stack from host buffers ------------------------------
-// For an attention-only stack every layer's inputs exist before the step starts, so they go to
-// the device in four copies, the 2 L kernels follow back to back on the same stream (nothing
-// between them: in overlap mode each decode launch starts under the tail of the previous one,
-// which the per-layer entry point's event waits prevent), and one copy brings all outputs back.
+// For an attention-only stack every layer's inputs exist before the step starts.  The layers go
+// in four chunks: each chunk's inputs travel in four copies on the cache's input stream, its
+// 2 x layers kernels follow back to back on the caller's stream once they have landed (nothing
+// between the kernels of a chunk: in overlap mode each decode launch starts under the tail of the
+// previous one, which the per-layer entry point's event waits prevent), and its outputs leave on
+// the output stream while the next chunk computes.  So the copies of all chunks but the first
+// (in) and the last (out) run under kernels.  The caller's stream ends up waiting for the last
+// output copy: synchronising it means the outputs are on the host.
+constexpr int kStackChunks = 4;
+
+static int stack_pipeline_init(spkv_cache *c) {
+  int rc = host_pipeline_init(c);
+  if (rc) return rc;
+  if (c->stack_ready) return SPKV_OK;
+  for (int i = 0; i < kStackChunks; ++i)
+    if (cudaEventCreateWithFlags(&c->ev_st_in[i], cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&c->ev_st_k[i], cudaEventDisableTiming) != cudaSuccess)
+      return SPKV_E_CUDA;
+  if (cudaEventCreateWithFlags(&c->ev_st_start, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&c->ev_st_done, cudaEventDisableTiming) != cudaSuccess)
+    return SPKV_E_CUDA;
+  c->stack_ready = true;
+  return SPKV_OK;
+}
+
 static size_t stack_inputs_bytes(const spkv_config_t *cfg, int32_t B, int32_t d_in, size_t *x, size_t *q, size_t *kv,
                                  size_t *lg) {
   *x = a256((size_t)cfg->n_layers * B * d_in * 2);
@@ -1051,20 +1072,45 @@ extern "C" int spkv_decode_stack_host(spkv_cache_t *cache, const spkv_predictor_
   const size_t x_l = (size_t)B * d_in * 2, q_l = (size_t)B * cfg.n_q_heads * kD * 2,
                kv_l = (size_t)B * cfg.n_kv_heads * kD * 2;
   cudaStream_t s = as_stream(stream);
-  if (cudaMemcpyAsync(d_x, h_x, x_l * L, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-      cudaMemcpyAsync(d_q, h_q, q_l * L, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-      cudaMemcpyAsync(d_k, h_k, kv_l * L, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-      cudaMemcpyAsync(d_v, h_v, kv_l * L, cudaMemcpyHostToDevice, s) != cudaSuccess)
+  int rc = stack_pipeline_init(cache);
+  if (rc) return rc;
+  const int nc = L < kStackChunks ? L : kStackChunks;
+  const char *hx = static_cast<const char *>(h_x), *hq = static_cast<const char *>(h_q),
+             *hk = static_cast<const char *>(h_k), *hv = static_cast<const char *>(h_v);
+  // the staging buffers are free once everything enqueued on the caller's stream so far has run
+  if (cudaEventRecord(cache->ev_st_start, s) != cudaSuccess ||
+      cudaStreamWaitEvent(cache->copy_in, cache->ev_st_start, 0) != cudaSuccess)
     return SPKV_E_CUDA;
-  cache->last_kind = kLastOther;  // the first append waits for the copies
-  for (int l = 0; l < L; ++l) {
-    int rc = spkv_score_append_evict(cache, l, &preds[l], d_seq_ids, B, d_x + l * x_l, d_k + l * kv_l, d_v + l * kv_l,
-                                     d_lg + (size_t)l * B * cfg.n_kv_heads, stream);
-    if (rc) return rc;
-    rc = spkv_decode_attention(cache, l, d_seq_ids, B, d_q + l * q_l, d_o + l * q_l, nullptr, sm_scale, p,
-                               spkv_decode_workspace_bytes(&cfg, B), stream);
-    if (rc) return rc;
+  for (int ci = 0; ci < nc; ++ci) {
+    const size_t l0 = (size_t)ci * L / nc, n = (size_t)(ci + 1) * L / nc - l0;
+    if (cudaMemcpyAsync(d_x + l0 * x_l, hx + l0 * x_l, n * x_l, cudaMemcpyHostToDevice, cache->copy_in) != cudaSuccess ||
+        cudaMemcpyAsync(d_q + l0 * q_l, hq + l0 * q_l, n * q_l, cudaMemcpyHostToDevice, cache->copy_in) != cudaSuccess ||
+        cudaMemcpyAsync(d_k + l0 * kv_l, hk + l0 * kv_l, n * kv_l, cudaMemcpyHostToDevice, cache->copy_in) != cudaSuccess ||
+        cudaMemcpyAsync(d_v + l0 * kv_l, hv + l0 * kv_l, n * kv_l, cudaMemcpyHostToDevice, cache->copy_in) != cudaSuccess ||
+        cudaEventRecord(cache->ev_st_in[ci], cache->copy_in) != cudaSuccess)
+      return SPKV_E_CUDA;
+  }
+  for (int ci = 0; ci < nc; ++ci) {
+    const int l0 = (int)((size_t)ci * L / nc), l1 = (int)((size_t)(ci + 1) * L / nc);
+    if (cudaStreamWaitEvent(s, cache->ev_st_in[ci], 0) != cudaSuccess) return SPKV_E_CUDA;
+    cache->last_kind = kLastOther;  // the chunk's first append waits for everything before it on the stream
+    for (int l = l0; l < l1; ++l) {
+      rc = spkv_score_append_evict(cache, l, &preds[l], d_seq_ids, B, d_x + l * x_l, d_k + l * kv_l, d_v + l * kv_l,
+                                   d_lg + (size_t)l * B * cfg.n_kv_heads, stream);
+      if (rc) return rc;
+      rc = spkv_decode_attention(cache, l, d_seq_ids, B, d_q + l * q_l, d_o + l * q_l, nullptr, sm_scale, p,
+                                 spkv_decode_workspace_bytes(&cfg, B), stream);
+      if (rc) return rc;
+    }
+    if (cudaEventRecord(cache->ev_st_k[ci], s) != cudaSuccess ||
+        cudaStreamWaitEvent(cache->copy_out, cache->ev_st_k[ci], 0) != cudaSuccess ||
+        cudaMemcpyAsync(static_cast<char *>(h_out) + l0 * q_l, d_o + l0 * q_l, (size_t)(l1 - l0) * q_l,
+                        cudaMemcpyDeviceToHost, cache->copy_out) != cudaSuccess)
+      return SPKV_E_CUDA;
   }
   cache->last_kind = kLastOther;
-  return check_stream_error(cudaMemcpyAsync(h_out, d_o, q_l * L, cudaMemcpyDeviceToHost, s));
+  if (cudaEventRecord(cache->ev_st_done, cache->copy_out) != cudaSuccess ||
+      cudaStreamWaitEvent(s, cache->ev_st_done, 0) != cudaSuccess)
+    return SPKV_E_CUDA;
+  return check_stream_error(cudaGetLastError());
 }

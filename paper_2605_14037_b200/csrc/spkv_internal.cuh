@@ -225,6 +225,9 @@ struct spkv_cache {
   cudaEvent_t ev_in[2], ev_k[2], ev_out[2];   // per slot: inputs landed, kernels done, output landed
   long long host_calls;                        // calls so far; slot = call & 1
   bool host_ready;
+  // spkv_decode_stack_host: per chunk of layers, inputs landed / kernels done; start and end of a call
+  cudaEvent_t ev_st_in[4], ev_st_k[4], ev_st_start, ev_st_done;
+  bool stack_ready;
 };
 
 namespace spkv {
