@@ -31,9 +31,6 @@
 // Shared memory: Q of both heads (64 KB) + 5 page stages.
 // Warps: 0 MMA issue, 1 page loader + TMEM allocation, 2-3 value conversion, 4-7 group 0,
 // 8-11 group 1.  All waits are bounded.
-#include <cstdlib>
-#include <cstring>
-
 #include "spkv_prefill_common.cuh"
 #include "spkv_tc5.cuh"
 
