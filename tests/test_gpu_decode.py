@@ -270,12 +270,14 @@ def test_overlap_mode_is_bit_identical_to_stream_ordered_launches(L, B, steps):
 
 
 @pytest.mark.parametrize("flags", [0, 1])
-def test_decode_stack_host_matches_device_calls(flags):
-    """spkv_decode_stack_host (all layers' inputs copied in at once, kernels back to back, one
-    copy out) against the device-pointer calls, bit for bit, with and without overlap mode."""
+@pytest.mark.parametrize("L", [1, 3, 5, 9])
+def test_decode_stack_host_matches_device_calls(flags, L):
+    """spkv_decode_stack_host (the layers in up to four chunks, each with its copies in, its
+    kernels back to back and its copy out) against the device-pointer calls, bit for bit, with
+    and without overlap mode, for layer counts below, at and above the number of chunks."""
     spkv = load()
     rng = np.random.default_rng(123 + flags)
-    L, B, Hq, Hkv, d_in, w, steps = 5, 3, 8, 2, 64, 16, 30
+    B, Hq, Hkv, d_in, w, steps = 3, 8, 2, 64, 16, 30
     mk = lambda f: spkv.Cache(n_layers=L, max_seqs=B, n_q_heads=Hq, n_kv_heads=Hkv, max_context=512,
                               pool_pages=L * B * Hkv * 2, window=w, tau=0.5, flags=f)
     ca, cb = mk(flags), mk(0)
