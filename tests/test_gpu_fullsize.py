@@ -1,10 +1,12 @@
-"""Parity at the benchmark's full size and launch configuration: one layer of the
-Llama-3-8B-shaped decode workload (batch 16, 32 query / 8 KV heads, context 32768, window 128,
-per-head keep rates ~ Beta(0.5, 2)).  The cache is built with 8192-pair prefill chunks and
-then stepped with batch-16 calls exactly as bench.py does.  Checked:
-  * compact-cache length of all 128 units == count of logits >= tau_logit among the pairs that
+"""Parity at the benchmark's full sizes and launch configuration: one layer of the
+Llama-3-8B-shaped decode workload (config 2: batch 16, 32 query / 8 KV heads, context 32768,
+window 128, per-head keep rates ~ Beta(0.5, 2)), of the long-context one (config 3: batch 4,
+context 131072, Beta(0.3, 3)) and of the 70B-shaped one (config 5: batch 8, 64 query / 8 KV
+heads, context 65536, Beta(0.5, 2.5)).  The cache is built with 8192-pair prefill chunks and
+then stepped with whole-batch calls exactly as bench.py does.  Checked:
+  * compact-cache length of all units == count of logits >= tau_logit among the pairs that
     left the window (kept-set identity), bit-exact;
-  * for two sampled sequences (16 units, CPU-generated K/V): kept positions and bytes bit-exact
+  * for the sampled sequences (8 units each, CPU-generated K/V): kept positions and bytes bit-exact
     against the oracle, sampled prefill outputs against the oracle's mask form, and the decode
     outputs of three steps against the oracle's streaming form, within the attention tolerance.
 """
@@ -21,13 +23,17 @@ from paper_2605_14037_b200 import synth
 pytestmark = pytest.mark.gpu
 
 
-def test_config2_one_layer_full_size():
+@pytest.mark.parametrize("B,Hq,Hkv,T,beta,sampled", [
+    (16, 32, 8, 32768, (0.5, 2.0), [3, 11]),
+    (4, 32, 8, 131072, (0.3, 3.0), [2]),
+    (8, 64, 8, 65536, (0.5, 2.5), [5]),
+], ids=["config2", "config3", "config5"])
+def test_one_layer_full_size(B, Hq, Hkv, T, beta, sampled):
     spkv = load()
-    B, Hq, Hkv, T, w, C, steps = 16, 32, 8, 32768, 128, 8192, 3
+    w, C, steps = 128, 8192, 3
     G = Hq // Hkv
-    sampled = [3, 11]
     rng = np.random.default_rng(1234)
-    rates = synth.keep_rates(rng, 1, Hkv, 0.5, 2.0)[0]
+    rates = synth.keep_rates(rng, 1, Hkv, *beta)[0]
     rates[0], rates[5] = 0.0, 0.97                       # a local-only head and a near-full head
     pages = int(np.ceil(rates * (T + steps) * 1.05 / 64 + 2).sum()) * B
     cache = spkv.Cache(n_layers=1, max_seqs=B, n_q_heads=Hq, n_kv_heads=Hkv, max_context=T + 128,
