@@ -109,3 +109,91 @@ def test_one_layer_full_size(B, Hq, Hkv, T, beta, sampled):
             compare_state(cache, 0, s, h, units[s][h])
     st = cache.spkv_cache_stats()
     assert abs(st.density_cache - want.sum() / (B * Hkv * (Tt - w))) < 1e-12
+
+
+def test_config4_one_layer_ragged_mixed_step():
+    """One layer of the mixed serving batch (config 4): 64 sequences with contexts drawn from
+    uniform[4096, 65536] as bench.py draws them; in a step sequences 0-7 take an 8192-pair prefill
+    chunk with queries and sequences 8-63 decode one token in one batched call.  One prefilling
+    and one decoding sequence have CPU-generated inputs and are checked against the oracle;
+    every unit's length against the count of open gates."""
+    spkv = load()
+    B, NP, Hq, Hkv, w, C = 64, 8, 32, 8, 128, 8192
+    G = Hq // Hkv
+    s_pre, s_dec = 5, 41
+    t_list = np.random.default_rng(4).integers(4096, 65536 + 1, size=B)       # bench.py's contexts
+    rng = np.random.default_rng(77)
+    rates = synth.keep_rates(rng, 1, Hkv, 0.5, 2.0)[0]
+    t_end = t_list + np.where(np.arange(B) < NP, C, 1)
+    pages = int(sum(np.ceil(rates * (t + 2) * 1.05 / 64 + 2).sum() for t in t_end))
+    cache = spkv.Cache(n_layers=1, max_seqs=B, n_q_heads=Hq, n_kv_heads=Hkv, max_context=65536 + C + 128,
+                       pool_pages=pages, window=w, tau=0.5)
+    tl = cache.spkv_tau_logit()
+    Tmax = int(t_end.max())
+    logit = np.stack([synth.logits_with_keep_rate(rng, (Tmax, B), float(r), tl) for r in rates], axis=-1)
+    Ks = {s: synth.normal_bf16(rng, (int(t_end[s]), Hkv, D)) for s in (s_pre, s_dec)}
+    Vs = {s: synth.normal_bf16(rng, (int(t_end[s]), Hkv, D)) for s in (s_pre, s_dec)}
+    q_pre = synth.normal_bf16(rng, (C, Hq, D))
+    gen = torch.Generator(device=dev())
+    gen.manual_seed(9)
+    lg_dev = torch.from_numpy(logit).to(dev())
+    rnd = lambda *shape: torch.randn(shape, generator=gen, device=dev()).to(torch.bfloat16)
+
+    def kv_of(s, a, b):
+        if s in Ks:
+            return to_dev_bf16(Ks[s][a:b]), to_dev_bf16(Vs[s][a:b])
+        return rnd(b - a, Hkv, D), rnd(b - a, Hkv, D)
+
+    for s in range(B):                                   # bring every sequence to its context
+        T0 = int(t_list[s])
+        for a in range(0, T0, C):
+            b = min(a + C, T0)
+            k, v = kv_of(s, a, b)
+            cache.spkv_prefill(0, s, k, v, lg_dev[a:b, s].contiguous())
+    assert cache.spkv_status() == 0
+
+    # the mixed step
+    out_pre = None
+    for s in range(NP):
+        T0 = int(t_list[s])
+        k, v = kv_of(s, T0, T0 + C)
+        o = cache.spkv_prefill(0, s, k, v, lg_dev[T0:T0 + C, s].contiguous(),
+                               q=to_dev_bf16(q_pre) if s == s_pre else rnd(C, Hq, D))
+        if s == s_pre:
+            out_pre = spkv.bits_from_bf16(o)
+    ids = torch.arange(NP, B, dtype=torch.int32, device=dev())
+    nd = B - NP
+    k_new, v_new, q_new = rnd(nd, Hkv, D), rnd(nd, Hkv, D), rnd(nd, Hq, D)
+    Td = int(t_list[s_dec])
+    k_new[s_dec - NP], v_new[s_dec - NP] = to_dev_bf16(Ks[s_dec][Td]), to_dev_bf16(Vs[s_dec][Td])
+    lg_step = torch.stack([lg_dev[int(t_list[s]), s] for s in range(NP, B)]).contiguous()
+    cache.spkv_append_evict(0, ids, k_new, v_new, lg_step)
+    out_dec = spkv.bits_from_bf16(cache.spkv_decode_attention(0, ids, q_new))
+    assert cache.spkv_status() == 0
+
+    scale = 1.0 / math.sqrt(D)
+    # prefilling sequence: sampled chunk queries against the mask form, state against the streaming form
+    Tp = int(t_list[s_pre])
+    for i in sorted({0, 1, 127, 128, C - 129, C - 1} | {int(x) for x in np.linspace(300, C - 300, 10)}):
+        for h in (1, 4, 6):
+            ref = oracle.mask_attend_row(np.ascontiguousarray(Ks[s_pre][:Tp + C, h]), np.ascontiguousarray(Vs[s_pre][:Tp + C, h]),
+                                         np.ascontiguousarray(logit[:Tp + C, s_pre, h]), Tp + i, w, tl,
+                                         np.ascontiguousarray(q_pre[i, h * G:(h + 1) * G]), scale)
+            assert_attn_close(out_pre[i, h * G:(h + 1) * G], ref, f"prefill i={i} h={h}")
+    q_bits = spkv.bits_from_bf16(q_new)
+    for s, T1 in ((s_pre, Tp + C), (s_dec, Td + 1)):
+        for h in range(Hkv):
+            u = oracle.Unit(w, D)
+            u.prefill(np.ascontiguousarray(Ks[s][:T1, h]), np.ascontiguousarray(Vs[s][:T1, h]),
+                      np.ascontiguousarray(logit[:T1, s, h]), tl)
+            if h in (0, 3, 7):
+                compare_state(cache, 0, s, h, u)
+            if s == s_dec:
+                ref = u.attend(np.ascontiguousarray(q_bits[s - NP, h * G:(h + 1) * G]), scale)
+                assert_attn_close(out_dec[s - NP, h * G:(h + 1) * G], ref, f"decode h={h}")
+    ln, tt = cache.spkv_read_lengths(0)
+    for s in range(B):
+        T1 = int(t_end[s])
+        assert tt[s].tolist() == [T1] * Hkv
+        want = (logit[:T1 - w, s] >= np.float32(tl)).sum(axis=0)
+        assert np.array_equal(ln[s], want.astype(np.int32)), s
