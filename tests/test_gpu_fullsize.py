@@ -197,3 +197,65 @@ def test_config4_one_layer_ragged_mixed_step():
         assert tt[s].tolist() == [T1] * Hkv
         want = (logit[:T1 - w, s] >= np.float32(tl)).sum(axis=0)
         assert np.array_equal(ln[s], want.astype(np.int32)), s
+
+
+def test_config1_every_step_of_the_chain():
+    """Config 1 (1 layer, batch 1, 8 query / 2 KV heads, context 4096, linear predictor on a
+    512-wide input, ~20 % kept): the whole chain score -> append/evict -> decode attention at
+    EVERY step against the oracle, with the keep decisions taken on the GPU's own logits
+    (inputs whose oracle logit lies in the rounding band of the threshold are resampled, so
+    both sides decide alike); then the same tokens through one prefill call must leave the
+    same state, bit for bit, and the same outputs within the tolerance."""
+    spkv = load()
+    Hq, Hkv, T, w, d_in = 8, 2, 4096, 128, 512
+    G = Hq // Hkv
+    rng = np.random.default_rng(101)
+    mk = lambda: spkv.Cache(n_layers=1, max_seqs=1, n_q_heads=Hq, n_kv_heads=Hkv, max_context=T + 128,
+                            pool_pages=2 * (T // 64 + 2), window=w, tau=0.5)
+    cache = mk()
+    tl = cache.spkv_tau_logit()
+    W = synth.linear_predictor(rng, Hkv, d_in)
+    b = synth.bias_for_keep_rate(W, [0.2, 0.2], tl)
+    x = synth.normal_bf16(rng, (T, d_in))
+    for _ in range(10):
+        ref_lg = oracle.score_linear(x, W, b)
+        near = (np.abs(ref_lg - float(tl)) < 1e-3).any(axis=1)
+        if not near.any():
+            break
+        x[near] = synth.normal_bf16(rng, (int(near.sum()), d_in))
+    assert not near.any()
+    K, V = synth.normal_bf16(rng, (T, Hkv, D)), synth.normal_bf16(rng, (T, Hkv, D))
+    q = synth.normal_bf16(rng, (T, Hq, D))
+    pred = spkv.make_predictor(to_dev_bf16(W), torch.from_numpy(b).to(dev()))
+    xd, Kd, Vd, qd = to_dev_bf16(x), to_dev_bf16(K), to_dev_bf16(V), to_dev_bf16(q)
+    ids = torch.zeros(1, dtype=torch.int32, device=dev())
+    outs = torch.empty((T, Hq, D), dtype=torch.bfloat16, device=dev())
+    lgs = torch.empty((T, Hkv), dtype=torch.float32, device=dev())
+    for t in range(T):
+        cache.spkv_score_append_evict(0, pred, ids, xd[t:t + 1], Kd[t:t + 1], Vd[t:t + 1], logits_out=lgs[t:t + 1])
+        cache.spkv_decode_attention(0, ids, qd[t:t + 1], out=outs[t:t + 1])
+    assert cache.spkv_status() == 0
+    got = spkv.bits_from_bf16(outs)
+    gpu_lg = lgs.cpu().numpy()
+    assert np.abs(gpu_lg - ref_lg).max() < 1e-3
+    assert np.array_equal(gpu_lg >= np.float32(tl), ref_lg >= float(tl))       # same decisions
+    scale = 1.0 / math.sqrt(D)
+    units = []
+    for h in range(Hkv):
+        u = oracle.Unit(w, D)
+        ref = u.prefill(np.ascontiguousarray(K[:, h]), np.ascontiguousarray(V[:, h]),
+                        np.ascontiguousarray(gpu_lg[:, h]), tl, np.ascontiguousarray(q[:, h * G:(h + 1) * G]), scale)
+        assert_attn_close(got[:, h * G:(h + 1) * G], ref, f"every step, kv head {h}")
+        compare_state(cache, 0, 0, h, u)
+        units.append((u, ref))
+    kept = [len(u) for u, _ in units]
+    assert all(0.15 * (T - w) < n < 0.25 * (T - w) for n in kept), kept
+    # the same tokens through one prefill call
+    cache2 = mk()
+    lg2 = cache2.spkv_score(pred, xd)
+    assert torch.equal(lg2, lgs)
+    out2 = spkv.bits_from_bf16(cache2.spkv_prefill(0, 0, Kd, Vd, lg2, q=qd))
+    assert cache2.spkv_status() == 0
+    for h in range(Hkv):
+        compare_state(cache2, 0, 0, h, units[h][0])
+        assert_attn_close(out2[:, h * G:(h + 1) * G], units[h][1], f"prefill form, kv head {h}")
