@@ -340,3 +340,78 @@ def test_decode_float32_output_at_2e_5(kernel_rows):
                     worst = max(worst, float(err.max()))
     assert cache.spkv_status() == 0
     print("worst abs error of the float32 rows:", worst)
+
+
+@pytest.mark.parametrize("L,B", [(4, 16), (2, 3), (3, 5), (1, 2)])
+def test_graph_replay_in_overlap_mode_matches_eager_launches(L, B):
+    """The benchmark's launch configuration: one step of the layer stack (fused score + append,
+    decode, per layer) captured once into a CUDA graph on an overlap-mode cache and replayed
+    step after step, the step's inputs copied into fixed staging tensors before each replay.
+    Outputs and final cache state must equal, bit for bit, those of a plain cache that launches
+    every kernel eagerly and stream-ordered."""
+    spkv = load()
+    rng = np.random.default_rng(900 + L + B)
+    Hq, Hkv, d_in, w, T0, steps = 8, 2, 64, 128, 500, 40
+    mk = lambda flags: spkv.Cache(n_layers=L, max_seqs=B, n_q_heads=Hq, n_kv_heads=Hkv, max_context=2048,
+                                  pool_pages=L * B * Hkv * 12, window=w, tau=0.5, flags=flags)
+    ca, cb = mk(spkv.FLAG_OVERLAP), mk(0)
+    tl = ca.spkv_tau_logit()
+    preds = []
+    for l in range(L):
+        W = synth.linear_predictor(rng, Hkv, d_in)
+        b = synth.bias_for_keep_rate(W, [0.3, 0.8], tl)
+        preds.append(spkv.make_predictor(to_dev_bf16(W), torch.from_numpy(b).to(dev())))
+    bf = lambda shape: to_dev_bf16(synth.normal_bf16(rng, shape))
+    for l in range(L):
+        for s in range(B):
+            k, v = bf((T0, Hkv, D)), bf((T0, Hkv, D))
+            lg = torch.from_numpy(synth.logits_with_keep_rate(rng, (T0, Hkv), 0.5, tl)).to(dev())
+            for c in (ca, cb):
+                c.spkv_prefill(l, s, k, v, lg)
+    ids = torch.arange(B, dtype=torch.int32, device=dev())
+    xs, qs = torch.empty((L, B, d_in), dtype=torch.bfloat16, device=dev()), torch.empty((L, B, Hq, D), dtype=torch.bfloat16, device=dev())
+    ks, vs = torch.empty((L, B, Hkv, D), dtype=torch.bfloat16, device=dev()), torch.empty((L, B, Hkv, D), dtype=torch.bfloat16, device=dev())
+    out_a = torch.empty((L, B, Hq, D), dtype=torch.bfloat16, device=dev())
+    ca.decode_workspace(B)                  # allocate before the capture
+
+    def layer_calls(c, x, q, k, v, o):
+        for l in range(L):
+            c.spkv_score_append_evict(l, preds[l], ids, x[l], k[l], v[l])
+            c.spkv_decode_attention(l, ids, q[l], out=o[l])
+
+    inputs = [(bf((L, B, d_in)), bf((L, B, Hq, D)), bf((L, B, Hkv, D)), bf((L, B, Hkv, D))) for _ in range(steps + 1)]
+
+    def stage(i):
+        x, q, k, v = inputs[i]
+        xs.copy_(x); qs.copy_(q); ks.copy_(k); vs.copy_(v)
+
+    # warm-up step outside the capture (both caches take it), then capture one step
+    stage(0)
+    side = torch.cuda.Stream(device=dev())
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        layer_calls(ca, xs, qs, ks, vs, out_a)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    out_b = torch.empty_like(out_a)
+    layer_calls(cb, *inputs[0], out_b)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        layer_calls(ca, xs, qs, ks, vs, out_a)
+    # the capture itself launched nothing: replay it for steps 1..n
+    for i in range(1, steps + 1):
+        stage(i)
+        graph.replay()
+        layer_calls(cb, *inputs[i], out_b)
+        torch.cuda.synchronize()
+        assert torch.equal(out_a.view(torch.int16), out_b.view(torch.int16)), i
+    assert ca.spkv_status() == 0 and cb.spkv_status() == 0
+    for l in range(L):
+        la, ta = ca.spkv_read_lengths(l)
+        lb, tb = cb.spkv_read_lengths(l)
+        assert np.array_equal(la, lb) and np.array_equal(ta, tb)
+        for s in range(B):
+            for h in range(Hkv):
+                pa, ka, va = ca.spkv_read_kept(l, s, h)
+                pb, kb, vb = cb.spkv_read_kept(l, s, h)
+                assert np.array_equal(pa, pb) and np.array_equal(ka, kb) and np.array_equal(va, vb)
