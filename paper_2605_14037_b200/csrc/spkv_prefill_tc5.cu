@@ -1,4 +1,7 @@
-// Chunk attention of spkv_prefill on the 5th-generation tensor cores (tcgen05.mma, TMEM).
+// Chunk attention of spkv_prefill on the 5th-generation tensor cores (tcgen05.mma, TMEM): the
+// one-head kernel, the first tcgen05 version, kept for comparison (SPKV_PREFILL_KERNEL=tc5x1; the
+// default is the two-head fp16 kernel in spkv_prefill_tc5x2h.cu), and the staging kernel that
+// every tcgen05 attention kernel runs behind.
 //
 // One block = 128 consecutive queries of one query head.  Keys/values arrive as 64-pair pages
 // -- first the compact-cache pages that hold the kept pairs visible to the tile (a prefix of the
@@ -323,7 +326,8 @@ int launch_prefill_attn_tc5(const PrefillArgs &a, cudaStream_t s) {
     return e && e[0] == 'b';
   }();
   prefill_stage_kernel<<<dim3(a.n_stage_pages, a.c.Hkv), 256, 0, s>>>(a);
-  if (a.c.G % 2 == 0 && !one_head) return bf16_pv ? launch_prefill_attn_tc5x2(a, s) : launch_prefill_attn_tc5x2h(a, s);
+  if (!one_head && !bf16_pv) return launch_prefill_attn_tc5x2h(a, s);   // any G: an odd group's last block has one head
+  if (!one_head && a.c.G % 2 == 0) return launch_prefill_attn_tc5x2(a, s);
   prefill_attn_tc5_kernel<<<dim3(((a.C + 127) / 128) * a.c.Hq), tc5::kThreads, tc5::kSmemBytes, s>>>(a);
   return check_stream_error(cudaGetLastError());
 }

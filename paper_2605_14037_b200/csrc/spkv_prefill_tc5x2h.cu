@@ -1,8 +1,9 @@
 // Chunk attention of spkv_prefill on tcgen05, two query heads per block, P.V in fp16.
 //
 // Same tiling as the two-term bf16 kernel next door (one block = 128 consecutive queries of two
-// query heads that share a KV head, Eq. 5; every 32 KB page is fetched once and feeds both; one
-// softmax group of 128 threads per head, thread = query row = TMEM lane).  Two things differ:
+// query heads that share a KV head -- of one, for the last head of an odd group --, Eq. 5;
+// every 32 KB page is fetched once and feeds both; one softmax group of 128 threads per head,
+// thread = query row = TMEM lane).  Two things differ:
 //
 // * P is ONE fp16 term (11 significant bits; the two-term bf16 split carries 16 but costs a second
 //   P.V pass).  The tensor cores want both operands in the same type, so warps 2-3 rewrite the
@@ -66,8 +67,11 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + kSBar + B_COUNT * 8);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   int kvh, pair, xtile;
-  prefill_work_item(a, blockIdx.x, (a.C + 127) / 128, c.G >> 1, kvh, pair, xtile);
+  prefill_work_item(a, blockIdx.x, (a.C + 127) / 128, (c.G + 1) >> 1, kvh, pair, xtile);
   const int hq0 = kvh * c.G + pair * 2, i0 = xtile * 128;
+  // an odd number of query heads per KV head leaves the last block of a KV head with one head:
+  // its second group and the MMAs of head 1 stay idle
+  const bool two = pair * 2 + 1 < c.G;
   const int32_t *hdr = unit_ws(a, kvh);
   const int32_t *E = hdr + kHdrInts;
   const int len0 = hdr[H_LEN0], n_old = hdr[H_NOLD], N = hdr[H_N];
@@ -118,7 +122,8 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
   for (int x = tid; x < 2 * 128 * 16; x += kThreads) {
     const int h = x >> 11, r = (x >> 4) & 127, ch = x & 15;
     uint4 val = make_uint4(0, 0, 0, 0);
-    if (i0 + r < a.C) val = *reinterpret_cast<const uint4 *>(a.q + ((size_t)(i0 + r) * c.Hq + hq0 + h) * kD + ch * 8);
+    if (i0 + r < a.C && (h == 0 || two))
+      val = *reinterpret_cast<const uint4 *>(a.q + ((size_t)(i0 + r) * c.Hq + hq0 + h) * kD + ch * 8);
     *reinterpret_cast<uint4 *>(smem + kSQ + h * 32768 + (ch >> 3) * 16384 + r * 128 + (((ch & 7) ^ (r & 7)) << 4)) = val;
   }
   fence_async_smem();
@@ -198,7 +203,7 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
     wait_page(0);
     if (!failed) {
       issue_qk(0, 0);
-      issue_qk(1, 0);
+      if (two) issue_qk(1, 0);
     }
     for (int j = 0; j < n_tiles && !failed; ++j) {
       const bool more = j + 1 < n_tiles;
@@ -215,13 +220,13 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
       issue_pv(0, j);
       if (failed) break;
       TC5H_STAMP(traced && lane == 0, 13, j);
-      if (more) {
+      if (more && two) {
         wait_s_free(1, j);
         if (failed) break;
         issue_qk(1, j + 1);
       }
       TC5H_STAMP(traced && lane == 0, 12, j);
-      issue_pv(1, j);
+      if (two) issue_pv(1, j);
       if (failed) break;
       umma_commit(&bar[B_KV_EMPTY + (j % kStages)]);  // page j has no reader left
     }
@@ -252,7 +257,8 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
     const uint32_t t_lane = tbase + ((uint32_t)((warp & 3) * 32) << 16);
     const uint32_t t_s = t_lane + h * 64, t_o = t_lane + 256 + h * 128;
     float m_ref = -INFINITY, l = 0.f;
-    for (int j = 0; j < n_tiles; ++j) {
+    const int n_mine = (h == 0 || two) ? n_tiles : 0;   // the idle group of a one-head block has no pages
+    for (int j = 0; j < n_mine; ++j) {
       if (!mbar_wait_bounded(&bar[B_S_FULL + h], j & 1)) { failed = true; break; }
       TC5H_STAMP(traced && row == 0, h * 4 + 0, j);
       fence_after();
@@ -353,7 +359,9 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
       mbar_arrive(&bar[B_P_FULL + 2 * h + (j & 1)]);
       TC5H_STAMP(traced && row == 0, h * 4 + 3, j);
     }
-    if (!failed && mbar_wait_bounded(&bar[B_O_DONE + 2 * h + ((n_tiles - 1) & 1)], 0)) {
+    if (n_mine == 0) {
+      // nothing to write
+    } else if (!failed && mbar_wait_bounded(&bar[B_O_DONE + 2 * h + ((n_tiles - 1) & 1)], 0)) {
       fence_after();
       const float inv = l > 0.f ? 1.f / l : 0.f;  // the bias of P cancels between O and l
       __nv_bfloat16 *orow = a.out + ((size_t)i * c.Hq + hq) * kD;
@@ -395,7 +403,7 @@ int launch_prefill_attn_tc5x2h(const PrefillArgs &a, cudaStream_t s) {
   if (cudaFuncSetAttribute(prefill_attn_tc5x2h_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            tc5x2h::kSmemBytes) != cudaSuccess)
     return SPKV_E_CUDA;
-  prefill_attn_tc5x2h_kernel<<<dim3(((a.C + 127) / 128) * a.c.Hkv * (a.c.G / 2)), tc5x2h::kThreads, tc5x2h::kSmemBytes,
+  prefill_attn_tc5x2h_kernel<<<dim3(((a.C + 127) / 128) * a.c.Hkv * ((a.c.G + 1) / 2)), tc5x2h::kThreads, tc5x2h::kSmemBytes,
                                s>>>(a);
   return check_stream_error(cudaGetLastError());
 }
