@@ -364,6 +364,7 @@ extern "C" int spkv_prefill(spkv_cache_t *cache, int32_t layer, int32_t seq, int
   a.stage_pages = reinterpret_cast<__nv_bfloat16 *>(static_cast<char *>(d_workspace) +
                                                     prefill_plan_bytes(&cache->cfg, C));
   a.n_stage_pages = prefill_stage_pages(&cache->cfg, C);
+  a.pair_tiles = 0;
   cudaStream_t s = as_stream(stream);
   cache->last_kind = kLastOther;
 

@@ -18,6 +18,7 @@ struct PrefillArgs {
   int ws_stride;
   __nv_bfloat16 *stage_pages;      // [Hkv][n_stage_pages] pages: old ring pairs + chunk pairs in
   int n_stage_pages;               //   position order, page format (tensor-core kernel only)
+  int pair_tiles;                  // fp16 two-slot kernel: a single head's blocks take two query tiles each
 };
 
 __device__ inline int32_t *unit_ws(const PrefillArgs &a, int kvh) { return a.ws + (size_t)kvh * a.ws_stride; }
@@ -28,13 +29,12 @@ __device__ inline int32_t *unit_ws(const PrefillArgs &a, int kvh) { return a.ws 
 // chunk (the plan kernel has counted them), and inside a head the query tiles run from the end
 // of the chunk backwards.  Item -> (KV head, which of its `blocks_per_kvh` head groups, query
 // tile).  Called by whole warps at kernel entry; every warp computes the same answer.
-__device__ inline void prefill_work_item(const PrefillArgs &a, int item, int n_xtiles, int blocks_per_kvh, int &kvh,
-                                         int &sub, int &xtile) {
-  const int r = item / n_xtiles, rank = r / blocks_per_kvh, lane = threadIdx.x & 31, Hkv = a.c.Hkv;
-  xtile = n_xtiles - 1 - item % n_xtiles;
-  sub = r % blocks_per_kvh;
-  kvh = rank;
-  if (Hkv > 32) return;  // more KV heads than lanes: plain order
+//
+// The KV head with the rank-th most keys per query in this chunk (ties by index).  Called by whole
+// warps; every warp computes the same answer.  More KV heads than lanes: plain order.
+__device__ inline int prefill_kvh_by_rank(const PrefillArgs &a, int rank) {
+  const int lane = threadIdx.x & 31, Hkv = a.c.Hkv;
+  if (Hkv > 32) return rank;
   int key = -1;
   if (lane < Hkv) {
     const int32_t *hdr = unit_ws(a, lane);
@@ -45,7 +45,14 @@ __device__ inline void prefill_work_item(const PrefillArgs &a, int item, int n_x
     const int other = __shfl_sync(0xffffffffu, key, k);
     my_rank += (other > key || (other == key && k < lane)) ? 1 : 0;
   }
-  kvh = __ffs(__ballot_sync(0xffffffffu, lane < Hkv && my_rank == rank)) - 1;
+  return __ffs(__ballot_sync(0xffffffffu, lane < Hkv && my_rank == rank)) - 1;
+}
+__device__ inline void prefill_work_item(const PrefillArgs &a, int item, int n_xtiles, int blocks_per_kvh, int &kvh,
+                                         int &sub, int &xtile) {
+  const int r = item / n_xtiles;
+  xtile = n_xtiles - 1 - item % n_xtiles;
+  sub = r % blocks_per_kvh;
+  kvh = prefill_kvh_by_rank(a, r / blocks_per_kvh);
 }
 
 

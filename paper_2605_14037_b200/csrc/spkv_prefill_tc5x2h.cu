@@ -1,9 +1,11 @@
 // Chunk attention of spkv_prefill on tcgen05, two query heads per block, P.V in fp16.
 //
-// Same tiling as the two-term bf16 kernel next door (one block = 128 consecutive queries of two
-// query heads that share a KV head -- of one, for the last head of an odd group --, Eq. 5;
-// every 32 KB page is fetched once and feeds both; one softmax group of 128 threads per head,
-// thread = query row = TMEM lane).  Two things differ:
+// Same tiling as the two-term bf16 kernel next door: one block = two 128-row slots that walk the
+// same pages -- two query heads that share a KV head on one tile of 128 consecutive queries
+// (Eq. 5), or, for the last head of an odd group (G = 1: every head), two consecutive query tiles
+// of that head; every 32 KB page is fetched once and feeds both slots; one softmax group of 128
+// threads per slot, thread = query row = TMEM lane.  ("Head h" below means slot h.)  Two things
+// differ:
 //
 // * P is ONE fp16 term (11 significant bits; the two-term bf16 split carries 16 but costs a second
 //   P.V pass).  The tensor cores want both operands in the same type, so warps 2-3 rewrite the
@@ -66,12 +68,29 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
   uint64_t *bar = reinterpret_cast<uint64_t *>(smem + kSBar);
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + kSBar + B_COUNT * 8);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  int kvh, pair, xtile;
-  prefill_work_item(a, blockIdx.x, (a.C + 127) / 128, (c.G + 1) >> 1, kvh, pair, xtile);
-  const int hq0 = kvh * c.G + pair * 2, i0 = xtile * 128;
-  // an odd number of query heads per KV head leaves the last block of a KV head with one head:
-  // its second group and the MMAs of head 1 stay idle
-  const bool two = pair * 2 + 1 < c.G;
+  // A block holds two 128-row slots that walk the same pages: two query heads of a KV head on
+  // one query tile, or -- for the last head of an odd group (G = 1: every head) -- two consecutive
+  // query tiles of that one head (one tile and an idle slot when the launch would otherwise have
+  // too few blocks to fill the GPU: a.pair_tiles = 0).  Work order: KV heads by keys per query, heaviest first; inside
+  // a head the head pairs tile by tile from the end of the chunk backwards, then the single head's
+  // tile pairs likewise.
+  const int n_xtiles = (a.C + 127) / 128, n_xpairs = a.pair_tiles ? (n_xtiles + 1) / 2 : n_xtiles;
+  const int per_kvh = (c.G >> 1) * n_xtiles + (c.G & 1) * n_xpairs;
+  const int kvh = prefill_kvh_by_rank(a, blockIdx.x / per_kvh), rem = blockIdx.x % per_kvh;
+  int hq_s[2], i0_s[2];
+  bool two;   // is slot 1 in use
+  if (rem < (c.G >> 1) * n_xtiles) {
+    const int pair = rem / n_xtiles, xtile = n_xtiles - 1 - rem % n_xtiles;
+    hq_s[0] = kvh * c.G + pair * 2; hq_s[1] = hq_s[0] + 1;
+    i0_s[0] = i0_s[1] = xtile * 128;
+    two = true;
+  } else {
+    const int xp = n_xpairs - 1 - (rem - (c.G >> 1) * n_xtiles);
+    hq_s[0] = hq_s[1] = kvh * c.G + c.G - 1;
+    i0_s[0] = a.pair_tiles ? xp * 256 : xp * 128;
+    i0_s[1] = i0_s[0] + 128;
+    two = a.pair_tiles && i0_s[1] < a.C;
+  }
   const int32_t *hdr = unit_ws(a, kvh);
   const int32_t *E = hdr + kHdrInts;
   const int len0 = hdr[H_LEN0], n_old = hdr[H_NOLD], N = hdr[H_N];
@@ -90,10 +109,11 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
   }
   // kept pairs visible to chunk query i: the first nvis(i) pairs of the compact cache
   auto nvis = [&](int i) { return len0 + E[min(max(i + n_old - c.w + 1, 0), N)]; };
-  const int i_last = min(i0 + 127, a.C - 1);
+  // the last query of the block (slot 1 never starts before slot 0) sees the most kept pairs
+  const int i_first = i0_s[0], i_last = min((two ? i0_s[1] : i0_s[0]) + 127, a.C - 1);
   const int n_ptiles = (nvis(i_last) + kP - 1) / kP;
-  // band, in staging indices (query i is staging pair n_old + i)
-  const int sp_lo = max(0, i0 + n_old - c.w + 1) / kP, sp_hi = (i_last + n_old) / kP;
+  // band of both slots together, in staging indices (query i is staging pair n_old + i)
+  const int sp_lo = max(0, i_first + n_old - c.w + 1) / kP, sp_hi = (i_last + n_old) / kP;
   const int n_tiles = n_ptiles + (sp_hi - sp_lo + 1);
 
   if (tid == 0) {
@@ -122,8 +142,8 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
   for (int x = tid; x < 2 * 128 * 16; x += kThreads) {
     const int h = x >> 11, r = (x >> 4) & 127, ch = x & 15;
     uint4 val = make_uint4(0, 0, 0, 0);
-    if (i0 + r < a.C && (h == 0 || two))
-      val = *reinterpret_cast<const uint4 *>(a.q + ((size_t)(i0 + r) * c.Hq + hq0 + h) * kD + ch * 8);
+    if (i0_s[h] + r < a.C && (h == 0 || two))
+      val = *reinterpret_cast<const uint4 *>(a.q + ((size_t)(i0_s[h] + r) * c.Hq + hq_s[h]) * kD + ch * 8);
     *reinterpret_cast<uint4 *>(smem + kSQ + h * 32768 + (ch >> 3) * 16384 + r * 128 + (((ch & 7) ^ (r & 7)) << 4)) = val;
   }
   fence_async_smem();
@@ -250,7 +270,7 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
     }
   } else {
     // ---------------------------------------------------------------- softmax groups
-    const int h = (warp >> 2) - 1, row = tid & 127, i = i0 + row, hq = hq0 + h;
+    const int h = (warp >> 2) - 1, row = tid & 127, i = i0_s[h] + row, hq = hq_s[h];
     const bool row_ok = i < a.C;
     const int nv = row_ok ? nvis(i) : 0;
     const int jq = n_old + i;  // staging index of this row's own pair
@@ -399,12 +419,23 @@ extern "C" int spkv_debug_tc5h_trace(long long *host_out) {
 }
 #endif
 
-int launch_prefill_attn_tc5x2h(const PrefillArgs &a, cudaStream_t s) {
+int launch_prefill_attn_tc5x2h(const PrefillArgs &a_in, cudaStream_t s) {
+  PrefillArgs a = a_in;
   if (cudaFuncSetAttribute(prefill_attn_tc5x2h_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            tc5x2h::kSmemBytes) != cudaSuccess)
     return SPKV_E_CUDA;
-  prefill_attn_tc5x2h_kernel<<<dim3(((a.C + 127) / 128) * a.c.Hkv * ((a.c.G + 1) / 2)), tc5x2h::kThreads, tc5x2h::kSmemBytes,
-                               s>>>(a);
+  const int n_xtiles = (a.C + 127) / 128;
+  // A single head's blocks take two query tiles each (the page walk then feeds 256 rows, as with
+  // a head pair) when that still leaves two waves of blocks; a small launch keeps one tile per
+  // block, whose finer grain balances better over the SMs.
+  static const int sms = [] {
+    int dev = 0, n = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    return n;
+  }();
+  a.pair_tiles = ((a.c.G / 2) * n_xtiles + (a.c.G & 1) * ((n_xtiles + 1) / 2)) * a.c.Hkv >= 2 * sms;
+  const int per_kvh = (a.c.G / 2) * n_xtiles + (a.c.G & 1) * (a.pair_tiles ? (n_xtiles + 1) / 2 : n_xtiles);
+  prefill_attn_tc5x2h_kernel<<<dim3(per_kvh * a.c.Hkv), tc5x2h::kThreads, tc5x2h::kSmemBytes, s>>>(a);
   return check_stream_error(cudaGetLastError());
 }
 

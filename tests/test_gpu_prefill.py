@@ -203,3 +203,23 @@ def test_prefill_scores_that_grow_or_fall_with_position(direction):
     for h in range(Hkv):
         compare_state(cache, 0, 0, h, units[h])
     assert_attn_close(got, ref, f"direction={direction}")
+
+
+@pytest.mark.parametrize("G,Hkv,chunks", [(1, 32, [2432, 600]), (3, 10, [2400, 257])])
+def test_prefill_single_head_blocks_take_two_query_tiles(G, Hkv, chunks):
+    """Odd query-group sizes in launches large enough for the last head of a group to run with
+    two consecutive query tiles per block (two waves of blocks or more): an odd and an even number
+    of tiles, then a smaller ragged chunk on top of that past (one tile per block again)."""
+    spkv = load()
+    w, Hq, T = 128, G * Hkv, sum(chunks)
+    rates = [((3 * i) % 10) / 10.0 for i in range(Hkv)]
+    cache = spkv.Cache(n_layers=1, max_seqs=1, n_q_heads=Hq, n_kv_heads=Hkv, max_context=4096,
+                       pool_pages=int(sum(rates) * T / 64) + 3 * Hkv + 8, window=w, tau=0.5)
+    tl = cache.spkv_tau_logit()
+    wl = Workload(4000 + G + len(chunks), T, 1, Hq, Hkv, rates, tl)
+    got = prefill_in_chunks(spkv, cache, 0, 0, wl, 0, chunks)
+    assert cache.spkv_status() == 0
+    units, ref = oracle_prefill(wl, 0, w, tl, G, T, 1.0 / math.sqrt(D))
+    for h in range(Hkv):
+        compare_state(cache, 0, 0, h, units[h])
+    assert_attn_close(got, ref, f"G={G} Hkv={Hkv} chunks={chunks}")
