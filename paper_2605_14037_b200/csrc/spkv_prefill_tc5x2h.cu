@@ -60,6 +60,8 @@ __device__ long long g_tc5h_trace[16][2048];
 #define TC5H_STAMP(cond, who, j) do { } while (0)
 #endif
 
+// kEvenG: every block is a head pair on one tile (the branches for single heads compile away).
+template <bool kEvenG>
 __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kernel(PrefillArgs a) {
   using namespace tc5;
   using namespace tc5x2h;
@@ -77,19 +79,19 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
   const int n_xtiles = (a.C + 127) / 128, n_xpairs = a.pair_tiles ? (n_xtiles + 1) / 2 : n_xtiles;
   const int per_kvh = (c.G >> 1) * n_xtiles + (c.G & 1) * n_xpairs;
   const int kvh = prefill_kvh_by_rank(a, blockIdx.x / per_kvh), rem = blockIdx.x % per_kvh;
-  int hq_s[2], i0_s[2];
+  int hq_s0, hq_s1, i0_s0, i0_s1;   // slot h: query head and first query row
   bool two;   // is slot 1 in use
-  if (rem < (c.G >> 1) * n_xtiles) {
+  if (kEvenG || rem < (c.G >> 1) * n_xtiles) {
     const int pair = rem / n_xtiles, xtile = n_xtiles - 1 - rem % n_xtiles;
-    hq_s[0] = kvh * c.G + pair * 2; hq_s[1] = hq_s[0] + 1;
-    i0_s[0] = i0_s[1] = xtile * 128;
+    hq_s0 = kvh * c.G + pair * 2; hq_s1 = hq_s0 + 1;
+    i0_s0 = i0_s1 = xtile * 128;
     two = true;
   } else {
     const int xp = n_xpairs - 1 - (rem - (c.G >> 1) * n_xtiles);
-    hq_s[0] = hq_s[1] = kvh * c.G + c.G - 1;
-    i0_s[0] = a.pair_tiles ? xp * 256 : xp * 128;
-    i0_s[1] = i0_s[0] + 128;
-    two = a.pair_tiles && i0_s[1] < a.C;
+    hq_s0 = hq_s1 = kvh * c.G + c.G - 1;
+    i0_s0 = a.pair_tiles ? xp * 256 : xp * 128;
+    i0_s1 = i0_s0 + 128;
+    two = a.pair_tiles && i0_s1 < a.C;
   }
   const int32_t *hdr = unit_ws(a, kvh);
   const int32_t *E = hdr + kHdrInts;
@@ -110,7 +112,8 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
   // kept pairs visible to chunk query i: the first nvis(i) pairs of the compact cache
   auto nvis = [&](int i) { return len0 + E[min(max(i + n_old - c.w + 1, 0), N)]; };
   // the last query of the block (slot 1 never starts before slot 0) sees the most kept pairs
-  const int i_first = i0_s[0], i_last = min((two ? i0_s[1] : i0_s[0]) + 127, a.C - 1);
+  if (kEvenG) two = true;
+  const int i_first = i0_s0, i_last = min((two ? i0_s1 : i0_s0) + 127, a.C - 1);
   const int n_ptiles = (nvis(i_last) + kP - 1) / kP;
   // band of both slots together, in staging indices (query i is staging pair n_old + i)
   const int sp_lo = max(0, i_first + n_old - c.w + 1) / kP, sp_hi = (i_last + n_old) / kP;
@@ -142,8 +145,9 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
   for (int x = tid; x < 2 * 128 * 16; x += kThreads) {
     const int h = x >> 11, r = (x >> 4) & 127, ch = x & 15;
     uint4 val = make_uint4(0, 0, 0, 0);
-    if (i0_s[h] + r < a.C && (h == 0 || two))
-      val = *reinterpret_cast<const uint4 *>(a.q + ((size_t)(i0_s[h] + r) * c.Hq + hq_s[h]) * kD + ch * 8);
+    const int i0h = h ? i0_s1 : i0_s0, hqh = h ? hq_s1 : hq_s0;
+    if (i0h + r < a.C && (h == 0 || two))
+      val = *reinterpret_cast<const uint4 *>(a.q + ((size_t)(i0h + r) * c.Hq + hqh) * kD + ch * 8);
     *reinterpret_cast<uint4 *>(smem + kSQ + h * 32768 + (ch >> 3) * 16384 + r * 128 + (((ch & 7) ^ (r & 7)) << 4)) = val;
   }
   fence_async_smem();
@@ -270,7 +274,7 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
     }
   } else {
     // ---------------------------------------------------------------- softmax groups
-    const int h = (warp >> 2) - 1, row = tid & 127, i = i0_s[h] + row, hq = hq_s[h];
+    const int h = (warp >> 2) - 1, row = tid & 127, i = (h ? i0_s1 : i0_s0) + row, hq = h ? hq_s1 : hq_s0;
     const bool row_ok = i < a.C;
     const int nv = row_ok ? nvis(i) : 0;
     const int jq = n_old + i;  // staging index of this row's own pair
@@ -421,8 +425,8 @@ extern "C" int spkv_debug_tc5h_trace(long long *host_out) {
 
 int launch_prefill_attn_tc5x2h(const PrefillArgs &a_in, cudaStream_t s) {
   PrefillArgs a = a_in;
-  if (cudaFuncSetAttribute(prefill_attn_tc5x2h_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           tc5x2h::kSmemBytes) != cudaSuccess)
+  auto kernel = (a.c.G & 1) ? prefill_attn_tc5x2h_kernel<false> : prefill_attn_tc5x2h_kernel<true>;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc5x2h::kSmemBytes) != cudaSuccess)
     return SPKV_E_CUDA;
   const int n_xtiles = (a.C + 127) / 128;
   // A single head's blocks take two query tiles each (the page walk then feeds 256 rows, as with
@@ -435,7 +439,7 @@ int launch_prefill_attn_tc5x2h(const PrefillArgs &a_in, cudaStream_t s) {
   }();
   a.pair_tiles = ((a.c.G / 2) * n_xtiles + (a.c.G & 1) * ((n_xtiles + 1) / 2)) * a.c.Hkv >= 2 * sms;
   const int per_kvh = (a.c.G / 2) * n_xtiles + (a.c.G & 1) * (a.pair_tiles ? (n_xtiles + 1) / 2 : n_xtiles);
-  prefill_attn_tc5x2h_kernel<<<dim3(per_kvh * a.c.Hkv), tc5x2h::kThreads, tc5x2h::kSmemBytes, s>>>(a);
+  kernel<<<dim3(per_kvh * a.c.Hkv), tc5x2h::kThreads, tc5x2h::kSmemBytes, s>>>(a);
   return check_stream_error(cudaGetLastError());
 }
 
