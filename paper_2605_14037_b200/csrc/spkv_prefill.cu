@@ -333,8 +333,10 @@ static int prefill_stage_pages(const spkv_config_t *cfg, int C) { return (C + cf
 
 extern "C" size_t spkv_prefill_workspace_bytes(const spkv_config_t *cfg, int32_t C) {
   if (!cfg || C < 0) return 0;
-  // plan (header + prefix sums per KV head), then the staging pages of the chunk attention
-  return prefill_plan_bytes(cfg, C) + (size_t)cfg->n_kv_heads * prefill_stage_pages(cfg, C) * kPageBytes;
+  // plan (header + prefix sums per KV head), then the staging pages of the chunk attention, then
+  // (small chunks only) the partial results of split page walks
+  return prefill_plan_bytes(cfg, C) + (size_t)cfg->n_kv_heads * prefill_stage_pages(cfg, C) * kPageBytes +
+         prefill_split_bytes(cfg, C);
 }
 
 extern "C" int spkv_prefill(spkv_cache_t *cache, int32_t layer, int32_t seq, int32_t C,
@@ -365,6 +367,11 @@ extern "C" int spkv_prefill(spkv_cache_t *cache, int32_t layer, int32_t seq, int
                                                     prefill_plan_bytes(&cache->cfg, C));
   a.n_stage_pages = prefill_stage_pages(&cache->cfg, C);
   a.pair_tiles = 0;
+  a.n_split = 1;
+  a.partials = prefill_split_bytes(&cache->cfg, C)
+                   ? reinterpret_cast<float *>(reinterpret_cast<char *>(a.stage_pages) +
+                                               (size_t)v.Hkv * a.n_stage_pages * kPageBytes)
+                   : nullptr;
   cudaStream_t s = as_stream(stream);
   cache->last_kind = kLastOther;
 

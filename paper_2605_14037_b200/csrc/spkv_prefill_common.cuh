@@ -19,6 +19,8 @@ struct PrefillArgs {
   __nv_bfloat16 *stage_pages;      // [Hkv][n_stage_pages] pages: old ring pairs + chunk pairs in
   int n_stage_pages;               //   position order, page format (tensor-core kernel only)
   int pair_tiles;                  // fp16 two-slot kernel: a single head's blocks take two query tiles each
+  int n_split;                     // fp16 two-slot kernel: blocks per page walk (split over the pages), >= 1
+  float *partials;                 // [walk][slot][split]: 128 rows x (128 O + pad) and (m, l); n_split > 1 only
 };
 
 __device__ inline int32_t *unit_ws(const PrefillArgs &a, int kvh) { return a.ws + (size_t)kvh * a.ws_stride; }
@@ -60,5 +62,6 @@ __device__ inline void prefill_work_item(const PrefillArgs &a, int item, int n_x
 int launch_prefill_attn_tc5(const PrefillArgs &a, cudaStream_t s);
 int launch_prefill_attn_tc5x2(const PrefillArgs &a, cudaStream_t s);
 int launch_prefill_attn_tc5x2h(const PrefillArgs &a, cudaStream_t s);
+size_t prefill_split_bytes(const spkv_config_t *cfg, int C);   // partial results of split page walks (small chunks)
 
 }  // namespace spkv

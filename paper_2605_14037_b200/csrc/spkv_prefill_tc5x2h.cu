@@ -34,6 +34,8 @@
 // Shared memory: Q of both heads (64 KB) + 5 page stages.
 // Warps: 0 MMA issue, 1 page loader + TMEM allocation, 2-3 value conversion, 4-7 group 0,
 // 8-11 group 1.  All waits are bounded.
+#include <algorithm>
+
 #include "spkv_prefill_common.cuh"
 #include "spkv_tc5.cuh"
 
@@ -51,6 +53,8 @@ enum { B_KV_FULL = 0, B_KV_EMPTY = 8, B_V_READY = 16 /* [stage] */, B_S_FULL = 2
        B_P_FULL = 28 /* [2h+b] */, B_O_DONE = 32 /* [2h+b] */, B_COUNT = 36 };
 constexpr int kConvThreads = 64;           // warps 2-3
 constexpr float kPBias = 7.f;              // P is stored as 2^7 p
+constexpr int kPartFloats = 128 * 128 + 128 * 2;   // one partial result: O of 128 rows, then (m, l) per row
+constexpr int kMaxSplit = 16;
 }  // namespace tc5x2h
 
 #ifdef SPKV_TC5_TRACE
@@ -59,6 +63,49 @@ __device__ long long g_tc5h_trace[16][2048];
 #else
 #define TC5H_STAMP(cond, who, j) do { } while (0)
 #endif
+
+// A page walk serves two 128-row slots: two query heads of a KV head on one query tile, or -- for
+// the last head of an odd group (G = 1: every head) -- two consecutive query tiles of that one
+// head (one tile and an idle slot when the launch would otherwise have too few blocks to fill
+// the GPU: a.pair_tiles = 0).  Work order: KV heads by keys per query, heaviest first; inside a
+// head the head pairs tile by tile from the end of the chunk backwards, then the single head's
+// tile pairs likewise.  Called by whole warps.
+struct WalkSlots {
+  int kvh, hq0, hq1, i00, i01;   // slot h: query head hq<h>, first query row i0<h>
+  bool two;                      // is slot 1 in use
+};
+template <bool kEvenG>
+__device__ inline WalkSlots walk_slots(const PrefillArgs &a, int walk) {
+  const CacheView &c = a.c;
+  const int n_xtiles = (a.C + 127) / 128, n_xpairs = a.pair_tiles ? (n_xtiles + 1) / 2 : n_xtiles;
+  const int per_kvh = (c.G >> 1) * n_xtiles + (c.G & 1) * n_xpairs;
+  WalkSlots w;
+  w.kvh = prefill_kvh_by_rank(a, walk / per_kvh);
+  const int rem = walk % per_kvh;
+  if (kEvenG || rem < (c.G >> 1) * n_xtiles) {
+    const int pair = rem / n_xtiles, xtile = n_xtiles - 1 - rem % n_xtiles;
+    w.hq0 = w.kvh * c.G + pair * 2; w.hq1 = w.hq0 + 1;
+    w.i00 = w.i01 = xtile * 128;
+    w.two = true;
+  } else {
+    const int xp = n_xpairs - 1 - (rem - (c.G >> 1) * n_xtiles);
+    w.hq0 = w.hq1 = w.kvh * c.G + c.G - 1;
+    w.i00 = a.pair_tiles ? xp * 256 : xp * 128;
+    w.i01 = w.i00 + 128;
+    w.two = a.pair_tiles && w.i01 < a.C;
+  }
+  return w;
+}
+// the power of two that brings the unit's largest |v| into [2^14, 2^15), and its inverse
+__device__ inline void value_scale(const CacheView &c, int u, float &v_scale, float &v_unscale) {
+  v_scale = v_unscale = 1.f;
+  const uint32_t vm = c.vmax[u];
+  if (vm) {
+    const int k = min(14 - ((int)(vm >> 23) - 127), 126);
+    v_scale = __int_as_float((127 + k) << 23);
+    v_unscale = __int_as_float((127 - k) << 23);
+  }
+}
 
 // kEvenG: every block is a head pair on one tile (the branches for single heads compile away).
 template <bool kEvenG>
@@ -70,29 +117,11 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
   uint64_t *bar = reinterpret_cast<uint64_t *>(smem + kSBar);
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + kSBar + B_COUNT * 8);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  // A block holds two 128-row slots that walk the same pages: two query heads of a KV head on
-  // one query tile, or -- for the last head of an odd group (G = 1: every head) -- two consecutive
-  // query tiles of that one head (one tile and an idle slot when the launch would otherwise have
-  // too few blocks to fill the GPU: a.pair_tiles = 0).  Work order: KV heads by keys per query, heaviest first; inside
-  // a head the head pairs tile by tile from the end of the chunk backwards, then the single head's
-  // tile pairs likewise.
-  const int n_xtiles = (a.C + 127) / 128, n_xpairs = a.pair_tiles ? (n_xtiles + 1) / 2 : n_xtiles;
-  const int per_kvh = (c.G >> 1) * n_xtiles + (c.G & 1) * n_xpairs;
-  const int kvh = prefill_kvh_by_rank(a, blockIdx.x / per_kvh), rem = blockIdx.x % per_kvh;
-  int hq_s0, hq_s1, i0_s0, i0_s1;   // slot h: query head and first query row
-  bool two;   // is slot 1 in use
-  if (kEvenG || rem < (c.G >> 1) * n_xtiles) {
-    const int pair = rem / n_xtiles, xtile = n_xtiles - 1 - rem % n_xtiles;
-    hq_s0 = kvh * c.G + pair * 2; hq_s1 = hq_s0 + 1;
-    i0_s0 = i0_s1 = xtile * 128;
-    two = true;
-  } else {
-    const int xp = n_xpairs - 1 - (rem - (c.G >> 1) * n_xtiles);
-    hq_s0 = hq_s1 = kvh * c.G + c.G - 1;
-    i0_s0 = a.pair_tiles ? xp * 256 : xp * 128;
-    i0_s1 = i0_s0 + 128;
-    two = a.pair_tiles && i0_s1 < a.C;
-  }
+  // a.n_split blocks share one page walk (small launches: see the launcher)
+  const int walk = blockIdx.x / a.n_split, split = blockIdx.x % a.n_split;
+  const WalkSlots ws = walk_slots<kEvenG>(a, walk);
+  const int kvh = ws.kvh, hq_s0 = ws.hq0, hq_s1 = ws.hq1, i0_s0 = ws.i00, i0_s1 = ws.i01;
+  bool two = ws.two;
   const int32_t *hdr = unit_ws(a, kvh);
   const int32_t *E = hdr + kHdrInts;
   const int len0 = hdr[H_LEN0], n_old = hdr[H_NOLD], N = hdr[H_N];
@@ -100,15 +129,8 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
   // The values are multiplied by 2^k with the unit's largest |v| brought into [2^14, 2^15) (every
   // value the unit holds or this chunk brings is covered by vmax); the epilogue multiplies by
   // 2^-k.  Both are exact.
-  float v_scale = 1.f, v_unscale = 1.f;
-  {
-    const uint32_t vm = c.vmax[u];
-    if (vm) {
-      const int k = min(14 - ((int)(vm >> 23) - 127), 126);
-      v_scale = __int_as_float((127 + k) << 23);
-      v_unscale = __int_as_float((127 - k) << 23);
-    }
-  }
+  float v_scale, v_unscale;
+  value_scale(c, u, v_scale, v_unscale);
   // kept pairs visible to chunk query i: the first nvis(i) pairs of the compact cache
   auto nvis = [&](int i) { return len0 + E[min(max(i + n_old - c.w + 1, 0), N)]; };
   // the last query of the block (slot 1 never starts before slot 0) sees the most kept pairs
@@ -117,7 +139,11 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
   const int n_ptiles = (nvis(i_last) + kP - 1) / kP;
   // band of both slots together, in staging indices (query i is staging pair n_old + i)
   const int sp_lo = max(0, i_first + n_old - c.w + 1) / kP, sp_hi = (i_last + n_old) / kP;
-  const int n_tiles = n_ptiles + (sp_hi - sp_lo + 1);
+  const int n_tiles_all = n_ptiles + (sp_hi - sp_lo + 1);
+  // this block's share of the walk: pages [j_begin, j_begin + n_tiles) of the list (compact-cache
+  // pages, then band pages); page numbers below are local, j_begin + j is the page's place in the list
+  const int j_begin = (int)((long long)n_tiles_all * split / a.n_split);
+  const int n_tiles = (int)((long long)n_tiles_all * (split + 1) / a.n_split) - j_begin;
 
   if (tid == 0) {
     for (int i = 0; i < kStages; ++i) {
@@ -169,7 +195,7 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
     // ---------------------------------------------------------------- page loader
     int j = 0;
     for (int base = 0; base < n_tiles && !failed; base += 32) {
-      const int jl = base + lane;
+      const int jl = j_begin + base + lane;
       int64_t src_off = 0;
       if (jl < n_ptiles) src_off = (int64_t)c.table[(size_t)u * c.max_pages + jl] * kPageElems;
       const int cnt = min(32, n_tiles - base);
@@ -180,8 +206,9 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
           if (j >= kStages && !mbar_wait_bounded(&bar[B_KV_EMPTY + s], ((j / kStages) - 1) & 1)) failed = true;
           if (!failed) {
             const __nv_bfloat16 *src =
-                j < n_ptiles ? c.pages + off
-                             : a.stage_pages + ((size_t)kvh * a.n_stage_pages + sp_lo + (j - n_ptiles)) * kPageElems;
+                j_begin + j < n_ptiles
+                    ? c.pages + off
+                    : a.stage_pages + ((size_t)kvh * a.n_stage_pages + sp_lo + (j_begin + j - n_ptiles)) * kPageElems;
             mbar_arrive_expect_tx(&bar[B_KV_FULL + s], kPageBytes);
             bulk_load(smem + kSKV + s * kPageBytes, src, kPageBytes, &bar[B_KV_FULL + s]);
           }
@@ -224,8 +251,8 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
       // the last two P.V have no later Q.K^T whose S_FULL would vouch for their completion
       if (jj + 2 >= n_tiles) umma_commit(&bar[B_O_DONE + 2 * h + (jj & 1)]);
     };
-    wait_page(0);
-    if (!failed) {
+    if (n_tiles > 0) wait_page(0);
+    if (!failed && n_tiles > 0) {
       issue_qk(0, 0);
       if (two) issue_qk(1, 0);
     }
@@ -302,14 +329,15 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
       // visibility: compact-cache page j -> first nv pairs; staging page -> the band of this row.
       // v keeps the raw scores (masked ones become -inf); the scale is folded into the exponent,
       // and pages that every row of the warp sees in full skip the masking altogether.
-      if (j < n_ptiles) {
-        const int base = j * kP;
+      const int jg = j_begin + j;   // the page's place in the list
+      if (jg < n_ptiles) {
+        const int base = jg * kP;
         if (!__all_sync(0xffffffffu, base + kP <= nv)) {
 #pragma unroll
           for (int x = 0; x < 64; ++x) v[x] = (base + x < nv) ? v[x] : -INFINITY;
         }
       } else {
-        const int base = (sp_lo + j - n_ptiles) * kP;
+        const int base = (sp_lo + jg - n_ptiles) * kP;
 #pragma unroll
         for (int x = 0; x < 64; ++x) {
           const int jj = base + x;
@@ -383,8 +411,33 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
       mbar_arrive(&bar[B_P_FULL + 2 * h + (j & 1)]);
       TC5H_STAMP(traced && row == 0, h * 4 + 3, j);
     }
-    if (n_mine == 0) {
-      // nothing to write
+    if (h == 1 && !two) {
+      // idle slot: nothing to write
+    } else if (a.n_split > 1) {
+      // a share of a split walk: the unnormalised row (fp32, in the scaled units) and its (m, l)
+      // go to the partial results; prefill_merge_kernel puts the shares together
+      float *part = a.partials + ((size_t)(walk * 2 + h) * a.n_split + split) * kPartFloats;
+      if (n_tiles == 0) {
+        part[128 * 128 + row * 2] = -INFINITY;
+        part[128 * 128 + row * 2 + 1] = 0.f;
+      } else if (!failed && mbar_wait_bounded(&bar[B_O_DONE + 2 * h + ((n_tiles - 1) & 1)], 0)) {
+        fence_after();
+#pragma unroll
+        for (int q8 = 0; q8 < 8; ++q8) {
+          float t16[16];
+          tmem_ld16(t_o + q8 * 16, t16);
+          tmem_ld_wait();
+          float4 *dst = reinterpret_cast<float4 *>(part + row * 128 + q8 * 16);
+          dst[0] = make_float4(t16[0], t16[1], t16[2], t16[3]);
+          dst[1] = make_float4(t16[4], t16[5], t16[6], t16[7]);
+          dst[2] = make_float4(t16[8], t16[9], t16[10], t16[11]);
+          dst[3] = make_float4(t16[12], t16[13], t16[14], t16[15]);
+        }
+        part[128 * 128 + row * 2] = m_ref;
+        part[128 * 128 + row * 2 + 1] = l;
+      } else {
+        failed = true;
+      }
     } else if (!failed && mbar_wait_bounded(&bar[B_O_DONE + 2 * h + ((n_tiles - 1) & 1)], 0)) {
       fence_after();
       const float inv = l > 0.f ? 1.f / l : 0.f;  // the bias of P cancels between O and l
@@ -423,6 +476,76 @@ extern "C" int spkv_debug_tc5h_trace(long long *host_out) {
 }
 #endif
 
+// Puts the shares of a split page walk together: out = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s
+// (M = max_s m_s; the m are log2-domain reference maxima, the O and l carry the same bias and value
+// scale in every share).  grid (walks, 2 slots), 256 threads: thread = (row, 16-dim group) x 4.
+template <bool kEvenG>
+__global__ void __launch_bounds__(256) prefill_merge_kernel(PrefillArgs a) {
+  using namespace tc5x2h;
+  const CacheView &c = a.c;
+  const int walk = blockIdx.x, h = blockIdx.y, S = a.n_split;
+  const WalkSlots ws = walk_slots<kEvenG>(a, walk);
+  if (h == 1 && !ws.two) return;
+  const int hq = h ? ws.hq1 : ws.hq0, i0 = h ? ws.i01 : ws.i00;
+  float v_scale, v_unscale;
+  value_scale(c, unit_index(c, a.layer, a.seq, ws.kvh), v_scale, v_unscale);
+  const float *part = a.partials + (size_t)(walk * 2 + h) * S * kPartFloats;
+  __shared__ float s_w[kMaxSplit][128];   // weight of share s for a row, already divided by the row sum
+  for (int row = threadIdx.x; row < 128; row += blockDim.x) {
+    float M = -INFINITY;
+    for (int s = 0; s < S; ++s) M = fmaxf(M, part[(size_t)s * kPartFloats + 128 * 128 + row * 2]);
+    float L = 0.f;
+    for (int s = 0; s < S; ++s) {
+      const float m = part[(size_t)s * kPartFloats + 128 * 128 + row * 2];
+      const float wgt = m == -INFINITY ? 0.f : exp2f(m - M);
+      s_w[s][row] = wgt;
+      L += wgt * part[(size_t)s * kPartFloats + 128 * 128 + row * 2 + 1];
+    }
+    const float inv = L > 0.f ? 1.f / L : 0.f;
+    for (int s = 0; s < S; ++s) s_w[s][row] *= inv;
+  }
+  __syncthreads();
+  for (int x = threadIdx.x; x < 128 * 8; x += blockDim.x) {
+    const int row = x >> 3, g = x & 7, i = i0 + row;
+    if (i >= a.C) continue;
+    float acc[16];
+#pragma unroll
+    for (int d = 0; d < 16; ++d) acc[d] = 0.f;
+    for (int s = 0; s < S; ++s) {
+      const float wgt = s_w[s][row];
+      if (wgt == 0.f) continue;   // an empty share has written no O
+      const float4 *src = reinterpret_cast<const float4 *>(part + (size_t)s * kPartFloats + row * 128 + g * 16);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const float4 v = src[q];
+        acc[4 * q] += wgt * v.x; acc[4 * q + 1] += wgt * v.y; acc[4 * q + 2] += wgt * v.z; acc[4 * q + 3] += wgt * v.w;
+      }
+    }
+    uint4 w0, w1;
+    w0.x = pack_bf16(acc[0] * v_unscale, acc[1] * v_unscale);   w0.y = pack_bf16(acc[2] * v_unscale, acc[3] * v_unscale);
+    w0.z = pack_bf16(acc[4] * v_unscale, acc[5] * v_unscale);   w0.w = pack_bf16(acc[6] * v_unscale, acc[7] * v_unscale);
+    w1.x = pack_bf16(acc[8] * v_unscale, acc[9] * v_unscale);   w1.y = pack_bf16(acc[10] * v_unscale, acc[11] * v_unscale);
+    w1.z = pack_bf16(acc[12] * v_unscale, acc[13] * v_unscale); w1.w = pack_bf16(acc[14] * v_unscale, acc[15] * v_unscale);
+    __nv_bfloat16 *orow = a.out + ((size_t)i * c.Hq + hq) * kD + g * 16;
+    *reinterpret_cast<uint4 *>(orow) = w0;
+    *reinterpret_cast<uint4 *>(orow + 8) = w1;
+  }
+}
+
+// Number of blocks that share a page walk.  A chunk of a few hundred tokens has only a handful of
+// walks (tiles x KV heads x head pairs) however long the context is; cutting each walk into
+// shares, as the decode kernel cuts a unit into page ranges, puts the other SMs to work.
+int prefill_split_count(int n_walks, int sms) {
+  if (n_walks >= sms) return 1;
+  return std::min(tc5x2h::kMaxSplit, (2 * sms + n_walks - 1) / n_walks);
+}
+size_t prefill_split_bytes(const spkv_config_t *cfg, int C) {
+  const int n_xtiles = (C + 127) / 128, G = cfg->n_q_heads / cfg->n_kv_heads;
+  const int n_walks = ((G / 2) * n_xtiles + (G & 1) * n_xtiles) * cfg->n_kv_heads;
+  const int S = prefill_split_count(n_walks, 192);   // an upper bound for any GPU of up to 192 SMs
+  return S > 1 ? (size_t)n_walks * 2 * S * tc5x2h::kPartFloats * 4 : 0;
+}
+
 int launch_prefill_attn_tc5x2h(const PrefillArgs &a_in, cudaStream_t s) {
   PrefillArgs a = a_in;
   auto kernel = (a.c.G & 1) ? prefill_attn_tc5x2h_kernel<false> : prefill_attn_tc5x2h_kernel<true>;
@@ -439,7 +562,13 @@ int launch_prefill_attn_tc5x2h(const PrefillArgs &a_in, cudaStream_t s) {
   }();
   a.pair_tiles = ((a.c.G / 2) * n_xtiles + (a.c.G & 1) * ((n_xtiles + 1) / 2)) * a.c.Hkv >= 2 * sms;
   const int per_kvh = (a.c.G / 2) * n_xtiles + (a.c.G & 1) * (a.pair_tiles ? (n_xtiles + 1) / 2 : n_xtiles);
-  kernel<<<dim3(per_kvh * a.c.Hkv), tc5x2h::kThreads, tc5x2h::kSmemBytes, s>>>(a);
+  const int n_walks = per_kvh * a.c.Hkv;
+  a.n_split = a.partials ? prefill_split_count(n_walks, std::min(sms, 192)) : 1;
+  kernel<<<dim3(n_walks * a.n_split), tc5x2h::kThreads, tc5x2h::kSmemBytes, s>>>(a);
+  if (a.n_split > 1) {
+    if (a.c.G & 1) prefill_merge_kernel<false><<<dim3(n_walks, 2), 256, 0, s>>>(a);
+    else           prefill_merge_kernel<true><<<dim3(n_walks, 2), 256, 0, s>>>(a);
+  }
   return check_stream_error(cudaGetLastError());
 }
 

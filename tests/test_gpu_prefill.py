@@ -223,3 +223,37 @@ def test_prefill_single_head_blocks_take_two_query_tiles(G, Hkv, chunks):
     for h in range(Hkv):
         compare_state(cache, 0, 0, h, units[h])
     assert_attn_close(got, ref, f"G={G} Hkv={Hkv} chunks={chunks}")
+
+
+@pytest.mark.parametrize("G,Hkv,small", [(4, 2, [48, 1, 130]), (1, 3, [16, 200]), (3, 2, [257])])
+def test_small_chunks_on_a_long_past_split_their_page_walks(G, Hkv, small):
+    """Chunks of a few tokens on a 20 k past: the launch has only a handful of page walks, each
+    hundreds of pages long, so every walk is cut into shares over several blocks and the shares
+    are merged by their log-sum-exp weights (some shares of the shortest heads are empty).
+    Every row of the small chunks against the mask form; state against the streaming form."""
+    spkv = load()
+    w, T0, Hq = 128, 20000, G * Hkv
+    T = T0 + sum(small)
+    rates = [0.02, 0.7, 0.3][:Hkv]
+    cache = spkv.Cache(n_layers=1, max_seqs=1, n_q_heads=Hq, n_kv_heads=Hkv, max_context=32768,
+                       pool_pages=int(sum(rates) * T / 64) + 3 * Hkv + 8, window=w, tau=0.5)
+    tl = cache.spkv_tau_logit()
+    wl = Workload(5000 + G, T, 1, Hq, Hkv, rates, tl)
+    prefill_in_chunks(spkv, cache, 0, 0, wl, 0, [8192, 8192, T0 - 16384], with_q=False)
+    K, V, Q = to_dev_bf16(wl.K[:, 0]), to_dev_bf16(wl.V[:, 0]), to_dev_bf16(wl.q[:, 0])
+    lg = torch.from_numpy(np.ascontiguousarray(wl.logit[:, 0])).to(dev())
+    outs, a = [], T0
+    for c in small:
+        outs.append(spkv.bits_from_bf16(cache.spkv_prefill(0, 0, K[a:a + c], V[a:a + c], lg[a:a + c], q=Q[a:a + c])))
+        a += c
+    assert cache.spkv_status() == 0
+    out = np.concatenate(outs)
+    scale = 1.0 / math.sqrt(D)
+    for h in range(Hkv):
+        Kh, Vh, Lh = (np.ascontiguousarray(x) for x in (wl.K[:, 0, h], wl.V[:, 0, h], wl.logit[:, 0, h]))
+        for t in range(T0, T, 3 if T - T0 > 100 else 1):
+            ref = oracle.mask_attend_row(Kh, Vh, Lh, t, w, tl, np.ascontiguousarray(wl.q[t, 0, h * G:(h + 1) * G]), scale)
+            assert_attn_close(out[t - T0, h * G:(h + 1) * G], ref, f"t={t} kvh={h}")
+        u = oracle.Unit(w, D)
+        u.prefill(Kh, Vh, Lh, tl)
+        compare_state(cache, 0, 0, h, u)
