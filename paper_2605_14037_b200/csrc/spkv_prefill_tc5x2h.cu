@@ -27,6 +27,10 @@
 // (special-function unit, the scarce resource) run under the load / maximum / hand-over phases of
 // the other instead of both queueing for the same unit at the same time.
 //
+// A launch with fewer page walks than SMs (a chunk of a few hundred tokens) cuts every walk into
+// up to 16 shares of consecutive pages, one block each; a share writes its unnormalised rows and
+// their (m, l), and prefill_merge_kernel combines the shares by their log-sum-exp weights.
+//
 // No unit is saturated (tensor pipe ~54 % active, special-function unit ~41 %, issue slots ~54 %):
 // the page period is the length of the chain scores -> softmax -> P -> MMA warp -> next scores.
 // (Computing part of the exponentials by polynomial on the FMA pipe, which helps when the
