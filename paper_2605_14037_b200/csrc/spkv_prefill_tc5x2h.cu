@@ -59,6 +59,7 @@ constexpr int kConvThreads = 64;           // warps 2-3
 constexpr float kPBias = 7.f;              // P is stored as 2^7 p
 constexpr int kPartFloats = 128 * 128 + 128 * 2;   // one partial result: O of 128 rows, then (m, l) per row
 constexpr int kMaxSplit = 16;
+constexpr int kMinSharePages = 16;          // a walk is not cut into shares shorter than this
 }  // namespace tc5x2h
 
 #ifdef SPKV_TC5_TRACE
@@ -146,8 +147,22 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
   const int n_tiles_all = n_ptiles + (sp_hi - sp_lo + 1);
   // this block's share of the walk: pages [j_begin, j_begin + n_tiles) of the list (compact-cache
   // pages, then band pages); page numbers below are local, j_begin + j is the page's place in the list
-  const int j_begin = (int)((long long)n_tiles_all * split / a.n_split);
-  const int n_tiles = (int)((long long)n_tiles_all * (split + 1) / a.n_split) - j_begin;
+  // (a walk takes as many of its a.n_split blocks as it has runs of kMinSharePages pages; the
+  // others find an empty share and leave at once)
+  const int n_shares = min(a.n_split, (n_tiles_all + kMinSharePages - 1) / kMinSharePages);
+  const int j_begin = split < n_shares ? (int)((long long)n_tiles_all * split / n_shares) : n_tiles_all;
+  const int n_tiles = split < n_shares ? (int)((long long)n_tiles_all * (split + 1) / n_shares) - j_begin : 0;
+  if (n_tiles == 0) {  // empty share (split walks only): says so in its partial result and leaves
+    if (warp >= 4) {
+      const int h = (warp >> 2) - 1;
+      if (h == 0 || two) {
+        float *part = a.partials + ((size_t)(walk * 2 + h) * a.n_split + split) * kPartFloats;
+        part[128 * 128 + (tid & 127) * 2] = -INFINITY;
+        part[128 * 128 + (tid & 127) * 2 + 1] = 0.f;
+      }
+    }
+    return;
+  }
 
   if (tid == 0) {
     for (int i = 0; i < kStages; ++i) {
@@ -539,15 +554,25 @@ __global__ void __launch_bounds__(256) prefill_merge_kernel(PrefillArgs a) {
 // Number of blocks that share a page walk.  A chunk of a few hundred tokens has only a handful of
 // walks (tiles x KV heads x head pairs) however long the context is; cutting each walk into
 // shares, as the decode kernel cuts a unit into page ranges, puts the other SMs to work.
+// Measured on a 32 k past, 32 query / 8 KV heads (TFLOP/s useful, whole call): with fewer walks
+// than SMs two waves of shares are best; a launch of one to two and a half waves of whole walks
+// is as slow as its longest walk (the heaviest head: ~0.5 ms) and gains from about six waves of
+// shares (chunk 1536: 460 -> 670, 2048: 600 -> 730); from there on whole walks win.
 int prefill_split_count(int n_walks, int sms) {
-  if (n_walks >= sms) return 1;
-  return std::min(tc5x2h::kMaxSplit, (2 * sms + n_walks - 1) / n_walks);
+  if (2 * n_walks >= 5 * sms) return 1;
+  const int target = n_walks < sms ? 2 * sms : 6 * sms;
+  return std::min(tc5x2h::kMaxSplit, (target + n_walks - 1) / n_walks);
+}
+// partial results the workspace holds: walks (one query tile per single head) x shares, for a GPU
+// of up to 192 SMs; the launcher never uses more (fewer walks or fewer SMs mean fewer blocks)
+static long long split_slots(int C, int G, int Hkv) {
+  const int n_xtiles = (C + 127) / 128;
+  const int n_walks = ((G / 2) * n_xtiles + (G & 1) * n_xtiles) * Hkv;
+  const int S = prefill_split_count(n_walks, 192);
+  return S > 1 ? (long long)n_walks * S : 0;
 }
 size_t prefill_split_bytes(const spkv_config_t *cfg, int C) {
-  const int n_xtiles = (C + 127) / 128, G = cfg->n_q_heads / cfg->n_kv_heads;
-  const int n_walks = ((G / 2) * n_xtiles + (G & 1) * n_xtiles) * cfg->n_kv_heads;
-  const int S = prefill_split_count(n_walks, 192);   // an upper bound for any GPU of up to 192 SMs
-  return S > 1 ? (size_t)n_walks * 2 * S * tc5x2h::kPartFloats * 4 : 0;
+  return (size_t)split_slots(C, cfg->n_q_heads / cfg->n_kv_heads, cfg->n_kv_heads) * 2 * tc5x2h::kPartFloats * 4;
 }
 
 int launch_prefill_attn_tc5x2h(const PrefillArgs &a_in, cudaStream_t s) {
@@ -568,6 +593,7 @@ int launch_prefill_attn_tc5x2h(const PrefillArgs &a_in, cudaStream_t s) {
   const int per_kvh = (a.c.G / 2) * n_xtiles + (a.c.G & 1) * (a.pair_tiles ? (n_xtiles + 1) / 2 : n_xtiles);
   const int n_walks = per_kvh * a.c.Hkv;
   a.n_split = a.partials ? prefill_split_count(n_walks, std::min(sms, 192)) : 1;
+  a.n_split = (int)std::max(1LL, std::min<long long>(a.n_split, split_slots(a.C, a.c.G, a.c.Hkv) / n_walks));
   kernel<<<dim3(n_walks * a.n_split), tc5x2h::kThreads, tc5x2h::kSmemBytes, s>>>(a);
   if (a.n_split > 1) {
     if (a.c.G & 1) prefill_merge_kernel<false><<<dim3(n_walks, 2), 256, 0, s>>>(a);
