@@ -51,52 +51,112 @@ def peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while a region runs."""
+    """Samples the SM clock and the throttle reasons every 20 ms while a region runs (NVML,
+    read-only queries, from a thread of this process; nvidia-smi every 100 ms if NVML cannot be
+    loaded).  Samples carry the time they were taken, so that a part of the region can be looked
+    at by itself (`window`)."""
 
     Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
+    REASONS = ((0x8, "hw_slowdown"), (0x40, "hw_thermal_slowdown"), (0x20, "sw_thermal_slowdown"),
+               (0x4, "sw_power_cap"))
 
-    def __init__(self, index):
-        self.index, self.proc = index, None
+    def __init__(self, index, period_s=0.02):
+        self.index, self.period, self.proc, self.thread = index, period_s, None, None
+        self.samples = []          # (perf_counter time, sm MHz, [reasons])
+        self.max_mhz = None
+        self.result = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+
+    def _nvml_loop(self, nv, handle):
+        while not self._stop.is_set():
+            try:
+                mhz = nv.nvmlDeviceGetClockInfo(handle, nv.NVML_CLOCK_SM)
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(handle)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(handle)
+                self.samples.append((time.perf_counter(), float(mhz), [n for bit, n in self.REASONS if mask & bit]))
+            except Exception:
+                pass
+            self._stop.wait(self.period)
 
     def __enter__(self):
+        import threading
+        self._stop = threading.Event()
         try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
-                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            import pynvml as nv
+            nv.nvmlInit()
+            # NVML numbers devices like nvidia-smi; CUDA_VISIBLE_DEVICES may renumber CUDA's
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+            idx = self.index
+            if vis and all(v.strip().isdigit() for v in vis.split(",")) and self.index < len(vis.split(",")):
+                idx = int(vis.split(",")[self.index])
+            handle = nv.nvmlDeviceGetHandleByIndex(idx)
+            self.max_mhz = float(nv.nvmlDeviceGetMaxClockInfo(handle, nv.NVML_CLOCK_SM))
+            self.thread = threading.Thread(target=self._nvml_loop, args=(nv, handle), daemon=True)
+            self.thread.start()
         except Exception:
-            self.proc = None
+            self.thread = None
+            try:
+                self.t_start = time.perf_counter()
+                self.proc = subprocess.Popen(
+                    ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                     "--format=csv,noheader,nounits", "-lms", "100"],
+                    stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            except Exception:
+                self.proc = None
         return self
 
     def __exit__(self, *exc):
-        self.result = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
-        if not self.proc:
-            return
-        time.sleep(0.15)
-        self.proc.terminate()
-        try:
-            out, _ = self.proc.communicate(timeout=5)
-        except Exception:
-            self.proc.kill()
-            return
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in out.strip().splitlines():
-            parts = [p.strip() for p in line.split(",")]
-            if len(parts) < 6:
-                continue
+        if self.thread is not None:
+            self._stop.set()
+            self.thread.join(timeout=2)
+        elif self.proc:
+            time.sleep(0.15)
+            self.proc.terminate()
             try:
-                sm.append(float(parts[0])); mx.append(float(parts[1]))
-            except ValueError:
-                continue
-            for n, v in zip(names, parts[2:6]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
-        if sm:
-            sm.sort()
-            self.result = {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(mx), "reasons": sorted(reasons)}
+                out, _ = self.proc.communicate(timeout=5)
+            except Exception:
+                self.proc.kill()
+                out = ""
+            names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+            lines = [l for l in out.strip().splitlines() if len(l.split(",")) >= 6]
+            t_end = time.perf_counter()
+            for i, line in enumerate(lines):
+                parts = [p.strip() for p in line.split(",")]
+                try:
+                    mhz, mx = float(parts[0]), float(parts[1])
+                except ValueError:
+                    continue
+                self.max_mhz = mx
+                # nvidia-smi prints no time we can align: spread the lines evenly over the region
+                t = self.t_start + (t_end - self.t_start) * (i + 0.5) / len(lines)
+                self.samples.append((t, mhz, [n for n, v in zip(names, parts[2:6]) if v.lower().startswith("active")]))
+        self.result = self.window(None, None)
+        self.result["samples_under_load"] = len(self.samples)
+
+    def window(self, t0, t1):
+        """Median SM clock and the reasons seen among the samples taken in [t0, t1] (all if None)."""
+        sel = [x for x in self.samples if (t0 is None or x[0] >= t0) and (t1 is None or x[0] <= t1)]
+        if not sel:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": []}
+        mhz = sorted(x[1] for x in sel)
+        return {"sm_mhz": mhz[len(mhz) // 2], "sm_max_mhz": self.max_mhz,
+                "reasons": sorted({r for x in sel for r in x[2]})}
+
+
+def median(xs):
+    xs = sorted(xs)
+    n = len(xs)
+    return xs[n // 2] if n % 2 else 0.5 * (xs[n // 2 - 1] + xs[n // 2])
+
+
+def plan_repeats(first_region_s, min_total_s=2.0, min_repeats=5, max_repeats=200):
+    """How often the K-step region is timed: until at least `min_total_s` of device time has been
+    measured, never fewer than `min_repeats` regions (and never more than `max_repeats`)."""
+    need = int(math.ceil(min_total_s / max(first_region_s, 1e-9)))
+    return max(min_repeats, min(max_repeats, need))
 
 
 def max_over_ranks(x, dist=None, device=None):
@@ -209,7 +269,9 @@ def run_ours(args):
     K, Wm = args.steps, args.warmup
     e2e_steps = min(K, args.e2e_steps)
     roof_steps = min(K, 8)
-    total_steps = Wm + K + 2 * (e2e_steps + 3) + roof_steps + 3
+    # every repeat of the timed region starts from the same checkpoint, so the cache (and the
+    # per-step inputs) only have to cover ONE pass over the phases below
+    total_steps = Wm + K + 2 * (e2e_steps + 3) + roof_steps + 3 + 1
     hbm_peak, peak_kind = peaks()
 
     def barrier():
@@ -259,6 +321,9 @@ def run_ours(args):
             step_no[0] += 1
 
         def layer_calls(stream=None, events=None):
+            # the inputs were staged by torch copies on this stream, not by the library: the first
+            # launch must wait for them even in overlap mode
+            cache.spkv_note_foreign_work()
             for l in range(L):
                 cache.spkv_score_append_evict(l, preds[l], ids, xs[l], ks[l], vs[l],
                                               logits_out=logits[l], stream=stream)
@@ -291,20 +356,64 @@ def run_ours(args):
             step()
         cache.check()
         st0 = cache.spkv_cache_stats()
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        with ClockSampler(local) as clk:
-            torch.cuda.nvtx.range_push("timed_region")      # lets a profiler pick out the timed launches
-            e0.record()
+        # The timed region is exactly K steps.  It is timed R times -- until >= 2 s of device time
+        # have been measured, at least 5 times -- each time from the same state: the cache is rolled
+        # back to a checkpoint taken here (metadata + ring pages; outside the timed region), and the
+        # same inputs are replayed.  `value` is the median region.
+        ckpt = cache.spkv_cache_checkpoint()
+        step_mark = step_no[0]
+        # settle: the same region replayed untimed until the GPU has been under this load for about a
+        # second -- a B200 starts at its maximum clock and drops to what its power limit sustains
+        # within the first ~0.5 s; the repeats below then all measure the sustained state
+        settle_regions, t_settle = 0, time.perf_counter()
+        while args.settle_seconds > 0 and time.perf_counter() - t_settle < args.settle_seconds:
             for _ in range(K):
                 step()
-            e1.record()
             torch.cuda.synchronize()
-            torch.cuda.nvtx.range_pop()
-        barrier()
-        ms = max_ranks(e0.elapsed_time(e1))
+            cache.spkv_cache_rollback(ckpt)
+            step_no[0] = step_mark
+            settle_regions += 1
+        regions, marks = [], []
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        st1 = None
+        with ClockSampler(local) as clk:
+            n_rep = 1
+            r = 0
+            while r < n_rep:
+                if r > 0:
+                    cache.spkv_cache_rollback(ckpt)
+                    step_no[0] = step_mark
+                barrier()
+                t_a = time.perf_counter()
+                torch.cuda.nvtx.range_push("timed_region")      # lets a profiler pick out the timed launches
+                e0.record()
+                for _ in range(K):
+                    step()
+                e1.record()
+                torch.cuda.synchronize()
+                torch.cuda.nvtx.range_pop()
+                t_b = time.perf_counter()
+                barrier()
+                regions.append(max_ranks(e0.elapsed_time(e1)))
+                marks.append((t_a, t_b))
+                if r == 0:
+                    st1 = cache.spkv_cache_stats()
+                    n_rep = int(max_ranks(plan_repeats(regions[0] * 1e-3)))
+                r += 1
+        ms = median(regions)
+        per_rep_clock = [clk.window(a, b)["sm_mhz"] for a, b in marks]
+        repeats = {"n": len(regions), "min": min(regions) / K, "median": ms / K, "max": max(regions) / K,
+                   "unit": "ms_per_step", "spread": (max(regions) - min(regions)) / ms,
+                   "timed_device_s": sum(regions) * 1e-3,
+                   "ms_per_step_each": [round(x / K, 5) for x in regions],
+                   "sm_mhz_each": per_rep_clock,
+                   # region time x median SM clock: flat if a slow repeat is a clock dip, not if it is contention
+                   "ms_x_ghz_each": [round(x / K * c * 1e-3, 5) if c else None for x, c in zip(regions, per_rep_clock)],
+                   "settle": {"seconds": args.settle_seconds, "untimed_regions": settle_regions},
+                   "how": "each repeat = the same K steps replayed from a checkpoint of the cache "
+                          "(spkv_cache_rollback, outside the timed region); value = median; before the first "
+                          "repeat the region is replayed untimed until the clocks have settled under load"}
         cache.check()
-        st1 = cache.spkv_cache_stats()
 
         # decode-kernel duration, measured with events around every launch (no graph)
         evs = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
@@ -324,7 +433,9 @@ def run_ours(args):
 
         scale_l = L_full / L          # > 1 only for a dense run on a layer subset
         ms *= scale_l
-        res = dict(layers_measured=L, ms_per_step=ms / K, tokens_per_s=world * B * K / (ms * 1e-3),
+        for k_ in ("min", "median", "max"):
+            repeats[k_] *= scale_l
+        res = dict(layers_measured=L, ms_per_step=ms / K, tokens_per_s=world * B * K / (ms * 1e-3), repeats=repeats,
                    kv_gb_per_step=scale_l * 0.5 * (st0.bytes_resident + st1.bytes_resident) / 1e9,
                    density=st1.density_cache, launch_bytes=launch_bytes, launch_s=launch_s,
                    clocks=clk.result, graph=graph is not None)
@@ -408,7 +519,7 @@ def run_ours(args):
                    "l2": "inputs larger than L2 (K/V read per step >> 126 MB)" if sp["kv_gb_per_step"] > 0.5
                          else "working set smaller than L2: latency-bound case",
                    "cuda_graph": sp["graph"], "launch_overlap": "SPKV_FLAG_OVERLAP", "parallelism": "replicas only" if world > 1 else "single GPU"},
-        "clocks": sp["clocks"],
+        "clocks": sp["clocks"], "repeats": sp["repeats"],
         "gpu_launches": 2 * L * K,
         # In overlap mode consecutive decode launches run under each other's head and tail, so a
         # launch has no duration of its own inside the timed region: `achieved` is the algorithmic
@@ -517,12 +628,16 @@ def run_config4(args):
         pre_ms = sum(a.elapsed_time(b) for a, b, _ in timers)
         dec_ms = sum(b.elapsed_time(c_) for _, b, c_ in timers)
         st1 = cache.spkv_cache_stats()
-        # useful prefill flops: visible keys per (query, head) = kept before + kept inside the chunk so far + window
+        # Useful prefill flops from the REALISED cache lengths.  A query sees the kept pairs of its unit
+        # with position <= t - w, plus the w pairs of its window.  Over the timed region a unit's K * C
+        # queries all see the n0 pairs kept before it, and a pair kept during it (n1 - n0 of them, from
+        # the lengths read before and after) is seen by the queries that come at least w later -- half
+        # of the region's queries on average, the gates being independent of position.
+        lens1 = [cache.spkv_read_lengths(l)[0][:NP].astype(np.int64) for l in range(L)]
         keys = 0.0
         for l in range(L):
-            for kk in range(K):
-                kept_before = lens0[l].sum(axis=0) + kk * NP * rates[l] * C      # [Hkv], summed over the 8 sequences
-                keys += float(((kept_before + NP * (rates[l] * C / 2 + W)) * (Hq // Hkv) * C).sum())
+            n0, n1 = lens0[l].astype(np.float64), lens1[l].astype(np.float64)          # [NP, Hkv]
+            keys += float(((n0 + 0.5 * (n1 - n0) + W) * (K * C) * (Hq // Hkv)).sum())
         # decode bytes: kept + window pairs of the 56 decoding sequences (their share of the resident bytes)
         lens_all = np.stack([cache.spkv_read_lengths(l)[0] for l in range(L)]).astype(np.int64)   # [L, B, Hkv]
         dec_bytes = float((lens_all[:, NP:].sum() + L * nd * Hkv * W) * 512 + L * nd * Hq * 512)
@@ -614,9 +729,12 @@ def cpu_baseline(cfg, budget_s=20.0, steps=None):
         t_used += time.perf_counter() - t0
         done += 1
     per_step_full = (t_used / done) * (L * B * Hkv / n)
+    kept = sum(len(u) for u in units)
+    density = kept / max(1, sum(max(Tb + done - W, 0) for _ in units))
     return {"value": B / per_step_full, "unit": "tokens/s", "cores": oracle.threads(), "kind": "oracle",
-            "sample": f"{n} units ({n_seq} sequences x {Hkv} KV heads of one layer, context {T}), "
+            "sample": f"{n} units ({n_seq} sequences x {Hkv} KV heads of layer 0, context {T}), "
                       f"{done} decode steps (append + attend), scaled by units to {L} layers x batch {B}",
+            "sample_density": density, "sample_kept_pairs": kept,
             "seconds": t_used}
 
 
@@ -637,10 +755,21 @@ def run_reference(args):
         "data": "synthetic",
         "config": {"workload": cfg["name"], "layers": L, "batch": B, "context": cfg["T"], "window": W,
                    "tau": TAU},
-        "cpu_baseline": {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")},
+        "cpu_baseline": {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample", "sample_density")},
         "e2e": {"value": cb["value"], "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line))
+
+
+def replica_launch_command(n, argv, port=None):
+    """The torchrun command line that runs this script as `n` replicas on one node."""
+    if port is None:
+        import socket
+        with socket.socket() as sock:
+            sock.bind(("127.0.0.1", 0))
+            port = sock.getsockname()[1]
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n),
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *argv]
 
 
 def main():
@@ -657,9 +786,15 @@ def main():
     ap.add_argument("--layers", type=int, default=0,
                     help="override the layer count (small profiling captures only; not a bench line)")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--settle-seconds", type=float, default=1.0,
+                    help="untimed replay of the timed region before the first repeat (clocks settle under load)")
     ap.add_argument("--sweep-tau", default="",
                     help="comma-separated thresholds: one decode measurement per tau, nothing else")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # replicas only: N independent copies of the workload, one process per GPU; started here
+        # the way a launcher would start them
+        sys.exit(subprocess.call(replica_launch_command(args.gpus, sys.argv[1:])))
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     if args.impl == "reference":

@@ -57,8 +57,14 @@ enum {
   SPKV_E_SCRATCH_LIMIT = -10,   /* request larger than the library's built-in scratch  */
   SPKV_E_ORDER_DECODE = -11,    /* device, overlap mode: a decode launch gave up waiting for the
                                    appends of its layer / the previous user of its workspace */
-  SPKV_E_ORDER_APPEND = -12     /* device, overlap mode: an append gave up waiting for the decode
+  SPKV_E_ORDER_APPEND = -12,    /* device, overlap mode: an append gave up waiting for the decode
                                    launches of its layer                                  */
+  SPKV_E_BOUNDS_PAGE = -13,     /* device, SPKV_FLAG_DEBUG_BOUNDS: a page index read from a page
+                                   table or the free stack names no pool page; the access was
+                                   skipped or redirected to a page of the unit's own          */
+  SPKV_E_CANARY = -14,          /* SPKV_FLAG_DEBUG_BOUNDS: a canary block between two regions of
+                                   the arena no longer holds its pattern                      */
+  SPKV_E_ATTACH = -15           /* spkv_cache_attach: no cache of this configuration in the arena */
 };
 
 typedef struct {
@@ -72,7 +78,7 @@ typedef struct {
   int32_t max_context;  /* upper bound on kept pairs per unit (sizes the page tables)   */
   int64_t pool_pages;   /* pages shared by all compact caches                           */
   float tau;            /* utility threshold in [0,1]; <= 0 keeps all, >= 1 keeps none  */
-  int32_t flags;        /* 0 or SPKV_FLAG_OVERLAP                                       */
+  int32_t flags;        /* 0 or an OR of SPKV_FLAG_* (below)                            */
   int32_t sink_tokens;  /* >= 0: the first sink_tokens positions of every sequence are
                            kept in the compact cache whatever their utility (the paper's
                            "Fixed Attention Sinks" ablation; its evaluation protocol uses
@@ -96,6 +102,22 @@ typedef struct {
  * earlier work, as any stream-ordered kernel does).  Any other call of the library (prefill,
  * score, reset, ...) is a full synchronisation point either way. */
 #define SPKV_FLAG_OVERLAP 1
+
+/* SPKV_FLAG_PREFILL_PV_BF16 (off by default): the chunk attention of spkv_prefill multiplies the
+ * softmax weights into the values as two bf16 terms (16 significant bits, bf16's exponent range)
+ * for every unit.  By default it uses one fp16 term (11 bits) on values rescaled by a power of
+ * two -- a third less tensor-core work -- and switches a unit to the two-term form by itself when
+ * the largest |value| its queries can see is 2^20 or more (see spkv_prefill).  Set the flag when
+ * the extra five bits matter more than the speed. */
+#define SPKV_FLAG_PREFILL_PV_BF16 2
+
+/* SPKV_FLAG_DEBUG_BOUNDS (off by default; a debugging aid for integrations, since memory checkers
+ * are not always available): every page index a kernel reads from a page table or from the free
+ * stack is checked against the pool's range before it is used; a violation sets the sticky status
+ * SPKV_E_BOUNDS_PAGE and the access is skipped (writes) or redirected to a page of the unit's own
+ * (reads), so that nothing outside the arena is touched.  spkv_status additionally verifies the
+ * 256-byte canary blocks that separate the metadata regions of the arena (SPKV_E_CANARY). */
+#define SPKV_FLAG_DEBUG_BOUNDS 4
 
 /* Utility predictor f of Eq. 1 (the sigmoid is never evaluated: the decision is taken
  * in logit space, u >= tau  <=>  logit >= log(tau/(1-tau))).
@@ -143,6 +165,52 @@ int spkv_arena_bytes(const spkv_config_t *cfg, size_t *out_bytes);
  * window kept by metadata); here the capacity is fixed at creation instead of grown. */
 int spkv_cache_create(const spkv_config_t *cfg, void *d_arena, size_t arena_bytes,
                       spkv_stream_t stream, spkv_cache_t **out);
+
+/* Snapshot / resume.  The arena is position-independent (it holds offsets and page indices, no
+ * pointers), so a snapshot of a cache is a plain copy of its arena made by the caller (device to
+ * device, to the host, to a file), and a copy placed in device memory again -- at any 256-byte
+ * aligned address, in this or a later process -- becomes a cache by attaching to it.
+ * spkv_cache_attach checks the header cache_create wrote (magic, layout version, a hash of every
+ * configuration field that fixes the layout; tau and flags may differ and take effect as given)
+ * and returns a handle without initialising anything; SPKV_E_ATTACH if the header does not
+ * match.  Synchronises `stream`.  Two handles on one arena must not be used at the same time. */
+int spkv_cache_attach(const spkv_config_t *cfg, void *d_arena, size_t arena_bytes,
+                      spkv_stream_t stream, spkv_cache_t **out);
+
+/* Checkpoint / rollback of a live cache without copying its pool: saves (restores) the metadata
+ * and the ring pages -- everything appends and prefill chunks change IN PLACE; the pairs they add
+ * to the pool land behind the saved lengths and are simply forgotten by a rollback.  Valid as long
+ * as no spkv_cache_reset_seq came between the two (it hands pages to other units).  Use: replaying
+ * the same decode steps (benchmark repeats, speculative tokens that were rejected).
+ *   d_buf: device, >= spkv_cache_checkpoint_bytes(cache) bytes.  Asynchronous on `stream`; a full
+ *   synchronisation point for SPKV_FLAG_OVERLAP. */
+size_t spkv_cache_checkpoint_bytes(const spkv_cache_t *cache);
+int spkv_cache_checkpoint(spkv_cache_t *cache, void *d_buf, size_t bytes, spkv_stream_t stream);
+int spkv_cache_rollback(spkv_cache_t *cache, const void *d_buf, size_t bytes, spkv_stream_t stream);
+
+/* SPKV_FLAG_OVERLAP only: tells the cache that work it did not launch (a copy, another library's
+ * kernel) was enqueued on the stream after its previous call and produces inputs of its next one.
+ * The next hot-path launch then waits for everything earlier on the stream, as it does after any
+ * other call of the library.  Call it before a step whose inputs were staged on the same stream,
+ * and before capturing a CUDA graph of a step. */
+int spkv_note_foreign_work(spkv_cache_t *cache);
+
+/* Safe-step budget (paper, Appendix "Inference Kernels": capacity checks are amortised by a budget
+ * of steps that cannot exhaust the headroom).  The number of further decode steps the listed
+ * sequences can take, all layers and KV heads, before a page-table or pool limit COULD be hit,
+ * assuming the worst case that every pair leaving a window is kept.  While the answer is n > 0
+ * the next n steps cannot raise SPKV_E_POOL_EXHAUSTED / SPKV_E_CONTEXT_OVERFLOW (other sequences
+ * sharing the pool must be counted in by listing them).  h_seq_ids: HOST array of B ids, B = 0 =
+ * every sequence.  Synchronises `stream`.  spkv_safe_steps_from_lengths is the arithmetic alone
+ * (host only): h_len / h_t [n_units] kept pairs / pairs received of the units to count. */
+int spkv_safe_steps(spkv_cache_t *cache, const int32_t *h_seq_ids, int32_t B, spkv_stream_t stream,
+                    int64_t *out_steps);
+int spkv_safe_steps_from_lengths(const spkv_config_t *cfg, const int32_t *h_len, const int32_t *h_t,
+                                 int64_t n_units, int64_t pages_free, int64_t *out_steps);
+
+/* Byte offsets of the arena's canary blocks (256 bytes of 0xC5 each, one after every metadata
+ * region), for tools that want to verify them themselves.  Host only; *n_out = their number. */
+int spkv_arena_canaries(const spkv_config_t *cfg, size_t *h_offsets, int32_t cap, int32_t *n_out);
 
 /* Frees the host handle only (the arena belongs to the caller). */
 int spkv_cache_destroy(spkv_cache_t *cache);
@@ -241,7 +309,11 @@ int spkv_decode_attention_f32(spkv_cache_t *cache, int32_t layer, const int32_t 
  *   - All calls on a device share the one array and it keeps the previous call's contents;
  *     the entry point clears the part that must start at zero on `stream` before the
  *     kernel.  Two calls whose GPU work overlaps (different streams, no dependency) race on
- *     it: keep such calls ordered. */
+ *     it: keep such calls ordered.  A call that is refused (any error code) has not touched
+ *     the array.
+ *   - That clearing is an ordinary stream operation, so in SPKV_FLAG_OVERLAP mode a launch made
+ *     through this entry point starts only after everything earlier on `stream` has finished
+ *     (it never runs under the tail of the previous decode launch). */
 #define SPKV_STATIC_SCRATCH_BYTES (6u << 20)
 int spkv_decode_attention_static(spkv_cache_t *cache, int32_t layer, const int32_t *d_seq_ids,
                                  int32_t B, const void *d_q, void *d_out, float *d_lse_opt,
@@ -256,7 +328,14 @@ size_t spkv_prefill_workspace_bytes(const spkv_config_t *cfg, int32_t C);
  * that leave the window (ballot + prefix sum, ascending position), tensor-core attention
  * of every query of the chunk over compact cache U window (Eq. 3-5), ring update.
  *   d_q [C, n_q_heads, 128], d_k/d_v [C, n_kv_heads, 128] bf16, d_logits [C, n_kv_heads],
- *   d_out [C, n_q_heads, 128] bf16.  d_q = d_out = NULL builds the cache state only. */
+ *   d_out [C, n_q_heads, 128] bf16.  d_q = d_out = NULL builds the cache state only.
+ *   With queries, sm_scale must be positive and finite (SPKV_E_INVALID otherwise).
+ * Precision of the weights-times-values product: one fp16 term on values rescaled by a power
+ * of two taken from the largest finite |value| the chunk's queries can see (compact cache,
+ * window, chunk); exact for every value within 2^28 of that maximum, off by at most 2^-39 of
+ * it below; a weight below 2^-32 of its row's running maximum is dropped.  A unit where that
+ * largest |value| reaches 2^20 -- and every unit under SPKV_FLAG_PREFILL_PV_BF16 -- takes two
+ * bf16 terms on the unscaled values instead (no scaling, no dropped weights). */
 int spkv_prefill(spkv_cache_t *cache, int32_t layer, int32_t seq, int32_t C, const void *d_q,
                  const void *d_k, const void *d_v, const float *d_logits, void *d_out,
                  float sm_scale, void *d_workspace, size_t workspace_bytes,
@@ -341,6 +420,17 @@ const char *spkv_error_string(int code);
  *   d_status: device, one int32, set to SPKV_E_TIMEOUT if a bounded wait ran out.  Asynchronous. */
 int spkv_stream_read(const void *d_buf, size_t bytes, unsigned long long *d_sink, int32_t *d_status,
                      spkv_stream_t stream);
+
+/* Self-test of the library's bounded device waits (no counterpart in the paper).  Every copy
+ * pipeline of the library waits on its copies with a clock limit; when a wait runs out the kernel
+ * records SPKV_E_TIMEOUT, stops issuing, waits (bounded) for the copies it still has in flight and
+ * returns -- the context stays usable.  This call runs that error path on purpose and harmlessly:
+ * one thread arms a barrier for 64 bytes more than the single 32 KB copy it issues delivers, waits
+ * `limit_clocks` cycles, and then drains as described.
+ *   d_buf: device, 16-byte aligned, >= 32 KB readable; d_status: device, four int32:
+ *   [0] SPKV_E_TIMEOUT (the wait ran out, as it must), [1] 1 = the copy in flight was waited for,
+ *   [2] clocks the first wait lasted, [3] 1 = the copied data is in place.  Asynchronous. */
+int spkv_wait_selftest(const void *d_buf, long long limit_clocks, int32_t *d_status, spkv_stream_t stream);
 
 #ifdef __cplusplus
 }

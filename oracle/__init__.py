@@ -75,6 +75,14 @@ def lib():
         l.orcB_attend_all.argtypes = [_u16p, _u16p, _f32p, C.c_int, C.c_int, C.c_float, _u16p,
                                       C.c_int, C.c_int, C.c_double, _f64p]
         l.orcB_density.restype = None
+        l.orc_gate_log_bias.argtypes = [C.c_float, C.c_double, C.c_float]
+        l.orc_gate_log_bias.restype = C.c_double
+        l.orcB_attend_row_soft.argtypes = [_u16p, _u16p, _f32p, C.c_int, C.c_int, C.c_int, C.c_double, C.c_float,
+                                           _u16p, C.c_int, C.c_int, C.c_double, _f64p, C.c_void_p]
+        l.orcB_attend_row_soft.restype = None
+        l.orcB_attend_all_soft.argtypes = [_u16p, _u16p, _f32p, C.c_int, C.c_int, C.c_double, C.c_float, _u16p,
+                                           C.c_int, C.c_int, C.c_double, _f64p, C.c_void_p]
+        l.orcB_attend_all_soft.restype = None
         l.orcB_density.argtypes = [_f32p, C.c_int, C.c_int, C.c_float, C.POINTER(C.c_double),
                                    C.POINTER(C.c_double)]
         l.orcA_new.restype = C.c_void_p
@@ -178,6 +186,36 @@ def mask_attend_all(K, V, logit, w, tau_l, q, scale, n_sink=0):
     lib().orcB_attend_all_sinks(K, V, logit, T, int(w), float(tau_l), int(n_sink), q, G, D,
                                 float(scale), out)
     return out
+
+
+def gate_log_bias(logit, alpha=0.0, tau_l=0.0) -> float:
+    """log of the (annealed) gate of one position: Eq. 6 with the gate of Eq. 7."""
+    return float(lib().orc_gate_log_bias(float(np.float32(logit)), float(alpha), float(tau_l)))
+
+
+def soft_attend_row(K, V, logit, t, w, q, scale, alpha=0.0, tau_l=0.0, want_lse=False):
+    """Soft-gated forward (Eq. 6; alpha > 0: the annealed gate of Eq. 7), one query position t.
+    K,V [T,D]; q [G,D] -> [G,D]."""
+    K, V, q, logit = _u16(K), _u16(V), _u16(q), _f32(logit)
+    T, D = K.shape
+    G = q.shape[0]
+    out = np.empty((G, D), np.float64)
+    lse = np.empty(G, np.float64)
+    lib().orcB_attend_row_soft(K, V, logit, T, int(t), int(w), float(alpha), float(tau_l), q, G, D,
+                               float(scale), out, lse.ctypes.data)
+    return (out, lse) if want_lse else out
+
+
+def soft_attend_all(K, V, logit, w, q, scale, alpha=0.0, tau_l=0.0, want_lse=False):
+    """Soft-gated forward for every position.  q [T,G,D] -> [T,G,D] (O(T^2))."""
+    K, V, q, logit = _u16(K), _u16(V), _u16(q), _f32(logit)
+    T, D = K.shape
+    G = q.shape[1]
+    out = np.empty((T, G, D), np.float64)
+    lse = np.empty((T, G), np.float64)
+    lib().orcB_attend_all_soft(K, V, logit, T, int(w), float(alpha), float(tau_l), q, G, D, float(scale),
+                               out, lse.ctypes.data)
+    return (out, lse) if want_lse else out
 
 
 def density(logit, w, tau_l):

@@ -6,7 +6,8 @@
  * library; it shares no code with it and nothing in the product path may call
  * it.  Only tests, the smoke check and the benchmark's CPU-baseline leg use it.
  *
- * Two independent formulations of the same definition live here:
+ * Two independent formulations of the same definition live here (and, after them, the
+ * soft-gated whole-sequence forward of the paper's training section, Eq. 6-7):
  *
  *   "mask form"      (orcB_*)  Eq. 2-5 of the paper written out literally:
  *                    threshold every position, build the additive bias
@@ -168,6 +169,72 @@ void orcB_attend_all(const uint16_t *K, const uint16_t *V, const float *logit, i
                      int w, float tau_logit, const uint16_t *q /*[T][G][D]*/, int G, int D,
                      double scale, double *out /*[T][G][D]*/) {
   orcB_attend_all_sinks(K, V, logit, T, w, tau_logit, 0, q, G, D, scale, out);
+}
+
+/* ------------------------------ soft-gated forward (Eq. 6 and Eq. 7: the training-time form) */
+
+/*
+ * Gate of one position.  u = sigma(logit) (Eq. 1).  During the annealed switch to hard gating the
+ * paper interpolates u~ = (1 - alpha) u + alpha 1[u >= tau] (Eq. 7): alpha = 0 is soft gating,
+ * alpha = 1 the binary gate.  The threshold is applied as everywhere else, on the float32 logit.
+ * Returns the additive bias log u~ (Eq. 6 with u~ for u); -inf when u~ = 0.
+ * For alpha = 0 the logarithm of the sigmoid is taken without forming the sigmoid:
+ * log sigma(l) = -log(1 + e^-l), finite for every finite l.  (The epsilon the paper's listing
+ * adds inside the logarithm is a guard for gradients; it is not part of Eq. 6 and not here.)
+ */
+double orc_gate_log_bias(float logit, double alpha, float tau_logit) {
+  double l = (double)logit;
+  if (alpha == 0.0) return l >= 0.0 ? -log1p(exp(-l)) : l - log1p(exp(l));
+  double u = orc_sigmoid(l);
+  double z = (logit >= tau_logit) ? 1.0 : 0.0;                 /* Eq. 2 */
+  double u_tilde = (1.0 - alpha) * u + alpha * z;              /* Eq. 7 */
+  return log(u_tilde);                                         /* log(0) = -inf */
+}
+
+/*
+ * Soft-gated attention for one query position t of one KV head over the whole sequence:
+ * the bias of Eq. 4 with the binary gate replaced by log u~_s (Eq. 6).  Three regions of a row:
+ * the window 0 <= t - s < w has bias 0 whatever the gate; an earlier position has bias
+ * log u~_s; a future position -inf.  Arguments as orcB_attend_row; alpha as above.
+ */
+void orcB_attend_row_soft(const uint16_t *K, const uint16_t *V, const float *logit, int T,
+                          int t, int w, double alpha, float tau_logit, const uint16_t *q, int G,
+                          int D, double scale, double *out, double *lse) {
+  double *a = (double *)malloc(sizeof(double) * (size_t)T);   /* biased, scaled scores of the row */
+  for (int g = 0; g < G; ++g) {
+    const uint16_t *qg = q + (size_t)g * D;
+    double top = -INFINITY;
+    for (int s = 0; s < T; ++s) {
+      double bias_ts;
+      if (s > t) bias_ts = -INFINITY;                                      /* future          */
+      else if (t - s < w) bias_ts = 0.0;                                   /* sliding window  */
+      else bias_ts = orc_gate_log_bias(logit[s], alpha, tau_logit);        /* long range: log u~_s */
+      double qk = 0.0;
+      for (int i = 0; i < D; ++i) qk += bf16_widen(qg[i]) * bf16_widen(K[(size_t)s * D + i]);
+      a[s] = qk * scale + bias_ts;
+      if (a[s] > top) top = a[s];
+    }
+    double z_row = 0.0;
+    for (int s = 0; s < T; ++s) z_row += exp(a[s] - top);
+    for (int i = 0; i < D; ++i) out[(size_t)g * D + i] = 0.0;
+    for (int s = 0; s < T; ++s) {
+      double weight = exp(a[s] - top) / z_row;
+      if (weight == 0.0) continue;
+      for (int i = 0; i < D; ++i) out[(size_t)g * D + i] += weight * bf16_widen(V[(size_t)s * D + i]);
+    }
+    if (lse) lse[g] = top + log(z_row);
+  }
+  free(a);
+}
+
+/* Soft-gated forward for every position (O(T^2)), rows in parallel. */
+void orcB_attend_all_soft(const uint16_t *K, const uint16_t *V, const float *logit, int T, int w,
+                          double alpha, float tau_logit, const uint16_t *q /*[T][G][D]*/, int G,
+                          int D, double scale, double *out /*[T][G][D]*/, double *lse /*[T][G] or NULL*/) {
+#pragma omp parallel for schedule(dynamic, 8)
+  for (int t = 0; t < T; ++t)
+    orcB_attend_row_soft(K, V, logit, T, t, w, alpha, tau_logit, q + (size_t)t * G * D, G, D, scale,
+                         out + (size_t)t * G * D, lse ? lse + (size_t)t * G : NULL);
 }
 
 /* Eq. 8 gate density over one (layer, head): mean of z over all T positions,

@@ -12,7 +12,8 @@ namespace spkv {
 
 // Pops a free page (lane 0) and clears its value block, so that rows past a page's
 // valid count always hold zeros (the attention kernels multiply them by weight 0).
-// Returns the global page index or -1.
+// Returns the global page index, -1 when the pool is empty, -2 when the index popped from the stack
+// failed the debug bounds check (status set already).
 __device__ inline int alloc_page(const CacheView &c, int lane) {
   int page = -1;
   if (lane == 0) {
@@ -20,7 +21,7 @@ __device__ inline int alloc_page(const CacheView &c, int lane) {
     if (top <= 0) {
       atomicAdd(&c.status[1], 1);
     } else {
-      page = __ldcg(&c.free_stack[top - 1]);
+      page = checked_page(c, __ldcg(&c.free_stack[top - 1]), -2);
     }
   }
   page = __shfl_sync(0xffffffffu, page, 0);
@@ -78,30 +79,33 @@ __device__ inline void append_unit(const CacheView &c, int layer, const int32_t 
         err = SPKV_E_CONTEXT_OVERFLOW;
       } else if (prow == 0) {
         page = alloc_page(c, lane);
-        if (page < 0) err = SPKV_E_POOL_EXHAUSTED;
+        if (page == -1) err = SPKV_E_POOL_EXHAUSTED;
+        else if (page < 0) err = SPKV_E_BOUNDS_PAGE;
         else if (lane == 0) c.table[(size_t)u * c.max_pages + pj] = page;
       } else {
-        page = __ldcg(&c.table[(size_t)u * c.max_pages + pj]);
+        page = checked_page(c, __ldcg(&c.table[(size_t)u * c.max_pages + pj]), -2);
+        if (page < 0) err = SPKV_E_BOUNDS_PAGE;   // the evicted pair is dropped, as on exhaustion
       }
       if (err) {
         if (lane == 0) set_status(c, err);
       } else {
         __syncwarp();
         __nv_bfloat16 *dst = c.pages + (int64_t)page * kPageElems;
-        *reinterpret_cast<uint4 *>(dst + blk + swz_off(prow, chunk)) = __ldcg(ring_cell);
+        const uint4 kept = __ldcg(ring_cell);
+        *reinterpret_cast<uint4 *>(dst + blk + swz_off(prow, chunk)) = kept;
+        // the compact cache's largest |value| (the prefill attention picks its value scale by it)
+        const uint32_t vm = __reduce_max_sync(0xffffffffu, lane < 16 ? 0u : chunk_abs_max_bf16(kept));
         if (lane == 0) {
           c.pos_pool[((int64_t)page - c.n_ring_pages_total) * kP + prow] = t - c.w;
           c.len[u] = n + 1;
+          note_vmax(c, u, vm);
         }
       }
     }
   }
   const uint4 *src = (lane < 16 ? k_new : v_new) + (size_t)item * 16 + chunk;
-  const uint4 cell = *src;
-  *ring_cell = cell;
-  const uint32_t vm = __reduce_max_sync(0xffffffffu, lane < 16 ? 0u : chunk_abs_max_bf16(cell));
+  *ring_cell = *src;
   if (lane == 0) {
-    note_vmax(c, u, vm);
     c.ring_logit[(size_t)u * c.w + slot] = new_logit;
     c.t[u] = t + 1;
   }

@@ -3,6 +3,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <algorithm>
 #include <new>
 #include <vector>
 
@@ -41,20 +42,43 @@ static void make_layout(const spkv_config_t *c, Layout *l) {
   size_t ring_pages = (c->window + kP - 1) / kP;
   size_t max_pages = ((size_t)c->max_context + kP - 1) / kP;
   size_t o = 0;
-  l->off_header = o; o = align_up(o + 256, 256);
-  l->off_t = o;      o = align_up(o + units * 4, 256);
-  l->off_len = o;    o = align_up(o + units * 4, 256);
-  l->off_table = o;  o = align_up(o + units * max_pages * 4, 256);
-  l->off_free = o;   o = align_up(o + (size_t)c->pool_pages * 4, 256);
-  l->off_pos = o;    o = align_up(o + (size_t)c->pool_pages * kP * 4, 256);
-  l->off_rlogit = o; o = align_up(o + units * (size_t)c->window * 4, 256);
-  l->off_htau = o;   o = align_up(o + (size_t)c->n_layers * c->n_kv_heads * 4, 256);
-  l->off_sync = o;   o = align_up(o + (size_t)c->n_layers * 4 * 8, 256);
-  l->off_vmax = o;   o = align_up(o + units * 4, 256);
+  int n_can = 0;
+  // a region of `bytes` bytes at the current offset, followed by its canary block
+  auto region = [&](size_t bytes) {
+    const size_t at = o;
+    o = align_up(o + bytes, 256);
+    l->canary[n_can++] = o;
+    o += kCanaryBytes;
+    return at;
+  };
+  l->off_header = region(256);
+  l->off_t = region(units * 4);
+  l->off_len = region(units * 4);
+  l->off_table = region(units * max_pages * 4);
+  l->off_free = region((size_t)c->pool_pages * 4);
+  l->off_pos = region((size_t)c->pool_pages * kP * 4);
+  l->off_rlogit = region(units * (size_t)c->window * 4);
+  l->off_htau = region((size_t)c->n_layers * c->n_kv_heads * 4);
+  l->off_sync = region((size_t)c->n_layers * 4 * 8);
+  l->off_vmax = region(units * 4);
   o = align_up(o, 1024);
   l->off_pages = o;  o += (units * ring_pages + (size_t)c->pool_pages) * kPageBytes;
   l->total = o;
 }
+
+// What an arena must agree on with a configuration to be attached to: everything that fixes the
+// layout (FNV-1a over the fields; tau and flags are run-time settings and may differ).
+static uint64_t layout_hash(const spkv_config_t *c) {
+  const int64_t f[] = {c->n_layers, c->max_seqs, c->n_q_heads, c->n_kv_heads, c->head_dim, c->window,
+                       c->page_tokens, c->max_context, c->pool_pages, c->sink_tokens};
+  uint64_t h = 1469598103934665603ULL;
+  for (int64_t v : f)
+    for (int b = 0; b < 8; ++b) { h ^= (uint64_t)(v >> (8 * b)) & 0xff; h *= 1099511628211ULL; }
+  return h;
+}
+constexpr uint32_t kMagic = 0x564B5053u;   // "SPKV"
+constexpr uint32_t kLayoutVersion = 2;
+constexpr int kHdrMagicWord = 8;            // int32 index of {magic, version, hash lo, hash hi} in the header
 
 // value = NaN clears the override
 __global__ void set_head_tau_kernel(float *head_tau, int first, int count, float value) {
@@ -102,14 +126,8 @@ extern "C" int spkv_arena_bytes(const spkv_config_t *cfg, size_t *out_bytes) {
   return SPKV_OK;
 }
 
-extern "C" int spkv_cache_create(const spkv_config_t *cfg, void *d_arena, size_t arena_bytes,
-                                 spkv_stream_t stream, spkv_cache_t **out) {
-  int rc = validate(cfg);
-  if (rc) return rc;
-  if (!d_arena || !out || ((uintptr_t)d_arena & 255)) return SPKV_E_INVALID;
-  Layout l;
-  make_layout(cfg, &l);
-  if (arena_bytes < l.total) return SPKV_E_ARENA_TOO_SMALL;
+// Host handle over an arena laid out for `cfg` (nothing is enqueued).
+static int make_handle(const spkv_config_t *cfg, void *d_arena, const Layout &l, spkv_cache **out) {
   spkv_cache *c = new (std::nothrow) spkv_cache();
   if (!c) return SPKV_E_INVALID;
   c->cfg = *cfg;
@@ -134,6 +152,7 @@ extern "C" int spkv_cache_create(const spkv_config_t *cfg, void *d_arena, size_t
   v.G = cfg->n_q_heads / cfg->n_kv_heads;
   v.w = cfg->window;
   v.n_sink = cfg->sink_tokens;
+  v.debug_bounds = (cfg->flags & SPKV_FLAG_DEBUG_BOUNDS) ? 1 : 0;
   v.ring_pages = (cfg->window + kP - 1) / kP;
   v.max_pages = (cfg->max_context + kP - 1) / kP;
   v.n_units = cfg->n_layers * cfg->max_seqs * cfg->n_kv_heads;
@@ -150,7 +169,6 @@ extern "C" int spkv_cache_create(const spkv_config_t *cfg, void *d_arena, size_t
   v.sync_ctr = reinterpret_cast<unsigned long long *>(base + l.off_sync);
   v.vmax = reinterpret_cast<uint32_t *>(base + l.off_vmax);
   v.pages = reinterpret_cast<__nv_bfloat16 *>(base + l.off_pages);
-
   int dev = 0;
   cudaDeviceProp prop;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
@@ -159,17 +177,41 @@ extern "C" int spkv_cache_create(const spkv_config_t *cfg, void *d_arena, size_t
     return SPKV_E_CUDA;
   }
   c->sm_count = prop.multiProcessorCount;
+  *out = c;
+  return SPKV_OK;
+}
 
+extern "C" int spkv_cache_create(const spkv_config_t *cfg, void *d_arena, size_t arena_bytes,
+                                 spkv_stream_t stream, spkv_cache_t **out) {
+  int rc = validate(cfg);
+  if (rc) return rc;
+  if (!d_arena || !out || ((uintptr_t)d_arena & 255)) return SPKV_E_INVALID;
+  Layout l;
+  make_layout(cfg, &l);
+  if (arena_bytes < l.total) return SPKV_E_ARENA_TOO_SMALL;
+  spkv_cache *c = nullptr;
+  rc = make_handle(cfg, d_arena, l, &c);
+  if (rc) return rc;
+  char *base = static_cast<char *>(d_arena);
+  const CacheView &v = c->view;
   cudaStream_t s = as_stream(stream);
   // metadata and ring pages start at zero; pool pages are zeroed when first allocated
   cudaError_t e = cudaMemsetAsync(base, 0, l.off_pages + (size_t)v.n_ring_pages_total * kPageBytes, s);
+  for (int i = 0; i < kCanaries && e == cudaSuccess; ++i)
+    e = cudaMemsetAsync(base + l.canary[i], kCanaryByte, kCanaryBytes, s);
+  if (e == cudaSuccess) {
+    // what spkv_cache_attach recognises the arena by (pageable host source: copied before the call returns)
+    const uint64_t h = layout_hash(cfg);
+    const uint32_t id[4] = {kMagic, kLayoutVersion, (uint32_t)h, (uint32_t)(h >> 32)};
+    e = cudaMemcpyAsync(v.status + kHdrMagicWord, id, sizeof id, cudaMemcpyHostToDevice, s);
+  }
   if (e == cudaSuccess) {
     const int nh = v.L * v.Hkv;
     set_head_tau_kernel<<<(nh + 255) / 256, 256, 0, s>>>(v.head_tau, 0, nh, NAN);
   }
   if (e == cudaSuccess && v.pool_pages > 0) {
     int64_t n = v.pool_pages;
-    init_free_stack_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(v.free_stack, &v.status[1], n,
+    init_free_stack_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(v.free_stack, &c->view.status[1], n,
                                                                       v.n_ring_pages_total);
     e = cudaGetLastError();
   }
@@ -180,6 +222,126 @@ extern "C" int spkv_cache_create(const spkv_config_t *cfg, void *d_arena, size_t
   }
   *out = c;
   return SPKV_OK;
+}
+
+extern "C" int spkv_cache_attach(const spkv_config_t *cfg, void *d_arena, size_t arena_bytes,
+                                 spkv_stream_t stream, spkv_cache_t **out) {
+  int rc = validate(cfg);
+  if (rc) return rc;
+  if (!d_arena || !out || ((uintptr_t)d_arena & 255)) return SPKV_E_INVALID;
+  Layout l;
+  make_layout(cfg, &l);
+  if (arena_bytes < l.total) return SPKV_E_ARENA_TOO_SMALL;
+  uint32_t id[4] = {0, 0, 0, 0};
+  if (cudaStreamSynchronize(as_stream(stream)) != cudaSuccess ||
+      cudaMemcpy(id, static_cast<char *>(d_arena) + l.off_header + kHdrMagicWord * 4, sizeof id,
+                 cudaMemcpyDeviceToHost) != cudaSuccess)
+    return SPKV_E_CUDA;
+  const uint64_t h = layout_hash(cfg);
+  if (id[0] != kMagic || id[1] != kLayoutVersion || id[2] != (uint32_t)h || id[3] != (uint32_t)(h >> 32))
+    return SPKV_E_ATTACH;
+  spkv_cache *c = nullptr;
+  rc = make_handle(cfg, d_arena, l, &c);
+  if (rc) return rc;
+  *out = c;
+  return SPKV_OK;
+}
+
+// ---- checkpoint / rollback of everything a decode or prefill call can change in place ---------
+static size_t checkpoint_bytes(const spkv_cache *c) {
+  return c->layout.off_pages + (size_t)c->view.n_ring_pages_total * kPageBytes;
+}
+extern "C" size_t spkv_cache_checkpoint_bytes(const spkv_cache_t *cache) { return cache ? checkpoint_bytes(cache) : 0; }
+
+extern "C" int spkv_cache_checkpoint(spkv_cache_t *cache, void *d_buf, size_t bytes, spkv_stream_t stream) {
+  if (!cache || !d_buf) return SPKV_E_INVALID;
+  if (bytes < checkpoint_bytes(cache)) return SPKV_E_WORKSPACE;
+  cache->last_kind = kLastOther;
+  return check_stream_error(
+      cudaMemcpyAsync(d_buf, cache->arena, checkpoint_bytes(cache), cudaMemcpyDeviceToDevice, as_stream(stream)));
+}
+
+extern "C" int spkv_cache_rollback(spkv_cache_t *cache, const void *d_buf, size_t bytes, spkv_stream_t stream) {
+  if (!cache || !d_buf) return SPKV_E_INVALID;
+  if (bytes < checkpoint_bytes(cache)) return SPKV_E_WORKSPACE;
+  cache->last_kind = kLastOther;
+  return check_stream_error(
+      cudaMemcpyAsync(cache->arena, d_buf, checkpoint_bytes(cache), cudaMemcpyDeviceToDevice, as_stream(stream)));
+}
+
+extern "C" int spkv_note_foreign_work(spkv_cache_t *cache) {
+  if (!cache) return SPKV_E_INVALID;
+  cache->last_kind = kLastOther;
+  return SPKV_OK;
+}
+
+extern "C" int spkv_arena_canaries(const spkv_config_t *cfg, size_t *h_offsets, int32_t cap, int32_t *n_out) {
+  int rc = validate(cfg);
+  if (rc) return rc;
+  Layout l;
+  make_layout(cfg, &l);
+  if (n_out) *n_out = kCanaries;
+  for (int i = 0; h_offsets && i < kCanaries && i < cap; ++i) h_offsets[i] = l.canary[i];
+  return SPKV_OK;
+}
+
+// ---- safe-step budget -----------------------------------------------------------------------
+// Worst case over n further steps: every pair that leaves a unit's window is kept.  A unit that has
+// received t pairs and keeps len then holds len + e(n) pairs, e(n) = max(t + n - w, 0) - max(t - w, 0),
+// and needs ceil((len + e(n)) / 64) - ceil(len / 64) new pages; it must also stay within its page table.
+static bool steps_fit(const spkv_config_t *cfg, const int32_t *len, const int32_t *t, int64_t n_units,
+                      int64_t pages_free, int64_t n) {
+  const int64_t w = cfg->window, max_pages = ((int64_t)cfg->max_context + kP - 1) / kP;
+  int64_t need = 0;
+  for (int64_t u = 0; u < n_units; ++u) {
+    const int64_t ev = std::max<int64_t>(t[u] + n - w, 0) - std::max<int64_t>(t[u] - w, 0);
+    const int64_t p0 = ((int64_t)len[u] + kP - 1) / kP, p1 = ((int64_t)len[u] + ev + kP - 1) / kP;
+    if (p1 > max_pages) return false;
+    need += p1 - p0;
+    if (need > pages_free) return false;
+  }
+  return true;
+}
+
+extern "C" int spkv_safe_steps_from_lengths(const spkv_config_t *cfg, const int32_t *h_len, const int32_t *h_t,
+                                            int64_t n_units, int64_t pages_free, int64_t *out_steps) {
+  int rc = validate(cfg);
+  if (rc) return rc;
+  if (!h_len || !h_t || !out_steps || n_units < 0 || pages_free < 0) return SPKV_E_INVALID;
+  int64_t lo = 0, hi = (int64_t)1 << 31;   // steps_fit(lo) holds (no step needs nothing); find the last n that fits
+  if (steps_fit(cfg, h_len, h_t, n_units, pages_free, hi)) { *out_steps = hi; return SPKV_OK; }
+  while (hi - lo > 1) {
+    const int64_t mid = lo + (hi - lo) / 2;
+    if (steps_fit(cfg, h_len, h_t, n_units, pages_free, mid)) lo = mid; else hi = mid;
+  }
+  *out_steps = lo;
+  return SPKV_OK;
+}
+
+extern "C" int spkv_safe_steps(spkv_cache_t *cache, const int32_t *h_seq_ids, int32_t B, spkv_stream_t stream,
+                               int64_t *out_steps) {
+  if (!cache || !out_steps || B < 0 || (B > 0 && !h_seq_ids)) return SPKV_E_INVALID;
+  const CacheView &v = cache->view;
+  for (int b = 0; b < B; ++b)
+    if (h_seq_ids[b] < 0 || h_seq_ids[b] >= v.S) return SPKV_E_INVALID;
+  if (cudaStreamSynchronize(as_stream(stream)) != cudaSuccess) return SPKV_E_CUDA;
+  std::vector<int32_t> t(v.n_units), len(v.n_units);
+  int32_t hdr[2];
+  if (cudaMemcpy(t.data(), v.t, (size_t)v.n_units * 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
+      cudaMemcpy(len.data(), v.len, (size_t)v.n_units * 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
+      cudaMemcpy(hdr, v.status, 8, cudaMemcpyDeviceToHost) != cudaSuccess)
+    return SPKV_E_CUDA;
+  // the units of the listed sequences (every layer and KV head); B = 0: all sequences
+  std::vector<int32_t> sl, st;
+  for (int l = 0; l < v.L; ++l)
+    for (int b = 0; b < (B ? B : v.S); ++b)
+      for (int h = 0; h < v.Hkv; ++h) {
+        const int u = (l * v.S + (B ? h_seq_ids[b] : b)) * v.Hkv + h;
+        sl.push_back(len[u]);
+        st.push_back(t[u]);
+      }
+  return spkv_safe_steps_from_lengths(&cache->cfg, sl.data(), st.data(), (int64_t)sl.size(),
+                                      hdr[1] > 0 ? hdr[1] : 0, out_steps);
 }
 
 extern "C" int spkv_cache_destroy(spkv_cache_t *cache) {
@@ -239,6 +401,17 @@ extern "C" int spkv_status(spkv_cache_t *cache, spkv_stream_t stream) {
   int32_t st = 0;
   if (cudaStreamSynchronize(as_stream(stream)) != cudaSuccess) return SPKV_E_CUDA;
   if (cudaMemcpy(&st, cache->view.status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return SPKV_E_CUDA;
+  if (st == SPKV_OK && (cache->cfg.flags & SPKV_FLAG_DEBUG_BOUNDS)) {
+    // the canary blocks between the metadata regions must still hold their pattern
+    unsigned char blk[kCanaryBytes];
+    for (int i = 0; i < kCanaries; ++i) {
+      if (cudaMemcpy(blk, static_cast<char *>(cache->arena) + cache->layout.canary[i], kCanaryBytes,
+                     cudaMemcpyDeviceToHost) != cudaSuccess)
+        return SPKV_E_CUDA;
+      for (int b = 0; b < kCanaryBytes; ++b)
+        if (blk[b] != kCanaryByte) return SPKV_E_CANARY;
+    }
+  }
   return st;
 }
 
@@ -390,6 +563,9 @@ extern "C" const char *spkv_error_string(int code) {
     case SPKV_E_SCRATCH_LIMIT: return "request exceeds the built-in scratch area";
     case SPKV_E_ORDER_DECODE: return "overlap mode: decode launch gave up waiting for its append / workspace";
     case SPKV_E_ORDER_APPEND: return "overlap mode: append gave up waiting for its layer's decode launches";
+    case SPKV_E_BOUNDS_PAGE: return "debug bounds: page index outside the pool";
+    case SPKV_E_CANARY: return "debug bounds: a canary block between arena regions was overwritten";
+    case SPKV_E_ATTACH: return "arena does not hold a cache of this configuration";
     default: return "unknown error";
   }
 }

@@ -39,9 +39,9 @@
 //       the partial + arrival count + last-arriver merge) while the consumers stream on.
 //
 // Why tensor cores in a bandwidth-bound kernel: per 512 B pair the group needs 2*G*128
-// multiply-adds.  On the CUDA cores (spkv_decode_simt.cu) that is, with bf16 unpacking and
-// the reductions, several hundred issue slots per pair and SM, and the issue rate, not
-// HBM, limits the kernel from G = 4 on.  As MMA tiles it is 24 instructions per page and
+// multiply-adds.  On the CUDA cores that is, with bf16 unpacking and the reductions, several
+// hundred issue slots per pair and SM (174 warp instructions per pair at G = 4 in an earlier
+// CUDA-core version of this kernel), and the issue rate, not HBM, limits the kernel from G = 4 on.  As MMA tiles it is 24 instructions per page and
 // warp, and the page stream alone sets the pace.
 //
 // Every wait is bounded (about a second).  A consumer warp whose page never lands records
@@ -49,7 +49,7 @@
 // leave at the same page; a producer whose stage is never released records the error and
 // stops issuing, after which the consumers run into their own limit.  Before the block
 // exits the producer waits (bounded again) for the copies it still has in flight.
-#include <stdlib.h>
+#include <atomic>
 
 #include "spkv_decode_common.cuh"
 #include "spkv_mma.cuh"
@@ -356,7 +356,8 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
         if (j >= 0) {
           const int u = s_unit[item], len = s_len[item], nk = (len + kP - 1) / kP;
           if (j < nk) {
-            gq.gpage = __ldcg(&c.table[(size_t)u * c.max_pages + j]);
+            // (debug bounds: a table entry that names no pool page is read from the unit's ring instead)
+            gq.gpage = checked_page(c, __ldcg(&c.table[(size_t)u * c.max_pages + j]), (int)ring_page(c, u, 0));
             gq.valid = min(kP, len - j * kP);
           } else {
             gq.gpage = (int)ring_page(c, u, j - nk);
@@ -764,17 +765,27 @@ extern "C" size_t spkv_decode_workspace_bytes(const spkv_config_t *cfg, int32_t 
   return 2 * decode_ws_layout(B * cfg->n_kv_heads, cfg->n_q_heads / cfg->n_kv_heads).total;
 }
 
+// Argument checks of a decode call that need no workspace (B > 0 on SPKV_OK with *empty = false).
+static int decode_check_args(const spkv_cache_t *cache, int32_t layer, const int32_t *d_seq_ids, int32_t B,
+                             const void *d_q, const void *d_out, const float *d_out_f32, bool *empty) {
+  *empty = false;
+  if (!cache || layer < 0 || layer >= cache->cfg.n_layers || B < 0 || B > cache->cfg.max_seqs)
+    return SPKV_E_INVALID;
+  if (B == 0) { *empty = true; return SPKV_OK; }
+  if (!d_seq_ids || !d_q || !d_out) return SPKV_E_INVALID;
+  if (((uintptr_t)d_q | (uintptr_t)d_out | (uintptr_t)d_out_f32) & 15) return SPKV_E_INVALID;
+  if (B * cache->view.Hkv > 1024) return SPKV_E_UNSUPPORTED;
+  return SPKV_OK;
+}
+
 static int decode_attention_impl(spkv_cache_t *cache, int32_t layer, const int32_t *d_seq_ids, int32_t B,
                                  const void *d_q, void *d_out, float *d_out_f32, float *d_lse_opt, float sm_scale,
                                  void *d_workspace, size_t workspace_bytes, spkv_stream_t stream) {
-  if (!cache || layer < 0 || layer >= cache->cfg.n_layers || B < 0 || B > cache->cfg.max_seqs)
-    return SPKV_E_INVALID;
-  if (B == 0) return SPKV_OK;
-  if (!d_seq_ids || !d_q || !d_out) return SPKV_E_INVALID;
-  if (((uintptr_t)d_q | (uintptr_t)d_out | (uintptr_t)d_out_f32) & 15) return SPKV_E_INVALID;
+  bool empty;
+  const int rc_args = decode_check_args(cache, layer, d_seq_ids, B, d_q, d_out, d_out_f32, &empty);
+  if (rc_args || empty) return rc_args;
   const CacheView &v = cache->view;
   const int n_items = B * v.Hkv;
-  if (n_items > 1024) return SPKV_E_UNSUPPORTED;
   const DecodeWs wl = decode_ws_layout(n_items, v.G);
   if (!d_workspace || ((uintptr_t)d_workspace & 255) || workspace_bytes < 2 * wl.total) return SPKV_E_WORKSPACE;
 
@@ -786,16 +797,8 @@ static int decode_attention_impl(spkv_cache_t *cache, int32_t layer, const int32
   a.out_f32 = d_out_f32;
   a.lse = d_lse_opt;
   a.scale_log2 = sm_scale * kLog2e;
-  static const int snap_env = [] {
-    const char *e = getenv("SPKV_DECODE_SNAP");  // tuning knob: snapping distance of the range cuts
-    return e ? atoi(e) : 6;
-  }();
-  a.snap = snap_env;
-  static const int min_pos_env = [] {
-    const char *e = getenv("SPKV_DECODE_MINPOS");  // tuning knob: least positions per block of a large launch
-    return e ? max(4, atoi(e)) : 56;
-  }();
-  a.min_pos = min_pos_env;
+  a.snap = 6;       // measured best on the 32 K and 128 K workloads (0, 2, 4, 6, 8, 12 tried)
+  a.min_pos = 56;   // likewise (32 ... 96 tried)
   // Two consecutive decode launches may overlap (the next one starts on the SMs this one
   // has left): they alternate between the two halves of the workspace.  A third cannot
   // join: it needs every block of the second resident, i.e. every SM left by the first.
@@ -825,15 +828,6 @@ static int decode_attention_impl(spkv_cache_t *cache, int32_t layer, const int32
   a.part_acc = reinterpret_cast<float *>(ws + wl.off_acc);
 
   cudaStream_t s = as_stream(stream);
-  static const bool use_simt = [] {
-    const char *e = getenv("SPKV_DECODE_KERNEL");  // "simt": the CUDA-core comparison kernel
-    return e && e[0] == 's';
-  }();
-  if (use_simt) {  // plain launch, not counted in the overlap bookkeeping: the next launch waits for it
-    cache->last_kind = kLastOther;
-    return launch_decode_simt(a, cache->sm_count, s);
-  }
-
   int GP = 1;
   while (GP < v.G) GP <<= 1;
   // as many page stages as fit beside the two merge buffers
@@ -881,36 +875,36 @@ static __device__ __align__(256) unsigned char g_static_scratch[SPKV_STATIC_SCRA
 
 namespace {
 constexpr int kMaxDevices = 64;
-void *g_scratch_ptr[kMaxDevices];  // device address of g_static_scratch, per device
-bool g_scratch_ready[kMaxDevices];
+// device address of g_static_scratch per device; non-null = looked up (published with release
+// order, so a thread that reads it non-null reads the address the lookup returned)
+std::atomic<void *> g_scratch_ptr[kMaxDevices];
 }  // namespace
 
 extern "C" int spkv_decode_attention_static(spkv_cache_t *cache, int32_t layer, const int32_t *d_seq_ids,
                                             int32_t B, const void *d_q, void *d_out, float *d_lse_opt,
                                             float sm_scale, spkv_stream_t stream) {
-  if (!cache || B < 0) return SPKV_E_INVALID;
+  // every refusal comes before anything touches the shared array
+  bool empty;
+  const int rc_args = decode_check_args(cache, layer, d_seq_ids, B, d_q, d_out, nullptr, &empty);
+  if (rc_args || empty) return rc_args;
   const size_t need = spkv_decode_workspace_bytes(&cache->cfg, B);
   if (need > (size_t)SPKV_STATIC_SCRATCH_BYTES) return SPKV_E_SCRATCH_LIMIT;
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SPKV_E_CUDA;
-  if (!g_scratch_ready[dev]) {
+  void *scratch = g_scratch_ptr[dev].load(std::memory_order_acquire);
+  if (!scratch) {
     // In host code `g_static_scratch` names a host-side stand-in, not device memory: the
     // address a kernel may use has to be asked for, once per device, with that device current.
-    void *p = nullptr;
-    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return SPKV_E_CUDA;
-    g_scratch_ptr[dev] = p;
-    g_scratch_ready[dev] = true;
+    if (cudaGetSymbolAddress(&scratch, g_static_scratch) != cudaSuccess || !scratch) return SPKV_E_CUDA;
+    g_scratch_ptr[dev].store(scratch, std::memory_order_release);
   }
-  void *scratch = g_scratch_ptr[dev];
-  if (B > 0) {
-    // the array keeps whatever the previous call left: the arrival counters must start at zero
-    const size_t counters =
-        decode_ws_layout(B * cache->cfg.n_kv_heads, cache->cfg.n_q_heads / cache->cfg.n_kv_heads).off_ml;
-    for (int half = 0; half < 2; ++half)
-      if (cudaMemsetAsync(static_cast<char *>(scratch) + half * (need / 2), 0, counters,
-                          as_stream(stream)) != cudaSuccess)
-        return SPKV_E_CUDA;
-  }
+  // the array keeps whatever the previous call left: the arrival counters must start at zero
+  const size_t counters =
+      decode_ws_layout(B * cache->cfg.n_kv_heads, cache->cfg.n_q_heads / cache->cfg.n_kv_heads).off_ml;
+  for (int half = 0; half < 2; ++half)
+    if (cudaMemsetAsync(static_cast<char *>(scratch) + half * (need / 2), 0, counters,
+                        as_stream(stream)) != cudaSuccess)
+      return SPKV_E_CUDA;
   return spkv_decode_attention(cache, layer, d_seq_ids, B, d_q, d_out, d_lse_opt, sm_scale, scratch,
                                SPKV_STATIC_SCRATCH_BYTES, stream);
 }

@@ -1,5 +1,4 @@
-// Declarations shared by the decode-attention kernels (tensor-core main kernel and the
-// CUDA-core comparison kernel): arguments, workspace layout, block scan.
+// Declarations of the decode-attention kernel: arguments, workspace layout, block scan.
 #pragma once
 #include "spkv_internal.cuh"
 
@@ -27,10 +26,6 @@ struct DecodeArgs {
   int32_t *group_counters; // [n_items][kMaxGrid / 8] arrival counters of the first-level merge groups
   float *part_ml;          // [slots][G][2]
   float *part_acc;         // [slots][G][128]
-};
-
-struct ItemInfo {  // per item, in shared memory
-  int unit, len, n_ring, nk;
 };
 
 // Exclusive prefix sum over s_np[0..n) -> s_pre[0..n], s_pre[n] = total.  All threads call.
@@ -82,7 +77,5 @@ inline DecodeWs decode_ws_layout(int n_items, int G) {
   w.total = w.off_acc + slots * G * kD * 4;
   return w;
 }
-
-int launch_decode_simt(const DecodeArgs &a, int sm_count, cudaStream_t s);
 
 }  // namespace spkv

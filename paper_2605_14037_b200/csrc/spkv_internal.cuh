@@ -1,7 +1,8 @@
 // Internal declarations shared by the translation units of libspkv.so.
 //
 // Arena layout (all offsets 256-byte aligned, computed by spkv_layout()):
-//   header      : status word, free-page counter
+//   header      : status word, free-page counter, magic + layout version + configuration hash
+//   (every metadata region is followed by a 256-byte canary block of 0xC5 bytes)
 //   t[]         : pairs received per unit                       int32 [n_units]
 //   len[]       : kept pairs per unit                           int32 [n_units]
 //   table[]     : page table per unit (global page indices)     int32 [n_units][max_pages]
@@ -9,7 +10,7 @@
 //   pos_pool[]  : position of every kept pair, by pool page     int32 [pool_pages][P]
 //   ring_logit[]: stored logit per ring slot                    f32   [n_units][w]
 //   head_tau[]  : per-(layer, KV head) threshold override       f32   [L][Hkv]  (NaN: none)
-//   vmax[]      : largest finite |value| a unit has received    u32   [n_units] (fp32 bit pattern)
+//   vmax[]      : largest finite |value| in a unit's compact cache u32 [n_units] (fp32 bit pattern)
 //   sync_ctr[]  : blocks started / finished per layer and kernel u64   [L][4]    (launch overlap)
 //   pages       : ring pages of every unit ([n_units][ring_pages]) followed by the pool
 //
@@ -40,6 +41,7 @@ constexpr int kMaxGroup = 16;      // query heads per KV head supported by the k
 struct CacheView {
   int32_t L, S, Hq, Hkv, G, w, ring_pages, max_pages, n_units;
   int32_t n_sink;       // positions < n_sink are kept whatever their logit (sink tokens)
+  int32_t debug_bounds; // SPKV_FLAG_DEBUG_BOUNDS: page indices read from tables are range-checked
   int64_t pool_pages, n_ring_pages_total;
   int32_t *status;      // [0] sticky status, [1] free_top
   int32_t *t;
@@ -50,15 +52,20 @@ struct CacheView {
   float *ring_logit;
   float *head_tau;      // [L][Hkv] logit-space threshold of a (layer, KV head); NaN = the cache-wide one
   unsigned long long *sync_ctr;  // [L][4]: append blocks started, finished; decode blocks started, finished
-  // [n_units] bit pattern of the largest finite |v| the unit has received since its sequence was
-  // reset.  The prefill attention multiplies P.V in fp16 and scales the values by a power of two
-  // taken from this word, so that any bf16 value range fits.
+  // [n_units] bit pattern of the largest finite |v| among the pairs the unit's compact cache holds
+  // (raised when a pair is kept, cleared when the sequence is reset).  The prefill attention
+  // multiplies P.V in fp16 after scaling the values by a power of two; it takes that factor from
+  // the largest |v| its queries can see: this word, the ring and the chunk.
   uint32_t *vmax;
   __nv_bfloat16 *pages;
 };
 
+constexpr int kCanaries = 10;          // one 256-byte block after each metadata region
+constexpr int kCanaryBytes = 256;
+constexpr unsigned char kCanaryByte = 0xC5;
 struct Layout {
   size_t off_header, off_t, off_len, off_table, off_free, off_pos, off_rlogit, off_htau, off_sync, off_vmax, off_pages, total;
+  size_t canary[kCanaries];
 };
 
 // largest finite |x| among the eight bf16 of a 16-byte chunk, as the upper half of an fp32 bit
@@ -74,8 +81,7 @@ __device__ inline uint32_t chunk_abs_max_bf16(const uint4 &v) {
   }
   return m << 16;
 }
-// one thread; the result is not used, so this is a fire-and-forget reduction (reading the word
-// first to skip the atomic would put an L2 round trip at the end of every append)
+// one thread; the result is not used, so this is a fire-and-forget reduction
 __device__ inline void note_vmax(const CacheView &c, int u, uint32_t m) {
   if (m) atomicMax(&c.vmax[u], m);
 }
@@ -90,6 +96,18 @@ __device__ inline int unit_index(const CacheView &c, int layer, int seq, int kvh
 }
 
 __device__ inline void set_status(const CacheView &c, int code) { atomicCAS(c.status, 0, code); }
+
+// ---- SPKV_FLAG_DEBUG_BOUNDS: page indices that come out of memory (page tables, free stack) ----
+__device__ inline bool pool_page_ok(const CacheView &c, int page) {
+  return (int64_t)page >= c.n_ring_pages_total && (int64_t)page < c.n_ring_pages_total + c.pool_pages;
+}
+// `page` if the check is off or the index names a pool page; otherwise the violation is recorded
+// in the status word and `fallback` is returned (a page that is safe to read, or -1 = skip)
+__device__ inline int checked_page(const CacheView &c, int page, int fallback) {
+  if (!c.debug_bounds || pool_page_ok(c, page)) return page;
+  set_status(c, SPKV_E_BOUNDS_PAGE);
+  return fallback;
+}
 
 // threshold in force for a (layer, KV head): its own if one was set, else the cache-wide one
 __device__ inline float head_threshold(const CacheView &c, int layer, int kvh, float tau_logit) {

@@ -1,6 +1,6 @@
-// Warp-level building blocks of the attention kernels: bf16 tensor-core tiles
-// (mma.sync m16n8k16, operands fetched with ldmatrix from swizzled shared memory),
-// the online-softmax update, and the mbarrier / bulk-copy primitives of the page pipeline.
+// Warp-level building blocks of the attention kernels: the bf16 tensor-core tiles of the decode
+// kernel (mma.sync m16n8k16, operands fetched with ldmatrix from swizzled shared memory) with
+// their online-softmax update, and the mbarrier / bulk-copy primitives of the page pipelines.
 //
 // Shared-memory image of a key or value block (identical to its image in HBM): two slabs
 // (dims 0-63 | 64-127) of 64 rows x 128 B; 16-byte chunk c (0-7) of a slab row r is stored at
@@ -49,114 +49,6 @@ __device__ inline float fast_exp2(float x) {
 // Byte offset of (row, logical 16-byte chunk) inside a swizzled key/value block.
 __device__ inline uint32_t blk_off(int row, int chunk) {
   return (uint32_t)((chunk >> 3) * 8192 + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
-}
-
-// Loads the A fragments of a 16 x 128 query tile straight from global memory.
-// row_ptr(r) returns the address of row r's 128 bf16 (or nullptr for a padding row).
-template <class RowPtr>
-__device__ inline void load_q_frags(uint32_t (&qf)[8][4], RowPtr row_ptr, int lane) {
-  const int g = lane >> 2, t = lane & 3;
-  const __nv_bfloat16 *r0 = row_ptr(g), *r1 = row_ptr(g + 8);
-#pragma unroll
-  for (int kk = 0; kk < 8; ++kk) {
-    const int c = kk * 16 + t * 2;
-    qf[kk][0] = r0 ? *reinterpret_cast<const uint32_t *>(r0 + c) : 0u;
-    qf[kk][1] = r1 ? *reinterpret_cast<const uint32_t *>(r1 + c) : 0u;
-    qf[kk][2] = r0 ? *reinterpret_cast<const uint32_t *>(r0 + c + 8) : 0u;
-    qf[kk][3] = r1 ? *reinterpret_cast<const uint32_t *>(r1 + c + 8) : 0u;
-  }
-}
-
-// s[n][.] = Q (16 x 128) . K^T for keys tok0 + 8n .. tok0 + 8n + 7, n < NT/8.
-template <int NT>
-__device__ inline void qk_tile(float (&s)[NT / 8][4], const uint32_t (&qf)[8][4], uint32_t sK,
-                               int tok0, int lane) {
-#pragma unroll
-  for (int n = 0; n < NT / 8; ++n) s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f;
-  const int mi = lane >> 3, ri = lane & 7;
-#pragma unroll
-  for (int kk = 0; kk < 8; ++kk) {
-#pragma unroll
-    for (int jp = 0; jp < NT / 16; ++jp) {
-      uint32_t b[4];
-      const int tok = tok0 + jp * 16 + (mi >> 1) * 8 + ri;
-      ldsm_x4(b, sK + blk_off(tok, 2 * kk + (mi & 1)));
-      mma_bf16_16816(s[2 * jp], qf[kk], b[0], b[1]);
-      mma_bf16_16816(s[2 * jp + 1], qf[kk], b[2], b[3]);
-    }
-  }
-}
-
-// Online-softmax update with the NT keys of this tile, then O += P . V.
-// visible(h, col): is key `col` (tile-local index tok0-based: col in [tok0, tok0+NT))
-// visible to row (g + 8h)?  m/l/o are per-thread state for rows g and g+8; l is a
-// per-thread partial sum (reduce over the 4 lanes of a quad at the end).
-template <int NT, class Visible>
-__device__ inline void softmax_pv_tile(float (&s)[NT / 8][4], Visible visible, float scale_log2,
-                                       float (&m)[2], float (&l)[2], float (&o)[16][4], uint32_t sV,
-                                       int tok0, int lane) {
-  const int t = lane & 3;
-  float mx[2] = {-INFINITY, -INFINITY};
-#pragma unroll
-  for (int n = 0; n < NT / 8; ++n)
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const int h = e >> 1;
-      const int col = tok0 + n * 8 + t * 2 + (e & 1);
-      const float v = visible(h, col) ? s[n][e] * scale_log2 : -INFINITY;
-      s[n][e] = v;
-      mx[h] = fmaxf(mx[h], v);
-    }
-  float ms[2];
-#pragma unroll
-  for (int h = 0; h < 2; ++h) {
-    mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 1));
-    mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 2));
-    const float mn = fmaxf(m[h], mx[h]);
-    ms[h] = mn == -INFINITY ? 0.f : mn;  // a row that has seen no key yet
-    const float corr = fast_exp2(m[h] - ms[h]);
-    m[h] = mn;
-    l[h] *= corr;
-#pragma unroll
-    for (int n = 0; n < 16; ++n) {
-      o[n][2 * h] *= corr;
-      o[n][2 * h + 1] *= corr;
-    }
-  }
-#pragma unroll
-  for (int n = 0; n < NT / 8; ++n)
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const float p = fast_exp2(s[n][e] - ms[e >> 1]);
-      s[n][e] = p;
-      l[e >> 1] += p;
-    }
-  // P is split into two bf16 terms, P = hi + lo (lo = P - bf16(P)), each multiplied into V:
-  // the weights then carry ~16 mantissa bits, so that the result keeps float32-accumulation
-  // accuracy even when large value terms cancel (a single bf16 P would err by 2^-9 sum p|v|).
-  const int mi = lane >> 3, ri = lane & 7;
-#pragma unroll
-  for (int kk = 0; kk < NT / 16; ++kk) {
-    uint32_t a[4], alo[4];
-#pragma unroll
-    for (int x = 0; x < 4; ++x) {
-      const float p0 = s[2 * kk + (x >> 1)][(x & 1) * 2], p1 = s[2 * kk + (x >> 1)][(x & 1) * 2 + 1];
-      const __nv_bfloat162 hi = __floats2bfloat162_rn(p0, p1);
-      const float2 hf = __bfloat1622float2(hi);
-      a[x] = *reinterpret_cast<const uint32_t *>(&hi);
-      alo[x] = pack_bf16(p0 - hf.x, p1 - hf.y);
-    }
-    const int tok = tok0 + kk * 16 + (mi & 1) * 8 + ri;
-#pragma unroll
-    for (int jn = 0; jn < 8; ++jn) {
-      uint32_t b[4];
-      ldsm_x4_trans(b, sV + blk_off(tok, 2 * jn + (mi >> 1)));
-      mma_bf16_16816(o[2 * jn], a, b[0], b[1]);
-      mma_bf16_16816(o[2 * jn + 1], a, b[2], b[3]);
-      mma_bf16_16816(o[2 * jn], alo, b[0], b[1]);
-      mma_bf16_16816(o[2 * jn + 1], alo, b[2], b[3]);
-    }
-  }
 }
 
 // ---- "keys as rows" tiles for decode --------------------------------------------------------
@@ -261,7 +153,10 @@ __device__ inline void softmax_pv_tile_t(float (&s)[NH][4], int n_valid, float s
       p[e] = fast_exp2(v[e] - ms[e & 1]);
       l[hn][e & 1] += p[e];
     }
-    // P = hi + lo in bf16 (see softmax_pv_tile), transposed into B-fragment layout
+    // P is split into two bf16 terms, P = hi + lo (lo = P - bf16(P)), each multiplied into V: the
+    // weights then carry ~16 mantissa bits, so that the result keeps float32-accumulation accuracy
+    // even when large value terms cancel (a single bf16 P would err by 2^-9 sum p|v|).
+    // Transposed into B-fragment layout.
     const __nv_bfloat162 h0 = __floats2bfloat162_rn(p[0], p[1]), h1 = __floats2bfloat162_rn(p[2], p[3]);
     const float2 f0 = __bfloat1622float2(h0), f1 = __bfloat1622float2(h1);
     bhi[hn][0] = movmatrix_trans(*reinterpret_cast<const uint32_t *>(&h0));
@@ -307,14 +202,20 @@ __device__ inline bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
       : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up after ~2^31 clock cycles (about a second) and returns false.
-__device__ inline bool mbar_wait_bounded(uint64_t *bar, uint32_t parity) {
+// Bounded wait: gives up after `limit` clock cycles (default ~2^31, about a second) and returns false.
+constexpr long long kWaitClocks = 1LL << 31;
+__device__ inline bool mbar_wait_bounded(uint64_t *bar, uint32_t parity, long long limit = kWaitClocks) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   while (!mbar_try_wait(bar, parity)) {
-    if (clock64() - t0 > (1LL << 31)) return false;
+    if (clock64() - t0 > limit) return false;
   }
   return true;
+}
+// Counts `bytes` as arrived on the barrier's current phase without any copy (used to close a
+// phase that was armed for more bytes than were ever sent).
+__device__ inline void mbar_complete_tx(uint64_t *bar, uint32_t bytes) {
+  asm volatile("mbarrier.complete_tx.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
 // 1-D bulk copy; src, dst 16-byte aligned, bytes a multiple of 16.
 __device__ inline void bulk_load(void *smem_dst, const void *gmem_src, uint32_t bytes, uint64_t *bar) {
@@ -322,13 +223,5 @@ __device__ inline void bulk_load(void *smem_dst, const void *gmem_src, uint32_t 
       "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
       ::"r"(smem_u32(smem_dst)), "l"(gmem_src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
-
-// ---- cp.async (16-byte) for gathered tiles ---------------------------------------------
-__device__ inline void cp_async16(uint32_t smem_dst, const void *gmem_src) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
-}
-__device__ inline void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ inline void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 }  // namespace spkv

@@ -2,7 +2,7 @@
 //
 // By definition the result equals C x (append/evict, decode attention) -- the paper's
 // chunked-prefill protocol, cache compressed after every chunk (Section "Sparse decoding
-// approximation"), attention per Eq. 3-5.  It is computed in four launches:
+// approximation"), attention per Eq. 3-5.  It is computed in five launches:
 //
 //  A  plan     one block per KV head: thresholds the old ring pairs and the chunk pairs in
 //              position order ("staging" sequence of N = min(t0,w) + C pairs), exclusive
@@ -11,8 +11,11 @@
 //  B  scatter  stream compaction proper: every flagged staging pair whose position is
 //              <= t_last - w is copied to compact-cache index len0 + E[j] (ascending
 //              position, so order and indices are unique and bit-exact).
-//  ATT attention of every query of the chunk (tensor cores, bf16 mma.sync m16n8k16, fp32
-//              accumulation, online softmax) over
+//  STG stage    the old ring pairs and the chunk's pairs, in position order, rewritten as pages
+//              in the workspace ("staging pages"), so that every key/value tile of the
+//              attention -- compact-cache page or band page -- is the same 32 KB image.
+//  ATT attention of every query of the chunk (tcgen05 tensor cores, fp32 accumulation, online
+//              softmax; spkv_prefill_tc5x2h.cu) over
 //                (a) the first nvis(t) = len0 + E[t - w - p0 + 1] pairs of the compact cache
 //                    (the kept pairs with position <= t - w: a prefix, because the cache is in
 //                    ascending position order), and
@@ -23,10 +26,7 @@
 //              are advanced.
 //
 // Workspace per KV head: a 64-int header followed by E[0..N] (int32).
-#include <stdlib.h>
-
 #include "spkv_prefill_common.cuh"
-#include "spkv_mma.cuh"
 
 namespace spkv {
 
@@ -87,12 +87,14 @@ __global__ void __launch_bounds__(1024) prefill_plan_kernel(PrefillArgs a) {
     if (pages1 > c.max_pages) {
       fail = SPKV_E_CONTEXT_OVERFLOW;
     } else if (n_new > 0) {
-      const int top = atomicSub(&c.status[1], n_new);
-      if (top < n_new) {
-        atomicAdd(&c.status[1], n_new);
-        fail = SPKV_E_POOL_EXHAUSTED;
-      } else {
-        s_pages_base = top;
+      // all n_new pages or none: the counter only ever moves by what is really taken, so the
+      // blocks of the other KV heads never see a number lower than the pool holds
+      int top = atomicAdd(&c.status[1], 0);
+      for (;;) {
+        if (top < n_new) { fail = SPKV_E_POOL_EXHAUSTED; break; }
+        const int seen = atomicCAS(&c.status[1], top, top - n_new);
+        if (seen == top) { s_pages_base = top; break; }
+        top = seen;
       }
     }
     if (fail) set_status(c, fail);
@@ -101,14 +103,17 @@ __global__ void __launch_bounds__(1024) prefill_plan_kernel(PrefillArgs a) {
     hdr[H_NCOMMIT] = fail ? 0 : n_commit;
     hdr[H_LEN1] = fail ? len0 : len1;
     hdr[H_FAIL] = fail;
+    hdr[H_VMAX] = (int32_t)c.vmax[u];   // the kept pairs so far; the stage kernel adds ring and chunk
   }
   __syncthreads();
   if (s_fail || n_new == 0) return;
+  // (debug bounds: an index from the stack that names no pool page is recorded; the scatter kernel
+  // skips what would go there)
   for (int i = tid; i < n_new; i += blockDim.x)
-    c.table[(size_t)u * c.max_pages + pages0 + i] = c.free_stack[s_pages_base - 1 - i];
+    c.table[(size_t)u * c.max_pages + pages0 + i] = checked_page(c, c.free_stack[s_pages_base - 1 - i], -1);
   __syncthreads();
   // rows past the final length of a freshly popped last page must read as zeros
-  if (len1 % kP) {
+  if (len1 % kP && c.table[(size_t)u * c.max_pages + pages1 - 1] >= 0) {
     const int last = c.table[(size_t)u * c.max_pages + pages1 - 1];
     uint4 *vb = reinterpret_cast<uint4 *>(c.pages + (int64_t)last * kPageElems + kBlockElems);
     for (int i = tid; i < kBlockElems * 2 / 16; i += blockDim.x) vb[i] = make_uint4(0, 0, 0, 0);
@@ -154,17 +159,18 @@ __global__ void __launch_bounds__(256) prefill_scatter_kernel(PrefillArgs a) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int chunk = lane & 15, blk = (lane >> 4) * kBlockElems;
   const int j0 = (blockIdx.x * 8 + warp) * 8;
-  uint32_t vm = 0;  // largest |v| among the chunk's own pairs that this warp keeps
+  uint32_t vm = 0;  // largest |v| among the pairs this warp appends to the compact cache
   for (int j = j0; j < min(j0 + 8, n_leave); ++j) {
     const int e = E[j];
     if (E[j + 1] == e) continue;  // not flagged
     const int idx = len0 + e;
-    const int page = c.table[(size_t)u * c.max_pages + idx / kP];
+    const int page = checked_page(c, c.table[(size_t)u * c.max_pages + idx / kP], -1);
+    if (page < 0) continue;   // debug bounds: recorded, the pair is not written
     const int drow = idx % kP;
     const SrcRow s = staging_row(a, u, kvh, t0, n_old, j);
     const uint4 val = load_chunk(lane < 16 ? s.k : s.v, s.row, chunk);
     *reinterpret_cast<uint4 *>(c.pages + (int64_t)page * kPageElems + blk + swz_off(drow, chunk)) = val;
-    if (lane >= 16 && j >= n_old) vm = max(vm, chunk_abs_max_bf16(val));
+    if (lane >= 16) vm = max(vm, chunk_abs_max_bf16(val));
     if (lane == 0) c.pos_pool[((int64_t)page - c.n_ring_pages_total) * kP + drow] = t0 - n_old + j;
   }
   vm = __reduce_max_sync(0xffffffffu, vm);
@@ -189,11 +195,7 @@ __global__ void __launch_bounds__(256) prefill_ring_kernel(PrefillArgs a) {
     const size_t off = ((size_t)i * c.Hkv + kvh) * kD;
     const uint4 val = *reinterpret_cast<const uint4 *>((lane < 16 ? a.k : a.v) + off + chunk * 8);
     *reinterpret_cast<uint4 *>(pg + blk + swz_off(row, chunk)) = val;
-    const uint32_t vm = __reduce_max_sync(0xffffffffu, lane < 16 ? 0u : chunk_abs_max_bf16(val));
-    if (lane == 0) {
-      c.ring_logit[(size_t)u * c.w + slot] = a.logits[(size_t)i * c.Hkv + kvh];
-      if (vm) note_vmax(c, u, vm);
-    }
+    if (lane == 0) c.ring_logit[(size_t)u * c.w + slot] = a.logits[(size_t)i * c.Hkv + kvh];
   }
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     c.t[u] = t0 + a.C;
@@ -201,119 +203,37 @@ __global__ void __launch_bounds__(256) prefill_ring_kernel(PrefillArgs a) {
   }
 }
 
-// ------------------------------------------------------------------ ATT: chunk attention
-// grid (ceil(C/64), Hq); 4 warps x 16 query rows; K/V tiles of 64 keys, double buffered.
-constexpr int kAttnSmem = 2 * kPageBytes;
-
-__global__ void __launch_bounds__(128) prefill_attn_kernel(PrefillArgs a) {
-  extern __shared__ __align__(128) unsigned char smem[];
+// ------------------------------------------------------------------ STG: staging pages
+// Old ring pairs and chunk pairs, in position order, rewritten as pages (workspace).
+// grid (n_stage_pages, Hkv), 256 threads: 8 warps x 8 rows.
+__global__ void __launch_bounds__(256) prefill_stage_kernel(PrefillArgs a) {
   const CacheView &c = a.c;
-  const int hq = blockIdx.y, kvh = hq / c.G;
-  const int i0 = blockIdx.x * 64;
-  const int32_t *hdr = unit_ws(a, kvh);
-  const int32_t *E = hdr + kHdrInts;
-  const int t0 = hdr[H_T0], len0 = hdr[H_LEN0], n_old = hdr[H_NOLD], N = hdr[H_N];
-  const int p0 = t0 - n_old;
+  const int kvh = blockIdx.y, sp = blockIdx.x;
+  int32_t *hdr = unit_ws(a, kvh);
+  const int t0 = hdr[H_T0], n_old = hdr[H_NOLD], N = hdr[H_N];
   const int u = unit_index(c, a.layer, a.seq, kvh);
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int g = lane >> 2;
-
-  // kept pairs visible to chunk query i: those with position <= t0 + i - w
-  auto nvis = [&](int i) { return len0 + E[min(max(i + n_old - c.w + 1, 0), N)]; };
-  const int i_last = min(i0 + 63, a.C - 1);
-  const int nv_lo = nvis(i0), nv_hi = nvis(i_last);
-  const int n_ptiles = (nv_hi + kP - 1) / kP;
-  const int s_lo = max(p0, t0 + i0 - c.w + 1), s_hi = t0 + i_last;  // band positions
-  const int n_btiles = (s_hi - s_lo + 1 + 63) / 64;
-  const int n_tiles = n_ptiles + n_btiles;
-
-  // rows of this thread
-  const int ra = i0 + warp * 16 + g, rb = ra + 8;
-  const int nv_a = ra < a.C ? nvis(ra) : 0, nv_b = rb < a.C ? nvis(rb) : 0;
-  const int ta = t0 + ra, tb = t0 + rb;
-
-  uint32_t qf[8][4];
-  load_q_frags(qf, [&](int r) -> const __nv_bfloat16 * {
-    const int i = i0 + warp * 16 + r;
-    return i < a.C ? a.q + ((size_t)i * c.Hq + hq) * kD : nullptr;
-  }, lane);
-
-  auto load_tile = [&](int tile, int buf) {
-    unsigned char *dst = smem + buf * kPageBytes;
-    if (tile < n_ptiles) {
-      const int page = c.table[(size_t)u * c.max_pages + tile];
-      const unsigned char *src = reinterpret_cast<const unsigned char *>(c.pages + (int64_t)page * kPageElems);
-      for (int x = tid; x < kPageBytes / 16; x += 128) cp_async16(smem_u32(dst + x * 16), src + x * 16);
-    } else {
-      // gather 64 band rows (ring slots or chunk rows) into the swizzled image
-      const int s_base = s_lo + (tile - n_ptiles) * 64;
-      for (int x = tid; x < 64 * 32; x += 128) {
-        const int r = x >> 5, part = x & 31, chunk = part & 15, isv = part >> 4;
-        const int s = s_base + r;
-        const uint32_t d = smem_u32(dst + isv * (kBlockElems * 2)) + blk_off(r, chunk);
-        if (s <= s_hi) {
-          const SrcRow sr = staging_row(a, u, kvh, t0, n_old, s - p0);
-          const __nv_bfloat16 *rowp = isv ? sr.v : sr.k;
-          cp_async16(d, rowp + (sr.row >= 0 ? swz_off(sr.row, chunk) : chunk * 8));
-        } else {
-          *reinterpret_cast<uint4 *>(dst + isv * (kBlockElems * 2) + blk_off(r, chunk)) = make_uint4(0, 0, 0, 0);
-        }
-      }
-    }
-    cp_async_commit();
-  };
-
-  float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f}, o[16][4];
-#pragma unroll
-  for (int n = 0; n < 16; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
-
-  load_tile(0, 0);
-  for (int tile = 0; tile < n_tiles; ++tile) {
-    const int buf = tile & 1;
-    if (tile + 1 < n_tiles) {
-      load_tile(tile + 1, buf ^ 1);
-      cp_async_wait<1>();
-    } else {
-      cp_async_wait<0>();
-    }
-    __syncthreads();
-    const uint32_t sK = smem_u32(smem + buf * kPageBytes), sV = sK + kBlockElems * 2;
-    float s[8][4];
-    qk_tile<64>(s, qf, sK, 0, lane);
-    if (tile < n_ptiles) {
-      const int base = tile * kP;
-      if (base + kP <= nv_lo) {
-        softmax_pv_tile<64>(s, [](int, int) { return true; }, a.scale_log2, m, l, o, sV, 0, lane);
+  __nv_bfloat16 *page = a.stage_pages + ((size_t)kvh * a.n_stage_pages + sp) * kPageElems;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int chunk = lane & 15, blk = (lane >> 4) * kBlockElems;
+  uint32_t vm = 0;  // largest |v| among the values this lane moves
+  for (int r = warp * 8; r < warp * 8 + 8; ++r) {
+    const int j = sp * kP + r;
+    uint4 val = make_uint4(0, 0, 0, 0);  // rows past the last pair read as zeros
+    if (j < N) {
+      if (j < n_old) {
+        const int slot = (t0 - n_old + j) % c.w;
+        const __nv_bfloat16 *pg = c.pages + ring_page(c, u, slot / kP) * kPageElems;
+        val = *reinterpret_cast<const uint4 *>(pg + blk + swz_off(slot % kP, chunk));
       } else {
-        softmax_pv_tile<64>(s, [&](int h, int col) { return base + col < (h ? nv_b : nv_a); },
-                            a.scale_log2, m, l, o, sV, 0, lane);
+        const __nv_bfloat16 *src = (lane < 16 ? a.k : a.v) + ((size_t)(j - n_old) * c.Hkv + kvh) * kD;
+        val = *reinterpret_cast<const uint4 *>(src + chunk * 8);
       }
-    } else {
-      const int s_base = s_lo + (tile - n_ptiles) * 64;
-      softmax_pv_tile<64>(s, [&](int h, int col) {
-        const int sp = s_base + col, tq = h ? tb : ta;
-        return sp <= tq && sp > tq - c.w && sp <= s_hi;
-      }, a.scale_log2, m, l, o, sV, 0, lane);
+      if (lane >= 16) vm = max(vm, chunk_abs_max_bf16(val));
     }
-    __syncthreads();
+    *reinterpret_cast<uint4 *>(page + blk + swz_off(r, chunk)) = val;
   }
-  // finish: reduce l over the quad, normalise, store bf16
-#pragma unroll
-  for (int h = 0; h < 2; ++h) {
-    l[h] += __shfl_xor_sync(0xffffffffu, l[h], 1);
-    l[h] += __shfl_xor_sync(0xffffffffu, l[h], 2);
-  }
-  const int t4 = lane & 3;
-#pragma unroll
-  for (int h = 0; h < 2; ++h) {
-    const int i = h ? rb : ra;
-    if (i >= a.C) continue;
-    const float inv = 1.f / l[h];
-    __nv_bfloat16 *orow = a.out + ((size_t)i * c.Hq + hq) * kD;
-#pragma unroll
-    for (int n = 0; n < 16; ++n)
-      *reinterpret_cast<uint32_t *>(orow + n * 8 + t4 * 2) = pack_bf16(o[n][2 * h] * inv, o[n][2 * h + 1] * inv);
-  }
+  vm = __reduce_max_sync(0xffffffffu, vm);
+  if (lane == 0 && vm) atomicMax(reinterpret_cast<uint32_t *>(&hdr[H_VMAX]), vm);
 }
 
 static size_t prefill_ws_stride_ints(int C, int w) {
@@ -347,6 +267,8 @@ extern "C" int spkv_prefill(spkv_cache_t *cache, int32_t layer, int32_t seq, int
     return SPKV_E_INVALID;
   if (C == 0) return SPKV_OK;
   if (!d_k || !d_v || !d_logits || ((d_q == nullptr) != (d_out == nullptr))) return SPKV_E_INVALID;
+  // the attention kernel folds the scale into the exponent and takes row maxima before scaling
+  if (d_q && !(sm_scale > 0.f && sm_scale < INFINITY)) return SPKV_E_INVALID;
   if (((uintptr_t)d_k | (uintptr_t)d_v | (uintptr_t)d_q | (uintptr_t)d_out) & 15) return SPKV_E_INVALID;
   const CacheView &v = cache->view;
   if (!d_workspace || ((uintptr_t)d_workspace & 255) ||
@@ -368,6 +290,7 @@ extern "C" int spkv_prefill(spkv_cache_t *cache, int32_t layer, int32_t seq, int
   a.n_stage_pages = prefill_stage_pages(&cache->cfg, C);
   a.pair_tiles = 0;
   a.n_split = 1;
+  a.force_wide = (cache->cfg.flags & SPKV_FLAG_PREFILL_PV_BF16) ? 1 : 0;
   a.partials = prefill_split_bytes(&cache->cfg, C)
                    ? reinterpret_cast<float *>(reinterpret_cast<char *>(a.stage_pages) +
                                                (size_t)v.Hkv * a.n_stage_pages * kPageBytes)
@@ -378,18 +301,10 @@ extern "C" int spkv_prefill(spkv_cache_t *cache, int32_t layer, int32_t seq, int
   prefill_plan_kernel<<<v.Hkv, 1024, 0, s>>>(a);
   // at most max(min(t0,w) + C - w, 0) <= C pairs leave the window
   prefill_scatter_kernel<<<dim3((C + 63) / 64, v.Hkv), 256, 0, s>>>(a);
-  static const bool use_mma_sync = [] {
-    const char *e = getenv("SPKV_PREFILL_KERNEL");  // "mma": the mma.sync comparison kernel
-    return e && e[0] == 'm';
-  }();
-  if (d_q && !use_mma_sync && sm_scale > 0.f) {  // the tcgen05 kernel folds a positive scale into the exponent
-    int rc = launch_prefill_attn_tc5(a, s);
+  if (d_q) {
+    prefill_stage_kernel<<<dim3(a.n_stage_pages, v.Hkv), 256, 0, s>>>(a);
+    const int rc = launch_prefill_attn_tc5x2h(a, s);
     if (rc) return rc;
-  } else if (d_q) {
-    if (cudaFuncSetAttribute(prefill_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             kAttnSmem) != cudaSuccess)
-      return SPKV_E_CUDA;
-    prefill_attn_kernel<<<dim3((C + 63) / 64, v.Hq), 128, kAttnSmem, s>>>(a);
   }
   const int n_ring = C < v.w ? C : v.w;
   prefill_ring_kernel<<<dim3((n_ring + 7) / 8, v.Hkv), 256, 0, s>>>(a);

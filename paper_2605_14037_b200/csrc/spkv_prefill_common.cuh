@@ -5,7 +5,10 @@
 namespace spkv {
 
 constexpr int kHdrInts = 64;
-enum { H_T0 = 0, H_LEN0, H_NOLD, H_N, H_NCOMMIT, H_LEN1, H_FAIL };
+enum { H_T0 = 0, H_LEN0, H_NOLD, H_N, H_NCOMMIT, H_LEN1, H_FAIL,
+       // fp32 bit pattern of the largest finite |value| a query of this call can see: the unit's kept
+       // pairs so far (plan kernel) and every staged pair, old ring and chunk (stage kernel)
+       H_VMAX };
 
 struct PrefillArgs {
   CacheView c;
@@ -21,16 +24,16 @@ struct PrefillArgs {
   int pair_tiles;                  // fp16 two-slot kernel: a single head's blocks take two query tiles each
   int n_split;                     // fp16 two-slot kernel: blocks per page walk (split over the pages), >= 1
   float *partials;                 // [walk][slot][split]: 128 rows x (128 O + pad) and (m, l); n_split > 1 only
+  int force_wide;                  // SPKV_FLAG_PREFILL_PV_BF16: every unit takes the two-term bf16 P.V
 };
 
 __device__ inline int32_t *unit_ws(const PrefillArgs &a, int kvh) { return a.ws + (size_t)kvh * a.ws_stride; }
 
-// Work order of the tensor-core attention kernels (1-D grid, blocks start in index order):
+// Work order of the tensor-core attention kernel (1-D grid, blocks start in index order):
 // heaviest blocks first, so that the last wave is made of short ones.  A block's length is the
 // number of pages it walks: KV heads are taken by descending number of kept pairs after the
 // chunk (the plan kernel has counted them), and inside a head the query tiles run from the end
-// of the chunk backwards.  Item -> (KV head, which of its `blocks_per_kvh` head groups, query
-// tile).  Called by whole warps at kernel entry; every warp computes the same answer.
+// of the chunk backwards.
 //
 // The KV head with the rank-th most keys per query in this chunk (ties by index).  Called by whole
 // warps; every warp computes the same answer.  More KV heads than lanes: plain order.
@@ -49,18 +52,7 @@ __device__ inline int prefill_kvh_by_rank(const PrefillArgs &a, int rank) {
   }
   return __ffs(__ballot_sync(0xffffffffu, lane < Hkv && my_rank == rank)) - 1;
 }
-__device__ inline void prefill_work_item(const PrefillArgs &a, int item, int n_xtiles, int blocks_per_kvh, int &kvh,
-                                         int &sub, int &xtile) {
-  const int r = item / n_xtiles;
-  xtile = n_xtiles - 1 - item % n_xtiles;
-  sub = r % blocks_per_kvh;
-  kvh = prefill_kvh_by_rank(a, r / blocks_per_kvh);
-}
-
-
-// staging pages + chunk attention on tcgen05 (two heads per block when G is even)
-int launch_prefill_attn_tc5(const PrefillArgs &a, cudaStream_t s);
-int launch_prefill_attn_tc5x2(const PrefillArgs &a, cudaStream_t s);
+// chunk attention on tcgen05 (two 128-row slots per block), after the staging pages were written
 int launch_prefill_attn_tc5x2h(const PrefillArgs &a, cudaStream_t s);
 size_t prefill_split_bytes(const spkv_config_t *cfg, int C);   // partial results of split page walks (small chunks)
 

@@ -1,18 +1,32 @@
-// Chunk attention of spkv_prefill on tcgen05, two query heads per block, P.V in fp16.
+// Chunk attention of spkv_prefill on tcgen05 (Eq. 3-5 for every query of a chunk), two query heads
+// per block, P.V in fp16 -- or, for a unit whose values span too wide a range for that, in two
+// bf16 terms.
 //
-// Same tiling as the two-term bf16 kernel next door: one block = two 128-row slots that walk the
-// same pages -- two query heads that share a KV head on one tile of 128 consecutive queries
-// (Eq. 5), or, for the last head of an odd group (G = 1: every head), two consecutive query tiles
-// of that head; every 32 KB page is fetched once and feeds both slots; one softmax group of 128
-// threads per slot, thread = query row = TMEM lane.  ("Head h" below means slot h.)  Two things
-// differ:
+// One block = two 128-row slots that walk the same pages -- two query heads that share a KV head
+// on one tile of 128 consecutive queries (Eq. 5: head j reads KV head j / G), or, for the last head
+// of an odd group (G = 1: every head), two consecutive query tiles of that head; every 32 KB page
+// is fetched once and feeds both slots; one softmax group of 128 threads per slot, thread = query
+// row = TMEM lane.  ("Head h" below means slot h.)  Per page and slot: S = Q K^T (8 MMAs M128 N64
+// K16, S in tensor memory), softmax in registers, O += P V with P taken from tensor memory.
 //
-// * P is ONE fp16 term (11 significant bits; the two-term bf16 split carries 16 but costs a second
-//   P.V pass).  The tensor cores want both operands in the same type, so warps 2-3 rewrite the
-//   value block of every page from bf16 to fp16 in shared memory, multiplied by a power of two
-//   that brings the largest |v| the unit has ever received into [2^14, 2^15) -- any bf16 range
-//   fits, and the epilogue undoes the factor exactly.  P carries a bias of 2^7 (p <= 2^8 under the
-//   lazy rescale), which cancels between O and the row sum.
+// * P is ONE fp16 term (11 significant bits).  The tensor cores want both operands in the same
+//   type, so warps 2-3 rewrite the value block of every page from bf16 to fp16 in shared memory,
+//   multiplied by a power of two that brings the largest |v| a query of this call can see (the
+//   unit's kept pairs, the old ring, the chunk: H_VMAX of the plan header) into [2^14, 2^15); the
+//   epilogue undoes the factor exactly.  A bf16 value converts to fp16 without loss unless it is
+//   more than 2^28 below that maximum, where fp16 goes subnormal: such a value is off by at most
+//   2^-39 of the maximum.  P carries a bias of 2^7 (p <= 2^8 under the lazy rescale), which
+//   cancels between O and the row sum.
+//
+// * "Wide" units: an fp16 P also drops weights below 2^-32 of the row's reference maximum, which
+//   is harmless unless such a key carries a value many orders above the others: at max|v| = 2^20
+//   a dropped key is worth at most 2^-12 in the output, the value flush above 2^-19.  When the
+//   maximum is 2^20 or more the blocks of
+//   such a unit -- and every block when the cache was created with SPKV_FLAG_PREFILL_PV_BF16 --
+//   leave the values in bf16 and split P into hi + lo bf16 terms (16 significant bits, bf16's
+//   exponent range): 8 P.V MMAs per page instead of 4, one P buffer per head instead of two (a
+//   group then waits for P.V of the previous page before it overwrites P).  Same pipeline, same
+//   barriers; the branch is uniform per block.
 //
 // * P has tensor-memory columns of its own instead of overwriting the scores it came from.  A
 //   group copies its row of S into registers and hands the S buffer back at once, so Q.K^T of the
@@ -21,7 +35,8 @@
 //   formed one dependent loop whose latency, not the tensor pipe, set the pace.
 //
 // Tensor memory (512 columns): S of head h at [64 h, +64); P buffer b of head h at
-// [128 + 32 (2h + b), +32) (two fp16 per column); O of head h at [256 + 128 h, +128).
+// [128 + 32 (2h + b), +32) (two fp16 per column; a wide unit: hi at [128 + 64 h, +32), lo in the
+// 32 columns after it); O of head h at [256 + 128 h, +128).
 // MMA order per page j:  QK0(j+1) | PV0(j) | QK1(j+1) | PV1(j).  The two heads' scores become
 // ready half a page apart, which keeps the two groups out of step: the exponentials of one
 // (special-function unit, the scarce resource) run under the load / maximum / hand-over phases of
@@ -33,8 +48,6 @@
 //
 // No unit is saturated (tensor pipe ~54 % active, special-function unit ~41 %, issue slots ~54 %):
 // the page period is the length of the chain scores -> softmax -> P -> MMA warp -> next scores.
-// (Computing part of the exponentials by polynomial on the FMA pipe, which helps when the
-// special-function unit is the limit, only added instructions here and was dropped.)
 // Shared memory: Q of both heads (64 KB) + 5 page stages.
 // Warps: 0 MMA issue, 1 page loader + TMEM allocation, 2-3 value conversion, 4-7 group 0,
 // 8-11 group 1.  All waits are bounded.
@@ -101,15 +114,18 @@ __device__ inline WalkSlots walk_slots(const PrefillArgs &a, int walk) {
   }
   return w;
 }
-// the power of two that brings the unit's largest |v| into [2^14, 2^15), and its inverse
-__device__ inline void value_scale(const CacheView &c, int u, float &v_scale, float &v_unscale) {
+// Is the unit "wide" (two-term bf16 P.V), and otherwise the power of two that brings the largest
+// visible |v| into [2^14, 2^15), with its inverse.  vm: fp32 bit pattern of that largest |v|.
+constexpr uint32_t kWideFrom = 0x49800000u;   // 2^20
+__device__ inline bool value_scale(uint32_t vm, int force_wide, float &v_scale, float &v_unscale) {
   v_scale = v_unscale = 1.f;
-  const uint32_t vm = c.vmax[u];
+  if (force_wide || vm >= kWideFrom) return true;
   if (vm) {
     const int k = min(14 - ((int)(vm >> 23) - 127), 126);
     v_scale = __int_as_float((127 + k) << 23);
     v_unscale = __int_as_float((127 - k) << 23);
   }
+  return false;
 }
 
 // kEvenG: every block is a head pair on one tile (the branches for single heads compile away).
@@ -131,11 +147,10 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
   const int32_t *E = hdr + kHdrInts;
   const int len0 = hdr[H_LEN0], n_old = hdr[H_NOLD], N = hdr[H_N];
   const int u = unit_index(c, a.layer, a.seq, kvh);
-  // The values are multiplied by 2^k with the unit's largest |v| brought into [2^14, 2^15) (every
-  // value the unit holds or this chunk brings is covered by vmax); the epilogue multiplies by
-  // 2^-k.  Both are exact.
+  // fp16 P.V: the values are multiplied by 2^k with the largest visible |v| brought into
+  // [2^14, 2^15); the epilogue multiplies by 2^-k.  A wide unit keeps bf16 values (factor 1).
   float v_scale, v_unscale;
-  value_scale(c, u, v_scale, v_unscale);
+  const bool wide = value_scale((uint32_t)hdr[H_VMAX], a.force_wide, v_scale, v_unscale);
   // kept pairs visible to chunk query i: the first nvis(i) pairs of the compact cache
   auto nvis = [&](int i) { return len0 + E[min(max(i + n_old - c.w + 1, 0), N)]; };
   // the last query of the block (slot 1 never starts before slot 0) sees the most kept pairs
@@ -216,7 +231,8 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
     for (int base = 0; base < n_tiles && !failed; base += 32) {
       const int jl = j_begin + base + lane;
       int64_t src_off = 0;
-      if (jl < n_ptiles) src_off = (int64_t)c.table[(size_t)u * c.max_pages + jl] * kPageElems;
+      if (jl < n_ptiles)   // (debug bounds: an entry that names no pool page is read from the unit's ring instead)
+        src_off = (int64_t)checked_page(c, c.table[(size_t)u * c.max_pages + jl], (int)ring_page(c, u, 0)) * kPageElems;
       const int cnt = min(32, n_tiles - base);
       for (int x = 0; x < cnt; ++x, ++j) {
         const int64_t off = __shfl_sync(0xffffffffu, src_off, x);
@@ -241,7 +257,8 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
         mbar_wait_bounded(&bar[B_KV_FULL + (k % kStages)], (k / kStages) & 1);
   } else if (warp == 0) {
     // ---------------------------------------------------------------- MMA issue (whole warp, one elected lane issues)
-    constexpr uint32_t idesc_qk = instr_desc(128, 64, false), idesc_pv = instr_desc(128, 128, true, true);
+    constexpr uint32_t idesc_qk = instr_desc(128, 64, false), idesc_pv = instr_desc(128, 128, true, true),
+                       idesc_pv_bf16 = instr_desc(128, 128, true, false);
     const uint32_t sQ = smem_u32(smem + kSQ);
     auto wait_page = [&](int jj) {
       if (!mbar_wait_bounded(&bar[B_KV_FULL + jj % kStages], (jj / kStages) & 1)) failed = true;
@@ -265,8 +282,12 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
       fence_after();
       if (failed) return;
       const uint32_t sV = smem_u32(smem + kSKV + (jj % kStages) * kPageBytes) + kBlockElems * 2;
-      umma_pv_page_f16(tbase + 256 + h * 128, tbase + 128 + (2 * h + (jj & 1)) * 32, smem_desc(sV, 8192, 1024), idesc_pv,
-                       jj > 0 ? 1u : 0u);
+      if (wide)
+        umma_pv_page(tbase + 256 + h * 128, tbase + 128 + h * 64, smem_desc(sV, 8192, 1024), idesc_pv_bf16,
+                     jj > 0 ? 1u : 0u);
+      else
+        umma_pv_page_f16(tbase + 256 + h * 128, tbase + 128 + (2 * h + (jj & 1)) * 32, smem_desc(sV, 8192, 1024),
+                         idesc_pv, jj > 0 ? 1u : 0u);
       // the last two P.V have no later Q.K^T whose S_FULL would vouch for their completion
       if (jj + 2 >= n_tiles) umma_commit(&bar[B_O_DONE + 2 * h + (jj & 1)]);
     };
@@ -302,14 +323,15 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
     }
   } else if (warp < 4) {
     // ---------------------------------------------------------------- value converter (warps 2-3)
-    // bf16 -> fp16 in place, in the swizzled layout the copy left (element positions do not move)
+    // bf16 -> fp16 in place, in the swizzled layout the copy left (element positions do not move);
+    // a wide unit's values stay as they are
     const int ct = tid - 64;
     for (int j = 0; j < n_tiles; ++j) {
       const int s = j % kStages;
       if (!mbar_wait_bounded(&bar[B_KV_FULL + s], (j / kStages) & 1)) { failed = true; break; }
       uint4 *vb = reinterpret_cast<uint4 *>(smem + kSKV + s * kPageBytes + kBlockElems * 2) + ct;
 #pragma unroll 8
-      for (int x = 0; x < 16; ++x) {
+      for (int x = 0; x < (wide ? 0 : 16); ++x) {
         uint4 r = vb[x * kConvThreads];
         r.x = bf16x2_to_f16x2(r.x, v_scale); r.y = bf16x2_to_f16x2(r.y, v_scale);
         r.z = bf16x2_to_f16x2(r.z, v_scale); r.w = bf16x2_to_f16x2(r.w, v_scale);
@@ -401,24 +423,56 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
       m_ref = m_new;
       TC5H_STAMP(traced && row == 0, h * 4 + 2, j);
       const float ms = m_ref == -INFINITY ? 0.f : m_ref;
-      // two elements per instruction where the hardware has a packed form (fma, add)
-      const uint64_t sc2 = pack2(a.scale_log2, a.scale_log2), nms2 = pack2(kPBias - ms, kPBias - ms);
+      // two elements per instruction where the hardware has a packed form (fma, add, sub)
+      const float bias = wide ? 0.f : kPBias;
+      const uint64_t sc2 = pack2(a.scale_log2, a.scale_log2), nms2 = pack2(bias - ms, bias - ms);
       uint64_t l2a = pack2(0.f, 0.f), l2b = l2a;
-      // P buffer (j & 1) is free: S_FULL(j) completed after P.V(j-2)
-      const uint32_t t_p = t_lane + 128 + (2 * h + (j & 1)) * 32;
-#pragma unroll
-      for (int q2 = 0; q2 < 2; ++q2) {  // 32 keys -> 16 columns of fp16 pairs
-        uint32_t ph[16];
-#pragma unroll
-        for (int x = 0; x < 16; ++x) {
-          float e0, e1;
-          unpack2(fma2(pack2(v[q2 * 32 + 2 * x], v[q2 * 32 + 2 * x + 1]), sc2, nms2), e0, e1);
-          const float p0 = fast_exp2(e0), p1 = fast_exp2(e1);
-          const uint64_t p2 = pack2(p0, p1);
-          if (x & 1) l2b = add2(l2b, p2); else l2a = add2(l2a, p2);
-          ph[x] = pack_f16(p0, p1);
+      if (wide) {
+        // one P buffer per head: P.V of the previous page must have read it.  Q.K^T(j+1) is issued
+        // after P.V(j-1) and needs nothing more from this group, so S_FULL(j+1) vouches for it
+        // (waiting on it here does not consume the phase); the last page has its own barrier.
+        if (j > 0 && !(j + 1 < n_tiles ? mbar_wait_bounded(&bar[B_S_FULL + h], (j + 1) & 1)
+                                       : mbar_wait_bounded(&bar[B_O_DONE + 2 * h + ((j - 1) & 1)], 0))) {
+          failed = true;
+          break;
         }
-        tmem_st16u(t_p + q2 * 16, ph);
+        fence_after();
+        const uint32_t t_p = t_lane + 128 + h * 64;
+#pragma unroll
+        for (int q2 = 0; q2 < 2; ++q2) {  // 32 keys -> 16 columns of hi, 16 of lo
+          uint32_t hi[16], lo[16];
+#pragma unroll
+          for (int x = 0; x < 16; ++x) {
+            float e0, e1, r0, r1;
+            unpack2(fma2(pack2(v[q2 * 32 + 2 * x], v[q2 * 32 + 2 * x + 1]), sc2, nms2), e0, e1);
+            const float p0 = fast_exp2(e0), p1 = fast_exp2(e1);
+            const uint64_t p2 = pack2(p0, p1);
+            if (x & 1) l2b = add2(l2b, p2); else l2a = add2(l2a, p2);
+            const __nv_bfloat162 hb = __floats2bfloat162_rn(p0, p1);
+            hi[x] = *reinterpret_cast<const uint32_t *>(&hb);
+            unpack2(sub2(p2, pack2(__uint_as_float(hi[x] << 16), __uint_as_float(hi[x] & 0xffff0000u))), r0, r1);
+            lo[x] = pack_bf16(r0, r1);
+          }
+          tmem_st16u(t_p + q2 * 16, hi);
+          tmem_st16u(t_p + 32 + q2 * 16, lo);
+        }
+      } else {
+        // P buffer (j & 1) is free: S_FULL(j) completed after P.V(j-2)
+        const uint32_t t_p = t_lane + 128 + (2 * h + (j & 1)) * 32;
+#pragma unroll
+        for (int q2 = 0; q2 < 2; ++q2) {  // 32 keys -> 16 columns of fp16 pairs
+          uint32_t ph[16];
+#pragma unroll
+          for (int x = 0; x < 16; ++x) {
+            float e0, e1;
+            unpack2(fma2(pack2(v[q2 * 32 + 2 * x], v[q2 * 32 + 2 * x + 1]), sc2, nms2), e0, e1);
+            const float p0 = fast_exp2(e0), p1 = fast_exp2(e1);
+            const uint64_t p2 = pack2(p0, p1);
+            if (x & 1) l2b = add2(l2b, p2); else l2a = add2(l2a, p2);
+            ph[x] = pack_f16(p0, p1);
+          }
+          tmem_st16u(t_p + q2 * 16, ph);
+        }
       }
       {
         float la, lb;
@@ -507,7 +561,7 @@ __global__ void __launch_bounds__(256) prefill_merge_kernel(PrefillArgs a) {
   if (h == 1 && !ws.two) return;
   const int hq = h ? ws.hq1 : ws.hq0, i0 = h ? ws.i01 : ws.i00;
   float v_scale, v_unscale;
-  value_scale(c, unit_index(c, a.layer, a.seq, ws.kvh), v_scale, v_unscale);
+  value_scale((uint32_t)unit_ws(a, ws.kvh)[H_VMAX], a.force_wide, v_scale, v_unscale);
   const float *part = a.partials + (size_t)(walk * 2 + h) * S * kPartFloats;
   __shared__ float s_w[kMaxSplit][128];   // weight of share s for a row, already divided by the row sum
   for (int row = threadIdx.x; row < 128; row += blockDim.x) {

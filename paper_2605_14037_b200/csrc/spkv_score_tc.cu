@@ -245,12 +245,8 @@ namespace spkv {
 // covers (the caller then uses the CUDA-core kernel), < 0 on error.
 int launch_score_mlp_tc(spkv_cache *cache, const spkv_predictor_t *p, const void *d_x, int n_tok, float *d_logits,
                         uint8_t *d_flags, cudaStream_t s) {
-  static const bool off = [] {
-    const char *e = getenv("SPKV_SCORE_KERNEL");  // "simt": always the CUDA-core kernel
-    return e && e[0] == 's';
-  }();
   const int Hkv = cache->view.Hkv, heads8 = (Hkv + 7) & ~7;
-  if (off || n_tok < 64 || p->hidden < 16 || p->hidden > sctc::kMaxHidden || (p->hidden & 15) ||
+  if (n_tok < 64 || p->hidden < 16 || p->hidden > sctc::kMaxHidden || (p->hidden & 15) ||
       p->hidden * heads8 > sctc::kMaxW2Floats || (p->d_in & 7) || ((uintptr_t)d_x & 15) || ((uintptr_t)p->d_W1 & 15) ||
       !encode_tiled())
     return 1;

@@ -48,9 +48,45 @@ __global__ void __launch_bounds__(32) stream_read_kernel(const unsigned char *bu
   atomicAdd(sink, sum);
 }
 
+// Self-test of the bounded waits, the error path every copy pipeline of the library shares: one
+// thread arms an mbarrier for 64 bytes more than the one 32 KB bulk copy it issues will ever
+// deliver, so the wait must run out after `limit` clocks.  It then records SPKV_E_TIMEOUT,
+// closes the phase by counting the missing bytes in itself and waits (bounded again, default
+// limit) for the copy that IS in flight, so that nothing lands in shared memory after the block
+// has gone -- what the real kernels do before they leave.  status: [0] SPKV_E_TIMEOUT if the first
+// wait ran out, 0 if it did not; [1] 1 if the copy was then seen complete; [2] clocks the first
+// wait lasted; [3] 1 if the first word in shared memory equals the first word of the buffer.
+__global__ void __launch_bounds__(32) wait_selftest_kernel(const unsigned char *buf, long long limit, int *status) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  uint64_t *bar = reinterpret_cast<uint64_t *>(smem + kPageBytes);
+  if (threadIdx.x != 0) return;
+  mbar_init(bar, 1);
+  mbar_fence_init();
+  mbar_arrive_expect_tx(bar, kPageBytes + 64);
+  bulk_load(smem, buf, kPageBytes, bar);
+  const long long t0 = clock64();
+  const bool arrived = mbar_wait_bounded(bar, 0, limit);
+  status[2] = (int)min(clock64() - t0, (long long)0x7fffffff);
+  status[0] = arrived ? 0 : SPKV_E_TIMEOUT;
+  if (!arrived) mbar_complete_tx(bar, 64);
+  const bool drained = mbar_wait_bounded(bar, 0);
+  status[1] = drained ? 1 : 0;
+  status[3] = drained && *reinterpret_cast<const unsigned int *>(smem) == *reinterpret_cast<const unsigned int *>(buf);
+}
+
 }  // namespace spkv
 
 using namespace spkv;
+
+extern "C" int spkv_wait_selftest(const void *d_buf, long long limit_clocks, int32_t *d_status, spkv_stream_t stream) {
+  if (!d_buf || !d_status || ((uintptr_t)d_buf & 15) || limit_clocks < 1) return SPKV_E_INVALID;
+  if (cudaFuncSetAttribute(wait_selftest_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPageBytes + 64) !=
+      cudaSuccess)
+    return SPKV_E_CUDA;
+  wait_selftest_kernel<<<1, 32, kPageBytes + 64, as_stream(stream)>>>(static_cast<const unsigned char *>(d_buf),
+                                                                     limit_clocks, d_status);
+  return check_stream_error(cudaGetLastError());
+}
 
 extern "C" int spkv_stream_read(const void *d_buf, size_t bytes, unsigned long long *d_sink, int32_t *d_status,
                                 spkv_stream_t stream) {

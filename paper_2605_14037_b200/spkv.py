@@ -23,11 +23,14 @@ SPKV_OK = 0
 ERRORS = {
     -1: "SPKV_E_INVALID", -2: "SPKV_E_ARENA_TOO_SMALL", -3: "SPKV_E_UNSUPPORTED", -4: "SPKV_E_CUDA",
     -5: "SPKV_E_POOL_EXHAUSTED", -6: "SPKV_E_CONTEXT_OVERFLOW", -7: "SPKV_E_WORKSPACE",
-    -8: "SPKV_E_TIMEOUT", -9: "SPKV_E_BOUNDS", -10: "SPKV_E_SCRATCH_LIMIT", -11: "SPKV_E_ORDER_DECODE", -12: "SPKV_E_ORDER_APPEND",
+    -8: "SPKV_E_TIMEOUT", -9: "SPKV_E_BOUNDS", -10: "SPKV_E_SCRATCH_LIMIT", -11: "SPKV_E_ORDER_DECODE",
+    -12: "SPKV_E_ORDER_APPEND", -13: "SPKV_E_BOUNDS_PAGE", -14: "SPKV_E_CANARY", -15: "SPKV_E_ATTACH",
 }
 
 
-FLAG_OVERLAP = 1   # SPKV_FLAG_OVERLAP
+FLAG_OVERLAP = 1          # SPKV_FLAG_OVERLAP
+FLAG_PREFILL_PV_BF16 = 2  # SPKV_FLAG_PREFILL_PV_BF16
+FLAG_DEBUG_BOUNDS = 4      # SPKV_FLAG_DEBUG_BOUNDS
 
 
 class Config(C.Structure):
@@ -74,6 +77,14 @@ def lib():
     protos = {
         "spkv_arena_bytes": (C.c_int, [cfgp, C.POINTER(sz)]),
         "spkv_cache_create": (C.c_int, [cfgp, vp, sz, vp, C.POINTER(vp)]),
+        "spkv_cache_attach": (C.c_int, [cfgp, vp, sz, vp, C.POINTER(vp)]),
+        "spkv_cache_checkpoint_bytes": (sz, [vp]),
+        "spkv_cache_checkpoint": (C.c_int, [vp, vp, sz, vp]),
+        "spkv_cache_rollback": (C.c_int, [vp, vp, sz, vp]),
+        "spkv_note_foreign_work": (C.c_int, [vp]),
+        "spkv_safe_steps": (C.c_int, [vp, vp, i32, vp, C.POINTER(C.c_int64)]),
+        "spkv_safe_steps_from_lengths": (C.c_int, [cfgp, vp, vp, C.c_int64, C.c_int64, C.POINTER(C.c_int64)]),
+        "spkv_arena_canaries": (C.c_int, [cfgp, C.POINTER(sz), i32, C.POINTER(i32)]),
         "spkv_cache_destroy": (C.c_int, [vp]),
         "spkv_cache_reset_seq": (C.c_int, [vp, i32, vp]),
         "spkv_set_tau": (C.c_int, [vp, f32]),
@@ -84,6 +95,7 @@ def lib():
         "spkv_decode_workspace_bytes": (sz, [cfgp, i32]),
         "spkv_decode_attention": (C.c_int, [vp, i32, vp, i32, vp, vp, vp, f32, vp, sz, vp]),
         "spkv_stream_read": (C.c_int, [vp, sz, vp, vp, vp]),
+        "spkv_wait_selftest": (C.c_int, [vp, C.c_longlong, vp, vp]),
         "spkv_decode_attention_f32": (C.c_int, [vp, i32, vp, i32, vp, vp, vp, vp, f32, vp, sz, vp]),
         "spkv_decode_attention_static": (C.c_int, [vp, i32, vp, i32, vp, vp, vp, f32, vp]),
         "spkv_prefill_workspace_bytes": (sz, [cfgp, i32]),
@@ -164,6 +176,51 @@ class Cache:
         self._ws = {}
         self.G = n_q_heads // n_kv_heads
         self.default_scale = 1.0 / math.sqrt(head_dim)
+
+    @classmethod
+    def attach(cls, arena, cfg, tau=None, flags=None):
+        """A Cache over an arena tensor that already holds one (a copy of another cache's arena):
+        spkv_cache_attach.  `cfg` is the Config the arena was created with; tau / flags override."""
+        self = cls.__new__(cls)
+        self.cfg = Config.from_buffer_copy(cfg)
+        if tau is not None:
+            self.cfg.tau = tau
+        if flags is not None:
+            self.cfg.flags = flags
+        self.device = arena.device
+        self.arena, self.arena_bytes = arena, arena.numel()
+        h = C.c_void_p()
+        with torch.cuda.device(self.device):
+            _check(lib().spkv_cache_attach(C.byref(self.cfg), _ptr(arena), arena.numel(), _stream(), C.byref(h)),
+                   "spkv_cache_attach")
+        self._h, self._ws = h, {}
+        self.G = self.cfg.n_q_heads // self.cfg.n_kv_heads
+        self.default_scale = 1.0 / math.sqrt(self.cfg.head_dim)
+        return self
+
+    def spkv_cache_checkpoint(self, buf=None, stream=None):
+        """Saves metadata + ring pages into `buf` (allocated when None); returns the buffer."""
+        n = lib().spkv_cache_checkpoint_bytes(self._h)
+        if buf is None:
+            buf = torch.empty(n, dtype=torch.uint8, device=self.device)
+        _check(lib().spkv_cache_checkpoint(self._h, _ptr(buf), buf.numel(), _stream(stream)), "spkv_cache_checkpoint")
+        return buf
+
+    def spkv_cache_rollback(self, buf, stream=None):
+        _check(lib().spkv_cache_rollback(self._h, _ptr(buf), buf.numel(), _stream(stream)), "spkv_cache_rollback")
+
+    def spkv_note_foreign_work(self):
+        _check(lib().spkv_note_foreign_work(self._h), "spkv_note_foreign_work")
+
+    def spkv_safe_steps(self, seq_ids=None, stream=None) -> int:
+        """Decode steps the listed sequences (host ints; None = all) can take before the pool or a
+        page table could run out, every evicted pair assumed kept."""
+        import numpy as np
+        ids = np.ascontiguousarray(np.asarray([] if seq_ids is None else seq_ids, dtype=np.int32))
+        out = C.c_int64()
+        _check(lib().spkv_safe_steps(self._h, ids.ctypes.data if ids.size else None, int(ids.size),
+                                     _stream(stream), C.byref(out)), "spkv_safe_steps")
+        return int(out.value)
 
     def close(self):
         if getattr(self, "_h", None):
@@ -390,8 +447,17 @@ def spkv_stream_read(buf, passes=5, stream=None):
     e1.record()
     e1.synchronize()
     if int(status.item()) != 0:
-        raise SpkvError(f"spkv_stream_read: {ERRORS.get(int(status.item()), status.item())}")
+        raise SpkvError(int(status.item()), "spkv_stream_read")
     return nbytes * passes / (e0.elapsed_time(e1) * 1e-3) / 1e9
+
+
+def spkv_wait_selftest(buf, limit_clocks, stream=None):
+    """Runs the library's bounded-wait error path once (see spkv.h); returns the four status
+    words [code, drained, clocks waited, data in place] as a list."""
+    status = torch.zeros(4, dtype=torch.int32, device=buf.device)
+    _check(lib().spkv_wait_selftest(_ptr(buf), int(limit_clocks), _ptr(status), _stream(stream)),
+           "spkv_wait_selftest")
+    return status.cpu().tolist()
 
 
 def bf16_from_bits(bits, device):

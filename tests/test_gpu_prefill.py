@@ -257,3 +257,82 @@ def test_small_chunks_on_a_long_past_split_their_page_walks(G, Hkv, small):
         u = oracle.Unit(w, D)
         u.prefill(Kh, Vh, Lh, tl)
         compare_state(cache, 0, 0, h, u)
+
+
+@pytest.mark.parametrize("G,Hkv,w", [(4, 2, 128), (3, 2, 100), (1, 3, 128), (8, 1, 4)])
+def test_prefill_with_two_term_bf16_weights(G, Hkv, w):
+    """SPKV_FLAG_PREFILL_PV_BF16: every unit multiplies the softmax weights into the values as
+    two bf16 terms (the form a unit with a very wide value range takes by itself).  Same chunkings,
+    same oracle, same tolerance as the default path; even and odd groups, a partially filled first
+    chunk, a one-token chunk."""
+    spkv = load()
+    T, Hq = 700, G * Hkv
+    rates = [0.25, 0.7, 0.5][:Hkv]
+    cache = spkv.Cache(n_layers=1, max_seqs=1, n_q_heads=Hq, n_kv_heads=Hkv, max_context=2048,
+                       pool_pages=40 + 12 * Hkv, window=w, tau=0.5, flags=spkv.FLAG_PREFILL_PV_BF16)
+    tl = cache.spkv_tau_logit()
+    wl = Workload(910 + w + G, T, 1, Hq, Hkv, rates, tl)
+    got = prefill_in_chunks(spkv, cache, 0, 0, wl, 0, [70, 1, 200, 129, 300])
+    assert cache.spkv_status() == 0
+    units, ref = oracle_prefill(wl, 0, w, tl, G, T, 1.0 / math.sqrt(D))
+    for h in range(Hkv):
+        compare_state(cache, 0, 0, h, units[h])
+    assert_attn_close(got, ref, f"two-term bf16, w={w} G={G}")
+
+
+def test_two_term_bf16_weights_on_split_page_walks_and_rescaled_rows():
+    """The flag on the two harder paths: page walks cut into shares (a small chunk on a 20 k past)
+    and rows whose accumulator is rescaled on every page (scores growing with position)."""
+    from paper_2605_14037_b200 import synth
+    spkv = load()
+    w, T0, G, Hkv = 128, 20000, 4, 2
+    Hq, small = G * Hkv, [48, 130]
+    T = T0 + sum(small)
+    rates = [0.05, 0.6]
+    cache = spkv.Cache(n_layers=1, max_seqs=1, n_q_heads=Hq, n_kv_heads=Hkv, max_context=32768,
+                       pool_pages=int(sum(rates) * T / 64) + 3 * Hkv + 8, window=w, tau=0.5,
+                       flags=spkv.FLAG_PREFILL_PV_BF16)
+    tl = cache.spkv_tau_logit()
+    wl = Workload(5100, T, 1, Hq, Hkv, rates, tl)
+    Kf = synth.bf16_bits_to_f32(wl.K)
+    Kf[T0 - 1500:, 0, 1, 0] = 0.25 * np.arange(1500 + sum(small), dtype=np.float32)   # KV head 1: scores grow
+    wl.K = synth.to_bf16_bits(Kf)
+    qf = synth.bf16_bits_to_f32(wl.q)
+    qf[:, 0, G, :] = 0.0
+    qf[:, 0, G, 0] = 8.0                    # first query head of KV head 1 looks at that dimension only
+    wl.q = synth.to_bf16_bits(qf)
+    prefill_in_chunks(spkv, cache, 0, 0, wl, 0, [8192, 8192, T0 - 16384], with_q=False)
+    K, V, Q = to_dev_bf16(wl.K[:, 0]), to_dev_bf16(wl.V[:, 0]), to_dev_bf16(wl.q[:, 0])
+    lg = torch.from_numpy(np.ascontiguousarray(wl.logit[:, 0])).to(dev())
+    outs, a = [], T0
+    for c in small:
+        outs.append(spkv.bits_from_bf16(cache.spkv_prefill(0, 0, K[a:a + c], V[a:a + c], lg[a:a + c], q=Q[a:a + c])))
+        a += c
+    assert cache.spkv_status() == 0
+    out = np.concatenate(outs)
+    scale = 1.0 / math.sqrt(D)
+    for h in range(Hkv):
+        Kh, Vh, Lh = (np.ascontiguousarray(x) for x in (wl.K[:, 0, h], wl.V[:, 0, h], wl.logit[:, 0, h]))
+        for t in range(T0, T, 2):
+            ref = oracle.mask_attend_row(Kh, Vh, Lh, t, w, tl, np.ascontiguousarray(wl.q[t, 0, h * G:(h + 1) * G]), scale)
+            assert_attn_close(out[t - T0, h * G:(h + 1) * G], ref, f"t={t} kvh={h}")
+
+
+@pytest.mark.parametrize("scale", [0.0, -0.1, float("inf"), float("nan")])
+def test_prefill_refuses_a_scale_that_is_not_positive_and_finite(scale):
+    """The chunk attention takes row maxima before scaling, which needs a positive scale: any other
+    value is an argument error, reported before anything is launched (the cache is unchanged).
+    Building the state only (no queries) does not look at the scale."""
+    spkv = load()
+    cache = spkv.Cache(n_layers=1, max_seqs=1, n_q_heads=4, n_kv_heads=2, max_context=1024,
+                       pool_pages=8, window=16, tau=0.5)
+    wl = Workload(77, 40, 1, 4, 2, [0.5, 0.5], cache.spkv_tau_logit())
+    K, V, Q = to_dev_bf16(wl.K[:, 0]), to_dev_bf16(wl.V[:, 0]), to_dev_bf16(wl.q[:, 0])
+    lg = torch.from_numpy(np.ascontiguousarray(wl.logit[:, 0])).to(dev())
+    with pytest.raises(spkv.SpkvError) as e:
+        cache.spkv_prefill(0, 0, K, V, lg, q=Q, sm_scale=scale)
+    assert e.value.code == -1
+    ln, tt = cache.spkv_read_lengths(0)
+    assert (tt == 0).all() and (ln == 0).all() and cache.spkv_status() == 0
+    cache.spkv_prefill(0, 0, K, V, lg, sm_scale=scale)          # state only
+    assert cache.spkv_status() == 0 and (cache.spkv_read_lengths(0)[1] == 40).all()

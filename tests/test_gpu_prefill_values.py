@@ -1,9 +1,11 @@
-"""GPU parity of the chunk attention under value ranges far from 1.  The paired tcgen05 kernel
+"""GPU parity of the chunk attention under value ranges far from 1.  The tcgen05 kernel
 multiplies P.V in fp16 after scaling the values by a power of two chosen from the largest |v|
-the unit has received; these cases make that scale matter: values near the top and the bottom
-of the bf16 range (a different one per KV head), a range that grows between chunks through
-appended tokens, and a sequence reset that has to forget the old range.  The tolerance is
-the usual one in units of the head's value scale."""
+its queries can see, and switches a unit to two bf16 terms when that maximum reaches 2^20; these
+cases make that matter: values near the top and the bottom of the bf16 range (a different one
+per KV head), a range that grows between chunks through appended tokens, a sequence reset that
+has to forget the old range -- all with the usual tolerance in units of the head's value scale
+-- and, at the plain tolerance of every other attention test, a single outlier among ordinary
+values: kept and visible, or discarded long before the queries that are checked."""
 import math
 
 import numpy as np
@@ -11,7 +13,7 @@ import pytest
 import torch
 
 import oracle
-from gpu_util import ABS_TOL, D, REL_TOL, Workload, compare_state, dev, load, to_dev_bf16
+from gpu_util import ABS_TOL, D, REL_TOL, Workload, assert_attn_close, compare_state, dev, load, to_dev_bf16
 from paper_2605_14037_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -97,3 +99,73 @@ def test_reset_forgets_the_value_range():
                         np.ascontiguousarray(wl.q[:, 0, h * G:(h + 1) * G]), sm)
         compare_state(cache, 0, 0, h, u)
         assert_close_scaled(out[:, h * G:(h + 1) * G], ref, 2.0 ** -20, f"after reset head {h}")
+
+
+def outlier_case(spkv, spread_log2, kept, flags=0, seed=77):
+    """N(0,1) values with ONE element of 2^spread_log2 in each KV head, at position 40 (dimension 5
+    of head 0, dimension 100 of head 1).  kept: the outlier's logit passes the threshold, so it
+    stays visible for ever; otherwise it is discarded when it leaves the window, 600 positions
+    before the first query that is checked.  Returns outputs of the last two chunks and the
+    oracle's, every element to be held to the plain tolerance."""
+    w, Hq, Hkv, G = 64, 4, 2, 2
+    chunks = [300, 40, 500, 300]
+    T = sum(chunks)
+    cache = spkv.Cache(n_layers=1, max_seqs=1, n_q_heads=Hq, n_kv_heads=Hkv, max_context=2048,
+                       pool_pages=48, window=w, tau=0.5, flags=flags)
+    tl = cache.spkv_tau_logit()
+    wl = Workload(seed, T, 1, Hq, Hkv, [0.3, 0.6], tl)
+    Vf = synth.bf16_bits_to_f32(wl.V)
+    Vf[40, 0, 0, 5] = np.float32(2.0 ** spread_log2)
+    Vf[40, 0, 1, 100] = np.float32(-(2.0 ** spread_log2))
+    wl.V = synth.to_bf16_bits(Vf)
+    wl.logit[40, 0, :] = np.float32(tl + 3.0) if kept else np.float32(tl - 3.0)
+    sm = 1.0 / math.sqrt(D)
+    refs, units = [], []
+    for h in range(Hkv):
+        u = oracle.Unit(w, D)
+        refs.append(u.prefill(np.ascontiguousarray(wl.K[:, 0, h]), np.ascontiguousarray(wl.V[:, 0, h]),
+                              np.ascontiguousarray(wl.logit[:, 0, h]), tl,
+                              np.ascontiguousarray(wl.q[:, 0, h * G:(h + 1) * G]), sm))
+        units.append(u)
+    K, V, Q = to_dev_bf16(wl.K), to_dev_bf16(wl.V), to_dev_bf16(wl.q)
+    lg = torch.from_numpy(wl.logit).to(dev())
+    ids = torch.zeros(1, dtype=torch.int32, device=dev())
+    outs, a = [], 0
+    for ci, c in enumerate(chunks):
+        if ci == 1:                      # the second stretch goes token by token through the append
+            for t in range(a, a + c):
+                cache.spkv_append_evict(0, ids, K[t], V[t], lg[t])
+            outs.append(None)
+        else:
+            outs.append(spkv.bits_from_bf16(cache.spkv_prefill(0, 0, K[a:a + c, 0], V[a:a + c, 0],
+                                                               lg[a:a + c, 0].contiguous(), q=Q[a:a + c, 0])))
+        a += c
+    assert cache.spkv_status() == 0
+    for h in range(Hkv):
+        compare_state(cache, 0, 0, h, units[h])
+    a2 = chunks[0] + chunks[1]
+    ref = np.concatenate(refs, axis=1)
+    return (np.concatenate(outs[2:]), ref[a2:]), (outs[0], ref[:chunks[0]])
+
+
+@pytest.mark.parametrize("spread_log2,kept", [(19, True), (20, True), (20, False), (35, True), (35, False),
+                                              (100, True), (100, False)])
+def test_one_outlier_among_ordinary_values_meets_the_plain_tolerance(spread_log2, kept):
+    """A 2^19 outlier keeps the unit on the fp16 path (every N(0,1) value of any weight stays a
+    normal fp16 number after the scaling); 2^20 and more make it a wide unit while the outlier is visible
+    (two bf16 terms, no scaling); once the outlier has been discarded the unit is an ordinary
+    one again and must be as accurate as if it had never seen it."""
+    spkv = load()
+    (late, late_ref), (first, first_ref) = outlier_case(spkv, spread_log2, kept)
+    assert_attn_close(late, late_ref, f"2^{spread_log2} kept={kept}: queries long after the outlier")
+    assert_attn_close(first, first_ref, f"2^{spread_log2} kept={kept}: chunk that holds the outlier")
+    if not kept:    # the outlier is invisible to the late queries: outputs of ordinary size
+        assert np.abs(late_ref).max() < 8.0
+
+
+def test_two_term_bf16_flag_meets_the_plain_tolerance_too():
+    spkv = load()
+    for kept in (True, False):
+        (late, late_ref), (first, first_ref) = outlier_case(spkv, 12, kept, flags=spkv.FLAG_PREFILL_PV_BF16)
+        assert_attn_close(late, late_ref, f"flag, kept={kept}: late queries")
+        assert_attn_close(first, first_ref, f"flag, kept={kept}: first chunk")

@@ -40,3 +40,24 @@ def test_stream_read_rejects_bad_arguments_and_ignores_less_than_a_page():
     assert f(C.c_void_p(buf.data_ptr() + 4), 36000, C.c_void_p(sink.data_ptr()), C.c_void_p(status.data_ptr()), s) != 0
     assert f(C.c_void_p(buf.data_ptr()), 1000, C.c_void_p(sink.data_ptr()), C.c_void_p(status.data_ptr()), s) == 0
     assert spkv.spkv_stream_read(buf, passes=2) > 0
+
+
+def test_a_bounded_wait_runs_out_and_the_context_stays_usable():
+    """Failure path without a fault: a barrier armed for more bytes than its copy delivers.  The
+    wait gives up after the limit it was given (about a millisecond here), the kernel reports
+    SPKV_E_TIMEOUT, waits for the copy it has in flight and returns; the next calls on the same
+    context work as if nothing had happened."""
+    spkv = load()
+    words = np.arange(8192 * 2, dtype=np.uint32) + 77
+    buf = torch.from_numpy(words.view(np.uint8).copy()).to(dev())
+    limit = 2_000_000                      # clocks: ~1 ms at ~2 GHz
+    code, drained, waited, data_ok = spkv.spkv_wait_selftest(buf, limit)
+    assert code == -8 and spkv.lib().spkv_error_string(code) == b"bounded device wait ran out"
+    assert drained == 1 and data_ok == 1
+    assert limit <= waited < 50 * limit, waited
+    # a second run gives the same answer, and ordinary work follows without an error
+    assert spkv.spkv_wait_selftest(buf, limit // 4)[:2] == [-8, 1]
+    assert torch.cuda.current_stream().query() in (True, False)
+    torch.cuda.synchronize()
+    assert spkv.spkv_stream_read(buf, passes=1) > 0
+    assert spkv.lib().spkv_wait_selftest(None, limit, None, None) == -1

@@ -92,3 +92,73 @@ def test_workspace_sizes_and_error_strings(spkv):
     assert l.spkv_cache_destroy(None) == -1
     assert l.spkv_set_tau(None, 0.5) == -1
     assert l.spkv_status(None, None) == -1
+
+
+def brute_force_safe_steps(w, max_context, lens, ts, pages_free, cap=5000):
+    """Steps n = 1, 2, ... with every evicted pair kept, page by page, until a unit would need a
+    page the pool no longer has or its table has no room for."""
+    lens, ts, free = list(lens), list(ts), pages_free
+    max_pages = (max_context + 63) // 64
+    for n in range(cap):
+        for u in range(len(lens)):
+            if ts[u] >= w:                      # the pair of position t - w leaves the window and is kept
+                if lens[u] % 64 == 0:
+                    if lens[u] // 64 >= max_pages or free == 0:
+                        return n
+                    free -= 1
+                lens[u] += 1
+            ts[u] += 1
+    return cap
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_safe_step_budget_equals_a_page_by_page_simulation(spkv, seed):
+    """The safe-step budget of the paper's inference appendix: the closed-form count the library
+    uses against a literal simulation of the worst case."""
+    import numpy as np
+    rng = np.random.default_rng(seed)
+    w = int(rng.choice([1, 16, 128, 200]))
+    n_units = int(rng.integers(1, 12))
+    ts = rng.integers(0, 3 * w + 5, size=n_units).astype(np.int32)
+    lens = np.array([rng.integers(0, max(t - w, 0) + 1) for t in ts], dtype=np.int32)
+    free = int(rng.integers(0, 12))
+    max_context = int(rng.choice([256, 1024, 1 << 20]))
+    c = cfg(spkv, window=w, max_context=max_context)
+    out = C.c_int64()
+    rc = spkv.lib().spkv_safe_steps_from_lengths(C.byref(c), lens.ctypes.data, ts.ctypes.data, n_units, free,
+                                                 C.byref(out))
+    assert rc == 0
+    assert out.value == brute_force_safe_steps(w, max_context, lens, ts, free), (w, lens, ts, free)
+
+
+def test_safe_step_budget_special_cases(spkv):
+    import numpy as np
+    c = cfg(spkv, window=128, max_context=1 << 20)
+    out = C.c_int64()
+    f = spkv.lib().spkv_safe_steps_from_lengths
+
+    def one(ln, t, free):
+        a, b = np.array([ln], np.int32), np.array([t], np.int32)     # kept alive across the call
+        return f(C.byref(c), a.ctypes.data, b.ctypes.data, 1, free, C.byref(out)), out.value
+
+    assert one(0, 0, 0) == (0, 128)           # an empty unit evicts nothing for w steps
+    assert one(0, 128, 0) == (0, 0)           # the next step may need a page and none is free
+    assert one(1, 500, 0) == (0, 63)          # 63 rows left in the unit's last page
+    assert one(64, 500, 1) == (0, 64)         # one page buys 64 steps
+    assert one(0, 0, 3) == (0, 128 + 3 * 64)
+    assert f(C.byref(c), None, None, 1, 0, C.byref(out)) == -1
+    empty = np.zeros(1, np.int32)
+    assert f(C.byref(c), empty.ctypes.data, empty.ctypes.data, 0, 0, C.byref(out)) == 0
+    assert out.value == 1 << 31               # nothing to count: no limit
+
+
+def test_canary_blocks_lie_between_the_metadata_regions(spkv):
+    c = cfg(spkv)
+    n, total = C.c_int32(), C.c_size_t()
+    offs = (C.c_size_t * 16)()
+    assert spkv.lib().spkv_arena_canaries(C.byref(c), offs, 16, C.byref(n)) == 0
+    assert spkv.lib().spkv_arena_bytes(C.byref(c), C.byref(total)) == 0
+    o = list(offs)[:n.value]
+    assert n.value == 10 and o == sorted(o) and o[0] == 256 and all(x % 256 == 0 for x in o)
+    units = 2 * 3 * 2
+    assert o[-1] + 256 <= total.value - (units * 2 + 100) * 32768     # all before the pages

@@ -33,6 +33,19 @@ MUTANTS = [
     ("silu_is_plain_sigmoid", "a[j] = z * orc_sigmoid(z);", "a[j] = orc_sigmoid(z);", 1),
     ("tau_logit_sign", "return (float)log(tau / (1.0 - tau));", "return (float)log((1.0 - tau) / tau);", 1),
     ("softmax_without_normalisation", "double p = exp(score[s] - mx) / denom;", "double p = exp(score[s] - mx);", 1),
+    ("soft_gate_inside_the_window_too", "else if (t - s < w) bias_ts = 0.0;", "else if (t - s < 0) bias_ts = 0.0;", 1),
+    ("soft_window_one_too_wide", "else if (t - s < w) bias_ts = 0.0;", "else if (t - s <= w) bias_ts = 0.0;", 1),
+    ("soft_future_visible", "if (s > t) bias_ts = -INFINITY;", "if (s > t + 1) bias_ts = -INFINITY;", 1),
+    ("soft_gate_without_logarithm", "return log(u_tilde);", "return u_tilde - 1.0;", 1),
+    ("soft_gate_dropped_term", ": l - log1p(exp(l));", ": -log1p(exp(l));", 1),
+    ("anneal_weights_swapped", "double u_tilde = (1.0 - alpha) * u + alpha * z;", "double u_tilde = alpha * u + (1.0 - alpha) * z;", 1),
+    ("anneal_threshold_exclusive", "double z = (logit >= tau_logit) ? 1.0 : 0.0;", "double z = (logit > tau_logit) ? 1.0 : 0.0;", 1),
+    ("soft_scale_dropped", "a[s] = qk * scale + bias_ts;", "a[s] = qk + bias_ts;", 1),
+    ("soft_scores_against_values", "qk += bf16_widen(qg[i]) * bf16_widen(K[(size_t)s * D + i]);",
+     "qk += bf16_widen(qg[i]) * bf16_widen(V[(size_t)s * D + i]);", 1),
+    ("soft_all_heads_use_head_0", "const uint16_t *qg = q + (size_t)g * D;", "const uint16_t *qg = q;", 1),
+    ("soft_lse_without_max", "if (lse) lse[g] = top + log(z_row);", "if (lse) lse[g] = log(z_row);", 1),
+    ("soft_unnormalised", "double weight = exp(a[s] - top) / z_row;", "double weight = exp(a[s] - top);", 1),
     ("keep_all_and_keep_none_swapped", "if (!(tau > 0.0)) return -INFINITY;", "if (!(tau > 0.0)) return INFINITY;", 1),
 ]
 
@@ -49,7 +62,8 @@ def test_planted_mistake_is_caught(tmp_path, name, old, new, count):
     env = dict(os.environ, SPKV_ORACLE_LIB=str(lib))
     r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider",
                         os.path.join(ROOT, "tests", "test_oracle_pins.py"),
-                        os.path.join(ROOT, "tests", "test_oracle_sinks.py")],
+                        os.path.join(ROOT, "tests", "test_oracle_sinks.py"),
+                        os.path.join(ROOT, "tests", "test_oracle_soft.py")],
                        cwd=ROOT, env=env, capture_output=True, text=True, timeout=600)
     out = r.stdout + r.stderr
     assert r.returncode == 1 and " failed" in out, f"mutant {name} survived the pins:\n{out[-800:]}"

@@ -75,6 +75,17 @@ def test_static_scratch_rejects_requests_beyond_its_size():
     assert spkv.lib().spkv_error_string(rc) == b"request exceeds the built-in scratch area"
     torch.cuda.synchronize()
     assert bool((out == 7.0).all())              # refused calls touch nothing
+    # argument errors are refused as spkv_decode_attention refuses them, before the shared array is
+    # touched: a bad layer, a missing query tensor, a batch larger than the cache has slots
+    f, s0 = spkv.lib().spkv_decode_attention_static, C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    ok_args = (C.c_void_p(ids.data_ptr()), 4, C.c_void_p(q.data_ptr()), C.c_void_p(out.data_ptr()), None, 0.1, s0)
+    assert f(cache._h, 1, *ok_args) == -1
+    assert f(cache._h, 0, C.c_void_p(ids.data_ptr()), 4, None, C.c_void_p(out.data_ptr()), None, 0.1, s0) == -1
+    assert f(cache._h, 0, C.c_void_p(ids.data_ptr()), 65, C.c_void_p(q.data_ptr()), C.c_void_p(out.data_ptr()),
+             None, 0.1, s0) == -1
+    assert f(None, 0, *ok_args) == -1
+    torch.cuda.synchronize()
+    assert bool((out == 7.0).all())
     # a batch that fits is accepted by the same cache
     small = torch.arange(4, dtype=torch.int32, device=dev())
     k = torch.zeros((4, 8, 128), dtype=torch.bfloat16, device=dev())
