@@ -402,8 +402,11 @@ def run_ours(args):
                 r += 1
         ms = median(regions)
         per_rep_clock = [clk.window(a, b)["sm_mhz"] for a, b in marks]
+        srt = sorted(regions)
+        p10, p90 = srt[len(srt) // 10], srt[len(srt) - 1 - len(srt) // 10]
         repeats = {"n": len(regions), "min": min(regions) / K, "median": ms / K, "max": max(regions) / K,
                    "unit": "ms_per_step", "spread": (max(regions) - min(regions)) / ms,
+                   "p10": p10 / K, "p90": p90 / K, "spread_p10_p90": (p90 - p10) / ms,
                    "timed_device_s": sum(regions) * 1e-3,
                    "ms_per_step_each": [round(x / K, 5) for x in regions],
                    "sm_mhz_each": per_rep_clock,
@@ -433,7 +436,7 @@ def run_ours(args):
 
         scale_l = L_full / L          # > 1 only for a dense run on a layer subset
         ms *= scale_l
-        for k_ in ("min", "median", "max"):
+        for k_ in ("min", "median", "max", "p10", "p90"):
             repeats[k_] *= scale_l
         res = dict(layers_measured=L, ms_per_step=ms / K, tokens_per_s=world * B * K / (ms * 1e-3), repeats=repeats,
                    kv_gb_per_step=scale_l * 0.5 * (st0.bytes_resident + st1.bytes_resident) / 1e9,
@@ -687,6 +690,91 @@ def run_config4(args):
 
 
 
+def run_softgate(args):
+    """Soft-gated whole-sequence forward (the paper's training-time attention, Eq. 6) on one
+    sequence of --softgate-T tokens with the head shape of the 8 B model: useful TFLOP/s against the
+    sustained bf16 peak, and beside it the hard-gated forward of the same sequence through
+    spkv_prefill (kept pairs compacted, so its work shrinks with the density)."""
+    import numpy as np
+    import torch
+
+    from paper_2605_14037_b200 import build as spkv_build
+    spkv_build.build()
+    from paper_2605_14037_b200 import spkv
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    T, Hq, Hkv = args.softgate_T, 32, 8
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(0)
+    rnd = lambda *shape: torch.randn(shape, generator=gen, device=dev).to(torch.bfloat16)
+    q, k, v = rnd(T, Hq, 128), rnd(T, Hkv, 128), rnd(T, Hkv, 128)
+    # gates: logits N(b_h, 1) with b_h such that head h would keep a fraction r_h at tau = 0.5
+    rates = np.random.default_rng(0).beta(0.5, 2.0, size=Hkv).clip(0.01, 0.99)
+    from statistics import NormalDist
+    bias = torch.tensor([NormalDist().inv_cdf(float(r)) for r in rates], dtype=torch.float32, device=dev)
+    logits = torch.randn((T, Hkv), generator=gen, device=dev) + bias
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            peak, peak_kind = float(json.load(f)["bf16_tflops_sustained"]), "of measured (sustained)"
+    except Exception:
+        peak, peak_kind = 1400.0, "of fallback (sustained)"
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def timed(fn):
+        for _ in range(max(3, args.warmup)):
+            fn()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        while time.perf_counter() - t0 < args.settle_seconds:
+            fn()
+            torch.cuda.synchronize()
+        times = []
+        with ClockSampler(0) as clk:
+            while len(times) < 5 or (sum(times) < 2000.0 and len(times) < 200):
+                a, b = ev(), ev()
+                a.record(); fn(); b.record()
+                torch.cuda.synchronize()
+                times.append(a.elapsed_time(b))
+        return median(times), times, clk.result
+
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    soft_out = torch.empty_like(q)
+    soft_ms, soft_all, clocks = timed(lambda: spkv.spkv_softgate_forward(q, k, v, logits, window=W, out=soft_out,
+                                                                       status=status))
+    assert int(status.item()) == 0, "a bounded wait ran out in the soft-gated forward"
+    flops = 4.0 * 128 * Hq * T * (T + 1) / 2
+    # hard-gated forward of the same tokens: spkv_prefill on an empty sequence with C = T
+    kept = int((logits >= 0).sum().item())
+    cache = spkv.Cache(n_layers=1, max_seqs=1, n_q_heads=Hq, n_kv_heads=Hkv, max_context=T + 64,
+                       pool_pages=kept // 64 + 2 * Hkv + 8, window=W, tau=TAU, device=dev)
+    out = torch.empty_like(q)
+
+    def hard():
+        cache.spkv_cache_reset_seq(0)
+        cache.spkv_prefill(0, 0, k, v, logits, q=q, out=out)
+
+    hard_ms, _, _ = timed(hard)
+    cache.check()
+    st = cache.spkv_cache_stats()
+    line = {
+        "metric": "soft-gated whole-sequence forward (Eq. 6), useful TFLOP/s", "value": flops / (soft_ms * 1e-3) / 1e12,
+        "unit": "TFLOP/s", "n_gpus": 1, "steps": len(soft_all), "warmup": max(3, args.warmup), "ms_per_step": soft_ms,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"softgate_forward_T{T}_q{Hq}_kv{Hkv}", "tokens": T, "q_heads": Hq, "kv_heads": Hkv,
+                   "window": W, "alpha": 0.0, "l2": "q and out (2 x %.0f MB) stream from HBM; K/V pages are re-read from L2" % (T * Hq * 256 / 1e6)},
+        "clocks": clocks,
+        "repeats": {"n": len(soft_all), "min": min(soft_all), "median": soft_ms, "max": max(soft_all), "unit": "ms"},
+        "gpu_launches": 3 + (1 if T < 4000 else 0),
+        "roofline": {"bound": "tensor", "kernel": "prefill_attn_tc5x2h_kernel<.., soft>", "achieved": flops / (soft_ms * 1e-3) / 1e12,
+                     "peak": peak, "unit": "TFLOP/s", "frac": flops / (soft_ms * 1e-3) / 1e12 / peak, "peak_kind": peak_kind,
+                     "flops_per_launch": flops, "traffic": None},
+        "hard_gated": {"ms": hard_ms, "density": st.density_cache, "speedup_over_soft": soft_ms / hard_ms,
+                       "how": "spkv_prefill of the same tokens on an empty sequence, tau = 0.5 (reset + prefill timed)"},
+        "e2e": None,
+    }
+    print(json.dumps(line))
+
+
 def load_traffic(workload, launch_bytes):
     """DRAM bytes per decode launch from the committed ncu summary, if there is one."""
     try:
@@ -788,6 +876,8 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--settle-seconds", type=float, default=1.0,
                     help="untimed replay of the timed region before the first repeat (clocks settle under load)")
+    ap.add_argument("--softgate-T", type=int, default=0,
+                    help="measure the soft-gated whole-sequence forward on this many tokens instead (not the bench line)")
     ap.add_argument("--sweep-tau", default="",
                     help="comma-separated thresholds: one decode measurement per tau, nothing else")
     args = ap.parse_args()
@@ -799,6 +889,9 @@ def main():
         args.warmup = 3
     if args.impl == "reference":
         run_reference(args)
+    elif args.softgate_T > 0:
+        if int(os.environ.get("RANK", "0")) == 0:
+            run_softgate(args)
     elif args.config == 4:
         if int(os.environ.get("RANK", "0")) == 0:
             run_config4(args)

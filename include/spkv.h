@@ -83,6 +83,15 @@ typedef struct {
                            kept in the compact cache whatever their utility (the paper's
                            "Fixed Attention Sinks" ablation; its evaluation protocol uses
                            4).  0 = the method as defined by Eq. 2-4.                      */
+  const uint8_t *h_local_only; /* HOST array [n_layers * n_kv_heads] or NULL, read only while
+                           spkv_arena_bytes / spkv_cache_create / spkv_cache_attach run: a
+                           non-zero entry declares that (layer, KV head) local-only for the
+                           life of the cache (the paper's static hybrid layouts: sliding-window
+                           heads beside global ones).  Such a head keeps nothing, sink positions
+                           included, so its units get no page table (the arena is smaller by
+                           max_context / 64 * 4 bytes per unit), the fused score + append does
+                           not compute its utility (the logit is written as 0), and
+                           spkv_set_head_tau refuses to change it.  n_kv_heads <= 64.        */
 } spkv_config_t;
 
 /* SPKV_FLAG_OVERLAP (off by default): consecutive hot-path launches on one stream overlap where
@@ -228,7 +237,8 @@ int spkv_set_tau(spkv_cache_t *cache, float tau);
  * (window attention, nothing is ever kept: its compact cache and page table stay empty),
  * tau <= 0 makes it a full-attention head, NaN returns it to the cache-wide threshold.
  * kv_head = -1 addresses every KV head of the layer.  spkv_score's optional flags follow the
- * cache-wide threshold only. */
+ * cache-wide threshold only.  A head that only ever needs the window is better declared in
+ * spkv_config_t.h_local_only: it then costs no page table and no scoring. */
 int spkv_set_head_tau(spkv_cache_t *cache, int32_t layer, int32_t kv_head, float tau,
                       spkv_stream_t stream);
 
@@ -340,6 +350,34 @@ int spkv_prefill(spkv_cache_t *cache, int32_t layer, int32_t seq, int32_t C, con
                  const void *d_k, const void *d_v, const float *d_logits, void *d_out,
                  float sm_scale, void *d_workspace, size_t workspace_bytes,
                  spkv_stream_t stream);
+
+/* Soft-gated whole-sequence forward: the attention the paper trains with (Section "Training",
+ * "Phase 1. Soft Gated Training", Eq. 6; the annealed gate of "Phase 2", Eq. 7; kernel notes in
+ * "Training Efficiency"), forward only.  Causal attention of all T queries over all T keys of one
+ * sequence in which key s gets, for query t,
+ *     bias 0                 if 0 <= t - s < window      (the local window is never gated)
+ *     bias log u~_s          if t - s >= window          (Eq. 6)
+ *     -inf                   if s > t,
+ * u~_s = (1 - alpha) sigma(logit_s) + alpha 1[logit_s >= tau_logit] (Eq. 7; alpha = 0: soft gating,
+ * alpha = 1: the binary gate, i.e. the hard-gated forward of Eq. 3-5), one gate per KV head shared
+ * by its query-head group.  log sigma is evaluated without forming the sigmoid; the epsilon the
+ * paper's listing adds inside the logarithm guards gradients and is not applied.
+ * No cache is involved and nothing is kept between calls.
+ *   d_q [T, n_q_heads, 128], d_k/d_v [T, n_kv_heads, 128] bf16, d_logits [T, n_kv_heads] float32
+ *   -> d_out [T, n_q_heads, 128] bf16, d_lse_opt [T, n_q_heads] float32 (natural-log sum-exp of
+ *   the biased scaled scores; may be NULL).  head_dim is 128, n_q_heads / n_kv_heads <= 16.
+ *   alpha in [0, 1]; tau as in spkv_config_t; sm_scale positive and finite;
+ *   flags: 0 or SPKV_FLAG_PREFILL_PV_BF16 (precision of weights x values as in spkv_prefill);
+ *   d_workspace: >= spkv_softgate_workspace_bytes(T, n_q_heads, n_kv_heads) bytes, 256-byte
+ *   aligned (K and V are rewritten there as 64-key pages: about the size of K + V);
+ *   d_status: device, one int32 that the caller has set to 0: SPKV_E_TIMEOUT is stored there if a
+ *   bounded wait inside the kernel ran out.  Asynchronous on `stream`. */
+size_t spkv_softgate_workspace_bytes(int32_t T, int32_t n_q_heads, int32_t n_kv_heads);
+int spkv_softgate_forward(int32_t T, int32_t n_q_heads, int32_t n_kv_heads, int32_t window,
+                          const void *d_q, const void *d_k, const void *d_v, const float *d_logits,
+                          float alpha, float tau, float sm_scale, int32_t flags, void *d_out,
+                          float *d_lse_opt, void *d_workspace, size_t workspace_bytes,
+                          int32_t *d_status, spkv_stream_t stream);
 
 /* One decode step of one layer from HOST buffers (pinned memory, or the copies are not
  * asynchronous): score -> append/evict -> decode attention with the inputs copied in and the

@@ -37,7 +37,8 @@ __device__ inline void append_unit(const CacheView &c, int layer, const int32_t 
                                    const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new,
                                    const float *__restrict__ logits, float tau_logit,
                                    const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__restrict__ W,
-                                   const float *__restrict__ bias, int d_in, float *__restrict__ logits_out) {
+                                   const float *__restrict__ bias, int d_in, float *__restrict__ logits_out,
+                                   unsigned long long local_mask) {
   const int lane = threadIdx.x & 31;
   const int item = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (item >= B * c.Hkv) return;
@@ -48,9 +49,15 @@ __device__ inline void append_unit(const CacheView &c, int layer, const int32_t 
     return;
   }
   const int u = unit_index(c, layer, seq, kvh);
+  // a head declared local-only keeps nothing and has no page table: its utility is never looked
+  // at, so it is not computed either (its logit is written as 0)
+  const bool local_only = (local_mask >> kvh) & 1ULL;
   // fused scoring (Eq. 1, linear predictor): this unit's logit for the new pair
   float new_logit;
-  if (x) {
+  if (local_only) {
+    new_logit = 0.f;
+    if (x && logits_out && lane == 0) logits_out[item] = 0.f;
+  } else if (x) {
     new_logit = warp_dot_bf16(x + (size_t)b * d_in, W + (size_t)kvh * d_in, d_in, lane) + bias[kvh];
     if (logits_out && lane == 0) logits_out[item] = new_logit;
   } else {
@@ -67,12 +74,13 @@ __device__ inline void append_unit(const CacheView &c, int layer, const int32_t 
   __nv_bfloat16 *ring = c.pages + ring_page(c, u, slot / kP) * kPageElems;
   uint4 *ring_cell = reinterpret_cast<uint4 *>(ring + blk + swz_off(row, chunk));
 
-  if (t >= c.w) {
+  if (t >= c.w && !local_only) {
     // the pair of position t - w leaves the window: threshold decision on its stored logit
     // (sink positions are kept regardless)
     const float lg = __ldcg(&c.ring_logit[(size_t)u * c.w + slot]);
     if (lg >= head_threshold(c, layer, kvh, tau_logit) || t - c.w < c.n_sink) {
       const int n = __ldcg(&c.len[u]);
+      int32_t *table = unit_table(c, unit_table_row(c, u));
       const int pj = n / kP, prow = n % kP;
       int page = -1, err = 0;
       if (pj >= c.max_pages) {
@@ -81,9 +89,9 @@ __device__ inline void append_unit(const CacheView &c, int layer, const int32_t 
         page = alloc_page(c, lane);
         if (page == -1) err = SPKV_E_POOL_EXHAUSTED;
         else if (page < 0) err = SPKV_E_BOUNDS_PAGE;
-        else if (lane == 0) c.table[(size_t)u * c.max_pages + pj] = page;
+        else if (lane == 0) table[pj] = page;
       } else {
-        page = checked_page(c, __ldcg(&c.table[(size_t)u * c.max_pages + pj]), -2);
+        page = checked_page(c, __ldcg(&table[pj]), -2);
         if (page < 0) err = SPKV_E_BOUNDS_PAGE;   // the evicted pair is dropped, as on exhaustion
       }
       if (err) {
@@ -117,7 +125,7 @@ append_evict_kernel(CacheView c, int layer, const int32_t *__restrict__ seq_ids,
                     const float *__restrict__ logits, float tau_logit,
                     const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__restrict__ W,
                     const float *__restrict__ bias, int d_in, float *__restrict__ logits_out,
-                    int wait_prev) {
+                    int wait_prev, unsigned long long local_mask) {
   // Every block counts itself in before dependents may launch and out when it is done: that is
   // what later kernels that skip griddepcontrol.wait order themselves by.
   if (threadIdx.x == 0) sync_count_start(c, layer, kSyncAppStart);
@@ -132,7 +140,7 @@ append_evict_kernel(CacheView c, int layer, const int32_t *__restrict__ seq_ids,
   else if (threadIdx.x == 0 && !sync_wait_finished(c, layer, kSyncDecStart)) set_status(c, SPKV_E_ORDER_APPEND);
   __syncthreads();
   pdl_trigger();
-  append_unit(c, layer, seq_ids, B, k_new, v_new, logits, tau_logit, x, W, bias, d_in, logits_out);
+  append_unit(c, layer, seq_ids, B, k_new, v_new, logits, tau_logit, x, W, bias, d_in, logits_out, local_mask);
   __syncthreads();
   if (threadIdx.x == 0) sync_count_finish(c, layer, kSyncAppFin);
 }
@@ -184,7 +192,7 @@ extern "C" int spkv_append_evict(spkv_cache_t *cache, int32_t layer, const int32
   return launch_append(cache, items, as_stream(stream), cache->view, layer, d_seq_ids, B,
                        static_cast<const uint4 *>(d_k), static_cast<const uint4 *>(d_v), d_logits,
                        cache->tau_logit, (const __nv_bfloat16 *)nullptr, (const __nv_bfloat16 *)nullptr,
-                       (const float *)nullptr, 0, (float *)nullptr, wait_prev);
+                       (const float *)nullptr, 0, (float *)nullptr, wait_prev, cache->local_mask[layer]);
 }
 
 extern "C" int spkv_score_append_evict(spkv_cache_t *cache, int32_t layer, const spkv_predictor_t *pred,
@@ -212,5 +220,5 @@ extern "C" int spkv_score_append_evict(spkv_cache_t *cache, int32_t layer, const
                        static_cast<const uint4 *>(d_k), static_cast<const uint4 *>(d_v), (const float *)nullptr,
                        cache->tau_logit, static_cast<const __nv_bfloat16 *>(d_x),
                        static_cast<const __nv_bfloat16 *>(pred->d_W1), pred->d_b1, pred->d_in, d_logits_out,
-                       wait_prev);
+                       wait_prev, cache->local_mask[layer]);
 }

@@ -34,6 +34,7 @@ static int validate(const spkv_config_t *c) {
   int64_t ring_pages = (c->window + kP - 1) / kP;
   if (units > (1 << 24)) return SPKV_E_INVALID;
   if (units * ring_pages + c->pool_pages > 0x7fffffffLL) return SPKV_E_INVALID;
+  if (c->h_local_only && c->n_kv_heads > 64) return SPKV_E_UNSUPPORTED;   // one bit per KV head of a layer
   return SPKV_OK;
 }
 
@@ -41,6 +42,11 @@ static void make_layout(const spkv_config_t *c, Layout *l) {
   size_t units = (size_t)c->n_layers * c->max_seqs * c->n_kv_heads;
   size_t ring_pages = (c->window + kP - 1) / kP;
   size_t max_pages = ((size_t)c->max_context + kP - 1) / kP;
+  // units of a head declared local-only have no page table
+  size_t global_heads = (size_t)c->n_layers * c->n_kv_heads;
+  if (c->h_local_only)
+    for (size_t i = 0, n = global_heads; i < n; ++i) global_heads -= c->h_local_only[i] ? 1 : 0;
+  l->n_table_rows = global_heads * c->max_seqs;
   size_t o = 0;
   int n_can = 0;
   // a region of `bytes` bytes at the current offset, followed by its canary block
@@ -54,13 +60,14 @@ static void make_layout(const spkv_config_t *c, Layout *l) {
   l->off_header = region(256);
   l->off_t = region(units * 4);
   l->off_len = region(units * 4);
-  l->off_table = region(units * max_pages * 4);
+  l->off_table = region(l->n_table_rows * max_pages * 4);
   l->off_free = region((size_t)c->pool_pages * 4);
   l->off_pos = region((size_t)c->pool_pages * kP * 4);
   l->off_rlogit = region(units * (size_t)c->window * 4);
   l->off_htau = region((size_t)c->n_layers * c->n_kv_heads * 4);
   l->off_sync = region((size_t)c->n_layers * 4 * 8);
   l->off_vmax = region(units * 4);
+  l->off_trow = region(units * 4);
   o = align_up(o, 1024);
   l->off_pages = o;  o += (units * ring_pages + (size_t)c->pool_pages) * kPageBytes;
   l->total = o;
@@ -74,10 +81,12 @@ static uint64_t layout_hash(const spkv_config_t *c) {
   uint64_t h = 1469598103934665603ULL;
   for (int64_t v : f)
     for (int b = 0; b < 8; ++b) { h ^= (uint64_t)(v >> (8 * b)) & 0xff; h *= 1099511628211ULL; }
+  if (c->h_local_only)   // which heads have no page table is part of the layout
+    for (int i = 0; i < c->n_layers * c->n_kv_heads; ++i) { h ^= c->h_local_only[i] ? 1 : 0; h *= 1099511628211ULL; }
   return h;
 }
 constexpr uint32_t kMagic = 0x564B5053u;   // "SPKV"
-constexpr uint32_t kLayoutVersion = 2;
+constexpr uint32_t kLayoutVersion = 3;
 constexpr int kHdrMagicWord = 8;            // int32 index of {magic, version, hash lo, hash hi} in the header
 
 // value = NaN clears the override
@@ -102,8 +111,8 @@ __global__ void reset_seq_kernel(CacheView c, int seq) {
   __shared__ int base;
   if (threadIdx.x == 0) base = n_pages ? atomicAdd(&c.status[1], n_pages) : 0;
   __syncthreads();
-  for (int j = threadIdx.x; j < n_pages; j += blockDim.x)
-    c.free_stack[base + j] = c.table[(size_t)u * c.max_pages + j];
+  for (int j = threadIdx.x; j < n_pages; j += blockDim.x)   // (n_pages > 0: the unit has a page table)
+    c.free_stack[base + j] = unit_table(c, c.table_row[u])[j];
   uint4 *ring = reinterpret_cast<uint4 *>(c.pages + ring_page(c, u, 0) * kPageElems);
   const int n16 = c.ring_pages * (kPageBytes / 16);
   for (int i = threadIdx.x; i < n16; i += blockDim.x) ring[i] = make_uint4(0, 0, 0, 0);
@@ -142,7 +151,16 @@ static int make_handle(const spkv_config_t *cfg, void *d_arena, const Layout &l,
   c->last_decode_items = -1;
   c->last_decode_ws = nullptr;
   c->appends_pending = new (std::nothrow) int[cfg->n_layers]();
-  if (!c->appends_pending) { delete c; return SPKV_E_INVALID; }
+  c->local_mask = new (std::nothrow) unsigned long long[cfg->n_layers]();
+  if (!c->appends_pending || !c->local_mask) {
+    delete[] c->appends_pending; delete[] c->local_mask; delete c;
+    return SPKV_E_INVALID;
+  }
+  if (cfg->h_local_only)
+    for (int l2 = 0; l2 < cfg->n_layers; ++l2)
+      for (int h = 0; h < cfg->n_kv_heads; ++h)
+        if (cfg->h_local_only[l2 * cfg->n_kv_heads + h]) c->local_mask[l2] |= 1ULL << h;
+  c->cfg.h_local_only = nullptr;   // the caller's array is read during this call only
   c->host_ready = false;
   c->stack_ready = false;
   c->host_calls = 0;
@@ -168,17 +186,25 @@ static int make_handle(const spkv_config_t *cfg, void *d_arena, const Layout &l,
   v.head_tau = reinterpret_cast<float *>(base + l.off_htau);
   v.sync_ctr = reinterpret_cast<unsigned long long *>(base + l.off_sync);
   v.vmax = reinterpret_cast<uint32_t *>(base + l.off_vmax);
+  v.table_row = reinterpret_cast<int32_t *>(base + l.off_trow);
   v.pages = reinterpret_cast<__nv_bfloat16 *>(base + l.off_pages);
   int dev = 0;
   cudaDeviceProp prop;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
     delete[] c->appends_pending;
+    delete[] c->local_mask;
     delete c;
     return SPKV_E_CUDA;
   }
   c->sm_count = prop.multiProcessorCount;
   *out = c;
   return SPKV_OK;
+}
+
+static void free_handle(spkv_cache *c) {
+  delete[] c->appends_pending;
+  delete[] c->local_mask;
+  delete c;
 }
 
 extern "C" int spkv_cache_create(const spkv_config_t *cfg, void *d_arena, size_t arena_bytes,
@@ -208,6 +234,20 @@ extern "C" int spkv_cache_create(const spkv_config_t *cfg, void *d_arena, size_t
   if (e == cudaSuccess) {
     const int nh = v.L * v.Hkv;
     set_head_tau_kernel<<<(nh + 255) / 256, 256, 0, s>>>(v.head_tau, 0, nh, NAN);
+    // page-table rows in (layer, sequence, KV head) order, local-only heads skipped; such a head
+    // also carries the keep-nothing threshold for good
+    std::vector<int32_t> rows((size_t)v.n_units);
+    int32_t next = 0;
+    for (int l2 = 0; l2 < v.L; ++l2)
+      for (int sq = 0; sq < v.S; ++sq)
+        for (int h = 0; h < v.Hkv; ++h)
+          rows[((size_t)l2 * v.S + sq) * v.Hkv + h] = ((c->local_mask[l2] >> h) & 1ULL) ? -1 : next++;
+    e = cudaMemcpyAsync(v.table_row, rows.data(), rows.size() * 4, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);   // `rows` is pageable host memory about to go away
+    for (int l2 = 0; l2 < v.L && e == cudaSuccess; ++l2)
+      for (int h = 0; h < v.Hkv; ++h)
+        if ((c->local_mask[l2] >> h) & 1ULL)
+          set_head_tau_kernel<<<1, 32, 0, s>>>(v.head_tau, l2 * v.Hkv + h, 1, INFINITY);
   }
   if (e == cudaSuccess && v.pool_pages > 0) {
     int64_t n = v.pool_pages;
@@ -216,8 +256,7 @@ extern "C" int spkv_cache_create(const spkv_config_t *cfg, void *d_arena, size_t
     e = cudaGetLastError();
   }
   if (e != cudaSuccess) {
-    delete[] c->appends_pending;
-    delete c;
+    free_handle(c);
     return SPKV_E_CUDA;
   }
   *out = c;
@@ -336,6 +375,7 @@ extern "C" int spkv_safe_steps(spkv_cache_t *cache, const int32_t *h_seq_ids, in
   for (int l = 0; l < v.L; ++l)
     for (int b = 0; b < (B ? B : v.S); ++b)
       for (int h = 0; h < v.Hkv; ++h) {
+        if ((cache->local_mask[l] >> h) & 1ULL) continue;   // a local-only head never needs a page
         const int u = (l * v.S + (B ? h_seq_ids[b] : b)) * v.Hkv + h;
         sl.push_back(len[u]);
         st.push_back(t[u]);
@@ -363,8 +403,7 @@ extern "C" int spkv_cache_destroy(spkv_cache_t *cache) {
     cudaStreamDestroy(cache->copy_in);
     cudaStreamDestroy(cache->copy_out);
   }
-  delete[] cache->appends_pending;
-  delete cache;
+  free_handle(cache);
   return SPKV_OK;
 }
 
@@ -386,6 +425,9 @@ extern "C" int spkv_set_head_tau(spkv_cache_t *cache, int32_t layer, int32_t kv_
                                  spkv_stream_t stream) {
   if (!cache || layer < 0 || layer >= cache->view.L || kv_head < -1 || kv_head >= cache->view.Hkv)
     return SPKV_E_INVALID;
+  // a head declared local-only at creation has no page table: it stays local-only
+  const unsigned long long target = kv_head < 0 ? ~0ULL : 1ULL << kv_head;
+  if (cache->local_mask[layer] & target) return SPKV_E_INVALID;
   const float value = tau != tau ? NAN : tau_to_logit(tau);
   const int first = layer * cache->view.Hkv + (kv_head < 0 ? 0 : kv_head);
   const int count = kv_head < 0 ? cache->view.Hkv : 1;
@@ -460,7 +502,10 @@ extern "C" int spkv_read_kept(spkv_cache_t *cache, int32_t layer, int32_t seq, i
   int n_pages = (n + kP - 1) / kP;
   if (n_pages == 0) return SPKV_OK;
   std::vector<int32_t> table(n_pages);
-  if (cudaMemcpy(table.data(), v.table + (size_t)u * v.max_pages, (size_t)n_pages * 4,
+  int32_t trow = -1;
+  if (cudaMemcpy(&trow, v.table_row + u, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return SPKV_E_CUDA;
+  if (trow < 0 || (size_t)trow >= cache->layout.n_table_rows) return SPKV_E_INVALID;
+  if (cudaMemcpy(table.data(), v.table + (size_t)trow * v.max_pages, (size_t)n_pages * 4,
                  cudaMemcpyDeviceToHost) != cudaSuccess)
     return SPKV_E_CUDA;
   std::vector<uint16_t> tmp(kPageElems);

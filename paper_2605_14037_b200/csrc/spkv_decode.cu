@@ -69,7 +69,7 @@ struct StageMeta {  // valid rows (bits 0-7) | flags (8-11) | item (12+)
 };
 
 struct TcSmem {  // offsets into dynamic shared memory, computed on host and device alike
-  int n_stages, red_bufs, stage_bytes, off_bar, off_meta, off_np, off_pre, off_unit, off_len, off_ring,
+  int n_stages, red_bufs, stage_bytes, off_bar, off_meta, off_np, off_pre, off_unit, off_len, off_ring, off_row,
       off_tmp, off_cut, off_red, off_mrg, off_flags, total;
 };
 __host__ __device__ inline TcSmem tc_smem_layout(int n_items, int GP, int n_stages, int red_bufs) {
@@ -86,6 +86,7 @@ __host__ __device__ inline TcSmem tc_smem_layout(int n_items, int GP, int n_stag
   L.off_unit = o;  o += n_items * 4;
   L.off_len = o;   o += n_items * 4;
   L.off_ring = o;  o += n_items * 4;
+  L.off_row = o;   o += n_items * 4;
   L.off_tmp = o;   o += 64 * 4;
   L.off_cut = o;   o += (kMaxGrid + 1) * 4;
   o = (o + 15) / 16 * 16;
@@ -235,6 +236,7 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
   int *s_unit = reinterpret_cast<int *>(smem + L.off_unit);
   int *s_len = reinterpret_cast<int *>(smem + L.off_len);
   int *s_ring = reinterpret_cast<int *>(smem + L.off_ring);
+  int *s_row = reinterpret_cast<int *>(smem + L.off_row);   // the unit's page-table row (-1: a local-only head)
   int *s_tmp = reinterpret_cast<int *>(smem + L.off_tmp);
   int *s_cut = reinterpret_cast<int *>(smem + L.off_cut);
   float *s_red = reinterpret_cast<float *>(smem + L.off_red);
@@ -290,9 +292,10 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
   for (int i = tid; i < n; i += kTcThreads) {
     const int b = i / c.Hkv, kvh = i % c.Hkv;
     const int seq = (a.wait_mode == 1 && i == tid) ? seq_first : a.seq_ids[b];
-    int np = 0, u = 0, len = 0, n_ring = 0;
+    int np = 0, u = 0, len = 0, n_ring = 0, trow = -1;
     if (seq >= 0 && seq < c.S) {
       u = unit_index(c, a.layer, seq, kvh);
+      trow = unit_table_row(c, u);
       // (L2 loads: in overlap mode the writer may be a kernel that ended after this block began,
       // and an SM's L1 is not coherent with other SMs' stores)
       len = __ldcg(&c.len[u]);
@@ -302,7 +305,7 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
       set_status(c, SPKV_E_BOUNDS);
     }
     s_np[i] = np > 0 ? np + 1 : 0;  // + the marker position
-    s_unit[i] = u; s_len[i] = len; s_ring[i] = n_ring;
+    s_unit[i] = u; s_len[i] = len; s_ring[i] = n_ring; s_row[i] = trow;
     if (np == 0 && blockIdx.x == 0) {  // nothing to attend to: defined output
       for (int g = 0; g < a.G; ++g) {
         __nv_bfloat16 *o = a.out + ((size_t)b * c.Hq + kvh * a.G + g) * kD;
@@ -357,7 +360,7 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
           const int u = s_unit[item], len = s_len[item], nk = (len + kP - 1) / kP;
           if (j < nk) {
             // (debug bounds: a table entry that names no pool page is read from the unit's ring instead)
-            gq.gpage = checked_page(c, __ldcg(&c.table[(size_t)u * c.max_pages + j]), (int)ring_page(c, u, 0));
+            gq.gpage = checked_page(c, __ldcg(&unit_table(c, s_row[item])[j]), (int)ring_page(c, u, 0));
             gq.valid = min(kP, len - j * kP);
           } else {
             gq.gpage = (int)ring_page(c, u, j - nk);

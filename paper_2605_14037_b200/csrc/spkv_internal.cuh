@@ -5,13 +5,15 @@
 //   (every metadata region is followed by a 256-byte canary block of 0xC5 bytes)
 //   t[]         : pairs received per unit                       int32 [n_units]
 //   len[]       : kept pairs per unit                           int32 [n_units]
-//   table[]     : page table per unit (global page indices)     int32 [n_units][max_pages]
+//   table[]     : page table per unit that can keep pairs        int32 [rows][max_pages]
+//                 (units of heads declared local-only at creation have none)
 //   free_stack[]: LIFO of free pool pages (global page indices) int32 [pool_pages]
 //   pos_pool[]  : position of every kept pair, by pool page     int32 [pool_pages][P]
 //   ring_logit[]: stored logit per ring slot                    f32   [n_units][w]
 //   head_tau[]  : per-(layer, KV head) threshold override       f32   [L][Hkv]  (NaN: none)
 //   vmax[]      : largest finite |value| in a unit's compact cache u32 [n_units] (fp32 bit pattern)
 //   sync_ctr[]  : blocks started / finished per layer and kernel u64   [L][4]    (launch overlap)
+//   table_row[] : row of a unit in table[], -1 = none            int32 [n_units]
 //   pages       : ring pages of every unit ([n_units][ring_pages]) followed by the pool
 //
 // A page holds P = 64 pairs: a 16 KB key block followed by a 16 KB value block.  Each
@@ -46,7 +48,8 @@ struct CacheView {
   int32_t *status;      // [0] sticky status, [1] free_top
   int32_t *t;
   int32_t *len;
-  int32_t *table;
+  int32_t *table;       // [table rows][max_pages]: a row per unit that can keep pairs
+  int32_t *table_row;   // [n_units]: the unit's row in `table`, -1 for a unit of a local-only head
   int32_t *free_stack;
   int32_t *pos_pool;
   float *ring_logit;
@@ -60,11 +63,13 @@ struct CacheView {
   __nv_bfloat16 *pages;
 };
 
-constexpr int kCanaries = 10;          // one 256-byte block after each metadata region
+constexpr int kCanaries = 11;          // one 256-byte block after each metadata region
 constexpr int kCanaryBytes = 256;
 constexpr unsigned char kCanaryByte = 0xC5;
 struct Layout {
-  size_t off_header, off_t, off_len, off_table, off_free, off_pos, off_rlogit, off_htau, off_sync, off_vmax, off_pages, total;
+  size_t off_header, off_t, off_len, off_table, off_free, off_pos, off_rlogit, off_htau, off_sync, off_vmax, off_trow,
+      off_pages, total;
+  size_t n_table_rows;
   size_t canary[kCanaries];
 };
 
@@ -114,6 +119,10 @@ __device__ inline float head_threshold(const CacheView &c, int layer, int kvh, f
   const float own = __ldcg(&c.head_tau[layer * c.Hkv + kvh]);
   return own != own ? tau_logit : own;
 }
+
+// page table of a unit (the caller knows the unit has one: row >= 0)
+__device__ inline int32_t *unit_table(const CacheView &c, int row) { return c.table + (size_t)row * c.max_pages; }
+__device__ inline int unit_table_row(const CacheView &c, int u) { return __ldcg(&c.table_row[u]); }
 
 // global page index of ring page j of a unit
 __device__ inline int64_t ring_page(const CacheView &c, int unit, int j) {
@@ -238,6 +247,7 @@ struct spkv_cache {
   int last_decode_items;    // units of the previous decode launch (the workspace halves depend on it)
   void *last_decode_ws;     // and its workspace
   int *appends_pending;     // [n_layers] appends since the layer's last decode launch
+  unsigned long long *local_mask;   // [n_layers] bit h set: KV head h of the layer was declared local-only
   // spkv_decode_step_host: copy streams and events of its two-slot pipeline (made on first use)
   cudaStream_t copy_in, copy_out;
   cudaEvent_t ev_in[2], ev_k[2], ev_out[2];   // per slot: inputs landed, kernels done, output landed

@@ -39,6 +39,7 @@ __global__ void __launch_bounds__(1024) prefill_plan_kernel(PrefillArgs a) {
   int32_t *E = hdr + kHdrInts;
   const int t0 = c.t[u], len0 = c.len[u];
   const float thr = head_threshold(c, a.layer, kvh, a.tau_logit);
+  const int trow = c.table_row[u];   // -1: a head declared local-only keeps nothing, sinks included
   const int n_old = min(t0, c.w), p0 = t0 - n_old;
   const int N = n_old + a.C;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -52,7 +53,7 @@ __global__ void __launch_bounds__(1024) prefill_plan_kernel(PrefillArgs a) {
     if (j < N) {
       const float lg = j < n_old ? c.ring_logit[(size_t)u * c.w + (p0 + j) % c.w]
                                  : a.logits[(size_t)(j - n_old) * c.Hkv + kvh];
-      flag = lg >= thr || p0 + j < c.n_sink;  // Eq. 2 on the float32 logit; sink positions always
+      flag = trow >= 0 && (lg >= thr || p0 + j < c.n_sink);  // Eq. 2 on the float32 logit; sink positions always
     }
     const unsigned ballot = __ballot_sync(0xffffffffu, flag);
     const int before = __popc(ballot & ((1u << lane) - 1u));
@@ -109,12 +110,13 @@ __global__ void __launch_bounds__(1024) prefill_plan_kernel(PrefillArgs a) {
   if (s_fail || n_new == 0) return;
   // (debug bounds: an index from the stack that names no pool page is recorded; the scatter kernel
   // skips what would go there)
+  int32_t *table = unit_table(c, trow);   // n_new > 0: the unit keeps pairs, so it has a table
   for (int i = tid; i < n_new; i += blockDim.x)
-    c.table[(size_t)u * c.max_pages + pages0 + i] = checked_page(c, c.free_stack[s_pages_base - 1 - i], -1);
+    table[pages0 + i] = checked_page(c, c.free_stack[s_pages_base - 1 - i], -1);
   __syncthreads();
   // rows past the final length of a freshly popped last page must read as zeros
-  if (len1 % kP && c.table[(size_t)u * c.max_pages + pages1 - 1] >= 0) {
-    const int last = c.table[(size_t)u * c.max_pages + pages1 - 1];
+  if (len1 % kP && table[pages1 - 1] >= 0) {
+    const int last = table[pages1 - 1];
     uint4 *vb = reinterpret_cast<uint4 *>(c.pages + (int64_t)last * kPageElems + kBlockElems);
     for (int i = tid; i < kBlockElems * 2 / 16; i += blockDim.x) vb[i] = make_uint4(0, 0, 0, 0);
   }
@@ -159,12 +161,13 @@ __global__ void __launch_bounds__(256) prefill_scatter_kernel(PrefillArgs a) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int chunk = lane & 15, blk = (lane >> 4) * kBlockElems;
   const int j0 = (blockIdx.x * 8 + warp) * 8;
+  const int trow = c.table_row[u];
   uint32_t vm = 0;  // largest |v| among the pairs this warp appends to the compact cache
   for (int j = j0; j < min(j0 + 8, n_leave); ++j) {
     const int e = E[j];
     if (E[j + 1] == e) continue;  // not flagged
     const int idx = len0 + e;
-    const int page = checked_page(c, c.table[(size_t)u * c.max_pages + idx / kP], -1);
+    const int page = checked_page(c, unit_table(c, trow)[idx / kP], -1);
     if (page < 0) continue;   // debug bounds: recorded, the pair is not written
     const int drow = idx % kP;
     const SrcRow s = staging_row(a, u, kvh, t0, n_old, j);
@@ -236,6 +239,11 @@ __global__ void __launch_bounds__(256) prefill_stage_kernel(PrefillArgs a) {
   if (lane == 0 && vm) atomicMax(reinterpret_cast<uint32_t *>(&hdr[H_VMAX]), vm);
 }
 
+int launch_prefill_stage(const PrefillArgs &a, cudaStream_t s) {
+  prefill_stage_kernel<<<dim3(a.n_stage_pages, a.c.Hkv), 256, 0, s>>>(a);
+  return check_stream_error(cudaGetLastError());
+}
+
 static size_t prefill_ws_stride_ints(int C, int w) {
   size_t ints = kHdrInts + (size_t)C + w + 2;
   return (ints + 63) / 64 * 64;
@@ -291,6 +299,9 @@ extern "C" int spkv_prefill(spkv_cache_t *cache, int32_t layer, int32_t seq, int
   a.pair_tiles = 0;
   a.n_split = 1;
   a.force_wide = (cache->cfg.flags & SPKV_FLAG_PREFILL_PV_BF16) ? 1 : 0;
+  a.soft = 0;
+  a.gate2 = nullptr;
+  a.lse = nullptr;
   a.partials = prefill_split_bytes(&cache->cfg, C)
                    ? reinterpret_cast<float *>(reinterpret_cast<char *>(a.stage_pages) +
                                                (size_t)v.Hkv * a.n_stage_pages * kPageBytes)
@@ -302,8 +313,8 @@ extern "C" int spkv_prefill(spkv_cache_t *cache, int32_t layer, int32_t seq, int
   // at most max(min(t0,w) + C - w, 0) <= C pairs leave the window
   prefill_scatter_kernel<<<dim3((C + 63) / 64, v.Hkv), 256, 0, s>>>(a);
   if (d_q) {
-    prefill_stage_kernel<<<dim3(a.n_stage_pages, v.Hkv), 256, 0, s>>>(a);
-    const int rc = launch_prefill_attn_tc5x2h(a, s);
+    int rc = launch_prefill_stage(a, s);
+    if (!rc) rc = launch_prefill_attn_tc5x2h(a, s);
     if (rc) return rc;
   }
   const int n_ring = C < v.w ? C : v.w;

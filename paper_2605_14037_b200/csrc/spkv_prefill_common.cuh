@@ -25,6 +25,12 @@ struct PrefillArgs {
   int n_split;                     // fp16 two-slot kernel: blocks per page walk (split over the pages), >= 1
   float *partials;                 // [walk][slot][split]: 128 rows x (128 O + pad) and (m, l); n_split > 1 only
   int force_wide;                  // SPKV_FLAG_PREFILL_PV_BF16: every unit takes the two-term bf16 P.V
+  // Soft-gated whole-sequence forward (spkv_softgate_forward; Eq. 6): no cache behind the call,
+  // the staging sequence is the whole sequence, a query walks every causal page of it, and a key
+  // beyond the query's window gets the bias gate2[key] (log2 of its gate) instead of a mask.
+  int soft;
+  const float *gate2;              // [Hkv][n_stage_pages * 64] (soft only)
+  float *lse;                      // [C][Hq] natural-log sum-exp of the biased scaled scores, or null
 };
 
 __device__ inline int32_t *unit_ws(const PrefillArgs &a, int kvh) { return a.ws + (size_t)kvh * a.ws_stride; }
@@ -39,7 +45,7 @@ __device__ inline int32_t *unit_ws(const PrefillArgs &a, int kvh) { return a.ws 
 // warps; every warp computes the same answer.  More KV heads than lanes: plain order.
 __device__ inline int prefill_kvh_by_rank(const PrefillArgs &a, int rank) {
   const int lane = threadIdx.x & 31, Hkv = a.c.Hkv;
-  if (Hkv > 32) return rank;
+  if (Hkv > 32 || a.soft) return rank;   // (soft-gated forward: every KV head walks the same pages)
   int key = -1;
   if (lane < Hkv) {
     const int32_t *hdr = unit_ws(a, lane);
@@ -52,7 +58,9 @@ __device__ inline int prefill_kvh_by_rank(const PrefillArgs &a, int rank) {
   }
   return __ffs(__ballot_sync(0xffffffffu, lane < Hkv && my_rank == rank)) - 1;
 }
-// chunk attention on tcgen05 (two 128-row slots per block), after the staging pages were written
+// staging pages (old ring pairs + chunk pairs as pages in the workspace), then the chunk attention
+// on tcgen05 (two 128-row slots per block)
+int launch_prefill_stage(const PrefillArgs &a, cudaStream_t s);
 int launch_prefill_attn_tc5x2h(const PrefillArgs &a, cudaStream_t s);
 size_t prefill_split_bytes(const spkv_config_t *cfg, int C);   // partial results of split page walks (small chunks)
 

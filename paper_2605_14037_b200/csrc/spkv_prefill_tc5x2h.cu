@@ -65,7 +65,8 @@ constexpr int kSQ = 0;                     // 2 x 32 KB: Q of head 0, head 1 (tw
 constexpr int kStages = 5;
 constexpr int kSKV = 65536;                // kStages x 32 KB
 constexpr int kSBar = kSKV + kStages * kPageBytes;
-constexpr int kSmemBytes = kSBar + 512;
+constexpr int kSGate = kSBar + 512;        // kStages x 64 floats: gate bias of a stage's keys (soft-gated forward)
+constexpr int kSmemBytes = kSGate + kStages * kP * 4;
 enum { B_KV_FULL = 0, B_KV_EMPTY = 8, B_V_READY = 16 /* [stage] */, B_S_FULL = 24 /* [h] */, B_S_FREE = 26 /* [h] */,
        B_P_FULL = 28 /* [2h+b] */, B_O_DONE = 32 /* [2h+b] */, B_COUNT = 36 };
 constexpr int kConvThreads = 64;           // warps 2-3
@@ -129,7 +130,11 @@ __device__ inline bool value_scale(uint32_t vm, int force_wide, float &v_scale, 
 }
 
 // kEvenG: every block is a head pair on one tile (the branches for single heads compile away).
-template <bool kEvenG>
+// kSoft: the soft-gated whole-sequence forward (Eq. 6): no compact-cache pages, the walk covers
+// every causal page of the sequence, and a key beyond a query's window is not masked but biased
+// by the logarithm of its gate.  The gate biases of a page's 64 keys travel with the page into
+// shared memory (one 256-byte bulk copy on the same barrier), once per page for all 256 rows.
+template <bool kEvenG, bool kSoft>
 __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kernel(PrefillArgs a) {
   using namespace tc5;
   using namespace tc5x2h;
@@ -152,13 +157,14 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
   float v_scale, v_unscale;
   const bool wide = value_scale((uint32_t)hdr[H_VMAX], a.force_wide, v_scale, v_unscale);
   // kept pairs visible to chunk query i: the first nvis(i) pairs of the compact cache
-  auto nvis = [&](int i) { return len0 + E[min(max(i + n_old - c.w + 1, 0), N)]; };
+  auto nvis = [&](int i) { return kSoft ? 0 : len0 + E[min(max(i + n_old - c.w + 1, 0), N)]; };
   // the last query of the block (slot 1 never starts before slot 0) sees the most kept pairs
   if (kEvenG) two = true;
   const int i_first = i0_s0, i_last = min((two ? i0_s1 : i0_s0) + 127, a.C - 1);
   const int n_ptiles = (nvis(i_last) + kP - 1) / kP;
-  // band of both slots together, in staging indices (query i is staging pair n_old + i)
-  const int sp_lo = max(0, i_first + n_old - c.w + 1) / kP, sp_hi = (i_last + n_old) / kP;
+  // band of both slots together, in staging indices (query i is staging pair n_old + i); the
+  // soft-gated forward walks every page from the start of the sequence
+  const int sp_lo = kSoft ? 0 : max(0, i_first + n_old - c.w + 1) / kP, sp_hi = (i_last + n_old) / kP;
   const int n_tiles_all = n_ptiles + (sp_hi - sp_lo + 1);
   // this block's share of the walk: pages [j_begin, j_begin + n_tiles) of the list (compact-cache
   // pages, then band pages); page numbers below are local, j_begin + j is the page's place in the list
@@ -232,7 +238,7 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
       const int jl = j_begin + base + lane;
       int64_t src_off = 0;
       if (jl < n_ptiles)   // (debug bounds: an entry that names no pool page is read from the unit's ring instead)
-        src_off = (int64_t)checked_page(c, c.table[(size_t)u * c.max_pages + jl], (int)ring_page(c, u, 0)) * kPageElems;
+        src_off = (int64_t)checked_page(c, unit_table(c, c.table_row[u])[jl], (int)ring_page(c, u, 0)) * kPageElems;
       const int cnt = min(32, n_tiles - base);
       for (int x = 0; x < cnt; ++x, ++j) {
         const int64_t off = __shfl_sync(0xffffffffu, src_off, x);
@@ -244,8 +250,11 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
                 j_begin + j < n_ptiles
                     ? c.pages + off
                     : a.stage_pages + ((size_t)kvh * a.n_stage_pages + sp_lo + (j_begin + j - n_ptiles)) * kPageElems;
-            mbar_arrive_expect_tx(&bar[B_KV_FULL + s], kPageBytes);
+            mbar_arrive_expect_tx(&bar[B_KV_FULL + s], kPageBytes + (kSoft ? kP * 4 : 0));
             bulk_load(smem + kSKV + s * kPageBytes, src, kPageBytes, &bar[B_KV_FULL + s]);
+            if (kSoft)   // the gate biases of the page's 64 keys
+              bulk_load(smem + kSGate + s * kP * 4,
+                        a.gate2 + ((size_t)kvh * a.n_stage_pages + (j_begin + j)) * kP, kP * 4, &bar[B_KV_FULL + s]);
           }
         }
         failed = __shfl_sync(0xffffffffu, (int)failed, 0) != 0;
@@ -371,7 +380,39 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
       // v keeps the raw scores (masked ones become -inf); the scale is folded into the exponent,
       // and pages that every row of the warp sees in full skip the masking altogether.
       const int jg = j_begin + j;   // the page's place in the list
-      if (jg < n_ptiles) {
+      float mx;
+      if (kSoft) {
+        // Eq. 6: score * scale + bias, bias = 0 inside the window, log2 of the key's gate before
+        // it, -inf for the future.  v becomes the biased score in the log2 domain.
+        const int base = jg * kP;
+        // the copy that brought the page also brought its gate biases (completed before the scores
+        // were committed; observing the barrier here makes the bytes visible to this thread)
+        if (!mbar_wait_bounded(&bar[B_KV_FULL + j % kStages], (j / kStages) & 1)) { failed = true; break; }
+        const float4 *gs = reinterpret_cast<const float4 *>(smem + kSGate + (j % kStages) * kP * 4);
+        if (__all_sync(0xffffffffu, row_ok && base + kP - 1 <= jq - c.w)) {
+          // the whole page lies before the window of every row of this warp: gate bias everywhere
+#pragma unroll
+          for (int x4 = 0; x4 < 16; ++x4) {
+            const float4 g4 = gs[x4];
+            v[4 * x4] = fmaf(v[4 * x4], a.scale_log2, g4.x);
+            v[4 * x4 + 1] = fmaf(v[4 * x4 + 1], a.scale_log2, g4.y);
+            v[4 * x4 + 2] = fmaf(v[4 * x4 + 2], a.scale_log2, g4.z);
+            v[4 * x4 + 3] = fmaf(v[4 * x4 + 3], a.scale_log2, g4.w);
+          }
+        } else {
+#pragma unroll
+          for (int x4 = 0; x4 < 16; ++x4) {
+            const float4 g4 = gs[x4];
+            const float gg[4] = {g4.x, g4.y, g4.z, g4.w};
+#pragma unroll
+            for (int y = 0; y < 4; ++y) {
+              const int jj = base + 4 * x4 + y;
+              const float sc = fmaf(v[4 * x4 + y], a.scale_log2, jj > jq - c.w ? 0.f : gg[y]);
+              v[4 * x4 + y] = (row_ok && jj <= jq) ? sc : -INFINITY;
+            }
+          }
+        }
+      } else if (jg < n_ptiles) {
         const int base = jg * kP;
         if (!__all_sync(0xffffffffu, base + kP <= nv)) {
 #pragma unroll
@@ -393,7 +434,8 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
         mx2 = max3(mx2, v[x + 4], v[x + 5]);
         mx3 = max3(mx3, v[x + 6], v[x + 7]);
       }
-      const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * a.scale_log2;  // scale > 0 (host-checked)
+      // (the hard-gated path keeps raw scores in v and folds the scale, > 0, into the exponent)
+      mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * (kSoft ? 1.f : a.scale_log2);
       // the reference maximum moves only when the row maximum outgrows it by 2^8
       const bool grow = mx > m_ref + 8.f;
       const float m_new = grow ? mx : m_ref;
@@ -444,7 +486,8 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
 #pragma unroll
           for (int x = 0; x < 16; ++x) {
             float e0, e1, r0, r1;
-            unpack2(fma2(pack2(v[q2 * 32 + 2 * x], v[q2 * 32 + 2 * x + 1]), sc2, nms2), e0, e1);
+            const uint64_t v2 = pack2(v[q2 * 32 + 2 * x], v[q2 * 32 + 2 * x + 1]);
+            unpack2(kSoft ? add2(v2, nms2) : fma2(v2, sc2, nms2), e0, e1);
             const float p0 = fast_exp2(e0), p1 = fast_exp2(e1);
             const uint64_t p2 = pack2(p0, p1);
             if (x & 1) l2b = add2(l2b, p2); else l2a = add2(l2a, p2);
@@ -465,7 +508,8 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
 #pragma unroll
           for (int x = 0; x < 16; ++x) {
             float e0, e1;
-            unpack2(fma2(pack2(v[q2 * 32 + 2 * x], v[q2 * 32 + 2 * x + 1]), sc2, nms2), e0, e1);
+            const uint64_t v2 = pack2(v[q2 * 32 + 2 * x], v[q2 * 32 + 2 * x + 1]);
+            unpack2(kSoft ? add2(v2, nms2) : fma2(v2, sc2, nms2), e0, e1);
             const float p0 = fast_exp2(e0), p1 = fast_exp2(e1);
             const uint64_t p2 = pack2(p0, p1);
             if (x & 1) l2b = add2(l2b, p2); else l2a = add2(l2a, p2);
@@ -515,6 +559,8 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
       fence_after();
       const float inv = l > 0.f ? 1.f / l : 0.f;  // the bias of P cancels between O and l
       __nv_bfloat16 *orow = a.out + ((size_t)i * c.Hq + hq) * kD;
+      if (a.lse && row_ok)   // l = sum 2^(s - m_ref + bias)
+        a.lse[(size_t)i * c.Hq + hq] = (m_ref - (wide ? 0.f : kPBias) + log2f(l)) * 0.6931471805599453f;
 #pragma unroll
       for (int q8 = 0; q8 < 8; ++q8) {
         float t16[16];
@@ -561,7 +607,7 @@ __global__ void __launch_bounds__(256) prefill_merge_kernel(PrefillArgs a) {
   if (h == 1 && !ws.two) return;
   const int hq = h ? ws.hq1 : ws.hq0, i0 = h ? ws.i01 : ws.i00;
   float v_scale, v_unscale;
-  value_scale((uint32_t)unit_ws(a, ws.kvh)[H_VMAX], a.force_wide, v_scale, v_unscale);
+  const bool wide = value_scale((uint32_t)unit_ws(a, ws.kvh)[H_VMAX], a.force_wide, v_scale, v_unscale);
   const float *part = a.partials + (size_t)(walk * 2 + h) * S * kPartFloats;
   __shared__ float s_w[kMaxSplit][128];   // weight of share s for a row, already divided by the row sum
   for (int row = threadIdx.x; row < 128; row += blockDim.x) {
@@ -576,6 +622,8 @@ __global__ void __launch_bounds__(256) prefill_merge_kernel(PrefillArgs a) {
     }
     const float inv = L > 0.f ? 1.f / L : 0.f;
     for (int s = 0; s < S; ++s) s_w[s][row] *= inv;
+    if (a.lse && i0 + row < a.C)   // the shares' l carry the same bias of P as the unsplit kernel's
+      a.lse[(size_t)(i0 + row) * c.Hq + hq] = (M - (wide ? 0.f : kPBias) + log2f(L)) * 0.6931471805599453f;
   }
   __syncthreads();
   for (int x = threadIdx.x; x < 128 * 8; x += blockDim.x) {
@@ -631,7 +679,8 @@ size_t prefill_split_bytes(const spkv_config_t *cfg, int C) {
 
 int launch_prefill_attn_tc5x2h(const PrefillArgs &a_in, cudaStream_t s) {
   PrefillArgs a = a_in;
-  auto kernel = (a.c.G & 1) ? prefill_attn_tc5x2h_kernel<false> : prefill_attn_tc5x2h_kernel<true>;
+  auto kernel = a.soft ? ((a.c.G & 1) ? prefill_attn_tc5x2h_kernel<false, true> : prefill_attn_tc5x2h_kernel<true, true>)
+                       : ((a.c.G & 1) ? prefill_attn_tc5x2h_kernel<false, false> : prefill_attn_tc5x2h_kernel<true, false>);
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc5x2h::kSmemBytes) != cudaSuccess)
     return SPKV_E_CUDA;
   const int n_xtiles = (a.C + 127) / 128;

@@ -37,7 +37,8 @@ class Config(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("max_seqs", C.c_int32), ("n_q_heads", C.c_int32),
                 ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("window", C.c_int32),
                 ("page_tokens", C.c_int32), ("max_context", C.c_int32), ("pool_pages", C.c_int64),
-                ("tau", C.c_float), ("flags", C.c_int32), ("sink_tokens", C.c_int32)]
+                ("tau", C.c_float), ("flags", C.c_int32), ("sink_tokens", C.c_int32),
+                ("h_local_only", C.c_void_p)]
 
 
 class Predictor(C.Structure):
@@ -100,6 +101,9 @@ def lib():
         "spkv_decode_attention_static": (C.c_int, [vp, i32, vp, i32, vp, vp, vp, f32, vp]),
         "spkv_prefill_workspace_bytes": (sz, [cfgp, i32]),
         "spkv_prefill": (C.c_int, [vp, i32, i32, i32, vp, vp, vp, vp, vp, f32, vp, sz, vp]),
+        "spkv_softgate_workspace_bytes": (sz, [i32, i32, i32]),
+        "spkv_softgate_forward": (C.c_int, [i32, i32, i32, i32, vp, vp, vp, vp, f32, f32, f32, i32, vp, vp, vp, sz,
+                                            vp, vp]),
         "spkv_decode_step_staging_bytes": (sz, [cfgp, i32, i32]),
         "spkv_decode_step_host": (C.c_int, [vp, i32, pp, vp, i32, vp, vp, vp, vp, vp, f32, vp, sz, vp]),
         "spkv_decode_step_host_flush": (C.c_int, [vp, vp]),
@@ -160,9 +164,17 @@ class Cache:
 
     def __init__(self, n_layers, max_seqs, n_q_heads, n_kv_heads, max_context, pool_pages,
                  window=128, tau=0.5, device="cuda:0", head_dim=128, page_tokens=64, sink_tokens=0,
-                 flags=0):
+                 flags=0, local_only=None):
+        """local_only: optional [n_layers, n_kv_heads] array, non-zero = that head is declared
+        local-only (window attention, no page table, not scored by the fused append)."""
+        import numpy as np
+        self._local_only = None
+        if local_only is not None:
+            self._local_only = np.ascontiguousarray(np.asarray(local_only) != 0, dtype=np.uint8)
+            assert self._local_only.shape == (n_layers, n_kv_heads)
         self.cfg = Config(n_layers, max_seqs, n_q_heads, n_kv_heads, head_dim, window, page_tokens,
-                          max_context, pool_pages, tau, flags, sink_tokens)
+                          max_context, pool_pages, tau, flags, sink_tokens,
+                          self._local_only.ctypes.data if self._local_only is not None else None)
         self.device = torch.device(device)
         n = C.c_size_t()
         _check(lib().spkv_arena_bytes(C.byref(self.cfg), C.byref(n)), "spkv_arena_bytes")
@@ -449,6 +461,38 @@ def spkv_stream_read(buf, passes=5, stream=None):
     if int(status.item()) != 0:
         raise SpkvError(int(status.item()), "spkv_stream_read")
     return nbytes * passes / (e0.elapsed_time(e1) * 1e-3) / 1e9
+
+
+_softgate_ws = {}
+
+
+def spkv_softgate_forward(q, k, v, logits, window=128, alpha=0.0, tau=0.5, sm_scale=None, flags=0, out=None,
+                          want_lse=False, stream=None, status=None):
+    """Soft-gated whole-sequence forward (Eq. 6 / Eq. 7; see spkv.h).  q [T,Hq,128], k, v [T,Hkv,128]
+    bf16, logits [T,Hkv] float32 on one device -> out [T,Hq,128] bf16 (and lse [T,Hq] float32).
+    status: an int32 device tensor of one zero that receives the device-side verdict; when given,
+    the call does not synchronise and the caller reads it; otherwise the call waits and raises."""
+    T, Hq, Hkv = q.shape[0], q.shape[1], k.shape[1]
+    if out is None:
+        out = torch.empty_like(q)
+    lse = torch.empty((T, Hq), dtype=torch.float32, device=q.device) if want_lse else None
+    nbytes = lib().spkv_softgate_workspace_bytes(T, Hq, Hkv)
+    ws = _softgate_ws.get(q.device)
+    if ws is None or ws.numel() < nbytes:
+        ws = _softgate_ws[q.device] = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=q.device)
+    own_status = status is None
+    if own_status:
+        status = torch.zeros(1, dtype=torch.int32, device=q.device)
+    _check(lib().spkv_softgate_forward(
+        T, Hq, Hkv, window, _ptr(q, torch.bfloat16), _ptr(k, torch.bfloat16), _ptr(v, torch.bfloat16),
+        _ptr(logits, torch.float32), alpha, tau, 1.0 / math.sqrt(q.shape[2]) if sm_scale is None else sm_scale,
+        flags, _ptr(out, torch.bfloat16), _ptr(lse), _ptr(ws), ws.numel(), _ptr(status), _stream(stream)),
+        "spkv_softgate_forward")
+    if own_status:
+        code = int(status.item())      # synchronises: the status word is the call's device-side verdict
+        if code != 0:
+            raise SpkvError(code, "spkv_softgate_forward (device)")
+    return (out, lse) if want_lse else out
 
 
 def spkv_wait_selftest(buf, limit_clocks, stream=None):

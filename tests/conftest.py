@@ -13,6 +13,8 @@ def pytest_configure(config):
 
 
 def pytest_collection_modifyitems(config, items):
+    if not any("gpu" in item.keywords for item in items):
+        return          # nothing to decide: do not pay for importing torch
     try:
         import torch
         has_gpu = torch.cuda.is_available()

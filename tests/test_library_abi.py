@@ -159,6 +159,27 @@ def test_canary_blocks_lie_between_the_metadata_regions(spkv):
     assert spkv.lib().spkv_arena_canaries(C.byref(c), offs, 16, C.byref(n)) == 0
     assert spkv.lib().spkv_arena_bytes(C.byref(c), C.byref(total)) == 0
     o = list(offs)[:n.value]
-    assert n.value == 10 and o == sorted(o) and o[0] == 256 and all(x % 256 == 0 for x in o)
+    assert n.value == 11 and o == sorted(o) and o[0] == 256 and all(x % 256 == 0 for x in o)
     units = 2 * 3 * 2
     assert o[-1] + 256 <= total.value - (units * 2 + 100) * 32768     # all before the pages
+
+
+def test_local_only_heads_cost_no_page_table(spkv):
+    """Static hybrid layout declared at creation: the arena shrinks by exactly the page tables of the
+    local-only heads' units."""
+    import numpy as np
+    n_all, n_some, n_none = C.c_size_t(), C.c_size_t(), C.c_size_t()
+    c = cfg(spkv, n_layers=3, max_seqs=5, n_q_heads=8, n_kv_heads=4, max_context=64 * 1024)
+    assert spkv.lib().spkv_arena_bytes(C.byref(c), C.byref(n_all)) == 0
+    flags = np.zeros((3, 4), np.uint8)
+    flags[0, :] = 1
+    flags[2, 1] = 1                       # 5 of the 12 heads
+    c.h_local_only = flags.ctypes.data
+    assert spkv.lib().spkv_arena_bytes(C.byref(c), C.byref(n_some)) == 0
+    assert n_all.value - n_some.value == 5 * 5 * 1024 * 4          # heads x sequences x entries x 4 bytes
+    flags[:] = 1
+    assert spkv.lib().spkv_arena_bytes(C.byref(c), C.byref(n_none)) == 0
+    assert n_all.value - n_none.value == 12 * 5 * 1024 * 4
+    big = cfg(spkv, n_q_heads=130, n_kv_heads=65)
+    big.h_local_only = flags.ctypes.data
+    assert spkv.lib().spkv_arena_bytes(C.byref(big), C.byref(n_none)) == -3

@@ -60,10 +60,11 @@ def test_planted_mistake_is_caught(tmp_path, name, old, new, count):
     src.write_text(mutated)
     subprocess.check_call(["gcc", "-O1", "-std=c99", "-fPIC", "-shared", "-fopenmp", "-o", str(lib), str(src), "-lm"])
     env = dict(os.environ, SPKV_ORACLE_LIB=str(lib))
+    # the pins of the part of the oracle the mistake sits in (soft-gated forward / everything else)
+    soft = name.startswith(("soft_", "anneal_"))
+    files = ["test_oracle_soft.py"] if soft else ["test_oracle_pins.py", "test_oracle_sinks.py"]
     r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider",
-                        os.path.join(ROOT, "tests", "test_oracle_pins.py"),
-                        os.path.join(ROOT, "tests", "test_oracle_sinks.py"),
-                        os.path.join(ROOT, "tests", "test_oracle_soft.py")],
+                        *[os.path.join(ROOT, "tests", f) for f in files]],
                        cwd=ROOT, env=env, capture_output=True, text=True, timeout=600)
     out = r.stdout + r.stderr
     assert r.returncode == 1 and " failed" in out, f"mutant {name} survived the pins:\n{out[-800:]}"
