@@ -190,11 +190,18 @@ class Cache:
         self.default_scale = 1.0 / math.sqrt(head_dim)
 
     @classmethod
-    def attach(cls, arena, cfg, tau=None, flags=None):
+    def attach(cls, arena, cfg, tau=None, flags=None, local_only=None):
         """A Cache over an arena tensor that already holds one (a copy of another cache's arena):
-        spkv_cache_attach.  `cfg` is the Config the arena was created with; tau / flags override."""
+        spkv_cache_attach.  `cfg` is the Config the arena was created with; tau / flags override;
+        local_only as at creation (it is part of the layout and has to be given again)."""
+        import numpy as np
         self = cls.__new__(cls)
         self.cfg = Config.from_buffer_copy(cfg)
+        self._local_only = None
+        if local_only is not None:
+            self._local_only = np.ascontiguousarray(np.asarray(local_only) != 0, dtype=np.uint8)
+            assert self._local_only.shape == (cfg.n_layers, cfg.n_kv_heads)
+        self.cfg.h_local_only = self._local_only.ctypes.data if self._local_only is not None else None
         if tau is not None:
             self.cfg.tau = tau
         if flags is not None:
