@@ -285,7 +285,11 @@ size_t spkv_decode_workspace_bytes(const spkv_config_t *cfg, int32_t B);
  *   d_lse_opt [B, n_q_heads] float32 natural-log sum-exp of the scaled scores, or NULL;
  *   d_workspace: >= spkv_decode_workspace_bytes(cfg, B) bytes, 256-byte aligned, used by
  *   this cache only; it must have been zero-filled once before its first use and is then
- *   left alone by the caller (consecutive calls alternate between its two halves). */
+ *   left alone by the caller (consecutive calls alternate between its two halves).
+ *   Under SPKV_FLAG_OVERLAP a launch starts beneath the tail of the previous decode launch only
+ *   if both calls were given the SAME workspace and batch size (the two then use different
+ *   halves); with another workspace or batch the launch is an ordinary stream-ordered one --
+ *   the result is the same, only the overlap is lost. */
 int spkv_decode_attention(spkv_cache_t *cache, int32_t layer, const int32_t *d_seq_ids,
                           int32_t B, const void *d_q, void *d_out, float *d_lse_opt,
                           float sm_scale, void *d_workspace, size_t workspace_bytes,
