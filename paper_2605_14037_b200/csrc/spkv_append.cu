@@ -51,7 +51,7 @@ __device__ inline void append_unit(const CacheView &c, int layer, const int32_t 
   const int u = unit_index(c, layer, seq, kvh);
   // a head declared local-only keeps nothing and has no page table: its utility is never looked
   // at, so it is not computed either (its logit is written as 0)
-  const bool local_only = (local_mask >> kvh) & 1ULL;
+  const bool local_only = kvh < 64 && ((local_mask >> kvh) & 1ULL);
   // fused scoring (Eq. 1, linear predictor): this unit's logit for the new pair
   float new_logit;
   if (local_only) {

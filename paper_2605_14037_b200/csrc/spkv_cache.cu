@@ -95,6 +95,21 @@ __global__ void set_head_tau_kernel(float *head_tau, int first, int count, float
   if (i < count) head_tau[first + i] = value;
 }
 
+// Page-table rows of one layer's units: row = base_row + seq * (global heads of the layer) + rank of
+// the head among them; -1 for the units of a local-only head, whose threshold becomes +inf.
+__global__ void init_table_rows_kernel(int32_t *table_row, float *head_tau, int layer, int S, int Hkv,
+                                       unsigned long long local_mask, int32_t base_row) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= S * Hkv) return;
+  const int seq = i / Hkv, h = i % Hkv;
+  const bool local = Hkv <= 64 && ((local_mask >> h) & 1ULL);
+  const unsigned long long all = Hkv >= 64 ? ~0ULL : ((1ULL << Hkv) - 1ULL);
+  const int n_global = Hkv <= 64 ? __popcll(~local_mask & all) : Hkv;
+  const int rank = Hkv <= 64 ? __popcll(~local_mask & ((1ULL << h) - 1ULL)) : h;
+  table_row[((size_t)layer * S + seq) * Hkv + h] = local ? -1 : base_row + seq * n_global + rank;
+  if (local && seq == 0) head_tau[layer * Hkv + h] = INFINITY;
+}
+
 __global__ void init_free_stack_kernel(int32_t *stack, int32_t *free_top, int64_t pool_pages,
                                        int64_t first) {
   int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -236,18 +251,15 @@ extern "C" int spkv_cache_create(const spkv_config_t *cfg, void *d_arena, size_t
     set_head_tau_kernel<<<(nh + 255) / 256, 256, 0, s>>>(v.head_tau, 0, nh, NAN);
     // page-table rows in (layer, sequence, KV head) order, local-only heads skipped; such a head
     // also carries the keep-nothing threshold for good
-    std::vector<int32_t> rows((size_t)v.n_units);
-    int32_t next = 0;
-    for (int l2 = 0; l2 < v.L; ++l2)
-      for (int sq = 0; sq < v.S; ++sq)
-        for (int h = 0; h < v.Hkv; ++h)
-          rows[((size_t)l2 * v.S + sq) * v.Hkv + h] = ((c->local_mask[l2] >> h) & 1ULL) ? -1 : next++;
-    e = cudaMemcpyAsync(v.table_row, rows.data(), rows.size() * 4, cudaMemcpyHostToDevice, s);
-    if (e == cudaSuccess) e = cudaStreamSynchronize(s);   // `rows` is pageable host memory about to go away
-    for (int l2 = 0; l2 < v.L && e == cudaSuccess; ++l2)
-      for (int h = 0; h < v.Hkv; ++h)
-        if ((c->local_mask[l2] >> h) & 1ULL)
-          set_head_tau_kernel<<<1, 32, 0, s>>>(v.head_tau, l2 * v.Hkv + h, 1, INFINITY);
+    int32_t base_row = 0;
+    for (int l2 = 0; l2 < v.L; ++l2) {
+      const unsigned long long m = c->local_mask[l2];
+      init_table_rows_kernel<<<(v.S * v.Hkv + 255) / 256, 256, 0, s>>>(v.table_row, v.head_tau, l2, v.S, v.Hkv, m, base_row);
+      int n_global = 0;
+      for (int h = 0; h < v.Hkv; ++h) n_global += (h < 64 && ((m >> h) & 1ULL)) ? 0 : 1;
+      base_row += n_global * v.S;
+    }
+    e = cudaGetLastError();
   }
   if (e == cudaSuccess && v.pool_pages > 0) {
     int64_t n = v.pool_pages;
@@ -375,7 +387,7 @@ extern "C" int spkv_safe_steps(spkv_cache_t *cache, const int32_t *h_seq_ids, in
   for (int l = 0; l < v.L; ++l)
     for (int b = 0; b < (B ? B : v.S); ++b)
       for (int h = 0; h < v.Hkv; ++h) {
-        if ((cache->local_mask[l] >> h) & 1ULL) continue;   // a local-only head never needs a page
+        if (h < 64 && ((cache->local_mask[l] >> h) & 1ULL)) continue;   // a local-only head never needs a page
         const int u = (l * v.S + (B ? h_seq_ids[b] : b)) * v.Hkv + h;
         sl.push_back(len[u]);
         st.push_back(t[u]);
@@ -426,7 +438,7 @@ extern "C" int spkv_set_head_tau(spkv_cache_t *cache, int32_t layer, int32_t kv_
   if (!cache || layer < 0 || layer >= cache->view.L || kv_head < -1 || kv_head >= cache->view.Hkv)
     return SPKV_E_INVALID;
   // a head declared local-only at creation has no page table: it stays local-only
-  const unsigned long long target = kv_head < 0 ? ~0ULL : 1ULL << kv_head;
+  const unsigned long long target = kv_head < 0 ? ~0ULL : (kv_head < 64 ? 1ULL << kv_head : 0ULL);
   if (cache->local_mask[layer] & target) return SPKV_E_INVALID;
   const float value = tau != tau ? NAN : tau_to_logit(tau);
   const int first = layer * cache->view.Hkv + (kv_head < 0 ? 0 : kv_head);

@@ -35,13 +35,13 @@ def test_attach_to_a_copy_of_the_arena_continues_where_the_original_was():
     torch.cuda.synchronize()
     # snapshot = a plain copy of the arena, placed somewhere else (here through the host)
     copy = cache.arena.cpu().to(dev())
-    h = C.c_void_p()
+    hnd = C.c_void_p()
     s0 = C.c_void_p(torch.cuda.current_stream().cuda_stream)
     # which heads are local-only is part of the layout: an attach that declares some is refused
     flags = np.array([[1, 0]], np.uint8)
     wrong = spkv.Config.from_buffer_copy(cache.cfg)
     wrong.h_local_only = flags.ctypes.data
-    assert spkv.lib().spkv_cache_attach(C.byref(wrong), C.c_void_p(copy.data_ptr()), copy.numel(), s0, C.byref(h)) == -15
+    assert spkv.lib().spkv_cache_attach(C.byref(wrong), C.c_void_p(copy.data_ptr()), copy.numel(), s0, C.byref(hnd)) == -15
     twin = spkv.Cache.attach(copy, cache.cfg)
     feed(twin, wl, 300, T)
     feed(cache, wl, 300, T)
@@ -62,11 +62,11 @@ def test_attach_to_a_copy_of_the_arena_continues_where_the_original_was():
     assert spkv.lib().spkv_arena_bytes(C.byref(other), C.byref(n)) == 0
     big = torch.zeros(max(n.value, copy.numel()), dtype=torch.uint8, device=dev())
     big[:copy.numel()] = copy
-    assert spkv.lib().spkv_cache_attach(C.byref(other), C.c_void_p(big.data_ptr()), big.numel(), s0, C.byref(h)) == -15
+    assert spkv.lib().spkv_cache_attach(C.byref(other), C.c_void_p(big.data_ptr()), big.numel(), s0, C.byref(hnd)) == -15
     blank = torch.zeros(copy.numel(), dtype=torch.uint8, device=dev())
     assert spkv.lib().spkv_cache_attach(C.byref(cache.cfg), C.c_void_p(blank.data_ptr()), blank.numel(), s0,
-                                        C.byref(h)) == -15
-    assert spkv.lib().spkv_cache_attach(C.byref(cache.cfg), C.c_void_p(copy.data_ptr()), 1024, s0, C.byref(h)) == -2
+                                        C.byref(hnd)) == -15
+    assert spkv.lib().spkv_cache_attach(C.byref(cache.cfg), C.c_void_p(copy.data_ptr()), 1024, s0, C.byref(hnd)) == -2
 
 
 def test_rollback_replays_the_same_steps_bit_for_bit():

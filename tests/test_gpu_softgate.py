@@ -69,7 +69,8 @@ def test_softgate_forward_every_row(T, G, Hkv, w, alpha):
 
 
 @pytest.mark.parametrize("T,G,Hkv,alpha,flags", [(4096, 4, 2, 0.0, 0), (4096, 8, 1, 0.25, 0), (4096, 1, 4, 0.0, 2),
-                                                 (16384, 4, 2, 0.0, 0), (16384, 8, 2, 0.0, 0), (16500, 3, 2, 0.0, 0)])
+                                                 (16384, 4, 2, 0.0, 0), (16384, 8, 2, 0.0, 0), (16500, 3, 2, 0.0, 0),
+                                                 (32768, 4, 8, 0.0, 0)])      # the last: the shape bench.py --softgate-T times
 def test_softgate_forward_long_sequences_sampled_rows(T, G, Hkv, alpha, flags):
     """4 K and 16 K sequences (whole page walks, pages far before every window of a warp take the
     fast path): sampled rows around the tile, page and window boundaries and at the end."""
