@@ -17,7 +17,7 @@
  *     caller; the library never allocates or frees device memory.
  *   - `stream` is a cudaStream_t passed as a plain pointer (NULL = default stream).
  *     Calls only enqueue work on it; the only calls that synchronise are spkv_status,
- *     spkv_cache_stats and the spkv_read_* helpers.
+ *     spkv_cache_stats, spkv_safe_steps, spkv_cache_attach and the spkv_read_* helpers.
  *   - bf16 tensors are dense, row-major, 16-byte aligned.  head_dim is 128.
  *   - Argument errors are reported synchronously.  Errors found on the device (pool
  *     exhausted, context overflow, a bounded wait that ran out) are recorded in a sticky
