@@ -40,6 +40,7 @@ CONFIGS = {
     5: dict(name="config5_llama70b_b8_ctx64k", L=80, B=8, Hq=64, Hkv=8, T=65536, beta=(0.5, 2.5)),
 }
 W, D_IN, TAU, CHUNK = 128, 512, 0.5, 8192
+CACHE_FLAGS = [1]          # SPKV_FLAG_OVERLAP; --stream-ordered clears it
 
 
 def peaks():
@@ -217,7 +218,7 @@ def build_workload(spkv, synth, torch, cfg, dev, dense, total_steps, seed=0, tau
         pool_pages = int(per_seq.sum())
     cache = spkv.Cache(n_layers=L, max_seqs=B, n_q_heads=Hq, n_kv_heads=Hkv,
                        max_context=t_final + 64, pool_pages=pool_pages, window=W, tau=tau, device=dev,
-                       flags=spkv.FLAG_OVERLAP)   # attention-only stack, inputs staged before the step
+                       flags=CACHE_FLAGS[0])   # overlap: attention-only stack, inputs staged before the step
     preds, keep = [], []
     for l in range(L):
         Wl, bl = pred_np[l]
@@ -521,7 +522,7 @@ def run_ours(args):
                    "density": sp["density"], "kv_gb_per_step": sp["kv_gb_per_step"],
                    "l2": "inputs larger than L2 (K/V read per step >> 126 MB)" if sp["kv_gb_per_step"] > 0.5
                          else "working set smaller than L2: latency-bound case",
-                   "cuda_graph": sp["graph"], "launch_overlap": "SPKV_FLAG_OVERLAP", "parallelism": "replicas only" if world > 1 else "single GPU"},
+                   "cuda_graph": sp["graph"], "launch_overlap": "SPKV_FLAG_OVERLAP" if CACHE_FLAGS[0] else "off (stream-ordered launches)", "parallelism": "replicas only" if world > 1 else "single GPU"},
         "clocks": sp["clocks"], "repeats": sp["repeats"],
         "gpu_launches": 2 * L * K,
         # In overlap mode consecutive decode launches run under each other's head and tail, so a
@@ -876,6 +877,9 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--settle-seconds", type=float, default=1.0,
                     help="untimed replay of the timed region before the first repeat (clocks settle under load)")
+    ap.add_argument("--stream-ordered", action="store_true",
+                    help="create the cache without SPKV_FLAG_OVERLAP: every launch waits for the previous one, as "
+                         "in a model whose layers depend on each other (comparison run, not the bench line)")
     ap.add_argument("--softgate-T", type=int, default=0,
                     help="measure the soft-gated whole-sequence forward on this many tokens instead (not the bench line)")
     ap.add_argument("--sweep-tau", default="",
@@ -887,6 +891,8 @@ def main():
         sys.exit(subprocess.call(replica_launch_command(args.gpus, sys.argv[1:])))
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
+    if args.stream_ordered:
+        CACHE_FLAGS[0] = 0
     if args.impl == "reference":
         run_reference(args)
     elif args.softgate_T > 0:

@@ -108,7 +108,9 @@ typedef struct {
  * do not write the same d_out.  That holds for an attention-only stack (the benchmark) and for
  * a model that stages a whole step's inputs beforehand; a model that computes q, k, v of a
  * layer between the library's calls must leave the flag off (every launch then waits for all
- * earlier work, as any stream-ordered kernel does).  Any other call of the library (prefill,
+ * earlier work, as any stream-ordered kernel does; the library still issues its hot-path kernels
+ * as programmatic dependent launches, so their block-local set-up runs under the tail of the
+ * previous kernel, but they execute griddepcontrol.wait before touching an input or the cache).  Any other call of the library (prefill,
  * score, reset, ...) is a full synchronisation point either way. */
 #define SPKV_FLAG_OVERLAP 1
 

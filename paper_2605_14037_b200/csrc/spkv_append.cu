@@ -165,17 +165,19 @@ static int append_must_wait(spkv_cache *cache, int layer, cudaStream_t s) {
   return independent ? 0 : 1;
 }
 
-// Plain stream-ordered launch unless the cache is in overlap mode.  Blocks of two warps: small
-// enough to fit on an SM beside a resident decode block (320 threads x 168 registers leave
-// 11.7 K registers), which is what lets the append of the next layer run under the decode.
+// Every launch is a programmatic dependent launch: the blocks may become resident and run their
+// block-local prologue while the previous kernel of the stream is still finishing.  Without
+// SPKV_FLAG_OVERLAP (and in overlap mode whenever the host cannot vouch for the preceding launches)
+// the kernel then executes griddepcontrol.wait before it touches any input or the cache, i.e. it
+// is ordered after everything earlier on the stream exactly as a plain launch would be; only the
+// launch latency is hidden.  Blocks of two warps: small enough to fit on an SM beside a resident
+// decode block (320 threads x 168 registers leave 11.7 K registers), which is what lets the
+// append of the next layer run under the decode in overlap mode.
 constexpr int kAppendThreads = 64;
 template <class... Args>
 static int launch_append(spkv_cache *cache, int items, cudaStream_t s, Args... args) {
   const int per = kAppendThreads / 32, grid = (items + per - 1) / per;
-  if (!(cache->cfg.flags & SPKV_FLAG_OVERLAP)) {
-    append_evict_kernel<<<grid, kAppendThreads, 0, s>>>(args...);
-    return check_stream_error(cudaGetLastError());
-  }
+  (void)cache;
   return check_stream_error(launch_overlapped(append_evict_kernel, dim3(grid), dim3(kAppendThreads), 0, s, args...));
 }
 

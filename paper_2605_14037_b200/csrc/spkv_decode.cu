@@ -801,7 +801,9 @@ static int decode_attention_impl(spkv_cache_t *cache, int32_t layer, const int32
   a.lse = d_lse_opt;
   a.scale_log2 = sm_scale * kLog2e;
   a.snap = 6;       // measured best on the 32 K and 128 K workloads (0, 2, 4, 6, 8, 12 tried)
-  a.min_pos = 56;   // likewise (32 ... 96 tried)
+  // likewise (32 ... 96 tried) where launches overlap: the SMs a launch leaves idle work for its
+  // neighbours.  A stream-ordered launch has no neighbours to share with and takes every SM.
+  a.min_pos = (cache->cfg.flags & SPKV_FLAG_OVERLAP) ? 56 : 12;
   // Two consecutive decode launches may overlap (the next one starts on the SMs this one
   // has left): they alternate between the two halves of the workspace.  A third cannot
   // join: it needs every block of the second resident, i.e. every SM left by the first.
@@ -844,10 +846,8 @@ static int decode_attention_impl(spkv_cache_t *cache, int32_t layer, const int32
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total) != cudaSuccess)
     return SPKV_E_CUDA;
   const int grid = min(kMaxGrid, cache->sm_count);
-  if (!(cache->cfg.flags & SPKV_FLAG_OVERLAP)) {  // plain stream-ordered launch
-    kernel<<<grid, kTcThreads, L.total, s>>>(a, GP, n_stages, red_bufs);
-    return check_stream_error(cudaGetLastError());
-  }
+  // (a programmatic dependent launch in every mode: with wait_mode 0 the kernel runs only its
+  // block-local prologue before griddepcontrol.wait orders it after everything earlier on the stream)
   return check_stream_error(
       launch_overlapped(kernel, dim3(grid), dim3(kTcThreads), (size_t)L.total, s, a, GP, n_stages, red_bufs));
 }
