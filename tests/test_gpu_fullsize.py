@@ -23,12 +23,14 @@ from paper_2605_14037_b200 import synth
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("B,Hq,Hkv,T,beta,sampled", [
-    (16, 32, 8, 32768, (0.5, 2.0), [3, 11]),
-    (4, 32, 8, 131072, (0.3, 3.0), [2]),
-    (8, 64, 8, 65536, (0.5, 2.5), [5]),
-], ids=["config2", "config3", "config5"])
-def test_one_layer_full_size(B, Hq, Hkv, T, beta, sampled):
+@pytest.mark.parametrize("B,Hq,Hkv,T,beta,sampled,overlap", [
+    (16, 32, 8, 32768, (0.5, 2.0), [3, 11], True),
+    (4, 32, 8, 131072, (0.3, 3.0), [2], True),
+    (8, 64, 8, 65536, (0.5, 2.5), [5], True),
+    # without the overlap flag a launch takes every SM (shorter ranges, more units split over blocks)
+    (4, 32, 8, 131072, (0.3, 3.0), [1], False),
+], ids=["config2", "config3", "config5", "config3_stream_ordered"])
+def test_one_layer_full_size(B, Hq, Hkv, T, beta, sampled, overlap):
     spkv = load()
     w, C, steps = 128, 8192, 3
     G = Hq // Hkv
@@ -37,7 +39,8 @@ def test_one_layer_full_size(B, Hq, Hkv, T, beta, sampled):
     rates[0], rates[5] = 0.0, 0.97                       # a local-only head and a near-full head
     pages = int(np.ceil(rates * (T + steps) * 1.05 / 64 + 2).sum()) * B
     cache = spkv.Cache(n_layers=1, max_seqs=B, n_q_heads=Hq, n_kv_heads=Hkv, max_context=T + 128,
-                       pool_pages=pages, window=w, tau=0.5, flags=spkv.FLAG_OVERLAP)   # as bench.py creates it
+                       pool_pages=pages, window=w, tau=0.5,
+                       flags=spkv.FLAG_OVERLAP if overlap else 0)   # as bench.py creates it / --stream-ordered
     tl = cache.spkv_tau_logit()
     Tt = T + steps
     logit = np.stack([synth.logits_with_keep_rate(rng, (Tt, B), float(r), tl) for r in rates], axis=-1)
