@@ -803,7 +803,7 @@ static int decode_attention_impl(spkv_cache_t *cache, int32_t layer, const int32
   a.snap = 6;       // measured best on the 32 K and 128 K workloads (0, 2, 4, 6, 8, 12 tried)
   // likewise (32 ... 96 tried) where launches overlap: the SMs a launch leaves idle work for its
   // neighbours.  A stream-ordered launch has no neighbours to share with and takes every SM.
-  a.min_pos = (cache->cfg.flags & SPKV_FLAG_OVERLAP) ? 56 : 12;
+  a.min_pos = (cache->cfg.flags & SPKV_FLAG_OVERLAP) ? 56 : 4;
   // Two consecutive decode launches may overlap (the next one starts on the SMs this one
   // has left): they alternate between the two halves of the workspace.  A third cannot
   // join: it needs every block of the second resident, i.e. every SM left by the first.

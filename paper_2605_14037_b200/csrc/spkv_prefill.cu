@@ -32,6 +32,7 @@ namespace spkv {
 
 // ---------------------------------------------------------------- A: plan (flags + scan)
 __global__ void __launch_bounds__(1024) prefill_plan_kernel(PrefillArgs a) {
+  pdl_chain_link();
   const CacheView &c = a.c;
   const int kvh = blockIdx.x;
   const int u = unit_index(c, a.layer, a.seq, kvh);
@@ -150,6 +151,7 @@ __device__ inline uint4 load_chunk(const __nv_bfloat16 *rowbase, int row, int ch
 // ------------------------------------------------------------------ B: scatter (compact)
 // grid (ceil(n_leave_max / 64), Hkv); each warp moves 8 consecutive staging pairs.
 __global__ void __launch_bounds__(256) prefill_scatter_kernel(PrefillArgs a) {
+  pdl_chain_link();
   const CacheView &c = a.c;
   const int kvh = blockIdx.y;
   const int32_t *hdr = unit_ws(a, kvh);
@@ -183,6 +185,7 @@ __global__ void __launch_bounds__(256) prefill_scatter_kernel(PrefillArgs a) {
 // --------------------------------------------------------------------- C: ring update
 // grid (ceil(min(C,w) / 8), Hkv); one warp per pair.
 __global__ void __launch_bounds__(256) prefill_ring_kernel(PrefillArgs a) {
+  pdl_chain_link();
   const CacheView &c = a.c;
   const int kvh = blockIdx.y;
   const int32_t *hdr = unit_ws(a, kvh);
@@ -210,6 +213,7 @@ __global__ void __launch_bounds__(256) prefill_ring_kernel(PrefillArgs a) {
 // Old ring pairs and chunk pairs, in position order, rewritten as pages (workspace).
 // grid (n_stage_pages, Hkv), 256 threads: 8 warps x 8 rows.
 __global__ void __launch_bounds__(256) prefill_stage_kernel(PrefillArgs a) {
+  pdl_chain_link();
   const CacheView &c = a.c;
   const int kvh = blockIdx.y, sp = blockIdx.x;
   int32_t *hdr = unit_ws(a, kvh);
@@ -240,8 +244,7 @@ __global__ void __launch_bounds__(256) prefill_stage_kernel(PrefillArgs a) {
 }
 
 int launch_prefill_stage(const PrefillArgs &a, cudaStream_t s) {
-  prefill_stage_kernel<<<dim3(a.n_stage_pages, a.c.Hkv), 256, 0, s>>>(a);
-  return check_stream_error(cudaGetLastError());
+  return check_stream_error(launch_link(a.chained != 0, prefill_stage_kernel, dim3(a.n_stage_pages, a.c.Hkv), dim3(256), 0, s, a));
 }
 
 static size_t prefill_ws_stride_ints(int C, int w) {
@@ -302,6 +305,7 @@ extern "C" int spkv_prefill(spkv_cache_t *cache, int32_t layer, int32_t seq, int
   a.soft = 0;
   a.gate2 = nullptr;
   a.lse = nullptr;
+  a.chained = C < 64;   // measured: see pdl_chain_link
   a.partials = prefill_split_bytes(&cache->cfg, C)
                    ? reinterpret_cast<float *>(reinterpret_cast<char *>(a.stage_pages) +
                                                (size_t)v.Hkv * a.n_stage_pages * kPageBytes)
@@ -309,15 +313,15 @@ extern "C" int spkv_prefill(spkv_cache_t *cache, int32_t layer, int32_t seq, int
   cudaStream_t s = as_stream(stream);
   cache->last_kind = kLastOther;
 
-  prefill_plan_kernel<<<v.Hkv, 1024, 0, s>>>(a);
+  if (launch_link(a.chained != 0, prefill_plan_kernel, dim3(v.Hkv), dim3(1024), 0, s, a) != cudaSuccess) return SPKV_E_CUDA;
   // at most max(min(t0,w) + C - w, 0) <= C pairs leave the window
-  prefill_scatter_kernel<<<dim3((C + 63) / 64, v.Hkv), 256, 0, s>>>(a);
+  if (launch_link(a.chained != 0, prefill_scatter_kernel, dim3((C + 63) / 64, v.Hkv), dim3(256), 0, s, a) != cudaSuccess)
+    return SPKV_E_CUDA;
   if (d_q) {
     int rc = launch_prefill_stage(a, s);
     if (!rc) rc = launch_prefill_attn_tc5x2h(a, s);
     if (rc) return rc;
   }
   const int n_ring = C < v.w ? C : v.w;
-  prefill_ring_kernel<<<dim3((n_ring + 7) / 8, v.Hkv), 256, 0, s>>>(a);
-  return check_stream_error(cudaGetLastError());
+  return check_stream_error(launch_link(a.chained != 0, prefill_ring_kernel, dim3((n_ring + 7) / 8, v.Hkv), dim3(256), 0, s, a));
 }

@@ -31,6 +31,7 @@ struct PrefillArgs {
   int soft;
   const float *gate2;              // [Hkv][n_stage_pages * 64] (soft only)
   float *lse;                      // [C][Hq] natural-log sum-exp of the biased scaled scores, or null
+  int chained;                     // host: launch the call's kernels as a chain of dependent launches (small chunks)
 };
 
 __device__ inline int32_t *unit_ws(const PrefillArgs &a, int kvh) { return a.ws + (size_t)kvh * a.ws_stride; }

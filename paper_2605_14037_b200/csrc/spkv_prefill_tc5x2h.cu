@@ -139,6 +139,7 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
   using namespace tc5;
   using namespace tc5x2h;
   extern __shared__ __align__(1024) unsigned char smem[];
+  pdl_chain_link();
   const CacheView &c = a.c;
   uint64_t *bar = reinterpret_cast<uint64_t *>(smem + kSBar);
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + kSBar + B_COUNT * 8);
@@ -601,6 +602,7 @@ extern "C" int spkv_debug_tc5h_trace(long long *host_out) {
 template <bool kEvenG>
 __global__ void __launch_bounds__(256) prefill_merge_kernel(PrefillArgs a) {
   using namespace tc5x2h;
+  pdl_chain_link();
   const CacheView &c = a.c;
   const int walk = blockIdx.x, h = blockIdx.y, S = a.n_split;
   const WalkSlots ws = walk_slots<kEvenG>(a, walk);
@@ -697,10 +699,12 @@ int launch_prefill_attn_tc5x2h(const PrefillArgs &a_in, cudaStream_t s) {
   const int n_walks = per_kvh * a.c.Hkv;
   a.n_split = a.partials ? prefill_split_count(n_walks, std::min(sms, 192)) : 1;
   a.n_split = (int)std::max(1LL, std::min<long long>(a.n_split, split_slots(a.C, a.c.G, a.c.Hkv) / n_walks));
-  kernel<<<dim3(n_walks * a.n_split), tc5x2h::kThreads, tc5x2h::kSmemBytes, s>>>(a);
+  if (launch_link(a.chained != 0, kernel, dim3(n_walks * a.n_split), dim3(tc5x2h::kThreads), (size_t)tc5x2h::kSmemBytes, s,
+                  a) != cudaSuccess)
+    return SPKV_E_CUDA;
   if (a.n_split > 1) {
-    if (a.c.G & 1) prefill_merge_kernel<false><<<dim3(n_walks, 2), 256, 0, s>>>(a);
-    else           prefill_merge_kernel<true><<<dim3(n_walks, 2), 256, 0, s>>>(a);
+    auto merge = (a.c.G & 1) ? prefill_merge_kernel<false> : prefill_merge_kernel<true>;
+    if (launch_link(a.chained != 0, merge, dim3(n_walks, 2), dim3(256), 0, s, a) != cudaSuccess) return SPKV_E_CUDA;
   }
   return check_stream_error(cudaGetLastError());
 }

@@ -15,6 +15,7 @@ __global__ void __launch_bounds__(256)
 score_linear_kernel(const __nv_bfloat16 *__restrict__ x, int n_tok, int d_in,
                     const __nv_bfloat16 *__restrict__ W, const float *__restrict__ b, int Hkv,
                     float tau_logit, float *__restrict__ logits, uint8_t *__restrict__ flags) {
+  pdl_chain_link();
   const int lane = threadIdx.x & 31;
   const int tok = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (tok >= n_tok) return;
@@ -72,9 +73,9 @@ extern "C" int spkv_score(spkv_cache_t *cache, const spkv_predictor_t *p, const 
   cache->last_kind = kLastOther;
   const __nv_bfloat16 *x = static_cast<const __nv_bfloat16 *>(d_x);
   if (p->kind == 0) {
-    score_linear_kernel<<<(n_tok + 7) / 8, 256, 0, s>>>(
-        x, n_tok, p->d_in, static_cast<const __nv_bfloat16 *>(p->d_W1), p->d_b1, Hkv,
-        cache->tau_logit, d_logits_out, d_flags_out);
+    return check_stream_error(launch_link(
+        n_tok < 64, score_linear_kernel, dim3((n_tok + 7) / 8), dim3(256), 0, s, x, n_tok, (int)p->d_in,
+        static_cast<const __nv_bfloat16 *>(p->d_W1), p->d_b1, Hkv, cache->tau_logit, d_logits_out, d_flags_out));
   } else if (p->kind == 1) {
     if (!p->d_W2 || !p->d_b2 || p->hidden < 1 || p->hidden > 8192) return SPKV_E_INVALID;
     // chunks of tokens at model width go to the tensor cores; a handful of tokens (decode) or an

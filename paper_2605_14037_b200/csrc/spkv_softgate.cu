@@ -28,6 +28,7 @@ __device__ inline float gate_log2(float logit, float alpha, float tau_logit) {
 // grid (n_stage_pages, Hkv), 64 threads: the gate biases of one page of keys; block (0, kvh) also
 // writes the plan header the attention kernel reads (an empty cache, a "chunk" of T pairs).
 __global__ void __launch_bounds__(64) softgate_prepare_kernel(PrefillArgs a, float *gate2, float alpha) {
+  pdl_chain_link();
   const int kvh = blockIdx.y, s = blockIdx.x * kP + threadIdx.x;
   gate2[((size_t)kvh * a.n_stage_pages + blockIdx.x) * kP + threadIdx.x] =
       s < a.C ? gate_log2(a.logits[(size_t)s * a.c.Hkv + kvh], alpha, a.tau_logit) : 0.f;
@@ -104,8 +105,9 @@ extern "C" int spkv_softgate_forward(int32_t T, int32_t n_q_heads, int32_t n_kv_
   a.gate2 = reinterpret_cast<const float *>(ws + w.off_gate);
   a.lse = d_lse_opt;
   cudaStream_t s = as_stream(stream);
-  softgate_prepare_kernel<<<dim3(w.n_pages, n_kv_heads), 64, 0, s>>>(a, reinterpret_cast<float *>(ws + w.off_gate), alpha);
-  int rc = check_stream_error(cudaGetLastError());
+  a.chained = T < 64;
+  int rc = check_stream_error(launch_link(a.chained != 0, softgate_prepare_kernel, dim3(w.n_pages, n_kv_heads), dim3(64), 0, s,
+                                          a, reinterpret_cast<float *>(ws + w.off_gate), alpha));
   if (!rc) rc = launch_prefill_stage(a, s);
   if (!rc) rc = launch_prefill_attn_tc5x2h(a, s);
   return rc;
