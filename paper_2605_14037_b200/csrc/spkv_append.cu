@@ -52,6 +52,20 @@ __device__ inline void append_unit(const CacheView &c, int layer, const int32_t 
   // a head declared local-only keeps nothing and has no page table: its utility is never looked
   // at, so it is not computed either (its logit is written as 0)
   const bool local_only = kvh < 64 && ((local_mask >> kvh) & 1ULL);
+  // The kernel is a chain of dependent trips to memory, so the loads are issued in three rounds
+  // rather than where the control flow first needs them.  Round 1 (above): the sequence id.
+  // Round 2, everything that depends on the unit alone: pairs received, kept length, page-table
+  // row, the head's own threshold, and the new pair itself.  Metadata is read from L2 (in overlap
+  // mode this kernel does not start at a stream-wide synchronisation point, and an SM's L1 is not
+  // coherent with other SMs' stores).
+  const int t = __ldcg(&c.t[u]);
+  const int n = __ldcg(&c.len[u]);
+  const int trow = local_only ? -1 : unit_table_row(c, u);
+  const float thr = head_threshold(c, layer, kvh, tau_logit);
+  // lanes 0-15 move the key row, lanes 16-31 the value row, one 16-byte chunk each
+  const int chunk = lane & 15;
+  const int blk = (lane >> 4) * kBlockElems;
+  const uint4 new_cell = ((lane < 16 ? k_new : v_new) + (size_t)item * 16)[chunk];
   // fused scoring (Eq. 1, linear predictor): this unit's logit for the new pair
   float new_logit;
   if (local_only) {
@@ -63,56 +77,50 @@ __device__ inline void append_unit(const CacheView &c, int layer, const int32_t 
   } else {
     new_logit = logits[item];
   }
-  // metadata and the evicted pair are read from L2: in overlap mode this kernel does not start at a
-  // stream-wide synchronisation point, and an SM's L1 is not coherent with other SMs' stores
-  const int t = __ldcg(&c.t[u]);
   const int slot = t % c.w;
   const int row = slot % kP;
-  // lanes 0-15 move the key row, lanes 16-31 the value row, one 16-byte chunk each
-  const int chunk = lane & 15;
-  const int blk = (lane >> 4) * kBlockElems;
   __nv_bfloat16 *ring = c.pages + ring_page(c, u, slot / kP) * kPageElems;
   uint4 *ring_cell = reinterpret_cast<uint4 *>(ring + blk + swz_off(row, chunk));
+  // Round 3, what depends on t and the length: the stored logit of the pair that leaves the window,
+  // the pair itself and the page-table entry it would go to (read whether or not it is kept).
+  const bool leaves = t >= c.w && trow >= 0;
+  const int pj = n / kP, prow = n % kP;
+  int32_t *table = unit_table(c, trow >= 0 ? trow : 0);
+  const float lg = __ldcg(&c.ring_logit[(size_t)u * c.w + slot]);
+  const uint4 evictee = __ldcg(ring_cell);
+  const int page_at_tail = (leaves && prow != 0 && pj < c.max_pages) ? __ldcg(&table[pj]) : -1;
 
-  if (t >= c.w && !local_only) {
-    // the pair of position t - w leaves the window: threshold decision on its stored logit
+  if (leaves && (lg >= thr || t - c.w < c.n_sink)) {
+    // the pair of position t - w leaves the window and passes the threshold on its stored logit
     // (sink positions are kept regardless)
-    const float lg = __ldcg(&c.ring_logit[(size_t)u * c.w + slot]);
-    if (lg >= head_threshold(c, layer, kvh, tau_logit) || t - c.w < c.n_sink) {
-      const int n = __ldcg(&c.len[u]);
-      int32_t *table = unit_table(c, unit_table_row(c, u));
-      const int pj = n / kP, prow = n % kP;
-      int page = -1, err = 0;
-      if (pj >= c.max_pages) {
-        err = SPKV_E_CONTEXT_OVERFLOW;
-      } else if (prow == 0) {
-        page = alloc_page(c, lane);
-        if (page == -1) err = SPKV_E_POOL_EXHAUSTED;
-        else if (page < 0) err = SPKV_E_BOUNDS_PAGE;
-        else if (lane == 0) table[pj] = page;
-      } else {
-        page = checked_page(c, __ldcg(&table[pj]), -2);
-        if (page < 0) err = SPKV_E_BOUNDS_PAGE;   // the evicted pair is dropped, as on exhaustion
-      }
-      if (err) {
-        if (lane == 0) set_status(c, err);
-      } else {
-        __syncwarp();
-        __nv_bfloat16 *dst = c.pages + (int64_t)page * kPageElems;
-        const uint4 kept = __ldcg(ring_cell);
-        *reinterpret_cast<uint4 *>(dst + blk + swz_off(prow, chunk)) = kept;
-        // the compact cache's largest |value| (the prefill attention picks its value scale by it)
-        const uint32_t vm = __reduce_max_sync(0xffffffffu, lane < 16 ? 0u : chunk_abs_max_bf16(kept));
-        if (lane == 0) {
-          c.pos_pool[((int64_t)page - c.n_ring_pages_total) * kP + prow] = t - c.w;
-          c.len[u] = n + 1;
-          note_vmax(c, u, vm);
-        }
+    int page = -1, err = 0;
+    if (pj >= c.max_pages) {
+      err = SPKV_E_CONTEXT_OVERFLOW;
+    } else if (prow == 0) {
+      page = alloc_page(c, lane);
+      if (page == -1) err = SPKV_E_POOL_EXHAUSTED;
+      else if (page < 0) err = SPKV_E_BOUNDS_PAGE;
+      else if (lane == 0) table[pj] = page;
+    } else {
+      page = checked_page(c, page_at_tail, -2);
+      if (page < 0) err = SPKV_E_BOUNDS_PAGE;   // the evicted pair is dropped, as on exhaustion
+    }
+    if (err) {
+      if (lane == 0) set_status(c, err);
+    } else {
+      __syncwarp();
+      __nv_bfloat16 *dst = c.pages + (int64_t)page * kPageElems;
+      *reinterpret_cast<uint4 *>(dst + blk + swz_off(prow, chunk)) = evictee;
+      // the compact cache's largest |value| (the prefill attention picks its value scale by it)
+      const uint32_t vm = __reduce_max_sync(0xffffffffu, lane < 16 ? 0u : chunk_abs_max_bf16(evictee));
+      if (lane == 0) {
+        c.pos_pool[((int64_t)page - c.n_ring_pages_total) * kP + prow] = t - c.w;
+        c.len[u] = n + 1;
+        note_vmax(c, u, vm);
       }
     }
   }
-  const uint4 *src = (lane < 16 ? k_new : v_new) + (size_t)item * 16 + chunk;
-  *ring_cell = *src;
+  *ring_cell = new_cell;
   if (lane == 0) {
     c.ring_logit[(size_t)u * c.w + slot] = new_logit;
     c.t[u] = t + 1;
