@@ -811,17 +811,19 @@ static int decode_attention_impl(spkv_cache_t *cache, int32_t layer, const int32
   char *ws = static_cast<char *>(d_workspace) + (size_t)half * wl.total;
   cache->ws_toggle ^= 1;
   // Overlap mode: directly after this layer's append on the same stream the kernel need not wait
-  // for the whole stream, only for that append and for the previous user of its workspace half
-  // (which must be another layer: a block cannot tell its own launch's blocks from older ones).
+  // for the whole stream, only for that append and for the previous user of its workspace half.
+  // When that user was a decode launch of this same layer (one- and two-layer stacks), the wait
+  // for the append covers it: the append, launched after that decode, itself waited for every
+  // decode launch of its layer before it touched the cache.  (The kernel could not wait for it
+  // directly: a block cannot tell its own launch's count from older ones.)
   a.wait_mode = ((cache->cfg.flags & SPKV_FLAG_OVERLAP) && cache->last_kind == kLastAppend &&
                  cache->last_layer == layer && cache->last_stream == as_stream(stream) &&
-                 cache->half_last_layer[half] != layer &&
                  // same workspace, cut into the same halves, as the launch it may run beside
                  cache->last_decode_items == n_items && cache->last_decode_ws == d_workspace)
                     ? 1 : 0;
   cache->last_decode_items = n_items;
   cache->last_decode_ws = d_workspace;
-  a.prev_half_layer = cache->half_last_layer[half];
+  a.prev_half_layer = cache->half_last_layer[half] == layer ? -1 : cache->half_last_layer[half];
   cache->half_last_layer[half] = layer;
   cache->appends_pending[layer] = 0;
   cache->last_kind = kLastDecode;
