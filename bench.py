@@ -336,12 +336,16 @@ def run_ours(args):
             """CUDA graphs of steps first ... first + n - 1 (capturing runs nothing)."""
             if args.no_graph:
                 return
-            for step in range(first, first + n):
+            step = first
+            while step < first + n:
+                cnt = min(max(1, args.steps_per_graph), first + n - step)
                 if step not in graphs:
                     g = torch.cuda.CUDAGraph()
                     with torch.cuda.graph(g):
-                        layer_calls(step)
-                    graphs[step] = g
+                        for j in range(cnt):
+                            layer_calls(step + j)
+                    graphs[step] = (g, cnt)
+                step += graphs[step][1]
 
         if not args.no_graph:
             side = torch.cuda.Stream(device=dev)
@@ -354,12 +358,15 @@ def run_ours(args):
 
         def run_steps(n, events=None):
             """n steps starting at step number step_no[0]."""
-            for i in range(n):
+            i = 0
+            while i < n:
                 step = step_no[0] + i
-                if step in graphs and events is None:
-                    graphs[step].replay()
+                if step in graphs and events is None and graphs[step][1] <= n - i:
+                    graphs[step][0].replay()
+                    i += graphs[step][1]
                 else:
                     layer_calls(step, events=None if events is None else events[i])
+                    i += 1
             step_no[0] += n
 
         run_steps(Wm)
@@ -528,7 +535,7 @@ def run_ours(args):
                    "density": sp["density"], "kv_gb_per_step": sp["kv_gb_per_step"],
                    "l2": "inputs larger than L2 (K/V read per step >> 126 MB)" if sp["kv_gb_per_step"] > 0.5
                          else "working set smaller than L2: latency-bound case",
-                   "cuda_graph": sp["graph"], "launch_overlap": "SPKV_FLAG_OVERLAP" if CACHE_FLAGS[0] else "off (stream-ordered launches)", "parallelism": "replicas only" if world > 1 else "single GPU"},
+                   "cuda_graph": sp["graph"], "steps_per_graph": max(1, args.steps_per_graph), "launch_overlap": "SPKV_FLAG_OVERLAP" if CACHE_FLAGS[0] else "off (stream-ordered launches)", "parallelism": "replicas only" if world > 1 else "single GPU"},
         "clocks": sp["clocks"], "repeats": sp["repeats"],
         "gpu_launches": 2 * L * K,
         # In overlap mode consecutive decode launches run under each other's head and tail, so a
@@ -883,6 +890,9 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--settle-seconds", type=float, default=1.0,
                     help="untimed replay of the timed region before the first repeat (clocks settle under load)")
+    ap.add_argument("--steps-per-graph", type=int, default=1,
+                    help="steps captured in one CUDA graph (default 1; more shows the device time of a "
+                         "tiny step where the host's replay rate is the limit)")
     ap.add_argument("--stream-ordered", action="store_true",
                     help="create the cache without SPKV_FLAG_OVERLAP: every launch waits for the previous one, as "
                          "in a model whose layers depend on each other (comparison run, not the bench line)")
