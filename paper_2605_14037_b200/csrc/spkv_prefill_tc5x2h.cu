@@ -24,33 +24,48 @@
 //   maximum is 2^20 or more the blocks of
 //   such a unit -- and every block when the cache was created with SPKV_FLAG_PREFILL_PV_BF16 --
 //   leave the values in bf16 and split P into hi + lo bf16 terms (16 significant bits, bf16's
-//   exponent range): 8 P.V MMAs per page instead of 4, one P buffer per head instead of two (a
-//   group then waits for P.V of the previous page before it overwrites P).  Same pipeline, same
-//   barriers; the branch is uniform per block.
+//   exponent range): 8 P.V MMAs per page instead of 4.  The branch is uniform per block.
 //
-// * P has tensor-memory columns of its own instead of overwriting the scores it came from.  A
-//   group copies its row of S into registers and hands the S buffer back at once, so Q.K^T of the
-//   next page runs under the softmax of this one and never waits for P; only P.V does.  With P
-//   aliased onto S, Q.K^T(j+2) had to queue behind P.V(j), and scores, softmax and P.V of a head
-//   formed one dependent loop whose latency, not the tensor pipe, set the pace.
+// Two pipelines, chosen at compile time (kDeep = !kSoft): the hard-gated kernel runs the deep one,
+// the soft-gated kernel -- whose softmax groups do more per page (gate biases) and set the pace by
+// themselves -- the flat one; each measured 3-8 % faster than the other in its place.
 //
-// Tensor memory (512 columns): S of head h at [64 h, +64); P buffer b of head h at
-// [128 + 32 (2h + b), +32) (two fp16 per column; a wide unit: hi at [128 + 64 h, +32), lo in the
-// 32 columns after it); O of head h at [256 + 128 h, +128).
-// MMA order per page j:  QK0(j+1) | PV0(j) | QK1(j+1) | PV1(j).  The two heads' scores become
-// ready half a page apart, which keeps the two groups out of step: the exponentials of one
-// (special-function unit, the scarce resource) run under the load / maximum / hand-over phases of
-// the other instead of both queueing for the same unit at the same time.
+// * Deep (hard-gated).  Two score buffers per head, and P written back over the scores it came
+//   from.  A group copies its row of S(j) into registers, and when the exponentials are done
+//   stores P(j) into the first columns of the same buffer; Q.K^T(j+2) goes into that buffer after
+//   P.V(j) has read it (the tensor pipe runs a thread's MMAs in order), Q.K^T(j+1) went into the
+//   other one a page earlier.  So a group always finds its next scores waiting.  One MMA-issuing
+//   warp per head: the tensor pipe takes only a few instructions ahead, the issuing thread blocks
+//   until the pipe accepts an MMA, and whatever else that warp does -- wait for a P, commit, turn
+//   its loop -- is time in which it feeds the pipe nothing (measured: every 100 cycles of delay put
+//   into a single issuing warp's loop lengthened the page period by 75-83).  With a warp per
+//   head, each running  wait P(j) | PV(j) | QK(j+2) | commit  for its own head, one head's MMAs
+//   fill the gaps of the other's.
+//   Tensor memory (512 columns): score buffer b = j & 1 of head h at [64 (2h + b), +64), P(j) in
+//   its first 32 columns (two fp16 per column; a wide unit: hi in the first 32, lo in the other
+//   32); O of head h at [256 + 128 h, +128).
+//
+// * Flat (soft-gated).  One score buffer per head and P in columns of its own; a group copies its
+//   row of S into registers and hands the buffer back at once (S_FREE), so Q.K^T of the next page
+//   runs under the softmax of this one and only P.V waits for P.  One MMA warp, order per page j:
+//   QK0(j+1) | PV0(j) | QK1(j+1) | PV1(j): the two heads' scores become ready half a page apart,
+//   which keeps the two groups out of step.
+//   Tensor memory: S of head h at [64 h, +64); P buffer b of head h at [128 + 32 (2h + b), +32)
+//   (a wide unit: hi at [128 + 64 h, +32), lo in the 32 columns after it, one buffer per head:
+//   a group then waits for P.V of the previous page before it overwrites P); O as above.
 //
 // A launch with fewer page walks than SMs (a chunk of a few hundred tokens) cuts every walk into
 // up to 16 shares of consecutive pages, one block each; a share writes its unnormalised rows and
 // their (m, l), and prefill_merge_kernel combines the shares by their log-sum-exp weights.
 //
-// No unit is saturated (tensor pipe ~54 % active, special-function unit ~41 %, issue slots ~54 %):
-// the page period is the length of the chain scores -> softmax -> P -> MMA warp -> next scores.
-// Shared memory: Q of both heads (64 KB) + 5 page stages.
-// Warps: 0 MMA issue, 1 page loader + TMEM allocation, 2-3 value conversion, 4-7 group 0,
-// 8-11 group 1.  All waits are bounded.
+// What sets the pace of the deep pipeline is the softmax groups: with their scores always waiting
+// they are busy ~85 % of the page period, each slowed by the other (alone a group needs ~1060
+// cycles per page, side by side ~1550), and no unit is saturated (special-function unit ~60 %,
+// issue slots ~55 %); in the flat pipeline it is the chain scores -> softmax -> P -> MMA warp ->
+// next scores.
+// Shared memory: Q of both heads (64 KB) + 5 page stages (deep: pages j .. j+2 in use).
+// Warps: 0 MMA issue (deep: head 0), 1 page loader + TMEM allocation, 2-3 value conversion,
+// 4-7 group 0, 8-11 group 1, 12 MMA issue head 1 (deep only).  All waits are bounded.
 #include <algorithm>
 
 #include "spkv_prefill_common.cuh"
@@ -59,7 +74,12 @@
 namespace spkv {
 
 namespace tc5x2h {
-constexpr int kThreads = 384;
+constexpr int kThreads = 416;
+// Warp roles.  Both MMA-issuing warps sit on scheduler 0 (warp % 4), the loader on 1, the value
+// converters on 2 and 3; every scheduler also runs one warp of each softmax group.  (Measured:
+// the MMA warps on different schedulers, or the conversion spread over four warps, lose 1-4 %.)
+constexpr int kMmaWarp0 = 0, kMmaWarp1 = 12, kLoaderWarp = 1;
+__host__ __device__ constexpr bool is_conv(int w) { return w == 2 || w == 3; }
 constexpr int kTmemCols = 512;
 constexpr int kSQ = 0;                     // 2 x 32 KB: Q of head 0, head 1 (two slabs of 128 rows x 128 B each)
 constexpr int kStages = 5;
@@ -67,8 +87,8 @@ constexpr int kSKV = 65536;                // kStages x 32 KB
 constexpr int kSBar = kSKV + kStages * kPageBytes;
 constexpr int kSGate = kSBar + 512;        // kStages x 64 floats: gate bias of a stage's keys (soft-gated forward)
 constexpr int kSmemBytes = kSGate + kStages * kP * 4;
-enum { B_KV_FULL = 0, B_KV_EMPTY = 8, B_V_READY = 16 /* [stage] */, B_S_FULL = 24 /* [h] */, B_S_FREE = 26 /* [h] */,
-       B_P_FULL = 28 /* [2h+b] */, B_O_DONE = 32 /* [2h+b] */, B_COUNT = 36 };
+enum { B_KV_FULL = 0, B_KV_EMPTY = 8, B_V_READY = 16 /* [stage] */, B_S_FULL = 24 /* [2h+b] */,
+       B_P_FULL = 28 /* [2h+b] */, B_O_DONE = 32 /* [2h+b] */, B_S_FREE = 36 /* [h], flat pipeline only */, B_COUNT = 38 };
 constexpr int kConvThreads = 64;           // warps 2-3
 constexpr float kPBias = 7.f;              // P is stored as 2^7 p
 constexpr int kPartFloats = 128 * 128 + 128 * 2;   // one partial result: O of 128 rows, then (m, l) per row
@@ -78,7 +98,10 @@ constexpr int kMinSharePages = 16;          // a walk is not cut into shares sho
 
 #ifdef SPKV_TC5_TRACE
 __device__ long long g_tc5h_trace[16][2048];
-#define TC5H_STAMP(cond, who, j) do { if ((cond) && (j) < 2048) g_tc5h_trace[who][j] = clock64(); } while (0)
+#ifndef SPKV_TC5_TRACE_MASK
+#define SPKV_TC5_TRACE_MASK 0xffff
+#endif
+#define TC5H_STAMP(cond, who, j) do { if (((SPKV_TC5_TRACE_MASK >> (who)) & 1) && (cond) && (j) < 2048) g_tc5h_trace[who][j] = clock64(); } while (0)
 #else
 #define TC5H_STAMP(cond, who, j) do { } while (0)
 #endif
@@ -138,6 +161,7 @@ template <bool kEvenG, bool kSoft>
 __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kernel(PrefillArgs a) {
   using namespace tc5;
   using namespace tc5x2h;
+  constexpr bool kDeep = !kSoft;   // which of the two pipelines (see the head of the file)
   extern __shared__ __align__(1024) unsigned char smem[];
   pdl_chain_link();
   const CacheView &c = a.c;
@@ -175,7 +199,7 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
   const int j_begin = split < n_shares ? (int)((long long)n_tiles_all * split / n_shares) : n_tiles_all;
   const int n_tiles = split < n_shares ? (int)((long long)n_tiles_all * (split + 1) / n_shares) - j_begin : 0;
   if (n_tiles == 0) {  // empty share (split walks only): says so in its partial result and leaves
-    if (warp >= 4) {
+    if (warp >= 4 && warp < 12) {
       const int h = (warp >> 2) - 1;
       if (h == 0 || two) {
         float *part = a.partials + ((size_t)(walk * 2 + h) * a.n_split + split) * kPartFloats;
@@ -189,23 +213,26 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
   if (tid == 0) {
     for (int i = 0; i < kStages; ++i) {
       mbar_init(&bar[B_KV_FULL + i], 1);
-      mbar_init(&bar[B_KV_EMPTY + i], 1);
+      mbar_init(&bar[B_KV_EMPTY + i], (kDeep && (kEvenG || ws.two)) ? 2 : 1);   // one commit per MMA warp at work
       mbar_init(&bar[B_V_READY + i], kConvThreads);
     }
-    // S_FULL / S_FREE: one barrier per head, one phase per page -- the MMA thread commits the
-    // scores of page j+1 only after the group has freed the buffer of page j, and the group frees
-    // it only after seeing it full, so the two are never more than one phase apart.
-    // P_FULL / O_DONE: one per head and page parity -- a group may hand over P(j+1) before the MMA
-    // thread has looked at P(j).  P(j+2) cannot follow before that: it needs the scores of page
-    // j+2, whose Q.K^T is issued after P.V(j).  O_DONE is committed for the last two pages only.
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(&bar[B_S_FULL + i], 1);
-      mbar_init(&bar[B_S_FREE + i], 128);
-    }
+    // Deep pipeline.  S_FULL / P_FULL / O_DONE: one barrier per head and page parity b = j & 1 (the
+    // score buffer the page uses), one phase per two pages.  The scores of page j+2 go into the
+    // buffer of page j and are issued after P.V(j), which needs P(j): a barrier is never more than
+    // one phase ahead of the group that waits on it.  O_DONE is committed for the last two pages.
+    // Flat pipeline.  S_FULL / S_FREE: one barrier per head (index 2h), one phase per page -- the
+    // MMA thread commits the scores of page j+1 only after the group has freed the buffer of page
+    // j, and the group frees it only after seeing it full, so the two are never more than one
+    // phase apart.  P_FULL / O_DONE per head and page parity: a group may hand over P(j+1) before
+    // the MMA thread has looked at P(j); P(j+2) cannot follow before that, it needs the scores of
+    // page j+2, whose Q.K^T is issued after P.V(j).
     for (int i = 0; i < 4; ++i) {
+      mbar_init(&bar[B_S_FULL + i], 1);
       mbar_init(&bar[B_P_FULL + i], 128);
       mbar_init(&bar[B_O_DONE + i], 1);
     }
+    mbar_init(&bar[B_S_FREE + 0], 128);
+    mbar_init(&bar[B_S_FREE + 1], 128);
     mbar_fence_init();
   }
   // Q tiles -> per head two slabs of 128 rows x 128 B, 128-byte swizzle (rows past the chunk are zero)
@@ -218,7 +245,7 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
     *reinterpret_cast<uint4 *>(smem + kSQ + h * 32768 + (ch >> 3) * 16384 + r * 128 + (((ch & 7) ^ (r & 7)) << 4)) = val;
   }
   fence_async_smem();
-  if (warp == 1) {
+  if (warp == kLoaderWarp) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
                  "n"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -232,7 +259,7 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
   const bool traced = blockIdx.x == 0;
 #endif
 
-  if (warp == 1) {
+  if (warp == kLoaderWarp) {
     // ---------------------------------------------------------------- page loader
     int j = 0;
     for (int base = 0; base < n_tiles && !failed; base += 32) {
@@ -265,8 +292,64 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
     if (failed && lane == 0)  // do not leave while copies may still be landing
       for (int k = max(0, j - kStages); k < j; ++k)
         mbar_wait_bounded(&bar[B_KV_FULL + (k % kStages)], (k / kStages) & 1);
-  } else if (warp == 0) {
+  } else if (kDeep && (warp == kMmaWarp0 || warp == kMmaWarp1)) {
     // ---------------------------------------------------------------- MMA issue (whole warp, one elected lane issues)
+    // Deep pipeline: one warp per head.  Issuing blocks while the tensor pipe's short queue is
+    // full, and everything else the warp does (barrier waits, commits, its loop) is time in which
+    // it feeds the pipe nothing; the other head's warp fills those gaps.
+    const int h_first = warp == kMmaWarp0 ? 0 : 1;
+    const int h_count = (h_first == 0 || two) ? 1 : 0;
+    constexpr uint32_t idesc_qk = instr_desc(128, 64, false), idesc_pv = instr_desc(128, 128, true, true),
+                       idesc_pv_bf16 = instr_desc(128, 128, true, false);
+    constexpr uint32_t kStageUnits = kPageBytes >> 4;   // a page stage in descriptor address units
+    const uint32_t kv0 = smem_u32(smem + kSKV);
+    const uint64_t dQ0 = smem_desc(smem_u32(smem + kSQ), 16, 1024);   // head 1: 32 KB = 2048 units later
+    const uint64_t dK = smem_desc(kv0, 16, 1024), dV = smem_desc(kv0 + kBlockElems * 2, 8192, 1024);
+    // S_h = Q_h . K^T of the page in `stage` into score buffer b, committed at once
+    auto issue_qk = [&](int h, uint32_t stage, uint32_t ph, uint32_t b) {
+      if (!mbar_wait_bounded(&bar[B_KV_FULL + stage], ph)) { failed = true; return; }
+      fence_after();
+      umma_qk_page<16384 / 16, 8192 / 16>(tbase + (2 * h + b) * 64, dQ0 + h * 2048, dK + stage * kStageUnits, idesc_qk);
+      umma_commit(&bar[B_S_FULL + 2 * h + b]);
+    };
+    const int n_mine = h_count ? n_tiles : 0;
+    for (int jj = 0; jj < min(2, n_mine) && !failed; ++jj)   // the scores of the first two pages
+      for (int h = h_first; h < h_first + h_count && !failed; ++h) issue_qk(h, jj, 0, jj);
+    uint32_t st = 0, ph = 0, st2 = 2, ph2 = 0;   // stage and phase parity of pages j and j + 2
+    for (int j = 0; j < n_mine && !failed; ++j) {
+      const uint32_t b = j & 1;
+      TC5H_STAMP(traced && lane == 0, 15 - h_first, j);
+      if (!mbar_wait_bounded(&bar[B_V_READY + st], ph)) { failed = true; break; }
+      for (int h = h_first; h < h_first + h_count && !failed; ++h) {
+        // O_h += P_h(j) . V(j): A = P from tensor memory (it lies where the page's scores lay), B =
+        // the page's value block (fp16 by now), MN-major
+        if (!mbar_wait_bounded(&bar[B_P_FULL + 2 * h + b], (j >> 1) & 1)) { failed = true; break; }
+        TC5H_STAMP(traced && lane == 0, 8 + h, j);
+        fence_after();
+        const uint32_t t_p = tbase + (2 * h + b) * 64, t_o = tbase + 256 + h * 128;
+        if (wide)
+          umma_pv_page(t_o, t_p, dV + st * kStageUnits, idesc_pv_bf16, j > 0 ? 1u : 0u);
+        else
+          umma_pv_page_f16(t_o, t_p, dV + st * kStageUnits, idesc_pv, j > 0 ? 1u : 0u);
+        TC5H_STAMP(traced && lane == 0, 13 - h, j);
+        if (j + 2 < n_tiles) {
+          // the tensor pipe runs a thread's instructions in order: Q.K^T(j+2) overwrites the buffer
+          // only after P.V(j) has read P from it, and its S_FULL vouches for that P.V
+          issue_qk(h, st2, ph2, b);
+        } else {
+          umma_commit(&bar[B_O_DONE + 2 * h + b]);   // the last two P.V have no later Q.K^T
+        }
+        TC5H_STAMP(traced && lane == 0, 11 - h, j);
+      }
+      if (failed) break;
+      umma_commit(&bar[B_KV_EMPTY + st]);  // this warp's head(s) have no use for page j any more
+      if (++st == kStages) { st = 0; ph ^= 1; }
+      if (++st2 == kStages) { st2 = 0; ph2 ^= 1; }
+    }
+  } else if (!kDeep && warp == kMmaWarp0) {
+    // ---------------------------------------------------------------- MMA issue, flat pipeline (whole warp, one elected lane issues)
+    // Order per page j:  QK0(j+1) | PV0(j) | QK1(j+1) | PV1(j).  The two heads' scores become ready
+    // half a page apart, which keeps the two groups out of step.
     constexpr uint32_t idesc_qk = instr_desc(128, 64, false), idesc_pv = instr_desc(128, 128, true, true),
                        idesc_pv_bf16 = instr_desc(128, 128, true, false);
     const uint32_t sQ = smem_u32(smem + kSQ);
@@ -288,7 +371,6 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
     // O_h += P_h(jj) . V(jj): A from tensor memory, B = the page's value block (fp16 by now), MN-major
     auto issue_pv = [&](int h, int jj) {
       if (!mbar_wait_bounded(&bar[B_P_FULL + 2 * h + (jj & 1)], (jj >> 1) & 1)) failed = true;
-      TC5H_STAMP(traced && lane == 0, 8 + h, jj);
       fence_after();
       if (failed) return;
       const uint32_t sV = smem_u32(smem + kSKV + (jj % kStages) * kPageBytes) + kBlockElems * 2;
@@ -301,37 +383,33 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
       // the last two P.V have no later Q.K^T whose S_FULL would vouch for their completion
       if (jj + 2 >= n_tiles) umma_commit(&bar[B_O_DONE + 2 * h + (jj & 1)]);
     };
-    if (n_tiles > 0) wait_page(0);
-    if (!failed && n_tiles > 0) {
+    wait_page(0);
+    if (!failed) {
       issue_qk(0, 0);
       if (two) issue_qk(1, 0);
     }
     for (int j = 0; j < n_tiles && !failed; ++j) {
       const bool more = j + 1 < n_tiles;
-      TC5H_STAMP(traced && lane == 0, 15, j);
       if (more) {
         wait_page(j + 1);
         wait_s_free(0, j);
         if (failed) break;
         issue_qk(0, j + 1);
       }
-      TC5H_STAMP(traced && lane == 0, 14, j);
       if (!mbar_wait_bounded(&bar[B_V_READY + j % kStages], (j / kStages) & 1)) failed = true;
       if (failed) break;
       issue_pv(0, j);
       if (failed) break;
-      TC5H_STAMP(traced && lane == 0, 13, j);
       if (more && two) {
         wait_s_free(1, j);
         if (failed) break;
         issue_qk(1, j + 1);
       }
-      TC5H_STAMP(traced && lane == 0, 12, j);
       if (two) issue_pv(1, j);
       if (failed) break;
       umma_commit(&bar[B_KV_EMPTY + (j % kStages)]);  // page j has no reader left
     }
-  } else if (warp < 4) {
+  } else if (is_conv(warp)) {
     // ---------------------------------------------------------------- value converter (warps 2-3)
     // bf16 -> fp16 in place, in the swizzled layout the copy left (element positions do not move);
     // a wide unit's values stay as they are
@@ -340,8 +418,8 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
       const int s = j % kStages;
       if (!mbar_wait_bounded(&bar[B_KV_FULL + s], (j / kStages) & 1)) { failed = true; break; }
       uint4 *vb = reinterpret_cast<uint4 *>(smem + kSKV + s * kPageBytes + kBlockElems * 2) + ct;
-#pragma unroll 8
-      for (int x = 0; x < (wide ? 0 : 16); ++x) {
+#pragma unroll
+      for (int x = 0; x < (wide ? 0 : 1024 / kConvThreads); ++x) {
         uint4 r = vb[x * kConvThreads];
         r.x = bf16x2_to_f16x2(r.x, v_scale); r.y = bf16x2_to_f16x2(r.y, v_scale);
         r.z = bf16x2_to_f16x2(r.z, v_scale); r.w = bf16x2_to_f16x2(r.w, v_scale);
@@ -350,20 +428,27 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
       fence_async_smem();
       mbar_arrive(&bar[B_V_READY + s]);
     }
-  } else {
+  } else if (warp >= 4 && warp < 12) {
     // ---------------------------------------------------------------- softmax groups
     const int h = (warp >> 2) - 1, row = tid & 127, i = (h ? i0_s1 : i0_s0) + row, hq = h ? hq_s1 : hq_s0;
     const bool row_ok = i < a.C;
     const int nv = row_ok ? nvis(i) : 0;
     const int jq = n_old + i;  // staging index of this row's own pair
     const uint32_t t_lane = tbase + ((uint32_t)((warp & 3) * 32) << 16);
-    const uint32_t t_s = t_lane + h * 64, t_o = t_lane + 256 + h * 128;
+    const uint32_t t_o = t_lane + 256 + h * 128;
     float m_ref = -INFINITY, l = 0.f;
     const int n_mine = (h == 0 || two) ? n_tiles : 0;   // the idle group of a one-head block has no pages
+    // the scores of page jj are complete (waiting does not consume the phase)
+    auto s_full_wait = [&](int jj) {
+      return kDeep ? mbar_wait_bounded(&bar[B_S_FULL + 2 * h + (jj & 1)], (jj >> 1) & 1)
+                   : mbar_wait_bounded(&bar[B_S_FULL + h], jj & 1);
+    };
     for (int j = 0; j < n_mine; ++j) {
-      if (!mbar_wait_bounded(&bar[B_S_FULL + h], j & 1)) { failed = true; break; }
+      if (!s_full_wait(j)) { failed = true; break; }
       TC5H_STAMP(traced && row == 0, h * 4 + 0, j);
       fence_after();
+      // deep: the page's score buffer, and P goes back into it; flat: the head's one score buffer
+      const uint32_t t_s = t_lane + (kDeep ? (2 * h + (j & 1)) * 64 : h * 64);
       float v[64];
 #pragma unroll
       for (int q4 = 0; q4 < 4; ++q4) {
@@ -373,9 +458,10 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
         for (int x = 0; x < 16; ++x) v[q4 * 16 + x] = t16[x];
       }
       tmem_ld_wait();
-      // the scores are in registers: Q.K^T of the next page may overwrite the buffer
-      fence_before();
-      mbar_arrive(&bar[B_S_FREE + h]);
+      if (!kDeep) {   // the scores are in registers: Q.K^T of the next page may overwrite the buffer
+        fence_before();
+        mbar_arrive(&bar[B_S_FREE + h]);
+      }
       TC5H_STAMP(traced && row == 0, h * 4 + 1, j);
       // visibility: compact-cache page j -> first nv pairs; staging page -> the band of this row.
       // v keeps the raw scores (masked ones become -inf); the scale is folded into the exponent,
@@ -442,11 +528,9 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
       const float m_new = grow ? mx : m_ref;
       if (j > 0 && __any_sync(0xffffffffu, grow)) {
         // O is stable between the completion of PV(j-1) and the hand-over of P(j).  QK(j+1) is
-        // issued after PV(j-1) and needs nothing more from this group (the S buffer is free), so
-        // S_FULL(j+1) vouches for it (waiting on it here does not consume the phase); the last
-        // page has its own barrier.
-        if (!(j + 1 < n_tiles ? mbar_wait_bounded(&bar[B_S_FULL + h], (j + 1) & 1)
-                              : mbar_wait_bounded(&bar[B_O_DONE + 2 * h + ((j - 1) & 1)], 0))) {
+        // issued after PV(j-1) and needs nothing more from this group, so S_FULL(j+1) vouches for
+        // it (waiting on it here does not consume the phase); the last page has its own barrier.
+        if (!(j + 1 < n_tiles ? s_full_wait(j + 1) : mbar_wait_bounded(&bar[B_O_DONE + 2 * h + ((j - 1) & 1)], 0))) {
           failed = true;
           break;
         }
@@ -471,16 +555,17 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
       const uint64_t sc2 = pack2(a.scale_log2, a.scale_log2), nms2 = pack2(bias - ms, bias - ms);
       uint64_t l2a = pack2(0.f, 0.f), l2b = l2a;
       if (wide) {
-        // one P buffer per head: P.V of the previous page must have read it.  Q.K^T(j+1) is issued
-        // after P.V(j-1) and needs nothing more from this group, so S_FULL(j+1) vouches for it
-        // (waiting on it here does not consume the phase); the last page has its own barrier.
-        if (j > 0 && !(j + 1 < n_tiles ? mbar_wait_bounded(&bar[B_S_FULL + h], (j + 1) & 1)
-                                       : mbar_wait_bounded(&bar[B_O_DONE + 2 * h + ((j - 1) & 1)], 0))) {
+        // deep: hi in the first 32 columns of the page's score buffer, lo in the other 32.
+        // flat: one P buffer per head (hi, then lo): P.V of the previous page must have read it;
+        // Q.K^T(j+1) is issued after P.V(j-1), so S_FULL(j+1) vouches for it; the last page has its
+        // own barrier.
+        if (!kDeep && j > 0 &&
+            !(j + 1 < n_tiles ? s_full_wait(j + 1) : mbar_wait_bounded(&bar[B_O_DONE + 2 * h + ((j - 1) & 1)], 0))) {
           failed = true;
           break;
         }
-        fence_after();
-        const uint32_t t_p = t_lane + 128 + h * 64;
+        if (!kDeep) fence_after();
+        const uint32_t t_p = kDeep ? t_s : t_lane + 128 + h * 64;
 #pragma unroll
         for (int q2 = 0; q2 < 2; ++q2) {  // 32 keys -> 16 columns of hi, 16 of lo
           uint32_t hi[16], lo[16];
@@ -501,8 +586,9 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
           tmem_st16u(t_p + 32 + q2 * 16, lo);
         }
       } else {
-        // P buffer (j & 1) is free: S_FULL(j) completed after P.V(j-2)
-        const uint32_t t_p = t_lane + 128 + (2 * h + (j & 1)) * 32;
+        // deep: the first 32 columns of the page's score buffer; flat: P buffer j & 1 of the head
+        // (free: S_FULL(j) completed after P.V(j-2))
+        const uint32_t t_p = kDeep ? t_s : t_lane + 128 + (2 * h + (j & 1)) * 32;
 #pragma unroll
         for (int q2 = 0; q2 < 2; ++q2) {  // 32 keys -> 16 columns of fp16 pairs
           uint32_t ph[16];
@@ -586,7 +672,7 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
   if (failed) set_status(c, SPKV_E_TIMEOUT);
   fence_before();
   __syncthreads();
-  if (warp == 1)
+  if (warp == kLoaderWarp)
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tbase), "n"(tc5x2h::kTmemCols) : "memory");
 }
 
