@@ -22,7 +22,10 @@ struct PrefillArgs {
   __nv_bfloat16 *stage_pages;      // [Hkv][n_stage_pages] pages: old ring pairs + chunk pairs in
   int n_stage_pages;               //   position order, page format (tensor-core kernel only)
   int pair_tiles;                  // fp16 two-slot kernel: a single head's blocks take two query tiles each
-  int n_split;                     // fp16 two-slot kernel: blocks per page walk (split over the pages), >= 1
+  int n_split;                     // fp16 two-slot kernel: blocks per page walk (the most shares a walk is cut into), >= 1
+  int walks_per_kvh;               //   page walks per KV head, and
+  float split_unit;                //   SMs of the device (a walk's fair share of the launch = all pages / this);
+                                   //   0: fewer walks than SMs, every walk is cut into runs of 16 pages
   float *partials;                 // [walk][slot][split]: 128 rows x (128 O + pad) and (m, l); n_split > 1 only
   int force_wide;                  // SPKV_FLAG_PREFILL_PV_BF16: every unit takes the two-term bf16 P.V
   // Soft-gated whole-sequence forward (spkv_softgate_forward; Eq. 6): no cache behind the call,

@@ -152,6 +152,52 @@ __device__ inline bool value_scale(uint32_t vm, int force_wide, float &v_scale, 
   return false;
 }
 
+// Pages of a walk: the compact-cache pages its last query sees (*n_ptiles), then the band pages
+// sp_lo ... of the staging area; the soft-gated forward walks every page from the start.
+template <bool kSoft>
+__device__ inline int walk_pages(const PrefillArgs &a, const WalkSlots &w, int *n_ptiles, int *sp_lo) {
+  const int32_t *hdr = unit_ws(a, w.kvh);
+  const int32_t *E = hdr + kHdrInts;
+  const int len0 = hdr[H_LEN0], n_old = hdr[H_NOLD], N = hdr[H_N];
+  // the last query of the block (slot 1 never starts before slot 0) sees the most kept pairs
+  const int i_first = w.i00, i_last = min((w.two ? w.i01 : w.i00) + 127, a.C - 1);
+  const int nv = kSoft ? 0 : len0 + E[min(max(i_last + n_old - a.c.w + 1, 0), N)];
+  *n_ptiles = (nv + kP - 1) / kP;
+  *sp_lo = kSoft ? 0 : max(0, i_first + n_old - a.c.w + 1) / kP;
+  return *n_ptiles + ((i_last + n_old) / kP - *sp_lo + 1);
+}
+// Shares a walk of n_pages pages is cut into, one block each, when the launch has a.n_split
+// blocks per walk.  A launch with fewer walks than SMs cuts every walk into runs of 16 pages.
+// A launch of one to two and a half waves of walks cuts a walk only when it is long against the
+// launch's fair share per SM (all pages of all walks / SMs, estimated from the plan headers: a KV
+// head's walks see its kept pairs from before the call plus, on average, half of those the chunk
+// adds, and ~3 band pages): a share costs a block's start-up, its partial result (128 KB) and the
+// merge, which only pays where a walk would otherwise outlast the rest of the launch -- a KV
+// head that keeps far more than the others.  Walks that stay whole write their output directly.
+// (Measured, TFLOP/s useful, 32 k past: 32 query / 8 KV heads with keep rates 0 - 0.9, chunk 1536:
+// 660 against 630 with every walk cut in four and 414 uncut; 8 / 2 heads, rates 0.15 / 0.6, chunk
+// 8192: 941 against 861 and 973.)
+constexpr float kSplitThr = 1.25f, kSplitFrac = 0.6f;
+template <bool kSoft>
+__device__ inline int walk_shares(const PrefillArgs &a, int n_pages) {
+  if (a.n_split <= 1) return 1;   // (uniform over the block)
+  // fewer walks than SMs: as many shares as there are runs of kMinSharePages pages
+  if (a.split_unit == 0.f) return max(1, min(a.n_split, n_pages / tc5x2h::kMinSharePages));
+  // (called by whole warps: one lane per KV head, so that the headers are fetched side by side)
+  float total = 0.f;
+  for (int k = threadIdx.x & 31; k < a.c.Hkv; k += 32) {
+    const int32_t *hd = unit_ws(a, k);
+    const float kept = kSoft ? 0.5f * a.C : hd[H_LEN0] + 0.5f * (hd + kHdrInts)[hd[H_N]];
+    total += kept * (1.f / kP) + 3.f;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+  const float fair = total * a.walks_per_kvh / a.split_unit;
+  if (n_pages <= kSplitThr * fair || n_pages < 2 * tc5x2h::kMinSharePages) return 1;
+  const float share = fmaxf((float)tc5x2h::kMinSharePages, kSplitFrac * fair);
+  return max(1, min(a.n_split, (int)ceilf(n_pages / share)));
+}
+
 // kEvenG: every block is a head pair on one tile (the branches for single heads compile away).
 // kSoft: the soft-gated whole-sequence forward (Eq. 6): no compact-cache pages, the walk covers
 // every causal page of the sequence, and a key beyond a query's window is not masked but biased
@@ -183,32 +229,17 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
   const bool wide = value_scale((uint32_t)hdr[H_VMAX], a.force_wide, v_scale, v_unscale);
   // kept pairs visible to chunk query i: the first nvis(i) pairs of the compact cache
   auto nvis = [&](int i) { return kSoft ? 0 : len0 + E[min(max(i + n_old - c.w + 1, 0), N)]; };
-  // the last query of the block (slot 1 never starts before slot 0) sees the most kept pairs
   if (kEvenG) two = true;
-  const int i_first = i0_s0, i_last = min((two ? i0_s1 : i0_s0) + 127, a.C - 1);
-  const int n_ptiles = (nvis(i_last) + kP - 1) / kP;
-  // band of both slots together, in staging indices (query i is staging pair n_old + i); the
-  // soft-gated forward walks every page from the start of the sequence
-  const int sp_lo = kSoft ? 0 : max(0, i_first + n_old - c.w + 1) / kP, sp_hi = (i_last + n_old) / kP;
-  const int n_tiles_all = n_ptiles + (sp_hi - sp_lo + 1);
+  // band of both slots together, in staging indices (query i is staging pair n_old + i)
+  int n_ptiles, sp_lo;
+  const int n_tiles_all = walk_pages<kSoft>(a, ws, &n_ptiles, &sp_lo);
   // this block's share of the walk: pages [j_begin, j_begin + n_tiles) of the list (compact-cache
-  // pages, then band pages); page numbers below are local, j_begin + j is the page's place in the list
-  // (a walk takes as many of its a.n_split blocks as it has runs of kMinSharePages pages; the
-  // others find an empty share and leave at once)
-  const int n_shares = min(a.n_split, (n_tiles_all + kMinSharePages - 1) / kMinSharePages);
-  const int j_begin = split < n_shares ? (int)((long long)n_tiles_all * split / n_shares) : n_tiles_all;
-  const int n_tiles = split < n_shares ? (int)((long long)n_tiles_all * (split + 1) / n_shares) - j_begin : 0;
-  if (n_tiles == 0) {  // empty share (split walks only): says so in its partial result and leaves
-    if (warp >= 4 && warp < 12) {
-      const int h = (warp >> 2) - 1;
-      if (h == 0 || two) {
-        float *part = a.partials + ((size_t)(walk * 2 + h) * a.n_split + split) * kPartFloats;
-        part[128 * 128 + (tid & 127) * 2] = -INFINITY;
-        part[128 * 128 + (tid & 127) * 2 + 1] = 0.f;
-      }
-    }
-    return;
-  }
+  // pages, then band pages); page numbers below are local, j_begin + j is the page's place in the
+  // list.  The blocks of a walk beyond its number of shares leave at once.
+  const int n_shares = walk_shares<kSoft>(a, n_tiles_all);
+  if (split >= n_shares) return;
+  const int j_begin = (int)((long long)n_tiles_all * split / n_shares);
+  const int n_tiles = (int)((long long)n_tiles_all * (split + 1) / n_shares) - j_begin;
 
   if (tid == 0) {
     for (int i = 0; i < kStages; ++i) {
@@ -617,14 +648,11 @@ __global__ void __launch_bounds__(tc5x2h::kThreads, 1) prefill_attn_tc5x2h_kerne
     }
     if (h == 1 && !two) {
       // idle slot: nothing to write
-    } else if (a.n_split > 1) {
+    } else if (n_shares > 1) {
       // a share of a split walk: the unnormalised row (fp32, in the scaled units) and its (m, l)
       // go to the partial results; prefill_merge_kernel puts the shares together
       float *part = a.partials + ((size_t)(walk * 2 + h) * a.n_split + split) * kPartFloats;
-      if (n_tiles == 0) {
-        part[128 * 128 + row * 2] = -INFINITY;
-        part[128 * 128 + row * 2 + 1] = 0.f;
-      } else if (!failed && mbar_wait_bounded(&bar[B_O_DONE + 2 * h + ((n_tiles - 1) & 1)], 0)) {
+      if (!failed && mbar_wait_bounded(&bar[B_O_DONE + 2 * h + ((n_tiles - 1) & 1)], 0)) {
         fence_after();
 #pragma unroll
         for (int q8 = 0; q8 < 8; ++q8) {
@@ -684,61 +712,68 @@ extern "C" int spkv_debug_tc5h_trace(long long *host_out) {
 
 // Puts the shares of a split page walk together: out = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s
 // (M = max_s m_s; the m are log2-domain reference maxima, the O and l carry the same bias and value
-// scale in every share).  grid (walks, 2 slots), 256 threads: thread = (row, 16-dim group) x 4.
-template <bool kEvenG>
+// scale in every share).  grid (walks, 2 slots, 4 row quarters), 256 threads: 32 rows per block,
+// thread = (row, 16-dim group).
+template <bool kEvenG, bool kSoft>
 __global__ void __launch_bounds__(256) prefill_merge_kernel(PrefillArgs a) {
   using namespace tc5x2h;
   pdl_chain_link();
   const CacheView &c = a.c;
-  const int walk = blockIdx.x, h = blockIdx.y, S = a.n_split;
+  const int walk = blockIdx.x, h = blockIdx.y, row0 = blockIdx.z * 32;
   const WalkSlots ws = walk_slots<kEvenG>(a, walk);
   if (h == 1 && !ws.two) return;
+  int n_ptiles, sp_lo;
+  const int S = walk_shares<kSoft>(a, walk_pages<kSoft>(a, ws, &n_ptiles, &sp_lo));
+  if (S == 1) return;   // the walk stayed whole and wrote its output itself
   const int hq = h ? ws.hq1 : ws.hq0, i0 = h ? ws.i01 : ws.i00;
+  if (i0 + row0 >= a.C) return;
   float v_scale, v_unscale;
   const bool wide = value_scale((uint32_t)unit_ws(a, ws.kvh)[H_VMAX], a.force_wide, v_scale, v_unscale);
-  const float *part = a.partials + (size_t)(walk * 2 + h) * S * kPartFloats;
-  __shared__ float s_w[kMaxSplit][128];   // weight of share s for a row, already divided by the row sum
-  for (int row = threadIdx.x; row < 128; row += blockDim.x) {
-    float M = -INFINITY;
-    for (int s = 0; s < S; ++s) M = fmaxf(M, part[(size_t)s * kPartFloats + 128 * 128 + row * 2]);
-    float L = 0.f;
-    for (int s = 0; s < S; ++s) {
-      const float m = part[(size_t)s * kPartFloats + 128 * 128 + row * 2];
-      const float wgt = m == -INFINITY ? 0.f : exp2f(m - M);
-      s_w[s][row] = wgt;
-      L += wgt * part[(size_t)s * kPartFloats + 128 * 128 + row * 2 + 1];
+  const float *part = a.partials + (size_t)(walk * 2 + h) * a.n_split * kPartFloats;
+  __shared__ float s_w[kMaxSplit][32];   // weight of share s for a row, already divided by the row sum
+  if (threadIdx.x < 32) {
+    const int row = row0 + threadIdx.x;
+    float ms[kMaxSplit], M = -INFINITY;
+#pragma unroll
+    for (int s = 0; s < kMaxSplit; ++s) {
+      ms[s] = s < S ? part[(size_t)s * kPartFloats + 128 * 128 + row * 2] : -INFINITY;
+      M = fmaxf(M, ms[s]);
+    }
+    float L = 0.f, wg[kMaxSplit];
+#pragma unroll
+    for (int s = 0; s < kMaxSplit; ++s) {
+      wg[s] = ms[s] == -INFINITY ? 0.f : exp2f(ms[s] - M);
+      if (s < S) L += wg[s] * part[(size_t)s * kPartFloats + 128 * 128 + row * 2 + 1];
     }
     const float inv = L > 0.f ? 1.f / L : 0.f;
-    for (int s = 0; s < S; ++s) s_w[s][row] *= inv;
+#pragma unroll
+    for (int s = 0; s < kMaxSplit; ++s) s_w[s][threadIdx.x] = wg[s] * inv;
     if (a.lse && i0 + row < a.C)   // the shares' l carry the same bias of P as the unsplit kernel's
       a.lse[(size_t)(i0 + row) * c.Hq + hq] = (M - (wide ? 0.f : kPBias) + log2f(L)) * 0.6931471805599453f;
   }
   __syncthreads();
-  for (int x = threadIdx.x; x < 128 * 8; x += blockDim.x) {
-    const int row = x >> 3, g = x & 7, i = i0 + row;
-    if (i >= a.C) continue;
-    float acc[16];
+  const int r = threadIdx.x >> 3, g = threadIdx.x & 7, row = row0 + r, i = i0 + row;
+  if (i >= a.C) return;
+  float acc[16];
 #pragma unroll
-    for (int d = 0; d < 16; ++d) acc[d] = 0.f;
-    for (int s = 0; s < S; ++s) {
-      const float wgt = s_w[s][row];
-      if (wgt == 0.f) continue;   // an empty share has written no O
-      const float4 *src = reinterpret_cast<const float4 *>(part + (size_t)s * kPartFloats + row * 128 + g * 16);
+  for (int d = 0; d < 16; ++d) acc[d] = 0.f;
+  for (int s = 0; s < S; ++s) {
+    const float wgt = s_w[s][r];
+    const float4 *src = reinterpret_cast<const float4 *>(part + (size_t)s * kPartFloats + row * 128 + g * 16);
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const float4 v = src[q];
-        acc[4 * q] += wgt * v.x; acc[4 * q + 1] += wgt * v.y; acc[4 * q + 2] += wgt * v.z; acc[4 * q + 3] += wgt * v.w;
-      }
+    for (int q = 0; q < 4; ++q) {
+      const float4 v = src[q];
+      acc[4 * q] += wgt * v.x; acc[4 * q + 1] += wgt * v.y; acc[4 * q + 2] += wgt * v.z; acc[4 * q + 3] += wgt * v.w;
     }
-    uint4 w0, w1;
-    w0.x = pack_bf16(acc[0] * v_unscale, acc[1] * v_unscale);   w0.y = pack_bf16(acc[2] * v_unscale, acc[3] * v_unscale);
-    w0.z = pack_bf16(acc[4] * v_unscale, acc[5] * v_unscale);   w0.w = pack_bf16(acc[6] * v_unscale, acc[7] * v_unscale);
-    w1.x = pack_bf16(acc[8] * v_unscale, acc[9] * v_unscale);   w1.y = pack_bf16(acc[10] * v_unscale, acc[11] * v_unscale);
-    w1.z = pack_bf16(acc[12] * v_unscale, acc[13] * v_unscale); w1.w = pack_bf16(acc[14] * v_unscale, acc[15] * v_unscale);
-    __nv_bfloat16 *orow = a.out + ((size_t)i * c.Hq + hq) * kD + g * 16;
-    *reinterpret_cast<uint4 *>(orow) = w0;
-    *reinterpret_cast<uint4 *>(orow + 8) = w1;
   }
+  uint4 w0, w1;
+  w0.x = pack_bf16(acc[0] * v_unscale, acc[1] * v_unscale);   w0.y = pack_bf16(acc[2] * v_unscale, acc[3] * v_unscale);
+  w0.z = pack_bf16(acc[4] * v_unscale, acc[5] * v_unscale);   w0.w = pack_bf16(acc[6] * v_unscale, acc[7] * v_unscale);
+  w1.x = pack_bf16(acc[8] * v_unscale, acc[9] * v_unscale);   w1.y = pack_bf16(acc[10] * v_unscale, acc[11] * v_unscale);
+  w1.z = pack_bf16(acc[12] * v_unscale, acc[13] * v_unscale); w1.w = pack_bf16(acc[14] * v_unscale, acc[15] * v_unscale);
+  __nv_bfloat16 *orow = a.out + ((size_t)i * c.Hq + hq) * kD + g * 16;
+  *reinterpret_cast<uint4 *>(orow) = w0;
+  *reinterpret_cast<uint4 *>(orow + 8) = w1;
 }
 
 // Number of blocks that share a page walk.  A chunk of a few hundred tokens has only a handful of
@@ -785,12 +820,15 @@ int launch_prefill_attn_tc5x2h(const PrefillArgs &a_in, cudaStream_t s) {
   const int n_walks = per_kvh * a.c.Hkv;
   a.n_split = a.partials ? prefill_split_count(n_walks, std::min(sms, 192)) : 1;
   a.n_split = (int)std::max(1LL, std::min<long long>(a.n_split, split_slots(a.C, a.c.G, a.c.Hkv) / n_walks));
+  a.walks_per_kvh = per_kvh;
+  a.split_unit = n_walks < sms ? 0.f : (float)sms;
   if (launch_link(a.chained != 0, kernel, dim3(n_walks * a.n_split), dim3(tc5x2h::kThreads), (size_t)tc5x2h::kSmemBytes, s,
                   a) != cudaSuccess)
     return SPKV_E_CUDA;
   if (a.n_split > 1) {
-    auto merge = (a.c.G & 1) ? prefill_merge_kernel<false> : prefill_merge_kernel<true>;
-    if (launch_link(a.chained != 0, merge, dim3(n_walks, 2), dim3(256), 0, s, a) != cudaSuccess) return SPKV_E_CUDA;
+    auto merge = a.soft ? ((a.c.G & 1) ? prefill_merge_kernel<false, true> : prefill_merge_kernel<true, true>)
+                        : ((a.c.G & 1) ? prefill_merge_kernel<false, false> : prefill_merge_kernel<true, false>);
+    if (launch_link(a.chained != 0, merge, dim3(n_walks, 2, 4), dim3(256), 0, s, a) != cudaSuccess) return SPKV_E_CUDA;
   }
   return check_stream_error(cudaGetLastError());
 }
