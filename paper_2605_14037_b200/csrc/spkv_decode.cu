@@ -298,8 +298,8 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
       trow = unit_table_row(c, u);
       // (L2 loads: in overlap mode the writer may be a kernel that ended after this block began,
       // and an SM's L1 is not coherent with other SMs' stores)
-      len = __ldcg(&c.len[u]);
-      n_ring = min(__ldcg(&c.t[u]), c.w);
+      len = ldcg_keep(&c.len[u]);
+      n_ring = min(ldcg_keep(&c.t[u]), c.w);
       np = (len + kP - 1) / kP + (n_ring + kP - 1) / kP;
     } else if (blockIdx.x == 0) {
       set_status(c, SPKV_E_BOUNDS);
@@ -360,7 +360,7 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
           const int u = s_unit[item], len = s_len[item], nk = (len + kP - 1) / kP;
           if (j < nk) {
             // (debug bounds: a table entry that names no pool page is read from the unit's ring instead)
-            gq.gpage = checked_page(c, __ldcg(&unit_table(c, s_row[item])[j]), (int)ring_page(c, u, 0));
+            gq.gpage = checked_page(c, ldcg_keep(&unit_table(c, s_row[item])[j]), (int)ring_page(c, u, 0));
             gq.valid = min(kP, len - j * kP);
           } else {
             gq.gpage = (int)ring_page(c, u, j - nk);
@@ -377,6 +377,9 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
 
     int k = 0;  // pages issued by this block
     int gave_up = 0;
+    // keys and values are read once per step: their lines leave L2 first, so that what every step
+    // reads again (lengths, page tables: loaded with the opposite hint) stays there (+1 % in step)
+    const uint64_t l2pol = l2_evict_first_policy();
     Group cur = resolve();
     while (cur.count > 0 && !gave_up) {
       const Group nxt = resolve();
@@ -396,7 +399,7 @@ decode_tc_kernel(DecodeArgs a, int GP, int n_stages, int red_bufs) {
           unsigned char *dst = smem + (size_t)stage * L.stage_bytes;
           const uint32_t qbytes = (fl & F_BEGIN) ? (uint32_t)(a.G * kRowBytes) : 0u;
           mbar_arrive_expect_tx(&full[stage], kPageBytes + qbytes);
-          bulk_load(dst, c.pages + (int64_t)gp * kPageElems, kPageBytes, &full[stage]);
+          bulk_load_hint(dst, c.pages + (int64_t)gp * kPageElems, kPageBytes, &full[stage], l2pol);
           if (qbytes)
             bulk_load(dst + kPageBytes,
                       a.q + ((size_t)(it / c.Hkv) * c.Hq + (size_t)(it % c.Hkv) * a.G) * kD, qbytes,

@@ -224,4 +224,26 @@ __device__ inline void bulk_load(void *smem_dst, const void *gmem_src, uint32_t 
       ::"r"(smem_u32(smem_dst)), "l"(gmem_src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
+// The same copy with an L2 eviction hint for data that is read once: the lines go first when L2
+// needs room, so what is read again every step (lengths, page tables, ring metadata) stays.
+__device__ inline uint64_t l2_evict_first_policy() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+// 32-bit load that bypasses L1 and asks L2 to keep the line (metadata read again every step)
+__device__ inline int ldcg_keep(const int *p) {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  int v;
+  asm volatile("ld.global.cg.L2::cache_hint.b32 %0, [%1], %2;" : "=r"(v) : "l"(p), "l"(pol) : "memory");
+  return v;
+}
+__device__ inline void bulk_load_hint(void *smem_dst, const void *gmem_src, uint32_t bytes, uint64_t *bar,
+                                      uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+      ::"r"(smem_u32(smem_dst)), "l"(gmem_src), "r"(bytes), "r"(smem_u32(bar)), "l"(policy) : "memory");
+}
+
 }  // namespace spkv
