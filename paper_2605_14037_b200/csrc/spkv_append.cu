@@ -58,8 +58,8 @@ __device__ inline void append_unit(const CacheView &c, int layer, const int32_t 
   // row, the head's own threshold, and the new pair itself.  Metadata is read from L2 (in overlap
   // mode this kernel does not start at a stream-wide synchronisation point, and an SM's L1 is not
   // coherent with other SMs' stores).
-  const int t = __ldcg(&c.t[u]);
-  const int n = __ldcg(&c.len[u]);
+  const int t = ldcg_keep(&c.t[u]);
+  const int n = ldcg_keep(&c.len[u]);
   const int trow = local_only ? -1 : unit_table_row(c, u);
   const float thr = head_threshold(c, layer, kvh, tau_logit);
   // lanes 0-15 move the key row, lanes 16-31 the value row, one 16-byte chunk each
@@ -88,7 +88,7 @@ __device__ inline void append_unit(const CacheView &c, int layer, const int32_t 
   int32_t *table = unit_table(c, trow >= 0 ? trow : 0);
   const float lg = __ldcg(&c.ring_logit[(size_t)u * c.w + slot]);
   const uint4 evictee = __ldcg(ring_cell);
-  const int page_at_tail = (leaves && prow != 0 && pj < c.max_pages) ? __ldcg(&table[pj]) : -1;
+  const int page_at_tail = (leaves && prow != 0 && pj < c.max_pages) ? ldcg_keep(&table[pj]) : -1;
 
   if (leaves && (lg >= thr || t - c.w < c.n_sink)) {
     // the pair of position t - w leaves the window and passes the threshold on its stored logit

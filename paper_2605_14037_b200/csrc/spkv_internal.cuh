@@ -122,7 +122,17 @@ __device__ inline float head_threshold(const CacheView &c, int layer, int kvh, f
 
 // page table of a unit (the caller knows the unit has one: row >= 0)
 __device__ inline int32_t *unit_table(const CacheView &c, int row) { return c.table + (size_t)row * c.max_pages; }
-__device__ inline int unit_table_row(const CacheView &c, int u) { return __ldcg(&c.table_row[u]); }
+// 32-bit load that bypasses L1 (an SM's L1 is not coherent with other SMs' stores) and asks L2 to
+// keep the line: for the metadata every step reads again (lengths, page tables), which the
+// streaming reads of keys and values -- issued with the opposite hint -- would otherwise push out.
+__device__ inline int ldcg_keep(const int *p) {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  int v;
+  asm volatile("ld.global.cg.L2::cache_hint.b32 %0, [%1], %2;" : "=r"(v) : "l"(p), "l"(pol) : "memory");
+  return v;
+}
+__device__ inline int unit_table_row(const CacheView &c, int u) { return ldcg_keep(&c.table_row[u]); }
 
 // global page index of ring page j of a unit
 __device__ inline int64_t ring_page(const CacheView &c, int unit, int j) {

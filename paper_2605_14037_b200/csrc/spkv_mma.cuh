@@ -231,14 +231,6 @@ __device__ inline uint64_t l2_evict_first_policy() {
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
   return pol;
 }
-// 32-bit load that bypasses L1 and asks L2 to keep the line (metadata read again every step)
-__device__ inline int ldcg_keep(const int *p) {
-  uint64_t pol;
-  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
-  int v;
-  asm volatile("ld.global.cg.L2::cache_hint.b32 %0, [%1], %2;" : "=r"(v) : "l"(p), "l"(pol) : "memory");
-  return v;
-}
 __device__ inline void bulk_load_hint(void *smem_dst, const void *gmem_src, uint32_t bytes, uint64_t *bar,
                                       uint64_t policy) {
   asm volatile(
