@@ -549,8 +549,8 @@ def run_ours(args):
                      "read_ceiling": {"gbs": sp.get("read_ceiling_gbs"),
                                       "frac": in_step / sp["read_ceiling_gbs"] if sp.get("read_ceiling_gbs") else None,
                                       "how": "spkv_stream_read over the cache arena: 32 KB bulk copies into shared "
-                                             "memory, one block per SM, nothing else (the measured peak above is a "
-                                             "copy: half writes)"},
+                                             "memory, one block per SM, pages handed out by an atomic counter, "
+                                             "nothing else (the measured peak above is a copy: half writes)"},
                      "bytes_per_launch": sp["launch_bytes"], "launch_period_us": sp["ms_per_step"] * 1e3 / L,
                      "how": "algorithmic K/V, Q, O bytes of a step over the step time measured with CUDA events "
                             "around the timed region (graph replay, launches overlapped, append included)",

@@ -406,7 +406,8 @@ int spkv_decode_step_host(spkv_cache_t *cache, int32_t layer, const spkv_predict
 int spkv_decode_step_host_flush(spkv_cache_t *cache, spkv_stream_t stream);
 
 /* One decode step of the WHOLE layer stack from host buffers, for an attention-only stack whose
- * inputs all exist before the step.  The layers go in four chunks: a chunk's inputs are copied
+ * inputs all exist before the step.  The layers go in three chunks (a short head, the bulk, a
+ * short tail; one chunk per layer below four layers): a chunk's inputs are copied
  * on a stream of the cache's own, its kernels (per layer score -> append/evict -> decode
  * attention, back to back) run on `stream` once they have landed, and its outputs are copied
  * back on another stream of the cache's own while the next chunk computes.  `stream` ends up
@@ -457,10 +458,14 @@ const char *spkv_error_string(int code);
 
 /* Measurement aid (no counterpart in the paper): streams `bytes` bytes (rounded down to whole
  * 32 KB pages) from device memory through shared memory with the bulk copies the decode kernel
- * uses, one block per SM, and does nothing else with them.  Timed by the caller with events it
- * gives the read-only HBM rate of this GPU, the ceiling of a kernel that only reads (the usual
- * copy figure is half writes).
- *   d_buf: device, 16-byte aligned; d_sink: device, one 64-bit word (a checksum is added to it);
+ * uses, one block per SM, and does nothing else with them.  The pages are handed out one by one
+ * through an atomic counter, so that SMs that draw faster take more of them (an even split ends
+ * with its slowest SM: about 3 % less on a B200).  Timed by the caller with events it gives the
+ * read-only HBM rate of this GPU, the ceiling of a kernel that only reads (the usual copy figure
+ * is half writes).
+ *   d_buf: device, 16-byte aligned; d_sink: device, TWO 64-bit words: [0] a checksum is added to
+ *   it, [1] the page counter, zero before the first call and left at zero by every call (calls
+ *   that share it must not overlap on the GPU);
  *   d_status: device, one int32, set to SPKV_E_TIMEOUT if a bounded wait ran out.  Asynchronous. */
 int spkv_stream_read(const void *d_buf, size_t bytes, unsigned long long *d_sink, int32_t *d_status,
                      spkv_stream_t stream);

@@ -399,7 +399,7 @@ extern "C" int spkv_safe_steps(spkv_cache_t *cache, const int32_t *h_seq_ids, in
 extern "C" int spkv_cache_destroy(spkv_cache_t *cache) {
   if (!cache) return SPKV_E_INVALID;
   if (cache->stack_ready) {
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < kStackChunks; ++i) {
       cudaEventDestroy(cache->ev_st_in[i]);
       cudaEventDestroy(cache->ev_st_k[i]);
     }

@@ -1012,14 +1012,18 @@ extern "C" int spkv_decode_step_host_flush(spkv_cache_t *cache, spkv_stream_t st
 
 // ---- one decode step of the WHOLE layer stack from host buffers ------------------------------
 // For an attention-only stack every layer's inputs exist before the step starts.  The layers go
-// in four chunks: each chunk's inputs travel in four copies on the cache's input stream, its
-// 2 x layers kernels follow back to back on the caller's stream once they have landed (nothing
-// between the kernels of a chunk: in overlap mode each decode launch starts under the tail of the
-// previous one, which the per-layer entry point's event waits prevent), and its outputs leave on
-// the output stream while the next chunk computes.  So the copies of all chunks but the first
-// (in) and the last (out) run under kernels.  The caller's stream ends up waiting for the last
-// output copy: synchronising it means the outputs are on the host.
-constexpr int kStackChunks = 4;
+// in three chunks -- a short head (a sixteenth of the stack), the bulk, a short tail: each chunk's
+// inputs travel in four copies on the cache's input stream, its 2 x layers kernels follow back to
+// back on the caller's stream once they have landed (nothing between the kernels of a chunk: in
+// overlap mode each decode launch starts under the tail of the previous one, which the per-layer
+// entry point's event waits prevent), and its outputs leave on the output stream while the next
+// chunk computes.  Only the head's inputs and the tail's outputs travel with nothing running
+// beside them, so those two are small; the bulk's inputs land under the head's kernels and its
+// outputs leave under the tail's.  Every chunk boundary costs an event wait on the caller's
+// stream, across which consecutive launches do not overlap, so there are no more chunks than
+// that (32 layers, batch 16: 2 + 28 + 2 layers 7440 tokens/s; four chunks of 8 7150; 2 + 14 +
+// 14 + 2 7340; 1 + 30 + 1 7290; one chunk 6920).  The caller's stream ends up waiting for the
+// last output copy: synchronising it means the outputs are on the host.
 
 static int stack_pipeline_init(spkv_cache *c) {
   int rc = host_pipeline_init(c);
@@ -1076,7 +1080,20 @@ extern "C" int spkv_decode_stack_host(spkv_cache_t *cache, const spkv_predictor_
   cudaStream_t s = as_stream(stream);
   int rc = stack_pipeline_init(cache);
   if (rc) return rc;
-  const int nc = L < kStackChunks ? L : kStackChunks;
+  // chunks of layers: a short head, the bulk, a short tail (fewer chunks for a short stack)
+  int bounds[kStackChunks + 1];
+  int nc;
+  {
+    const int h = L / 16 > 1 ? L / 16 : 1;
+    bounds[0] = 0;
+    if (L >= 4 * h) {
+      nc = 3;
+      bounds[1] = h; bounds[2] = L - h; bounds[3] = L;
+    } else {
+      nc = L < kStackChunks ? L : kStackChunks;
+      for (int ci = 1; ci <= nc; ++ci) bounds[ci] = (int)((size_t)ci * L / nc);
+    }
+  }
   const char *hx = static_cast<const char *>(h_x), *hq = static_cast<const char *>(h_q),
              *hk = static_cast<const char *>(h_k), *hv = static_cast<const char *>(h_v);
   // the staging buffers are free once everything enqueued on the caller's stream so far has run
@@ -1084,7 +1101,7 @@ extern "C" int spkv_decode_stack_host(spkv_cache_t *cache, const spkv_predictor_
       cudaStreamWaitEvent(cache->copy_in, cache->ev_st_start, 0) != cudaSuccess)
     return SPKV_E_CUDA;
   for (int ci = 0; ci < nc; ++ci) {
-    const size_t l0 = (size_t)ci * L / nc, n = (size_t)(ci + 1) * L / nc - l0;
+    const size_t l0 = (size_t)bounds[ci], n = (size_t)bounds[ci + 1] - l0;
     if (cudaMemcpyAsync(d_x + l0 * x_l, hx + l0 * x_l, n * x_l, cudaMemcpyHostToDevice, cache->copy_in) != cudaSuccess ||
         cudaMemcpyAsync(d_q + l0 * q_l, hq + l0 * q_l, n * q_l, cudaMemcpyHostToDevice, cache->copy_in) != cudaSuccess ||
         cudaMemcpyAsync(d_k + l0 * kv_l, hk + l0 * kv_l, n * kv_l, cudaMemcpyHostToDevice, cache->copy_in) != cudaSuccess ||
@@ -1093,7 +1110,7 @@ extern "C" int spkv_decode_stack_host(spkv_cache_t *cache, const spkv_predictor_
       return SPKV_E_CUDA;
   }
   for (int ci = 0; ci < nc; ++ci) {
-    const int l0 = (int)((size_t)ci * L / nc), l1 = (int)((size_t)(ci + 1) * L / nc);
+    const int l0 = bounds[ci], l1 = bounds[ci + 1];
     if (cudaStreamWaitEvent(s, cache->ev_st_in[ci], 0) != cudaSuccess) return SPKV_E_CUDA;
     cache->last_kind = kLastOther;  // the chunk's first append waits for everything before it on the stream
     for (int l = l0; l < l1; ++l) {

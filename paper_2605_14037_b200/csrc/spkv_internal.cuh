@@ -39,6 +39,7 @@ constexpr int kBlockElems = kP * kD;        // bf16 elements in a key (or value)
 constexpr int kPageElems = 2 * kBlockElems; // 16384 elements = 32 KB
 constexpr int kPageBytes = kPageElems * 2;
 constexpr int kMaxGroup = 16;      // query heads per KV head supported by the kernels
+constexpr int kStackChunks = 4;    // most chunks spkv_decode_stack_host cuts the layer stack into
 
 struct CacheView {
   int32_t L, S, Hq, Hkv, G, w, ring_pages, max_pages, n_units;
@@ -285,7 +286,7 @@ struct spkv_cache {
   long long host_calls;                        // calls so far; slot = call & 1
   bool host_ready;
   // spkv_decode_stack_host: per chunk of layers, inputs landed / kernels done; start and end of a call
-  cudaEvent_t ev_st_in[4], ev_st_k[4], ev_st_start, ev_st_done;
+  cudaEvent_t ev_st_in[spkv::kStackChunks], ev_st_k[spkv::kStackChunks], ev_st_start, ev_st_done;
   bool stack_ready;
 };
 

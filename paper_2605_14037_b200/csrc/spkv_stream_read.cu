@@ -1,7 +1,7 @@
 // Measurement aid (no counterpart in the paper): how fast can this GPU READ from HBM with the
 // copy mechanism the decode kernel uses?  The decode path only reads its K/V pages, while the
 // usual bandwidth figure is a copy (half reads, half writes); this kernel streams a buffer
-// through shared memory in 32 KB bulk copies, six in flight per block, one block per SM, and does
+// through shared memory in 32 KB bulk copies, five in flight per block, one block per SM, and does
 // nothing else with it (one word per page goes into a checksum so that the copies are not dead).
 #include "spkv_internal.cuh"
 #include "spkv_mma.cuh"
@@ -9,11 +9,18 @@
 namespace spkv {
 
 namespace {
-constexpr int kReadStages = 6;
+constexpr int kReadStages = 5;
 constexpr int kReadSmem = kReadStages * kPageBytes + 64;
 }  // namespace
 
-// grid = SMs, 32 threads; block b takes pages b, b + grid, ...  status[0] != 0 on a timed-out wait.
+// grid = SMs, 32 threads.  Pages are handed out one at a time by an atomic counter (sink[1]) rather
+// than split evenly: SMs do not draw from HBM at the same rate -- under full load, with the same
+// bytes in flight, the fastest takes about a fifth more pages than the mean and the slowest a
+// fifth less, the same SMs in every run -- and an even split ends when the slowest SM does
+// (measured on one B200: 7.30 TB/s with an even split, 7.54 TB/s with the counter).  Every block
+// claims until the counter has run past n_pages, i.e. fails exactly once; the claim that brings
+// it to n_pages + gridDim.x is the launch's last and its owner leaves the counter at zero.
+// status[0] != 0 on a timed-out wait.
 __global__ void __launch_bounds__(32) stream_read_kernel(const unsigned char *buf, long long n_pages,
                                                          unsigned long long *sink, int *status) {
   extern __shared__ __align__(1024) unsigned char smem[];
@@ -27,7 +34,12 @@ __global__ void __launch_bounds__(32) stream_read_kernel(const unsigned char *bu
   unsigned long long sum = 0;
   long long k = 0;
   bool failed = false;
-  for (long long p = blockIdx.x; p < n_pages && !failed; p += gridDim.x, ++k) {
+  for (;; ++k) {
+    const long long p = (long long)atomicAdd(&sink[1], 1ULL);
+    if (p >= n_pages) {
+      if (p == n_pages + (long long)gridDim.x - 1) sink[1] = 0;
+      break;
+    }
     const int s = (int)(k % kReadStages);
     if (k >= kReadStages) {  // the copy that used this stage before has landed
       if (!mbar_wait_bounded(&full[s], (uint32_t)((k / kReadStages) - 1) & 1)) { failed = true; break; }

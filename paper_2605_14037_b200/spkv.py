@@ -453,7 +453,7 @@ class Cache:
 def spkv_stream_read(buf, passes=5, stream=None):
     """Read-only HBM rate in GB/s: streams the uint8 tensor `buf` through spkv_stream_read
     `passes` times (after one warm-up pass), timed with CUDA events on the launching stream."""
-    sink = torch.zeros(1, dtype=torch.int64, device=buf.device)
+    sink = torch.zeros(2, dtype=torch.int64, device=buf.device)   # checksum, page counter
     status = torch.zeros(1, dtype=torch.int32, device=buf.device)
     nbytes = buf.numel() // 32768 * 32768
     call = lambda: _check(lib().spkv_stream_read(_ptr(buf), nbytes, _ptr(sink), _ptr(status), _stream(stream)),

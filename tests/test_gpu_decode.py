@@ -270,11 +270,12 @@ def test_overlap_mode_is_bit_identical_to_stream_ordered_launches(L, B, steps):
 
 
 @pytest.mark.parametrize("flags", [0, 1])
-@pytest.mark.parametrize("L", [1, 3, 5, 9])
+@pytest.mark.parametrize("L", [1, 3, 4, 5, 9, 33])
 def test_decode_stack_host_matches_device_calls(flags, L):
-    """spkv_decode_stack_host (the layers in up to four chunks, each with its copies in, its
-    kernels back to back and its copy out) against the device-pointer calls, bit for bit, with
-    and without overlap mode, for layer counts below, at and above the number of chunks."""
+    """spkv_decode_stack_host (the layers in chunks -- head, bulk, tail -- each with its copies in,
+    its kernels back to back and its copy out) against the device-pointer calls, bit for bit,
+    with and without overlap mode, for stacks too short for three chunks, just long enough, and
+    long enough for a head and tail of two layers."""
     spkv = load()
     rng = np.random.default_rng(123 + flags)
     B, Hq, Hkv, d_in, w, steps = 3, 8, 2, 64, 16, 30

@@ -1,5 +1,6 @@
 """The read-stream measurement aid: it must touch every 32 KB page of the buffer exactly once
-(its checksum adds the first 32-bit word of each page) and report no timed-out wait."""
+(its checksum adds the first 32-bit word of each page), leave its page counter at zero for the
+next call, and report no timed-out wait."""
 import ctypes as C
 
 import numpy as np
@@ -18,7 +19,7 @@ def test_stream_read_visits_every_page_once(n_pages, tail):
     first = np.random.default_rng(n_pages).integers(0, 2 ** 32, size=n_pages, dtype=np.uint64).astype(np.uint32)
     words[np.arange(n_pages) * 8192] = first
     buf = torch.from_numpy(words.view(np.uint8)[:n_pages * 32768 + tail].copy()).to(dev())
-    sink = torch.zeros(1, dtype=torch.int64, device=dev())
+    sink = torch.zeros(2, dtype=torch.int64, device=dev())      # checksum, page counter
     status = torch.zeros(1, dtype=torch.int32, device=dev())
     for rep in range(3):
         rc = spkv.lib().spkv_stream_read(C.c_void_p(buf.data_ptr()), buf.numel(), C.c_void_p(sink.data_ptr()),
@@ -26,13 +27,14 @@ def test_stream_read_visits_every_page_once(n_pages, tail):
         assert rc == 0
     torch.cuda.synchronize()
     assert int(status.item()) == 0
-    assert int(sink.item()) == 3 * int(first.astype(np.uint64).sum())
+    assert int(sink[0].item()) == 3 * int(first.astype(np.uint64).sum())
+    assert int(sink[1].item()) == 0          # the last claim of every launch clears the counter
 
 
 def test_stream_read_rejects_bad_arguments_and_ignores_less_than_a_page():
     spkv = load()
     buf = torch.zeros(40000, dtype=torch.uint8, device=dev())
-    sink = torch.zeros(1, dtype=torch.int64, device=dev())
+    sink = torch.zeros(2, dtype=torch.int64, device=dev())
     status = torch.zeros(1, dtype=torch.int32, device=dev())
     s = C.c_void_p(torch.cuda.current_stream().cuda_stream)
     f = spkv.lib().spkv_stream_read
