@@ -322,6 +322,10 @@ def run_ours(args):
             xs, qs, ks, vs = x_all[step], q_in[step % n_in], k_in[step % n_in], v_in[step % n_in]
             # the first launch of a step waits for everything before it on the stream even in overlap
             # mode (the previous step's reads of the cache, a rollback copy)
+            if not args.per_layer and events is None:
+                # the whole stack in two launches: appends of every layer, one persistent decode kernel
+                cache.spkv_decode_stack(preds, ids, xs, qs, ks, vs, out=out, logits_out=logits, stream=stream)
+                return
             cache.spkv_note_foreign_work()
             for l in range(L):
                 cache.spkv_score_append_evict(l, preds[l], ids, xs[l], ks[l], vs[l],
@@ -893,6 +897,9 @@ def main():
     ap.add_argument("--steps-per-graph", type=int, default=1,
                     help="steps captured in one CUDA graph (default 1; more shows the device time of a "
                          "tiny step where the host's replay rate is the limit)")
+    ap.add_argument("--per-layer", action="store_true",
+                    help="time the step as 2 L per-layer calls (spkv_score_append_evict, spkv_decode_attention) "
+                         "instead of one spkv_decode_stack call (comparison run, not the bench line)")
     ap.add_argument("--stream-ordered", action="store_true",
                     help="create the cache without SPKV_FLAG_OVERLAP: every launch waits for the previous one, as "
                          "in a model whose layers depend on each other (comparison run, not the bench line)")

@@ -405,6 +405,27 @@ int spkv_decode_step_host(spkv_cache_t *cache, int32_t layer, const spkv_predict
                           void *d_staging, size_t staging_bytes, spkv_stream_t stream);
 int spkv_decode_step_host_flush(spkv_cache_t *cache, spkv_stream_t stream);
 
+/* One decode step of the WHOLE layer stack from device buffers, for an attention-only stack whose
+ * inputs all exist before the step (Eq. 1-5 per layer; Appendix "Inference Kernels": fused token
+ * append, sparse decode): the same results as, layer by layer, spkv_score_append_evict followed
+ * by spkv_decode_attention, bit for bit, in two launches -- the appends of every layer, then one
+ * persistent decode-attention kernel whose blocks take page ranges of all layers from one list,
+ * so that their page streams never stop between layers.  Ordinary stream-ordered launches (no
+ * SPKV_FLAG_OVERLAP contract); no synchronisation.
+ *   preds [n_layers]: HOST array of predictors with the same d_in (linear predictors and up to 128
+ *   layers take the two launches; otherwise the call falls back to the per-layer calls);
+ *   d_x [L, B, d_in], d_q [L, B, n_q_heads, 128], d_k/d_v [L, B, n_kv_heads, 128] bf16, 16-byte
+ *   aligned -> d_out [L, B, n_q_heads, 128] bf16; d_logits_out [L, B, n_kv_heads] float32 or NULL
+ *   (required by two-layer predictors); d_lse_opt [L, B, n_q_heads] float32 or NULL;
+ *   d_workspace: >= spkv_decode_stack_workspace_bytes(cfg, B) bytes, 256-byte aligned, used by this
+ *   cache only, zero-filled once before its first use and then left alone.  After a sticky
+ *   SPKV_E_TIMEOUT it must be zero-filled again. */
+size_t spkv_decode_stack_workspace_bytes(const spkv_config_t *cfg, int32_t B);
+int spkv_decode_stack(spkv_cache_t *cache, const spkv_predictor_t *preds, const int32_t *d_seq_ids,
+                      int32_t B, const void *d_x, const void *d_q, const void *d_k, const void *d_v,
+                      void *d_out, float *d_logits_out, float *d_lse_opt, float sm_scale,
+                      void *d_workspace, size_t workspace_bytes, spkv_stream_t stream);
+
 /* One decode step of the WHOLE layer stack from host buffers, for an attention-only stack whose
  * inputs all exist before the step.  The layers go in three chunks (a short head, the bulk, a
  * short tail; one chunk per layer below four layers): a chunk's inputs are copied

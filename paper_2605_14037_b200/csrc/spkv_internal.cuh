@@ -294,6 +294,16 @@ namespace spkv {
 int check_stream_error(cudaError_t e);
 inline cudaStream_t as_stream(spkv_stream_t s) { return reinterpret_cast<cudaStream_t>(s); }
 float tau_to_logit(float tau);
+// per-layer linear predictors and local-only masks of a stack step, passed to kernels by value
+constexpr int kMaxStackLayers = 128;
+struct StackPreds {
+  const __nv_bfloat16 *W[kMaxStackLayers];
+  const float *bias[kMaxStackLayers];
+  unsigned long long local_mask[kMaxStackLayers];
+};
+int launch_append_stack(spkv_cache *cache, const StackPreds &sp, int n_layers, const int32_t *d_seq_ids, int B,
+                        const void *d_k, const void *d_v, const void *d_x, int d_in, float *d_logits_out,
+                        cudaStream_t s);
 int launch_score_mlp_tc(spkv_cache *cache, const spkv_predictor_t *p, const void *d_x, int n_tok, float *d_logits,
                         uint8_t *d_flags, cudaStream_t s);
 }  // namespace spkv

@@ -109,6 +109,8 @@ def lib():
         "spkv_decode_step_host_flush": (C.c_int, [vp, vp]),
         "spkv_decode_stack_staging_bytes": (sz, [cfgp, i32, i32]),
         "spkv_decode_stack_host": (C.c_int, [vp, vp, vp, i32, vp, vp, vp, vp, vp, f32, vp, sz, vp]),
+        "spkv_decode_stack_workspace_bytes": (sz, [cfgp, i32]),
+        "spkv_decode_stack": (C.c_int, [vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, f32, vp, sz, vp]),
         "spkv_status": (C.c_int, [vp, vp]),
         "spkv_clear_status": (C.c_int, [vp, vp]),
         "spkv_cache_stats": (C.c_int, [vp, vp, C.POINTER(Stats)]),
@@ -361,6 +363,24 @@ class Cache:
             C.c_void_p(h_v.data_ptr()), C.c_void_p(h_out.data_ptr()),
             self.default_scale if sm_scale is None else sm_scale, _ptr(st), st.numel(),
             _stream(stream)), "spkv_decode_step_host")
+
+    def spkv_decode_stack(self, preds, seq_ids, x, q, k, v, out=None, logits_out=None, lse=None, sm_scale=None,
+                          stream=None):
+        """One decode step of all layers from device tensors [L, B, ...]: the appends of every layer in
+        one launch, decode attention of every layer in one persistent launch."""
+        B, L = seq_ids.numel(), self.cfg.n_layers
+        assert len(preds) == L and q.shape[0] == L
+        arr = (Predictor * L)(*preds)
+        if out is None:
+            out = torch.empty_like(q)
+        ws = self._workspace("decode_stack", lib().spkv_decode_stack_workspace_bytes(C.byref(self.cfg), B))
+        _check(lib().spkv_decode_stack(
+            self._h, C.cast(arr, C.c_void_p), _ptr(seq_ids, torch.int32), B, _ptr(x, torch.bfloat16),
+            _ptr(q, torch.bfloat16), _ptr(k, torch.bfloat16), _ptr(v, torch.bfloat16), _ptr(out, torch.bfloat16),
+            _ptr(logits_out, torch.float32), _ptr(lse, torch.float32),
+            self.default_scale if sm_scale is None else sm_scale, _ptr(ws), ws.numel(), _stream(stream)),
+            "spkv_decode_stack")
+        return out
 
     def spkv_decode_stack_host(self, preds, seq_ids, h_x, h_q, h_k, h_v, h_out, sm_scale=None, stream=None):
         """One decode step of all layers from host (pinned) tensors [L, B, ...]; enqueues four
