@@ -408,7 +408,7 @@ int spkv_decode_step_host_flush(spkv_cache_t *cache, spkv_stream_t stream);
 /* One decode step of the WHOLE layer stack from device buffers, for an attention-only stack whose
  * inputs all exist before the step (Eq. 1-5 per layer; Appendix "Inference Kernels": fused token
  * append, sparse decode): the same results as, layer by layer, spkv_score_append_evict followed
- * by spkv_decode_attention, bit for bit, in two launches -- the appends of every layer, then one
+ * by spkv_decode_attention on the same cache, bit for bit, in two launches -- the appends of every layer, then one
  * persistent decode-attention kernel whose blocks take page ranges of all layers from one list,
  * so that their page streams never stop between layers.  Ordinary stream-ordered launches (no
  * SPKV_FLAG_OVERLAP contract); no synchronisation.
@@ -429,8 +429,8 @@ int spkv_decode_stack(spkv_cache_t *cache, const spkv_predictor_t *preds, const 
 /* One decode step of the WHOLE layer stack from host buffers, for an attention-only stack whose
  * inputs all exist before the step.  The layers go in three chunks (a short head, the bulk, a
  * short tail; one chunk per layer below four layers): a chunk's inputs are copied
- * on a stream of the cache's own, its kernels (per layer score -> append/evict -> decode
- * attention, back to back) run on `stream` once they have landed, and its outputs are copied
+ * on a stream of the cache's own, its kernels (spkv_decode_stack's two launches over the chunk's
+ * layers) run on `stream` once they have landed, and its outputs are copied
  * back on another stream of the cache's own while the next chunk computes.  `stream` ends up
  * waiting for the last output copy, so synchronising `stream` means h_out is complete; the host
  * buffers must stay untouched until then (pinned memory, or the copies serialise).  No

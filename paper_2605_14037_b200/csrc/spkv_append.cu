@@ -154,27 +154,27 @@ append_evict_kernel(CacheView c, int layer, const int32_t *__restrict__ seq_ids,
 }
 
 // The appends of every layer of a stack step in one launch (spkv_decode_stack): warp g owns unit
-// g % items of layer g / items.  Inputs and logits are laid out layer after layer.  A plain
+// g % items of layer layer0 + g / items.  Inputs and logits are laid out layer after layer, layer0's first.  A plain
 // stream-ordered launch: no overlap bookkeeping.
 __global__ void __launch_bounds__(128)
-append_stack_kernel(CacheView c, StackPreds sp, int n_layers, const int32_t *__restrict__ seq_ids, int B,
+append_stack_kernel(CacheView c, StackPreds sp, int layer0, int n_layers, const int32_t *__restrict__ seq_ids, int B,
                     const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new,
                     const __nv_bfloat16 *__restrict__ x, int d_in, float *__restrict__ logits_out, float tau_logit) {
   const int items = B * c.Hkv;
   const long long g = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int layer = (int)(g / items), item = (int)(g % items);
   if (layer >= n_layers) return;
-  append_unit(c, layer, item, seq_ids, B, k_new + (size_t)layer * items * 16, v_new + (size_t)layer * items * 16,
+  append_unit(c, layer0 + layer, item, seq_ids, B, k_new + (size_t)layer * items * 16, v_new + (size_t)layer * items * 16,
               nullptr, tau_logit, x + (size_t)layer * B * d_in, sp.W[layer], sp.bias[layer], d_in,
               logits_out ? logits_out + (size_t)layer * items : nullptr, sp.local_mask[layer]);
 }
 
-int launch_append_stack(spkv_cache *cache, const StackPreds &sp, int n_layers, const int32_t *d_seq_ids, int B,
+int launch_append_stack(spkv_cache *cache, const StackPreds &sp, int layer0, int n_layers, const int32_t *d_seq_ids, int B,
                         const void *d_k, const void *d_v, const void *d_x, int d_in, float *d_logits_out,
                         cudaStream_t s) {
   const long long warps = (long long)n_layers * B * cache->view.Hkv;
   const int grid = (int)((warps + 3) / 4);
-  append_stack_kernel<<<grid, 128, 0, s>>>(cache->view, sp, n_layers, d_seq_ids, B, static_cast<const uint4 *>(d_k),
+  append_stack_kernel<<<grid, 128, 0, s>>>(cache->view, sp, layer0, n_layers, d_seq_ids, B, static_cast<const uint4 *>(d_k),
                                            static_cast<const uint4 *>(d_v), static_cast<const __nv_bfloat16 *>(d_x), d_in,
                                            d_logits_out, cache->tau_logit);
   return check_stream_error(cudaGetLastError());

@@ -677,18 +677,15 @@ extern "C" int spkv_decode_step_host_flush(spkv_cache_t *cache, spkv_stream_t st
 // ---- one decode step of the WHOLE layer stack from host buffers ------------------------------
 // For an attention-only stack every layer's inputs exist before the step starts.  The layers go
 // in three chunks -- a short head (a sixteenth of the stack), the bulk, a short tail: each chunk's
-// inputs travel in four copies on the cache's input stream, its 2 x layers kernels follow back to
-// back on the caller's stream once they have landed (nothing between the kernels of a chunk: in
-// overlap mode each decode launch starts under the tail of the previous one, which the per-layer
-// entry point's event waits prevent), and its outputs leave on the output stream while the next
-// chunk computes.  Only the head's inputs and the tail's outputs travel with nothing running
+// inputs travel in four copies on the cache's input stream, its two launches (the appends of its
+// layers, one persistent decode kernel over its layers: spkv_decode_stack's) follow on the
+// caller's stream once they have landed, and its outputs leave on the output stream while the
+// next chunk computes.  Only the head's inputs and the tail's outputs travel with nothing running
 // beside them, so those two are small; the bulk's inputs land under the head's kernels and its
-// outputs leave under the tail's.  Every chunk boundary costs an event wait on the caller's
-// stream, across which consecutive launches do not overlap, so there are no more chunks than
-// that (32 layers, batch 16: 2 + 28 + 2 layers 7440 tokens/s; four chunks of 8 7150; 2 + 14 +
-// 14 + 2 7340; 1 + 30 + 1 7290; one chunk 6920).  The caller's stream ends up waiting for the
-// last output copy: synchronising it means the outputs are on the host.
-
+// outputs leave under the tail's.  (Measured with per-layer launches, 32 layers, batch 16:
+// 2 + 28 + 2 layers 7440 tokens/s; four chunks of 8 7150; 2 + 14 + 14 + 2 7340; 1 + 30 + 1 7290;
+// one chunk 6920.)  The caller's stream ends up waiting for the last output copy: synchronising it
+// means the outputs are on the host.
 static int stack_pipeline_init(spkv_cache *c) {
   int rc = host_pipeline_init(c);
   if (rc) return rc;
@@ -716,7 +713,7 @@ static size_t stack_inputs_bytes(const spkv_config_t *cfg, int32_t B, int32_t d_
 extern "C" size_t spkv_decode_stack_staging_bytes(const spkv_config_t *cfg, int32_t B, int32_t d_in) {
   if (!cfg || B < 0 || d_in < 0) return 0;
   size_t x, q, kv, lg;
-  return stack_inputs_bytes(cfg, B, d_in, &x, &q, &kv, &lg) + spkv_decode_workspace_bytes(cfg, B);
+  return stack_inputs_bytes(cfg, B, d_in, &x, &q, &kv, &lg) + spkv_decode_stack_workspace_bytes(cfg, B);
 }
 
 extern "C" int spkv_decode_stack_host(spkv_cache_t *cache, const spkv_predictor_t *preds, const int32_t *d_seq_ids,
@@ -776,15 +773,10 @@ extern "C" int spkv_decode_stack_host(spkv_cache_t *cache, const spkv_predictor_
   for (int ci = 0; ci < nc; ++ci) {
     const int l0 = bounds[ci], l1 = bounds[ci + 1];
     if (cudaStreamWaitEvent(s, cache->ev_st_in[ci], 0) != cudaSuccess) return SPKV_E_CUDA;
-    cache->last_kind = kLastOther;  // the chunk's first append waits for everything before it on the stream
-    for (int l = l0; l < l1; ++l) {
-      rc = spkv_score_append_evict(cache, l, &preds[l], d_seq_ids, B, d_x + l * x_l, d_k + l * kv_l, d_v + l * kv_l,
-                                   d_lg + (size_t)l * B * cfg.n_kv_heads, stream);
-      if (rc) return rc;
-      rc = spkv_decode_attention(cache, l, d_seq_ids, B, d_q + l * q_l, d_o + l * q_l, nullptr, sm_scale, p,
-                                 spkv_decode_workspace_bytes(&cfg, B), stream);
-      if (rc) return rc;
-    }
+    // the chunk's layers: their appends in one launch, their decode attention in one persistent launch
+    rc = decode_stack_layers(cache, l0, l1, preds, d_seq_ids, B, d_x, d_q, d_k, d_v, d_o, d_lg, nullptr, sm_scale, p,
+                             spkv_decode_stack_workspace_bytes(&cfg, B), stream);
+    if (rc) return rc;
     if (cudaEventRecord(cache->ev_st_k[ci], s) != cudaSuccess ||
         cudaStreamWaitEvent(cache->copy_out, cache->ev_st_k[ci], 0) != cudaSuccess ||
         cudaMemcpyAsync(static_cast<char *>(h_out) + l0 * q_l, d_o + l0 * q_l, (size_t)(l1 - l0) * q_l,

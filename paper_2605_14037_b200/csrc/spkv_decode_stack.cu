@@ -41,15 +41,15 @@ enum { F_LAYER = 8 };  // stage flag: no page, "the producer has left this layer
 
 struct StackArgs {
   CacheView c;
-  int n_layers, B, n_items, G;
+  int layer0, n_layers, B, n_items, G;   // layers layer0 ... layer0 + n_layers - 1 of the cache
   const int32_t *seq_ids;
-  const __nv_bfloat16 *q;  // [L][B][Hq][128]
+  const __nv_bfloat16 *q;  // [L][B][Hq][128], first row: layer0's
   __nv_bfloat16 *out;      // [L][B][Hq][128]
   float *lse;              // [L][B][Hq] or null
   float scale_log2;
   int snap, min_pos;
   int32_t *claim;          // the launch's range counter
-  char *ws;                // per-layer regions: arrival counters, partial results
+  char *ws;                // per-layer regions (from layer0's on): arrival counters, partial results
   size_t ws_layer_bytes, off_gcnt, off_ml, off_acc;
 };
 
@@ -154,7 +154,7 @@ decode_stack_kernel(StackArgs a, int GP, int n_stages) {
         const int seq = s_seq[b];
         int np = 0, u = 0, len = 0, n_ring = 0, trow = -1;
         if (seq >= 0 && seq < c.S) {
-          u = unit_index(c, l, seq, kvh);
+          u = unit_index(c, a.layer0 + l, seq, kvh);
           trow = unit_table_row(c, u);
           len = ldcg_keep(&c.len[u]);
           n_ring = min(ldcg_keep(&c.t[u]), c.w);
@@ -205,7 +205,9 @@ decode_stack_kernel(StackArgs a, int GP, int n_stages) {
     }
   } else if (warp == kConsumerWarps) {
     // ------------------------------------------------------------------ producer warp
-    struct Group { int gpage, valid, flags, item, count, chunk, layer; };
+    // kind 0: nothing follows; 1: `count` positions of a range; 2: no pages, only the news that the
+    // producer has moved on from layer `mark`
+    struct Group { int gpage, valid, flags, item, count, chunk, layer, kind, mark; };
     int k = 0;          // stages used so far (pages and markers)
     int gave_up = 0;
     int layer = -1;     // layer whose plan is in use (-1: none yet)
@@ -231,48 +233,60 @@ decode_stack_kernel(StackArgs a, int GP, int n_stages) {
       }
       ++k;
     };
-    // moves on to layer `to` (every layer in between is visited: its marker, then the next plan)
-    auto enter_layer = [&](int to) {
-      while (layer < to && !gave_up) {
-        if (layer >= 0) marker(F_LAYER, layer);
-        if (gave_up) break;
-        ++layer;
-        int ok = 1;
-        if (lane == 0) ok = wait_or_flag(&plan_ready[layer & 1], (layer >> 1) & 1, c);
-        if (!__shfl_sync(0xffffffffu, ok, 0)) gave_up = 1;
-        P = plan_of(layer);
-      }
-    };
-    // Claims ranges until one is not empty (warp-uniform).  Every block claims until the counter has
-    // run past the list, i.e. fails exactly once: the claim that brings the counter to
-    // n_ranges + gridDim.x is the launch's last, and its owner leaves the counter at zero.
-    auto next_range = [&]() {
-      for (;;) {
-        const int g = __shfl_sync(0xffffffffu, pending, 0);
-        if (g >= n_ranges) {
-          if (g == n_ranges + NB - 1 && lane == 0) *a.claim = 0;
-          return false;
+    // The range held for this block (claimed, not yet walked), or the end of the list.  Every block
+    // claims until the counter has run past the list, i.e. fails exactly once: the claim that brings
+    // the counter to n_ranges + gridDim.x is the launch's last, and its owner leaves it at zero.
+    // A block whose list is exhausted still visits the remaining layers (markers only): the planner
+    // walks them all, each only after this block has left the layer two before it.
+    bool have_g = false, finishing = false;
+    int tgt_layer = 0, g_cidx = 0;
+    // Resolves the next (up to) 32 positions of the range (markers come out with valid = 0), taking a
+    // new range when the current one is done.  Entering the next layer is a step of its own -- one
+    // layer per call, a group of kind 2 -- because the marker of the layer left must go down the
+    // pipeline behind that layer's last pages and before this warp waits for a later plan.
+    auto resolve = [&]() {
+      Group gq = {0, 0, 0, 0, 0, 0, 0, 0, -1};
+      if (!more) return gq;
+      while (cur_base >= r_pe) {
+        if (!have_g && !finishing) {
+          const int g = __shfl_sync(0xffffffffu, pending, 0);
+          if (g >= n_ranges) {
+            if (g == n_ranges + NB - 1 && lane == 0) *a.claim = 0;
+            finishing = true;
+            tgt_layer = a.n_layers - 1;
+          } else {
+            if (lane == 0) pending = atomicAdd(a.claim, 1);
+            have_g = true;
+            tgt_layer = g / NB;
+            g_cidx = g % NB;
+          }
         }
-        if (lane == 0) pending = atomicAdd(a.claim, 1);
-        enter_layer(g / NB);
-        if (gave_up) return false;
-        cidx = g % NB;
-        const int VP = P[PL.hdr], nb_eff = P[PL.hdr + 1];
-        if (VP == 0 || cidx >= nb_eff) continue;
+        if (layer < tgt_layer) {
+          gq.kind = 2;
+          gq.mark = layer;  // (-1 before the first layer: nothing to tell)
+          ++layer;
+          int ok = 1;
+          if (lane == 0) ok = wait_or_flag(&plan_ready[layer & 1], (layer >> 1) & 1, c);
+          if (!__shfl_sync(0xffffffffu, ok, 0)) {
+            gave_up = 1;
+            more = false;
+            gq.kind = 0;
+          }
+          P = plan_of(layer);
+          return gq;
+        }
+        if (finishing) {
+          more = false;
+          return gq;
+        }
+        have_g = false;
+        cidx = g_cidx;
+        if (P[PL.hdr] == 0 || cidx >= P[PL.hdr + 1]) continue;  // the layer has fewer ranges than the numbering
         r_ps = P[PL.cut + cidx];
         r_pe = P[PL.cut + cidx + 1];
         cur_base = r_ps;
-        if (r_pe > r_ps) return true;
       }
-    };
-    // resolves the next (up to) 32 positions of the range; markers come out with valid = 0
-    auto resolve = [&]() {
-      Group gq = {0, 0, 0, 0, 0, 0, 0};
-      if (!more) return gq;
-      if (cur_base >= r_pe && !next_range()) {
-        more = false;
-        return gq;
-      }
+      gq.kind = 1;
       gq.chunk = cidx;
       gq.layer = layer;
       gq.count = min(32, r_pe - cur_base);
@@ -305,7 +319,9 @@ decode_stack_kernel(StackArgs a, int GP, int n_stages) {
 
     const uint64_t l2pol = l2_evict_first_policy();  // keys and values are read once per step
     Group cur = resolve();
-    while (cur.count > 0 && !gave_up) {
+    while (cur.kind != 0 && !gave_up) {
+      if (cur.mark >= 0) marker(F_LAYER, cur.mark);  // before the next resolve, which may wait for a plan that needs it
+      if (gave_up) break;
       const Group nxt = resolve();  // resolved before this group is issued: its table loads overlap the copies
       for (int i = 0; i < cur.count; ++i) {
         const int gp = __shfl_sync(0xffffffffu, cur.gpage, i), va = __shfl_sync(0xffffffffu, cur.valid, i);
@@ -335,9 +351,6 @@ decode_stack_kernel(StackArgs a, int GP, int n_stages) {
       }
       cur = nxt;
     }
-    // The list is exhausted.  The planner still walks the remaining layers, each of which it may
-    // only plan once this block has left the layer two before it: visit them all (markers only).
-    if (!gave_up) enter_layer(a.n_layers - 1);
     if (!gave_up) marker(F_STOP, 0);  // tell the consumers that nothing follows
     if (lane == 0 && gave_up) {
       // do not leave while copies may still be landing in shared memory
@@ -492,17 +505,21 @@ extern "C" size_t spkv_decode_stack_workspace_bytes(const spkv_config_t *cfg, in
   return 256 + (size_t)cfg->n_layers * per_layer + spkv_decode_workspace_bytes(cfg, B);
 }
 
-extern "C" int spkv_decode_stack(spkv_cache_t *cache, const spkv_predictor_t *preds, const int32_t *d_seq_ids, int32_t B,
-                                 const void *d_x, const void *d_q, const void *d_k, const void *d_v, void *d_out,
-                                 float *d_logits_out, float *d_lse_opt, float sm_scale, void *d_workspace,
-                                 size_t workspace_bytes, spkv_stream_t stream) {
-  if (!cache || !preds || B < 0 || B > cache->cfg.max_seqs) return SPKV_E_INVALID;
+// Layers l0 ... l1 - 1 of a stack step.  The input and output pointers name layer 0's rows (the
+// whole stack's arrays), whatever the range.
+int spkv::decode_stack_layers(spkv_cache *cache, int l0, int l1, const spkv_predictor_t *preds, const int32_t *d_seq_ids,
+                              int32_t B, const void *d_x, const void *d_q, const void *d_k, const void *d_v, void *d_out,
+                              float *d_logits_out, float *d_lse_opt, float sm_scale, void *d_workspace,
+                              size_t workspace_bytes, spkv_stream_t stream) {
+  if (!cache || !preds || B < 0 || B > cache->cfg.max_seqs || l0 < 0 || l1 > cache->cfg.n_layers || l0 > l1)
+    return SPKV_E_INVALID;
+  if (l0 == l1) return SPKV_OK;
   if (B == 0) return SPKV_OK;
   if (!d_seq_ids || !d_x || !d_q || !d_k || !d_v || !d_out) return SPKV_E_INVALID;
   if (((uintptr_t)d_x | (uintptr_t)d_q | (uintptr_t)d_k | (uintptr_t)d_v | (uintptr_t)d_out) & 15) return SPKV_E_INVALID;
   const spkv_config_t &cfg = cache->cfg;
   const CacheView &v = cache->view;
-  const int L = cfg.n_layers, n_items = B * v.Hkv, d_in = preds[0].d_in;
+  const int L = cfg.n_layers, n_items = B * v.Hkv, d_in = preds[0].d_in, nl = l1 - l0;
   if (n_items > 1024) return SPKV_E_UNSUPPORTED;
   for (int l = 0; l < L; ++l)
     if (preds[l].d_in != d_in) return SPKV_E_INVALID;
@@ -514,13 +531,13 @@ extern "C" int spkv_decode_stack(spkv_cache_t *cache, const spkv_predictor_t *pr
   const size_t x_l = (size_t)B * d_in * 2, q_l = (size_t)B * cfg.n_q_heads * kD * 2, kv_l = (size_t)n_items * kD * 2;
   cudaStream_t s = as_stream(stream);
 
-  bool fused = L <= kMaxStackLayers && d_in >= 8 && (d_in & 7) == 0 && (x_l & 15) == 0;
-  for (int l = 0; l < L && fused; ++l)
+  bool fused = nl <= kMaxStackLayers && d_in >= 8 && (d_in & 7) == 0 && (x_l & 15) == 0;
+  for (int l = l0; l < l1 && fused; ++l)
     fused = preds[l].kind == 0 && preds[l].d_W1 && preds[l].d_b1 && ((uintptr_t)preds[l].d_W1 & 15) == 0;
   if (!fused) {
     // two-layer predictors (scored by a kernel of their own) and very deep stacks: layer by layer
     void *ws1 = ws + 256 + (size_t)L * per_layer;
-    for (int l = 0; l < L; ++l) {
+    for (int l = l0; l < l1; ++l) {
       float *lg = d_logits_out ? d_logits_out + (size_t)l * n_items : nullptr;
       int rc = spkv_score_append_evict(cache, l, &preds[l], d_seq_ids, B, static_cast<const char *>(d_x) + l * x_l,
                                        static_cast<const char *>(d_k) + l * kv_l,
@@ -539,25 +556,29 @@ extern "C" int spkv_decode_stack(spkv_cache_t *cache, const spkv_predictor_t *pr
   // wait for it, and the next per-layer call must wait for them
   cache->last_kind = kLastOther;
   StackPreds sp;
-  for (int l = 0; l < L; ++l) {
-    sp.W[l] = static_cast<const __nv_bfloat16 *>(preds[l].d_W1);
-    sp.bias[l] = preds[l].d_b1;
-    sp.local_mask[l] = cache->local_mask[l];
+  for (int l = l0; l < l1; ++l) {
+    sp.W[l - l0] = static_cast<const __nv_bfloat16 *>(preds[l].d_W1);
+    sp.bias[l - l0] = preds[l].d_b1;
+    sp.local_mask[l - l0] = cache->local_mask[l];
   }
-  int rc = launch_append_stack(cache, sp, L, d_seq_ids, B, d_k, d_v, d_x, d_in, d_logits_out, s);
+  int rc = launch_append_stack(cache, sp, l0, nl, d_seq_ids, B, static_cast<const char *>(d_k) + l0 * kv_l,
+                               static_cast<const char *>(d_v) + l0 * kv_l, static_cast<const char *>(d_x) + l0 * x_l, d_in,
+                               d_logits_out ? d_logits_out + (size_t)l0 * n_items : nullptr, s);
   if (rc) return rc;
 
   StackArgs a;
-  a.c = v; a.n_layers = L; a.B = B; a.n_items = n_items; a.G = v.G;
+  a.c = v; a.layer0 = l0; a.n_layers = nl; a.B = B; a.n_items = n_items; a.G = v.G;
   a.seq_ids = d_seq_ids;
-  a.q = static_cast<const __nv_bfloat16 *>(d_q);
-  a.out = static_cast<__nv_bfloat16 *>(d_out);
-  a.lse = d_lse_opt;
+  a.q = reinterpret_cast<const __nv_bfloat16 *>(static_cast<const char *>(d_q) + l0 * q_l);
+  a.out = reinterpret_cast<__nv_bfloat16 *>(static_cast<char *>(d_out) + l0 * q_l);
+  a.lse = d_lse_opt ? d_lse_opt + (size_t)l0 * B * cfg.n_q_heads : nullptr;
   a.scale_log2 = sm_scale * kLog2e;
   a.snap = 6;
-  a.min_pos = 56;
+  // the per-layer kernel's rule, so that both paths cut a layer's pages the same way: a cache in
+  // overlap mode gives a range at least 56 positions when the layer has half a grid of such ranges
+  a.min_pos = (cfg.flags & SPKV_FLAG_OVERLAP) ? 56 : 4;
   a.claim = reinterpret_cast<int32_t *>(ws);
-  a.ws = ws + 256;
+  a.ws = ws + 256 + (size_t)l0 * per_layer;
   a.ws_layer_bytes = per_layer;
   a.off_gcnt = wl.off_gcnt; a.off_ml = wl.off_ml; a.off_acc = wl.off_acc;
   int GP = 1;
@@ -573,4 +594,13 @@ extern "C" int spkv_decode_stack(spkv_cache_t *cache, const spkv_predictor_t *pr
   const int grid = min(kMaxGrid, cache->sm_count);
   kernel<<<grid, kStackThreads, SL.total, s>>>(a, GP, n_stages);
   return check_stream_error(cudaGetLastError());
+}
+
+extern "C" int spkv_decode_stack(spkv_cache_t *cache, const spkv_predictor_t *preds, const int32_t *d_seq_ids, int32_t B,
+                                 const void *d_x, const void *d_q, const void *d_k, const void *d_v, void *d_out,
+                                 float *d_logits_out, float *d_lse_opt, float sm_scale, void *d_workspace,
+                                 size_t workspace_bytes, spkv_stream_t stream) {
+  if (!cache) return SPKV_E_INVALID;
+  return decode_stack_layers(cache, 0, cache->cfg.n_layers, preds, d_seq_ids, B, d_x, d_q, d_k, d_v, d_out, d_logits_out,
+                             d_lse_opt, sm_scale, d_workspace, workspace_bytes, stream);
 }

@@ -301,9 +301,13 @@ struct StackPreds {
   const float *bias[kMaxStackLayers];
   unsigned long long local_mask[kMaxStackLayers];
 };
-int launch_append_stack(spkv_cache *cache, const StackPreds &sp, int n_layers, const int32_t *d_seq_ids, int B,
+int launch_append_stack(spkv_cache *cache, const StackPreds &sp, int layer0, int n_layers, const int32_t *d_seq_ids, int B,
                         const void *d_k, const void *d_v, const void *d_x, int d_in, float *d_logits_out,
                         cudaStream_t s);
+int decode_stack_layers(spkv_cache *cache, int l0, int l1, const spkv_predictor_t *preds, const int32_t *d_seq_ids,
+                        int32_t B, const void *d_x, const void *d_q, const void *d_k, const void *d_v, void *d_out,
+                        float *d_logits_out, float *d_lse_opt, float sm_scale, void *d_workspace, size_t workspace_bytes,
+                        spkv_stream_t stream);
 int launch_score_mlp_tc(spkv_cache *cache, const spkv_predictor_t *p, const void *d_x, int n_tok, float *d_logits,
                         uint8_t *d_flags, cudaStream_t s);
 }  // namespace spkv

@@ -1,8 +1,8 @@
 """spkv_decode_stack: one decode step of the whole layer stack in two launches (the appends of
 every layer, then one persistent decode-attention kernel over all layers).  Checked against the
 oracle's streaming form unit by unit (state bit-exact, outputs at the attention tolerance), and
-against the per-layer calls it replaces (a cache in overlap mode cuts its page ranges the same
-way: same state, logits and outputs, bit for bit)."""
+against the per-layer calls it replaces on a second cache with the same flags (same state,
+logits and outputs, bit for bit)."""
 import math
 
 import numpy as np
@@ -22,7 +22,7 @@ def make_stack(spkv, rng, L, B, Hq, Hkv, T0, w, rates, d_in, tau=0.5, flags=0, m
     pool = pool_pages if pool_pages is not None else L * B * Hkv * ((T0 + 200) // 64 + 3)
     mk = lambda f: spkv.Cache(n_layers=L, max_seqs=B, n_q_heads=Hq, n_kv_heads=Hkv, max_context=max_context,
                               pool_pages=pool, window=w, tau=tau, flags=f)
-    ca, cb = mk(flags), mk(1)
+    ca, cb = mk(flags), mk(flags)
     tl = ca.spkv_tau_logit()
     preds, units = [], [[[oracle.Unit(w, D) for _ in range(Hkv)] for _ in range(B)] for _ in range(L)]
     for l in range(L):
@@ -47,6 +47,7 @@ def make_stack(spkv, rng, L, B, Hq, Hkv, T0, w, rates, d_in, tau=0.5, flags=0, m
     return ca, cb, preds, units, tl
 
 
+@pytest.mark.parametrize("flags", [0, 1])
 @pytest.mark.parametrize("L,B,Hq,Hkv,T0,w,rates,steps", [
     (3, 2, 8, 2, 700, 128, [0.3, 0.9], 3),                       # a few units, split over many blocks
     (5, 3, 8, 2, 300, 16, [0.0, 1.0], 4),                        # local-only and keep-all heads, tiny window
@@ -55,11 +56,11 @@ def make_stack(spkv, rng, L, B, Hq, Hkv, T0, w, rates, d_in, tau=0.5, flags=0, m
     (1, 2, 6, 2, 400, 100, [0.4, 0.7], 3),                       # one layer, odd group, odd window
     (7, 2, 4, 4, 0, 128, [0.5, 0.5, 0.5, 0.5], 5),               # from an empty cache
 ])
-def test_stack_step_matches_oracle_and_per_layer_calls(L, B, Hq, Hkv, T0, w, rates, steps):
+def test_stack_step_matches_oracle_and_per_layer_calls(L, B, Hq, Hkv, T0, w, rates, steps, flags):
     spkv = load()
     rng = np.random.default_rng(1000 + L * 7 + B)
     d_in, G = 64, Hq // Hkv
-    ca, cb, preds, units, tl = make_stack(spkv, rng, L, B, Hq, Hkv, T0, w, rates, d_in)
+    ca, cb, preds, units, tl = make_stack(spkv, rng, L, B, Hq, Hkv, T0, w, rates, d_in, flags=flags)
     ids = torch.arange(B, dtype=torch.int32, device=dev())
     scale = 1.0 / math.sqrt(D)
     for t in range(steps):
