@@ -539,15 +539,20 @@ def run_ours(args):
                    "density": sp["density"], "kv_gb_per_step": sp["kv_gb_per_step"],
                    "l2": "inputs larger than L2 (K/V read per step >> 126 MB)" if sp["kv_gb_per_step"] > 0.5
                          else "working set smaller than L2: latency-bound case",
-                   "cuda_graph": sp["graph"], "steps_per_graph": max(1, args.steps_per_graph), "launch_overlap": "SPKV_FLAG_OVERLAP" if CACHE_FLAGS[0] else "off (stream-ordered launches)", "parallelism": "replicas only" if world > 1 else "single GPU"},
+                   "cuda_graph": sp["graph"], "steps_per_graph": max(1, args.steps_per_graph),
+                   "step_api": "2 L per-layer calls" if args.per_layer else "spkv_decode_stack (2 launches per step)",
+                   "launch_overlap": ("SPKV_FLAG_OVERLAP" if CACHE_FLAGS[0] else "off (stream-ordered launches)") if args.per_layer
+                                     else "not used (plain stream-ordered launches)", "parallelism": "replicas only" if world > 1 else "single GPU"},
         "clocks": sp["clocks"], "repeats": sp["repeats"],
-        "gpu_launches": 2 * L * K,
-        # In overlap mode consecutive decode launches run under each other's head and tail, so a
-        # launch has no duration of its own inside the timed region: `achieved` is the algorithmic
-        # bytes of a launch over the average launch PERIOD there (step time / launches per step;
-        # conservative: the period also holds the fused append).  The same launch timed alone
+        "gpu_launches": (2 * L if args.per_layer else 2) * K,
+        # One step = one spkv_decode_stack call: the appends of every layer (one launch) and ONE
+        # persistent decode kernel over all layers.  `achieved` is the algorithmic bytes of the step
+        # over the step time (conservative: the step time also holds the append launch).  With
+        # --per-layer the step is 2 L launches that overlap in SPKV_FLAG_OVERLAP mode, and `achieved`
+        # is a launch's bytes over the average launch period.  A per-layer decode launch timed alone
         # (events around it, no graph, nothing overlapping) is reported beside it.
-        "roofline": {"bound": "hbm", "kernel": "decode_tc_kernel", "achieved": in_step, "peak": hbm_peak,
+        "roofline": {"bound": "hbm", "kernel": "decode_tc_kernel" if args.per_layer else "decode_stack_kernel",
+                     "achieved": in_step, "peak": hbm_peak,
                      "unit": "GB/s", "frac": in_step / hbm_peak, "peak_kind": f"of {peak_kind}",
                      "frac_of_nominal_8TBs": in_step / 8000.0,
                      "read_ceiling": {"gbs": sp.get("read_ceiling_gbs"),
@@ -555,13 +560,15 @@ def run_ours(args):
                                       "how": "spkv_stream_read over the cache arena: 32 KB bulk copies into shared "
                                              "memory, one block per SM, pages handed out by an atomic counter, "
                                              "nothing else (the measured peak above is a copy: half writes)"},
-                     "bytes_per_launch": sp["launch_bytes"], "launch_period_us": sp["ms_per_step"] * 1e3 / L,
+                     "bytes_per_launch": sp["launch_bytes"] * (1 if args.per_layer else L),
+                     "bytes_per_layer": sp["launch_bytes"], "us_per_layer": sp["ms_per_step"] * 1e3 / L,
                      "how": "algorithmic K/V, Q, O bytes of a step over the step time measured with CUDA events "
-                            "around the timed region (graph replay, launches overlapped, append included)",
-                     "launch_alone": {"achieved": achieved, "frac": achieved / hbm_peak,
-                                      "launch_us": sp["launch_s"] * 1e6,
-                                      "how": "decode launches bracketed by CUDA events, no graph, no overlap with neighbours"},
-                     "traffic": load_traffic(cfg["name"], sp["launch_bytes"])},
+                            "around the timed region (graph replay, append launch included)",
+                     "per_layer_launch_alone": {"kernel": "decode_tc_kernel", "achieved": achieved,
+                                                "frac": achieved / hbm_peak, "launch_us": sp["launch_s"] * 1e6,
+                                                "how": "one layer's spkv_decode_attention launch bracketed by CUDA "
+                                                       "events, no graph, nothing overlapping"},
+                     "traffic": load_traffic(cfg["name"], sp["launch_bytes"] * (1 if args.per_layer else L))},
         "e2e": sp.get("e2e"),
     }
     if dn is not None:
@@ -617,18 +624,22 @@ def run_config4(args):
         lg_p = torch.empty((C, Hkv), dtype=torch.float32, device=dev)
 
         def step(timers=None):
+            a, b, c_ = ev(), ev(), ev()
+            a.record()
             for l in range(L):
-                a, b, c_ = ev(), ev(), ev()
-                a.record()
                 for s in range(NP):                                           # sequences 0..7 prefill
                     cache.spkv_score(preds[l], xp, logits=lg_p)
                     cache.spkv_prefill(l, s, kp, vp, lg_p, q=qp, out=out_p)
-                b.record()
-                cache.spkv_score_append_evict(l, preds[l], dec_ids, xq[l], kd[l], vd[l])
-                cache.spkv_decode_attention(l, dec_ids, qd[l], out=out_d[l])
-                c_.record()
-                if timers is not None:
-                    timers.append((a, b, c_))
+            b.record()
+            if args.per_layer:
+                for l in range(L):
+                    cache.spkv_score_append_evict(l, preds[l], dec_ids, xq[l], kd[l], vd[l])
+                    cache.spkv_decode_attention(l, dec_ids, qd[l], out=out_d[l])
+            else:                                                             # sequences 8..63 decode: all layers, two launches
+                cache.spkv_decode_stack(preds, dec_ids, xq, qd, kd, vd, out=out_d)
+            c_.record()
+            if timers is not None:
+                timers.append((a, b, c_))
 
         for _ in range(Wm):
             step()
@@ -693,7 +704,7 @@ def run_config4(args):
                    "contexts": "uniform[4096, 65536], seeded", "keep_rates": "beta(0.5, 2.0)",
                    "density": sp["density"], "resident_gb": sp["resident_gb"],
                    "l2": "inputs larger than L2", "cuda_graph": False},
-        "clocks": sp["clocks"], "gpu_launches": K * L * (NP * 6 + 2),
+        "clocks": sp["clocks"], "gpu_launches": K * (L * NP * 6 + (2 * L if args.per_layer else 2)),
         "decode": {"tokens_per_s": K * nd / (sp["dec_ms"] * 1e-3), "ms_per_step": sp["dec_ms"] / K,
                    "achieved_gbs": sp["dec_gbs"], "frac_of_measured_hbm": sp["dec_gbs"] / hbm_peak},
         "prefill": {"tokens_per_s": K * NP * C / (sp["pre_ms"] * 1e-3), "ms_per_step": sp["pre_ms"] / K,

@@ -48,6 +48,7 @@ struct StackArgs {
   float *lse;              // [L][B][Hq] or null
   float scale_log2;
   int snap, min_pos;
+  int nb;                  // ranges per layer in the list (a layer with fewer leaves the rest empty)
   int32_t *claim;          // the launch's range counter
   char *ws;                // per-layer regions (from layer0's on): arrival counters, partial results
   size_t ws_layer_bytes, off_gcnt, off_ml, off_acc;
@@ -115,7 +116,7 @@ decode_stack_kernel(StackArgs a, int GP, int n_stages) {
   auto plan_of = [&](int layer) { return reinterpret_cast<int *>(smem + L.off_plan + (layer & 1) * L.plan_bytes); };
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int NB = (int)gridDim.x;                 // ranges per layer in the global numbering
+  const int NB = a.nb;                           // ranges per layer in the global numbering
   const int n_ranges = a.n_layers * NB;
 
   if (tid == 0) {
@@ -251,7 +252,7 @@ decode_stack_kernel(StackArgs a, int GP, int n_stages) {
         if (!have_g && !finishing) {
           const int g = __shfl_sync(0xffffffffu, pending, 0);
           if (g >= n_ranges) {
-            if (g == n_ranges + NB - 1 && lane == 0) *a.claim = 0;
+            if (g == n_ranges + (int)gridDim.x - 1 && lane == 0) *a.claim = 0;
             finishing = true;
             tgt_layer = a.n_layers - 1;
           } else {
@@ -577,6 +578,7 @@ int spkv::decode_stack_layers(spkv_cache *cache, int l0, int l1, const spkv_pred
   // the per-layer kernel's rule, so that both paths cut a layer's pages the same way: a cache in
   // overlap mode gives a range at least 56 positions when the layer has half a grid of such ranges
   a.min_pos = (cfg.flags & SPKV_FLAG_OVERLAP) ? 56 : 4;
+  a.nb = min(kMaxGrid, cache->sm_count);
   a.claim = reinterpret_cast<int32_t *>(ws);
   a.ws = ws + 256 + (size_t)l0 * per_layer;
   a.ws_layer_bytes = per_layer;
