@@ -262,3 +262,78 @@ def test_config1_every_step_of_the_chain():
     for h in range(Hkv):
         compare_state(cache2, 0, 0, h, units[h][0])
         assert_attn_close(out2[:, h * G:(h + 1) * G], units[h][1], f"prefill form, kv head {h}")
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,T,beta,sampled", [
+    (16, 32, 8, 32768, (0.5, 2.0), 11),
+    (4, 32, 8, 131072, (0.3, 3.0), 2),
+], ids=["config2", "config3"])
+def test_two_layers_full_size_stack_step(B, Hq, Hkv, T, beta, sampled):
+    """The launch configuration bench.py times: decode steps through spkv_decode_stack (the appends
+    of every layer in one launch, one persistent decode kernel over the layers), two layers at
+    the shapes of configs 2 and 3.  The new tokens are scored by the layers' linear predictors
+    inside the call; the oracle is fed the float32 logits the call returns.  Checked for the
+    sampled sequence (both layers, all KV heads): decode outputs of three steps against the
+    oracle's streaming form, final state bit-exact; for every unit: the kept-set identity."""
+    spkv = load()
+    L, w, C, steps, d_in = 2, 128, 8192, 3, 64
+    G = Hq // Hkv
+    rng = np.random.default_rng(4321)
+    rates = synth.keep_rates(rng, L, Hkv, *beta)
+    rates[0, 0], rates[0, 5], rates[1, 2] = 0.0, 0.97, 1.0         # local-only, near-full and full heads
+    pages = int(np.ceil(rates * (T + steps) * 1.05 / 64 + 2).sum()) * B
+    cache = spkv.Cache(n_layers=L, max_seqs=B, n_q_heads=Hq, n_kv_heads=Hkv, max_context=T + 128,
+                       pool_pages=pages, window=w, tau=0.5, flags=spkv.FLAG_OVERLAP)   # as bench.py creates it
+    tl = cache.spkv_tau_logit()
+    logit = np.stack([np.stack([synth.logits_with_keep_rate(rng, (T, B), float(r), tl) for r in rates[l]], axis=-1)
+                      for l in range(L)])                           # [L, T, B, Hkv]
+    Ks = synth.normal_bf16(rng, (L, T + steps, Hkv, D))              # the sampled sequence's pairs
+    Vs = synth.normal_bf16(rng, (L, T + steps, Hkv, D))
+    gen = torch.Generator(device=dev())
+    gen.manual_seed(9)
+    preds = []
+    for l in range(L):
+        Wl = synth.linear_predictor(rng, Hkv, d_in)
+        preds.append(spkv.make_predictor(to_dev_bf16(Wl), torch.from_numpy(
+            synth.bias_for_keep_rate(Wl, rates[l], tl)).to(dev())))
+        lg_dev = torch.from_numpy(logit[l]).to(dev())
+        for s in range(B):
+            if s == sampled:
+                Kd, Vd = to_dev_bf16(Ks[l, :T]), to_dev_bf16(Vs[l, :T])
+            else:
+                Kd = torch.randn((T, Hkv, D), generator=gen, device=dev()).to(torch.bfloat16)
+                Vd = torch.randn((T, Hkv, D), generator=gen, device=dev()).to(torch.bfloat16)
+            for a in range(0, T, C):
+                cache.spkv_prefill(l, s, Kd[a:a + C], Vd[a:a + C], lg_dev[a:a + C, s].contiguous())
+    assert cache.spkv_status() == 0
+    units = [[oracle.Unit(w, D) for _ in range(Hkv)] for _ in range(L)]
+    for l in range(L):
+        for h in range(Hkv):
+            units[l][h].prefill(np.ascontiguousarray(Ks[l, :T, h]), np.ascontiguousarray(Vs[l, :T, h]),
+                                np.ascontiguousarray(logit[l, :T, sampled, h]), tl)
+    ids = torch.arange(B, dtype=torch.int32, device=dev())
+    scale = 1.0 / math.sqrt(D)
+    for step in range(steps):
+        t = T + step
+        x = torch.randn((L, B, d_in), generator=gen, device=dev()).to(torch.bfloat16)
+        k_new = torch.randn((L, B, Hkv, D), generator=gen, device=dev()).to(torch.bfloat16)
+        v_new = torch.randn((L, B, Hkv, D), generator=gen, device=dev()).to(torch.bfloat16)
+        q_new = torch.randn((L, B, Hq, D), generator=gen, device=dev()).to(torch.bfloat16)
+        for l in range(L):
+            k_new[l, sampled], v_new[l, sampled] = to_dev_bf16(Ks[l, t]), to_dev_bf16(Vs[l, t])
+        lg_new = torch.empty((L, B, Hkv), dtype=torch.float32, device=dev())
+        out = spkv.bits_from_bf16(cache.spkv_decode_stack(preds, ids, x, q_new, k_new, v_new, logits_out=lg_new))
+        q_bits, lg_host = spkv.bits_from_bf16(q_new), lg_new.cpu().numpy()
+        for l in range(L):
+            for h in range(Hkv):
+                units[l][h].append(Ks[l, t, h], Vs[l, t, h], lg_host[l, sampled, h], tl)
+                ref = units[l][h].attend(np.ascontiguousarray(q_bits[l, sampled, h * G:(h + 1) * G]), scale)
+                assert_attn_close(out[l, sampled, h * G:(h + 1) * G], ref, f"stack step={step} layer={l} h={h}")
+    assert cache.spkv_status() == 0
+    for l in range(L):
+        ln, tt = cache.spkv_read_lengths(l)
+        want = (logit[l, :T + steps - w] >= np.float32(tl)).sum(axis=0)      # [B, Hkv]: all from the prefill logits
+        assert np.array_equal(ln, want.astype(np.int32)) and (tt == T + steps).all()
+        for h in (0, 2, 5):
+            compare_state(cache, l, sampled, h, units[l][h])
+    assert cache.spkv_read_lengths(0)[0][:, 0].max() == 0 and cache.spkv_read_lengths(1)[0][:, 2].min() == T + steps - w
