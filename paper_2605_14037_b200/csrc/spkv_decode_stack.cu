@@ -23,9 +23,9 @@
 // counters live in per-layer regions of the workspace, merged by whoever arrives last.
 //
 // Warps: 8 consumers (two groups taking alternate pages), producer, epilogue, planner.
-// Shared memory: page stages, two hand-over buffers, two plans (layer parity).
+// Shared memory: page stages, two hand-over buffers, two to four plans (layer modulo their number).
 // Hand-shakes inside the block (mbarriers, every wait bounded):
-//   plan_ready[p]  planner -> producer: the plan of a layer of parity p is complete;
+//   plan_ready[p]  planner -> producer: the plan in buffer p is complete;
 //   plan_free[p]   epilogue -> planner: nobody needs that plan any more.  The producer sends a
 //                  marker down the page pipeline when it moves on to the next layer; the
 //                  consumers pass it on, and the epilogue warp, which sees it after the last segment
@@ -37,6 +37,7 @@
 namespace spkv {
 
 constexpr int kStackThreads = (kConsumerWarps + 3) * 32;  // + producer, epilogue, planner
+constexpr int kMaxPlans = 4;  // plan buffers: the planner may be this many layers ahead of the epilogue warp
 enum { F_LAYER = 8 };  // stage flag: no page, "the producer has left this layer"
 
 struct StackArgs {
@@ -72,22 +73,23 @@ __host__ __device__ inline StackPlan stack_plan_layout(int n) {
 }
 
 struct StackSmem {
-  int n_stages, stage_bytes, off_bar, off_meta, off_seq, off_np, off_plan, plan_bytes, off_red, off_mrg, off_flags,
+  int n_stages, n_plans, stage_bytes, off_bar, off_meta, off_seq, off_np, off_plan, plan_bytes, off_red, off_mrg, off_flags,
       total;
 };
-__host__ __device__ inline StackSmem stack_smem_layout(int n_items, int B, int GP, int n_stages) {
+__host__ __device__ inline StackSmem stack_smem_layout(int n_items, int B, int GP, int n_stages, int n_plans) {
   StackSmem L;
   L.n_stages = n_stages;
+  L.n_plans = n_plans;
   L.stage_bytes = kPageBytes + GP * kRowBytes;
   int o = n_stages * L.stage_bytes;
   o = (o + 15) / 16 * 16;
-  L.off_bar = o;   o += (2 * kMaxStages + 8) * 8;  // full[], empty[], red_full[2], red_empty[2], plan_ready[2], plan_free[2]
+  L.off_bar = o;   o += (2 * kMaxStages + 4 + 2 * kMaxPlans) * 8;  // full[], empty[], red_full[2], red_empty[2], plan_ready[], plan_free[]
   L.off_meta = o;  o += kMaxStages * (int)sizeof(StageMeta);
   L.off_seq = o;   o += B * 4;
   L.off_np = o;    o += n_items * 4;
   o = (o + 15) / 16 * 16;
   L.plan_bytes = stack_plan_layout(n_items).ints * 4;
-  L.off_plan = o;  o += 2 * L.plan_bytes;
+  L.off_plan = o;  o += n_plans * L.plan_bytes;
   L.off_red = o;   o += 2 * kConsumerWarps * GP * 132 * 4;
   L.off_mrg = o;   o += kMergeCap * 8;
   L.off_flags = o; o += 32;
@@ -97,23 +99,23 @@ __host__ __device__ inline StackSmem stack_smem_layout(int n_items, int B, int G
 
 template <int NH>  // 8-head tiles on the N side: 1 for G <= 8, 2 for G <= 16
 __global__ void __launch_bounds__(kStackThreads, 1)
-decode_stack_kernel(StackArgs a, int GP, int n_stages) {
+decode_stack_kernel(StackArgs a, int GP, int n_stages, int n_plans) {
   extern __shared__ __align__(1024) unsigned char smem[];
   const CacheView &c = a.c;
   const int n = a.n_items;
-  const StackSmem L = stack_smem_layout(n, a.B, GP, n_stages);
+  const StackSmem L = stack_smem_layout(n, a.B, GP, n_stages, n_plans);
   const StackPlan PL = stack_plan_layout(n);
   uint64_t *full = reinterpret_cast<uint64_t *>(smem + L.off_bar);
   uint64_t *empty = full + kMaxStages;
   uint64_t *red_full = empty + kMaxStages, *red_empty = red_full + 2;
-  uint64_t *plan_ready = red_empty + 2, *plan_free = plan_ready + 2;
+  uint64_t *plan_ready = red_empty + 2, *plan_free = plan_ready + kMaxPlans;
   volatile StageMeta *s_meta = reinterpret_cast<volatile StageMeta *>(smem + L.off_meta);
   int *s_seq = reinterpret_cast<int *>(smem + L.off_seq);
   int *s_np = reinterpret_cast<int *>(smem + L.off_np);
   float *s_red = reinterpret_cast<float *>(smem + L.off_red);
   float2 *s_mrg = reinterpret_cast<float2 *>(smem + L.off_mrg);
   volatile int *s_redmeta = reinterpret_cast<volatile int *>(smem + L.off_flags);  // [rb]: item, [2+rb]: range, [4+rb]: layer
-  auto plan_of = [&](int layer) { return reinterpret_cast<int *>(smem + L.off_plan + (layer & 1) * L.plan_bytes); };
+  auto plan_of = [&](int layer) { return reinterpret_cast<int *>(smem + L.off_plan + (layer % n_plans) * L.plan_bytes); };
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int NB = a.nb;                           // ranges per layer in the global numbering
@@ -127,6 +129,8 @@ decode_stack_kernel(StackArgs a, int GP, int n_stages) {
     for (int i = 0; i < 2; ++i) {
       mbar_init(&red_full[i], kConsumerWarps);
       mbar_init(&red_empty[i], 1);
+    }
+    for (int i = 0; i < n_plans; ++i) {
       mbar_init(&plan_ready[i], 1);
       mbar_init(&plan_free[i], 1);
     }
@@ -148,7 +152,7 @@ decode_stack_kernel(StackArgs a, int GP, int n_stages) {
     // cuts -- what the per-layer kernel's whole block does before its first page, here by one warp
     // while the previous layer streams.
     for (int l = 0; l < a.n_layers; ++l) {
-      if (l >= 2 && !wait_or_flag(&plan_free[l & 1], ((l >> 1) - 1) & 1, c)) break;
+      if (l >= n_plans && !wait_or_flag(&plan_free[l % n_plans], ((l / n_plans) - 1) & 1, c)) break;
       int *P = plan_of(l);
       for (int i = lane; i < n; i += 32) {
         const int b = i / c.Hkv, kvh = i % c.Hkv;
@@ -202,7 +206,7 @@ decode_stack_kernel(StackArgs a, int GP, int n_stages) {
         P[PL.hdr + 1] = nb_eff;
       }
       __syncwarp();
-      if (lane == 0) mbar_arrive(&plan_ready[l & 1]);
+      if (lane == 0) mbar_arrive(&plan_ready[l % n_plans]);
     }
   } else if (warp == kConsumerWarps) {
     // ------------------------------------------------------------------ producer warp
@@ -267,7 +271,7 @@ decode_stack_kernel(StackArgs a, int GP, int n_stages) {
           gq.mark = layer;  // (-1 before the first layer: nothing to tell)
           ++layer;
           int ok = 1;
-          if (lane == 0) ok = wait_or_flag(&plan_ready[layer & 1], (layer >> 1) & 1, c);
+          if (lane == 0) ok = wait_or_flag(&plan_ready[layer % n_plans], (layer / n_plans) & 1, c);
           if (!__shfl_sync(0xffffffffu, ok, 0)) {
             gave_up = 1;
             more = false;
@@ -473,7 +477,7 @@ decode_stack_kernel(StackArgs a, int GP, int n_stages) {
       if (item == -2) {  // every segment of `layer` has passed: the planner may reuse its plan
         __syncwarp();
         if (lane == 0) {
-          mbar_arrive(&plan_free[layer & 1]);
+          mbar_arrive(&plan_free[layer % n_plans]);
           mbar_arrive(&red_empty[rb]);
         }
         continue;
@@ -586,15 +590,19 @@ int spkv::decode_stack_layers(spkv_cache *cache, int l0, int l1, const spkv_pred
   int GP = 1;
   while (GP < v.G) GP <<= 1;
   const int limit = 227 * 1024;
-  int n_stages = 6;
-  StackSmem SL = stack_smem_layout(n_items, B, GP, n_stages);
-  while (SL.total > limit && n_stages > 2) SL = stack_smem_layout(n_items, B, GP, --n_stages);
+  // as many page stages as fit beside two plans; then as many plans (up to four: small layers are
+  // paced by how far ahead the planner may run) as fit without costing a stage
+  int n_stages = 6, n_plans = 2;
+  StackSmem SL = stack_smem_layout(n_items, B, GP, n_stages, n_plans);
+  while (SL.total > limit && n_stages > 2) SL = stack_smem_layout(n_items, B, GP, --n_stages, n_plans);
   if (SL.total > limit) return SPKV_E_UNSUPPORTED;
-  void (*kernel)(StackArgs, int, int) = GP > 8 ? decode_stack_kernel<2> : decode_stack_kernel<1>;
+  while (n_plans < kMaxPlans && stack_smem_layout(n_items, B, GP, n_stages, n_plans + 1).total <= limit)
+    SL = stack_smem_layout(n_items, B, GP, n_stages, ++n_plans);
+  void (*kernel)(StackArgs, int, int, int) = GP > 8 ? decode_stack_kernel<2> : decode_stack_kernel<1>;
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SL.total) != cudaSuccess)
     return SPKV_E_CUDA;
   const int grid = min(kMaxGrid, cache->sm_count);
-  kernel<<<grid, kStackThreads, SL.total, s>>>(a, GP, n_stages);
+  kernel<<<grid, kStackThreads, SL.total, s>>>(a, GP, n_stages, n_plans);
   return check_stream_error(cudaGetLastError());
 }
 
