@@ -84,6 +84,11 @@ def test_workspace_sizes_and_error_strings(spkv):
     assert 0 < a < b
     assert l.spkv_decode_step_staging_bytes(C.byref(c), 3, 512) > b
     assert l.spkv_prefill_workspace_bytes(C.byref(c), 8192) > 0
+    # the stack step keeps arrival counters and partial results per layer (one half of a per-layer
+    # workspace each), one counter word, and a per-layer workspace for its fallback path
+    per_layer = (b // 2 + 255) // 256 * 256
+    assert l.spkv_decode_stack_workspace_bytes(C.byref(c), 3) == 256 + c.n_layers * per_layer + b
+    assert l.spkv_decode_stack_workspace_bytes(None, 3) == 0
     assert l.spkv_error_string(0) == b"ok"
     seen = {l.spkv_error_string(code) for code in range(-10, 1)}
     assert len(seen) == 11 and b"unknown error" not in seen
