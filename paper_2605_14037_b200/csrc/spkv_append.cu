@@ -160,6 +160,10 @@ __global__ void __launch_bounds__(128)
 append_stack_kernel(CacheView c, StackPreds sp, int layer0, int n_layers, const int32_t *__restrict__ seq_ids, int B,
                     const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new,
                     const __nv_bfloat16 *__restrict__ x, int d_in, float *__restrict__ logits_out, float tau_logit) {
+  // the decode launch behind this one is a programmatic dependent launch: let its blocks become
+  // resident and run their block-local set-up now (they wait for this grid to complete before they
+  // read the cache)
+  pdl_trigger();
   const int items = B * c.Hkv;
   const long long g = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int layer = (int)(g / items), item = (int)(g % items);

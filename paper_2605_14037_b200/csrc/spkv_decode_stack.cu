@@ -144,6 +144,10 @@ decode_stack_kernel(StackArgs a, int GP, int n_stages, int n_plans) {
         make_uint4(0, 0, 0, 0);
   }
   for (int i = tid; i < a.B; i += kStackThreads) s_seq[i] = a.seq_ids[i];
+  // Everything above touched only this block's shared memory and an input of the call; the launch
+  // is a programmatic dependent one, so it may have run under the tail of the append launch.  From
+  // here on the cache is read: wait for that launch (and everything before it) to complete.
+  pdl_wait();
   __syncthreads();
 
   if (warp == kConsumerWarps + 2) {
@@ -602,8 +606,8 @@ int spkv::decode_stack_layers(spkv_cache *cache, int l0, int l1, const spkv_pred
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SL.total) != cudaSuccess)
     return SPKV_E_CUDA;
   const int grid = min(kMaxGrid, cache->sm_count);
-  kernel<<<grid, kStackThreads, SL.total, s>>>(a, GP, n_stages, n_plans);
-  return check_stream_error(cudaGetLastError());
+  return check_stream_error(
+      launch_overlapped(kernel, dim3(grid), dim3(kStackThreads), (size_t)SL.total, s, a, GP, n_stages, n_plans));
 }
 
 extern "C" int spkv_decode_stack(spkv_cache_t *cache, const spkv_predictor_t *preds, const int32_t *d_seq_ids, int32_t B,
