@@ -905,9 +905,9 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--settle-seconds", type=float, default=1.0,
                     help="untimed replay of the timed region before the first repeat (clocks settle under load)")
-    ap.add_argument("--steps-per-graph", type=int, default=1,
-                    help="steps captured in one CUDA graph (default 1; more shows the device time of a "
-                         "tiny step where the host's replay rate is the limit)")
+    ap.add_argument("--steps-per-graph", type=int, default=0,
+                    help="steps captured in one CUDA graph (default: 1, and 16 for the tiny config 1, whose "
+                         "step is shorter than the time the host needs to replay a graph)")
     ap.add_argument("--per-layer", action="store_true",
                     help="time the step as 2 L per-layer calls (spkv_score_append_evict, spkv_decode_attention) "
                          "instead of one spkv_decode_stack call (comparison run, not the bench line)")
@@ -925,6 +925,8 @@ def main():
         sys.exit(subprocess.call(replica_launch_command(args.gpus, sys.argv[1:])))
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
+    if args.steps_per_graph <= 0:
+        args.steps_per_graph = 16 if args.config == 1 else 1
     if args.stream_ordered:
         CACHE_FLAGS[0] = 0
     if args.impl == "reference":

@@ -127,3 +127,45 @@ def test_stack_step_repeats_bit_for_bit_and_refuses_bad_arguments():
     assert f(*args(B=0)) == 0
     torch.cuda.synchronize()
     assert ca.spkv_status() == 0
+
+
+def test_stack_step_with_sinks_local_only_heads_and_per_head_thresholds():
+    """The variants of the cache go through the stack step unchanged: sink tokens, a head declared
+    local-only at creation (no page table), per-head thresholds set at run time, range checks on.
+    Compared bit for bit with the per-layer calls (which test_gpu_sinks / test_gpu_hybrid hold
+    against the oracle) from an empty cache over enough steps for evictions and second pages."""
+    spkv = load()
+    rng = np.random.default_rng(5)
+    L, B, Hq, Hkv, w, d_in, steps = 3, 2, 8, 4, 16, 64, 150
+    local = np.zeros((L, Hkv), dtype=np.uint8)
+    local[1, 2] = 1
+    mk = lambda: spkv.Cache(n_layers=L, max_seqs=B, n_q_heads=Hq, n_kv_heads=Hkv, max_context=512, pool_pages=96,
+                            window=w, tau=0.5, sink_tokens=3, local_only=local, flags=spkv.FLAG_DEBUG_BOUNDS)
+    ca, cb = mk(), mk()
+    for c_ in (ca, cb):
+        c_.spkv_set_head_tau(0, 1, 1.0)        # a local-only head declared at run time
+        c_.spkv_set_head_tau(2, 0, 0.0)        # a full-attention head
+    tl = ca.spkv_tau_logit()
+    preds = []
+    for l in range(L):
+        W = synth.linear_predictor(rng, Hkv, d_in)
+        preds.append(spkv.make_predictor(to_dev_bf16(W), torch.from_numpy(
+            synth.bias_for_keep_rate(W, [0.2, 0.5, 0.8, 0.4], tl)).to(dev())))
+    ids = torch.tensor([1, 0], dtype=torch.int32, device=dev())
+    for t in range(steps):
+        x, q = to_dev_bf16(synth.normal_bf16(rng, (L, B, d_in))), to_dev_bf16(synth.normal_bf16(rng, (L, B, Hq, D)))
+        k, v = to_dev_bf16(synth.normal_bf16(rng, (L, B, Hkv, D))), to_dev_bf16(synth.normal_bf16(rng, (L, B, Hkv, D)))
+        out_a = ca.spkv_decode_stack(preds, ids, x, q, k, v)
+        for l in range(L):
+            cb.spkv_score_append_evict(l, preds[l], ids, x[l], k[l], v[l])
+            out_b = cb.spkv_decode_attention(l, ids, q[l])
+            assert torch.equal(out_a[l].view(torch.int16), out_b.view(torch.int16)), (t, l)
+    assert ca.spkv_status() == 0 and cb.spkv_status() == 0
+    for l in range(L):
+        la, lb = ca.spkv_read_lengths(l)[0], cb.spkv_read_lengths(l)[0]
+        assert np.array_equal(la, lb)
+    assert ca.spkv_read_lengths(1)[0][:, 2].max() == 0                   # declared local-only: not even the sinks
+    assert (ca.spkv_read_lengths(0)[0][:, 1] == 3).all()                 # threshold 1 at run time: the sinks only
+    assert ca.spkv_read_lengths(2)[0][:, 0].min() == steps - w          # the full-attention head kept every evictee
+    for h in (0, 3):
+        assert ca.spkv_read_kept(1, 1, h)[0][:3].tolist() == [0, 1, 2]   # the sinks lead the cache
