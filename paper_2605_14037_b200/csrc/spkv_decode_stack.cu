@@ -246,7 +246,7 @@ decode_stack_kernel(StackArgs a, int GP, int n_stages, int n_plans) {
     // claims until the counter has run past the list, i.e. fails exactly once: the claim that brings
     // the counter to n_ranges + gridDim.x is the launch's last, and its owner leaves it at zero.
     // A block whose list is exhausted still visits the remaining layers (markers only): the planner
-    // walks them all, each only after this block has left the layer two before it.
+    // walks them all, each only after this block has left the layer that held its plan buffer before.
     bool have_g = false, finishing = false;
     int tgt_layer = 0, g_cidx = 0;
     // Resolves the next (up to) 32 positions of the range (markers come out with valid = 0), taking a
