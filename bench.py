@@ -574,7 +574,9 @@ def run_ours(args):
     if dn is not None:
         dn_ach = dn["launch_bytes"] / dn["launch_s"] / 1e9
         line["dense"] = {"tokens_per_s": dn["tokens_per_s"], "ms_per_step": dn["ms_per_step"],
-                         "kv_gb_per_step": dn["kv_gb_per_step"], "achieved_gbs": dn_ach,
+                         "kv_gb_per_step": dn["kv_gb_per_step"],
+                         "in_step_gbs": dn["kv_gb_per_step"] / dn["ms_per_step"] * 1e3,   # K/V bytes of a step over its time
+                         "achieved_gbs": dn_ach,                                          # one per-layer launch, timed alone
                          "layers_measured": dn["layers_measured"],
                          "scaled_from_layer_subset": dn["layers_measured"] != L,
                          "frac": dn_ach / hbm_peak,
