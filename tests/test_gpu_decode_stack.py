@@ -55,6 +55,8 @@ def make_stack(spkv, rng, L, B, Hq, Hkv, T0, w, rates, d_in, tau=0.5, flags=0, m
     (4, 1, 16, 1, 1500, 128, [0.6], 2),                          # 16 query heads per KV head
     (1, 2, 6, 2, 400, 100, [0.4, 0.7], 3),                       # one layer, odd group, odd window
     (7, 2, 4, 4, 0, 128, [0.5, 0.5, 0.5, 0.5], 5),               # from an empty cache
+    (33, 1, 4, 1, 0, 16, [0.5], 40),                             # many tiny layers: the plan buffers wrap many times
+    (12, 2, 8, 2, 90, 16, [0.0, 1.0], 6),                        # layers of a page or two: most blocks visit them empty-handed
 ])
 def test_stack_step_matches_oracle_and_per_layer_calls(L, B, Hq, Hkv, T0, w, rates, steps, flags):
     spkv = load()
