@@ -412,8 +412,9 @@ int spkv_decode_step_host_flush(spkv_cache_t *cache, spkv_stream_t stream);
  * persistent decode-attention kernel whose blocks take page ranges of all layers from one list,
  * so that their page streams never stop between layers.  Ordinary stream-ordered launches (no
  * SPKV_FLAG_OVERLAP contract); no synchronisation.
- *   preds [n_layers]: HOST array of predictors with the same d_in (linear predictors and up to 128
- *   layers take the two launches; otherwise the call falls back to the per-layer calls);
+ *   preds [n_layers]: HOST array of predictors with the same d_in (linear predictors, up to 128
+ *   layers and a batch whose per-layer plans fit in shared memory take the two launches; otherwise
+ *   the call makes the per-layer calls itself);
  *   d_x [L, B, d_in], d_q [L, B, n_q_heads, 128], d_k/d_v [L, B, n_kv_heads, 128] bf16, 16-byte
  *   aligned -> d_out [L, B, n_q_heads, 128] bf16; d_logits_out [L, B, n_kv_heads] float32 or NULL
  *   (required by two-layer predictors); d_lse_opt [L, B, n_q_heads] float32 or NULL;

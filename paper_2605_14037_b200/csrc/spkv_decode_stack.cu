@@ -540,11 +540,25 @@ int spkv::decode_stack_layers(spkv_cache *cache, int l0, int l1, const spkv_pred
   const size_t x_l = (size_t)B * d_in * 2, q_l = (size_t)B * cfg.n_q_heads * kD * 2, kv_l = (size_t)n_items * kD * 2;
   cudaStream_t s = as_stream(stream);
 
-  bool fused = nl <= kMaxStackLayers && d_in >= 8 && (d_in & 7) == 0 && (x_l & 15) == 0;
+  // shared memory of the persistent kernel: as many page stages as fit beside two plans; then as
+  // many plans (up to four: small layers are paced by how far ahead the planner may run) as fit
+  // without costing a stage
+  int GP = 1;
+  while (GP < v.G) GP <<= 1;
+  const int limit = 227 * 1024;
+  int n_stages = 6, n_plans = 2;
+  StackSmem SL = stack_smem_layout(n_items, B, GP, n_stages, n_plans);
+  while (SL.total > limit && n_stages > 2) SL = stack_smem_layout(n_items, B, GP, --n_stages, n_plans);
+  while (SL.total <= limit && n_plans < kMaxPlans &&
+         stack_smem_layout(n_items, B, GP, n_stages, n_plans + 1).total <= limit)
+    SL = stack_smem_layout(n_items, B, GP, n_stages, ++n_plans);
+
+  bool fused = nl <= kMaxStackLayers && d_in >= 8 && (d_in & 7) == 0 && (x_l & 15) == 0 && SL.total <= limit;
   for (int l = l0; l < l1 && fused; ++l)
     fused = preds[l].kind == 0 && preds[l].d_W1 && preds[l].d_b1 && ((uintptr_t)preds[l].d_W1 & 15) == 0;
   if (!fused) {
-    // two-layer predictors (scored by a kernel of their own) and very deep stacks: layer by layer
+    // two-layer predictors (scored by a kernel of their own), very deep stacks, and batches whose
+    // plans leave no room for two page stages: layer by layer
     void *ws1 = ws + 256 + (size_t)L * per_layer;
     for (int l = l0; l < l1; ++l) {
       float *lg = d_logits_out ? d_logits_out + (size_t)l * n_items : nullptr;
@@ -591,17 +605,6 @@ int spkv::decode_stack_layers(spkv_cache *cache, int l0, int l1, const spkv_pred
   a.ws = ws + 256 + (size_t)l0 * per_layer;
   a.ws_layer_bytes = per_layer;
   a.off_gcnt = wl.off_gcnt; a.off_ml = wl.off_ml; a.off_acc = wl.off_acc;
-  int GP = 1;
-  while (GP < v.G) GP <<= 1;
-  const int limit = 227 * 1024;
-  // as many page stages as fit beside two plans; then as many plans (up to four: small layers are
-  // paced by how far ahead the planner may run) as fit without costing a stage
-  int n_stages = 6, n_plans = 2;
-  StackSmem SL = stack_smem_layout(n_items, B, GP, n_stages, n_plans);
-  while (SL.total > limit && n_stages > 2) SL = stack_smem_layout(n_items, B, GP, --n_stages, n_plans);
-  if (SL.total > limit) return SPKV_E_UNSUPPORTED;
-  while (n_plans < kMaxPlans && stack_smem_layout(n_items, B, GP, n_stages, n_plans + 1).total <= limit)
-    SL = stack_smem_layout(n_items, B, GP, n_stages, ++n_plans);
   void (*kernel)(StackArgs, int, int, int) = GP > 8 ? decode_stack_kernel<2> : decode_stack_kernel<1>;
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SL.total) != cudaSuccess)
     return SPKV_E_CUDA;

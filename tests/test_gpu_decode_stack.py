@@ -171,3 +171,36 @@ def test_stack_step_with_sinks_local_only_heads_and_per_head_thresholds():
     assert ca.spkv_read_lengths(2)[0][:, 0].min() == steps - w          # the full-attention head kept every evictee
     for h in (0, 3):
         assert ca.spkv_read_kept(1, 1, h)[0][:3].tolist() == [0, 1, 2]   # the sinks lead the cache
+
+
+def test_stack_step_with_two_layer_predictors_makes_the_per_layer_calls():
+    """Two-layer predictors are scored by a kernel of their own, so the stack call falls back to the
+    per-layer calls inside the library: same results as making them oneself, logits required."""
+    spkv = load()
+    rng = np.random.default_rng(11)
+    L, B, Hq, Hkv, w, d_in, hidden, steps = 3, 2, 8, 2, 16, 64, 32, 40
+    mk = lambda: spkv.Cache(n_layers=L, max_seqs=B, n_q_heads=Hq, n_kv_heads=Hkv, max_context=256, pool_pages=48,
+                            window=w, tau=0.5)
+    ca, cb = mk(), mk()
+    preds = []
+    for l in range(L):
+        W1 = to_dev_bf16(synth.normal_bf16(rng, (hidden, d_in)))
+        W2 = to_dev_bf16(synth.normal_bf16(rng, (Hkv, hidden)))
+        b1 = torch.from_numpy(rng.standard_normal(hidden).astype(np.float32)).to(dev())
+        b2 = torch.from_numpy(rng.standard_normal(Hkv).astype(np.float32)).to(dev())
+        preds.append(spkv.make_predictor(W1, b1, W2, b2))
+    ids = torch.arange(B, dtype=torch.int32, device=dev())
+    for t in range(steps):
+        x, q = to_dev_bf16(synth.normal_bf16(rng, (L, B, d_in))), to_dev_bf16(synth.normal_bf16(rng, (L, B, Hq, D)))
+        k, v = to_dev_bf16(synth.normal_bf16(rng, (L, B, Hkv, D))), to_dev_bf16(synth.normal_bf16(rng, (L, B, Hkv, D)))
+        lg_a = torch.empty((L, B, Hkv), dtype=torch.float32, device=dev())
+        out_a = ca.spkv_decode_stack(preds, ids, x, q, k, v, logits_out=lg_a)
+        for l in range(L):
+            lg_b = torch.empty((B, Hkv), dtype=torch.float32, device=dev())
+            cb.spkv_score_append_evict(l, preds[l], ids, x[l], k[l], v[l], logits_out=lg_b)
+            out_b = cb.spkv_decode_attention(l, ids, q[l])
+            assert torch.equal(lg_a[l].view(torch.int32), lg_b.view(torch.int32)), (t, l)
+            assert torch.equal(out_a[l].view(torch.int16), out_b.view(torch.int16)), (t, l)
+    assert ca.spkv_status() == 0 and cb.spkv_status() == 0
+    with pytest.raises(spkv.SpkvError):                       # two-layer predictors need the logits buffer
+        ca.spkv_decode_stack(preds, ids, x, q, k, v)
