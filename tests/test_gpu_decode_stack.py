@@ -204,3 +204,34 @@ def test_stack_step_with_two_layer_predictors_makes_the_per_layer_calls():
     assert ca.spkv_status() == 0 and cb.spkv_status() == 0
     with pytest.raises(spkv.SpkvError):                       # two-layer predictors need the logits buffer
         ca.spkv_decode_stack(preds, ids, x, q, k, v)
+
+
+def test_stack_step_replayed_from_a_cuda_graph_matches_eager_calls():
+    """bench.py replays the stack step as a CUDA graph: a captured step, replayed with fresh inputs
+    copied into its buffers, against eager calls on a second cache -- outputs and final lengths,
+    bit for bit, over enough steps for evictions."""
+    spkv = load()
+    rng = np.random.default_rng(21)
+    L, B, Hq, Hkv, d_in, steps = 4, 3, 8, 2, 64, 12
+    ca, cb, preds, units, tl = make_stack(spkv, rng, L, B, Hq, Hkv, 600, 128, [0.3, 0.8], d_in, flags=1)
+    ids = torch.arange(B, dtype=torch.int32, device=dev())
+    bufs = [torch.zeros(shape, dtype=torch.bfloat16, device=dev())
+            for shape in ((L, B, d_in), (L, B, Hq, D), (L, B, Hkv, D), (L, B, Hkv, D))]
+    out_g = torch.zeros((L, B, Hq, D), dtype=torch.bfloat16, device=dev())
+    ca.spkv_decode_stack(preds, ids, *bufs, out=out_g)          # warm-up outside the capture (same step on both caches)
+    cb.spkv_decode_stack(preds, ids, *bufs)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):                                    # capturing runs nothing
+        ca.spkv_decode_stack(preds, ids, *bufs, out=out_g)
+    for t in range(steps):
+        fresh = [to_dev_bf16(synth.normal_bf16(rng, tuple(b.shape))) for b in bufs]
+        for b, f in zip(bufs, fresh):
+            b.copy_(f)
+        g.replay()
+        want = cb.spkv_decode_stack(preds, ids, *fresh)
+        torch.cuda.synchronize()
+        assert torch.equal(out_g.view(torch.int16), want.view(torch.int16)), t
+    assert ca.spkv_status() == 0 and cb.spkv_status() == 0
+    for l in range(L):
+        assert np.array_equal(ca.spkv_read_lengths(l)[0], cb.spkv_read_lengths(l)[0])
