@@ -192,6 +192,53 @@ __device__ inline void merge_rows(const float *g_acc /* first slot, + lane * 4 *
 }
 
 
+// ---- the consumer warps' state for one segment (shared by the per-layer and the stack kernel) ----
+// A consumer warp keeps, for its 16 of every page's 64 pairs, the query fragments of the group's
+// heads (qb) and the running maximum, sum and output accumulators (m, l, o) in the MMA tiles'
+// register layout: lane = 4 g + t4 holds heads 2 t4, 2 t4 + 1 of every 8-head tile.
+
+// First page of a segment: the group's query rows (in the stage, behind the page) -> fragments;
+// accumulators cleared.
+template <int NH>
+__device__ inline void segment_begin(uint32_t (&qb)[NH][8][2], float (&m)[NH][2], float (&l)[NH][2],
+                                     float (&o)[NH][8][4], const __nv_bfloat16 *qs, int GP, int lane) {
+  load_q_frags_t<NH>(qb, [&](int h) -> const __nv_bfloat16 * { return h < GP ? qs + h * kD : nullptr; }, lane);
+#pragma unroll
+  for (int hn = 0; hn < NH; ++hn) {
+    m[hn][0] = m[hn][1] = -INFINITY;
+    l[hn][0] = l[hn][1] = 0.f;
+#pragma unroll
+    for (int mt = 0; mt < 8; ++mt) o[hn][mt][0] = o[hn][mt][1] = o[hn][mt][2] = o[hn][mt][3] = 0.f;
+  }
+}
+
+// Last page of a segment: this warp's (m, l, O) of the G heads into its rows of the hand-over
+// buffer `red` ([warp][GP][132]: 128 output dims, then m and l), for the epilogue warp.
+template <int NH>
+__device__ inline void segment_hand_over(float *red, int warp, int GP, int G, const float (&m)[NH][2],
+                                         const float (&l)[NH][2], const float (&o)[NH][8][4], int lane) {
+  const int g = lane >> 2, t4 = lane & 3;
+#pragma unroll
+  for (int hn = 0; hn < NH; ++hn)
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      float lv = l[hn][j];
+      lv += __shfl_xor_sync(0xffffffffu, lv, 4);
+      lv += __shfl_xor_sync(0xffffffffu, lv, 8);
+      lv += __shfl_xor_sync(0xffffffffu, lv, 16);
+      const int h = hn * 8 + t4 * 2 + j;
+      if (h < G) {
+        float *dst = red + ((size_t)warp * GP + h) * 132;
+#pragma unroll
+        for (int mt = 0; mt < 8; ++mt) {
+          dst[mt * 16 + g] = o[hn][mt][j];
+          dst[mt * 16 + 8 + g] = o[hn][mt][2 + j];
+        }
+        if (g == 0) { dst[128] = m[hn][j]; dst[129] = lv; }
+      }
+    }
+}
+
 // Where the segments of one launch (or of one layer of a stack launch) put their results.
 struct SegOut {
   __nv_bfloat16 *out;       // [B][Hq][128]

@@ -372,7 +372,6 @@ decode_stack_kernel(StackArgs a, int GP, int n_stages, int n_plans) {
     // S^T = K Q^T and O^T += V^T P^T as m16n8k16 tiles, online softmax in registers)
     uint32_t qb[NH][8][2];
     float m[NH][2], l[NH][2], o[NH][8][4];
-    const int g = lane >> 2, t4 = lane & 3;
     int seg_k = 0;  // pages of the current segment so far: group g takes those with seg_k % 2 == g, so that a
                     // segment's sums do not depend on what the block streamed before it
     int n_seg = 0;  // hand-overs so far (segments and layer markers)
@@ -407,16 +406,7 @@ decode_stack_kernel(StackArgs a, int GP, int n_stages, int n_plans) {
       unsigned char *sbase = smem + (size_t)stage * L.stage_bytes;
       if (flags & F_BEGIN) {
         seg_k = 0;
-        const __nv_bfloat16 *qs = reinterpret_cast<const __nv_bfloat16 *>(sbase + kPageBytes);
-        load_q_frags_t<NH>(qb, [&](int h) -> const __nv_bfloat16 * { return h < GP ? qs + h * kD : nullptr; },
-                           lane);
-#pragma unroll
-        for (int hn = 0; hn < NH; ++hn) {
-          m[hn][0] = m[hn][1] = -INFINITY;
-          l[hn][0] = l[hn][1] = 0.f;
-#pragma unroll
-          for (int mt = 0; mt < 8; ++mt) o[hn][mt][0] = o[hn][mt][1] = o[hn][mt][2] = o[hn][mt][3] = 0.f;
-        }
+        segment_begin<NH>(qb, m, l, o, reinterpret_cast<const __nv_bfloat16 *>(sbase + kPageBytes), GP, lane);
       }
       const int tok0 = (warp & 3) * 16;
       if ((seg_k & 1) == (warp >> 2) && tok0 < valid) {
@@ -433,26 +423,7 @@ decode_stack_kernel(StackArgs a, int GP, int n_stages, int n_plans) {
       // last page of the segment: hand this warp's (m, l, O) to the epilogue warp
       int rb;
       if (!hand_over_begin(rb)) break;
-      float *red = s_red + (size_t)rb * kConsumerWarps * GP * 132;
-#pragma unroll
-      for (int hn = 0; hn < NH; ++hn)
-#pragma unroll
-        for (int j = 0; j < 2; ++j) {
-          float lv = l[hn][j];
-          lv += __shfl_xor_sync(0xffffffffu, lv, 4);
-          lv += __shfl_xor_sync(0xffffffffu, lv, 8);
-          lv += __shfl_xor_sync(0xffffffffu, lv, 16);
-          const int h = hn * 8 + t4 * 2 + j;
-          if (h < a.G) {
-            float *dst = red + ((size_t)warp * GP + h) * 132;
-#pragma unroll
-            for (int mt = 0; mt < 8; ++mt) {
-              dst[mt * 16 + g] = o[hn][mt][j];
-              dst[mt * 16 + 8 + g] = o[hn][mt][2 + j];
-            }
-            if (g == 0) { dst[128] = m[hn][j]; dst[129] = lv; }
-          }
-        }
+      segment_hand_over<NH>(s_red + (size_t)rb * kConsumerWarps * GP * 132, warp, GP, a.G, m, l, o, lane);
       if (tid == 0) {
         s_redmeta[rb] = item;
         s_redmeta[2 + rb] = chunk;
