@@ -1,19 +1,22 @@
 #!/usr/bin/env python
 """SP-KV decode benchmark (one JSON line).
 
-A step = one decode token for every sequence of the batch through the whole layer stack:
-per layer  spkv_score_append_evict (score + append/evict fused) -> spkv_decode_attention  (the library is the
-attention path only; there are no projections or MLPs).  Inputs are synthetic and seeded,
+A step = one decode token for every sequence of the batch through the whole layer stack: per layer
+score + append/evict, then decode attention (the library is the attention path only; there are no
+projections or MLPs).  The step is ONE spkv_decode_stack call -- the appends of every layer in one
+launch, decode attention of every layer in one persistent launch; --per-layer times it as 2 L calls
+(spkv_score_append_evict -> spkv_decode_attention per layer).  Inputs are synthetic and seeded,
 shaped like the paper's decode workloads (see paper_2605_14037_b200/synth.py); the cache is
 brought to the configured context length with spkv_prefill before timing.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config 2] [--impl reference]
 
 value        whole-job decode tokens/s, inputs resident in HBM, one CUDA-graph replay per step
-e2e          the same through spkv_decode_step_host with pinned HOST buffers (H2D + D2H timed)
-roofline     decode-attention kernel: algorithmic bytes (kept + window K/V, Q, O) per launch over
-             the average launch period in the timed region (launches overlap), against the
-             measured HBM copy bandwidth; the same launch timed alone is reported beside it
+e2e          the same through spkv_decode_stack_host with pinned HOST buffers (H2D + D2H timed);
+             the per-layer spkv_decode_step_host beside it
+roofline     decode-attention kernel: algorithmic bytes (kept + window K/V, Q, O) of a step over the
+             step time, against the measured HBM copy bandwidth, the nominal 8 TB/s and a read-only
+             stream the library measures itself; one per-layer launch timed alone beside it
 dense        same library, tau = -inf (every pair kept): the full-cache decode baseline
 cpu_baseline the CPU oracle timed on a bounded sample of the same workload
 """

@@ -1,6 +1,8 @@
 // Step 3 of the hot path: ragged split-K decode attention (Eq. 3-5) over
-// ring window U compact cache, log-sum-exp merge fused in.  Main (tensor-core) kernel and
-// the host entry points.
+// ring window U compact cache, log-sum-exp merge fused in.  The kernel that takes one layer per
+// launch, and the host entry points.  (spkv_decode_stack.cu holds the kernel that takes every
+// layer of a step in one launch; the two share their consumers, epilogue and range cuts through
+// spkv_decode_common.cuh.)
 //
 // Work decomposition.  The call covers n_items = B * n_kv_heads units.  Unit i owns np_i
 // pages (its kept pages followed by its ring pages).  All page lists are laid end to end
